@@ -1,0 +1,356 @@
+"""Physical packing of Cassandra-1 speculation data (oracle): weight blobs and KV records.
+
+Test infrastructure only; see the package docstring.
+
+The paper fixes the *content* (a bitmap, a sign+mantissa field per kept value, a unary
+exponent code per kept value; Sec. 4.2, 5.1) and asks for fully packed superblocks that
+are read contiguously (Sec. 5.3); the concrete byte layout below is this build's own.
+
+Common rules
+  * every stream is a sequence of 32-bit little-endian words, filled MSB first;
+  * a field of width F = 8 - t never straddles a word: a word holds floor(32/F) fields;
+  * unary codewords are contiguous and may straddle words;
+  * unused bits are zero.
+
+Weight blob  (rows N x cols K, row-major source)
+  word  0      magic 'CASW'            word  7  chunk_cols C (multiple of 32)
+  word  1      version (1)             word  8  n_seg
+  word  2      N                       word  9  n_rowblocks = ceil(N/32)
+  word  3      K                       word 10  kept per row = K - floor(K*p/1000)
+  word  4      p (per-mille)           word 11  directory byte offset (384)
+  word  5      t                       word 12  body byte offset
+  word  6      seg_cols (mult. of C)   word 13/14  total bytes (lo/hi)
+  bytes 128..383   codebook: rank -> exponent value
+  directory: one entry of four words per superblock sb = rowblock*n_seg + seg:
+      {byte offset / 16, W_f, W_u, n_chunks}
+  superblock = 32 rows x one column segment, four sections, each word-interleaved over
+  the 32 rows (word j of row r sits at index j*32 + r):
+      chunk table  n_chunks words/row : (index of the chunk's first field << 20) | bit
+                                        offset of the chunk's first codeword
+      bitmap       seg_cols/32 words/row (1 = kept), column c at bit 31 - c%32
+      fields       W_f words/row  (max over the 32 rows of ceil(kept_in_seg / per_word))
+      unary        W_u words/row  (max over the 32 rows)
+
+KV record (one token, one KV head, K or V; d = head_dim)
+  bitmap d/32 words, fields W_f = ceil(kept/per_word) words, unary: variable word count.
+"""
+from __future__ import annotations
+
+import dataclasses
+
+import numpy as np
+
+from . import codec
+
+MAGIC = 0x57534143
+VERSION = 1
+HEADER_BYTES = 128
+CODEBOOK_BYTES = 256
+DIR_OFFSET = HEADER_BYTES + CODEBOOK_BYTES
+ROWS_PER_BLOCK = 32
+
+
+def fields_per_word(t: int) -> int:
+    return 32 // (8 - t)
+
+
+def bits_to_words(bits: np.ndarray) -> np.ndarray:
+    """Bit k of the sequence -> word k//32, bit position 31 - k%32."""
+    bits = np.asarray(bits, dtype=np.uint8)
+    n_words = (bits.size + 31) // 32
+    padded = np.zeros(n_words * 32, dtype=np.uint8)
+    padded[: bits.size] = bits
+    by = np.packbits(padded).reshape(n_words, 4).astype(np.uint32)      # big bit order inside bytes
+    return (by[:, 0] << 24) | (by[:, 1] << 16) | (by[:, 2] << 8) | by[:, 3]
+
+
+def words_to_bits(words: np.ndarray) -> np.ndarray:
+    w = np.asarray(words, dtype=np.uint32)
+    by = np.stack([(w >> 24) & 0xFF, (w >> 16) & 0xFF, (w >> 8) & 0xFF, w & 0xFF], axis=1).astype(np.uint8)
+    return np.unpackbits(by.reshape(-1))
+
+
+def pack_fields(fields: np.ndarray, t: int) -> np.ndarray:
+    width = 8 - t
+    per = fields_per_word(t)
+    fields = np.asarray(fields, dtype=np.uint32)
+    n_words = (fields.size + per - 1) // per
+    out = np.zeros(n_words, dtype=np.uint32)
+    for j in range(fields.size):
+        out[j // per] |= np.uint32(int(fields[j]) << (32 - width * (j % per + 1)))
+    return out
+
+
+def unpack_fields(words: np.ndarray, n: int, t: int) -> np.ndarray:
+    width = 8 - t
+    per = fields_per_word(t)
+    out = np.zeros(n, dtype=np.uint32)
+    for j in range(n):
+        out[j] = (int(words[j // per]) >> (32 - width * (j % per + 1))) & ((1 << width) - 1)
+    return out
+
+
+def _pack_fields_fast(fields: np.ndarray, t: int) -> np.ndarray:
+    width = 8 - t
+    per = fields_per_word(t)
+    fields = np.asarray(fields, dtype=np.uint32)
+    n_words = (fields.size + per - 1) // per
+    padded = np.zeros(n_words * per, dtype=np.uint32)
+    padded[: fields.size] = fields
+    padded = padded.reshape(n_words, per)
+    shifts = np.array([32 - width * (j + 1) for j in range(per)], dtype=np.uint32)
+    return np.bitwise_or.reduce(padded << shifts[None, :], axis=1).astype(np.uint32) if n_words else padded.reshape(0)
+
+
+@dataclasses.dataclass
+class WeightBlobInfo:
+    rows: int
+    cols: int
+    p: int
+    t: int
+    seg_cols: int
+    chunk_cols: int
+    n_seg: int
+    n_rowblocks: int
+    kept_per_row: int
+    body_offset: int
+    total_bytes: int
+    codebook: np.ndarray          # rank -> exponent
+    directory: np.ndarray         # [n_sb, 4] uint32
+
+
+def auto_seg_cols(cols: int, chunk_cols: int, seg_cols: int) -> int:
+    k_pad = (cols + 31) // 32 * 32
+    seg = min(seg_cols, (k_pad + chunk_cols - 1) // chunk_cols * chunk_cols)
+    return seg
+
+
+def _segment_cols(k_pad: int, seg_cols: int, seg: int) -> int:
+    return min(seg_cols, k_pad - seg * seg_cols)
+
+
+def encode_weight_blob(w_bits: np.ndarray, act_norm: np.ndarray | None, p: int, t: int,
+                       seg_cols: int = 2048, chunk_cols: int = 256,
+                       rowblocks=None):
+    """Encode a bf16 matrix into a blob.  Returns (blob as uint32 words, WeightBlobInfo).
+
+    With `rowblocks` (an iterable of row-block indices) only those superblocks' bodies are
+    produced -- returned as {sb_index: words} together with header/codebook/sizes -- so that a
+    large matrix can be spot-checked; the codebook always covers the whole matrix.
+    """
+    w_bits = np.asarray(w_bits, dtype=np.uint16)
+    n, k = w_bits.shape
+    if act_norm is None:
+        act_norm = np.ones(k, dtype=np.float32)
+    assert chunk_cols % 32 == 0 and seg_cols % chunk_cols == 0 and seg_cols <= 4096
+    keep = codec.keep_mask_weights(w_bits, act_norm, p)
+    counts = codec.exponent_counts(w_bits, keep)
+    rank_to_exp = codec.codebook_from_counts(counts)
+    exp_to_rank = codec.invert_codebook(rank_to_exp)
+
+    k_pad = (k + 31) // 32 * 32
+    seg_cols = auto_seg_cols(k, chunk_cols, seg_cols)
+    n_seg = (k_pad + seg_cols - 1) // seg_cols
+    n_rb = (n + ROWS_PER_BLOCK - 1) // ROWS_PER_BLOCK
+    per = fields_per_word(t)
+
+    _, e_all, _ = codec.split_fields(w_bits)
+    sel = range(n_rb) if rowblocks is None else list(rowblocks)
+    bodies: dict[int, np.ndarray] = {}
+    for rb in sel:
+        for seg in range(n_seg):
+            c0 = seg * seg_cols
+            scols = _segment_cols(k_pad, seg_cols, seg)
+            n_ch = (scols + chunk_cols - 1) // chunk_cols
+            rows_tab, rows_bm, rows_f, rows_u = [], [], [], []
+            for rr in range(ROWS_PER_BLOCK):
+                r = rb * ROWS_PER_BLOCK + rr
+                km = np.zeros(scols, dtype=bool)
+                if r < n:
+                    c1 = min(k, c0 + scols)
+                    km[: c1 - c0] = keep[r, c0:c1]
+                idx = np.flatnonzero(km)
+                if idx.size:
+                    vals = w_bits[r, c0 + idx]
+                    fields = codec.spec_field(vals, t)
+                    ranks = exp_to_rank[e_all[r, c0 + idx]]
+                else:
+                    fields = np.zeros(0, dtype=np.uint32)
+                    ranks = np.zeros(0, dtype=np.int64)
+                # chunk table: running count of kept values and of code bits at each chunk start
+                tab = np.zeros(n_ch, dtype=np.uint32)
+                code_len = ranks + 1
+                cum_bits = np.concatenate(([0], np.cumsum(code_len)))
+                for ch in range(n_ch):
+                    first = int(np.searchsorted(idx, ch * chunk_cols))      # kept values before the chunk
+                    bit_off = int(cum_bits[first])
+                    if first >= (1 << 12) or bit_off >= (1 << 20):
+                        raise ValueError("chunk table overflow")
+                    tab[ch] = (first << 20) | bit_off
+                rows_tab.append(tab)
+                rows_bm.append(bits_to_words(km.astype(np.uint8)))
+                rows_f.append(_pack_fields_fast(fields, t))
+                rows_u.append(bits_to_words(codec.unary_encode_fast(ranks)) if ranks.size else np.zeros(0, np.uint32))
+            w_f = max(x.size for x in rows_f)
+            w_u = max(x.size for x in rows_u)
+
+            def interleave(rows, width):
+                sec = np.zeros((width, ROWS_PER_BLOCK), dtype=np.uint32)
+                for rr, x in enumerate(rows):
+                    sec[: x.size, rr] = x
+                return sec.reshape(-1)
+
+            body = np.concatenate([
+                interleave(rows_tab, n_ch), interleave(rows_bm, scols // 32),
+                interleave(rows_f, w_f), interleave(rows_u, w_u)])
+            bodies[rb * n_seg + seg] = (body, w_f, w_u, n_ch)
+
+    info = dict(rows=n, cols=k, p=p, t=t, seg_cols=seg_cols, chunk_cols=chunk_cols, n_seg=n_seg,
+                n_rowblocks=n_rb, kept_per_row=k - codec.n_pruned(k, p), codebook=rank_to_exp,
+                counts=counts, keep=keep)
+    if rowblocks is not None:
+        return bodies, info
+
+    n_sb = n_rb * n_seg
+    body_off = (DIR_OFFSET + 16 * n_sb + 127) // 128 * 128
+    directory = np.zeros((n_sb, 4), dtype=np.uint32)
+    off = body_off
+    parts = []
+    for sb in range(n_sb):
+        body, w_f, w_u, n_ch = bodies[sb]
+        directory[sb] = (off // 16, w_f, w_u, n_ch)
+        off += body.size * 4
+        parts.append(body)
+    total = off
+    header = np.zeros(HEADER_BYTES // 4, dtype=np.uint32)
+    header[:15] = (MAGIC, VERSION, n, k, p, t, seg_cols, chunk_cols, n_seg, n_rb,
+                   k - codec.n_pruned(k, p), DIR_OFFSET, body_off, total & 0xFFFFFFFF, total >> 32)
+    cb_words = np.frombuffer(rank_to_exp.tobytes(), dtype="<u4")
+    pad = np.zeros((body_off - DIR_OFFSET - 16 * n_sb) // 4, dtype=np.uint32)
+    blob = np.concatenate([header, cb_words, directory.reshape(-1), pad] + parts).astype(np.uint32)
+    assert blob.size * 4 == total
+    return blob, info
+
+
+def parse_weight_blob(blob: np.ndarray) -> WeightBlobInfo:
+    blob = np.asarray(blob, dtype=np.uint32)
+    h = blob[: HEADER_BYTES // 4]
+    if int(h[0]) != MAGIC or int(h[1]) != VERSION:
+        raise ValueError("bad magic/version")
+    n_sb = int(h[8]) * int(h[9])
+    cb = np.frombuffer(blob[HEADER_BYTES // 4: DIR_OFFSET // 4].tobytes(), dtype=np.uint8).copy()
+    d0 = int(h[11]) // 4
+    directory = blob[d0: d0 + 4 * n_sb].reshape(n_sb, 4).copy()
+    return WeightBlobInfo(rows=int(h[2]), cols=int(h[3]), p=int(h[4]), t=int(h[5]), seg_cols=int(h[6]),
+                          chunk_cols=int(h[7]), n_seg=int(h[8]), n_rowblocks=int(h[9]), kept_per_row=int(h[10]),
+                          body_offset=int(h[12]), total_bytes=int(h[13]) | (int(h[14]) << 32),
+                          codebook=cb, directory=directory)
+
+
+def decode_weight_blob(blob: np.ndarray, use_chunk_table: bool = False) -> np.ndarray:
+    """Draft decode of a whole blob -> bf16 bit patterns [N, K] (pruned -> +0, low mantissa -> 0).
+
+    With use_chunk_table, every chunk is decoded on its own, starting from the offsets the chunk
+    table gives (this is how a parallel decoder enters the streams)."""
+    blob = np.asarray(blob, dtype=np.uint32)
+    info = parse_weight_blob(blob)
+    n, k, t = info.rows, info.cols, info.t
+    k_pad = (k + 31) // 32 * 32
+    out = np.zeros((info.n_rowblocks * ROWS_PER_BLOCK, info.n_seg * info.seg_cols), dtype=np.uint16)
+    for sb in range(info.n_rowblocks * info.n_seg):
+        rb, seg = divmod(sb, info.n_seg)
+        off16, w_f, w_u, n_ch = (int(x) for x in info.directory[sb])
+        scols = _segment_cols(k_pad, info.seg_cols, seg)
+        base = off16 * 4
+        tab = blob[base: base + n_ch * 32].reshape(n_ch, 32); base += n_ch * 32
+        bm = blob[base: base + scols // 32 * 32].reshape(scols // 32, 32); base += scols // 32 * 32
+        fl = blob[base: base + w_f * 32].reshape(w_f, 32); base += w_f * 32
+        un = blob[base: base + w_u * 32].reshape(w_u, 32)
+        for rr in range(ROWS_PER_BLOCK):
+            km = words_to_bits(bm[:, rr]).astype(bool)
+            idx = np.flatnonzero(km)
+            if idx.size == 0:
+                continue
+            ubits = words_to_bits(un[:, rr])
+            if not use_chunk_table:
+                fields = unpack_fields(fl[:, rr], idx.size, t)
+                ranks = codec.unary_decode_fast(ubits, idx.size)
+            else:
+                fields = np.zeros(idx.size, dtype=np.uint32)
+                ranks = np.zeros(idx.size, dtype=np.int64)
+                per = fields_per_word(t)
+                for ch in range(n_ch):
+                    first, bit_off = int(tab[ch, rr]) >> 20, int(tab[ch, rr]) & 0xFFFFF
+                    cnt = int(km[ch * info.chunk_cols: (ch + 1) * info.chunk_cols].sum())
+                    if cnt == 0:
+                        continue
+                    width = 8 - t
+                    for j in range(first, first + cnt):
+                        fields[j] = (int(fl[j // per, rr]) >> (32 - width * (j % per + 1))) & ((1 << width) - 1)
+                    ranks[first: first + cnt] = codec.unary_decode_fast(ubits[bit_off:], cnt)
+            e = info.codebook[ranks].astype(np.uint16)
+            s = (fields >> (7 - t)).astype(np.uint16) & 1
+            m_hi = (fields & ((1 << (7 - t)) - 1)).astype(np.uint16)
+            vals = (s << 15) | (e << 7) | (m_hi << t)
+            out[rb * ROWS_PER_BLOCK + rr, seg * info.seg_cols + idx] = vals
+    return out[:n, :k]
+
+
+def blob_section_bits(blob: np.ndarray) -> dict:
+    """Bits spent per section over the whole blob (for the size closed form)."""
+    info = parse_weight_blob(blob)
+    k_pad = (info.cols + 31) // 32 * 32
+    tab = bm = fl = un = 0
+    for sb in range(info.n_rowblocks * info.n_seg):
+        _, w_f, w_u, n_ch = (int(x) for x in info.directory[sb])
+        scols = _segment_cols(k_pad, info.seg_cols, sb % info.n_seg)
+        tab += n_ch * 32 * 32
+        bm += scols * 32
+        fl += w_f * 32 * 32
+        un += w_u * 32 * 32
+    return dict(header=info.body_offset * 8, chunk_table=tab, bitmap=bm, fields=fl, unary=un,
+                total=info.total_bytes * 8)
+
+
+# --------------------------------------------------------------------------------------
+# KV records
+# --------------------------------------------------------------------------------------
+
+
+def kv_fixed_words(d: int, p: int, t: int) -> int:
+    kept = d - codec.n_pruned(d, p)
+    return d // 32 + (kept + fields_per_word(t) - 1) // fields_per_word(t)
+
+
+def encode_kv_token(x_bits: np.ndarray, p: int, t: int, exp_to_rank: np.ndarray):
+    """One token, one head: returns (bitmap words, field words, unary words)."""
+    x_bits = np.asarray(x_bits, dtype=np.uint16)
+    keep = codec.keep_mask_kv(x_bits, p)
+    idx = np.flatnonzero(keep)
+    _, e, _ = codec.split_fields(x_bits[idx])
+    ranks = np.asarray(exp_to_rank)[e]
+    return (bits_to_words(keep.astype(np.uint8)),
+            _pack_fields_fast(codec.spec_field(x_bits[idx], t), t),
+            bits_to_words(codec.unary_encode_fast(ranks)) if idx.size else np.zeros(0, np.uint32))
+
+
+def decode_kv_token(bm_words, field_words, unary_words, d: int, t: int, rank_to_exp: np.ndarray) -> np.ndarray:
+    keep = words_to_bits(bm_words)[:d].astype(bool)
+    idx = np.flatnonzero(keep)
+    out = np.zeros(d, dtype=np.uint16)
+    if idx.size == 0:
+        return out
+    fields = unpack_fields(field_words, idx.size, t)
+    ranks = codec.unary_decode_fast(words_to_bits(unary_words), idx.size)
+    e = np.asarray(rank_to_exp)[ranks].astype(np.uint16)
+    s = (fields >> (7 - t)).astype(np.uint16) & 1
+    m_hi = (fields & ((1 << (7 - t)) - 1)).astype(np.uint16)
+    out[idx] = (s << 15) | (e << 7) | (m_hi << t)
+    return out
+
+
+def kv_codebook(x_bits: np.ndarray, p: int) -> np.ndarray:
+    """Codebook of one (layer, K|V): exponent histogram of the kept values of all given tokens and
+    heads (x_bits [..., d])."""
+    keep = codec.keep_mask_kv(x_bits, p)
+    return codec.codebook_from_counts(codec.exponent_counts(x_bits, keep))

@@ -1,0 +1,224 @@
+"""Llama-style target and Cassandra draft forward passes, and the speculative loop (oracle).
+
+Test infrastructure only; see the package docstring.
+
+Target = the bf16 model (RMSNorm, RoPE, grouped-query attention, SwiGLU; Sec. 2.1).
+Draft  = the same graph evaluated on zero-padded reconstructions of the speculation data of
+the weights and of the KV cache (Sec. 4.1).  Accumulation is fp64; activations are rounded to
+bf16 at the same points as the CUDA path: norm outputs, projection outputs, RoPE outputs,
+attention output, SwiGLU output and after each residual add.  Logits stay unrounded.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+from . import codec, layout
+
+
+def _f(bits):
+    return codec.bf16_bits_to_f64(bits)
+
+
+def _r(x):
+    return codec.f64_to_bf16_bits(x)
+
+
+def rmsnorm(h_bits: np.ndarray, g_bits: np.ndarray, eps: float) -> np.ndarray:
+    h = _f(h_bits)
+    inv = 1.0 / np.sqrt(np.mean(h * h) + eps)
+    return _r(h * inv * _f(g_bits))
+
+
+def rope(v_bits: np.ndarray, pos: int, theta: float) -> np.ndarray:
+    """v [heads, d]; pairs (i, i + d/2) rotated by pos * theta^(-2i/d)."""
+    v = _f(v_bits)
+    d = v.shape[-1]
+    half = d // 2
+    i = np.arange(half, dtype=np.float64)
+    ang = float(pos) * theta ** (-2.0 * i / d)
+    c, s = np.cos(ang), np.sin(ang)
+    a, b = v[:, :half], v[:, half:]
+    return _r(np.concatenate([a * c - b * s, b * c + a * s], axis=1))
+
+
+def argmax_lowest(x: np.ndarray) -> int:
+    return int(np.argmax(x))          # numpy returns the first (lowest) index among equal maxima
+
+
+class Weights:
+    """Dense fp64 views of a model's matrices (exact bf16 values)."""
+
+    def __init__(self, shape, w_bits: dict):
+        self.shape = shape
+        self.layers = [{k: _f(v) if k.startswith("w") else np.asarray(v, dtype=np.uint16) for k, v in lw.items()}
+                       for lw in w_bits["layers"]]
+        self.embed_bits = np.asarray(w_bits["embed"], dtype=np.uint16)
+        self.lm_head = _f(w_bits["lm_head"])
+        self.norm_final = np.asarray(w_bits["norm_final"], dtype=np.uint16)
+
+
+def draft_weight_bits(w_bits: dict, act_norms: dict, p: int, t: int) -> dict:
+    """Speculation-data view of every projection and of lm_head (embeddings and norm gains stay bf16)."""
+    out = {"layers": []}
+    for li, lw in enumerate(w_bits["layers"]):
+        d = {}
+        for k, v in lw.items():
+            if k.startswith("w"):
+                v = np.asarray(v, dtype=np.uint16)
+                keep = codec.keep_mask_weights(v, act_norms["layers"][li][k], p)
+                d[k] = codec.draft_bits(v, keep, t)
+            else:
+                d[k] = v
+        out["layers"].append(d)
+    lm = np.asarray(w_bits["lm_head"], dtype=np.uint16)
+    out["lm_head"] = codec.draft_bits(lm, codec.keep_mask_weights(lm, act_norms["lm_head"], p), t)
+    out["embed"] = w_bits["embed"]
+    out["norm_final"] = w_bits["norm_final"]
+    return out
+
+
+class KVCache:
+    """Per layer: bf16 K/V as written by the target, and the draft's view of every position."""
+
+    def __init__(self, shape, max_seq: int):
+        s = shape
+        z = lambda: np.zeros((s.n_layers, max_seq, s.n_kv_heads, s.head_dim), dtype=np.uint16)
+        self.k, self.v = z(), z()            # target (bf16) cache
+        self.kd, self.vd = z(), z()          # zero-padded reconstruction of the compressed cache
+        self.n = 0                           # committed length
+
+
+def forward_token(W: Weights, kv: KVCache, tok: int, pos: int, draft: bool, kv_p: int, kv_t: int,
+                  calib: dict | None = None):
+    """One token at position `pos`.  Target mode writes K/V in both forms at `pos`; draft mode
+    writes only the draft view.  Returns the fp64 logits."""
+    s = W.shape
+    d = s.head_dim
+    g = s.n_q_heads // s.n_kv_heads
+    h = W.embed_bits[tok].copy()
+
+    def note(li, names, x_bits):
+        if calib is not None:
+            x = _f(x_bits)
+            for nm in names:
+                calib["layers"][li][nm] += x * x
+
+    for li, lw in enumerate(W.layers):
+        xn = rmsnorm(h, lw["norm_attn"], s.rms_eps)
+        note(li, ("wq", "wk", "wv"), xn)
+        x = _f(xn)
+        q = _r(lw["wq"] @ x).reshape(s.n_q_heads, d)
+        k = _r(lw["wk"] @ x).reshape(s.n_kv_heads, d)
+        v = _r(lw["wv"] @ x).reshape(s.n_kv_heads, d)
+        q = rope(q, pos, s.rope_theta)
+        k = rope(k, pos, s.rope_theta)
+        kd = codec.draft_bits(k, codec.keep_mask_kv(k, kv_p), kv_t)
+        vd = codec.draft_bits(v, codec.keep_mask_kv(v, kv_p), kv_t)
+        kv.kd[li, pos], kv.vd[li, pos] = kd, vd
+        if not draft:
+            kv.k[li, pos], kv.v[li, pos] = k, v
+        kc = _f((kv.kd if draft else kv.k)[li, : pos + 1])          # [pos+1, n_kv, d]
+        vc = _f((kv.vd if draft else kv.v)[li, : pos + 1])
+        qf = _f(q)
+        o = np.zeros((s.n_q_heads, d))
+        for hq in range(s.n_q_heads):
+            hk = hq // g
+            sc = (kc[:, hk, :] @ qf[hq]) / np.sqrt(float(d))
+            sc = sc - sc.max()
+            pr = np.exp(sc)
+            pr = pr / pr.sum()
+            o[hq] = pr @ vc[:, hk, :]
+        ob = _r(o.reshape(-1))
+        note(li, ("wo",), ob)
+        attn = _r(lw["wo"] @ _f(ob))
+        h = _r(_f(h) + _f(attn))
+        xn = rmsnorm(h, lw["norm_ffn"], s.rms_eps)
+        note(li, ("wg", "wu"), xn)
+        x = _f(xn)
+        gate = _f(_r(lw["wg"] @ x))
+        up = _f(_r(lw["wu"] @ x))
+        act = _r(gate / (1.0 + np.exp(-gate)) * up)
+        note(li, ("wd",), act)
+        down = _r(lw["wd"] @ _f(act))
+        h = _r(_f(h) + _f(down))
+    xn = rmsnorm(h, W.norm_final, s.rms_eps)
+    if calib is not None:
+        calib["lm_head"] += _f(xn) ** 2
+    return W.lm_head @ _f(xn)
+
+
+def new_calib(shape) -> dict:
+    from synth import llama_layer_shapes
+    return {"layers": [{k: np.zeros(c) for k, (_, c) in llama_layer_shapes(shape).items()}
+                       for _ in range(shape.n_layers)],
+            "lm_head": np.zeros(shape.hidden)}
+
+
+def calib_to_norms(calib: dict) -> dict:
+    """Per-input-channel L2 norms (fp32) from accumulated sums of squares."""
+    return {"layers": [{k: np.sqrt(v).astype(np.float32) for k, v in lw.items()} for lw in calib["layers"]],
+            "lm_head": np.sqrt(calib["lm_head"]).astype(np.float32)}
+
+
+def prefill(W: Weights, kv: KVCache, prompt, kv_p: int, kv_t: int, calib: dict | None = None):
+    """Target pass over the prompt; returns the logits of the last prompt token."""
+    logits = None
+    for pos, tok in enumerate(prompt):
+        logits = forward_token(W, kv, int(tok), pos, False, kv_p, kv_t, calib)
+    kv.n = len(prompt)
+    return logits
+
+
+def greedy_accept(draft_tokens, target_argmax):
+    """Number of accepted draft tokens: Eq. 1 specialised to greedy decoding, where the ratio
+    p_i/q_i is 1 if the target's own choice equals the drafted token and 0 otherwise."""
+    gamma = len(draft_tokens)
+    rejected = [i - 1 for i in range(1, gamma + 1) if draft_tokens[i - 1] != target_argmax[i - 1]]
+    return min(rejected + [gamma])
+
+
+def plain_greedy(W: Weights, kv: KVCache, first_tok: int, n_tokens: int, kv_p: int, kv_t: int):
+    """Autoregressive decoding with the target only.  `first_tok` is the token predicted from the
+    prompt; returns the n_tokens tokens that follow it."""
+    out = []
+    tok = first_tok
+    for _ in range(n_tokens):
+        logits = forward_token(W, kv, tok, kv.n, False, kv_p, kv_t)
+        kv.n += 1
+        tok = argmax_lowest(logits)
+        out.append(tok)
+    return out
+
+
+def speculative_greedy(W: Weights, Wd, kv: KVCache, first_tok: int, n_tokens: int, gamma: int,
+                       kv_p: int, kv_t: int, draft_fn=None, trace=None):
+    """Draft gamma tokens, verify gamma+1 rows with the target, accept the matching prefix,
+    emit the target's token at the first mismatch (or its bonus token), roll the cache back.
+
+    `draft_fn(i, tok, pos)` may replace the draft model (used to test losslessness with arbitrary
+    drafts).  Returns the emitted tokens (at least n_tokens)."""
+    out = []
+    last = first_tok
+    while len(out) < n_tokens:
+        n = kv.n
+        drafts = []
+        tok = last
+        for i in range(gamma):
+            if draft_fn is not None:
+                nxt = int(draft_fn(i, tok, n + i))
+            else:
+                nxt = argmax_lowest(forward_token(Wd, kv, tok, n + i, True, kv_p, kv_t))
+            drafts.append(nxt)
+            tok = nxt
+        rows = [last] + drafts
+        targ = []
+        for i, tk in enumerate(rows):                 # batched verification == row-by-row causal pass
+            targ.append(argmax_lowest(forward_token(W, kv, tk, n + i, False, kv_p, kv_t)))
+        a = greedy_accept(drafts, targ)
+        emitted = drafts[:a] + [targ[a]]
+        out.extend(emitted)
+        kv.n = n + a + 1                              # entries beyond are stale and get overwritten
+        last = targ[a]
+        if trace is not None:
+            trace.append(dict(n=n, drafts=drafts, target=targ, accepted=a))
+    return out
