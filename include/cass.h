@@ -1,0 +1,199 @@
+/*
+ * cass.h -- C boundary of the B200-native Cassandra self-speculative decode step.
+ *
+ * One draft pass reads only the speculation data (pruned, mantissa-truncated, unary-exponent-coded
+ * weights and KV cache; Sec. 4.1-4.2 of the paper), decodes it in registers and runs batch-1 GEMV and
+ * grouped-query decode attention on it; a bf16 verification pass over the gamma+1 drafted rows and a
+ * greedy accept/rollback close each step (Sec. 2.2).
+ *
+ * Conventions
+ *   - Every entry point returns 0 (CASS_OK) or a negative CASS_ERR_* code; nothing throws.
+ *   - Pointers are DEVICE pointers unless the name starts with h_ (host).  The caller owns every buffer.
+ *   - No entry point allocates or frees device memory; size queries say how much the caller must provide.
+ *   - `stream` is a cudaStream_t passed as void*; work is enqueued on it and the call returns without
+ *     synchronising, except where a comment says that the call synchronises.
+ *   - Kernels are built for sm_100a only.  On any other device the first launch fails and the call
+ *     returns CASS_ERR_CUDA (there is no fallback path).
+ *   - Device-side problems (capacity exceeded, bounded wait ran out) are recorded in the session's
+ *     status word, readable with cass_session_status().
+ */
+#ifndef CASS_H_
+#define CASS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    CASS_OK = 0,
+    CASS_ERR_INVALID_ARG = -1,
+    CASS_ERR_CAPACITY = -2,
+    CASS_ERR_UNSUPPORTED = -3,
+    CASS_ERR_TIMEOUT = -4,
+    CASS_ERR_CUDA = -5
+};
+
+enum { CASS_KV_BF16 = 1, CASS_KV_COMPRESSED = 2 };
+
+/* Format parameters.  p = pruning ratio in per-mille, t = number of LOW mantissa bits removed from the
+ * speculation data (Eq. 2's w_t / kv_t; 7 - t mantissa bits remain).  Paper default: 400 / 4 (Sec. 6.1, 7.2).
+ * w_seg_cols / w_chunk_cols: columns per superblock and per decode chunk (0 = 2048 / 256). */
+typedef struct cass_format {
+    int mode;                /* 1 = Cassandra-1 (unary exponent code) */
+    int w_prune_permille, w_trunc_bits;
+    int kv_prune_permille, kv_trunc_bits;
+    int w_seg_cols, w_chunk_cols;
+} cass_format;
+
+typedef struct cass_model_desc {
+    int n_layers, hidden, n_q_heads, n_kv_heads, head_dim, ffn, vocab;
+    int max_seq;             /* KV positions per sequence */
+    int max_batch;           /* sequences (this build: 1) */
+    int gamma_max;           /* largest draft length; verification takes up to 16 rows per call */
+    float rope_theta, rms_eps;
+} cass_model_desc;
+
+/* Device pointers to the bf16 target model.  Per layer: wqkv [(n_q+2 n_kv) d, hidden] (q rows, then k rows,
+ * then v rows), wo [hidden, n_q d], wgu [2 ffn, hidden] (gate rows, then up rows), wd [hidden, ffn],
+ * two RMSNorm gains [hidden].  All row-major, rows = output features. */
+typedef struct cass_layer_weights {
+    const void *wqkv, *wo, *wgu, *wd, *norm_attn, *norm_ffn;
+} cass_layer_weights;
+
+typedef struct cass_model_weights {
+    const cass_layer_weights* h_layers;   /* HOST array [n_layers] of device pointers */
+    const void *embed, *lm_head, *norm_final;
+} cass_model_weights;
+
+/* Device pointers to the encoded speculation data of the same matrices (cass_encode_weights output). */
+typedef struct cass_layer_blobs { const void *wqkv, *wo, *wgu, *wd; } cass_layer_blobs;
+typedef struct cass_model_blobs {
+    const cass_layer_blobs* h_layers;     /* HOST array [n_layers] */
+    const void* lm_head;
+} cass_model_blobs;
+
+/* ------------------------------------------------------------------------------------------------------
+ * Offline weight encoder (Sec. 4.2 "Unstructured Value Pruning" with the Wanda score, "Mantissa
+ * Truncation", "Exponent Compression" by unary coding; Sec. 5.1 encoder; Sec. 5.3 superblocks).
+ * ---------------------------------------------------------------------------------------------------- */
+
+/* Upper bound of the blob size this library accepts for a rows x cols matrix (allows a mean code length of
+ * 8 bits per kept value), and the scratch the encoder needs.  Host-only arithmetic. */
+int cass_encoded_weight_bytes(const cass_format* fmt, int rows, int cols, size_t* h_blob_bound,
+                              size_t* h_workspace_bytes);
+
+/* Encode W (bf16 [rows][cols], row-major) into `blob`.  act_norm: fp32 [cols] per-input-channel L2 norms of
+ * calibration activations, or NULL for all ones.  Per row the floor(cols*p/1000) lowest scores
+ * fp32(|W_ij|) * act_norm[j] are pruned (ties: lower column first); NaN scores are not supported.
+ * blob must be 128-byte aligned.  workspace: scratch of the size the query returned.  d_status: device int32,
+ * set to CASS_ERR_CAPACITY if blob_cap is too small (blob contents are then undefined), else left alone.
+ * The total size is also stored in the blob header (see cass_weight_blob_info). */
+int cass_encode_weights(const cass_format* fmt, const void* W_bf16, const float* act_norm, int rows, int cols,
+                        void* blob, size_t blob_cap, void* workspace, size_t workspace_bytes,
+                        int32_t* d_status, void* stream);
+
+typedef struct cass_blob_info {
+    int rows, cols, prune_permille, trunc_bits, seg_cols, chunk_cols, n_seg, n_rowblocks, kept_per_row;
+    int max_superblock_bytes;
+    uint64_t total_bytes;
+} cass_blob_info;
+
+/* Reads the blob header back to the host.  SYNCHRONISES `stream`. */
+int cass_weight_blob_info(const void* blob, cass_blob_info* h_info, void* stream);
+
+/* Test hook: zero-padded reconstruction (Sec. 4.1, draft inference) of a whole blob into bf16 [rows][cols]. */
+int cass_decode_weights(const void* blob, const cass_blob_info* h_info, void* W_bf16_out, void* stream);
+
+/* ------------------------------------------------------------------------------------------------------
+ * Draft GEMV on speculation data (Sec. 4.1 draft inference; decoder dataflow of Sec. 5.1 / Algorithm 1).
+ *   y[r] = sum_c decode(blob)[r][c] * x[c], fp32 accumulation, y rounded to bf16 (y_bf16) and/or kept fp32.
+ * x: bf16 [cols].  partial: fp32 scratch [n_seg][rows].  Either output pointer may be NULL.
+ * ---------------------------------------------------------------------------------------------------- */
+int cass_draft_gemv(const void* blob, const cass_blob_info* h_info, const void* x_bf16, float* partial,
+                    void* y_bf16, float* y_f32, int32_t* d_status, void* stream);
+
+/* ------------------------------------------------------------------------------------------------------
+ * Session: model, KV caches (bf16 and compressed), activations and step state in caller-provided memory.
+ * ---------------------------------------------------------------------------------------------------- */
+int cass_session_bytes(const cass_model_desc* desc, const cass_format* fmt, size_t* h_bytes);
+
+/* mem: device memory of at least cass_session_bytes, 256-byte aligned; it is zeroed here.  blobs may be NULL
+ * and supplied later with cass_session_set_blobs (after calibration).  *h_session is a host handle released
+ * with cass_session_destroy (which frees host memory only).  SYNCHRONISES `stream`. */
+int cass_session_init(void* mem, size_t bytes, const cass_model_desc* desc, const cass_format* fmt,
+                      const cass_model_weights* weights, const cass_model_blobs* blobs, void** h_session,
+                      void* stream);
+int cass_session_set_blobs(void* session, const cass_model_blobs* blobs, void* stream);   /* SYNCHRONISES */
+int cass_session_destroy(void* session);
+
+/* Forget all sequences: committed length 0, no draft in flight, KV codebooks cleared. */
+int cass_session_reset(void* session, void* stream);
+
+/* Reads the device status word and the committed length of sequence 0.  SYNCHRONISES `stream`. */
+int cass_session_status(void* session, int32_t* h_status, int32_t* h_len, void* stream);
+
+/* Wanda calibration (Sec. 4.2, Sec. 7.2 "Pre-Computation Cost"): while enabled, cass_verify accumulates the
+ * per-input-channel sums of squares of the activations entering each projection.  cass_calib_norms writes
+ * their square roots: fp32 [n_layers][4][max(hidden, ffn)] (inputs of wqkv, wo, wgu, wd) followed by
+ * fp32 [hidden] (input of lm_head). */
+int cass_calib_enable(void* session, int on, void* stream);
+int cass_calib_norms(void* session, float* norms_out, void* stream);
+size_t cass_calib_norms_count(const cass_model_desc* desc);
+
+/* Online KV encoder (Sec. 4.2 per-token magnitude pruning; Sec. 5.1 encoder).  Writes n_new tokens of one
+ * layer, starting at position start_pos of sequence 0, into the bf16 cache and/or the compressed cache
+ * (flags).  K, V: bf16 [n_new][n_kv_heads][head_dim]; K is expected post-RoPE.  Per token and head the
+ * floor(d*p/1000) smallest |x| are pruned (ties: lower channel first).  Positions must be appended in
+ * order: start_pos may not exceed the number of positions already in the compressed cache of that layer.
+ * The compressed cache uses the layer's frozen codebooks (cass_kv_build_codebook). */
+int cass_kv_append(void* session, int layer, const void* K_bf16, const void* V_bf16, int start_pos, int n_new,
+                   int flags, void* stream);
+
+/* Builds the exponent codebooks of every layer (one for K, one for V) from the kept values of the first
+ * n_tokens positions of the bf16 cache, freezes them, and encodes those positions into the compressed cache. */
+int cass_kv_build_codebook(void* session, int n_tokens, void* stream);
+
+/* Sets the committed length of sequence 0 (after prefill through cass_verify, or to roll back). */
+int cass_set_len(void* session, int len, void* stream);
+
+/* One draft token (Sec. 4.1 draft inference).  Reads the token id at tok_in, runs the draft model at position
+ * len + (tokens drafted since the last accept), appends that position's K/V to the compressed cache only,
+ * and writes the greedy next token to tok_out (lowest index on ties).  logits_opt: fp32 [vocab] or NULL. */
+int cass_draft_step(void* session, const int32_t* tok_in, int32_t* tok_out, float* logits_opt, void* stream);
+
+/* Target pass over g+1 rows (Sec. 2.2 verification; Sec. 4.1 target inference): toks[i] sits at position
+ * len + i; causal among the rows; K/V of those positions are (over)written in both caches; row i's greedy
+ * token goes to target_argmax[i].  g+1 <= 16.  g = 0 is plain autoregressive decoding.  Does not move len.
+ * logits_opt: fp32 [g+1][vocab] or NULL.  Row results do not depend on how many rows the call has. */
+int cass_verify(void* session, const int32_t* toks, int g, int32_t* target_argmax, float* logits_opt,
+                void* stream);
+
+/* Greedy acceptance (Sec. 2.2; Eq. 1 with p/q in {0,1}): a = min({i-1 : draft[i-1] != target_argmax[i-1]} U {g});
+ * out_tokens[0..a] = draft[0..a-1], target_argmax[a]; len += a + 1 (both caches are trimmed by that);
+ * the draft-in-flight counter returns to 0; *next_tok = target_argmax[a].  n_accepted, next_tok: device. */
+int cass_accept(void* session, const int32_t* draft, const int32_t* target_argmax, int g, int32_t* n_accepted,
+                int32_t* out_tokens, int32_t* next_tok, void* stream);
+
+/* Geometry of the compressed KV cache of (layer, kind 0=K 1=V, head) for tests: device pointers to the
+ * fixed-part blocks, the unary arena and the per-token word offsets, plus words per token in the fixed part. */
+typedef struct cass_kv_view {
+    const uint32_t* fixed; const uint32_t* arena; const uint32_t* offsets; const uint8_t* codebook;
+    const void* k_or_v_bf16;
+    int fixed_words_per_token, bitmap_words, arena_words;
+} cass_kv_view;
+int cass_kv_query(void* session, int layer, int kind, int head, cass_kv_view* h_view);
+
+/* Standalone draft attention / verify kernels are reached through cass_draft_step / cass_verify; the
+ * activations of the last call can be inspected for tests: which = 0 hidden state after the last layer
+ * (bf16 [rows][hidden]), 1 = layer-0 attention output (bf16 [rows][n_q d]). */
+int cass_debug_activation(void* session, int which, const void** d_ptr, int* h_rows, int* h_cols);
+
+const char* cass_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CASS_H_ */

@@ -23,12 +23,17 @@ Weight blob  (rows N x cols K, row-major source)
   bytes 128..383   codebook: rank -> exponent value
   directory: one entry of four words per superblock sb = rowblock*n_seg + seg:
       {byte offset / 16, W_f, W_u, n_chunks}
-  superblock = 32 rows x one column segment, four sections, each word-interleaved over
-  the 32 rows (word j of row r sits at index j*32 + r):
-      chunk table  n_chunks words/row : (index of the chunk's first field << 20) | bit
-                                        offset of the chunk's first codeword
+  word 15      largest superblock size in bytes
+  superblock = 32 rows x one column segment.  First an "irregular" mask: one word per chunk
+  (bit r set = row r of that chunk is irregular, see `chunk_is_irregular`), padded with zero
+  words to a multiple of 32 words.  Then four sections, each word-interleaved over the 32
+  rows (word j of row r sits at index j*32 + r):
+      chunk table  n_chunks+1 words/row : (index of the chunk's first field WORD << 20) | bit
+                                        offset of the chunk's first codeword; the last entry
+                                        holds the segment totals.  The fields of every chunk
+                                        start on a word boundary.
       bitmap       seg_cols/32 words/row (1 = kept), column c at bit 31 - c%32
-      fields       W_f words/row  (max over the 32 rows of ceil(kept_in_seg / per_word))
+      fields       W_f words/row  (max over the 32 rows of the sum over chunks of ceil(kept_in_chunk / per_word))
       unary        W_u words/row  (max over the 32 rows)
 
 KV record (one token, one KV head, K or V; d = head_dim)
@@ -129,6 +134,31 @@ def _segment_cols(k_pad: int, seg_cols: int, seg: int) -> int:
     return min(seg_cols, k_pad - seg * seg_cols)
 
 
+GROUP_COLS = 8      # kept columns per bitmap-walk group
+GROUP_CODES = 4     # codewords per unary-walk group
+
+
+def chunk_is_irregular(cols_in_chunk: np.ndarray, code_len: np.ndarray) -> bool:
+    """A hint for parallel decoders.  A (row, chunk) is regular when a decoder that looks at the
+    bitmap and at the unary stream through 32-bit windows never needs a second window inside a
+    group: (a) for every aligned group of 8 consecutive kept columns, the distance from the
+    column after the previous group's last kept column (the chunk start for the first group) to
+    the group's last kept column is below 32; (b) every aligned group of 4 consecutive codewords
+    is at most 32 bits long in total.  Groups are counted from the chunk's first kept value."""
+    cols = np.asarray(cols_in_chunk, dtype=np.int64)
+    lens = np.asarray(code_len, dtype=np.int64)
+    start = 0
+    for g in range(0, cols.size, GROUP_COLS):
+        last = int(cols[min(g + GROUP_COLS, cols.size) - 1])
+        if last - start >= 32:
+            return True
+        start = last + 1
+    for g in range(0, lens.size, GROUP_CODES):
+        if int(lens[g: g + GROUP_CODES].sum()) > 32:
+            return True
+    return False
+
+
 def encode_weight_blob(w_bits: np.ndarray, act_norm: np.ndarray | None, p: int, t: int,
                        seg_cols: int = 2048, chunk_cols: int = 256,
                        rowblocks=None):
@@ -142,7 +172,7 @@ def encode_weight_blob(w_bits: np.ndarray, act_norm: np.ndarray | None, p: int, 
     n, k = w_bits.shape
     if act_norm is None:
         act_norm = np.ones(k, dtype=np.float32)
-    assert chunk_cols % 32 == 0 and seg_cols % chunk_cols == 0 and seg_cols <= 4096
+    assert chunk_cols % 32 == 0 and seg_cols % chunk_cols == 0 and seg_cols <= 2048
     keep = codec.keep_mask_weights(w_bits, act_norm, p)
     counts = codec.exponent_counts(w_bits, keep)
     rank_to_exp = codec.codebook_from_counts(counts)
@@ -163,6 +193,7 @@ def encode_weight_blob(w_bits: np.ndarray, act_norm: np.ndarray | None, p: int, 
             scols = _segment_cols(k_pad, seg_cols, seg)
             n_ch = (scols + chunk_cols - 1) // chunk_cols
             rows_tab, rows_bm, rows_f, rows_u = [], [], [], []
+            irr = np.zeros((n_ch + 31) // 32 * 32, dtype=np.uint32)
             for rr in range(ROWS_PER_BLOCK):
                 r = rb * ROWS_PER_BLOCK + rr
                 km = np.zeros(scols, dtype=bool)
@@ -177,19 +208,29 @@ def encode_weight_blob(w_bits: np.ndarray, act_norm: np.ndarray | None, p: int, 
                 else:
                     fields = np.zeros(0, dtype=np.uint32)
                     ranks = np.zeros(0, dtype=np.int64)
-                # chunk table: running count of kept values and of code bits at each chunk start
-                tab = np.zeros(n_ch, dtype=np.uint32)
+                # chunk table: field-word index and code-bit offset at each chunk start.  The fields of a
+                # chunk start on a word boundary, so a decoder can enter the field stream at any chunk.
+                tab = np.zeros(n_ch + 1, dtype=np.uint32)
                 code_len = ranks + 1
                 cum_bits = np.concatenate(([0], np.cumsum(code_len)))
-                for ch in range(n_ch):
+                fparts = []
+                fword = 0
+                for ch in range(n_ch + 1):
                     first = int(np.searchsorted(idx, ch * chunk_cols))      # kept values before the chunk
                     bit_off = int(cum_bits[first])
-                    if first >= (1 << 12) or bit_off >= (1 << 20):
+                    if fword >= (1 << 12) or bit_off >= (1 << 20):
                         raise ValueError("chunk table overflow")
-                    tab[ch] = (first << 20) | bit_off
+                    tab[ch] = (fword << 20) | bit_off
+                    if ch < n_ch:
+                        last = int(np.searchsorted(idx, (ch + 1) * chunk_cols))
+                        fw = _pack_fields_fast(fields[first:last], t)
+                        fparts.append(fw)
+                        fword += fw.size
+                        if chunk_is_irregular(idx[first:last] - ch * chunk_cols, code_len[first:last]):
+                            irr[ch] |= np.uint32(1 << rr)
                 rows_tab.append(tab)
                 rows_bm.append(bits_to_words(km.astype(np.uint8)))
-                rows_f.append(_pack_fields_fast(fields, t))
+                rows_f.append(np.concatenate(fparts) if fparts else np.zeros(0, np.uint32))
                 rows_u.append(bits_to_words(codec.unary_encode_fast(ranks)) if ranks.size else np.zeros(0, np.uint32))
             w_f = max(x.size for x in rows_f)
             w_u = max(x.size for x in rows_u)
@@ -201,7 +242,7 @@ def encode_weight_blob(w_bits: np.ndarray, act_norm: np.ndarray | None, p: int, 
                 return sec.reshape(-1)
 
             body = np.concatenate([
-                interleave(rows_tab, n_ch), interleave(rows_bm, scols // 32),
+                irr, interleave(rows_tab, n_ch + 1), interleave(rows_bm, scols // 32),
                 interleave(rows_f, w_f), interleave(rows_u, w_u)])
             bodies[rb * n_seg + seg] = (body, w_f, w_u, n_ch)
 
@@ -223,8 +264,9 @@ def encode_weight_blob(w_bits: np.ndarray, act_norm: np.ndarray | None, p: int, 
         parts.append(body)
     total = off
     header = np.zeros(HEADER_BYTES // 4, dtype=np.uint32)
-    header[:15] = (MAGIC, VERSION, n, k, p, t, seg_cols, chunk_cols, n_seg, n_rb,
-                   k - codec.n_pruned(k, p), DIR_OFFSET, body_off, total & 0xFFFFFFFF, total >> 32)
+    header[:16] = (MAGIC, VERSION, n, k, p, t, seg_cols, chunk_cols, n_seg, n_rb,
+                   k - codec.n_pruned(k, p), DIR_OFFSET, body_off, total & 0xFFFFFFFF, total >> 32,
+                   max(b[0].size * 4 for b in bodies.values()))
     cb_words = np.frombuffer(rank_to_exp.tobytes(), dtype="<u4")
     pad = np.zeros((body_off - DIR_OFFSET - 16 * n_sb) // 4, dtype=np.uint32)
     blob = np.concatenate([header, cb_words, directory.reshape(-1), pad] + parts).astype(np.uint32)
@@ -261,8 +303,8 @@ def decode_weight_blob(blob: np.ndarray, use_chunk_table: bool = False) -> np.nd
         rb, seg = divmod(sb, info.n_seg)
         off16, w_f, w_u, n_ch = (int(x) for x in info.directory[sb])
         scols = _segment_cols(k_pad, info.seg_cols, seg)
-        base = off16 * 4
-        tab = blob[base: base + n_ch * 32].reshape(n_ch, 32); base += n_ch * 32
+        base = off16 * 4 + (n_ch + 31) // 32 * 32
+        tab = blob[base: base + (n_ch + 1) * 32].reshape(n_ch + 1, 32); base += (n_ch + 1) * 32
         bm = blob[base: base + scols // 32 * 32].reshape(scols // 32, 32); base += scols // 32 * 32
         fl = blob[base: base + w_f * 32].reshape(w_f, 32); base += w_f * 32
         un = blob[base: base + w_u * 32].reshape(w_u, 32)
@@ -272,22 +314,20 @@ def decode_weight_blob(blob: np.ndarray, use_chunk_table: bool = False) -> np.nd
             if idx.size == 0:
                 continue
             ubits = words_to_bits(un[:, rr])
+            fields = np.zeros(idx.size, dtype=np.uint32)
+            ranks = np.zeros(idx.size, dtype=np.int64)
             if not use_chunk_table:
-                fields = unpack_fields(fl[:, rr], idx.size, t)
                 ranks = codec.unary_decode_fast(ubits, idx.size)
-            else:
-                fields = np.zeros(idx.size, dtype=np.uint32)
-                ranks = np.zeros(idx.size, dtype=np.int64)
-                per = fields_per_word(t)
-                for ch in range(n_ch):
-                    first, bit_off = int(tab[ch, rr]) >> 20, int(tab[ch, rr]) & 0xFFFFF
-                    cnt = int(km[ch * info.chunk_cols: (ch + 1) * info.chunk_cols].sum())
-                    if cnt == 0:
-                        continue
-                    width = 8 - t
-                    for j in range(first, first + cnt):
-                        fields[j] = (int(fl[j // per, rr]) >> (32 - width * (j % per + 1))) & ((1 << width) - 1)
-                    ranks[first: first + cnt] = codec.unary_decode_fast(ubits[bit_off:], cnt)
+            done = 0
+            for ch in range(n_ch):
+                fword, bit_off = int(tab[ch, rr]) >> 20, int(tab[ch, rr]) & 0xFFFFF
+                cnt = int(km[ch * info.chunk_cols: (ch + 1) * info.chunk_cols].sum())
+                if cnt == 0:
+                    continue
+                fields[done: done + cnt] = unpack_fields(fl[fword:, rr], cnt, t)
+                if use_chunk_table:
+                    ranks[done: done + cnt] = codec.unary_decode_fast(ubits[bit_off:], cnt)
+                done += cnt
             e = info.codebook[ranks].astype(np.uint16)
             s = (fields >> (7 - t)).astype(np.uint16) & 1
             m_hi = (fields & ((1 << (7 - t)) - 1)).astype(np.uint16)
@@ -304,7 +344,7 @@ def blob_section_bits(blob: np.ndarray) -> dict:
     for sb in range(info.n_rowblocks * info.n_seg):
         _, w_f, w_u, n_ch = (int(x) for x in info.directory[sb])
         scols = _segment_cols(k_pad, info.seg_cols, sb % info.n_seg)
-        tab += n_ch * 32 * 32
+        tab += ((n_ch + 1) * 32 + (n_ch + 31) // 32 * 32) * 32
         bm += scols * 32
         fl += w_f * 32 * 32
         un += w_u * 32 * 32

@@ -1,0 +1,99 @@
+// Weight-blob format (device side): header indices, superblock geometry, and the generic
+// sequential decoder of one (row, chunk).
+//
+// Blob = header (128 B) | codebook rank->exponent (256 B) | directory (16 B per superblock) | bodies.
+// A superblock holds 32 rows x one column segment: an "irregular" mask (one word per chunk, padded to
+// 32 words), then chunk table, bitmap, fields and unary sections, each interleaved word by word over
+// the 32 rows.  All streams are filled MSB first.  See the format notes in the design document.
+#pragma once
+
+#include "common.cuh"
+
+namespace cass {
+
+enum BlobHeaderWord {
+    H_MAGIC = 0, H_VERSION, H_ROWS, H_COLS, H_P, H_T, H_SEG, H_CHUNK, H_NSEG, H_NRB, H_KEPT,
+    H_DIROFF, H_BODYOFF, H_TOTLO, H_TOTHI, H_MAXSB
+};
+constexpr uint32_t kBlobMagic = 0x57534143u;
+constexpr int kBlobHeaderBytes = 128;
+constexpr int kBlobCodebookBytes = 256;
+constexpr int kBlobDirOffset = kBlobHeaderBytes + kBlobCodebookBytes;
+
+// Word offsets of the sections of one superblock.
+struct SbGeom {
+    int n_ch;       // chunks in this segment
+    int bm_words;   // bitmap words per row
+    int w_f, w_u;   // field / unary words per row
+    int tab, bm, fl, un, total;   // section starts and total size, in words
+
+    __host__ __device__ static SbGeom make(int n_ch, int seg_cols_here, int w_f, int w_u) {
+        SbGeom g;
+        g.n_ch = n_ch;
+        g.bm_words = seg_cols_here / 32;
+        g.w_f = w_f;
+        g.w_u = w_u;
+        g.tab = ceil_div(n_ch, 32) * 32;
+        g.bm = g.tab + (n_ch + 1) * 32;
+        g.fl = g.bm + g.bm_words * 32;
+        g.un = g.fl + w_f * 32;
+        g.total = g.un + w_u * 32;
+        return g;
+    }
+};
+
+__host__ __device__ inline int seg_cols_of(int k_pad, int seg_cols, int seg) {
+    int rest = k_pad - seg * seg_cols;
+    return rest < seg_cols ? rest : seg_cols;
+}
+
+// Reads one codeword starting at absolute bit `ub` of a row's unary stream (words un[j*32]); returns the
+// number of zeros before the terminating one and advances ub past it.  Handles codewords of any length.
+// `limit_bits` bounds the scan so that a corrupt stream cannot run away.
+__device__ __forceinline__ int read_unary(const uint32_t* un_row, uint32_t& ub, uint32_t limit_bits) {
+    int rank = 0;
+    while (ub < limit_bits) {
+        uint32_t w = un_row[(ub >> 5) * 32] << (ub & 31);
+        int avail = 32 - (int)(ub & 31);
+        if (w) {
+            int s = __clz(w);
+            ub += s + 1;
+            return rank + s;
+        }
+        rank += avail;
+        ub += avail;
+    }
+    return rank;
+}
+
+// Generic decoder of one (row, chunk): calls emit(col_in_segment, bf16_bits) for every kept value, in
+// column order.  `sb` points at the superblock's first word (global or shared memory); `row` in [0,32).
+template <class Emit>
+__device__ inline void decode_chunk_generic(const uint32_t* sb, const SbGeom& g, int chunk_cols, int ch, int row,
+                                            int t, const uint8_t* rank_to_exp, Emit&& emit) {
+    const int F = 8 - t, per = 32 / F;
+    const uint32_t e0 = sb[g.tab + ch * 32 + row];
+    uint32_t fw = e0 >> 20, ub = e0 & 0xFFFFFu;
+    const uint32_t* fl_row = sb + g.fl + row;
+    const uint32_t* un_row = sb + g.un + row;
+    const uint32_t limit = (uint32_t)g.w_u * 32u;
+    const int w0 = ch * (chunk_cols / 32);
+    const int w1 = min(w0 + chunk_cols / 32, g.bm_words);
+    int k = 0;                                       // kept values seen in this chunk
+    for (int w = w0; w < w1; ++w) {
+        uint32_t bm = sb[g.bm + w * 32 + row];
+        while (bm) {
+            int s = __clz(bm);
+            bm &= ~(0x80000000u >> s);
+            uint32_t fword = fl_row[(fw + k / per) * 32];
+            uint32_t f = (fword >> (32 - F * (k % per + 1))) & ((1u << F) - 1u);
+            int rank = read_unary(un_row, ub, limit);
+            uint32_t e = rank_to_exp[rank & 255];
+            uint32_t sign = f >> (F - 1), mhi = f & ((1u << (F - 1)) - 1u);
+            emit(w * 32 + s, (uint16_t)((sign << 15) | (e << 7) | (mhi << t)));
+            ++k;
+        }
+    }
+}
+
+}  // namespace cass
