@@ -15,8 +15,27 @@ import numpy as np
 from . import codec, layout
 
 
+_ACC = np.float64      # accumulation type; fp64 is the oracle, fp32 only serves sensitivity studies
+
+
+class accumulate_in:
+    """Context manager: evaluate the model with another accumulation type (used to measure how far the bf16
+    rounding points amplify accumulation error, i.e. the noise floor of a logit comparison)."""
+
+    def __init__(self, dtype):
+        self.dtype = dtype
+
+    def __enter__(self):
+        global _ACC
+        self.prev, _ACC = _ACC, self.dtype
+
+    def __exit__(self, *a):
+        global _ACC
+        _ACC = self.prev
+
+
 def _f(bits):
-    return codec.bf16_bits_to_f64(bits)
+    return codec.bf16_bits_to_f64(bits).astype(_ACC)
 
 
 def _r(x):
@@ -49,7 +68,7 @@ class Weights:
     """Dense fp64 views of a model's matrices (exact bf16 values)."""
 
     def __init__(self, shape, w_bits: dict):
-        self.shape = shape
+        self.shape = shape          # matrices take the accumulation type in force at construction (fp64 by default)
         self.layers = [{k: _f(v) if k.startswith("w") else np.asarray(v, dtype=np.uint16) for k, v in lw.items()}
                        for lw in w_bits["layers"]]
         self.embed_bits = np.asarray(w_bits["embed"], dtype=np.uint16)
@@ -120,10 +139,10 @@ def forward_token(W: Weights, kv: KVCache, tok: int, pos: int, draft: bool, kv_p
         kc = _f((kv.kd if draft else kv.k)[li, : pos + 1])          # [pos+1, n_kv, d]
         vc = _f((kv.vd if draft else kv.v)[li, : pos + 1])
         qf = _f(q)
-        o = np.zeros((s.n_q_heads, d))
+        o = np.zeros((s.n_q_heads, d), dtype=_ACC)
         for hq in range(s.n_q_heads):
             hk = hq // g
-            sc = (kc[:, hk, :] @ qf[hq]) / np.sqrt(float(d))
+            sc = (kc[:, hk, :] @ qf[hq]) / _ACC(np.sqrt(float(d)))
             sc = sc - sc.max()
             pr = np.exp(sc)
             pr = pr / pr.sum()
@@ -137,7 +156,7 @@ def forward_token(W: Weights, kv: KVCache, tok: int, pos: int, draft: bool, kv_p
         x = _f(xn)
         gate = _f(_r(lw["wg"] @ x))
         up = _f(_r(lw["wu"] @ x))
-        act = _r(gate / (1.0 + np.exp(-gate)) * up)
+        act = _r(gate / (_ACC(1.0) + np.exp(-gate)) * up)
         note(li, ("wd",), act)
         down = _r(lw["wd"] @ _f(act))
         h = _r(_f(h) + _f(down))

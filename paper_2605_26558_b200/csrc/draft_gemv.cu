@@ -88,11 +88,12 @@ __device__ __forceinline__ float chunk_dot_fast(const uint32_t* __restrict__ sb,
 // T >= 0: fast path for regular chunks, generic path otherwise.  T = -1: generic path only (any t).
 template <int T>
 __global__ void __launch_bounds__(1024) k_draft_gemv(const uint32_t* __restrict__ blob, const uint16_t* __restrict__ x,
-                                                     float* __restrict__ partial, int32_t* __restrict__ d_status) {
+                                                     float* __restrict__ partial, int32_t* __restrict__ d_status,
+                                                     int max_sb /* shared-memory room for one superblock */, int seg_cols_host) {
     extern __shared__ __align__(128) uint8_t smem_raw[];
     const uint32_t* h = blob;
     const int n = h[H_ROWS], k = h[H_COLS], t = h[H_T], seg_cols = h[H_SEG], chunk_cols = h[H_CHUNK];
-    const int n_seg = h[H_NSEG], n_rb = h[H_NRB], max_sb = h[H_MAXSB];
+    const int n_seg = h[H_NSEG], n_rb = h[H_NRB];
     const int k_pad = ceil_div(k, 32) * 32;
     const int sb_i = blockIdx.x, rb = sb_i / n_seg, seg = sb_i % n_seg;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, n_warps = blockDim.x >> 5;
@@ -107,6 +108,12 @@ __global__ void __launch_bounds__(1024) k_draft_gemv(const uint32_t* __restrict_
     const int scols = seg_cols_of(k_pad, seg_cols, seg);
     const SbGeom g = SbGeom::make((int)dir[3], scols, (int)dir[1], (int)dir[2]);
     const uint32_t bytes = (uint32_t)g.total * 4u;
+    // The launch sized shared memory from the host's copy of the header; a blob that does not match it
+    // (larger superblock, other segment geometry) is refused instead of overrunning the buffer.
+    if (bytes > (uint32_t)max_sb || (int)blockDim.x < 32 * g.n_ch || seg_cols != seg_cols_host || g.n_ch > 32) {
+        if (tid == 0 && d_status) atomicExch(d_status, CASS_ERR_INVALID_ARG);
+        return;
+    }
 
     if (tid == 0) {
         mbar_init(bar, 1);
@@ -179,9 +186,13 @@ int launch_draft_gemv(const void* blob, const cass_blob_info& bi, const void* x_
     const uint16_t* x = (const uint16_t*)x_bf16;
 #define CASS_GEMV_LAUNCH(TT)                                                                                   \
     do {                                                                                                       \
-        CASS_CUDA_CHECK(cudaFuncSetAttribute(k_draft_gemv<TT>, cudaFuncAttributeMaxDynamicSharedMemorySize,    \
-                                             (int)smem));                                                      \
-        k_draft_gemv<TT><<<grid, block, smem, stream>>>(b, x, partial, d_status);                              \
+        static int attr_smem = 0;      /* largest size already granted to this instantiation */              \
+        if ((int)smem > attr_smem) {                                                                           \
+            CASS_CUDA_CHECK(cudaFuncSetAttribute(k_draft_gemv<TT>, cudaFuncAttributeMaxDynamicSharedMemorySize,\
+                                                 (int)smem));                                                  \
+            attr_smem = (int)smem;                                                                             \
+        }                                                                                                      \
+        k_draft_gemv<TT><<<grid, block, smem, stream>>>(b, x, partial, d_status, bi.max_superblock_bytes, bi.seg_cols);                              \
     } while (0)
     if (bi.trunc_bits == 4) CASS_GEMV_LAUNCH(4);
     else if (bi.trunc_bits == 0) CASS_GEMV_LAUNCH(0);

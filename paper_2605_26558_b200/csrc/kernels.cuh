@@ -5,9 +5,85 @@
 
 namespace cass {
 
+// Device-resident step state of one sequence; kernels read positions from here so that a captured graph of
+// launches can be replayed without host-side position arguments.
+struct DevState {
+    int32_t len;        // committed KV positions
+    int32_t inflight;   // draft tokens appended since the last accept
+    int32_t status;     // first device-side error (CASS_ERR_*), 0 if none
+    int32_t calib_on;
+};
+
+// Compressed KV cache of one (layer, K|V): per head a fixed part (bitmap + fields, 32-token blocks interleaved
+// word by word), an append-only arena of unary words and per-token word offsets.
+struct KvComp {
+    uint32_t* fixed;        // [n_kv][n_blocks][wpt][32]
+    uint32_t* arena;        // [n_kv][arena_words]
+    uint32_t* off;          // [n_kv][max_seq + 1]
+    uint8_t* rank_to_exp;   // [256]
+    uint8_t* exp_to_rank;   // [256]
+    unsigned long long* hist;   // [256]
+};
+
+struct KvGeom {
+    int n_kv, d, max_seq, n_blocks, wpt, bm_words, f_words, kept, n_prune, t, arena_words;
+};
+
+constexpr int kAttnChunk = 256;      // split-K granularity over the sequence (fixed absolute boundaries)
+
 size_t gemv_smem_bytes(const cass_blob_info& bi);
 // partial: fp32 [n_seg][n_rowblocks*32]; the caller sums the segments (fixed order) afterwards.
 int launch_draft_gemv(const void* blob, const cass_blob_info& bi, const void* x_bf16, float* partial,
                       int32_t* d_status, cudaStream_t stream);
+
+// ---- small ops (ops.cu) -------------------------------------------------------------------------------
+int launch_rope_table(float* cos_t, float* sin_t, int max_seq, int d, float theta, cudaStream_t s);
+int launch_embed(const int32_t* toks, const uint16_t* embed, uint16_t* h, int rows, int hidden, cudaStream_t s);
+int launch_rmsnorm(const uint16_t* h, const uint16_t* gain, uint16_t* out, int rows, int hidden, float eps,
+                   cudaStream_t s);
+// h = bf16(h + y); out = rmsnorm(h) * gain.  y comes either as bf16 [rows][hidden] or (rows == 1) as fp32 split-K
+// partials [n_seg][n_pad] that are summed in segment order and rounded to bf16 first.
+int launch_residual_rmsnorm(uint16_t* h, const uint16_t* y_bf16, const float* partial, int n_seg, int n_pad,
+                            const uint16_t* gain, uint16_t* out, int rows, int hidden, float eps, cudaStream_t s);
+// q and k of qkv (bf16 [rows][qkv_dim]) rotated in place at position base + row (base from state: len, or
+// len + inflight when use_inflight).  With partial != NULL (rows == 1) qkv is first formed from the partials.
+int launch_qkv_rope(uint16_t* qkv, const float* partial, int n_seg, int n_pad, const float* cos_t, const float* sin_t,
+                    const DevState* st, int use_inflight, int rows, int n_q, int n_kv, int d, cudaStream_t s);
+int launch_swiglu(const uint16_t* gu_bf16, const float* partial, int n_seg, int n_pad, uint16_t* act, int rows,
+                  int ffn, cudaStream_t s);
+// logits (fp32 [rows][vocab], or formed from partials when rows == 1) -> lowest-index argmax per row; optional copy
+// of the logits; bump_inflight adds 1 to the draft counter afterwards.
+int launch_argmax(const float* logits, const float* partial, int n_seg, int n_pad, int rows, int vocab, int32_t* out,
+                  float* logits_copy, DevState* st, int bump_inflight, cudaStream_t s);
+int launch_accept(DevState* st, const int32_t* draft, const int32_t* target, int g, int32_t* n_acc,
+                  int32_t* out_tokens, int32_t* next_tok, cudaStream_t s);
+int launch_calib_accum(const uint16_t* x, int rows, int cols, float* sumsq, const DevState* st, cudaStream_t s);
+int launch_sqrt(const float* in, float* out, size_t n, cudaStream_t s);
+
+// ---- KV encoder (kv.cu) -------------------------------------------------------------------------------
+// src_k/src_v: bf16 rows with `row_stride` elements between tokens and n_kv*d contiguous per token.
+// start_pos < 0: take the position from the state (len, or len + inflight when use_inflight).
+int launch_kv_append(const KvGeom& g, const KvComp& ck, const KvComp& cv, uint16_t* k_cache, uint16_t* v_cache,
+                     const uint16_t* src_k, const uint16_t* src_v, int row_stride, int start_pos, int use_inflight,
+                     int n_new, int flags, DevState* st, cudaStream_t s);
+int launch_kv_codebook(const KvGeom& g, const KvComp& ck, const KvComp& cv, const uint16_t* k_cache,
+                       const uint16_t* v_cache, int n_tokens, cudaStream_t s);
+
+// ---- attention ----------------------------------------------------------------------------------------
+struct AttnScratch {
+    float* o;     // [rows*n_q][n_chunks][d]
+    float* m;     // [rows*n_q][n_chunks]
+    float* l;     // [rows*n_q][n_chunks]
+};
+// Draft: one query row at position len + inflight over the compressed cache.
+int launch_draft_attn(const KvGeom& g, const KvComp& ck, const KvComp& cv, const uint16_t* qkv, int n_q,
+                      const DevState* st, const AttnScratch& sc, uint16_t* out, cudaStream_t s);
+// Verify: rows at positions len + r over the bf16 cache, causal.
+int launch_verify_attn(const KvGeom& g, const uint16_t* k_cache, const uint16_t* v_cache, const uint16_t* qkv,
+                       int rows, int n_q, const DevState* st, const AttnScratch& sc, uint16_t* out, cudaStream_t s);
+
+// ---- verification GEMM (verify_gemm.cu): Y[r][n] = sum_k W[n][k] X[r][k], bf16 in, fp32 accumulate -------------
+int launch_verify_gemm(const uint16_t* W, const uint16_t* X, int rows, int n, int k, uint16_t* y_bf16, float* y_f32,
+                       cudaStream_t s);
 
 }  // namespace cass

@@ -1,0 +1,202 @@
+// Online KV encoder (Sec. 4.2: per-token magnitude pruning of K and V, mantissa truncation, unary exponent
+// code; Sec. 5.1 encoder): one warp formats one (token, KV head, K|V) record; records are appended to the
+// compressed cache and, on request, the raw bf16 rows go to the target's cache.
+#include "kernels.cuh"
+
+namespace cass {
+
+constexpr int kKvMaxPerLane = 8;       // head_dim <= 256
+constexpr int kKvStageWords = 96;      // unary staging per token: up to 3072 code bits
+constexpr int kKvWarps = 8;
+constexpr int kKvFixMax = 72;        // head_dim 256, no truncation: 8 bitmap + 64 field words
+
+// Per-token selection: lane holds elements c = lane + 32 j.  keep[j] is set for the d - n_prune largest
+// |x| (ties: the lower channel is pruned first).  Key = (|x| bits << 8) | channel is unique.
+__device__ __forceinline__ void kv_select(const uint32_t (&bits)[kKvMaxPerLane], int nj, int n_prune, int lane,
+                                          bool (&keep)[kKvMaxPerLane]) {
+    uint32_t key[kKvMaxPerLane];
+    int below[kKvMaxPerLane];
+#pragma unroll
+    for (int j = 0; j < kKvMaxPerLane; ++j) {
+        key[j] = j < nj ? (((bits[j] & 0x7FFFu) << 8) | (uint32_t)(lane + 32 * j)) : 0xFFFFFFFFu;
+        below[j] = 0;
+    }
+    for (int jj = 0; jj < nj; ++jj) {
+        for (int src = 0; src < 32; ++src) {
+            uint32_t other = __shfl_sync(0xffffffffu, key[jj], src);
+#pragma unroll
+            for (int j = 0; j < kKvMaxPerLane; ++j) below[j] += other < key[j];
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < kKvMaxPerLane; ++j) keep[j] = j < nj && below[j] >= n_prune;
+}
+
+__global__ void __launch_bounds__(256) k_kv_hist(KvGeom g, KvComp ck, KvComp cv, const uint16_t* __restrict__ k_cache,
+                                                 const uint16_t* __restrict__ v_cache, int n_tokens) {
+    __shared__ unsigned int s_hist[256];
+    const int head = blockIdx.x, kind = blockIdx.y;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint16_t* cache = kind ? v_cache : k_cache;
+    s_hist[threadIdx.x] = 0;
+    __syncthreads();
+    const int nj = g.d / 32;
+    for (int t = blockIdx.z * kKvWarps + warp; t < n_tokens; t += gridDim.z * kKvWarps) {
+        uint32_t bits[kKvMaxPerLane];
+        bool keep[kKvMaxPerLane];
+        const uint16_t* src = cache + ((size_t)t * g.n_kv + head) * g.d;
+#pragma unroll
+        for (int j = 0; j < kKvMaxPerLane; ++j) bits[j] = j < nj ? src[lane + 32 * j] : 0;
+        kv_select(bits, nj, g.n_prune, lane, keep);
+#pragma unroll
+        for (int j = 0; j < kKvMaxPerLane; ++j)
+            if (keep[j]) atomicAdd(&s_hist[(bits[j] >> 7) & 0xFF], 1u);
+    }
+    __syncthreads();
+    unsigned long long* hist = kind ? cv.hist : ck.hist;
+    if (s_hist[threadIdx.x]) atomicAdd(&hist[threadIdx.x], (unsigned long long)s_hist[threadIdx.x]);
+}
+
+__global__ void k_kv_rank(KvComp ck, KvComp cv) {
+    __shared__ unsigned long long s[256];
+    KvComp c = blockIdx.x ? cv : ck;
+    int e = threadIdx.x;
+    s[e] = c.hist[e];
+    __syncthreads();
+    unsigned long long mine = s[e];
+    int rank = 0;
+    for (int o = 0; o < 256; ++o) rank += (s[o] > mine) || (s[o] == mine && o < e);
+    c.rank_to_exp[rank] = (uint8_t)e;
+    c.exp_to_rank[e] = (uint8_t)rank;
+}
+
+// grid (n_kv, 2): block of 8 warps walks the n_new tokens in batches of 8; offsets into the unary arena are
+// assigned sequentially by one thread per batch, so records stay densely packed in token order.
+__global__ void __launch_bounds__(256) k_kv_append(KvGeom g, KvComp ck, KvComp cv, uint16_t* __restrict__ k_cache,
+                                                   uint16_t* __restrict__ v_cache, const uint16_t* __restrict__ src_k,
+                                                   const uint16_t* __restrict__ src_v, int row_stride, int start_pos_arg,
+                                                   int use_inflight, int n_new, int flags, DevState* st) {
+    __shared__ uint32_t s_fix[kKvWarps][kKvFixMax];          // bitmap (<= 8) + field words (<= 64)
+    __shared__ uint32_t s_una[kKvWarps][kKvStageWords];
+    __shared__ uint32_t s_nw[kKvWarps], s_off[kKvWarps];
+    const int head = blockIdx.x, kind = blockIdx.y;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const KvComp c = kind ? cv : ck;
+    const uint16_t* src = kind ? src_v : src_k;
+    uint16_t* cache = kind ? v_cache : k_cache;
+    const int start_pos = start_pos_arg >= 0 ? start_pos_arg : st->len + (use_inflight ? st->inflight : 0);
+    const int nj = g.d / 32, t_bits = g.t, F = 8 - t_bits, per = 32 / F;
+    uint32_t* off = c.off + (size_t)head * (g.max_seq + 1);
+    uint32_t* arena = c.arena + (size_t)head * g.arena_words;
+    uint32_t* fixed = c.fixed + (size_t)head * g.n_blocks * g.wpt * 32;
+
+    for (int base = 0; base < n_new; base += kKvWarps) {
+        const int i = base + warp;
+        const bool active = i < n_new && start_pos + i < g.max_seq;
+        const int pos = start_pos + i;
+        uint32_t bits[kKvMaxPerLane];
+        bool keep[kKvMaxPerLane];
+        uint32_t n_words = 0;
+        if (active) {
+            const uint16_t* row = src + (size_t)i * row_stride + (size_t)head * g.d;
+#pragma unroll
+            for (int j = 0; j < kKvMaxPerLane; ++j) bits[j] = j < nj ? row[lane + 32 * j] : 0;
+            if (flags & CASS_KV_BF16) {
+                uint16_t* dst = cache + ((size_t)pos * g.n_kv + head) * g.d;
+#pragma unroll
+                for (int j = 0; j < kKvMaxPerLane; ++j)
+                    if (j < nj) dst[lane + 32 * j] = (uint16_t)bits[j];
+            }
+        }
+        if (flags & CASS_KV_COMPRESSED) {
+            if (active) {
+                kv_select(bits, nj, g.n_prune, lane, keep);
+                for (int w = lane; w < kKvFixMax; w += 32) s_fix[warp][w] = 0;
+                for (int w = lane; w < kKvStageWords; w += 32) s_una[warp][w] = 0;
+                __syncwarp();
+                uint32_t kbase = 0, ubase = 0;
+#pragma unroll
+                for (int j = 0; j < kKvMaxPerLane; ++j) {
+                    if (j < nj) {
+                        uint32_t bm = __brev(__ballot_sync(0xffffffffu, keep[j]));   // channel c at bit 31 - c%32
+                        if (lane == 0) s_fix[warp][j] = bm;
+                        uint32_t len = keep[j] ? (uint32_t)c.exp_to_rank[(bits[j] >> 7) & 0xFF] + 1u : 0u;
+                        uint32_t incl = len;
+#pragma unroll
+                        for (int o = 1; o < 32; o <<= 1) {
+                            uint32_t v = __shfl_up_sync(0xffffffffu, incl, o);
+                            if (lane >= o) incl += v;
+                        }
+                        if (keep[j]) {
+                            uint32_t k = kbase + (lane ? __popc(bm >> (32 - lane)) : 0u);
+                            uint32_t field = ((bits[j] >> 15) << (7 - t_bits)) | ((bits[j] & 0x7Fu) >> t_bits);
+                            atomicOr(&s_fix[warp][nj + k / per], field << (32 - F * (k % per + 1)));
+                            uint32_t p = ubase + incl - 1;
+                            if ((p >> 5) < (uint32_t)kKvStageWords) atomicOr(&s_una[warp][p >> 5], 0x80000000u >> (p & 31));
+                        }
+                        kbase += __popc(bm);
+                        ubase += __shfl_sync(0xffffffffu, incl, 31);
+                    }
+                }
+                n_words = (ubase + 31) / 32;
+                if (n_words > (uint32_t)kKvStageWords) {          // record too long for the staging buffer
+                    if (lane == 0) atomicCAS(&st->status, 0, CASS_ERR_CAPACITY);
+                    n_words = kKvStageWords;
+                }
+            }
+            if (lane == 0) s_nw[warp] = active ? n_words : 0u;
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                uint32_t o = off[start_pos + base];
+                for (int w = 0; w < kKvWarps; ++w) {
+                    int p = start_pos + base + w;
+                    if (base + w >= n_new || p >= g.max_seq) break;
+                    uint32_t nw = s_nw[w];
+                    if (o + nw > (uint32_t)g.arena_words) {           // arena full: keep offsets valid, drop the codes
+                        atomicCAS(&st->status, 0, CASS_ERR_CAPACITY);
+                        nw = 0;
+                        s_nw[w] = 0;
+                    }
+                    s_off[w] = o;
+                    o += nw;
+                    off[p + 1] = o;
+                }
+            }
+            __syncthreads();
+            if (active) {
+                uint32_t* blk = fixed + (size_t)(pos / 32) * g.wpt * 32 + (pos % 32);
+                for (int w = lane; w < g.wpt; w += 32) blk[w * 32] = s_fix[warp][w];
+                uint32_t o = s_off[warp], nw = s_nw[warp];
+                for (uint32_t w = lane; w < nw; w += 32) arena[o + w] = s_una[warp][w];
+            }
+            __syncthreads();
+        }
+    }
+}
+
+int launch_kv_append(const KvGeom& g, const KvComp& ck, const KvComp& cv, uint16_t* k_cache, uint16_t* v_cache,
+                     const uint16_t* src_k, const uint16_t* src_v, int row_stride, int start_pos, int use_inflight,
+                     int n_new, int flags, DevState* st, cudaStream_t s) {
+    if (n_new <= 0) return CASS_OK;
+    dim3 grid(g.n_kv, 2);
+    k_kv_append<<<grid, 256, 0, s>>>(g, ck, cv, k_cache, v_cache, src_k, src_v, row_stride, start_pos, use_inflight,
+                                     n_new, flags, st);
+    CASS_LAUNCH_CHECK();
+    return CASS_OK;
+}
+
+int launch_kv_codebook(const KvGeom& g, const KvComp& ck, const KvComp& cv, const uint16_t* k_cache,
+                       const uint16_t* v_cache, int n_tokens, cudaStream_t s) {
+    CASS_CUDA_CHECK(cudaMemsetAsync(ck.hist, 0, 256 * 8, s));
+    CASS_CUDA_CHECK(cudaMemsetAsync(cv.hist, 0, 256 * 8, s));
+    if (n_tokens > 0) {
+        dim3 grid(g.n_kv, 2, min(64, ceil_div(n_tokens, kKvWarps)));
+        k_kv_hist<<<grid, 256, 0, s>>>(g, ck, cv, k_cache, v_cache, n_tokens);
+        CASS_LAUNCH_CHECK();
+    }
+    k_kv_rank<<<2, 256, 0, s>>>(ck, cv);
+    CASS_LAUNCH_CHECK();
+    return CASS_OK;
+}
+
+}  // namespace cass

@@ -1,0 +1,266 @@
+// Small per-token operators of the decoder layer (Sec. 2.1): embedding gather, RMSNorm, RoPE, SwiGLU, residual
+// add, greedy argmax, and the greedy accept / rollback step (Sec. 2.2).  Activations are bf16 between
+// operators; arithmetic inside an operator is fp32.
+#include "kernels.cuh"
+
+namespace cass {
+
+__global__ void k_rope_table(float* __restrict__ cos_t, float* __restrict__ sin_t, int max_seq, int half, float theta) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= (size_t)max_seq * half) return;
+    int pos = (int)(i / half), j = (int)(i % half);
+    double inv = pow((double)theta, -2.0 * (double)j / (double)(2 * half));
+    double ang = (double)pos * inv;
+    cos_t[i] = (float)cos(ang);
+    sin_t[i] = (float)sin(ang);
+}
+
+__global__ void k_embed(const int32_t* __restrict__ toks, const uint16_t* __restrict__ embed, uint16_t* __restrict__ h,
+                        int hidden) {
+    int r = blockIdx.x;
+    const uint16_t* src = embed + (size_t)toks[r] * hidden;
+    for (int i = threadIdx.x; i < hidden; i += blockDim.x) h[(size_t)r * hidden + i] = src[i];
+}
+
+__device__ __forceinline__ float block_sum(float v, float* s_red) {
+    v = warp_sum(v);
+    int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+    __syncthreads();
+    if (lane == 0) s_red[warp] = v;
+    __syncthreads();
+    float t = 0.f;
+    for (int i = 0; i < nw; ++i) t += s_red[i];
+    return t;
+}
+
+// h (+= y) then out = h * rsqrt(mean(h^2) + eps) * gain, all rounded to bf16 where stored.
+__global__ void __launch_bounds__(1024) k_residual_rmsnorm(uint16_t* __restrict__ h, const uint16_t* __restrict__ y_bf16,
+                                                           const float* __restrict__ partial, int n_seg, int n_pad,
+                                                           const uint16_t* __restrict__ gain, uint16_t* __restrict__ out,
+                                                           int hidden, float eps) {
+    __shared__ float s_red[32];
+    const int r = blockIdx.x;
+    uint16_t* hr = h + (size_t)r * hidden;
+    float ss = 0.f;
+    for (int i = threadIdx.x; i < hidden; i += blockDim.x) {
+        float v = bf16_bits_to_float(hr[i]);
+        if (y_bf16 || partial) {
+            float y;
+            if (partial) {
+                float acc = 0.f;
+                for (int s = 0; s < n_seg; ++s) acc += partial[(size_t)s * n_pad + i];
+                y = round_bf16(acc);
+            } else {
+                y = bf16_bits_to_float(y_bf16[(size_t)r * hidden + i]);
+            }
+            v = round_bf16(v + y);
+            hr[i] = float_to_bf16_bits(v);
+        }
+        ss += v * v;
+    }
+    ss = block_sum(ss, s_red);
+    const float inv = 1.0f / sqrtf(ss / (float)hidden + eps);
+    if (out) {
+        for (int i = threadIdx.x; i < hidden; i += blockDim.x) {
+            float v = bf16_bits_to_float(hr[i]);
+            out[(size_t)r * hidden + i] = float_to_bf16_bits(v * inv * bf16_bits_to_float(gain[i]));
+        }
+    }
+}
+
+__global__ void k_qkv_rope(uint16_t* __restrict__ qkv, const float* __restrict__ partial, int n_seg, int n_pad,
+                           const float* __restrict__ cos_t, const float* __restrict__ sin_t,
+                           const DevState* __restrict__ st, int use_inflight, int n_q, int n_kv, int d) {
+    const int r = blockIdx.y, half = d / 2;
+    const int qkv_dim = (n_q + 2 * n_kv) * d;
+    const int pos = st->len + (use_inflight ? st->inflight : 0) + r;
+    uint16_t* row = qkv + (size_t)r * qkv_dim;
+    const int n_rot = (n_q + n_kv) * half;             // rotated pairs
+    const int n_items = n_rot + n_kv * d;              // + plain v elements
+    auto load = [&](int i) -> float {
+        if (partial) {
+            float acc = 0.f;
+            for (int s = 0; s < n_seg; ++s) acc += partial[(size_t)s * n_pad + i];
+            return round_bf16(acc);
+        }
+        return bf16_bits_to_float(row[i]);
+    };
+    for (int it = blockIdx.x * blockDim.x + threadIdx.x; it < n_items; it += gridDim.x * blockDim.x) {
+        if (it < n_rot) {
+            int head = it / half, j = it % half;
+            int ia = head * d + j, ib = ia + half;
+            float a = load(ia), b = load(ib);
+            float c = cos_t[(size_t)pos * half + j], s = sin_t[(size_t)pos * half + j];
+            row[ia] = float_to_bf16_bits(a * c - b * s);
+            row[ib] = float_to_bf16_bits(b * c + a * s);
+        } else if (partial) {
+            int i = (n_q + n_kv) * d + (it - n_rot);
+            row[i] = float_to_bf16_bits(load(i));
+        }
+    }
+}
+
+__global__ void k_swiglu(const uint16_t* __restrict__ gu, const float* __restrict__ partial, int n_seg, int n_pad,
+                         uint16_t* __restrict__ act, int ffn) {
+    const int r = blockIdx.y;
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < ffn; i += gridDim.x * blockDim.x) {
+        float g, u;
+        if (partial) {
+            float ag = 0.f, au = 0.f;
+            for (int s = 0; s < n_seg; ++s) {
+                ag += partial[(size_t)s * n_pad + i];
+                au += partial[(size_t)s * n_pad + ffn + i];
+            }
+            g = round_bf16(ag);
+            u = round_bf16(au);
+        } else {
+            g = bf16_bits_to_float(gu[(size_t)r * 2 * ffn + i]);
+            u = bf16_bits_to_float(gu[(size_t)r * 2 * ffn + ffn + i]);
+        }
+        float silu = g / (1.0f + expf(-g));
+        act[(size_t)r * ffn + i] = float_to_bf16_bits(silu * u);
+    }
+}
+
+__global__ void __launch_bounds__(1024) k_argmax(const float* __restrict__ logits, const float* __restrict__ partial,
+                                                 int n_seg, int n_pad, int vocab, int32_t* __restrict__ out,
+                                                 float* __restrict__ logits_copy, DevState* st, int bump_inflight) {
+    __shared__ float s_v[32];
+    __shared__ int s_i[32];
+    const int r = blockIdx.x;
+    float best = -INFINITY;
+    int best_i = 0x7fffffff;
+    for (int i = threadIdx.x; i < vocab; i += blockDim.x) {
+        float v;
+        if (partial) {
+            v = 0.f;
+            for (int s = 0; s < n_seg; ++s) v += partial[(size_t)s * n_pad + i];
+        } else {
+            v = logits[(size_t)r * vocab + i];
+        }
+        if (logits_copy) logits_copy[(size_t)r * vocab + i] = v;
+        if (v > best || (v == best && i < best_i)) { best = v; best_i = i; }
+    }
+    for (int o = 16; o > 0; o >>= 1) {
+        float ov = __shfl_xor_sync(0xffffffffu, best, o);
+        int oi = __shfl_xor_sync(0xffffffffu, best_i, o);
+        if (ov > best || (ov == best && oi < best_i)) { best = ov; best_i = oi; }
+    }
+    int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (lane == 0) { s_v[warp] = best; s_i[warp] = best_i; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int w = 1; w < (int)(blockDim.x >> 5); ++w)
+            if (s_v[w] > best || (s_v[w] == best && s_i[w] < best_i)) { best = s_v[w]; best_i = s_i[w]; }
+        out[r] = best_i == 0x7fffffff ? 0 : best_i;
+        if (bump_inflight && r == 0) st->inflight += 1;
+    }
+}
+
+// Greedy acceptance: a = min({i-1 : draft_i != target_{i-1}} U {g}); emit draft_1..draft_a and target_a.
+__global__ void k_accept(DevState* st, const int32_t* __restrict__ draft, const int32_t* __restrict__ target, int g,
+                         int32_t* n_acc, int32_t* out_tokens, int32_t* next_tok) {
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    int a = 0;
+    while (a < g && draft[a] == target[a]) ++a;
+    for (int i = 0; i < a; ++i) out_tokens[i] = draft[i];
+    out_tokens[a] = target[a];
+    for (int i = a + 1; i <= g; ++i) out_tokens[i] = -1;
+    *n_acc = a;
+    if (next_tok) *next_tok = target[a];
+    st->len += a + 1;
+    st->inflight = 0;
+}
+
+__global__ void k_calib_accum(const uint16_t* __restrict__ x, int rows, int cols, float* __restrict__ sumsq,
+                              const DevState* __restrict__ st) {
+    if (!st->calib_on) return;
+    int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= cols) return;
+    float acc = sumsq[c];
+    for (int r = 0; r < rows; ++r) {
+        float v = bf16_bits_to_float(x[(size_t)r * cols + c]);
+        acc += v * v;
+    }
+    sumsq[c] = acc;
+}
+
+__global__ void k_sqrt(const float* __restrict__ in, float* __restrict__ out, size_t n) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) out[i] = sqrtf(in[i]);
+}
+
+int launch_rope_table(float* cos_t, float* sin_t, int max_seq, int d, float theta, cudaStream_t s) {
+    size_t n = (size_t)max_seq * (d / 2);
+    k_rope_table<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(cos_t, sin_t, max_seq, d / 2, theta);
+    CASS_LAUNCH_CHECK();
+    return CASS_OK;
+}
+
+int launch_embed(const int32_t* toks, const uint16_t* embed, uint16_t* h, int rows, int hidden, cudaStream_t s) {
+    k_embed<<<rows, 256, 0, s>>>(toks, embed, h, hidden);
+    CASS_LAUNCH_CHECK();
+    return CASS_OK;
+}
+
+int launch_rmsnorm(const uint16_t* h, const uint16_t* gain, uint16_t* out, int rows, int hidden, float eps, cudaStream_t s) {
+    k_residual_rmsnorm<<<rows, 1024, 0, s>>>(const_cast<uint16_t*>(h), nullptr, nullptr, 0, 0, gain, out, hidden, eps);
+    CASS_LAUNCH_CHECK();
+    return CASS_OK;
+}
+
+int launch_residual_rmsnorm(uint16_t* h, const uint16_t* y_bf16, const float* partial, int n_seg, int n_pad,
+                            const uint16_t* gain, uint16_t* out, int rows, int hidden, float eps, cudaStream_t s) {
+    if (partial && rows != 1) return CASS_ERR_INVALID_ARG;
+    k_residual_rmsnorm<<<rows, 1024, 0, s>>>(h, y_bf16, partial, n_seg, n_pad, gain, out, hidden, eps);
+    CASS_LAUNCH_CHECK();
+    return CASS_OK;
+}
+
+int launch_qkv_rope(uint16_t* qkv, const float* partial, int n_seg, int n_pad, const float* cos_t, const float* sin_t,
+                    const DevState* st, int use_inflight, int rows, int n_q, int n_kv, int d, cudaStream_t s) {
+    if (partial && rows != 1) return CASS_ERR_INVALID_ARG;
+    int items = (n_q + n_kv) * (d / 2) + n_kv * d;
+    dim3 grid(ceil_div(items, 256), rows);
+    k_qkv_rope<<<grid, 256, 0, s>>>(qkv, partial, n_seg, n_pad, cos_t, sin_t, st, use_inflight, n_q, n_kv, d);
+    CASS_LAUNCH_CHECK();
+    return CASS_OK;
+}
+
+int launch_swiglu(const uint16_t* gu_bf16, const float* partial, int n_seg, int n_pad, uint16_t* act, int rows, int ffn,
+                  cudaStream_t s) {
+    if (partial && rows != 1) return CASS_ERR_INVALID_ARG;
+    dim3 grid(ceil_div(ffn, 256), rows);
+    k_swiglu<<<grid, 256, 0, s>>>(gu_bf16, partial, n_seg, n_pad, act, ffn);
+    CASS_LAUNCH_CHECK();
+    return CASS_OK;
+}
+
+int launch_argmax(const float* logits, const float* partial, int n_seg, int n_pad, int rows, int vocab, int32_t* out,
+                  float* logits_copy, DevState* st, int bump_inflight, cudaStream_t s) {
+    if (partial && rows != 1) return CASS_ERR_INVALID_ARG;
+    k_argmax<<<rows, 1024, 0, s>>>(logits, partial, n_seg, n_pad, vocab, out, logits_copy, st, bump_inflight);
+    CASS_LAUNCH_CHECK();
+    return CASS_OK;
+}
+
+int launch_accept(DevState* st, const int32_t* draft, const int32_t* target, int g, int32_t* n_acc, int32_t* out_tokens,
+                  int32_t* next_tok, cudaStream_t s) {
+    k_accept<<<1, 32, 0, s>>>(st, draft, target, g, n_acc, out_tokens, next_tok);
+    CASS_LAUNCH_CHECK();
+    return CASS_OK;
+}
+
+int launch_calib_accum(const uint16_t* x, int rows, int cols, float* sumsq, const DevState* st, cudaStream_t s) {
+    k_calib_accum<<<ceil_div(cols, 256), 256, 0, s>>>(x, rows, cols, sumsq, st);
+    CASS_LAUNCH_CHECK();
+    return CASS_OK;
+}
+
+int launch_sqrt(const float* in, float* out, size_t n, cudaStream_t s) {
+    k_sqrt<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(in, out, n);
+    CASS_LAUNCH_CHECK();
+    return CASS_OK;
+}
+
+}  // namespace cass
