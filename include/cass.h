@@ -104,13 +104,24 @@ typedef struct cass_blob_info {
 /* Reads the blob header back to the host.  SYNCHRONISES `stream`. */
 int cass_weight_blob_info(const void* blob, cass_blob_info* h_info, void* stream);
 
+/* Bits of speculation data in a blob, by kind (Sec. 4.2: one bitmap bit per value, sign + kept mantissa bits and
+ * one unary codeword per kept value), and what the physical layout adds around them (chunk tables, masks, padding,
+ * header, codebook, directory).  d_scratch: device memory of at least 8 bytes, 8-byte aligned.  SYNCHRONISES `stream`. */
+typedef struct cass_blob_stats {
+    uint64_t bitmap_bits, field_bits, code_bits;    /* content: rows*cols, rows*kept*(8-t), sum of codeword lengths */
+    uint64_t total_bits;                            /* whole blob */
+} cass_blob_stats;
+int cass_weight_blob_stats(const void* blob, const cass_blob_info* h_info, void* d_scratch, cass_blob_stats* h_stats,
+                           void* stream);
+
 /* Test hook: zero-padded reconstruction (Sec. 4.1, draft inference) of a whole blob into bf16 [rows][cols]. */
 int cass_decode_weights(const void* blob, const cass_blob_info* h_info, void* W_bf16_out, void* stream);
 
 /* ------------------------------------------------------------------------------------------------------
  * Draft GEMV on speculation data (Sec. 4.1 draft inference; decoder dataflow of Sec. 5.1 / Algorithm 1).
  *   y[r] = sum_c decode(blob)[r][c] * x[c], fp32 accumulation, y rounded to bf16 (y_bf16) and/or kept fp32.
- * x: bf16 [cols].  partial: fp32 scratch [n_seg][rows].  Either output pointer may be NULL.
+ * x: bf16 [cols].  partial: fp32 scratch [n_seg][n_rowblocks*32], which receives the per-segment sums.  Either
+ * output pointer may be NULL; with both NULL only `partial` is produced.
  * ---------------------------------------------------------------------------------------------------- */
 int cass_draft_gemv(const void* blob, const cass_blob_info* h_info, const void* x_bf16, float* partial,
                     void* y_bf16, float* y_f32, int32_t* d_status, void* stream);

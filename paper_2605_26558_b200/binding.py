@@ -65,6 +65,11 @@ class BlobInfo(C.Structure):
                 ("kept_per_row", C.c_int), ("max_superblock_bytes", C.c_int), ("total_bytes", C.c_uint64)]
 
 
+class BlobStats(C.Structure):
+    _fields_ = [("bitmap_bits", C.c_uint64), ("field_bits", C.c_uint64), ("code_bits", C.c_uint64),
+                ("total_bits", C.c_uint64)]
+
+
 class KVView(C.Structure):
     _fields_ = [("fixed", C.c_void_p), ("arena", C.c_void_p), ("offsets", C.c_void_p), ("codebook", C.c_void_p),
                 ("k_or_v_bf16", C.c_void_p), ("fixed_words_per_token", C.c_int), ("bitmap_words", C.c_int),
@@ -124,6 +129,13 @@ def cass_weight_blob_info(blob, stream=None) -> BlobInfo:
     info = BlobInfo()
     _check("cass_weight_blob_info", lib.cass_weight_blob_info(_ptr(blob), C.byref(info), _stream(stream)))
     return info
+
+
+def cass_weight_blob_stats(blob, info: BlobInfo, d_scratch, stream=None) -> BlobStats:
+    st = BlobStats()
+    _check("cass_weight_blob_stats", lib.cass_weight_blob_stats(_ptr(blob), C.byref(info), _ptr(d_scratch), C.byref(st),
+                                                                _stream(stream)))
+    return st
 
 
 def cass_decode_weights(blob, info: BlobInfo, out_bf16, stream=None):

@@ -212,6 +212,7 @@ extern "C" int cass_draft_gemv(const void* blob, const cass_blob_info* h_info, c
     cudaStream_t stream = (cudaStream_t)stream_;
     int rc = launch_draft_gemv(blob, *h_info, x_bf16, partial, d_status, stream);
     if (rc) return rc;
+    if (!y_bf16 && !y_f32) return CASS_OK;
     int n_pad = h_info->n_rowblocks * kRowsPerBlock;
     k_gemv_finish<<<ceil_div(h_info->rows, 256), 256, 0, stream>>>(partial, h_info->rows, n_pad, h_info->n_seg,
                                                                     (uint16_t*)y_bf16, y_f32);

@@ -317,9 +317,40 @@ __global__ void k_decode(const uint32_t* __restrict__ blob, uint16_t* __restrict
     }
 }
 
+// ---- content accounting: sum of the codeword lengths recorded in the chunk tables ------------------------
+__global__ void k_code_bits(const uint32_t* __restrict__ blob, unsigned long long* __restrict__ out) {
+    const uint32_t* h = blob;
+    const int k = h[H_COLS], seg_cols = h[H_SEG], n_seg = h[H_NSEG];
+    const int k_pad = ceil_div(k, 32) * 32;
+    const int sb = blockIdx.x, seg = sb % n_seg;
+    const uint32_t* dir = blob + kBlobDirOffset / 4 + sb * 4;
+    const SbGeom sg = SbGeom::make((int)dir[3], seg_cols_of(k_pad, seg_cols, seg), (int)dir[1], (int)dir[2]);
+    const uint32_t* body = blob + (size_t)dir[0] * 4;
+    unsigned int bits = body[sg.tab + sg.n_ch * 32 + threadIdx.x] & 0xFFFFFu;       // segment total of row threadIdx.x
+    bits = __reduce_add_sync(0xffffffffu, bits);
+    if (threadIdx.x == 0) atomicAdd(out, (unsigned long long)bits);
+}
+
 }  // namespace cass
 
 using namespace cass;
+
+extern "C" int cass_weight_blob_stats(const void* blob, const cass_blob_info* bi, void* d_scratch, cass_blob_stats* st,
+                                      void* stream_) {
+    if (!blob || !bi || !d_scratch || !st || ((uintptr_t)d_scratch & 7)) return CASS_ERR_INVALID_ARG;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    CASS_CUDA_CHECK(cudaMemsetAsync(d_scratch, 0, 8, stream));
+    k_code_bits<<<bi->n_rowblocks * bi->n_seg, 32, 0, stream>>>((const uint32_t*)blob, (unsigned long long*)d_scratch);
+    CASS_LAUNCH_CHECK();
+    unsigned long long code = 0;
+    CASS_CUDA_CHECK(cudaMemcpyAsync(&code, d_scratch, 8, cudaMemcpyDeviceToHost, stream));
+    CASS_CUDA_CHECK(cudaStreamSynchronize(stream));
+    st->bitmap_bits = (uint64_t)bi->rows * bi->cols;
+    st->field_bits = (uint64_t)bi->rows * bi->kept_per_row * (8 - bi->trunc_bits);
+    st->code_bits = code;
+    st->total_bits = bi->total_bytes * 8;
+    return CASS_OK;
+}
 
 extern "C" int cass_encoded_weight_bytes(const cass_format* fmt, int rows, int cols, size_t* h_blob_bound,
                                          size_t* h_workspace_bytes) {

@@ -110,7 +110,7 @@ class Engine:
     def encode_weights(self, norms: dict | None):
         """Runs the GPU weight encoder on the four matrices of every layer and on lm_head."""
         status = torch.zeros(1, dtype=torch.int32, device=self.device)
-        blobs = {"layers": [], "infos": []}
+        blobs = {"layers": [], "infos": {}}
         ws = None
 
         def enc(w, a):
@@ -127,10 +127,10 @@ class Engine:
             d = {}
             for nm in ("wqkv", "wo", "wgu", "wd"):
                 a = None if norms is None else norms["layers"][l][nm].to(self.device, torch.float32).contiguous()
-                d[nm], _ = enc(lw[nm], a)
+                d[nm], blobs["infos"][(l, nm)] = enc(lw[nm], a)
             blobs["layers"].append(d)
         a = None if norms is None else norms["lm_head"].to(self.device, torch.float32).contiguous()
-        blobs["lm_head"], _ = enc(self.w["lm_head"], a)
+        blobs["lm_head"], blobs["infos"]["lm_head"] = enc(self.w["lm_head"], a)
         if int(status.item()) != 0:
             raise B.CassError("cass_encode_weights(status)", int(status.item()))
         self.set_blobs(blobs)
