@@ -8,13 +8,18 @@ are read contiguously (Sec. 5.3); the concrete byte layout below is this build's
 
 Common rules
   * every stream is a sequence of 32-bit little-endian words, filled MSB first;
-  * a field of width F = 8 - t never straddles a word: a word holds floor(32/F) fields;
+  * a field of width F = 8 - t never straddles a word: a word holds floor(32/F) fields.  When F divides 32
+    (t = 0, 4, 6, 7) field j is stored "float-aligned and rotated": its sign bit and its 7-t mantissa bits
+    are first put where a binary32 number keeps them (sign at bit 31, mantissa from bit 22 downwards) and
+    that pattern is rotated right by F*j bits; the patterns of the 32/F fields of a word are disjoint and
+    fill it.  A decoder gets sign and mantissa of field j in place with one rotate and one mask.  For the
+    other t the fields are simply packed from the most significant end (field j at bits 31-F*j .. 32-F*(j+1));
   * unary codewords are contiguous and may straddle words;
   * unused bits are zero.
 
 Weight blob  (rows N x cols K, row-major source)
   word  0      magic 'CASW'            word  7  chunk_cols C (multiple of 32)
-  word  1      version (1)             word  8  n_seg
+  word  1      version (2)             word  8  n_seg
   word  2      N                       word  9  n_rowblocks = ceil(N/32)
   word  3      K                       word 10  kept per row = K - floor(K*p/1000)
   word  4      p (per-mille)           word 11  directory byte offset (384)
@@ -24,9 +29,7 @@ Weight blob  (rows N x cols K, row-major source)
   directory: one entry of four words per superblock sb = rowblock*n_seg + seg:
       {byte offset / 16, W_f, W_u, n_chunks}
   word 15      largest superblock size in bytes
-  superblock = 32 rows x one column segment.  First an "irregular" mask: one word per chunk
-  (bit r set = row r of that chunk is irregular, see `chunk_is_irregular`), padded with zero
-  words to a multiple of 32 words.  Then four sections, each word-interleaved over the 32
+  superblock = 32 rows x one column segment: four sections, each word-interleaved over the 32
   rows (word j of row r sits at index j*32 + r):
       chunk table  n_chunks+1 words/row : (index of the chunk's first field WORD << 20) | bit
                                         offset of the chunk's first codeword; the last entry
@@ -48,7 +51,7 @@ import numpy as np
 from . import codec
 
 MAGIC = 0x57534143
-VERSION = 1
+VERSION = 2
 HEADER_BYTES = 128
 CODEBOOK_BYTES = 256
 DIR_OFFSET = HEADER_BYTES + CODEBOOK_BYTES
@@ -75,36 +78,70 @@ def words_to_bits(words: np.ndarray) -> np.ndarray:
     return np.unpackbits(by.reshape(-1))
 
 
-def pack_fields(fields: np.ndarray, t: int) -> np.ndarray:
+def field_rotated(t: int) -> bool:
+    return 32 % (8 - t) == 0
+
+
+def field_bits_in_word(field: int, j: int, t: int) -> int:
+    """The bits field j contributes to its word (see the module docstring)."""
     width = 8 - t
+    field = int(field)
+    if field_rotated(t):
+        sign, mant = field >> (7 - t), field & ((1 << (7 - t)) - 1)
+        canon = (sign << 31) | (mant << (16 + t))             # binary32 sign and top mantissa positions
+        r = (width * j) % 32
+        return ((canon >> r) | (canon << (32 - r))) & 0xFFFFFFFF
+    return field << (32 - width * (j + 1))
+
+
+def field_from_word(word: int, j: int, t: int) -> int:
+    width = 8 - t
+    word = int(word)
+    if field_rotated(t):
+        r = (width * j) % 32
+        canon = ((word << r) | (word >> (32 - r))) & 0xFFFFFFFF
+        return ((canon >> 31) << (7 - t)) | ((canon >> (16 + t)) & ((1 << (7 - t)) - 1))
+    return (word >> (32 - width * (j + 1))) & ((1 << width) - 1)
+
+
+def pack_fields(fields: np.ndarray, t: int) -> np.ndarray:
     per = fields_per_word(t)
     fields = np.asarray(fields, dtype=np.uint32)
     n_words = (fields.size + per - 1) // per
     out = np.zeros(n_words, dtype=np.uint32)
     for j in range(fields.size):
-        out[j // per] |= np.uint32(int(fields[j]) << (32 - width * (j % per + 1)))
+        out[j // per] |= np.uint32(field_bits_in_word(fields[j], j % per, t))
     return out
 
 
 def unpack_fields(words: np.ndarray, n: int, t: int) -> np.ndarray:
-    width = 8 - t
     per = fields_per_word(t)
     out = np.zeros(n, dtype=np.uint32)
     for j in range(n):
-        out[j] = (int(words[j // per]) >> (32 - width * (j % per + 1))) & ((1 << width) - 1)
+        out[j] = field_from_word(words[j // per], j % per, t)
     return out
 
 
 def _pack_fields_fast(fields: np.ndarray, t: int) -> np.ndarray:
+    """Same words as `pack_fields`, vectorised."""
     width = 8 - t
     per = fields_per_word(t)
     fields = np.asarray(fields, dtype=np.uint32)
     n_words = (fields.size + per - 1) // per
-    padded = np.zeros(n_words * per, dtype=np.uint32)
+    if n_words == 0:
+        return np.zeros(0, dtype=np.uint32)
+    padded = np.zeros(n_words * per, dtype=np.uint64)
     padded[: fields.size] = fields
     padded = padded.reshape(n_words, per)
-    shifts = np.array([32 - width * (j + 1) for j in range(per)], dtype=np.uint32)
-    return np.bitwise_or.reduce(padded << shifts[None, :], axis=1).astype(np.uint32) if n_words else padded.reshape(0)
+    j = np.arange(per, dtype=np.uint64)[None, :]
+    if field_rotated(t):
+        sign, mant = padded >> np.uint64(7 - t), padded & np.uint64((1 << (7 - t)) - 1)
+        canon = (sign << np.uint64(31)) | (mant << np.uint64(16 + t))
+        r = (np.uint64(width) * j) % np.uint64(32)
+        bits = ((canon >> r) | (canon << (np.uint64(32) - r))) & np.uint64(0xFFFFFFFF)
+    else:
+        bits = padded << (np.uint64(32) - np.uint64(width) * (j + np.uint64(1)))
+    return np.bitwise_or.reduce(bits, axis=1).astype(np.uint32)
 
 
 @dataclasses.dataclass
@@ -132,31 +169,6 @@ def auto_seg_cols(cols: int, chunk_cols: int, seg_cols: int) -> int:
 
 def _segment_cols(k_pad: int, seg_cols: int, seg: int) -> int:
     return min(seg_cols, k_pad - seg * seg_cols)
-
-
-GROUP_COLS = 8      # kept columns per bitmap-walk group
-GROUP_CODES = 4     # codewords per unary-walk group
-
-
-def chunk_is_irregular(cols_in_chunk: np.ndarray, code_len: np.ndarray) -> bool:
-    """A hint for parallel decoders.  A (row, chunk) is regular when a decoder that looks at the
-    bitmap and at the unary stream through 32-bit windows never needs a second window inside a
-    group: (a) for every aligned group of 8 consecutive kept columns, the distance from the
-    column after the previous group's last kept column (the chunk start for the first group) to
-    the group's last kept column is below 32; (b) every aligned group of 4 consecutive codewords
-    is at most 32 bits long in total.  Groups are counted from the chunk's first kept value."""
-    cols = np.asarray(cols_in_chunk, dtype=np.int64)
-    lens = np.asarray(code_len, dtype=np.int64)
-    start = 0
-    for g in range(0, cols.size, GROUP_COLS):
-        last = int(cols[min(g + GROUP_COLS, cols.size) - 1])
-        if last - start >= 32:
-            return True
-        start = last + 1
-    for g in range(0, lens.size, GROUP_CODES):
-        if int(lens[g: g + GROUP_CODES].sum()) > 32:
-            return True
-    return False
 
 
 def encode_weight_blob(w_bits: np.ndarray, act_norm: np.ndarray | None, p: int, t: int,
@@ -193,7 +205,6 @@ def encode_weight_blob(w_bits: np.ndarray, act_norm: np.ndarray | None, p: int, 
             scols = _segment_cols(k_pad, seg_cols, seg)
             n_ch = (scols + chunk_cols - 1) // chunk_cols
             rows_tab, rows_bm, rows_f, rows_u = [], [], [], []
-            irr = np.zeros((n_ch + 31) // 32 * 32, dtype=np.uint32)
             for rr in range(ROWS_PER_BLOCK):
                 r = rb * ROWS_PER_BLOCK + rr
                 km = np.zeros(scols, dtype=bool)
@@ -226,8 +237,6 @@ def encode_weight_blob(w_bits: np.ndarray, act_norm: np.ndarray | None, p: int, 
                         fw = _pack_fields_fast(fields[first:last], t)
                         fparts.append(fw)
                         fword += fw.size
-                        if chunk_is_irregular(idx[first:last] - ch * chunk_cols, code_len[first:last]):
-                            irr[ch] |= np.uint32(1 << rr)
                 rows_tab.append(tab)
                 rows_bm.append(bits_to_words(km.astype(np.uint8)))
                 rows_f.append(np.concatenate(fparts) if fparts else np.zeros(0, np.uint32))
@@ -242,7 +251,7 @@ def encode_weight_blob(w_bits: np.ndarray, act_norm: np.ndarray | None, p: int, 
                 return sec.reshape(-1)
 
             body = np.concatenate([
-                irr, interleave(rows_tab, n_ch + 1), interleave(rows_bm, scols // 32),
+                interleave(rows_tab, n_ch + 1), interleave(rows_bm, scols // 32),
                 interleave(rows_f, w_f), interleave(rows_u, w_u)])
             bodies[rb * n_seg + seg] = (body, w_f, w_u, n_ch)
 
@@ -303,7 +312,7 @@ def decode_weight_blob(blob: np.ndarray, use_chunk_table: bool = False) -> np.nd
         rb, seg = divmod(sb, info.n_seg)
         off16, w_f, w_u, n_ch = (int(x) for x in info.directory[sb])
         scols = _segment_cols(k_pad, info.seg_cols, seg)
-        base = off16 * 4 + (n_ch + 31) // 32 * 32
+        base = off16 * 4
         tab = blob[base: base + (n_ch + 1) * 32].reshape(n_ch + 1, 32); base += (n_ch + 1) * 32
         bm = blob[base: base + scols // 32 * 32].reshape(scols // 32, 32); base += scols // 32 * 32
         fl = blob[base: base + w_f * 32].reshape(w_f, 32); base += w_f * 32
@@ -344,7 +353,7 @@ def blob_section_bits(blob: np.ndarray) -> dict:
     for sb in range(info.n_rowblocks * info.n_seg):
         _, w_f, w_u, n_ch = (int(x) for x in info.directory[sb])
         scols = _segment_cols(k_pad, info.seg_cols, sb % info.n_seg)
-        tab += ((n_ch + 1) * 32 + (n_ch + 31) // 32 * 32) * 32
+        tab += (n_ch + 1) * 32 * 32
         bm += scols * 32
         fl += w_f * 32 * 32
         un += w_u * 32 * 32

@@ -28,6 +28,34 @@ constexpr int kMaxVerifyRows = 16;
 __host__ __device__ inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 __host__ __device__ inline size_t align_up(size_t a, size_t b) { return (a + b - 1) / b * b; }
 
+// ---- sign + mantissa fields of the speculation data ----------------------------------------------------
+// A field is the sign bit followed by the 7-t kept mantissa bits (F = 8-t bits); a 32-bit word holds 32/F
+// fields and no field straddles words.  When F divides 32 field j is stored float-aligned and rotated: sign at
+// bit 31 and mantissa from bit 22 downwards, that pattern rotated right by F*j (the patterns of one word are
+// disjoint), so that one rotate-left and one mask put both where a binary32 (or, after >> 16, a bf16) value
+// keeps them.  Otherwise fields are packed from the most significant end.
+__host__ __device__ inline bool field_rotated(int t) { return 32 % (8 - t) == 0; }
+
+__device__ __forceinline__ uint32_t field_bits_in_word(uint32_t field, int j, int t) {
+    const int F = 8 - t;
+    if (field_rotated(t)) {
+        uint32_t canon = ((field >> (7 - t)) << 31) | ((field & ((1u << (7 - t)) - 1u)) << (16 + t));
+        return __funnelshift_r(canon, canon, (F * j) & 31);
+    }
+    return field << (32 - F * (j + 1));
+}
+
+// Sign and mantissa of field j of `word`, already at their bf16 positions (bit 15, bits 6..t).
+__device__ __forceinline__ uint32_t field_sign_mant_bf16(uint32_t word, int j, int t) {
+    const int F = 8 - t;
+    if (field_rotated(t)) {
+        uint32_t canon = __funnelshift_l(word, word, (F * j) & 31);
+        return (canon >> 16) & (0x8000u | (0x7Fu & ~((1u << t) - 1u)));
+    }
+    uint32_t f = (word >> (32 - F * (j + 1))) & ((1u << F) - 1u);
+    return ((f >> (F - 1)) << 15) | ((f & ((1u << (F - 1)) - 1u)) << t);
+}
+
 __device__ __forceinline__ float bf16_bits_to_float(uint32_t b) { return __uint_as_float(b << 16); }
 
 __device__ __forceinline__ uint16_t float_to_bf16_bits(float f) {

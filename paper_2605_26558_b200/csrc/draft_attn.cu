@@ -25,7 +25,6 @@ __device__ __forceinline__ void kv_decode_token(const uint32_t* fix, int fs, con
             int s = __clz(bm);
             bm &= ~(0x80000000u >> s);
             uint32_t fword = fix[(bm_words + k / per) * fs];
-            uint32_t f = (fword >> (32 - F * (k % per + 1))) & ((1u << F) - 1u);
             int rank = 0;
             while (ub < limit) {
                 uint32_t v = una[(ub >> 5) * us] << (ub & 31);
@@ -35,7 +34,7 @@ __device__ __forceinline__ void kv_decode_token(const uint32_t* fix, int fs, con
                 ub += avail;
             }
             uint32_t e = r2e[rank & 255];
-            uint32_t bits = ((f >> (F - 1)) << 15) | (e << 7) | ((f & ((1u << (F - 1)) - 1u)) << t);
+            uint32_t bits = field_sign_mant_bf16(fword, k % per, t) | (e << 7);
             emit(w * 32 + s, bits);
             ++k;
         }

@@ -2,32 +2,79 @@
 // the software form of the decoder dataflow of Sec. 5.1: bitmap de-sparsification, unary exponent decode
 // through a rank->exponent table, sign/mantissa concatenation).
 //
-// One CTA per superblock (32 rows x one column segment).  The whole superblock arrives in shared memory with
-// one bulk asynchronous copy (contiguous read, as Sec. 5.3 asks), then warp c decodes chunk c with lane = row:
-// every lane walks its own bitmap, field and unary streams, which are interleaved word by word so that all
-// shared-memory reads of the streams are conflict free.  Regular chunks (see the irregular mask of the format)
-// use 32-bit windows: one bitmap window per 8 kept values, one unary window per 4 codewords.
+// Work unit = one superblock (32 rows x one column segment).  A CTA owns one column segment (its slice of x
+// stays in shared memory as fp32) and walks the row blocks assigned to it; superblocks arrive through a
+// two-stage ring of bulk asynchronous copies (contiguous reads, as Sec. 5.3 asks), so the copy of the next
+// superblocks overlaps the decode of the current one.  Warp c decodes chunk c with lane = row: every lane
+// walks its own bitmap, field and unary streams, which are interleaved word by word over the 32 rows so that
+// all shared-memory reads of the streams are conflict free.
 #include "wblob.cuh"
 #include "kernels.cuh"
 
 namespace cass {
 
+constexpr int kGemvStages = 1;         // stages of the copy ring per CTA; several CTAs share an SM, so their copies and decodes overlap
+constexpr int kXSlack = 288;           // readable floats after the x slice: a window walk may run up to 8 x 32 + 8 columns past its start
+
+static size_t gemv_stage_bytes(const cass_blob_info& bi) { return align_up((size_t)bi.max_superblock_bytes + 256, 128); }
+
 size_t gemv_smem_bytes(const cass_blob_info& bi) {
     const int n_ch = ceil_div(bi.seg_cols, bi.chunk_cols);
-    return align_up((size_t)bi.max_superblock_bytes + 256, 128) + (size_t)(bi.seg_cols + 64) * 4 + 256 * 4 +
-           (size_t)n_ch * 32 * 4 + 64;
+    return kGemvStages * gemv_stage_bytes(bi) + (size_t)(bi.seg_cols + kXSlack) * 4 + 256 * 4 + (size_t)2 * n_ch * 32 * 4 + 64;
 }
 
-// Dot product of one regular (row, chunk) with x, lane = row.  T = truncated mantissa bits (0 or 4).
+__device__ __forceinline__ uint32_t shl_sat(uint32_t v, uint32_t s) {      // shift counts >= 32 give 0
+    uint32_t r;
+    asm("shl.b32 %0, %1, %2;" : "=r"(r) : "r"(v), "r"(s));
+    return r;
+}
+
+struct WalkState {
+    float acc;
+    uint32_t bpos, upos;
+};
+
+// Careful walk of `count` (<= 8) kept values of one row from column bpos / code bit upos on: any gap between
+// kept columns, any codeword length.  Used for the rare groups that do not fit the 32-bit windows.
+template <int T>
+__device__ __noinline__ WalkState group_slow(const uint32_t* bmS, const uint32_t* unS, const uint32_t* flG, int count,
+                                             WalkState st, uint32_t bpos_lim, uint32_t upos_lim, const float* xs,
+                                             const uint32_t* lut) {
+    constexpr int F = 8 - T, PER = 32 / F;
+    constexpr uint32_t MASK = 0x80000000u | (((1u << (7 - T)) - 1u) << (16 + T));
+    for (int e = 0; e < count; ++e) {
+        bool found = false;
+        while (st.bpos < bpos_lim) {
+            uint32_t w = bmS[(st.bpos >> 5) * 32] << (st.bpos & 31);
+            if (w) { st.bpos += __clz(w); found = true; break; }
+            st.bpos = (st.bpos | 31u) + 1u;
+        }
+        if (!found) break;                                   // corrupt stream: stop inside the buffers
+        const float xv = xs[st.bpos];
+        st.bpos += 1;
+        const int rank = read_unary(unS, st.upos, upos_lim);
+        const uint32_t fword = flG[(e / PER) * 32];
+        const uint32_t a = __funnelshift_l(fword, fword, (F * (e % PER)) & 31);
+        st.acc = fmaf(__uint_as_float((a & MASK) | lut[rank & 255]), xv, st.acc);
+    }
+    return st;
+}
+
+// Dot product of one chunk (32 rows, lane = row) with x.  T = truncated mantissa bits (0 or 4).  Every lane walks
+// its row in groups of 8 kept values through 32-bit windows: one bitmap window per group, one unary window per 4
+// codewords.  A group whose 8 kept columns span more than 32 columns, or whose 4 codewords take more than 32 bits,
+// shows up as a window that ran dry (a leading-zero count of 32); that lane then redoes the group with the careful
+// walk while the others wait.
 template <int T>
 __device__ __forceinline__ float chunk_dot_fast(const uint32_t* __restrict__ sb, const SbGeom& g, int ch, int lane,
                                                 int chunk_cols, const float* __restrict__ xs,
                                                 const uint32_t* __restrict__ lut) {
     constexpr int F = 8 - T, PER = 32 / F, NFW = kGroupCols / PER;       // field words per group of 8
-    constexpr uint32_t MANT = ((1u << (F - 1)) - 1u) << (T + 16);
-    static_assert(PER == 4 || PER == 8, "fast path handles 4 or 8 fields per word");
+    constexpr uint32_t MASK = 0x80000000u | (((1u << (7 - T)) - 1u) << (16 + T));   // sign + kept mantissa of a binary32
+    static_assert(32 % F == 0 && (PER == 4 || PER == 8), "fast path: rotated fields, 4 or 8 per word");
     const uint32_t e0 = sb[g.tab + ch * 32 + lane];
-    uint32_t fw = e0 >> 20, upos = e0 & 0xFFFFFu;
+    const uint32_t fw = e0 >> 20;
+    uint32_t upos = e0 & 0xFFFFFu;
     const uint32_t* bmS = sb + g.bm + lane;
     const uint32_t* flS = sb + g.fl + lane;
     const uint32_t* unS = sb + g.un + lane;
@@ -35,48 +82,59 @@ __device__ __forceinline__ float chunk_dot_fast(const uint32_t* __restrict__ sb,
     const int w0 = ch * wpc, w1 = min(w0 + wpc, g.bm_words);
     int m = 0;
     for (int w = w0; w < w1; ++w) m += __popc(bmS[w * 32]);
-    const int n_full = warp_min_i(m) / kGroupCols;
-    const int n_groups = ceil_div(warp_max_i(m), kGroupCols);
+    const int n_full = __reduce_min_sync(0xffffffffu, m) / kGroupCols;
+    const int n_groups = ceil_div(__reduce_max_sync(0xffffffffu, m), kGroupCols);
     uint32_t bpos = (uint32_t)(w0 * 32);
     const uint32_t bpos_lim = (uint32_t)(g.bm_words * 32), upos_lim = (uint32_t)(g.w_u * 32);
     float acc = 0.f;
 
     auto group = [&](int grp, bool tail) {
+        const WalkState st0 = {acc, bpos, upos};
         const uint32_t bw = bpos >> 5;
-        uint32_t bv = __funnelshift_l(bmS[(bw + 1) * 32], bmS[bw * 32], bpos);
+        uint32_t bv = __funnelshift_l(bmS[(bw + 1) * 32], bmS[bw * 32], bpos);     // 32 columns from bpos on
         const float* xg = xs + bpos;
         uint32_t fwd[NFW];
 #pragma unroll
         for (int i = 0; i < NFW; ++i) fwd[i] = flS[(fw + grp * NFW + i) * 32];
         const int rem = m - grp * kGroupCols;
-        int s = 0;
+        uint32_t adv = 0;                           // zero columns skipped so far in this window
+        uint32_t dry = 0;                           // bit 5 set: a window ran dry under a value that counts
 #pragma unroll
         for (int half = 0; half < kGroupCols / kGroupCodes; ++half) {
             const uint32_t uw = upos >> 5;
-            uint32_t uv = __funnelshift_l(unS[(uw + 1) * 32], unS[uw * 32], upos);
-            int tprev = -1;
+            uint32_t uv = __funnelshift_l(unS[(uw + 1) * 32], unS[uw * 32], upos); // 32 code bits from upos on
+            uint32_t usum = 0;
 #pragma unroll
             for (int j = 0; j < kGroupCodes; ++j) {
                 const int e = half * kGroupCodes + j;
-                s = __clz(bv);
-                const float xv = xg[s];
-                bv &= ~(0x80000000u >> s);
-                const int tt = __clz(uv);
-                const uint32_t eb = lut[tt - tprev - 1];
-                tprev = tt;
-                uv &= ~(0x80000000u >> tt);
-                constexpr int dummy = 0; (void)dummy;
-                const int sh = (32 - F * (e % PER + 1)) - (T + 16);
+                const uint32_t s = __clz(bv);                        // zeros before the next kept column
+                adv += s;
+                const float xv = xg[adv + e];
+                bv = shl_sat(shl_sat(bv, s), 1);
+                const uint32_t tt = __clz(uv);                       // rank = zeros before the terminating one
+                const uint32_t eb = lut[tt];
+                uv = shl_sat(shl_sat(uv, tt), 1);
+                usum += tt;
                 const uint32_t fword = fwd[e / PER];
-                const uint32_t a = sh >= 0 ? (fword >> (sh >= 0 ? sh : 0)) : (fword << (sh < 0 ? -sh : 0));
-                const uint32_t wb = (a & MANT) | eb | ((a << 8) & 0x80000000u);
-                if (!tail || e < rem) acc = fmaf(__uint_as_float(wb), xv, acc);
+                const uint32_t a = __funnelshift_l(fword, fword, (F * (e % PER)) & 31);
+                const uint32_t wb = (a & MASK) | eb;
+                if (!tail) {
+                    acc = fmaf(__uint_as_float(wb), xv, acc);
+                } else if (e < rem) {
+                    acc = fmaf(__uint_as_float(wb), xv, acc);
+                    dry |= s | tt;
+                }
             }
-            upos += (uint32_t)(tprev + 1);
-            if (tail) upos = min(upos, upos_lim);
+            if (!tail) dry |= (usum + kGroupCodes > 32u) ? 32u : 0u;
+            upos = min(upos + usum + kGroupCodes, upos_lim);      // rows that ran out of values stay inside the buffers
         }
-        bpos += (uint32_t)(s + 1);
-        if (tail) bpos = min(bpos, bpos_lim);
+        if (!tail) dry |= (adv + kGroupCols > 32u) ? 32u : 0u;
+        bpos = min(bpos + adv + kGroupCols, bpos_lim);
+        if (dry & 32u) {
+            const WalkState r = group_slow<T>(bmS, unS, flS + (fw + grp * NFW) * 32, min(rem, kGroupCols), st0, bpos_lim,
+                                              upos_lim, xs, lut);
+            acc = r.acc; bpos = r.bpos; upos = r.upos;
+        }
     };
 
     int grp = 0;
@@ -86,82 +144,109 @@ __device__ __forceinline__ float chunk_dot_fast(const uint32_t* __restrict__ sb,
 }
 
 // T >= 0: fast path for regular chunks, generic path otherwise.  T = -1: generic path only (any t).
+// grid = (n_seg, G): CTA (seg, j) handles the superblocks (rb, seg) for rb = j, j + G, ...
 template <int T>
 __global__ void __launch_bounds__(1024) k_draft_gemv(const uint32_t* __restrict__ blob, const uint16_t* __restrict__ x,
                                                      float* __restrict__ partial, int32_t* __restrict__ d_status,
-                                                     int max_sb /* shared-memory room for one superblock */, int seg_cols_host) {
+                                                     int stage_bytes, int max_sb, int seg_cols_host) {
     extern __shared__ __align__(128) uint8_t smem_raw[];
     const uint32_t* h = blob;
     const int n = h[H_ROWS], k = h[H_COLS], t = h[H_T], seg_cols = h[H_SEG], chunk_cols = h[H_CHUNK];
     const int n_seg = h[H_NSEG], n_rb = h[H_NRB];
     const int k_pad = ceil_div(k, 32) * 32;
-    const int sb_i = blockIdx.x, rb = sb_i / n_seg, seg = sb_i % n_seg;
+    const int seg = blockIdx.x, rb0 = blockIdx.y, rb_step = gridDim.y;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, n_warps = blockDim.x >> 5;
 
-    uint32_t* sb = reinterpret_cast<uint32_t*>(smem_raw);
-    float* xs = reinterpret_cast<float*>(smem_raw + align_up((size_t)max_sb + 256, 128));
-    uint32_t* lut = reinterpret_cast<uint32_t*>(xs + seg_cols + 64);
-    float* red = reinterpret_cast<float*>(lut + 256);
-    uint64_t* bar = reinterpret_cast<uint64_t*>(red + n_warps * 32);
+    float* xs = reinterpret_cast<float*>(smem_raw + (size_t)kGemvStages * stage_bytes);
+    uint32_t* lut = reinterpret_cast<uint32_t*>(xs + seg_cols + kXSlack);
+    float* red = reinterpret_cast<float*>(lut + 256);                       // [2][n_warps][32]
+    uint64_t* bar = reinterpret_cast<uint64_t*>(red + 2 * n_warps * 32);    // [kGemvStages]
+    __shared__ int s_skip[kGemvStages];
 
-    const uint32_t* dir = blob + kBlobDirOffset / 4 + sb_i * 4;
     const int scols = seg_cols_of(k_pad, seg_cols, seg);
-    const SbGeom g = SbGeom::make((int)dir[3], scols, (int)dir[1], (int)dir[2]);
-    const uint32_t bytes = (uint32_t)g.total * 4u;
-    // The launch sized shared memory from the host's copy of the header; a blob that does not match it
-    // (larger superblock, other segment geometry) is refused instead of overrunning the buffer.
-    if (bytes > (uint32_t)max_sb || (int)blockDim.x < 32 * g.n_ch || seg_cols != seg_cols_host || g.n_ch > 32) {
+    const int n_ch = ceil_div(scols, chunk_cols);
+    // The launch sized shared memory from the host's copy of the header; a blob that does not match it is
+    // refused instead of overrunning the buffers.
+    if (seg >= n_seg || (int)blockDim.x < 32 * n_ch || seg_cols != seg_cols_host || n_ch > 32) {
         if (tid == 0 && d_status) atomicExch(d_status, CASS_ERR_INVALID_ARG);
         return;
     }
+    const int n_tiles = rb0 < n_rb ? (n_rb - rb0 + rb_step - 1) / rb_step : 0;
 
     if (tid == 0) {
-        mbar_init(bar, 1);
+        for (int s = 0; s < kGemvStages; ++s) mbar_init(&bar[s], 1);
         fence_mbar_init();
     }
     __syncthreads();
-    if (tid == 0) {
-        const uint8_t* src = reinterpret_cast<const uint8_t*>(blob) + (size_t)dir[0] * 16;
-        mbar_expect_tx(bar, bytes);
-        for (uint32_t off = 0; off < bytes; off += 32768u) {
-            uint32_t nb = min(32768u, bytes - off);
-            bulk_g2s(smem_raw + off, src + off, nb, bar);
+
+    // thread 0: start the copy of tile i into stage i % kGemvStages
+    auto issue = [&](int i) {
+        const int s = i % kGemvStages;
+        const int sb_i = (rb0 + i * rb_step) * n_seg + seg;
+        const uint32_t* dir = blob + kBlobDirOffset / 4 + sb_i * 4;
+        const SbGeom g = SbGeom::make((int)dir[3], scols, (int)dir[1], (int)dir[2]);
+        const uint32_t bytes = (uint32_t)g.total * 4u;
+        if (bytes > (uint32_t)max_sb || (int)dir[3] != n_ch) {               // does not fit: skip the tile, flag it
+            s_skip[s] = 1;
+            if (d_status) atomicExch(d_status, CASS_ERR_INVALID_ARG);
+            mbar_expect_tx(&bar[s], 0);
+            return;
         }
+        s_skip[s] = 0;
+        const uint8_t* src = reinterpret_cast<const uint8_t*>(blob) + (size_t)dir[0] * 16;
+        uint8_t* dst = smem_raw + (size_t)s * stage_bytes;
+        mbar_expect_tx(&bar[s], bytes);
+        for (uint32_t off = 0; off < bytes; off += 32768u) bulk_g2s(dst + off, src + off, min(32768u, bytes - off), &bar[s]);
+    };
+    if (tid == 0) {
+        for (int i = 0; i < kGemvStages && i < n_tiles; ++i) issue(i);
     }
     // x of this segment (fp32), zero beyond the matrix, and the rank -> exponent table pre-shifted into place
     const int c0 = seg * seg_cols;
-    for (int i = tid; i < seg_cols + 64; i += blockDim.x) {
+    for (int i = tid; i < seg_cols + kXSlack; i += blockDim.x) {
         int c = c0 + i;
         xs[i] = (i < scols && c < k) ? bf16_bits_to_float(x[c]) : 0.f;
     }
     const uint8_t* cb = reinterpret_cast<const uint8_t*>(blob) + kBlobHeaderBytes;
     for (int i = tid; i < 256; i += blockDim.x) lut[i] = (uint32_t)cb[i] << 23;
-    // slack words after the superblock may be read (never used) by the window loads
-    for (int i = tid; i < 64; i += blockDim.x) sb[g.total + i] = 0;
     __syncthreads();
-    if (!mbar_wait_bounded(bar, 0)) {
-        if (d_status) atomicExch(d_status, CASS_ERR_TIMEOUT);
-        return;
-    }
 
-    float acc = 0.f;
-    if (warp < g.n_ch) {
-        const uint32_t irregular = sb[warp];
-        if (T >= 0 && irregular == 0u) {
-            acc = chunk_dot_fast<(T >= 0 ? T : 0)>(sb, g, warp, lane, chunk_cols, xs, lut);
-        } else {
-            decode_chunk_generic(sb, g, chunk_cols, warp, lane, t, cb, [&](int col, uint16_t bits) {
-                acc = fmaf(bf16_bits_to_float(bits), xs[col], acc);
-            });
+    for (int i = 0; i < n_tiles; ++i) {
+        const int s = i % kGemvStages;
+        const int rb = rb0 + i * rb_step;
+        if (!mbar_wait_bounded(&bar[s], (uint32_t)(i / kGemvStages) & 1u)) {
+            // give up: flag the error, let the copies still in flight into this CTA's buffers land (bounded), leave
+            if (d_status) atomicExch(d_status, CASS_ERR_TIMEOUT);
+            for (int j = i; j < n_tiles && j < i + kGemvStages; ++j)
+                mbar_wait_bounded(&bar[j % kGemvStages], (uint32_t)(j / kGemvStages) & 1u);
+            return;
         }
-    }
-    red[warp * 32 + lane] = acc;
-    __syncthreads();
-    if (warp == 0) {
-        float sum = 0.f;
-        for (int w = 0; w < n_warps; ++w) sum += red[w * 32 + lane];
-        int row = rb * kRowsPerBlock + lane;
-        if (row < n) partial[(size_t)seg * (n_rb * kRowsPerBlock) + row] = sum;
+        const uint32_t* sb = reinterpret_cast<const uint32_t*>(smem_raw + (size_t)s * stage_bytes);
+        float acc = 0.f;
+        if (warp < n_ch && !s_skip[s]) {
+            const uint32_t* dir = blob + kBlobDirOffset / 4 + (rb * n_seg + seg) * 4;
+            const SbGeom g = SbGeom::make(n_ch, scols, (int)dir[1], (int)dir[2]);
+            if (T >= 0) {
+                acc = chunk_dot_fast<(T >= 0 ? T : 0)>(sb, g, warp, lane, chunk_cols, xs, lut);
+            } else {
+                decode_chunk_generic(sb, g, chunk_cols, warp, lane, t, cb, [&](int col, uint16_t bits) {
+                    acc = fmaf(bf16_bits_to_float(bits), xs[col], acc);
+                });
+            }
+        }
+        float* red_i = red + (i & 1) * n_warps * 32;
+        red_i[warp * 32 + lane] = acc;
+        __syncthreads();                              // all reads of stage s are done; partial sums are visible
+        if (tid == 0 && i + kGemvStages < n_tiles) {
+            fence_proxy_async();
+            issue(i + kGemvStages);
+        }
+        if (warp == 0) {
+            float sum = 0.f;
+            for (int w = 0; w < n_ch; ++w) sum += red_i[w * 32 + lane];
+            int row = rb * kRowsPerBlock + lane;
+            if (row < n) partial[(size_t)seg * (n_rb * kRowsPerBlock) + row] = sum;
+        }
     }
 }
 
@@ -175,15 +260,34 @@ __global__ void k_gemv_finish(const float* __restrict__ partial, int n, int n_pa
     if (y_bf16) y_bf16[r] = float_to_bf16_bits(acc);
 }
 
+static int sm_count() {
+    static int n = 0;
+    if (n == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+            n = 148;
+    }
+    return n;
+}
+
 int launch_draft_gemv(const void* blob, const cass_blob_info& bi, const void* x_bf16, float* partial,
                       int32_t* d_status, cudaStream_t stream) {
     const int n_ch = ceil_div(bi.seg_cols, bi.chunk_cols);
     if (n_ch > 32) return CASS_ERR_UNSUPPORTED;
-    size_t smem = gemv_smem_bytes(bi);
+    const size_t smem = gemv_smem_bytes(bi);
     if (smem > 227 * 1024) return CASS_ERR_CAPACITY;
-    dim3 grid(bi.n_rowblocks * bi.n_seg), block(32 * n_ch);
+    const int threads = 32 * n_ch;
+    int per_sm = (int)((228 * 1024) / (smem + 1024));
+    if (per_sm > 2048 / threads) per_sm = 2048 / threads;
+    if (per_sm < 1) per_sm = 1;
+    int g = ceil_div(sm_count() * per_sm, bi.n_seg);
+    if (g > bi.n_rowblocks) g = bi.n_rowblocks;
+    if (g < 1) g = 1;
+    g = ceil_div(bi.n_rowblocks, ceil_div(bi.n_rowblocks, g));       // same number of rounds, evenly filled
+    dim3 grid(bi.n_seg, g), block(threads);
     const uint32_t* b = (const uint32_t*)blob;
     const uint16_t* x = (const uint16_t*)x_bf16;
+    const int stage = (int)gemv_stage_bytes(bi);
 #define CASS_GEMV_LAUNCH(TT)                                                                                   \
     do {                                                                                                       \
         static int attr_smem = 0;      /* largest size already granted to this instantiation */              \
@@ -192,7 +296,7 @@ int launch_draft_gemv(const void* blob, const cass_blob_info& bi, const void* x_
                                                  (int)smem));                                                  \
             attr_smem = (int)smem;                                                                             \
         }                                                                                                      \
-        k_draft_gemv<TT><<<grid, block, smem, stream>>>(b, x, partial, d_status, bi.max_superblock_bytes, bi.seg_cols);                              \
+        k_draft_gemv<TT><<<grid, block, smem, stream>>>(b, x, partial, d_status, stage, bi.max_superblock_bytes, bi.seg_cols); \
     } while (0)
     if (bi.trunc_bits == 4) CASS_GEMV_LAUNCH(4);
     else if (bi.trunc_bits == 0) CASS_GEMV_LAUNCH(0);

@@ -201,7 +201,7 @@ __global__ void __launch_bounds__(1024) k_directory(EncGeom g, const uint32_t* _
         unsigned long long total = s_carry;
         uint32_t* h = blob;
         for (int i = 0; i < kBlobHeaderBytes / 4; ++i) h[i] = 0;
-        h[H_MAGIC] = kBlobMagic; h[H_VERSION] = 1; h[H_ROWS] = g.n; h[H_COLS] = g.k; h[H_P] = g.p; h[H_T] = g.t;
+        h[H_MAGIC] = kBlobMagic; h[H_VERSION] = kBlobVersion; h[H_ROWS] = g.n; h[H_COLS] = g.k; h[H_P] = g.p; h[H_T] = g.t;
         h[H_SEG] = g.seg_cols; h[H_CHUNK] = g.chunk_cols; h[H_NSEG] = g.n_seg; h[H_NRB] = g.n_rb;
         h[H_KEPT] = g.k - g.n_prune; h[H_DIROFF] = kBlobDirOffset; h[H_BODYOFF] = (uint32_t)body_off;
         h[H_TOTLO] = (uint32_t)total; h[H_TOTHI] = (uint32_t)(total >> 32); h[H_MAXSB] = s_maxsb;
@@ -258,7 +258,7 @@ __global__ void __launch_bounds__(1024) k_pack(const uint16_t* __restrict__ W, E
         if (kept) {
             uint32_t pre = lane ? __popc(bm >> (32 - lane)) : 0u;
             uint32_t k = k_in_chunk + pre;
-            atomicOr(&body[sg.fl + (fw + k / per) * 32 + r], field << (32 - F * (k % per + 1)));
+            atomicOr(&body[sg.fl + (fw + k / per) * 32 + r], field_bits_in_word(field, k % per, t));
             uint32_t pos = ub + incl - 1;
             atomicOr(&body[sg.un + (pos >> 5) * 32 + r], 0x80000000u >> (pos & 31));
         }
@@ -267,34 +267,6 @@ __global__ void __launch_bounds__(1024) k_pack(const uint16_t* __restrict__ W, E
     }
     fw += (k_in_chunk + per - 1) / per;
     if (lane == 0) body[sg.tab + sg.n_ch * 32 + r] = (fw << 20) | ub;
-    __syncthreads();
-
-    // Irregular-chunk hint: thread (row, chunk) walks its chunk once, sequentially.
-    for (int item = tid; item < sg.n_ch * 32; item += 1024) {
-        int ch = item >> 5, rr = item & 31;
-        int grow = rb * kRowsPerBlock + rr;
-        if (grow >= g.n) continue;
-        bool irregular = false;
-        int start = 0, kcnt = 0, last = 0, code_sum = 0;
-        int wa = ch * wpc, wb = min(wa + wpc, sg.bm_words);
-        for (int j = wa; j < wb; ++j) {
-            uint32_t bm = keepbm[(size_t)grow * words + w0 + j];
-            while (bm) {
-                int s = __clz(bm);
-                bm &= ~(0x80000000u >> s);
-                int col = (j - wa) * 32 + s;
-                int len = exp_to_rank[(W[(size_t)grow * g.k + (w0 + j) * 32 + s] >> 7) & 0xFF] + 1;
-                last = col;
-                code_sum += len;
-                ++kcnt;
-                if (kcnt % kGroupCodes == 0) { irregular |= code_sum > 32; code_sum = 0; }
-                if (kcnt % kGroupCols == 0) { irregular |= (last - start) >= 32; start = last + 1; }
-            }
-        }
-        if (kcnt % kGroupCodes) irregular |= code_sum > 32;
-        if (kcnt % kGroupCols) irregular |= (last - start) >= 32;
-        if (irregular) atomicOr(&body[ch], 1u << rr);
-    }
 }
 
 // ---- test hook: zero-padded reconstruction of the whole blob ---------------------------------------------
@@ -360,11 +332,11 @@ extern "C" int cass_encoded_weight_bytes(const cass_format* fmt, int rows, int c
     const int F = 8 - g.t, per = 32 / F;
     size_t n_sb = (size_t)g.n_rb * g.n_seg;
     int n_ch = ceil_div(g.seg_cols, g.chunk_cols);
-    // per superblock: mask + table + bitmap + fields (kept values + one padding word per chunk) + codes at a
+    // per superblock: table + bitmap + fields (kept values + one padding word per chunk) + codes at a
     // mean of 8 bits per kept value (+1 word of row padding)
     size_t kept_seg = (size_t)g.seg_cols;
     size_t words_row = (size_t)(n_ch + 1) + g.seg_cols / 32 + (kept_seg + per - 1) / per + n_ch + kept_seg * 8 / 32 + 1;
-    size_t sb_bytes = ((size_t)ceil_div(n_ch, 32) * 32 + words_row * 32) * 4;
+    size_t sb_bytes = words_row * 32 * 4;
     if (h_blob_bound) *h_blob_bound = align_up((size_t)kBlobDirOffset + 16 * n_sb, 128) + n_sb * sb_bytes;
     if (h_workspace_bytes) *h_workspace_bytes = carve(nullptr, g.n_pad, g.k_pad, g.n_seg).bytes;
     return CASS_OK;
@@ -410,7 +382,7 @@ extern "C" int cass_weight_blob_info(const void* blob, cass_blob_info* h_info, v
     cudaStream_t stream = (cudaStream_t)stream_;
     CASS_CUDA_CHECK(cudaMemcpyAsync(h, blob, sizeof(h), cudaMemcpyDeviceToHost, stream));
     CASS_CUDA_CHECK(cudaStreamSynchronize(stream));
-    if (h[H_MAGIC] != kBlobMagic || h[H_VERSION] != 1) return CASS_ERR_INVALID_ARG;
+    if (h[H_MAGIC] != kBlobMagic || h[H_VERSION] != kBlobVersion) return CASS_ERR_INVALID_ARG;
     h_info->rows = h[H_ROWS]; h_info->cols = h[H_COLS]; h_info->prune_permille = h[H_P]; h_info->trunc_bits = h[H_T];
     h_info->seg_cols = h[H_SEG]; h_info->chunk_cols = h[H_CHUNK]; h_info->n_seg = h[H_NSEG]; h_info->n_rowblocks = h[H_NRB];
     h_info->kept_per_row = h[H_KEPT]; h_info->max_superblock_bytes = h[H_MAXSB];

@@ -130,7 +130,7 @@ __global__ void __launch_bounds__(256) k_kv_append(KvGeom g, KvComp ck, KvComp c
                         if (keep[j]) {
                             uint32_t k = kbase + (lane ? __popc(bm >> (32 - lane)) : 0u);
                             uint32_t field = ((bits[j] >> 15) << (7 - t_bits)) | ((bits[j] & 0x7Fu) >> t_bits);
-                            atomicOr(&s_fix[warp][nj + k / per], field << (32 - F * (k % per + 1)));
+                            atomicOr(&s_fix[warp][nj + k / per], field_bits_in_word(field, k % per, t_bits));
                             uint32_t p = ubase + incl - 1;
                             if ((p >> 5) < (uint32_t)kKvStageWords) atomicOr(&s_una[warp][p >> 5], 0x80000000u >> (p & 31));
                         }

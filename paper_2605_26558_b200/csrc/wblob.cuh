@@ -2,9 +2,11 @@
 // sequential decoder of one (row, chunk).
 //
 // Blob = header (128 B) | codebook rank->exponent (256 B) | directory (16 B per superblock) | bodies.
-// A superblock holds 32 rows x one column segment: an "irregular" mask (one word per chunk, padded to
-// 32 words), then chunk table, bitmap, fields and unary sections, each interleaved word by word over
-// the 32 rows.  All streams are filled MSB first.  See the format notes in the design document.
+// A superblock holds 32 rows x one column segment: chunk table, bitmap, fields and unary sections, each
+// interleaved word by word over the 32 rows (word j of row r at index j*32 + r).  A chunk-table entry is
+// (index of the chunk's first field word << 20) | bit offset of the chunk's first codeword; the fields of
+// every chunk start on a word boundary; the last entry holds the segment totals.  Bit streams are filled
+// MSB first.
 #pragma once
 
 #include "common.cuh"
@@ -16,6 +18,7 @@ enum BlobHeaderWord {
     H_DIROFF, H_BODYOFF, H_TOTLO, H_TOTHI, H_MAXSB
 };
 constexpr uint32_t kBlobMagic = 0x57534143u;
+constexpr uint32_t kBlobVersion = 2;
 constexpr int kBlobHeaderBytes = 128;
 constexpr int kBlobCodebookBytes = 256;
 constexpr int kBlobDirOffset = kBlobHeaderBytes + kBlobCodebookBytes;
@@ -33,7 +36,7 @@ struct SbGeom {
         g.bm_words = seg_cols_here / 32;
         g.w_f = w_f;
         g.w_u = w_u;
-        g.tab = ceil_div(n_ch, 32) * 32;
+        g.tab = 0;
         g.bm = g.tab + (n_ch + 1) * 32;
         g.fl = g.bm + g.bm_words * 32;
         g.un = g.fl + w_f * 32;
@@ -71,7 +74,7 @@ __device__ __forceinline__ int read_unary(const uint32_t* un_row, uint32_t& ub, 
 template <class Emit>
 __device__ inline void decode_chunk_generic(const uint32_t* sb, const SbGeom& g, int chunk_cols, int ch, int row,
                                             int t, const uint8_t* rank_to_exp, Emit&& emit) {
-    const int F = 8 - t, per = 32 / F;
+    const int per = 32 / (8 - t);
     const uint32_t e0 = sb[g.tab + ch * 32 + row];
     uint32_t fw = e0 >> 20, ub = e0 & 0xFFFFFu;
     const uint32_t* fl_row = sb + g.fl + row;
@@ -86,11 +89,9 @@ __device__ inline void decode_chunk_generic(const uint32_t* sb, const SbGeom& g,
             int s = __clz(bm);
             bm &= ~(0x80000000u >> s);
             uint32_t fword = fl_row[(fw + k / per) * 32];
-            uint32_t f = (fword >> (32 - F * (k % per + 1))) & ((1u << F) - 1u);
             int rank = read_unary(un_row, ub, limit);
             uint32_t e = rank_to_exp[rank & 255];
-            uint32_t sign = f >> (F - 1), mhi = f & ((1u << (F - 1)) - 1u);
-            emit(w * 32 + s, (uint16_t)((sign << 15) | (e << 7) | (mhi << t)));
+            emit(w * 32 + s, (uint16_t)(field_sign_mant_bf16(fword, k % per, t) | (e << 7)));
             ++k;
         }
     }

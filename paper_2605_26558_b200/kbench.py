@@ -1,0 +1,115 @@
+"""Per-kernel microbenchmarks on one Llama-3-8B-shaped decoder layer (hidden 4096, 32 q / 8 kv heads of 128,
+FFN 14336; weights 0.02*Student-t(4) with 1 % outlier input channels; KV ~ N(0,1) with 2 % outlier channels in K).
+
+    python -m paper_2605_26558_b200.kbench [--kernel gemv|verify_gemm|all] [--copies C] [--iters I] [--json]
+
+Each kernel is timed with CUDA events over `--iters` passes across `--copies` distinct copies of its operands (so
+that the working set, copies x operand bytes, exceeds L2), after warm-up passes.  Bytes are the algorithmic bytes
+of the method (speculation-data content for the draft GEMV, bf16 weight bytes for verification).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+
+import torch
+
+from . import binding as B
+
+SHAPES = {                 # rows, cols of the fused matrices of one 8B layer
+    "wqkv": (6144, 4096),
+    "wo": (4096, 4096),
+    "wgu": (28672, 4096),
+    "wd": (4096, 14336),
+}
+
+
+def _peak():
+    p = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+def _time(fn, iters, warm=2):
+    for _ in range(warm):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / iters
+
+
+def encode(w, fmt, act=None):
+    rows, cols = w.shape
+    bound, ws_bytes = B.cass_encoded_weight_bytes(fmt, rows, cols)
+    blob = torch.empty(bound, dtype=torch.uint8, device=w.device)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=w.device)
+    status = torch.zeros(1, dtype=torch.int32, device=w.device)
+    B.cass_encode_weights(fmt, w, act, blob, ws, status)
+    info = B.cass_weight_blob_info(blob)
+    assert int(status.item()) == 0
+    return blob[: info.total_bytes].clone(), info
+
+
+def bench_gemv(name, copies, iters, fmt):
+    import synth
+    rows, cols = SHAPES[name]
+    dev = torch.device("cuda")
+    scratch = torch.zeros(8, dtype=torch.uint8, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    jobs, alg_bits, blob_bits = [], 0, 0
+    x = synth.activation_vector(cols, 1, "kbench/x", device=dev)[0].contiguous()
+    for c in range(copies):
+        w = synth.student_t_weight(rows, cols, c, f"kbench/{name}", device=dev)
+        blob, info = encode(w, fmt)
+        st = B.cass_weight_blob_stats(blob, info, scratch)
+        alg_bits += st.bitmap_bits + st.field_bits + st.code_bits + 16 * cols + 32 * rows * info.n_seg
+        blob_bits += st.total_bits
+        partial = torch.empty(info.n_seg * info.n_rowblocks * 32, dtype=torch.float32, device=dev)
+        jobs.append((blob, info, partial))
+        del w
+
+    def run():
+        for blob, info, partial in jobs:
+            B.cass_draft_gemv(blob, info, x, partial, None, None, status)
+
+    ms = _time(run, iters)
+    assert int(status.item()) == 0
+    peak, kind = _peak()
+    gbs = alg_bits / 8 / (ms * 1e-3) / 1e9
+    return {"kernel": "draft_gemv", "shape": name, "rows": rows, "cols": cols, "copies": copies,
+            "us_per_launch": ms * 1e3 / copies, "algorithmic_GBps": gbs, "frac_of_hbm_peak": gbs / peak,
+            "peak": f"{peak} GB/s ({kind})", "bits_per_element": alg_bits / copies / (rows * cols),
+            "blob_bits_per_element": blob_bits / copies / (rows * cols),
+            "dense_elements_per_s": rows * cols * copies / (ms * 1e-3)}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--kernel", default="gemv")
+    ap.add_argument("--shape", default="all")
+    ap.add_argument("--copies", type=int, default=0, help="distinct operand copies (0: enough to exceed 2x L2)")
+    ap.add_argument("--iters", type=int, default=5)
+    ap.add_argument("--p", type=int, default=400)
+    ap.add_argument("--t", type=int, default=4)
+    args = ap.parse_args()
+    fmt = B.default_format(w_p=args.p, w_t=args.t)
+    out = []
+    if args.kernel in ("gemv", "all"):
+        for name in (SHAPES if args.shape == "all" else [args.shape]):
+            rows, cols = SHAPES[name]
+            copies = args.copies or max(2, int(300e6 / (rows * cols * 0.64)) + 1)
+            out.append(bench_gemv(name, copies, args.iters, fmt))
+    for r in out:
+        print(json.dumps(r))
+
+
+if __name__ == "__main__":
+    main()

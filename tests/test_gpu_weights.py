@@ -88,8 +88,9 @@ def test_encode_decode_gemv(cass, rows, cols, p, t, seg, chunk):
     assert np.array_equal(_bits(y16), codec.f64_to_bf16_bits(y32.cpu().numpy().astype(np.float64)))
 
 
-def test_irregular_chunks_take_the_generic_path(cass):
-    """Rows with long zero runs in the bitmap and very rare exponents (long codewords)."""
+def test_long_gaps_and_long_codewords(cass):
+    """Rows with long zero runs in the bitmap and very rare exponents (long codewords): the window walk of the
+    draft GEMV has to fall back to its careful walk for those groups."""
     rows, cols = 64, 1024
     w = synth.student_t_weight(rows, cols, 3, "gpu/irregular").float()
     w[3, 100:400] = 0.0                       # pruned run longer than a 32-bit window
@@ -104,9 +105,9 @@ def test_irregular_chunks_take_the_generic_path(cass):
     want, oinfo = layout.encode_weight_blob(wb, None, 400, 4)
     got = blob[: info.total_bytes // 4].cpu().numpy().view(np.uint32)
     assert np.array_equal(got, want)
-    binfo = layout.parse_weight_blob(want)
-    irr = want[int(binfo.directory[0][0]) * 4: int(binfo.directory[0][0]) * 4 + 4]
-    assert irr.any(), "the case should exercise the irregular path"
+    inv = codec.invert_codebook(oinfo["codebook"])
+    code_len = inv[(wb >> 7) & 0xFF] + 1
+    assert (code_len[7][oinfo["keep"][7]] > 8).any() and not oinfo["keep"][3, 100:400].any(), "the case should be hard"
     x = synth.activation_vector(cols, 2, "gpu/x2")[0]
     partial = torch.zeros(info.n_seg * info.n_rowblocks * 32, dtype=torch.float32, device="cuda")
     y32 = torch.zeros(rows, dtype=torch.float32, device="cuda")

@@ -229,18 +229,37 @@ def test_blob_size_closed_form(golden_dir):
     assert abs((float(gold["spec_bits"]) + 0.6 * 4 + 0.4 * 16) - float(gold["total_bits"])) < 1e-9
 
 
-def test_field_packing_msb_first():
-    """Fields fill a word from its most significant end and never straddle words."""
-    assert list(layout.pack_fields([0xA, 0x1, 0xF], 4)) == [0xA1F00000]
-    assert list(layout.pack_fields(list(range(1, 10)), 4)) == [0x12345678, 0x90000000]
+def test_field_packing():
+    """Fields never straddle words.  For widths that do not divide 32 they fill a word from its most significant
+    end; for widths that do, field j is the binary32-aligned pattern (sign at bit 31, mantissa from bit 22 down)
+    rotated right by width*j, and the patterns of one word are disjoint and cover it."""
     assert list(layout.pack_fields([0x1F, 0x01, 0x10, 0x0A, 0x15, 0x00, 0x1F], 3)) == [
         (0x1F << 27) | (0x01 << 22) | (0x10 << 17) | (0x0A << 12) | (0x15 << 7) | (0x00 << 2), 0x1F << 27]
+    # t = 4: a nibble s,m2,m1,m0 of field 0 sits at bits 31, 22, 21, 20; field 1 is that pattern moved down by 4
+    assert list(layout.pack_fields([0b1000], 4)) == [0x80000000]
+    assert list(layout.pack_fields([0b0111], 4)) == [0x00700000]
+    assert list(layout.pack_fields([0, 0b1101], 4)) == [(1 << 27) | (0b101 << 16)]
+    assert list(layout.pack_fields([0] * 3 + [0b0100], 4)) == [1 << 10]               # bit 22 - 12
+    assert list(layout.pack_fields([0] * 6 + [0b0110], 4)) == [(1 << 30) | (1 << 29)]   # 22-24, 21-24 wrap around
+    assert list(layout.pack_fields([0xF] * 9, 4)) == [0xFFFFFFFF, 0x80700000]
+    for t in (0, 4, 6, 7):                           # disjoint cover of the word by the per-field patterns
+        per, full = layout.fields_per_word(t), (1 << (8 - t)) - 1
+        seen = 0
+        for j in range(per):
+            bits = layout.field_bits_in_word(full, j, t)
+            assert bits & seen == 0 and bin(bits).count("1") == 8 - t
+            seen |= bits
+        assert seen == 0xFFFFFFFF
+        # one rotate-left by width*j puts sign and mantissa where binary32 keeps them
+        w = int(layout.pack_fields([full] * per, t)[0])
+        assert w == 0xFFFFFFFF
     rng = np.random.default_rng(0)
     for t in range(8):
         f = rng.integers(0, 1 << (8 - t), 50).astype(np.uint32)
         w = layout.pack_fields(f, t)
         assert np.array_equal(w, layout._pack_fields_fast(f, t))
         assert np.array_equal(layout.unpack_fields(w, 50, t), f)
+        assert w.size == -(-50 // layout.fields_per_word(t))
     assert list(layout.bits_to_words([1] + [0] * 31 + [0, 1])) == [0x80000000, 0x40000000]
 
 
