@@ -8,6 +8,8 @@
 // superblocks overlaps the decode of the current one.  Warp c decodes chunk c with lane = row: every lane
 // walks its own bitmap, field and unary streams, which are interleaved word by word over the 32 rows so that
 // all shared-memory reads of the streams are conflict free.
+#include <type_traits>
+
 #include "wblob.cuh"
 #include "kernels.cuh"
 
@@ -60,11 +62,23 @@ __device__ __noinline__ WalkState group_slow(const uint32_t* bmS, const uint32_t
     return st;
 }
 
+__device__ __forceinline__ uint32_t lds_u32(uint32_t addr) {         // shared-space byte address
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v;
+}
+template <int OFF>
+__device__ __forceinline__ uint32_t lds_u32_off(uint32_t addr) {
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1+%2];" : "=r"(v) : "r"(addr), "n"(OFF));
+    return v;
+}
+
 // Dot product of one chunk (32 rows, lane = row) with x.  T = truncated mantissa bits (0 or 4).  Every lane walks
 // its row in groups of 8 kept values through 32-bit windows: one bitmap window per group, one unary window per 4
 // codewords.  A group whose 8 kept columns span more than 32 columns, or whose 4 codewords take more than 32 bits,
 // shows up as a window that ran dry (a leading-zero count of 32); that lane then redoes the group with the careful
-// walk while the others wait.
+// walk while the others wait.  The walk addresses shared memory through 32-bit shared-space addresses.
 template <int T>
 __device__ __forceinline__ float chunk_dot_fast(const uint32_t* __restrict__ sb, const SbGeom& g, int ch, int lane,
                                                 int chunk_cols, const float* __restrict__ xs,
@@ -78,6 +92,8 @@ __device__ __forceinline__ float chunk_dot_fast(const uint32_t* __restrict__ sb,
     const uint32_t* bmS = sb + g.bm + lane;
     const uint32_t* flS = sb + g.fl + lane;
     const uint32_t* unS = sb + g.un + lane;
+    const uint32_t bm_a = smem_u32(bmS), un_a = smem_u32(unS), xs_a = smem_u32(xs), lut_a = smem_u32(lut);
+    uint32_t fl_a = smem_u32(flS + fw * 32);
     const int wpc = chunk_cols / 32;
     const int w0 = ch * wpc, w1 = min(w0 + wpc, g.bm_words);
     int m = 0;
@@ -90,29 +106,30 @@ __device__ __forceinline__ float chunk_dot_fast(const uint32_t* __restrict__ sb,
 
     auto group = [&](int grp, bool tail) {
         const WalkState st0 = {acc, bpos, upos};
-        const uint32_t bw = bpos >> 5;
-        uint32_t bv = __funnelshift_l(bmS[(bw + 1) * 32], bmS[bw * 32], bpos);     // 32 columns from bpos on
-        const float* xg = xs + bpos;
+        const uint32_t ba = bm_a + (bpos >> 5) * 128u;
+        uint32_t bv = __funnelshift_l(lds_u32_off<128>(ba), lds_u32(ba), bpos);    // 32 columns from bpos on
+        const uint32_t xg = xs_a + bpos * 4u;
+        uint32_t xa = xg;                           // address of x[bpos + zero columns skipped so far]
         uint32_t fwd[NFW];
-#pragma unroll
-        for (int i = 0; i < NFW; ++i) fwd[i] = flS[(fw + grp * NFW + i) * 32];
+        fwd[0] = lds_u32(fl_a);
+        if (NFW > 1) fwd[NFW - 1] = lds_u32_off<128>(fl_a);
         const int rem = m - grp * kGroupCols;
-        uint32_t adv = 0;                           // zero columns skipped so far in this window
         uint32_t dry = 0;                           // bit 5 set: a window ran dry under a value that counts
+        uint32_t umax = 0;
 #pragma unroll
         for (int half = 0; half < kGroupCols / kGroupCodes; ++half) {
-            const uint32_t uw = upos >> 5;
-            uint32_t uv = __funnelshift_l(unS[(uw + 1) * 32], unS[uw * 32], upos); // 32 code bits from upos on
+            const uint32_t ua = un_a + (upos >> 5) * 128u;
+            uint32_t uv = __funnelshift_l(lds_u32_off<128>(ua), lds_u32(ua), upos);   // 32 code bits from upos on
             uint32_t usum = 0;
-#pragma unroll
-            for (int j = 0; j < kGroupCodes; ++j) {
-                const int e = half * kGroupCodes + j;
+            auto elem = [&](auto ec) {
+                constexpr int e = decltype(ec)::value;
                 const uint32_t s = __clz(bv);                        // zeros before the next kept column
-                adv += s;
-                const float xv = xg[adv + e];
+                xa += s * 4u;
+                float xv;
+                asm volatile("ld.shared.f32 %0, [%1+%2];" : "=f"(xv) : "r"(xa), "n"(4 * e));
                 bv = shl_sat(shl_sat(bv, s), 1);
                 const uint32_t tt = __clz(uv);                       // rank = zeros before the terminating one
-                const uint32_t eb = lut[tt];
+                const uint32_t eb = lds_u32(lut_a + tt * 4u);
                 uv = shl_sat(shl_sat(uv, tt), 1);
                 usum += tt;
                 const uint32_t fword = fwd[e / PER];
@@ -124,17 +141,29 @@ __device__ __forceinline__ float chunk_dot_fast(const uint32_t* __restrict__ sb,
                     acc = fmaf(__uint_as_float(wb), xv, acc);
                     dry |= s | tt;
                 }
+            };
+            if (half == 0) {
+                elem(std::integral_constant<int, 0>{}); elem(std::integral_constant<int, 1>{});
+                elem(std::integral_constant<int, 2>{}); elem(std::integral_constant<int, 3>{});
+            } else {
+                elem(std::integral_constant<int, 4>{}); elem(std::integral_constant<int, 5>{});
+                elem(std::integral_constant<int, 6>{}); elem(std::integral_constant<int, 7>{});
             }
-            if (!tail) dry |= (usum + kGroupCodes > 32u) ? 32u : 0u;
-            upos = min(upos + usum + kGroupCodes, upos_lim);      // rows that ran out of values stay inside the buffers
+            upos += usum + kGroupCodes;
+            if (tail) upos = min(upos, upos_lim);                 // rows that ran out of values stay inside the buffers
+            else umax = max(umax, usum);
         }
-        if (!tail) dry |= (adv + kGroupCols > 32u) ? 32u : 0u;
-        bpos = min(bpos + adv + kGroupCols, bpos_lim);
+        const uint32_t adv = (xa - xg) >> 2;        // zero columns skipped in this window
+        bpos += adv + kGroupCols;
+        if (tail) bpos = min(bpos, bpos_lim);
+        // full group: the 8 columns fit the window iff adv + 8 <= 32, the 4 codewords of a half iff usum + 4 <= 32
+        else dry = (uint32_t)__vimax3_s32((int)adv + 4, (int)umax, 0) > 28u ? 32u : 0u;
         if (dry & 32u) {
             const WalkState r = group_slow<T>(bmS, unS, flS + (fw + grp * NFW) * 32, min(rem, kGroupCols), st0, bpos_lim,
                                               upos_lim, xs, lut);
             acc = r.acc; bpos = r.bpos; upos = r.upos;
         }
+        fl_a += NFW * 128u;
     };
 
     int grp = 0;
@@ -283,7 +312,6 @@ int launch_draft_gemv(const void* blob, const cass_blob_info& bi, const void* x_
     int g = ceil_div(sm_count() * per_sm, bi.n_seg);
     if (g > bi.n_rowblocks) g = bi.n_rowblocks;
     if (g < 1) g = 1;
-    g = ceil_div(bi.n_rowblocks, ceil_div(bi.n_rowblocks, g));       // same number of rounds, evenly filled
     dim3 grid(bi.n_seg, g), block(threads);
     const uint32_t* b = (const uint32_t*)blob;
     const uint16_t* x = (const uint16_t*)x_bf16;
