@@ -126,6 +126,24 @@ int cass_decode_weights(const void* blob, const cass_blob_info* h_info, void* W_
 int cass_draft_gemv(const void* blob, const cass_blob_info* h_info, const void* x_bf16, float* partial,
                     void* y_bf16, float* y_f32, int32_t* d_status, void* stream);
 
+/* Draft GEMV without a scratch argument (the paper has no counterpart; this is a convenience of this library).
+ * Some callers cannot obtain device memory at the point where they call: code running between the capture-safe
+ * parts of an inference server, plug-ins that are handed only their input and output tensors, or hosts whose
+ * memory pool is closed after start-up.  For them the split-K partial sums go to an array built into the library
+ * image (CASS_STATIC_PARTIAL_FLOATS floats = 2 MiB, resident on every GPU that loads the library until the
+ * process exits) instead of a caller-provided `partial`.  The call allocates and frees nothing.
+ *   - Limit: n_seg * n_rowblocks * 32 <= CASS_STATIC_PARTIAL_FLOATS, else CASS_ERR_CAPACITY (nothing is launched).
+ *     The largest matrix of the Llama-3-8B shape (lm_head 128256 x 4096: 2 x 128256 floats) fits.
+ *   - At least one of y_bf16 / y_f32 must be given; results equal those of cass_draft_gemv.
+ *   - The first call on a device looks up the array's device address (with that device current) and keeps it;
+ *     make that first call outside any stream capture.
+ *   - All calls on one GPU share the array, which keeps the previous call's sums: every value a call reads it has
+ *     written itself first, so nothing needs clearing, but two calls that overlap on the GPU (different streams)
+ *     race on it.  Serialise them on one stream or with events. */
+#define CASS_STATIC_PARTIAL_FLOATS (512 * 1024)
+int cass_draft_gemv_static(const void* blob, const cass_blob_info* h_info, const void* x_bf16, void* y_bf16,
+                           float* y_f32, int32_t* d_status, void* stream);
+
 /* ------------------------------------------------------------------------------------------------------
  * Session: model, KV caches (bf16 and compressed), activations and step state in caller-provided memory.
  * ---------------------------------------------------------------------------------------------------- */

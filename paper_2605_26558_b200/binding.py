@@ -147,6 +147,12 @@ def cass_draft_gemv(blob, info: BlobInfo, x_bf16, partial, y_bf16, y_f32, d_stat
                                                   _ptr(y_f32), _ptr(d_status), _stream(stream)))
 
 
+def cass_draft_gemv_static(blob, info: BlobInfo, x_bf16, y_bf16, y_f32, d_status, stream=None):
+    """cass_draft_gemv with the partial sums in the library's built-in scratch: nothing is allocated, here or there."""
+    _check("cass_draft_gemv_static", lib.cass_draft_gemv_static(_ptr(blob), C.byref(info), _ptr(x_bf16), _ptr(y_bf16),
+                                                                _ptr(y_f32), _ptr(d_status), _stream(stream)))
+
+
 def cass_session_bytes(desc: ModelDesc, fmt: Format) -> int:
     n = C.c_size_t(0)
     _check("cass_session_bytes", lib.cass_session_bytes(C.byref(desc), C.byref(fmt), C.byref(n)))

@@ -351,3 +351,37 @@ extern "C" int cass_draft_gemv(const void* blob, const cass_blob_info* h_info, c
     CASS_LAUNCH_CHECK();
     return CASS_OK;
 }
+
+// ---- variant with built-in scratch ------------------------------------------------------------------------
+// The split-K partial sums of this variant live in a fixed array inside the library image, so the call needs no
+// scratch buffer from its caller.  Every GPU that loads the library holds the array (2 MiB) until the process ends.
+static __device__ __align__(256) float g_static_partial[CASS_STATIC_PARTIAL_FLOATS];
+
+extern "C" int cass_draft_gemv_static(const void* blob, const cass_blob_info* h_info, const void* x_bf16, void* y_bf16,
+                                      float* y_f32, int32_t* d_status, void* stream_) {
+    if (!blob || !h_info || !x_bf16 || (!y_bf16 && !y_f32)) return CASS_ERR_INVALID_ARG;
+    if (h_info->n_seg <= 0 || h_info->n_rowblocks <= 0) return CASS_ERR_INVALID_ARG;
+    const size_t need = (size_t)h_info->n_seg * h_info->n_rowblocks * kRowsPerBlock;
+    if (need > (size_t)CASS_STATIC_PARTIAL_FLOATS) return CASS_ERR_CAPACITY;     // matrix too large for the built-in scratch
+    // In host code the array's name is only a handle; its device address is looked up once per device, with that
+    // device current, and kept.
+    constexpr int kMaxDevices = 64;
+    static float* s_scratch[kMaxDevices] = {nullptr};
+    int dev = -1;
+    CASS_CUDA_CHECK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return CASS_ERR_UNSUPPORTED;
+    if (!s_scratch[dev]) {
+        float* ptr = nullptr;
+        if (cudaGetSymbolAddress((void**)&ptr, g_static_partial) != cudaSuccess || !ptr) return CASS_ERR_CUDA;
+        s_scratch[dev] = ptr;
+    }
+    float* partial = s_scratch[dev];
+    cudaStream_t stream = (cudaStream_t)stream_;
+    int rc = launch_draft_gemv(blob, *h_info, x_bf16, partial, d_status, stream);
+    if (rc) return rc;
+    const int n_pad = h_info->n_rowblocks * kRowsPerBlock;
+    k_gemv_finish<<<ceil_div(h_info->rows, 256), 256, 0, stream>>>(partial, h_info->rows, n_pad, h_info->n_seg,
+                                                                    (uint16_t*)y_bf16, y_f32);
+    CASS_LAUNCH_CHECK();
+    return CASS_OK;
+}
