@@ -170,6 +170,18 @@ def launches_per_step(n_layers: int, gamma: int) -> int:
     return gamma * draft + verify + 1
 
 
+def combine_replicas(ms, ms_e2e, emitted, e2e_emitted, world, device):
+    """Replicas only: the job's time is the slowest rank's, its work the sum over ranks (no data-path collective)."""
+    import torch
+    import torch.distributed as dist
+    if world <= 1:
+        return ms, ms_e2e, float(emitted), float(e2e_emitted)
+    vals = torch.tensor([ms, ms_e2e, float(emitted), float(e2e_emitted)], dtype=torch.float64, device=device)
+    mx = vals.clone(); dist.all_reduce(mx, op=dist.ReduceOp.MAX)
+    sm = vals.clone(); dist.all_reduce(sm, op=dist.ReduceOp.SUM)
+    return float(mx[0]), float(mx[1]), float(sm[2]), float(sm[3])
+
+
 def run_cass(args):
     import torch
     import torch.distributed as dist
@@ -322,14 +334,7 @@ def run_cass(args):
     st_code, _ = eng.status()
 
     # ---- gather over ranks ----
-    vals = torch.tensor([ms, ms_e2e, float(emitted), float(e2e_emitted)], dtype=torch.float64, device=dev)
-    if world > 1:
-        mx = vals.clone(); dist.all_reduce(mx, op=dist.ReduceOp.MAX)
-        sm = vals.clone(); dist.all_reduce(sm, op=dist.ReduceOp.SUM)
-        ms, ms_e2e = float(mx[0]), float(mx[1])
-        emitted_all, e2e_all = float(sm[2]), float(sm[3])
-    else:
-        emitted_all, e2e_all = float(emitted), float(e2e_emitted)
+    ms, ms_e2e, emitted_all, e2e_all = combine_replicas(ms, ms_e2e, emitted, e2e_emitted, world, dev)
 
     if rank == 0:
         cpu = None
