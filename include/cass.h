@@ -200,6 +200,16 @@ int cass_draft_step(void* session, const int32_t* tok_in, int32_t* tok_out, floa
 int cass_verify(void* session, const int32_t* toks, int g, int32_t* target_argmax, float* logits_opt,
                 void* stream);
 
+/* Stand-alone verification projection (Sec. 2.2: the gamma+1 rows are processed as one small batch, bound by
+ * the bf16 weight bytes): Y[r][j] = sum_c W[j][c] X[r][c] for r < rows <= 16, fp32 accumulation on the tensor
+ * cores.  W: bf16 [n][k] row-major, 16-byte aligned, k a multiple of 8.  X: bf16 buffer of 16 rows of k values,
+ * 16-byte aligned (rows beyond `rows` are read but do not influence the result).  scratch: device memory of
+ * cass_verify_gemm_scratch_bytes(n, k).  Outputs [rows][n]; either may be NULL.  A row's result does not depend
+ * on `rows`.  d_status (required) receives CASS_ERR_TIMEOUT if a bounded device wait runs out. */
+size_t cass_verify_gemm_scratch_bytes(int n, int k);
+int cass_verify_gemm(const void* W_bf16, const void* X_bf16, int rows, int n, int k, void* scratch, size_t scratch_bytes,
+                     void* y_bf16, float* y_f32, int32_t* d_status, void* stream);
+
 /* Greedy acceptance (Sec. 2.2; Eq. 1 with p/q in {0,1}): a = min({i-1 : draft[i-1] != target_argmax[i-1]} U {g});
  * out_tokens[0..a] = draft[0..a-1], target_argmax[a]; len += a + 1 (both caches are trimmed by that);
  * the draft-in-flight counter returns to 0; *next_tok = target_argmax[a].  n_accepted, next_tok: device. */

@@ -85,6 +85,7 @@ def _load() -> C.CDLL:
 
 lib = _load()
 lib.cass_version.restype = C.c_char_p
+lib.cass_verify_gemm_scratch_bytes.restype = C.c_size_t
 if hasattr(lib, "cass_calib_norms_count"):
     lib.cass_calib_norms_count.restype = C.c_size_t
 
@@ -216,6 +217,18 @@ def cass_draft_step(session, tok_in, tok_out, logits_opt=None, stream=None):
 
 def cass_verify(session, toks, g: int, target_argmax, logits_opt=None, stream=None):
     _check("cass_verify", lib.cass_verify(session, _ptr(toks), g, _ptr(target_argmax), _ptr(logits_opt), _stream(stream)))
+
+
+def cass_verify_gemm_scratch_bytes(n: int, k: int) -> int:
+    return int(lib.cass_verify_gemm_scratch_bytes(n, k))
+
+
+def cass_verify_gemm(w_bf16, x_bf16, rows: int, scratch, y_bf16, y_f32, d_status, stream=None):
+    n, k = w_bf16.shape
+    assert x_bf16.shape[0] == 16 and x_bf16.shape[1] == k
+    _check("cass_verify_gemm", lib.cass_verify_gemm(_ptr(w_bf16), _ptr(x_bf16), rows, n, k, _ptr(scratch),
+                                                    C.c_size_t(scratch.numel() * scratch.element_size()), _ptr(y_bf16),
+                                                    _ptr(y_f32), _ptr(d_status), _stream(stream)))
 
 
 def cass_accept(session, draft, target_argmax, g: int, n_accepted, out_tokens, next_tok, stream=None):

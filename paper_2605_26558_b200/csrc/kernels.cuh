@@ -82,8 +82,10 @@ int launch_draft_attn(const KvGeom& g, const KvComp& ck, const KvComp& cv, const
 int launch_verify_attn(const KvGeom& g, const uint16_t* k_cache, const uint16_t* v_cache, const uint16_t* qkv,
                        int rows, int n_q, const DevState* st, const AttnScratch& sc, uint16_t* out, cudaStream_t s);
 
-// ---- verification GEMM (verify_gemm.cu): Y[r][n] = sum_k W[n][k] X[r][k], bf16 in, fp32 accumulate -------------
-int launch_verify_gemm(const uint16_t* W, const uint16_t* X, int rows, int n, int k, uint16_t* y_bf16, float* y_f32,
-                       cudaStream_t s);
+// ---- verification GEMM (verify_gemm.cu): Y[r][n] = sum_k W[n][k] X[r][k], bf16 in, fp32 accumulate (tcgen05) ----
+// X is a buffer of 16 rows of k values (the first `rows` are used); partial: fp32 scratch of verify_gemm_partial_floats.
+size_t verify_gemm_partial_floats(int n, int k);
+int launch_verify_gemm(const uint16_t* W, const uint16_t* X, int rows, int n, int k, float* partial, uint16_t* y_bf16,
+                       float* y_f32, int32_t* d_status, cudaStream_t s);
 
 }  // namespace cass

@@ -37,7 +37,7 @@ struct Session {
     int calib_kmax;
     // activations (rows <= 16)
     uint16_t *h, *xn, *qkv, *attn, *y, *gu, *act;
-    float *logits, *partial;
+    float *logits, *partial, *vg_partial;
     size_t partial_floats;
     AttnScratch asc;
     int32_t* argmax_tmp;
@@ -125,6 +125,14 @@ static size_t layout(Session* s, uint8_t* base) {
     (void)segmax; (void)nmax;
     s->partial_floats = pf;
     s->partial = (float*)at(p.take(pf * 4));
+    {   // split-K scratch of the verification GEMMs
+        size_t c[5] = {verify_gemm_partial_floats(s->qkv_dim, d.hidden), verify_gemm_partial_floats(d.hidden, d.n_q_heads * d.head_dim),
+                       verify_gemm_partial_floats(2 * d.ffn, d.hidden), verify_gemm_partial_floats(d.hidden, d.ffn),
+                       verify_gemm_partial_floats(d.vocab, d.hidden)};
+        size_t m = 0;
+        for (size_t v : c) if (v > m) m = v;
+        s->vg_partial = (float*)at(p.take(m * 4));
+    }
     const int n_chunks = ceil_div(d.max_seq, kAttnChunk);
     size_t pairs = (size_t)R * d.n_q_heads;
     s->asc.o = (float*)at(p.take(pairs * n_chunks * d.head_dim * 4));
@@ -360,24 +368,24 @@ extern "C" int cass_verify(void* session, const int32_t* toks, int g, int32_t* t
     for (int l = 0; l < d.n_layers; ++l) {
         LayerDev& L = s->layers[l];
         RC(launch_calib_accum(s->xn, rows, d.hidden, L.calib[0], s->st, st));
-        RC(launch_verify_gemm((const uint16_t*)L.w.wqkv, s->xn, rows, s->qkv_dim, d.hidden, s->qkv, nullptr, st));
+        RC(launch_verify_gemm((const uint16_t*)L.w.wqkv, s->xn, rows, s->qkv_dim, d.hidden, s->vg_partial, s->qkv, nullptr, &s->st->status, st));
         RC(launch_qkv_rope(s->qkv, nullptr, 0, 0, s->cos_t, s->sin_t, s->st, 0, rows, d.n_q_heads, d.n_kv_heads, d.head_dim, st));
         RC(launch_kv_append(s->kg, L.ck, L.cv, L.kc, L.vc, s->qkv + qd, s->qkv + qd + d.n_kv_heads * d.head_dim, s->qkv_dim,
                             -1, 0, rows, kv_flags, s->st, st));
         RC(launch_verify_attn(s->kg, L.kc, L.vc, s->qkv, rows, d.n_q_heads, s->st, s->asc, s->attn, st));
         RC(launch_calib_accum(s->attn, rows, qd, L.calib[1], s->st, st));
-        RC(launch_verify_gemm((const uint16_t*)L.w.wo, s->attn, rows, d.hidden, qd, s->y, nullptr, st));
+        RC(launch_verify_gemm((const uint16_t*)L.w.wo, s->attn, rows, d.hidden, qd, s->vg_partial, s->y, nullptr, &s->st->status, st));
         RC(launch_residual_rmsnorm(s->h, s->y, nullptr, 0, 0, (const uint16_t*)L.w.norm_ffn, s->xn, rows, d.hidden, d.rms_eps, st));
         RC(launch_calib_accum(s->xn, rows, d.hidden, L.calib[2], s->st, st));
-        RC(launch_verify_gemm((const uint16_t*)L.w.wgu, s->xn, rows, 2 * d.ffn, d.hidden, s->gu, nullptr, st));
+        RC(launch_verify_gemm((const uint16_t*)L.w.wgu, s->xn, rows, 2 * d.ffn, d.hidden, s->vg_partial, s->gu, nullptr, &s->st->status, st));
         RC(launch_swiglu(s->gu, nullptr, 0, 0, s->act, rows, d.ffn, st));
         RC(launch_calib_accum(s->act, rows, d.ffn, L.calib[3], s->st, st));
-        RC(launch_verify_gemm((const uint16_t*)L.w.wd, s->act, rows, d.hidden, d.ffn, s->y, nullptr, st));
+        RC(launch_verify_gemm((const uint16_t*)L.w.wd, s->act, rows, d.hidden, d.ffn, s->vg_partial, s->y, nullptr, &s->st->status, st));
         const uint16_t* next_gain = (const uint16_t*)(l + 1 < d.n_layers ? s->layers[l + 1].w.norm_attn : s->norm_final);
         RC(launch_residual_rmsnorm(s->h, s->y, nullptr, 0, 0, next_gain, s->xn, rows, d.hidden, d.rms_eps, st));
     }
     RC(launch_calib_accum(s->xn, rows, d.hidden, s->calib_lm, s->st, st));
-    RC(launch_verify_gemm((const uint16_t*)s->lm_head, s->xn, rows, d.vocab, d.hidden, nullptr, s->logits, st));
+    RC(launch_verify_gemm((const uint16_t*)s->lm_head, s->xn, rows, d.vocab, d.hidden, s->vg_partial, nullptr, s->logits, &s->st->status, st));
     RC(launch_argmax(s->logits, nullptr, 0, 0, rows, d.vocab, target_argmax, logits_opt, s->st, 0, st));
     return CASS_OK;
 }

@@ -1,96 +1,250 @@
 // Verification projections (Sec. 2.2: the target model processes the gamma+1 drafted rows as one small batch,
 // memory-bound on the bf16 weights): Y[r][n] = sum_k W[n][k] X[r][k], bf16 operands, fp32 accumulation.
 //
-// CUDA-core version: every weight element is read once from HBM (streaming 16-byte loads) and multiplied
-// against all rows, which sit in shared memory.  The accumulation order of one output element depends only
-// on (n, k) and never on the number of rows in the call, so a row gives bit-identical results whether it is
-// verified alone or with others.
+// tcgen05 version, "swap-AB": the weights are the M operand (128 output features per CTA), the token rows the N
+// operand (always padded to 16 columns), the accumulator lives in tensor memory.  One CTA = one 128-feature tile x
+// one K range (split-K so that small matrices still fill the GPU); warp 0 streams 128x64 weight tiles and the
+// 16x64 activation tile through a ring of TMA loads (128-byte swizzle), warp 1 issues the MMAs, warps 2-5 read the
+// accumulator back and store fp32 partial sums; a second kernel adds the K ranges in fixed order.
+//
+// Row-count invariance: an accumulator column belongs to one token row, the tile shape, the K ranges and the order
+// of the MMAs depend on (n, k) only, so a row gives the same bits whether it is verified alone or with others.
+#include <cuda.h>
+
 #include "kernels.cuh"
 
 namespace cass {
 
-constexpr int kVgWarps = 8, kVgFeat = 4, kVgKT = 1024;
+constexpr int kTcBM = 128, kTcBN = 16, kTcBK = 64, kTcStages = 6;
+constexpr int kTcABytes = kTcBM * kTcBK * 2, kTcBBytes = kTcBN * kTcBK * 2;
+constexpr int kTcThreads = 192;
+constexpr int kTcSmem = kTcStages * (kTcABytes + kTcBBytes) + 256 + 1024;     // + barriers + alignment slack
+constexpr int kTcTmemCols = 32;
 
-__device__ __forceinline__ uint4 ld_stream(const uint4* p) {
-    uint4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
-    return v;
+// ---- tensor maps ------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+    }
+    return fn;
 }
 
-template <int RT>
-__global__ void __launch_bounds__(256) k_verify_gemm(const uint16_t* __restrict__ W, const uint16_t* __restrict__ X,
-                                                     int rows, int n, int k, uint16_t* __restrict__ y_bf16,
-                                                     float* __restrict__ y_f32) {
-    __shared__ __align__(16) uint16_t xs[RT][kVgKT];
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int n0 = (blockIdx.x * kVgWarps + warp) * kVgFeat;
-    float acc[kVgFeat][RT];
-#pragma unroll
-    for (int f = 0; f < kVgFeat; ++f)
-#pragma unroll
-        for (int r = 0; r < RT; ++r) acc[f][r] = 0.f;
+// bf16 matrix [rows][cols] row-major -> map with a (box_rows x 64)-element box, 128-byte swizzle, zero fill outside.
+static int make_map(CUtensorMap* m, const void* ptr, int rows, int cols, int box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return CASS_ERR_CUDA;
+    cuuint64_t gdim[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t gstride[1] = {(cuuint64_t)cols * 2};
+    cuuint32_t box[2] = {(cuuint32_t)kTcBK, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), gdim, gstride, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? CASS_OK : CASS_ERR_INVALID_ARG;
+}
 
-    for (int kt = 0; kt < k; kt += kVgKT) {
-        __syncthreads();
-        for (int i = tid; i < RT * (kVgKT / 8); i += 256) {
-            int r = i / (kVgKT / 8), c8 = i % (kVgKT / 8);
-            uint4 v = make_uint4(0, 0, 0, 0);
-            if (r < rows && kt + c8 * 8 < k) v = *reinterpret_cast<const uint4*>(X + (size_t)r * k + kt + c8 * 8);
-            *reinterpret_cast<uint4*>(&xs[r][c8 * 8]) = v;
+// ---- PTX wrappers -----------------------------------------------------------------------------------------
+__device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(
+                     smem_u32(smem_dst)),
+                 "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y)
+                 : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_commit(uint64_t* bar) {      // arrives on `bar` when all MMAs issued so far are done
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+// Shared-memory operand descriptor: K-major tile, rows of 64 bf16 (128 bytes), 128-byte swizzle, groups of 8 rows
+// 1024 bytes apart.
+__device__ __forceinline__ uint64_t tc_smem_desc(const void* p) {
+    uint64_t d = (uint64_t)((smem_u32(p) & 0x3FFFFu) >> 4);
+    d |= (uint64_t)(1024 >> 4) << 32;      // stride between 8-row groups
+    d |= 1ull << 46;                       // descriptor version of this architecture
+    d |= 2ull << 61;                       // 128-byte swizzle
+    return d;
+}
+
+// Instruction descriptor of kind::f16: D fp32, A and B bf16, both K-major, M = 128, N = 16.
+constexpr uint32_t kTcIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kTcBN >> 3) << 17) | ((uint32_t)(kTcBM >> 4) << 24);
+
+__device__ __forceinline__ void tc_mma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
+        "l"(adesc), "l"(bdesc), "r"(kTcIdesc), "r"(accumulate)
+        : "memory");
+}
+
+// grid (m tiles, k splits).  partial: fp32 [k splits][16][n].
+__global__ void __launch_bounds__(kTcThreads) k_verify_gemm_tc(const __grid_constant__ CUtensorMap map_w,
+                                                                const __grid_constant__ CUtensorMap map_x,
+                                                                float* __restrict__ partial, int rows, int n,
+                                                                int kb_total, int kb_per_split, int32_t* __restrict__ d_status) {
+    extern __shared__ uint8_t smem_dyn[];
+    uint8_t* base = reinterpret_cast<uint8_t*>(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);     // swizzled tiles: 1024-byte aligned
+    uint8_t* sA = base;
+    uint8_t* sB = base + kTcStages * kTcABytes;
+    uint64_t* full = reinterpret_cast<uint64_t*>(sB + kTcStages * kTcBBytes);
+    uint64_t* empty = full + kTcStages;
+    uint64_t* acc_ready = empty + kTcStages;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_ready + 1);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int m0 = blockIdx.x * kTcBM, ks = blockIdx.y;
+    const int kb0 = ks * kb_per_split;
+    const int nkb = min(kb_per_split, kb_total - kb0);
+
+    if (tid == 0) {
+        for (int s = 0; s < kTcStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+        mbar_init(acc_ready, 1);
+        fence_mbar_init();
+    }
+    if (warp == 1) {                                   // one warp owns the tensor-memory allocation
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTcTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp == 0 && lane == 0) {
+        // ---- producer: TMA loads into the ring ----
+        for (int kb = 0; kb < nkb; ++kb) {
+            const int s = kb % kTcStages;
+            const uint32_t ph = (uint32_t)(kb / kTcStages) & 1u;
+            if (!mbar_wait_bounded(&empty[s], ph ^ 1u)) { atomicExch(d_status, CASS_ERR_TIMEOUT); break; }
+            mbar_expect_tx(&full[s], kTcABytes + kTcBBytes);
+            tma_load_2d(sA + s * kTcABytes, &map_w, (kb0 + kb) * kTcBK, m0, &full[s]);
+            tma_load_2d(sB + s * kTcBBytes, &map_x, (kb0 + kb) * kTcBK, 0, &full[s]);
         }
-        __syncthreads();
+    } else if (warp == 1 && lane == 0) {
+        // ---- MMA issuer ----
+        bool ok = true;
+        for (int kb = 0; kb < nkb && ok; ++kb) {
+            const int s = kb % kTcStages;
+            const uint32_t ph = (uint32_t)(kb / kTcStages) & 1u;
+            if (!mbar_wait_bounded(&full[s], ph)) { atomicExch(d_status, CASS_ERR_TIMEOUT); ok = false; break; }
+            tc_fence_after();
+            const uint64_t ad = tc_smem_desc(sA + s * kTcABytes), bd = tc_smem_desc(sB + s * kTcBBytes);
 #pragma unroll
-        for (int step = 0; step < kVgKT / 256; ++step) {
-            const int kk = (step * 32 + lane) * 8;
-            if (kt + kk >= k) continue;
-            uint4 wv[kVgFeat];
+            for (int kk = 0; kk < kTcBK / 16; ++kk)      // 16 bf16 = 32 bytes along K inside the swizzle row: +2 in the address field
+                tc_mma(tmem, ad + (uint64_t)(kk * 2), bd + (uint64_t)(kk * 2), (uint32_t)((kb | kk) != 0));
+            tc_commit(&empty[s]);                        // frees the stage once these MMAs have read it
+        }
+        tc_commit(acc_ready);                            // accumulator complete (or abandoned after a time-out)
+    } else if (warp >= 2) {
+        // ---- epilogue: warp w may read the 32 accumulator lanes of quarter w % 4 ----
+        if (mbar_wait_bounded(acc_ready, 0)) {
+            __syncwarp();
+            tc_fence_after();
+            const int q = warp & 3;
+            uint32_t v[16];
+            asm volatile(
+                "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+                : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+                  "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+                : "r"(tmem + ((uint32_t)(q * 32) << 16)));
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            const int feat = m0 + q * 32 + lane;
+            if (feat < n && nkb > 0) {
 #pragma unroll
-            for (int f = 0; f < kVgFeat; ++f) {
-                wv[f] = make_uint4(0, 0, 0, 0);
-                if (n0 + f < n) wv[f] = ld_stream(reinterpret_cast<const uint4*>(W + (size_t)(n0 + f) * k + kt + kk));
+                for (int r = 0; r < kTcBN; ++r)
+                    if (r < rows) partial[((size_t)ks * kTcBN + r) * n + feat] = __uint_as_float(v[r]);
             }
-#pragma unroll
-            for (int r = 0; r < RT; ++r) {
-                const uint4 xv = *reinterpret_cast<const uint4*>(&xs[r][kk]);
-                const uint32_t xw[4] = {xv.x, xv.y, xv.z, xv.w};
-#pragma unroll
-                for (int f = 0; f < kVgFeat; ++f) {
-                    const uint32_t ww[4] = {wv[f].x, wv[f].y, wv[f].z, wv[f].w};
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        acc[f][r] = fmaf(__uint_as_float(ww[q] << 16), __uint_as_float(xw[q] << 16), acc[f][r]);
-                        acc[f][r] = fmaf(__uint_as_float(ww[q] & 0xFFFF0000u), __uint_as_float(xw[q] & 0xFFFF0000u), acc[f][r]);
-                    }
-                }
-            }
+        } else {
+            atomicExch(d_status, CASS_ERR_TIMEOUT);
         }
     }
-#pragma unroll
-    for (int f = 0; f < kVgFeat; ++f)
-#pragma unroll
-        for (int r = 0; r < RT; ++r) {
-            float v = warp_sum(acc[f][r]);
-            if (lane == 0 && r < rows && n0 + f < n) {
-                if (y_f32) y_f32[(size_t)r * n + n0 + f] = v;
-                if (y_bf16) y_bf16[(size_t)r * n + n0 + f] = float_to_bf16_bits(v);
-            }
-        }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTcTmemCols) : "memory");
+    }
 }
 
-int launch_verify_gemm(const uint16_t* W, const uint16_t* X, int rows, int n, int k, uint16_t* y_bf16, float* y_f32,
-                       cudaStream_t s) {
-    if (rows < 1 || rows > kMaxVerifyRows || (k % 8)) return CASS_ERR_INVALID_ARG;
-    dim3 grid(ceil_div(n, kVgWarps * kVgFeat));
-#define CASS_VG(RT_) k_verify_gemm<RT_><<<grid, 256, 0, s>>>(W, X, rows, n, k, y_bf16, y_f32)
-    if (rows == 1) CASS_VG(1);
-    else if (rows <= 3) CASS_VG(3);
-    else if (rows <= 5) CASS_VG(5);
-    else if (rows <= 7) CASS_VG(7);
-    else if (rows <= 9) CASS_VG(9);
-    else CASS_VG(16);
-#undef CASS_VG
+__global__ void k_verify_gemm_finish(const float* __restrict__ partial, int rows, int n, int n_split,
+                                     uint16_t* __restrict__ y_bf16, float* __restrict__ y_f32) {
+    const int j = blockIdx.x * blockDim.x + threadIdx.x, r = blockIdx.y;
+    if (j >= n || r >= rows) return;
+    float acc = 0.f;
+    for (int s = 0; s < n_split; ++s) acc += partial[((size_t)s * kTcBN + r) * n + j];
+    if (y_f32) y_f32[(size_t)r * n + j] = acc;
+    if (y_bf16) y_bf16[(size_t)r * n + j] = float_to_bf16_bits(acc);
+}
+
+// K ranges: a function of (n, k) only.  Enough CTAs for about two per SM, at least 4 k-blocks per range.
+static void split_plan(int n, int k, int* kb_total, int* kb_per_split, int* n_split) {
+    const int tiles = ceil_div(n, kTcBM);
+    *kb_total = ceil_div(k, kTcBK);
+    int want = ceil_div(296, tiles);
+    int max_split = *kb_total / 4 > 0 ? *kb_total / 4 : 1;
+    if (want > max_split) want = max_split;
+    if (want < 1) want = 1;
+    *kb_per_split = ceil_div(*kb_total, want);
+    *n_split = ceil_div(*kb_total, *kb_per_split);
+}
+
+size_t verify_gemm_partial_floats(int n, int k) {
+    int kbt, kbs, ns;
+    split_plan(n, k, &kbt, &kbs, &ns);
+    return (size_t)ns * kTcBN * n;
+}
+
+int launch_verify_gemm(const uint16_t* W, const uint16_t* X, int rows, int n, int k, float* partial, uint16_t* y_bf16,
+                       float* y_f32, int32_t* d_status, cudaStream_t s) {
+    if (rows < 1 || rows > kMaxVerifyRows || (k % 8) || n < 1 || !partial || !d_status) return CASS_ERR_INVALID_ARG;
+    if (((uintptr_t)W & 15) || ((uintptr_t)X & 15)) return CASS_ERR_INVALID_ARG;
+    CUtensorMap mw, mx;
+    int rc = make_map(&mw, W, n, k, kTcBM);
+    if (rc) return rc;
+    rc = make_map(&mx, X, kMaxVerifyRows, k, kTcBN);      // the activation buffer always has 16 rows
+    if (rc) return rc;
+    int kbt, kbs, ns;
+    split_plan(n, k, &kbt, &kbs, &ns);
+    static bool attr = false;
+    if (!attr) {
+        CASS_CUDA_CHECK(cudaFuncSetAttribute(k_verify_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmem));
+        attr = true;
+    }
+    dim3 grid(ceil_div(n, kTcBM), ns);
+    k_verify_gemm_tc<<<grid, kTcThreads, kTcSmem, s>>>(mw, mx, partial, rows, n, kbt, kbs, d_status);
+    CASS_LAUNCH_CHECK();
+    dim3 g2(ceil_div(n, 256), rows);
+    k_verify_gemm_finish<<<g2, 256, 0, s>>>(partial, rows, n, ns, y_bf16, y_f32);
     CASS_LAUNCH_CHECK();
     return CASS_OK;
 }
 
 }  // namespace cass
+
+using namespace cass;
+
+extern "C" size_t cass_verify_gemm_scratch_bytes(int n, int k) {
+    if (n < 1 || k < 1) return 0;
+    return verify_gemm_partial_floats(n, k) * sizeof(float);
+}
+
+extern "C" int cass_verify_gemm(const void* W_bf16, const void* X_bf16, int rows, int n, int k, void* scratch,
+                                size_t scratch_bytes, void* y_bf16, float* y_f32, int32_t* d_status, void* stream) {
+    if (!W_bf16 || !X_bf16 || !scratch || (!y_bf16 && !y_f32)) return CASS_ERR_INVALID_ARG;
+    if (n < 1 || k < 1 || scratch_bytes < cass_verify_gemm_scratch_bytes(n, k)) return CASS_ERR_CAPACITY;
+    return launch_verify_gemm((const uint16_t*)W_bf16, (const uint16_t*)X_bf16, rows, n, k, (float*)scratch, (uint16_t*)y_bf16,
+                              y_f32, d_status, (cudaStream_t)stream);
+}

@@ -91,6 +91,30 @@ def bench_gemv(name, copies, iters, fmt):
             "dense_elements_per_s": rows * cols * copies / (ms * 1e-3)}
 
 
+def bench_verify_gemm(name, copies, iters, rows=5):
+    import synth
+    n, k = SHAPES[name]
+    dev = torch.device("cuda")
+    x = synth.activation_vector(k, 1, "kbench/xv", device=dev, rows=16).contiguous()
+    ws = [synth.student_t_weight(n, k, c, f"kbench/v{name}", device=dev) for c in range(copies)]
+    scratch = torch.empty(B.cass_verify_gemm_scratch_bytes(n, k), dtype=torch.uint8, device=dev)
+    y = torch.empty(rows, n, dtype=torch.bfloat16, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+
+    def run():
+        for w in ws:
+            B.cass_verify_gemm(w, x, rows, scratch, y, None, status)
+
+    ms = _time(run, iters)
+    assert int(status.item()) == 0
+    peak, kind = _peak()
+    byt = copies * (n * k * 2 + 16 * k * 2 + rows * n * 2)
+    gbs = byt / (ms * 1e-3) / 1e9
+    return {"kernel": "verify_gemm", "shape": name, "n": n, "k": k, "rows": rows, "copies": copies,
+            "us_per_call": ms * 1e3 / copies, "algorithmic_GBps": gbs, "frac_of_hbm_peak": gbs / peak,
+            "peak": f"{peak} GB/s ({kind})", "tflops": 2.0 * rows * n * k * copies / (ms * 1e-3) / 1e12}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--kernel", default="gemv")
@@ -107,6 +131,11 @@ def main():
             rows, cols = SHAPES[name]
             copies = args.copies or max(2, int(300e6 / (rows * cols * 0.64)) + 1)
             out.append(bench_gemv(name, copies, args.iters, fmt))
+    if args.kernel in ("verify_gemm", "all"):
+        for name in (SHAPES if args.shape == "all" else [args.shape]):
+            n, k = SHAPES[name]
+            copies = args.copies or max(2, int(300e6 / (n * k * 2)) + 1)
+            out.append(bench_verify_gemm(name, copies, args.iters))
     for r in out:
         print(json.dumps(r))
 
