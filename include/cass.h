@@ -200,6 +200,11 @@ int cass_draft_step(void* session, const int32_t* tok_in, int32_t* tok_out, floa
 int cass_verify(void* session, const int32_t* toks, int g, int32_t* target_argmax, float* logits_opt,
                 void* stream);
 
+/* Stand-alone draft attention of one layer (Sec. 4.1 draft inference over the KV speculation data of Sec. 4.2):
+ * q: bf16 [n_q_heads][head_dim] (post-RoPE); the query sees the first len + 1 positions of the layer's compressed
+ * cache (len = committed length, see cass_set_len; no draft in flight); out: bf16 [n_q_heads][head_dim]. */
+int cass_draft_attention(void* session, int layer, const void* q_bf16, void* out_bf16, void* stream);
+
 /* Stand-alone verification projection (Sec. 2.2: the gamma+1 rows are processed as one small batch, bound by
  * the bf16 weight bytes): Y[r][j] = sum_c W[j][c] X[r][c] for r < rows <= 16, fp32 accumulation on the tensor
  * cores.  W: bf16 [n][k] row-major, 16-byte aligned, k a multiple of 8.  X: bf16 buffer of 16 rows of k values,

@@ -219,6 +219,10 @@ def cass_verify(session, toks, g: int, target_argmax, logits_opt=None, stream=No
     _check("cass_verify", lib.cass_verify(session, _ptr(toks), g, _ptr(target_argmax), _ptr(logits_opt), _stream(stream)))
 
 
+def cass_draft_attention(session, layer: int, q_bf16, out_bf16, stream=None):
+    _check("cass_draft_attention", lib.cass_draft_attention(session, layer, _ptr(q_bf16), _ptr(out_bf16), _stream(stream)))
+
+
 def cass_verify_gemm_scratch_bytes(n: int, k: int) -> int:
     return int(lib.cass_verify_gemm_scratch_bytes(n, k))
 

@@ -1,142 +1,293 @@
 // Draft decode attention over the compressed KV cache (Sec. 4.1 draft inference; KV speculation data of
-// Sec. 4.2): grouped-query attention of one query row, split over the sequence in fixed 256-token chunks
-// with a log-sum-exp merge.  Lane = token: every lane walks its own token's record (bitmap, fields, unary
-// codes) and accumulates q.k for all query heads of the group; V records are decoded into a dense bf16 tile in
-// shared memory and multiplied by the chunk's probabilities.
+// Sec. 4.2): grouped-query attention of one query row, split over the sequence in fixed 64-token chunks with a
+// log-sum-exp merge.  One CTA = one (KV head, chunk): warps 0-1 decode the K records of 32 tokens each (lane =
+// token) and form q.k for all query heads of the group, warps 2-3 decode the V records of the same tokens into a
+// dense bf16 tile in shared memory; then the chunk's probabilities multiply the tile.  Records are walked like
+// the weight streams: 8 kept values per 32-bit bitmap window, 4 codewords per 32-bit unary window, with a
+// careful walk for the rare group that does not fit its windows.
+#include <type_traits>
+
 #include "kernels.cuh"
 
 namespace cass {
 
-constexpr int kDaWarps = kAttnChunk / 32;     // 8 warps, 32 tokens each
-constexpr int kDaUnaStage = 24;               // staged unary words per token; longer records are read in place
+constexpr int kDaTok = 64;                    // tokens per CTA
+constexpr int kDaThreads = 128;
+constexpr int kDaUnaStage = 32;               // staged unary words per token; longer records are read in place
 constexpr int kMaxGroup = 8;                  // query heads per KV head
+constexpr int kQStride = kMaxGroup * 4;       // bytes per column of the query tile q_s[col][8]
 
-// Sequential decode of one token's record.  fix: bitmap then field words with stride fs; una: words with stride us.
-template <class Emit>
-__device__ __forceinline__ void kv_decode_token(const uint32_t* fix, int fs, const uint32_t* una, int us, uint32_t n_una,
-                                                int bm_words, int t, const uint8_t* __restrict__ r2e, Emit&& emit) {
-    const int F = 8 - t, per = 32 / F;
-    uint32_t ub = 0;
-    const uint32_t limit = n_una * 32u;
-    int k = 0;
-    for (int w = 0; w < bm_words; ++w) {
-        uint32_t bm = fix[w * fs];
-        while (bm) {
-            int s = __clz(bm);
-            bm &= ~(0x80000000u >> s);
-            uint32_t fword = fix[(bm_words + k / per) * fs];
-            int rank = 0;
-            while (ub < limit) {
-                uint32_t v = una[(ub >> 5) * us] << (ub & 31);
-                int avail = 32 - (int)(ub & 31);
-                if (v) { int z = __clz(v); rank += z; ub += z + 1; break; }
-                rank += avail;
-                ub += avail;
-            }
-            uint32_t e = r2e[rank & 255];
-            uint32_t bits = field_sign_mant_bf16(fword, k % per, t) | (e << 7);
-            emit(w * 32 + s, bits);
-            ++k;
+__device__ __forceinline__ uint32_t da_shl(uint32_t v, uint32_t s) {
+    uint32_t r;
+    asm("shl.b32 %0, %1, %2;" : "=r"(r) : "r"(v), "r"(s));
+    return r;
+}
+__device__ __forceinline__ uint32_t da_lds(uint32_t a) {
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a));
+    return v;
+}
+
+// What happens to a decoded value.  K: multiply with the query tile; V: store into the token's dense row.
+struct EmitK {
+    float acc[kMaxGroup], g[kMaxGroup];
+    uint32_t q_a;
+    int G;
+    __device__ __forceinline__ void reset() {
+#pragma unroll
+        for (int i = 0; i < kMaxGroup; ++i) g[i] = 0.f;
+    }
+    __device__ __forceinline__ void fma_into(float (&dst)[kMaxGroup], uint32_t off, uint32_t wb) {
+        const float w = __uint_as_float(wb);
+        float4 a, b = make_float4(0.f, 0.f, 0.f, 0.f);
+        asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(a.x), "=f"(a.y), "=f"(a.z), "=f"(a.w) : "r"(q_a + off));
+        dst[0] = fmaf(w, a.x, dst[0]); dst[1] = fmaf(w, a.y, dst[1]); dst[2] = fmaf(w, a.z, dst[2]); dst[3] = fmaf(w, a.w, dst[3]);
+        if (G > 4) {
+            asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4+16];" : "=f"(b.x), "=f"(b.y), "=f"(b.z), "=f"(b.w) : "r"(q_a + off));
+            dst[4] = fmaf(w, b.x, dst[4]); dst[5] = fmaf(w, b.y, dst[5]); dst[6] = fmaf(w, b.z, dst[6]); dst[7] = fmaf(w, b.w, dst[7]);
         }
+    }
+    template <int E>
+    __device__ __forceinline__ void elem(uint32_t off, uint32_t wb, bool valid) { if (valid) fma_into(g, off, wb); }
+    __device__ __forceinline__ void commit(int) {
+#pragma unroll
+        for (int i = 0; i < kMaxGroup; ++i) acc[i] += g[i];
+    }
+    __device__ __forceinline__ void direct(uint32_t off, uint32_t wb) { fma_into(acc, off, wb); }
+    __device__ __forceinline__ void restart() {
+#pragma unroll
+        for (int i = 0; i < kMaxGroup; ++i) acc[i] = 0.f;
+    }
+};
+
+struct EmitV {
+    uint32_t row_a;                      // shared address of the token's dense row
+    uint32_t off[kGroupCols], wb[kGroupCols];
+    __device__ __forceinline__ void reset() {}
+    template <int E>
+    __device__ __forceinline__ void elem(uint32_t o, uint32_t w, bool) { off[E] = o; wb[E] = w; }
+    __device__ __forceinline__ void commit(int cnt) {
+#pragma unroll
+        for (int e = 0; e < kGroupCols; ++e)
+            if (e < cnt) asm volatile("st.shared.u16 [%0], %1;" ::"r"(row_a + off[e]), "h"((uint16_t)(wb[e] >> 16)));
+    }
+    __device__ __forceinline__ void direct(uint32_t o, uint32_t w) {
+        asm volatile("st.shared.u16 [%0], %1;" ::"r"(row_a + o), "h"((uint16_t)(w >> 16)));
+    }
+    __device__ __forceinline__ void restart() {}
+};
+
+// Careful walk of `count` kept values from column bpos / code bit upos on.  bm/fl: this token's words, `fs` words
+// apart; un: unary words `us` apart.  STRIDE: bytes per column on the emitter's side.
+template <int T, int STRIDE, class Emit>
+__device__ __forceinline__ void kv_group_slow(const uint32_t* bm, const uint32_t* fl, int fs, const uint32_t* un, int us,
+                                           int count, uint32_t& bpos, uint32_t& upos, uint32_t bpos_lim, uint32_t upos_lim,
+                                           const uint32_t* lut, Emit& em) {
+    constexpr int F = 8 - T, PER = 32 / F;
+    constexpr uint32_t MASK = 0x80000000u | (((1u << (7 - T)) - 1u) << (16 + T));
+    for (int e = 0; e < count; ++e) {
+        bool found = false;
+        while (bpos < bpos_lim) {
+            uint32_t w = bm[(bpos >> 5) * fs] << (bpos & 31);
+            if (w) { bpos += __clz(w); found = true; break; }
+            bpos = (bpos | 31u) + 1u;
+        }
+        if (!found) break;
+        const uint32_t col = bpos;
+        bpos += 1;
+        int rank = 0;
+        while (upos < upos_lim) {
+            uint32_t v = un[(upos >> 5) * us] << (upos & 31);
+            int avail = 32 - (int)(upos & 31);
+            if (v) { int z = __clz(v); rank += z; upos += z + 1; break; }
+            rank += avail;
+            upos += avail;
+        }
+        const uint32_t fword = fl[(e / PER) * fs];
+        const uint32_t a = __funnelshift_l(fword, fword, (F * (e % PER)) & 31);
+        em.direct(col * STRIDE, (a & MASK) | lut[rank & 255]);
     }
 }
 
-struct DaSmem {
-    // carved from dynamic shared memory by the kernel
-};
+// Walk of one record by one lane; `active` lanes emit, the others only keep the warp in step.
+// bm_a / fl_a / un_a: shared addresses of this lane's first bitmap / field / unary word (words 128 bytes apart).
+template <int T, int STRIDE, class Emit>
+__device__ __forceinline__ void kv_record_walk(const uint32_t* bmP, const uint32_t* flP, const uint32_t* unP, uint32_t lut_a,
+                                               const uint32_t* lutP, int kept, int d, uint32_t una_bits, bool active, Emit& em) {
+    constexpr int F = 8 - T, PER = 32 / F, NFW = kGroupCols / PER;
+    constexpr uint32_t MASK = 0x80000000u | (((1u << (7 - T)) - 1u) << (16 + T));
+    const uint32_t bm_a = smem_u32(bmP), un_a = smem_u32(unP);
+    uint32_t fl_a = smem_u32(flP);
+    uint32_t bpos = 0, upos = 0;
+    const uint32_t bpos_lim = (uint32_t)d, upos_lim = (uint32_t)kDaUnaStage * 32u;
+    const int n_groups = ceil_div(kept, kGroupCols);
+    for (int grp = 0; grp < n_groups; ++grp) {
+        const int cnt = min(kGroupCols, kept - grp * kGroupCols);
+        const bool tail = cnt < kGroupCols;
+        const uint32_t bpos0 = bpos, upos0 = upos;
+        const uint32_t ba = bm_a + (bpos >> 5) * 128u;
+        uint32_t bv = __funnelshift_l(da_lds(ba + 128u), da_lds(ba), bpos);
+        const uint32_t x0 = bpos * STRIDE;
+        uint32_t xa = x0;
+        uint32_t fwd[NFW];
+        fwd[0] = da_lds(fl_a);
+        if (NFW > 1) fwd[NFW - 1] = da_lds(fl_a + 128u);
+        uint32_t dry = 0, umax = 0;
+        em.reset();
+#pragma unroll
+        for (int half = 0; half < kGroupCols / kGroupCodes; ++half) {
+            const uint32_t ua = un_a + (upos >> 5) * 128u;
+            uint32_t uv = __funnelshift_l(da_lds(ua + 128u), da_lds(ua), upos);
+            uint32_t usum = 0;
+            auto elem = [&](auto ec) {
+                constexpr int e = decltype(ec)::value;
+                const uint32_t s = __clz(bv);
+                xa += s * STRIDE;
+                bv = da_shl(da_shl(bv, s), 1);
+                const uint32_t tt = __clz(uv);
+                const uint32_t eb = da_lds(lut_a + tt * 4u);
+                uv = da_shl(da_shl(uv, tt), 1);
+                usum += tt;
+                const uint32_t fword = fwd[e / PER];
+                const uint32_t a = __funnelshift_l(fword, fword, (F * (e % PER)) & 31);
+                const bool valid = active && (!tail || e < cnt);
+                em.template elem<e>(xa + e * STRIDE, (a & MASK) | eb, valid);
+                if (tail && e < cnt) dry |= s | tt;
+            };
+            if (half == 0) {
+                elem(std::integral_constant<int, 0>{}); elem(std::integral_constant<int, 1>{});
+                elem(std::integral_constant<int, 2>{}); elem(std::integral_constant<int, 3>{});
+            } else {
+                elem(std::integral_constant<int, 4>{}); elem(std::integral_constant<int, 5>{});
+                elem(std::integral_constant<int, 6>{}); elem(std::integral_constant<int, 7>{});
+            }
+            upos = min(upos + usum + kGroupCodes, upos_lim);
+            umax = max(umax, usum);
+        }
+        const uint32_t adv = (xa - x0) / STRIDE;
+        bpos = min(bpos + adv + kGroupCols, bpos_lim);
+        if (!tail) dry = (adv + kGroupCols > 32u || umax + kGroupCodes > 32u) ? 32u : 0u;
+        if (active) {
+            if (dry & 32u) {                           // a window ran dry: redo this group one value at a time
+                bpos = bpos0; upos = upos0;
+                kv_group_slow<T, STRIDE>(bmP, flP + grp * NFW * 32, 32, unP, 32, cnt, bpos, upos, bpos_lim, min(una_bits, upos_lim),
+                                         lutP, em);
+            } else {
+                em.commit(cnt);
+            }
+        }
+        fl_a += NFW * 128u;
+    }
+}
 
-__global__ void __launch_bounds__(256) k_draft_attn(KvGeom g, KvComp ck, KvComp cv, const uint16_t* __restrict__ qkv,
-                                                    int n_q, const DevState* __restrict__ st, AttnScratch sc,
-                                                    int n_chunks_alloc) {
+template <int T>
+__global__ void __launch_bounds__(kDaThreads) k_draft_attn(KvGeom g, KvComp ck, KvComp cv, const uint16_t* __restrict__ qkv,
+                                                           int n_q, const DevState* __restrict__ st, AttnScratch sc,
+                                                           int n_chunks_alloc) {
     extern __shared__ __align__(16) uint8_t smem[];
     const int chunk = blockIdx.x, head = blockIdx.y;
     const int cur_len = st->len + st->inflight + 1;            // positions visible to the drafted token
-    const int t0 = chunk * kAttnChunk;
+    const int t0 = chunk * kDaTok;
     if (t0 >= cur_len) return;
     const int G = n_q / g.n_kv, d = g.d;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
-    float* q_s = reinterpret_cast<float*>(smem);                              // [G][d]
-    float* sc_s = q_s + kMaxGroup * d;                                        // [G][256] scores -> probabilities
-    float* ml_s = sc_s + kMaxGroup * kAttnChunk;                              // [G][2]
-    uint32_t* fix_s = reinterpret_cast<uint32_t*>(ml_s + 2 * kMaxGroup);      // [8 warps][wpt][32]
-    uint32_t* una_s = fix_s + kDaWarps * g.wpt * 32;                          // [8 warps][kDaUnaStage][32]
-    uint16_t* v_s = reinterpret_cast<uint16_t*>(una_s + kDaWarps * kDaUnaStage * 32);   // [256][d] bf16
-    uint8_t* r2e_s = reinterpret_cast<uint8_t*>(v_s + kAttnChunk * d);        // [2][256]
+    float* q_s = reinterpret_cast<float*>(smem);                              // [d][8]
+    float* sc_s = q_s + d * kMaxGroup;                                        // [8][64] scores -> probabilities
+    float* ml_s = sc_s + kMaxGroup * kDaTok;                                  // [8][2]
+    uint32_t* lut_s = reinterpret_cast<uint32_t*>(ml_s + 2 * kMaxGroup);      // [2][256] rank -> exponent << 23
+    uint32_t* fix_s = lut_s + 512;                                            // [4 warps][wpt + 1][32]
+    uint32_t* una_s = fix_s + 4 * (g.wpt + 1) * 32;                           // [4 warps][kDaUnaStage + 2][32]
+    uint16_t* v_s = reinterpret_cast<uint16_t*>(una_s + 4 * (kDaUnaStage + 2) * 32);   // [64][d] bf16
 
     const float scale = rsqrtf((float)d);
-    for (int i = tid; i < G * d; i += 256) q_s[i] = bf16_bits_to_float(qkv[(size_t)head * G * d + i]);
-    for (int i = tid; i < 256; i += 256) { r2e_s[i] = ck.rank_to_exp[i]; r2e_s[256 + i] = cv.rank_to_exp[i]; }
-    for (int i = tid; i < kAttnChunk * d / 2; i += 256) reinterpret_cast<uint32_t*>(v_s)[i] = 0u;
+    for (int i = tid; i < d * kMaxGroup; i += kDaThreads) {
+        int col = i / kMaxGroup, gi = i % kMaxGroup;
+        q_s[i] = gi < G ? bf16_bits_to_float(qkv[(size_t)(head * G + gi) * d + col]) : 0.f;
+    }
+    for (int i = tid; i < 512; i += kDaThreads) lut_s[i] = (uint32_t)(i < 256 ? ck.rank_to_exp[i] : cv.rank_to_exp[i - 256]) << 23;
+    for (int i = tid; i < kDaTok * d / 2; i += kDaThreads) reinterpret_cast<uint32_t*>(v_s)[i] = 0u;
+
+    // stage this warp's 32 records: warps 0,1 -> K of tokens t0 + 32 w .., warps 2,3 -> V of the same tokens
+    const int kind = warp >> 1, tw = warp & 1;
+    const int tok = t0 + tw * 32 + lane;
+    const bool valid = tok < cur_len;
+    const KvComp& c = kind ? cv : ck;
+    uint32_t* my_fix = fix_s + warp * (g.wpt + 1) * 32;
+    uint32_t* my_una = una_s + warp * (kDaUnaStage + 2) * 32;
+    {
+        const uint32_t* fixed = c.fixed + ((size_t)head * g.n_blocks + tok / 32) * g.wpt * 32;
+        for (int w = 0; w < g.wpt; ++w) my_fix[w * 32 + lane] = fixed[w * 32 + lane];          // coalesced block copy
+        my_fix[g.wpt * 32 + lane] = 0u;
+    }
+    const uint32_t* off = c.off + (size_t)head * (g.max_seq + 1);
+    const uint32_t* arena = c.arena + (size_t)head * g.arena_words;
+    uint32_t o0 = 0, n_una = 0;
+    if (valid) { o0 = off[tok]; n_una = off[tok + 1] - o0; }
+    const bool staged = n_una <= (uint32_t)kDaUnaStage;
+    for (int w = 0; w < kDaUnaStage + 2; ++w) my_una[w * 32 + lane] = (staged && (uint32_t)w < n_una) ? arena[o0 + w] : 0u;
     __syncthreads();
 
-    const int tok = t0 + warp * 32 + lane;
-    const bool valid = tok < cur_len;
-    const int blk = tok / 32;                                               // same for the whole warp
-    uint32_t* my_fix = fix_s + warp * g.wpt * 32 + lane;
-    uint32_t* my_una = una_s + warp * kDaUnaStage * 32 + lane;
-
-    for (int kind = 0; kind < 2; ++kind) {
-        const KvComp& c = kind ? cv : ck;
-        const uint32_t* fixed = c.fixed + ((size_t)head * g.n_blocks + blk) * g.wpt * 32;
-        const uint32_t* off = c.off + (size_t)head * (g.max_seq + 1);
-        const uint32_t* arena = c.arena + (size_t)head * g.arena_words;
-        __syncwarp();
-        for (int w = 0; w < g.wpt; ++w) my_fix[w * 32] = fixed[w * 32 + lane];         // coalesced block copy
-        uint32_t o0 = 0, n_una = 0;
-        if (valid) { o0 = off[tok]; n_una = off[tok + 1] - o0; }
-        const bool staged = n_una <= (uint32_t)kDaUnaStage;
-        if (staged) for (uint32_t w = 0; w < n_una; ++w) my_una[w * 32] = arena[o0 + w];
-        __syncwarp();
-        const uint32_t* una = staged ? my_una : arena + o0;
-        const int us = staged ? 32 : 1;
-        if (kind == 0) {
-            float acc[kMaxGroup];
+    const uint32_t* lutP = lut_s + kind * 256;
+    if (kind == 0) {
+        EmitK em;
+        em.q_a = smem_u32(q_s);
+        em.G = G;
+        em.restart();
+        kv_record_walk<T, kQStride>(my_fix + lane, my_fix + g.bm_words * 32 + lane, my_una + lane, smem_u32(lutP), lutP, g.kept, d,
+                                    n_una * 32u, valid && staged, em);
+        if (valid && !staged) {                                               // very long record: walk it in place
+            uint32_t bpos = 0, upos = 0;
+            em.restart();
+            for (int grp = 0; grp * kGroupCols < g.kept; ++grp)
+                kv_group_slow<T, kQStride>(my_fix + lane, my_fix + (g.bm_words + grp * (kGroupCols * (8 - T) / 32)) * 32 + lane, 32,
+                                           arena + o0, 1, min(kGroupCols, g.kept - grp * kGroupCols), bpos, upos, (uint32_t)d,
+                                           n_una * 32u, lutP, em);
+        }
 #pragma unroll
-            for (int gi = 0; gi < kMaxGroup; ++gi) acc[gi] = 0.f;
-            if (valid) {
-                kv_decode_token(my_fix, 32, una, us, n_una, g.bm_words, g.t, r2e_s, [&](int col, uint32_t bits) {
-                    float kvv = bf16_bits_to_float(bits);
-#pragma unroll
-                    for (int gi = 0; gi < kMaxGroup; ++gi)
-                        if (gi < G) acc[gi] = fmaf(kvv, q_s[gi * d + col], acc[gi]);
-                });
-            }
-#pragma unroll
-            for (int gi = 0; gi < kMaxGroup; ++gi)
-                if (gi < G) sc_s[gi * kAttnChunk + warp * 32 + lane] = valid ? acc[gi] * scale : -INFINITY;
-        } else {
-            if (valid) {
-                uint16_t* vrow = v_s + (size_t)(warp * 32 + lane) * d;
-                kv_decode_token(my_fix, 32, una, us, n_una, g.bm_words, g.t, r2e_s + 256,
-                                [&](int col, uint32_t bits) { vrow[col] = (uint16_t)bits; });
-            }
+        for (int gi = 0; gi < kMaxGroup; ++gi)
+            if (gi < G) sc_s[gi * kDaTok + tw * 32 + lane] = valid ? em.acc[gi] * scale : -INFINITY;
+    } else {
+        EmitV em;
+        em.row_a = smem_u32(v_s + (size_t)(tw * 32 + lane) * d);
+        kv_record_walk<T, 2>(my_fix + lane, my_fix + g.bm_words * 32 + lane, my_una + lane, smem_u32(lutP), lutP, g.kept, d,
+                             n_una * 32u, valid && staged, em);
+        if (valid && !staged) {
+            uint32_t bpos = 0, upos = 0;
+            for (int grp = 0; grp * kGroupCols < g.kept; ++grp)
+                kv_group_slow<T, 2>(my_fix + lane, my_fix + (g.bm_words + grp * (kGroupCols * (8 - T) / 32)) * 32 + lane, 32,
+                                    arena + o0, 1, min(kGroupCols, g.kept - grp * kGroupCols), bpos, upos, (uint32_t)d,
+                                    n_una * 32u, lutP, em);
         }
     }
     __syncthreads();
-    // chunk softmax statistics: warp gi handles query head gi of the group
-    if (warp < G) {
-        float m = -INFINITY;
-        for (int i = lane; i < kAttnChunk; i += 32) m = fmaxf(m, sc_s[warp * kAttnChunk + i]);
-        m = warp_max(m);
-        float l = 0.f;
-        for (int i = lane; i < kAttnChunk; i += 32) {
-            float p = expf(sc_s[warp * kAttnChunk + i] - m);          // exp(-inf) = 0 for tokens beyond the end
-            sc_s[warp * kAttnChunk + i] = p;
-            l += p;
-        }
-        l = warp_sum(l);
-        if (lane == 0) { ml_s[warp * 2] = m; ml_s[warp * 2 + 1] = l; }
+    // chunk softmax statistics: warp w handles query heads w, w + 4
+    for (int gi = warp; gi < G; gi += kDaThreads / 32) {
+        float a = sc_s[gi * kDaTok + lane], b = sc_s[gi * kDaTok + 32 + lane];
+        const float m = warp_max(fmaxf(a, b));
+        a = expf(a - m);                                              // exp(-inf) = 0 for tokens beyond the end
+        b = expf(b - m);
+        sc_s[gi * kDaTok + lane] = a;
+        sc_s[gi * kDaTok + 32 + lane] = b;
+        const float l = warp_sum(a + b);
+        if (lane == 0) { ml_s[gi * 2] = m; ml_s[gi * 2 + 1] = l; }
     }
     __syncthreads();
     // o[gi][dim] = sum_t p[gi][t] * v[t][dim]
-    const int n_tok = min(kAttnChunk, cur_len - t0);
-    for (int item = tid; item < G * d; item += 256) {
-        int gi = item / d, dim = item % d;
-        float acc = 0.f;
-        for (int t = 0; t < n_tok; ++t) acc = fmaf(sc_s[gi * kAttnChunk + t], bf16_bits_to_float(v_s[(size_t)t * d + dim]), acc);
-        int hq = head * G + gi;
-        sc.o[((size_t)hq * n_chunks_alloc + chunk) * d + dim] = acc;
+    const int n_tok = min(kDaTok, cur_len - t0);
+    for (int dim = tid; dim < d; dim += kDaThreads) {
+        float acc[kMaxGroup];
+#pragma unroll
+        for (int gi = 0; gi < kMaxGroup; ++gi) acc[gi] = 0.f;
+        for (int t = 0; t < n_tok; ++t) {
+            const float v = bf16_bits_to_float(v_s[(size_t)t * d + dim]);
+#pragma unroll
+            for (int gi = 0; gi < kMaxGroup; ++gi)
+                if (gi < G) acc[gi] = fmaf(sc_s[gi * kDaTok + t], v, acc[gi]);
+        }
+#pragma unroll
+        for (int gi = 0; gi < kMaxGroup; ++gi)
+            if (gi < G) sc.o[((size_t)(head * G + gi) * n_chunks_alloc + chunk) * d + dim] = acc[gi];
     }
     if (tid < G) {
         int hq = head * G + tid;
@@ -146,12 +297,13 @@ __global__ void __launch_bounds__(256) k_draft_attn(KvGeom g, KvComp ck, KvComp 
 }
 
 // Merge the chunk partials of every (row, query head): out = sum_c e^{m_c - M} o_c / sum_c e^{m_c - M} l_c.
-// Row r sees positions < len + (draft: inflight + 1 | verify: r + 1).
-__global__ void k_attn_merge(AttnScratch sc, int n_chunks_alloc, int n_q, int d, const DevState* __restrict__ st,
-                             int draft_mode, uint16_t* __restrict__ out) {
+// Row r sees positions < len + (draft: inflight + 1 | verify: r + 1); chunks hold `chunk_tokens` positions.
+__global__ void k_attn_merge(AttnScratch sc, int n_chunks_alloc, int chunk_tokens, int n_q, int d,
+                             const DevState* __restrict__ st, int draft_mode, uint16_t* __restrict__ out) {
+    pdl_launch_dependents();
     const int hq = blockIdx.x, r = blockIdx.y;
     const int vis = st->len + (draft_mode ? st->inflight + 1 : r + 1);
-    const int n_ch = ceil_div(vis, kAttnChunk);
+    const int n_ch = ceil_div(vis, chunk_tokens);
     const size_t pair = (size_t)r * n_q + hq;
     float M = -INFINITY;
     for (int c = 0; c < n_ch; ++c) M = fmaxf(M, sc.m[pair * n_chunks_alloc + c]);
@@ -165,31 +317,41 @@ __global__ void k_attn_merge(AttnScratch sc, int n_chunks_alloc, int n_q, int d,
     }
 }
 
-int launch_attn_merge(const AttnScratch& sc, int n_chunks_alloc, int rows, int n_q, int d, const DevState* st,
-                      int draft_mode, uint16_t* out, cudaStream_t s) {
+int launch_attn_merge(const AttnScratch& sc, int n_chunks_alloc, int chunk_tokens, int rows, int n_q, int d,
+                      const DevState* st, int draft_mode, uint16_t* out, cudaStream_t s) {
     dim3 grid(n_q, rows);
-    k_attn_merge<<<grid, 128, 0, s>>>(sc, n_chunks_alloc, n_q, d, st, draft_mode, out);
+    k_attn_merge<<<grid, 128, 0, s>>>(sc, n_chunks_alloc, chunk_tokens, n_q, d, st, draft_mode, out);
     CASS_LAUNCH_CHECK();
     return CASS_OK;
+}
+
+size_t draft_attn_smem_bytes(const KvGeom& g) {
+    return (size_t)g.d * kMaxGroup * 4 + (size_t)kMaxGroup * kDaTok * 4 + 2 * kMaxGroup * 4 + 512 * 4 +
+           (size_t)4 * (g.wpt + 1) * 32 * 4 + (size_t)4 * (kDaUnaStage + 2) * 32 * 4 + (size_t)kDaTok * g.d * 2 + 64;
 }
 
 int launch_draft_attn(const KvGeom& g, const KvComp& ck, const KvComp& cv, const uint16_t* qkv, int n_q,
                       const DevState* st, const AttnScratch& sc, uint16_t* out, cudaStream_t s) {
     const int G = n_q / g.n_kv;
     if (G > kMaxGroup || g.d > 256 || g.d % 32) return CASS_ERR_UNSUPPORTED;
-    const int n_chunks = ceil_div(g.max_seq, kAttnChunk);
-    size_t smem = (size_t)kMaxGroup * g.d * 4 + (size_t)kMaxGroup * kAttnChunk * 4 + 2 * kMaxGroup * 4 +
-                  (size_t)kDaWarps * g.wpt * 32 * 4 + (size_t)kDaWarps * kDaUnaStage * 32 * 4 +
-                  (size_t)kAttnChunk * g.d * 2 + 512;
-    static size_t attr = 0;
-    if (smem > attr) {
-        CASS_CUDA_CHECK(cudaFuncSetAttribute(k_draft_attn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        attr = smem;
-    }
+    const int n_chunks = ceil_div(g.max_seq, kDaTok);
+    const size_t smem = draft_attn_smem_bytes(g);
     dim3 grid(n_chunks, g.n_kv);
-    k_draft_attn<<<grid, 256, smem, s>>>(g, ck, cv, qkv, n_q, st, sc, n_chunks);
+#define CASS_DA_LAUNCH(TT)                                                                                           \
+    do {                                                                                                             \
+        static size_t attr = 0;                                                                                      \
+        if (smem > attr) {                                                                                           \
+            CASS_CUDA_CHECK(cudaFuncSetAttribute(k_draft_attn<TT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
+            attr = smem;                                                                                             \
+        }                                                                                                            \
+        k_draft_attn<TT><<<grid, kDaThreads, smem, s>>>(g, ck, cv, qkv, n_q, st, sc, n_chunks);                      \
+    } while (0)
+    if (g.t == 4) CASS_DA_LAUNCH(4);
+    else if (g.t == 0) CASS_DA_LAUNCH(0);
+    else return CASS_ERR_UNSUPPORTED;
+#undef CASS_DA_LAUNCH
     CASS_LAUNCH_CHECK();
-    return launch_attn_merge(sc, n_chunks, 1, n_q, g.d, st, 1, out, s);
+    return launch_attn_merge(sc, n_chunks, kDaTok, 1, n_q, g.d, st, 1, out, s);
 }
 
 }  // namespace cass

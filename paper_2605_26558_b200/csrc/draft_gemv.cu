@@ -31,6 +31,17 @@ __device__ __forceinline__ uint32_t shl_sat(uint32_t v, uint32_t s) {      // sh
     return r;
 }
 
+__device__ __forceinline__ uint32_t bfind_u32(uint32_t v) {         // index of the most significant one, -1 if none
+    uint32_t r;
+    asm("bfind.u32 %0, %1;" : "=r"(r) : "r"(v));
+    return r;
+}
+__device__ __forceinline__ uint32_t mad_lo(uint32_t a, uint32_t b, uint32_t c) {
+    uint32_t r;
+    asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(c));
+    return r;
+}
+
 struct WalkState {
     float acc;
     uint32_t bpos, upos;
@@ -77,7 +88,7 @@ __device__ __forceinline__ uint32_t lds_u32_off(uint32_t addr) {
 // Dot product of one chunk (32 rows, lane = row) with x.  T = truncated mantissa bits (0 or 4).  Every lane walks
 // its row in groups of 8 kept values through 32-bit windows: one bitmap window per group, one unary window per 4
 // codewords.  A group whose 8 kept columns span more than 32 columns, or whose 4 codewords take more than 32 bits,
-// shows up as a window that ran dry (a leading-zero count of 32); that lane then redoes the group with the careful
+// shows up as a window that ran dry (no bit left to find); that lane then redoes the group with the careful
 // walk while the others wait.  The walk addresses shared memory through 32-bit shared-space addresses.
 template <int T>
 __device__ __forceinline__ float chunk_dot_fast(const uint32_t* __restrict__ sb, const SbGeom& g, int ch, int lane,
@@ -104,34 +115,38 @@ __device__ __forceinline__ float chunk_dot_fast(const uint32_t* __restrict__ sb,
     const uint32_t bpos_lim = (uint32_t)(g.bm_words * 32), upos_lim = (uint32_t)(g.w_u * 32);
     float acc = 0.f;
 
+    // Bit positions are counted from the least significant end (bfind): a window keeps its place and the bit
+    // just used is cleared, so a kept column is x[bpos + 31 - p] and a codeword's rank is the distance between two
+    // consecutive terminators.  A window that ran dry gives p = -1; once dry it stays dry, so the sign of the last
+    // position of each window tells whether the whole group fitted.
     auto group = [&](int grp, bool tail) {
         const WalkState st0 = {acc, bpos, upos};
         const uint32_t ba = bm_a + (bpos >> 5) * 128u;
         uint32_t bv = __funnelshift_l(lds_u32_off<128>(ba), lds_u32(ba), bpos);    // 32 columns from bpos on
-        const uint32_t xg = xs_a + bpos * 4u;
-        uint32_t xa = xg;                           // address of x[bpos + zero columns skipped so far]
+        const uint32_t xg = xs_a + bpos * 4u + 124u;                               // address of x[bpos + 31]
         uint32_t fwd[NFW];
         fwd[0] = lds_u32(fl_a);
         if (NFW > 1) fwd[NFW - 1] = lds_u32_off<128>(fl_a);
         const int rem = m - grp * kGroupCols;
-        uint32_t dry = 0;                           // bit 5 set: a window ran dry under a value that counts
-        uint32_t umax = 0;
+        uint32_t dry = 0;                           // sign bit set: a window ran dry under a value that counts
+        uint32_t p = 0;
 #pragma unroll
         for (int half = 0; half < kGroupCols / kGroupCodes; ++half) {
             const uint32_t ua = un_a + (upos >> 5) * 128u;
             uint32_t uv = __funnelshift_l(lds_u32_off<128>(ua), lds_u32(ua), upos);   // 32 code bits from upos on
-            uint32_t usum = 0;
-            auto elem = [&](auto ec) {
-                constexpr int e = decltype(ec)::value;
-                const uint32_t s = __clz(bv);                        // zeros before the next kept column
-                xa += s * 4u;
+            uint32_t la = lut_a + 124u;             // lut + 4 * (position of the previous terminator - 1); none yet: 32
+            uint32_t q = 0;
+#pragma unroll
+            for (int j = 0; j < kGroupCodes; ++j) {
+                const int e = half * kGroupCodes + j;
+                p = bfind_u32(bv);                                   // next kept column
                 float xv;
-                asm volatile("ld.shared.f32 %0, [%1+%2];" : "=f"(xv) : "r"(xa), "n"(4 * e));
-                bv = shl_sat(shl_sat(bv, s), 1);
-                const uint32_t tt = __clz(uv);                       // rank = zeros before the terminating one
-                const uint32_t eb = lds_u32(lut_a + tt * 4u);
-                uv = shl_sat(shl_sat(uv, tt), 1);
-                usum += tt;
+                asm volatile("ld.shared.f32 %0, [%1];" : "=f"(xv) : "r"(mad_lo(p, 0xFFFFFFFCu, xg)));
+                bv &= ~shl_sat(1u, p);
+                q = bfind_u32(uv);                                   // next terminator
+                const uint32_t eb = lds_u32(mad_lo(q, 0xFFFFFFFCu, la));          // lut[previous - q - 1]
+                la = mad_lo(q, 4u, lut_a - 4u);
+                uv &= ~shl_sat(1u, q);
                 const uint32_t fword = fwd[e / PER];
                 const uint32_t a = __funnelshift_l(fword, fword, (F * (e % PER)) & 31);
                 const uint32_t wb = (a & MASK) | eb;
@@ -139,26 +154,17 @@ __device__ __forceinline__ float chunk_dot_fast(const uint32_t* __restrict__ sb,
                     acc = fmaf(__uint_as_float(wb), xv, acc);
                 } else if (e < rem) {
                     acc = fmaf(__uint_as_float(wb), xv, acc);
-                    dry |= s | tt;
+                    dry |= p | q;
                 }
-            };
-            if (half == 0) {
-                elem(std::integral_constant<int, 0>{}); elem(std::integral_constant<int, 1>{});
-                elem(std::integral_constant<int, 2>{}); elem(std::integral_constant<int, 3>{});
-            } else {
-                elem(std::integral_constant<int, 4>{}); elem(std::integral_constant<int, 5>{});
-                elem(std::integral_constant<int, 6>{}); elem(std::integral_constant<int, 7>{});
             }
-            upos += usum + kGroupCodes;
-            if (tail) upos = min(upos, upos_lim);                 // rows that ran out of values stay inside the buffers
-            else umax = max(umax, usum);
+            upos += 32u - q;                                         // bits up to and including the last terminator
+            if (tail) upos = min(upos, upos_lim);                    // rows that ran out of values stay inside the buffers
+            else dry |= q;
         }
-        const uint32_t adv = (xa - xg) >> 2;        // zero columns skipped in this window
-        bpos += adv + kGroupCols;
+        bpos += 32u - p;
         if (tail) bpos = min(bpos, bpos_lim);
-        // full group: the 8 columns fit the window iff adv + 8 <= 32, the 4 codewords of a half iff usum + 4 <= 32
-        else dry = (uint32_t)__vimax3_s32((int)adv + 4, (int)umax, 0) > 28u ? 32u : 0u;
-        if (dry & 32u) {
+        else dry |= p;
+        if ((int32_t)dry < 0) {
             const WalkState r = group_slow<T>(bmS, unS, flS + (fw + grp * NFW) * 32, min(rem, kGroupCols), st0, bpos_lim,
                                               upos_lim, xs, lut);
             acc = r.acc; bpos = r.bpos; upos = r.upos;
@@ -230,14 +236,18 @@ __global__ void __launch_bounds__(1024) k_draft_gemv(const uint32_t* __restrict_
     if (tid == 0) {
         for (int i = 0; i < kGemvStages && i < n_tiles; ++i) issue(i);
     }
-    // x of this segment (fp32), zero beyond the matrix, and the rank -> exponent table pre-shifted into place
+    // the rank -> exponent table, pre-shifted into place
+    const uint8_t* cb = reinterpret_cast<const uint8_t*>(blob) + kBlobHeaderBytes;
+    for (int i = tid; i < 256; i += blockDim.x) lut[i] = (uint32_t)cb[i] << 23;
+    // Everything above touches only the blob, which no kernel writes.  When the launch allows this grid to start
+    // before its predecessor in the stream has finished, wait here: x and the scratch `partial` are the predecessor's.
+    pdl_wait();
+    // x of this segment (fp32), zero beyond the matrix
     const int c0 = seg * seg_cols;
     for (int i = tid; i < seg_cols + kXSlack; i += blockDim.x) {
         int c = c0 + i;
         xs[i] = (i < scols && c < k) ? bf16_bits_to_float(x[c]) : 0.f;
     }
-    const uint8_t* cb = reinterpret_cast<const uint8_t*>(blob) + kBlobHeaderBytes;
-    for (int i = tid; i < 256; i += blockDim.x) lut[i] = (uint32_t)cb[i] << 23;
     __syncthreads();
 
     for (int i = 0; i < n_tiles; ++i) {
@@ -324,7 +334,14 @@ int launch_draft_gemv(const void* blob, const cass_blob_info& bi, const void* x_
                                                  (int)smem));                                                  \
             attr_smem = (int)smem;                                                                             \
         }                                                                                                      \
-        k_draft_gemv<TT><<<grid, block, smem, stream>>>(b, x, partial, d_status, stage, bi.max_superblock_bytes, bi.seg_cols); \
+        cudaLaunchConfig_t cfg = {};                                                                           \
+        cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = stream;            \
+        cudaLaunchAttribute at[1];                                                                             \
+        at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   /* prologue may overlap the predecessor */ \
+        at[0].val.programmaticStreamSerializationAllowed = 1;                                                  \
+        cfg.attrs = at; cfg.numAttrs = 1;                                                                      \
+        CASS_CUDA_CHECK(cudaLaunchKernelEx(&cfg, k_draft_gemv<TT>, b, x, partial, d_status, stage,             \
+                                           (int)bi.max_superblock_bytes, (int)bi.seg_cols));                   \
     } while (0)
     if (bi.trunc_bits == 4) CASS_GEMV_LAUNCH(4);
     else if (bi.trunc_bits == 0) CASS_GEMV_LAUNCH(0);

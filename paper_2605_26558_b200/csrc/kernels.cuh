@@ -53,8 +53,9 @@ int launch_swiglu(const uint16_t* gu_bf16, const float* partial, int n_seg, int 
                   int ffn, cudaStream_t s);
 // logits (fp32 [rows][vocab], or formed from partials when rows == 1) -> lowest-index argmax per row; optional copy
 // of the logits; bump_inflight adds 1 to the draft counter afterwards.
+// tmp_v / tmp_i: scratch of 16 x 128 entries each.
 int launch_argmax(const float* logits, const float* partial, int n_seg, int n_pad, int rows, int vocab, int32_t* out,
-                  float* logits_copy, DevState* st, int bump_inflight, cudaStream_t s);
+                  float* logits_copy, float* tmp_v, int32_t* tmp_i, DevState* st, int bump_inflight, cudaStream_t s);
 int launch_accept(DevState* st, const int32_t* draft, const int32_t* target, int g, int32_t* n_acc,
                   int32_t* out_tokens, int32_t* next_tok, cudaStream_t s);
 int launch_calib_accum(const uint16_t* x, int rows, int cols, float* sumsq, const DevState* st, cudaStream_t s);

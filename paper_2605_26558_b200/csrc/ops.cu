@@ -33,37 +33,71 @@ __device__ __forceinline__ float block_sum(float v, float* s_red) {
     return t;
 }
 
-// h (+= y) then out = h * rsqrt(mean(h^2) + eps) * gain, all rounded to bf16 where stored.
+// h (+= y) then out = h * rsqrt(mean(h^2) + eps) * gain, all rounded to bf16 where stored.  Four values per thread
+// and iteration (16-byte loads of the fp32 partial sums); the updated values stay in registers for the second pass.
+constexpr int kNormMaxIter = 8;          // hidden <= 8 * 4 * blockDim.x
+
 __global__ void __launch_bounds__(1024) k_residual_rmsnorm(uint16_t* __restrict__ h, const uint16_t* __restrict__ y_bf16,
                                                            const float* __restrict__ partial, int n_seg, int n_pad,
                                                            const uint16_t* __restrict__ gain, uint16_t* __restrict__ out,
                                                            int hidden, float eps) {
     __shared__ float s_red[32];
+    pdl_launch_dependents();            // a following draft GEMV may start fetching its weights now
     const int r = blockIdx.x;
     uint16_t* hr = h + (size_t)r * hidden;
+    float vals[kNormMaxIter][4];
     float ss = 0.f;
-    for (int i = threadIdx.x; i < hidden; i += blockDim.x) {
-        float v = bf16_bits_to_float(hr[i]);
-        if (y_bf16 || partial) {
-            float y;
-            if (partial) {
-                float acc = 0.f;
-                for (int s = 0; s < n_seg; ++s) acc += partial[(size_t)s * n_pad + i];
-                y = round_bf16(acc);
-            } else {
-                y = bf16_bits_to_float(y_bf16[(size_t)r * hidden + i]);
+    const int step = blockDim.x * 4;
+#pragma unroll
+    for (int it = 0; it < kNormMaxIter; ++it) {
+        const int i = threadIdx.x * 4 + it * step;
+        if (i < hidden) {
+            const uint2 hv = *reinterpret_cast<const uint2*>(hr + i);
+            float v[4] = {__uint_as_float(hv.x << 16), __uint_as_float(hv.x & 0xFFFF0000u), __uint_as_float(hv.y << 16),
+                          __uint_as_float(hv.y & 0xFFFF0000u)};
+            if (y_bf16 || partial) {
+                float y[4];
+                if (partial) {
+                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                    for (int s = 0; s < n_seg; ++s) {
+                        const float4 p = *reinterpret_cast<const float4*>(partial + (size_t)s * n_pad + i);
+                        acc.x += p.x; acc.y += p.y; acc.z += p.z; acc.w += p.w;
+                    }
+                    y[0] = round_bf16(acc.x); y[1] = round_bf16(acc.y); y[2] = round_bf16(acc.z); y[3] = round_bf16(acc.w);
+                } else {
+                    const uint2 yv = *reinterpret_cast<const uint2*>(y_bf16 + (size_t)r * hidden + i);
+                    y[0] = __uint_as_float(yv.x << 16); y[1] = __uint_as_float(yv.x & 0xFFFF0000u);
+                    y[2] = __uint_as_float(yv.y << 16); y[3] = __uint_as_float(yv.y & 0xFFFF0000u);
+                }
+#pragma unroll
+                for (int q = 0; q < 4; ++q) v[q] = round_bf16(v[q] + y[q]);
+                uint2 o;
+                o.x = (uint32_t)float_to_bf16_bits(v[0]) | ((uint32_t)float_to_bf16_bits(v[1]) << 16);
+                o.y = (uint32_t)float_to_bf16_bits(v[2]) | ((uint32_t)float_to_bf16_bits(v[3]) << 16);
+                *reinterpret_cast<uint2*>(hr + i) = o;
             }
-            v = round_bf16(v + y);
-            hr[i] = float_to_bf16_bits(v);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) { vals[it][q] = v[q]; ss += v[q] * v[q]; }
         }
-        ss += v * v;
     }
     ss = block_sum(ss, s_red);
     const float inv = 1.0f / sqrtf(ss / (float)hidden + eps);
     if (out) {
-        for (int i = threadIdx.x; i < hidden; i += blockDim.x) {
-            float v = bf16_bits_to_float(hr[i]);
-            out[(size_t)r * hidden + i] = float_to_bf16_bits(v * inv * bf16_bits_to_float(gain[i]));
+#pragma unroll
+        for (int it = 0; it < kNormMaxIter; ++it) {
+            const int i = threadIdx.x * 4 + it * step;
+            if (i < hidden) {
+                const uint2 gv = *reinterpret_cast<const uint2*>(gain + i);
+                const float gq[4] = {__uint_as_float(gv.x << 16), __uint_as_float(gv.x & 0xFFFF0000u), __uint_as_float(gv.y << 16),
+                                     __uint_as_float(gv.y & 0xFFFF0000u)};
+                uint32_t ob[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) ob[q] = float_to_bf16_bits(vals[it][q] * inv * gq[q]);
+                uint2 o;
+                o.x = ob[0] | (ob[1] << 16);
+                o.y = ob[2] | (ob[3] << 16);
+                *reinterpret_cast<uint2*>(out + (size_t)r * hidden + i) = o;
+            }
         }
     }
 }
@@ -102,6 +136,7 @@ __global__ void k_qkv_rope(uint16_t* __restrict__ qkv, const float* __restrict__
 
 __global__ void k_swiglu(const uint16_t* __restrict__ gu, const float* __restrict__ partial, int n_seg, int n_pad,
                          uint16_t* __restrict__ act, int ffn) {
+    pdl_launch_dependents();
     const int r = blockIdx.y;
     for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < ffn; i += gridDim.x * blockDim.x) {
         float g, u;
@@ -122,15 +157,24 @@ __global__ void k_swiglu(const uint16_t* __restrict__ gu, const float* __restric
     }
 }
 
-__global__ void __launch_bounds__(1024) k_argmax(const float* __restrict__ logits, const float* __restrict__ partial,
-                                                 int n_seg, int n_pad, int vocab, int32_t* __restrict__ out,
-                                                 float* __restrict__ logits_copy, DevState* st, int bump_inflight) {
-    __shared__ float s_v[32];
-    __shared__ int s_i[32];
-    const int r = blockIdx.x;
+// Greedy token of each row, lowest index on ties, in two levels: slices of the vocabulary, then the slices' winners.
+constexpr int kArgmaxSlices = 128;
+
+__device__ __forceinline__ void argmax_combine(float& best, int& best_i, float ov, int oi) {
+    if (ov > best || (ov == best && oi < best_i)) { best = ov; best_i = oi; }
+}
+
+__global__ void __launch_bounds__(256) k_argmax_part(const float* __restrict__ logits, const float* __restrict__ partial,
+                                                     int n_seg, int n_pad, int vocab, float* __restrict__ tmp_v,
+                                                     int32_t* __restrict__ tmp_i, float* __restrict__ logits_copy) {
+    __shared__ float s_v[8];
+    __shared__ int s_i[8];
+    const int r = blockIdx.y, nsl = gridDim.x;
+    const int per = ceil_div(vocab, nsl);
+    const int lo = blockIdx.x * per, hi = min(vocab, lo + per);
     float best = -INFINITY;
     int best_i = 0x7fffffff;
-    for (int i = threadIdx.x; i < vocab; i += blockDim.x) {
+    for (int i = lo + threadIdx.x; i < hi; i += blockDim.x) {
         float v;
         if (partial) {
             v = 0.f;
@@ -139,19 +183,41 @@ __global__ void __launch_bounds__(1024) k_argmax(const float* __restrict__ logit
             v = logits[(size_t)r * vocab + i];
         }
         if (logits_copy) logits_copy[(size_t)r * vocab + i] = v;
-        if (v > best || (v == best && i < best_i)) { best = v; best_i = i; }
+        argmax_combine(best, best_i, v, i);
     }
     for (int o = 16; o > 0; o >>= 1) {
         float ov = __shfl_xor_sync(0xffffffffu, best, o);
         int oi = __shfl_xor_sync(0xffffffffu, best_i, o);
-        if (ov > best || (ov == best && oi < best_i)) { best = ov; best_i = oi; }
+        argmax_combine(best, best_i, ov, oi);
     }
-    int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     if (lane == 0) { s_v[warp] = best; s_i[warp] = best_i; }
     __syncthreads();
     if (threadIdx.x == 0) {
-        for (int w = 1; w < (int)(blockDim.x >> 5); ++w)
-            if (s_v[w] > best || (s_v[w] == best && s_i[w] < best_i)) { best = s_v[w]; best_i = s_i[w]; }
+        for (int w = 1; w < (int)(blockDim.x >> 5); ++w) argmax_combine(best, best_i, s_v[w], s_i[w]);
+        tmp_v[r * nsl + blockIdx.x] = best;
+        tmp_i[r * nsl + blockIdx.x] = best_i;
+    }
+}
+
+__global__ void __launch_bounds__(kArgmaxSlices) k_argmax_final(const float* __restrict__ tmp_v, const int32_t* __restrict__ tmp_i,
+                                                                int nsl, int32_t* __restrict__ out, DevState* st, int bump_inflight) {
+    __shared__ float s_v[kArgmaxSlices / 32];
+    __shared__ int s_i[kArgmaxSlices / 32];
+    const int r = blockIdx.x;
+    float best = -INFINITY;
+    int best_i = 0x7fffffff;
+    if ((int)threadIdx.x < nsl) { best = tmp_v[r * nsl + threadIdx.x]; best_i = tmp_i[r * nsl + threadIdx.x]; }
+    for (int o = 16; o > 0; o >>= 1) {
+        float ov = __shfl_xor_sync(0xffffffffu, best, o);
+        int oi = __shfl_xor_sync(0xffffffffu, best_i, o);
+        argmax_combine(best, best_i, ov, oi);
+    }
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (lane == 0) { s_v[warp] = best; s_i[warp] = best_i; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int w = 1; w < kArgmaxSlices / 32; ++w) argmax_combine(best, best_i, s_v[w], s_i[w]);
         out[r] = best_i == 0x7fffffff ? 0 : best_i;
         if (bump_inflight && r == 0) st->inflight += 1;
     }
@@ -203,8 +269,14 @@ int launch_embed(const int32_t* toks, const uint16_t* embed, uint16_t* h, int ro
     return CASS_OK;
 }
 
+static int norm_threads(int hidden) {
+    int t = ceil_div(ceil_div(hidden, 4), 32) * 32;
+    return t > 1024 ? 1024 : t;
+}
+
 int launch_rmsnorm(const uint16_t* h, const uint16_t* gain, uint16_t* out, int rows, int hidden, float eps, cudaStream_t s) {
-    k_residual_rmsnorm<<<rows, 1024, 0, s>>>(const_cast<uint16_t*>(h), nullptr, nullptr, 0, 0, gain, out, hidden, eps);
+    if (hidden % 4 || hidden > kNormMaxIter * 4 * 1024) return CASS_ERR_UNSUPPORTED;
+    k_residual_rmsnorm<<<rows, norm_threads(hidden), 0, s>>>(const_cast<uint16_t*>(h), nullptr, nullptr, 0, 0, gain, out, hidden, eps);
     CASS_LAUNCH_CHECK();
     return CASS_OK;
 }
@@ -212,7 +284,8 @@ int launch_rmsnorm(const uint16_t* h, const uint16_t* gain, uint16_t* out, int r
 int launch_residual_rmsnorm(uint16_t* h, const uint16_t* y_bf16, const float* partial, int n_seg, int n_pad,
                             const uint16_t* gain, uint16_t* out, int rows, int hidden, float eps, cudaStream_t s) {
     if (partial && rows != 1) return CASS_ERR_INVALID_ARG;
-    k_residual_rmsnorm<<<rows, 1024, 0, s>>>(h, y_bf16, partial, n_seg, n_pad, gain, out, hidden, eps);
+    if (hidden % 4 || hidden > kNormMaxIter * 4 * 1024) return CASS_ERR_UNSUPPORTED;
+    k_residual_rmsnorm<<<rows, norm_threads(hidden), 0, s>>>(h, y_bf16, partial, n_seg, n_pad, gain, out, hidden, eps);
     CASS_LAUNCH_CHECK();
     return CASS_OK;
 }
@@ -237,9 +310,14 @@ int launch_swiglu(const uint16_t* gu_bf16, const float* partial, int n_seg, int 
 }
 
 int launch_argmax(const float* logits, const float* partial, int n_seg, int n_pad, int rows, int vocab, int32_t* out,
-                  float* logits_copy, DevState* st, int bump_inflight, cudaStream_t s) {
+                  float* logits_copy, float* tmp_v, int32_t* tmp_i, DevState* st, int bump_inflight, cudaStream_t s) {
     if (partial && rows != 1) return CASS_ERR_INVALID_ARG;
-    k_argmax<<<rows, 1024, 0, s>>>(logits, partial, n_seg, n_pad, vocab, out, logits_copy, st, bump_inflight);
+    int nsl = ceil_div(vocab, 1024);
+    if (nsl > kArgmaxSlices) nsl = kArgmaxSlices;
+    dim3 grid(nsl, rows);
+    k_argmax_part<<<grid, 256, 0, s>>>(logits, partial, n_seg, n_pad, vocab, tmp_v, tmp_i, logits_copy);
+    CASS_LAUNCH_CHECK();
+    k_argmax_final<<<rows, kArgmaxSlices, 0, s>>>(tmp_v, tmp_i, nsl, out, st, bump_inflight);
     CASS_LAUNCH_CHECK();
     return CASS_OK;
 }

@@ -7,9 +7,6 @@
 
 namespace cass {
 
-int launch_attn_merge(const AttnScratch& sc, int n_chunks_alloc, int rows, int n_q, int d, const DevState* st,
-                      int draft_mode, uint16_t* out, cudaStream_t s);
-
 struct LayerDev {
     cass_layer_weights w;
     const void* blob[4];
@@ -41,6 +38,7 @@ struct Session {
     size_t partial_floats;
     AttnScratch asc;
     int32_t* argmax_tmp;
+    float* argmax_val;
     bool have_blobs, codebooks_ready;
     int qkv_dim, kmax;
 };
@@ -63,6 +61,7 @@ static int check_desc(const cass_model_desc* d, const cass_format* f) {
     if (d->gamma_max < 0 || d->gamma_max + 1 > kMaxVerifyRows) return CASS_ERR_INVALID_ARG;
     if (f->kv_prune_permille < 0 || f->kv_prune_permille > 999 || f->kv_trunc_bits < 0 || f->kv_trunc_bits > 7)
         return CASS_ERR_INVALID_ARG;
+    if (f->kv_trunc_bits != 0 && f->kv_trunc_bits != 4) return CASS_ERR_UNSUPPORTED;    // draft attention walks t = 0 or 4 records
     return CASS_OK;
 }
 
@@ -138,7 +137,8 @@ static size_t layout(Session* s, uint8_t* base) {
     s->asc.o = (float*)at(p.take(pairs * n_chunks * d.head_dim * 4));
     s->asc.m = (float*)at(p.take(pairs * n_chunks * 4));
     s->asc.l = (float*)at(p.take(pairs * n_chunks * 4));
-    s->argmax_tmp = (int32_t*)at(p.take(64 * 4));
+    s->argmax_tmp = (int32_t*)at(p.take(kMaxVerifyRows * 128 * 4));
+    s->argmax_val = (float*)at(p.take(kMaxVerifyRows * 128 * 4));
     s->layers.resize(d.n_layers);
     for (int l = 0; l < d.n_layers; ++l) {
         LayerDev& L = s->layers[l];
@@ -340,6 +340,15 @@ extern "C" int cass_kv_query(void* session, int layer, int kind, int head, cass_
     return CASS_OK;
 }
 
+extern "C" int cass_draft_attention(void* session, int layer, const void* q_bf16, void* out_bf16, void* stream_) {
+    if (!session || !q_bf16 || !out_bf16) return CASS_ERR_INVALID_ARG;
+    Session* s = (Session*)session;
+    if (layer < 0 || layer >= s->d.n_layers) return CASS_ERR_INVALID_ARG;
+    LayerDev& L = s->layers[layer];
+    return launch_draft_attn(s->kg, L.ck, L.cv, (const uint16_t*)q_bf16, s->d.n_q_heads, s->st, s->asc, (uint16_t*)out_bf16,
+                             (cudaStream_t)stream_);
+}
+
 extern "C" int cass_debug_activation(void* session, int which, const void** d_ptr, int* h_rows, int* h_cols) {
     if (!session || !d_ptr) return CASS_ERR_INVALID_ARG;
     Session* s = (Session*)session;
@@ -386,7 +395,7 @@ extern "C" int cass_verify(void* session, const int32_t* toks, int g, int32_t* t
     }
     RC(launch_calib_accum(s->xn, rows, d.hidden, s->calib_lm, s->st, st));
     RC(launch_verify_gemm((const uint16_t*)s->lm_head, s->xn, rows, d.vocab, d.hidden, s->vg_partial, nullptr, s->logits, &s->st->status, st));
-    RC(launch_argmax(s->logits, nullptr, 0, 0, rows, d.vocab, target_argmax, logits_opt, s->st, 0, st));
+    RC(launch_argmax(s->logits, nullptr, 0, 0, rows, d.vocab, target_argmax, logits_opt, s->argmax_val, s->argmax_tmp, s->st, 0, st));
     return CASS_OK;
 }
 
@@ -420,7 +429,7 @@ extern "C" int cass_draft_step(void* session, const int32_t* tok_in, int32_t* to
                                    d.rms_eps, st));
     }
     RC(launch_draft_gemv(s->lm_blob, s->lm_bi, s->xn, s->partial, status, st));
-    RC(launch_argmax(nullptr, s->partial, s->lm_bi.n_seg, s->lm_bi.n_rowblocks * 32, 1, d.vocab, tok_out, logits_opt, s->st, 1, st));
+    RC(launch_argmax(nullptr, s->partial, s->lm_bi.n_seg, s->lm_bi.n_rowblocks * 32, 1, d.vocab, tok_out, logits_opt, s->argmax_val, s->argmax_tmp, s->st, 1, st));
     return CASS_OK;
 }
 

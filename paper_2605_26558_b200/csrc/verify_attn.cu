@@ -115,8 +115,8 @@ __global__ void __launch_bounds__(256) k_verify_attn(KvGeom g, const uint16_t* _
     }
 }
 
-int launch_attn_merge(const AttnScratch& sc, int n_chunks_alloc, int rows, int n_q, int d, const DevState* st,
-                      int draft_mode, uint16_t* out, cudaStream_t s);
+int launch_attn_merge(const AttnScratch& sc, int n_chunks_alloc, int chunk_tokens, int rows, int n_q, int d,
+                      const DevState* st, int draft_mode, uint16_t* out, cudaStream_t s);
 
 int launch_verify_attn(const KvGeom& g, const uint16_t* k_cache, const uint16_t* v_cache, const uint16_t* qkv, int rows,
                        int n_q, const DevState* st, const AttnScratch& sc, uint16_t* out, cudaStream_t s) {
@@ -133,7 +133,7 @@ int launch_verify_attn(const KvGeom& g, const uint16_t* k_cache, const uint16_t*
     dim3 grid(n_chunks, g.n_kv);
     k_verify_attn<<<grid, 256, smem, s>>>(g, k_cache, v_cache, qkv, rows, n_q, st, sc, n_chunks);
     CASS_LAUNCH_CHECK();
-    return launch_attn_merge(sc, n_chunks, rows, n_q, g.d, st, 0, out, s);
+    return launch_attn_merge(sc, n_chunks, kAttnChunk, rows, n_q, g.d, st, 0, out, s);
 }
 
 }  // namespace cass

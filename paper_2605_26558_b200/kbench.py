@@ -115,16 +115,105 @@ def bench_verify_gemm(name, copies, iters, rows=5):
             "peak": f"{peak} GB/s ({kind})", "tflops": 2.0 * rows * n * k * copies / (ms * 1e-3) / 1e12}
 
 
+def bench_draft_attn(n_pos, layers, iters):
+    """Draft attention and the KV encoder on `layers` Llama-3-8B-shaped layers (32 q / 8 kv heads of 128) holding
+    n_pos synthetic positions each; the layers' compressed caches together exceed L2 for layers * n_pos >= 2.6e5."""
+    import synth
+    from . import engine
+    dev = torch.device("cuda")
+    shape = synth.ModelShape(n_layers=layers, hidden=256, n_q_heads=32, n_kv_heads=8, head_dim=128, ffn=256, vocab=256)
+    wt = synth.model_weights(shape, 0, device=dev, layers=[0])
+    lw = engine.fuse_layer_weights(wt["layers"][0])
+    gw = {"layers": [lw] * layers, "embed": wt["embed"], "lm_head": wt["lm_head"], "norm_final": wt["norm_final"]}
+    eng = engine.Engine(shape, gw, max_seq=(n_pos + 64 + 255) // 256 * 256, gamma_max=4)
+    n0 = min(n_pos, 512)
+    kvs = []
+    for l in range(layers):
+        k, v = synth.kv_fill(n_pos + 1, 8, 128, l, "kbench/kv", device=dev)
+        kvs.append((k, v))
+        B.cass_kv_append(eng.session, l, k[:n0].contiguous(), v[:n0].contiguous(), 0, n0, B.KV_BF16)
+    B.cass_kv_build_codebook(eng.session, n0)
+    for l, (k, v) in enumerate(kvs):
+        if n_pos > n0:
+            B.cass_kv_append(eng.session, l, k[n0:n_pos].contiguous(), v[n0:n_pos].contiguous(), n0, n_pos - n0,
+                             B.KV_BF16 | B.KV_COMPRESSED)
+    B.cass_set_len(eng.session, n_pos - 1)
+    q = synth.activation_vector(128, 2, "kbench/q", device=dev, rows=32).contiguous()
+    out = torch.zeros(32, 128, dtype=torch.bfloat16, device=dev)
+    base, mem32 = eng.mem.data_ptr(), eng.mem.view(torch.int32)
+    bytes_layer = 0
+    for kind in (0, 1):
+        for head in range(8):
+            view = B.cass_kv_query(eng.session, 0, kind, head)
+            oo = (view.offsets - base) // 4
+            una_words = int(mem32[oo + n_pos].item())
+            bytes_layer += 4 * (una_words + n_pos * view.fixed_words_per_token + n_pos + 1)
+    ms = _time(lambda: [B.cass_draft_attention(eng.session, l, q, out) for l in range(layers)], iters)
+    peak, kind_ = _peak()
+    gbs = bytes_layer * layers / (ms * 1e-3) / 1e9
+    res = [{"kernel": "draft_attn (+merge)", "positions": n_pos, "layers": layers, "us_per_layer": ms * 1e3 / layers,
+            "compressed_kv_bytes_per_layer": bytes_layer, "bf16_kv_bytes_per_layer": n_pos * 8 * 128 * 2 * 2,
+            "algorithmic_GBps": gbs, "frac_of_hbm_peak": gbs / peak, "peak": f"{peak} GB/s ({kind_})"}]
+    # KV encoder: one new token per layer, both caches
+    ms = _time(lambda: [B.cass_kv_append(eng.session, l, kvs[l][0][n_pos:], kvs[l][1][n_pos:], n_pos, 1,
+                                         B.KV_BF16 | B.KV_COMPRESSED) for l in range(layers)], iters)
+    res.append({"kernel": "kv_append (1 token, bf16 + compressed)", "positions": n_pos, "us_per_layer": ms * 1e3 / layers})
+    assert eng.status()[0] == 0
+    eng.close()
+    return res
+
+
+def step_breakdown(gamma=4, n_prompt=512, steps=3):
+    """Per-kernel device time of the speculative step on the full Llama-3-8B shape, from the CUPTI kernel trace of a
+    few eager steps (warm, not under ncu)."""
+    import re
+    import collections
+    import synth
+    from . import engine
+    from torch.profiler import profile, ProfilerActivity
+    dev = torch.device("cuda")
+    shape = synth.LLAMA3_8B
+    wt = synth.model_weights(shape, 0, device=dev)
+    gw = {"layers": [engine.fuse_layer_weights(lw) for lw in wt["layers"]], "embed": wt["embed"], "lm_head": wt["lm_head"],
+          "norm_final": wt["norm_final"]}
+    del wt
+    eng = engine.Engine(shape, gw, max_seq=n_prompt + 256, gamma_max=gamma)
+    eng.prefill(synth.random_prompt(n_prompt, shape.vocab, 0), calibrate=True)
+    eng.encode_weights(eng.calib_norms())
+    eng.build_kv_codebook()
+    for _ in range(2):
+        eng.step(gamma)
+    torch.cuda.synchronize()
+    with profile(activities=[ProfilerActivity.CUDA]) as prof:
+        for _ in range(steps):
+            eng.step(gamma)
+        torch.cuda.synchronize()
+    agg = collections.defaultdict(lambda: [0, 0.0])
+    for ev in prof.events():
+        if ev.device_type is not None and "cuda" in str(ev.device_type).lower() and ev.name.find("Memcpy") < 0 and ev.name.find("Memset") < 0:
+            name = re.sub(r"<.*|\(.*", "", ev.name).replace("void ", "").replace("cass::", "")
+            agg[name][0] += 1
+            agg[name][1] += ev.device_time_total if hasattr(ev, "device_time_total") else ev.cuda_time_total
+    tot = sum(v[1] for v in agg.values())
+    rows = [{"kernel": k, "launches_per_step": v[0] / steps, "us_per_step": v[1] / steps, "share": v[1] / tot,
+             "avg_us": v[1] / v[0]} for k, v in sorted(agg.items(), key=lambda kv: -kv[1][1])]
+    eng.close()
+    return [{"kernel": "step_breakdown", "gamma": gamma, "kernel_us_per_step": tot / steps}] + rows
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--kernel", default="gemv")
     ap.add_argument("--shape", default="all")
     ap.add_argument("--copies", type=int, default=0, help="distinct operand copies (0: enough to exceed 2x L2)")
     ap.add_argument("--iters", type=int, default=5)
+    ap.add_argument("--positions", type=int, default=0)
+    ap.add_argument("--chunk", type=int, default=0, help="columns per decode chunk of the weight format (0 = default 256)")
+    ap.add_argument("--seg", type=int, default=0, help="columns per superblock of the weight format (0 = default 2048)")
     ap.add_argument("--p", type=int, default=400)
     ap.add_argument("--t", type=int, default=4)
     args = ap.parse_args()
-    fmt = B.default_format(w_p=args.p, w_t=args.t)
+    fmt = B.default_format(w_p=args.p, w_t=args.t, chunk_cols=args.chunk, seg_cols=args.seg)
     out = []
     if args.kernel in ("gemv", "all"):
         for name in (SHAPES if args.shape == "all" else [args.shape]):
@@ -136,6 +225,11 @@ def main():
             n, k = SHAPES[name]
             copies = args.copies or max(2, int(300e6 / (n * k * 2)) + 1)
             out.append(bench_verify_gemm(name, copies, args.iters))
+    if args.kernel == "step":
+        out.extend(step_breakdown())
+    if args.kernel in ("attn", "all"):
+        for n_pos in ([args.positions] if args.positions else [4096, 32768]):
+            out.extend(bench_draft_attn(n_pos, max(2, int(3.0e5 / n_pos) + 1), args.iters))
     for r in out:
         print(json.dumps(r))
 

@@ -4,7 +4,7 @@ import pytest
 import torch
 
 import synth
-from oracle import codec
+from oracle import codec, layout
 
 pytestmark = pytest.mark.gpu
 TOL = 2e-2
@@ -59,3 +59,45 @@ def test_verify_gemm_rows_do_not_depend_on_the_batch(cass):
     x2[1:] = float("nan")                                      # other rows' contents cannot leak into row 0
     alone, _ = _run(cass, w, x2, 1)
     assert torch.equal(alone[0], full[0])
+
+
+@pytest.mark.parametrize("n_pos", [1, 63, 64, 65, 700, 4096])
+def test_draft_attention_llama_layer_shape(cass, n_pos):
+    """Draft attention of one Llama-3-8B-shaped layer (32 q / 8 kv heads of 128) over synthetic KV (N(0,1), outlier
+    channels in K) against the oracle: softmax(q . K_hat / sqrt(d)) V_hat on the zero-padded reconstruction."""
+    from paper_2605_26558_b200 import engine
+    shape = synth.ModelShape(n_layers=1, hidden=256, n_q_heads=32, n_kv_heads=8, head_dim=128, ffn=256, vocab=256)
+    wt = synth.model_weights(shape, 0, device="cuda")
+    gw = {"layers": [engine.fuse_layer_weights(lw) for lw in wt["layers"]], "embed": wt["embed"], "lm_head": wt["lm_head"],
+          "norm_final": wt["norm_final"]}
+    eng = engine.Engine(shape, gw, max_seq=4096 + 64, gamma_max=4)
+    k, v = synth.kv_fill(n_pos, 8, 128, 1, "ka/kv")
+    n0 = max(1, min(n_pos, 512))                     # codebooks come from the first positions, the rest is appended
+    cass.cass_kv_append(eng.session, 0, k[:n0].cuda().contiguous(), v[:n0].cuda().contiguous(), 0, n0, cass.KV_BF16)
+    cass.cass_kv_build_codebook(eng.session, n0)
+    if n_pos > n0:
+        cass.cass_kv_append(eng.session, 0, k[n0:].cuda().contiguous(), v[n0:].cuda().contiguous(), n0, n_pos - n0,
+                            cass.KV_BF16 | cass.KV_COMPRESSED)
+    cass.cass_set_len(eng.session, n_pos - 1)
+    q = synth.activation_vector(128, 2, "ka/q", rows=32)
+    out = torch.zeros(32, 128, dtype=torch.bfloat16, device="cuda")
+    cass.cass_draft_attention(eng.session, 0, q.cuda().contiguous(), out)
+    torch.cuda.synchronize()
+    assert eng.status()[0] == 0
+    kb, vb = _bits(k), _bits(v)
+    kd = codec.bf16_bits_to_f64(codec.draft_bits(kb, codec.keep_mask_kv(kb, 400), 4))
+    vd = codec.bf16_bits_to_f64(codec.draft_bits(vb, codec.keep_mask_kv(vb, 400), 4))
+    qf = codec.bf16_bits_to_f64(_bits(q))
+    want = np.zeros((32, 128))
+    for hq in range(32):
+        sc = kd[:, hq // 4, :] @ qf[hq] / np.sqrt(128.0)
+        p = np.exp(sc - sc.max())
+        want[hq] = (p / p.sum()) @ vd[:, hq // 4, :]
+    got = codec.bf16_bits_to_f64(_bits(out))
+    rms = float(np.sqrt(np.mean(want ** 2)))
+    # The output is rounded to bf16, so each element may be off by half an ulp (<= 2^-8 |value|) on top of the
+    # fp32-vs-fp64 difference, which is held to a twentieth of the 2e-2 bar.
+    err = np.abs(got - want)
+    assert (err <= 2.0 ** -8 * np.abs(want) + 0.05 * TOL * rms).all(), (err.max(), rms)
+    assert np.median(err) <= 0.1 * TOL * rms
+    eng.close()
