@@ -19,7 +19,7 @@ Common rules
 
 Weight blob  (rows N x cols K, row-major source)
   word  0      magic 'CASW'            word  7  chunk_cols C (multiple of 32)
-  word  1      version (2)             word  8  n_seg
+  word  1      version (3)             word  8  n_seg
   word  2      N                       word  9  n_rowblocks = ceil(N/32)
   word  3      K                       word 10  kept per row = K - floor(K*p/1000)
   word  4      p (per-mille)           word 11  directory byte offset (384)
@@ -27,16 +27,20 @@ Weight blob  (rows N x cols K, row-major source)
   word  6      seg_cols (mult. of C)   word 13/14  total bytes (lo/hi)
   bytes 128..383   codebook: rank -> exponent value
   directory: one entry of four words per superblock sb = rowblock*n_seg + seg:
-      {byte offset / 16, W_f, W_u, n_chunks}
+      {byte offset / 16, W_f, W_u, n_chunks | chunk_elems << 8}
   word 15      largest superblock size in bytes
   superblock = 32 rows x one column segment: four sections, each word-interleaved over the 32
   rows (word j of row r sits at index j*32 + r):
-      chunk table  n_chunks+1 words/row : (index of the chunk's first field WORD << 20) | bit
-                                        offset of the chunk's first codeword; the last entry
-                                        holds the segment totals.  The fields of every chunk
-                                        start on a word boundary.
+      chunk table  n_chunks+1 words/row : entry points for parallel decoders.  A row's kept values of
+                                        the segment are cut into n_chunks runs of E values (E, a multiple
+                                        of 8, is the superblock's chunk_elems: the smallest such number
+                                        with n_chunks * E >= the largest kept count among the 32 rows).
+                                        Entry c = (column of the row's value c*E << 20) | bit offset of
+                                        its codeword, or (segment columns << 20) | total code bits if the
+                                        row has no such value; the last entry is
+                                        (kept count << 20) | total code bits.
       bitmap       seg_cols/32 words/row (1 = kept), column c at bit 31 - c%32
-      fields       W_f words/row  (max over the 32 rows of the sum over chunks of ceil(kept_in_chunk / per_word))
+      fields       W_f words/row  (max over the 32 rows of ceil(kept / per_word))
       unary        W_u words/row  (max over the 32 rows)
 
 KV record (one token, one KV head, K or V; d = head_dim)
@@ -51,7 +55,7 @@ import numpy as np
 from . import codec
 
 MAGIC = 0x57534143
-VERSION = 2
+VERSION = 3
 HEADER_BYTES = 128
 CODEBOOK_BYTES = 256
 DIR_OFFSET = HEADER_BYTES + CODEBOOK_BYTES
@@ -171,6 +175,12 @@ def _segment_cols(k_pad: int, seg_cols: int, seg: int) -> int:
     return min(seg_cols, k_pad - seg * seg_cols)
 
 
+def chunk_elems_for(max_kept: int, n_ch: int) -> int:
+    """Values per decode chunk of a superblock: smallest multiple of 8 with n_ch * E >= max_kept (at least 8)."""
+    per_chunk = (max_kept + n_ch - 1) // n_ch
+    return max(8, (per_chunk + 7) // 8 * 8)
+
+
 def encode_weight_blob(w_bits: np.ndarray, act_norm: np.ndarray | None, p: int, t: int,
                        seg_cols: int = 2048, chunk_cols: int = 256,
                        rowblocks=None):
@@ -204,7 +214,7 @@ def encode_weight_blob(w_bits: np.ndarray, act_norm: np.ndarray | None, p: int, 
             c0 = seg * seg_cols
             scols = _segment_cols(k_pad, seg_cols, seg)
             n_ch = (scols + chunk_cols - 1) // chunk_cols
-            rows_tab, rows_bm, rows_f, rows_u = [], [], [], []
+            rows_bm, rows_f, rows_u, rows_idx, rows_cum = [], [], [], [], []
             for rr in range(ROWS_PER_BLOCK):
                 r = rb * ROWS_PER_BLOCK + rr
                 km = np.zeros(scols, dtype=bool)
@@ -219,28 +229,24 @@ def encode_weight_blob(w_bits: np.ndarray, act_norm: np.ndarray | None, p: int, 
                 else:
                     fields = np.zeros(0, dtype=np.uint32)
                     ranks = np.zeros(0, dtype=np.int64)
-                # chunk table: field-word index and code-bit offset at each chunk start.  The fields of a
-                # chunk start on a word boundary, so a decoder can enter the field stream at any chunk.
-                tab = np.zeros(n_ch + 1, dtype=np.uint32)
-                code_len = ranks + 1
-                cum_bits = np.concatenate(([0], np.cumsum(code_len)))
-                fparts = []
-                fword = 0
-                for ch in range(n_ch + 1):
-                    first = int(np.searchsorted(idx, ch * chunk_cols))      # kept values before the chunk
-                    bit_off = int(cum_bits[first])
-                    if fword >= (1 << 12) or bit_off >= (1 << 20):
-                        raise ValueError("chunk table overflow")
-                    tab[ch] = (fword << 20) | bit_off
-                    if ch < n_ch:
-                        last = int(np.searchsorted(idx, (ch + 1) * chunk_cols))
-                        fw = _pack_fields_fast(fields[first:last], t)
-                        fparts.append(fw)
-                        fword += fw.size
-                rows_tab.append(tab)
+                rows_idx.append(idx)
+                rows_cum.append(np.concatenate(([0], np.cumsum(ranks + 1))))
                 rows_bm.append(bits_to_words(km.astype(np.uint8)))
-                rows_f.append(np.concatenate(fparts) if fparts else np.zeros(0, np.uint32))
+                rows_f.append(_pack_fields_fast(fields, t))
                 rows_u.append(bits_to_words(codec.unary_encode_fast(ranks)) if ranks.size else np.zeros(0, np.uint32))
+            chunk_elems = chunk_elems_for(max(x.size for x in rows_idx), n_ch)
+            rows_tab = []
+            for idx, cum in zip(rows_idx, rows_cum):
+                # chunk table: where the row's value c * chunk_elems sits (column, first code bit)
+                tab = np.zeros(n_ch + 1, dtype=np.uint32)
+                total_bits = int(cum[-1])
+                if total_bits >= (1 << 20) or scols >= (1 << 12):
+                    raise ValueError("chunk table overflow")
+                for ch in range(n_ch):
+                    k0 = ch * chunk_elems
+                    tab[ch] = (int(idx[k0]) << 20) | int(cum[k0]) if k0 < idx.size else (scols << 20) | total_bits
+                tab[n_ch] = (idx.size << 20) | total_bits
+                rows_tab.append(tab)
             w_f = max(x.size for x in rows_f)
             w_u = max(x.size for x in rows_u)
 
@@ -253,7 +259,7 @@ def encode_weight_blob(w_bits: np.ndarray, act_norm: np.ndarray | None, p: int, 
             body = np.concatenate([
                 interleave(rows_tab, n_ch + 1), interleave(rows_bm, scols // 32),
                 interleave(rows_f, w_f), interleave(rows_u, w_u)])
-            bodies[rb * n_seg + seg] = (body, w_f, w_u, n_ch)
+            bodies[rb * n_seg + seg] = (body, w_f, w_u, n_ch | (chunk_elems << 8))
 
     info = dict(rows=n, cols=k, p=p, t=t, seg_cols=seg_cols, chunk_cols=chunk_cols, n_seg=n_seg,
                 n_rowblocks=n_rb, kept_per_row=k - codec.n_pruned(k, p), codebook=rank_to_exp,
@@ -301,7 +307,7 @@ def parse_weight_blob(blob: np.ndarray) -> WeightBlobInfo:
 def decode_weight_blob(blob: np.ndarray, use_chunk_table: bool = False) -> np.ndarray:
     """Draft decode of a whole blob -> bf16 bit patterns [N, K] (pruned -> +0, low mantissa -> 0).
 
-    With use_chunk_table, every chunk is decoded on its own, starting from the offsets the chunk
+    With use_chunk_table, every chunk is decoded on its own, starting from the column and code bit the chunk
     table gives (this is how a parallel decoder enters the streams)."""
     blob = np.asarray(blob, dtype=np.uint32)
     info = parse_weight_blob(blob)
@@ -310,7 +316,8 @@ def decode_weight_blob(blob: np.ndarray, use_chunk_table: bool = False) -> np.nd
     out = np.zeros((info.n_rowblocks * ROWS_PER_BLOCK, info.n_seg * info.seg_cols), dtype=np.uint16)
     for sb in range(info.n_rowblocks * info.n_seg):
         rb, seg = divmod(sb, info.n_seg)
-        off16, w_f, w_u, n_ch = (int(x) for x in info.directory[sb])
+        off16, w_f, w_u, w3 = (int(x) for x in info.directory[sb])
+        n_ch, chunk_elems = w3 & 0xFF, w3 >> 8
         scols = _segment_cols(k_pad, info.seg_cols, seg)
         base = off16 * 4
         tab = blob[base: base + (n_ch + 1) * 32].reshape(n_ch + 1, 32); base += (n_ch + 1) * 32
@@ -320,27 +327,28 @@ def decode_weight_blob(blob: np.ndarray, use_chunk_table: bool = False) -> np.nd
         for rr in range(ROWS_PER_BLOCK):
             km = words_to_bits(bm[:, rr]).astype(bool)
             idx = np.flatnonzero(km)
+            assert idx.size == int(tab[n_ch, rr]) >> 20
             if idx.size == 0:
                 continue
             ubits = words_to_bits(un[:, rr])
-            fields = np.zeros(idx.size, dtype=np.uint32)
-            ranks = np.zeros(idx.size, dtype=np.int64)
+            fields = unpack_fields(fl[:, rr], idx.size, t)
             if not use_chunk_table:
                 ranks = codec.unary_decode_fast(ubits, idx.size)
-            done = 0
-            for ch in range(n_ch):
-                fword, bit_off = int(tab[ch, rr]) >> 20, int(tab[ch, rr]) & 0xFFFFF
-                cnt = int(km[ch * info.chunk_cols: (ch + 1) * info.chunk_cols].sum())
-                if cnt == 0:
-                    continue
-                fields[done: done + cnt] = unpack_fields(fl[fword:, rr], cnt, t)
-                if use_chunk_table:
-                    ranks[done: done + cnt] = codec.unary_decode_fast(ubits[bit_off:], cnt)
-                done += cnt
+            else:
+                ranks = np.zeros(idx.size, dtype=np.int64)
+                for ch in range(n_ch):
+                    k0 = ch * chunk_elems
+                    cnt = min(chunk_elems, idx.size - k0)
+                    if cnt <= 0:
+                        assert int(tab[ch, rr]) >> 20 == scols
+                        continue
+                    col, bit_off = int(tab[ch, rr]) >> 20, int(tab[ch, rr]) & 0xFFFFF
+                    assert col == idx[k0]
+                    ranks[k0: k0 + cnt] = codec.unary_decode_fast(ubits[bit_off:], cnt)
             e = info.codebook[ranks].astype(np.uint16)
-            s = (fields >> (7 - t)).astype(np.uint16) & 1
+            s_ = (fields >> (7 - t)).astype(np.uint16) & 1
             m_hi = (fields & ((1 << (7 - t)) - 1)).astype(np.uint16)
-            vals = (s << 15) | (e << 7) | (m_hi << t)
+            vals = (s_ << 15) | (e << 7) | (m_hi << t)
             out[rb * ROWS_PER_BLOCK + rr, seg * info.seg_cols + idx] = vals
     return out[:n, :k]
 
@@ -351,7 +359,8 @@ def blob_section_bits(blob: np.ndarray) -> dict:
     k_pad = (info.cols + 31) // 32 * 32
     tab = bm = fl = un = 0
     for sb in range(info.n_rowblocks * info.n_seg):
-        _, w_f, w_u, n_ch = (int(x) for x in info.directory[sb])
+        _, w_f, w_u, w3 = (int(x) for x in info.directory[sb])
+        n_ch = w3 & 0xFF
         scols = _segment_cols(k_pad, info.seg_cols, sb % info.n_seg)
         tab += (n_ch + 1) * 32 * 32
         bm += scols * 32

@@ -11,7 +11,7 @@
 
 namespace cass {
 
-constexpr int kDaTok = 64;                    // tokens per CTA
+constexpr int kDaTok = kAttnChunk;            // tokens per CTA
 constexpr int kDaThreads = 128;
 constexpr int kDaUnaStage = 32;               // staged unary words per token; longer records are read in place
 constexpr int kMaxGroup = 8;                  // query heads per KV head
@@ -279,6 +279,7 @@ __global__ void __launch_bounds__(kDaThreads) k_draft_attn(KvGeom g, KvComp ck, 
         float acc[kMaxGroup];
 #pragma unroll
         for (int gi = 0; gi < kMaxGroup; ++gi) acc[gi] = 0.f;
+#pragma unroll 4
         for (int t = 0; t < n_tok; ++t) {
             const float v = bf16_bits_to_float(v_s[(size_t)t * d + dim]);
 #pragma unroll
@@ -298,21 +299,40 @@ __global__ void __launch_bounds__(kDaThreads) k_draft_attn(KvGeom g, KvComp ck, 
 
 // Merge the chunk partials of every (row, query head): out = sum_c e^{m_c - M} o_c / sum_c e^{m_c - M} l_c.
 // Row r sees positions < len + (draft: inflight + 1 | verify: r + 1); chunks hold `chunk_tokens` positions.
-__global__ void k_attn_merge(AttnScratch sc, int n_chunks_alloc, int chunk_tokens, int n_q, int d,
-                             const DevState* __restrict__ st, int draft_mode, uint16_t* __restrict__ out) {
+// The reductions run in a fixed order that depends on the number of visible chunks only.
+__global__ void __launch_bounds__(128) k_attn_merge(AttnScratch sc, int n_chunks_alloc, int chunk_tokens, int n_q, int d,
+                                                    const DevState* __restrict__ st, int draft_mode, uint16_t* __restrict__ out) {
+    extern __shared__ float w_s[];                  // [n_chunks_alloc] weights e^{m_c - M}
+    __shared__ float s_red[4];
     pdl_launch_dependents();
     const int hq = blockIdx.x, r = blockIdx.y;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int vis = st->len + (draft_mode ? st->inflight + 1 : r + 1);
     const int n_ch = ceil_div(vis, chunk_tokens);
     const size_t pair = (size_t)r * n_q + hq;
+    const float* mp = sc.m + pair * n_chunks_alloc;
+    const float* lp = sc.l + pair * n_chunks_alloc;
     float M = -INFINITY;
-    for (int c = 0; c < n_ch; ++c) M = fmaxf(M, sc.m[pair * n_chunks_alloc + c]);
+    for (int c = tid; c < n_ch; c += 128) M = fmaxf(M, mp[c]);
+    M = warp_max(M);
+    if (lane == 0) s_red[warp] = M;
+    __syncthreads();
+    M = fmaxf(fmaxf(s_red[0], s_red[1]), fmaxf(s_red[2], s_red[3]));
+    __syncthreads();
     float L = 0.f;
-    for (int c = 0; c < n_ch; ++c) L += expf(sc.m[pair * n_chunks_alloc + c] - M) * sc.l[pair * n_chunks_alloc + c];
-    for (int dim = threadIdx.x; dim < d; dim += blockDim.x) {
+    for (int c = tid; c < n_ch; c += 128) {
+        const float w = expf(mp[c] - M);
+        w_s[c] = w;
+        L += w * lp[c];
+    }
+    L = warp_sum(L);
+    if (lane == 0) s_red[warp] = L;
+    __syncthreads();
+    L = (s_red[0] + s_red[1]) + (s_red[2] + s_red[3]);
+    const float* op = sc.o + pair * n_chunks_alloc * d;
+    for (int dim = tid; dim < d; dim += 128) {
         float acc = 0.f;
-        for (int c = 0; c < n_ch; ++c)
-            acc += expf(sc.m[pair * n_chunks_alloc + c] - M) * sc.o[(pair * n_chunks_alloc + c) * d + dim];
+        for (int c = 0; c < n_ch; ++c) acc = fmaf(w_s[c], op[(size_t)c * d + dim], acc);
         out[((size_t)r * n_q + hq) * d + dim] = float_to_bf16_bits(acc / L);
     }
 }
@@ -320,7 +340,14 @@ __global__ void k_attn_merge(AttnScratch sc, int n_chunks_alloc, int chunk_token
 int launch_attn_merge(const AttnScratch& sc, int n_chunks_alloc, int chunk_tokens, int rows, int n_q, int d,
                       const DevState* st, int draft_mode, uint16_t* out, cudaStream_t s) {
     dim3 grid(n_q, rows);
-    k_attn_merge<<<grid, 128, 0, s>>>(sc, n_chunks_alloc, chunk_tokens, n_q, d, st, draft_mode, out);
+    const size_t smem = (size_t)n_chunks_alloc * 4;
+    if (smem > 200 * 1024) return CASS_ERR_CAPACITY;
+    static size_t attr = 48 * 1024;
+    if (smem > attr) {
+        CASS_CUDA_CHECK(cudaFuncSetAttribute(k_attn_merge, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        attr = smem;
+    }
+    k_attn_merge<<<grid, 128, smem, s>>>(sc, n_chunks_alloc, chunk_tokens, n_q, d, st, draft_mode, out);
     CASS_LAUNCH_CHECK();
     return CASS_OK;
 }

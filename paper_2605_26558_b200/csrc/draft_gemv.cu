@@ -92,26 +92,25 @@ __device__ __forceinline__ uint32_t lds_u32_off(uint32_t addr) {
 // walk while the others wait.  The walk addresses shared memory through 32-bit shared-space addresses.
 template <int T>
 __device__ __forceinline__ float chunk_dot_fast(const uint32_t* __restrict__ sb, const SbGeom& g, int ch, int lane,
-                                                int chunk_cols, const float* __restrict__ xs,
+                                                int chunk_elems, const float* __restrict__ xs,
                                                 const uint32_t* __restrict__ lut) {
     constexpr int F = 8 - T, PER = 32 / F, NFW = kGroupCols / PER;       // field words per group of 8
     constexpr uint32_t MASK = 0x80000000u | (((1u << (7 - T)) - 1u) << (16 + T));   // sign + kept mantissa of a binary32
     static_assert(32 % F == 0 && (PER == 4 || PER == 8), "fast path: rotated fields, 4 or 8 per word");
-    const uint32_t e0 = sb[g.tab + ch * 32 + lane];
-    const uint32_t fw = e0 >> 20;
+    const uint32_t e0 = sb[g.tab + ch * 32 + lane];            // where this row's value ch * chunk_elems sits
+    const uint32_t fw = (uint32_t)(ch * chunk_elems) / PER;    // its field word (chunk_elems is a multiple of 8)
     uint32_t upos = e0 & 0xFFFFFu;
     const uint32_t* bmS = sb + g.bm + lane;
     const uint32_t* flS = sb + g.fl + lane;
     const uint32_t* unS = sb + g.un + lane;
     const uint32_t bm_a = smem_u32(bmS), un_a = smem_u32(unS), xs_a = smem_u32(xs), lut_a = smem_u32(lut);
     uint32_t fl_a = smem_u32(flS + fw * 32);
-    const int wpc = chunk_cols / 32;
-    const int w0 = ch * wpc, w1 = min(w0 + wpc, g.bm_words);
-    int m = 0;
-    for (int w = w0; w < w1; ++w) m += __popc(bmS[w * 32]);
+    // every row has chunk_elems values in each chunk except its last ones, so the lanes of a warp stay in step
+    const int kept = (int)(sb[g.tab + g.n_ch * 32 + lane] >> 20);
+    const int m = max(0, min(chunk_elems, kept - ch * chunk_elems));
     const int n_full = __reduce_min_sync(0xffffffffu, m) / kGroupCols;
     const int n_groups = ceil_div(__reduce_max_sync(0xffffffffu, m), kGroupCols);
-    uint32_t bpos = (uint32_t)(w0 * 32);
+    uint32_t bpos = e0 >> 20;
     const uint32_t bpos_lim = (uint32_t)(g.bm_words * 32), upos_lim = (uint32_t)(g.w_u * 32);
     float acc = 0.f;
 
@@ -119,7 +118,8 @@ __device__ __forceinline__ float chunk_dot_fast(const uint32_t* __restrict__ sb,
     // just used is cleared, so a kept column is x[bpos + 31 - p] and a codeword's rank is the distance between two
     // consecutive terminators.  A window that ran dry gives p = -1; once dry it stays dry, so the sign of the last
     // position of each window tells whether the whole group fitted.
-    auto group = [&](int grp, bool tail) {
+    auto group = [&](int grp, auto tail_c) {
+        constexpr bool tail = decltype(tail_c)::value;         // two specialisations: full groups carry no per-value tests
         const WalkState st0 = {acc, bpos, upos};
         const uint32_t ba = bm_a + (bpos >> 5) * 128u;
         uint32_t bv = __funnelshift_l(lds_u32_off<128>(ba), lds_u32(ba), bpos);    // 32 columns from bpos on
@@ -173,8 +173,8 @@ __device__ __forceinline__ float chunk_dot_fast(const uint32_t* __restrict__ sb,
     };
 
     int grp = 0;
-    for (; grp < n_full; ++grp) group(grp, false);
-    for (; grp < n_groups; ++grp) group(grp, true);
+    for (; grp < n_full; ++grp) group(grp, std::false_type{});
+    for (; grp < n_groups; ++grp) group(grp, std::true_type{});
     return acc;
 }
 
@@ -219,9 +219,9 @@ __global__ void __launch_bounds__(1024) k_draft_gemv(const uint32_t* __restrict_
         const int s = i % kGemvStages;
         const int sb_i = (rb0 + i * rb_step) * n_seg + seg;
         const uint32_t* dir = blob + kBlobDirOffset / 4 + sb_i * 4;
-        const SbGeom g = SbGeom::make((int)dir[3], scols, (int)dir[1], (int)dir[2]);
+        const SbGeom g = SbGeom::make(dir_n_ch(dir[3]), scols, (int)dir[1], (int)dir[2]);
         const uint32_t bytes = (uint32_t)g.total * 4u;
-        if (bytes > (uint32_t)max_sb || (int)dir[3] != n_ch) {               // does not fit: skip the tile, flag it
+        if (bytes > (uint32_t)max_sb || dir_n_ch(dir[3]) != n_ch) {               // does not fit: skip the tile, flag it
             s_skip[s] = 1;
             if (d_status) atomicExch(d_status, CASS_ERR_INVALID_ARG);
             mbar_expect_tx(&bar[s], 0);
@@ -266,9 +266,9 @@ __global__ void __launch_bounds__(1024) k_draft_gemv(const uint32_t* __restrict_
             const uint32_t* dir = blob + kBlobDirOffset / 4 + (rb * n_seg + seg) * 4;
             const SbGeom g = SbGeom::make(n_ch, scols, (int)dir[1], (int)dir[2]);
             if (T >= 0) {
-                acc = chunk_dot_fast<(T >= 0 ? T : 0)>(sb, g, warp, lane, chunk_cols, xs, lut);
+                acc = chunk_dot_fast<(T >= 0 ? T : 0)>(sb, g, warp, lane, dir_chunk_elems(dir[3]), xs, lut);
             } else {
-                decode_chunk_generic(sb, g, chunk_cols, warp, lane, t, cb, [&](int col, uint16_t bits) {
+                decode_chunk_generic(sb, g, dir_chunk_elems(dir[3]), warp, lane, t, cb, [&](int col, uint16_t bits) {
                     acc = fmaf(bf16_bits_to_float(bits), xs[col], acc);
                 });
             }

@@ -122,31 +122,28 @@ __global__ void k_codebook(const unsigned long long* __restrict__ hist, uint8_t*
     exp_to_rank[e] = (uint8_t)rank;
 }
 
-// ---- E4: per (row, segment) sizes: field words (chunks start on word boundaries) and code bits ----------
+// ---- E4: per (row, segment) sizes: kept values and code bits ------------------------------------------------
 __global__ void k_sizes(const uint16_t* __restrict__ W, EncGeom g, const uint32_t* __restrict__ keepbm,
-                        const uint8_t* __restrict__ exp_to_rank, uint32_t* __restrict__ cnt_fw,
+                        const uint8_t* __restrict__ exp_to_rank, uint32_t* __restrict__ cnt_kept,
                         uint32_t* __restrict__ ubits) {
     int gw = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
     if (gw >= g.n_pad * g.n_seg) return;
     int row = gw / g.n_seg, seg = gw % g.n_seg;
-    uint32_t fw = 0, ub = 0;
+    uint32_t kept_n = 0, ub = 0;
     if (row < g.n) {
-        const int per = 32 / (8 - g.t);
-        const int words = g.k_pad / 32, wpc = g.chunk_cols / 32;
+        const int words = g.k_pad / 32;
         int scols = seg_cols_of(g.k_pad, g.seg_cols, seg);
         int w0 = seg * (g.seg_cols / 32), nw = scols / 32;
-        uint32_t in_chunk = 0;
         for (int j = 0; j < nw; ++j) {
             uint32_t bm = keepbm[(size_t)row * words + w0 + j];
             bool kept = (bm >> (31 - lane)) & 1u;
             uint32_t len = 0;
             if (kept) len = exp_to_rank[(W[(size_t)row * g.k + (w0 + j) * 32 + lane] >> 7) & 0xFF] + 1u;
             ub += __reduce_add_sync(0xffffffffu, len);
-            in_chunk += __popc(bm);
-            if ((j + 1) % wpc == 0 || j + 1 == nw) { fw += (in_chunk + per - 1) / per; in_chunk = 0; }
+            kept_n += __popc(bm);
         }
     }
-    if (lane == 0) { cnt_fw[gw] = fw; ubits[gw] = ub; }
+    if (lane == 0) { cnt_kept[gw] = kept_n; ubits[gw] = ub; }
 }
 
 // ---- E5: directory (exclusive scan of superblock sizes) and header -------------------------------------
@@ -164,15 +161,17 @@ __global__ void __launch_bounds__(1024) k_directory(EncGeom g, const uint32_t* _
     for (int base = 0; base < n_sb; base += 1024) {
         int sb = base + tid;
         unsigned long long bytes = 0;
-        uint32_t wf = 0, wu = 0;
+        uint32_t wf = 0, wu = 0, max_kept = 0;
         int n_ch = 0;
         if (sb < n_sb) {
             int rb = sb / g.n_seg, seg = sb % g.n_seg;
+            const uint32_t per = 32u / (8u - (uint32_t)g.t);
             for (int r = 0; r < kRowsPerBlock; ++r) {
                 int row = rb * kRowsPerBlock + r;
-                wf = max(wf, cnt_fw[row * g.n_seg + seg]);
+                max_kept = max(max_kept, cnt_fw[row * g.n_seg + seg]);
                 wu = max(wu, (ubits[row * g.n_seg + seg] + 31u) / 32u);
             }
+            wf = (max_kept + per - 1) / per;
             int scols = seg_cols_of(g.k_pad, g.seg_cols, seg);
             n_ch = ceil_div(scols, g.chunk_cols);
             bytes = (unsigned long long)SbGeom::make(n_ch, scols, (int)wf, (int)wu).total * 4ull;
@@ -191,7 +190,7 @@ __global__ void __launch_bounds__(1024) k_directory(EncGeom g, const uint32_t* _
             dir[sb * 4 + 0] = (uint32_t)(excl / 16);
             dir[sb * 4 + 1] = wf;
             dir[sb * 4 + 2] = wu;
-            dir[sb * 4 + 3] = (uint32_t)n_ch;
+            dir[sb * 4 + 3] = (uint32_t)n_ch | ((uint32_t)chunk_elems_for((int)max_kept, n_ch) << 8);
         }
         __syncthreads();
         if (tid == 1023) s_carry += s_scan[1023];
@@ -224,22 +223,19 @@ __global__ void __launch_bounds__(1024) k_pack(const uint16_t* __restrict__ W, E
     const int tid = threadIdx.x, lane = tid & 31, r = tid >> 5;
     const uint32_t* dir = blob + kBlobDirOffset / 4 + sb * 4;
     const int scols = seg_cols_of(g.k_pad, g.seg_cols, seg);
-    const SbGeom sg = SbGeom::make((int)dir[3], scols, (int)dir[1], (int)dir[2]);
+    const int n_ch = dir_n_ch(dir[3]);
+    const uint32_t E = (uint32_t)dir_chunk_elems(dir[3]);
+    const SbGeom sg = SbGeom::make(n_ch, scols, (int)dir[1], (int)dir[2]);
     uint32_t* body = blob + (size_t)dir[0] * 4;
     for (int i = tid; i < sg.total / 4; i += 1024) reinterpret_cast<uint4*>(body)[i] = make_uint4(0, 0, 0, 0);
     __syncthreads();
 
     const int row = rb * kRowsPerBlock + r;
     const int t = g.t, F = 8 - t, per = 32 / F;
-    const int words = g.k_pad / 32, wpc = g.chunk_cols / 32;
+    const int words = g.k_pad / 32;
     const int w0 = seg * (g.seg_cols / 32);
-    uint32_t fw = 0, ub = 0, k_in_chunk = 0;
+    uint32_t ub = 0, k_base = 0;
     for (int j = 0; j < sg.bm_words; ++j) {
-        if (j % wpc == 0) {
-            fw += (k_in_chunk + per - 1) / per;
-            k_in_chunk = 0;
-            if (lane == 0) body[sg.tab + (j / wpc) * 32 + r] = (fw << 20) | ub;
-        }
         uint32_t bm = row < g.n ? keepbm[(size_t)row * words + w0 + j] : 0u;
         if (lane == 0) body[sg.bm + j * 32 + r] = bm;
         bool kept = (bm >> (31 - lane)) & 1u;
@@ -257,16 +253,21 @@ __global__ void __launch_bounds__(1024) k_pack(const uint16_t* __restrict__ W, E
         }
         if (kept) {
             uint32_t pre = lane ? __popc(bm >> (32 - lane)) : 0u;
-            uint32_t k = k_in_chunk + pre;
-            atomicOr(&body[sg.fl + (fw + k / per) * 32 + r], field_bits_in_word(field, k % per, t));
-            uint32_t pos = ub + incl - 1;
+            uint32_t k = k_base + pre;
+            atomicOr(&body[sg.fl + (k / per) * 32 + r], field_bits_in_word(field, k % per, t));
+            uint32_t pos = ub + incl - 1;                                   // the codeword's terminating one
             atomicOr(&body[sg.un + (pos >> 5) * 32 + r], 0x80000000u >> (pos & 31));
+            if (k % E == 0 && k / E < (uint32_t)n_ch)                       // first value of a chunk: its column and first code bit
+                body[sg.tab + (k / E) * 32 + r] = ((uint32_t)(j * 32 + lane) << 20) | (pos + 1 - len);
         }
         ub += __shfl_sync(0xffffffffu, incl, 31);
-        k_in_chunk += __popc(bm);
+        k_base += __popc(bm);
     }
-    fw += (k_in_chunk + per - 1) / per;
-    if (lane == 0) body[sg.tab + sg.n_ch * 32 + r] = (fw << 20) | ub;
+    // chunks the row has no value for, and the totals
+    for (int c = lane; c <= n_ch; c += 32) {
+        if (c == n_ch) body[sg.tab + c * 32 + r] = (k_base << 20) | ub;
+        else if ((uint32_t)c * E >= k_base) body[sg.tab + c * 32 + r] = ((uint32_t)scols << 20) | ub;
+    }
 }
 
 // ---- test hook: zero-padded reconstruction of the whole blob ---------------------------------------------
@@ -276,13 +277,14 @@ __global__ void k_decode(const uint32_t* __restrict__ blob, uint16_t* __restrict
     const int k_pad = ceil_div(k, 32) * 32;
     const int sb = blockIdx.x, rb = sb / n_seg, seg = sb % n_seg;
     const uint32_t* dir = blob + kBlobDirOffset / 4 + sb * 4;
-    const SbGeom sg = SbGeom::make((int)dir[3], seg_cols_of(k_pad, seg_cols, seg), (int)dir[1], (int)dir[2]);
+    const SbGeom sg = SbGeom::make(dir_n_ch(dir[3]), seg_cols_of(k_pad, seg_cols, seg), (int)dir[1], (int)dir[2]);
+    const int chunk_elems = dir_chunk_elems(dir[3]);
     const uint32_t* body = blob + (size_t)dir[0] * 4;
     const uint8_t* cb = reinterpret_cast<const uint8_t*>(blob) + kBlobHeaderBytes;
     for (int item = threadIdx.x; item < sg.n_ch * 32; item += blockDim.x) {
         int ch = item >> 5, r = item & 31, row = rb * kRowsPerBlock + r;
         if (row >= n) continue;
-        decode_chunk_generic(body, sg, chunk_cols, ch, r, t, cb, [&](int col, uint16_t bits) {
+        decode_chunk_generic(body, sg, chunk_elems, ch, r, t, cb, [&](int col, uint16_t bits) {
             int c = seg * seg_cols + col;
             if (c < k) out[(size_t)row * k + c] = bits;
         });
@@ -296,7 +298,7 @@ __global__ void k_code_bits(const uint32_t* __restrict__ blob, unsigned long lon
     const int k_pad = ceil_div(k, 32) * 32;
     const int sb = blockIdx.x, seg = sb % n_seg;
     const uint32_t* dir = blob + kBlobDirOffset / 4 + sb * 4;
-    const SbGeom sg = SbGeom::make((int)dir[3], seg_cols_of(k_pad, seg_cols, seg), (int)dir[1], (int)dir[2]);
+    const SbGeom sg = SbGeom::make(dir_n_ch(dir[3]), seg_cols_of(k_pad, seg_cols, seg), (int)dir[1], (int)dir[2]);
     const uint32_t* body = blob + (size_t)dir[0] * 4;
     unsigned int bits = body[sg.tab + sg.n_ch * 32 + threadIdx.x] & 0xFFFFFu;       // segment total of row threadIdx.x
     bits = __reduce_add_sync(0xffffffffu, bits);

@@ -29,7 +29,7 @@ struct KvGeom {
     int n_kv, d, max_seq, n_blocks, wpt, bm_words, f_words, kept, n_prune, t, arena_words;
 };
 
-constexpr int kAttnChunk = 256;      // split-K granularity over the sequence (fixed absolute boundaries)
+constexpr int kAttnChunk = 64;       // split-K granularity over the sequence (fixed absolute boundaries)
 
 size_t gemv_smem_bytes(const cass_blob_info& bi);
 // partial: fp32 [n_seg][n_rowblocks*32]; the caller sums the segments (fixed order) afterwards.

@@ -18,7 +18,7 @@ enum BlobHeaderWord {
     H_DIROFF, H_BODYOFF, H_TOTLO, H_TOTHI, H_MAXSB
 };
 constexpr uint32_t kBlobMagic = 0x57534143u;
-constexpr uint32_t kBlobVersion = 2;
+constexpr uint32_t kBlobVersion = 3;
 constexpr int kBlobHeaderBytes = 128;
 constexpr int kBlobCodebookBytes = 256;
 constexpr int kBlobDirOffset = kBlobHeaderBytes + kBlobCodebookBytes;
@@ -45,6 +45,14 @@ struct SbGeom {
     }
 };
 
+__host__ __device__ inline int dir_n_ch(uint32_t w3) { return (int)(w3 & 0xFFu); }
+__host__ __device__ inline int dir_chunk_elems(uint32_t w3) { return (int)(w3 >> 8); }
+__host__ __device__ inline int chunk_elems_for(int max_kept, int n_ch) {       // smallest multiple of 8 with n_ch * E >= max_kept
+    int per_chunk = ceil_div(max_kept, n_ch);
+    int e = ceil_div(per_chunk, 8) * 8;
+    return e < 8 ? 8 : e;
+}
+
 __host__ __device__ inline int seg_cols_of(int k_pad, int seg_cols, int seg) {
     int rest = k_pad - seg * seg_cols;
     return rest < seg_cols ? rest : seg_cols;
@@ -69,31 +77,35 @@ __device__ __forceinline__ int read_unary(const uint32_t* un_row, uint32_t& ub, 
     return rank;
 }
 
-// Generic decoder of one (row, chunk): calls emit(col_in_segment, bf16_bits) for every kept value, in
+// Generic decoder of one (row, chunk): calls emit(col_in_segment, bf16_bits) for every kept value of the chunk, in
 // column order.  `sb` points at the superblock's first word (global or shared memory); `row` in [0,32).
 template <class Emit>
-__device__ inline void decode_chunk_generic(const uint32_t* sb, const SbGeom& g, int chunk_cols, int ch, int row,
+__device__ inline void decode_chunk_generic(const uint32_t* sb, const SbGeom& g, int chunk_elems, int ch, int row,
                                             int t, const uint8_t* rank_to_exp, Emit&& emit) {
     const int per = 32 / (8 - t);
     const uint32_t e0 = sb[g.tab + ch * 32 + row];
-    uint32_t fw = e0 >> 20, ub = e0 & 0xFFFFFu;
+    const int kept = (int)(sb[g.tab + g.n_ch * 32 + row] >> 20);
+    const int k0 = ch * chunk_elems;
+    const int cnt = min(chunk_elems, kept - k0);
+    if (cnt <= 0) return;
+    uint32_t col = e0 >> 20, ub = e0 & 0xFFFFFu;
     const uint32_t* fl_row = sb + g.fl + row;
     const uint32_t* un_row = sb + g.un + row;
     const uint32_t limit = (uint32_t)g.w_u * 32u;
-    const int w0 = ch * (chunk_cols / 32);
-    const int w1 = min(w0 + chunk_cols / 32, g.bm_words);
-    int k = 0;                                       // kept values seen in this chunk
-    for (int w = w0; w < w1; ++w) {
-        uint32_t bm = sb[g.bm + w * 32 + row];
-        while (bm) {
-            int s = __clz(bm);
-            bm &= ~(0x80000000u >> s);
-            uint32_t fword = fl_row[(fw + k / per) * 32];
-            int rank = read_unary(un_row, ub, limit);
-            uint32_t e = rank_to_exp[rank & 255];
-            emit(w * 32 + s, (uint16_t)(field_sign_mant_bf16(fword, k % per, t) | (e << 7)));
-            ++k;
+    const uint32_t col_lim = (uint32_t)g.bm_words * 32u;
+    for (int k = k0; k < k0 + cnt; ++k) {
+        bool found = false;
+        while (col < col_lim) {
+            uint32_t bm = sb[g.bm + (col >> 5) * 32 + row] << (col & 31);
+            if (bm) { col += __clz(bm); found = true; break; }
+            col = (col | 31u) + 1u;
         }
+        if (!found) return;                                   // corrupt stream: stop inside the buffers
+        uint32_t fword = fl_row[(k / per) * 32];
+        int rank = read_unary(un_row, ub, limit);
+        uint32_t e = rank_to_exp[rank & 255];
+        emit((int)col, (uint16_t)(field_sign_mant_bf16(fword, k % per, t) | (e << 7)));
+        col += 1;
     }
 }
 
