@@ -18,6 +18,20 @@
         if (cudaGetLastError() != cudaSuccess) return CASS_ERR_CUDA; \
     } while (0)
 
+// Launch with programmatic stream serialisation: the grid may be scheduled while its predecessor in the stream is
+// still running; every kernel launched this way calls pdl_wait() before it touches global memory, which returns
+// once the predecessor has completed and its writes are visible.
+#define CASS_PDL_LAUNCH(kernel_, grid_, block_, smem_, stream_, ...)                                              \
+    do {                                                                                                    \
+        cudaLaunchConfig_t _cfg = {};                                                                       \
+        _cfg.gridDim = (grid_); _cfg.blockDim = (block_); _cfg.dynamicSmemBytes = (smem_); _cfg.stream = (stream_); \
+        cudaLaunchAttribute _at[1];                                                                         \
+        _at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;                                     \
+        _at[0].val.programmaticStreamSerializationAllowed = 1;                                              \
+        _cfg.attrs = _at; _cfg.numAttrs = 1;                                                                \
+        if (cudaLaunchKernelEx(&_cfg, kernel_, __VA_ARGS__) != cudaSuccess) return CASS_ERR_CUDA;            \
+    } while (0)
+
 namespace cass {
 
 constexpr int kRowsPerBlock = 32;          // rows (or tokens) interleaved in one superblock

@@ -185,6 +185,8 @@ __global__ void __launch_bounds__(kDaThreads) k_draft_attn(KvGeom g, KvComp ck, 
                                                            int n_q, const DevState* __restrict__ st, AttnScratch sc,
                                                            int n_chunks_alloc) {
     extern __shared__ __align__(16) uint8_t smem[];
+    pdl_launch_dependents();
+    pdl_wait();
     const int chunk = blockIdx.x, head = blockIdx.y;
     const int cur_len = st->len + st->inflight + 1;            // positions visible to the drafted token
     const int t0 = chunk * kDaTok;
@@ -305,6 +307,7 @@ __global__ void __launch_bounds__(128) k_attn_merge(AttnScratch sc, int n_chunks
     extern __shared__ float w_s[];                  // [n_chunks_alloc] weights e^{m_c - M}
     __shared__ float s_red[4];
     pdl_launch_dependents();
+    pdl_wait();
     const int hq = blockIdx.x, r = blockIdx.y;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int vis = st->len + (draft_mode ? st->inflight + 1 : r + 1);
@@ -347,8 +350,7 @@ int launch_attn_merge(const AttnScratch& sc, int n_chunks_alloc, int chunk_token
         CASS_CUDA_CHECK(cudaFuncSetAttribute(k_attn_merge, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         attr = smem;
     }
-    k_attn_merge<<<grid, 128, smem, s>>>(sc, n_chunks_alloc, chunk_tokens, n_q, d, st, draft_mode, out);
-    CASS_LAUNCH_CHECK();
+    CASS_PDL_LAUNCH(k_attn_merge, grid, dim3(128), smem, s, sc, n_chunks_alloc, chunk_tokens, n_q, d, st, draft_mode, out);
     return CASS_OK;
 }
 
@@ -371,7 +373,7 @@ int launch_draft_attn(const KvGeom& g, const KvComp& ck, const KvComp& cv, const
             CASS_CUDA_CHECK(cudaFuncSetAttribute(k_draft_attn<TT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
             attr = smem;                                                                                             \
         }                                                                                                            \
-        k_draft_attn<TT><<<grid, kDaThreads, smem, s>>>(g, ck, cv, qkv, n_q, st, sc, n_chunks);                      \
+        CASS_PDL_LAUNCH(k_draft_attn<TT>, grid, dim3(kDaThreads), smem, s, g, ck, cv, qkv, n_q, st, sc, n_chunks);     \
     } while (0)
     if (g.t == 4) CASS_DA_LAUNCH(4);
     else if (g.t == 0) CASS_DA_LAUNCH(0);

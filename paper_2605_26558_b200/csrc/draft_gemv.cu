@@ -291,6 +291,7 @@ __global__ void __launch_bounds__(1024) k_draft_gemv(const uint32_t* __restrict_
 
 __global__ void k_gemv_finish(const float* __restrict__ partial, int n, int n_pad, int n_seg,
                               uint16_t* __restrict__ y_bf16, float* __restrict__ y_f32) {
+    pdl_wait();
     int r = blockIdx.x * blockDim.x + threadIdx.x;
     if (r >= n) return;
     float acc = 0.f;

@@ -79,6 +79,8 @@ __global__ void __launch_bounds__(256) k_kv_append(KvGeom g, KvComp ck, KvComp c
     __shared__ uint32_t s_fix[kKvWarps][kKvFixMax];          // bitmap (<= 8) + field words (<= 64)
     __shared__ uint32_t s_una[kKvWarps][kKvStageWords];
     __shared__ uint32_t s_nw[kKvWarps], s_off[kKvWarps];
+    pdl_launch_dependents();
+    pdl_wait();
     const int head = blockIdx.x, kind = blockIdx.y;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const KvComp c = kind ? cv : ck;
@@ -179,9 +181,8 @@ int launch_kv_append(const KvGeom& g, const KvComp& ck, const KvComp& cv, uint16
                      int n_new, int flags, DevState* st, cudaStream_t s) {
     if (n_new <= 0) return CASS_OK;
     dim3 grid(g.n_kv, 2);
-    k_kv_append<<<grid, 256, 0, s>>>(g, ck, cv, k_cache, v_cache, src_k, src_v, row_stride, start_pos, use_inflight,
-                                     n_new, flags, st);
-    CASS_LAUNCH_CHECK();
+    CASS_PDL_LAUNCH(k_kv_append, grid, dim3(256), 0, s, g, ck, cv, k_cache, v_cache, src_k, src_v, row_stride, start_pos,
+                    use_inflight, n_new, flags, st);
     return CASS_OK;
 }
 

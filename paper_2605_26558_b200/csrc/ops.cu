@@ -17,6 +17,8 @@ __global__ void k_rope_table(float* __restrict__ cos_t, float* __restrict__ sin_
 
 __global__ void k_embed(const int32_t* __restrict__ toks, const uint16_t* __restrict__ embed, uint16_t* __restrict__ h,
                         int hidden) {
+    pdl_launch_dependents();
+    pdl_wait();
     int r = blockIdx.x;
     const uint16_t* src = embed + (size_t)toks[r] * hidden;
     for (int i = threadIdx.x; i < hidden; i += blockDim.x) h[(size_t)r * hidden + i] = src[i];
@@ -43,6 +45,7 @@ __global__ void __launch_bounds__(1024) k_residual_rmsnorm(uint16_t* __restrict_
                                                            int hidden, float eps) {
     __shared__ float s_red[32];
     pdl_launch_dependents();            // a following draft GEMV may start fetching its weights now
+    pdl_wait();
     const int r = blockIdx.x;
     uint16_t* hr = h + (size_t)r * hidden;
     float vals[kNormMaxIter][4];
@@ -105,6 +108,8 @@ __global__ void __launch_bounds__(1024) k_residual_rmsnorm(uint16_t* __restrict_
 __global__ void k_qkv_rope(uint16_t* __restrict__ qkv, const float* __restrict__ partial, int n_seg, int n_pad,
                            const float* __restrict__ cos_t, const float* __restrict__ sin_t,
                            const DevState* __restrict__ st, int use_inflight, int n_q, int n_kv, int d) {
+    pdl_launch_dependents();
+    pdl_wait();
     const int r = blockIdx.y, half = d / 2;
     const int qkv_dim = (n_q + 2 * n_kv) * d;
     const int pos = st->len + (use_inflight ? st->inflight : 0) + r;
@@ -137,6 +142,7 @@ __global__ void k_qkv_rope(uint16_t* __restrict__ qkv, const float* __restrict__
 __global__ void k_swiglu(const uint16_t* __restrict__ gu, const float* __restrict__ partial, int n_seg, int n_pad,
                          uint16_t* __restrict__ act, int ffn) {
     pdl_launch_dependents();
+    pdl_wait();
     const int r = blockIdx.y;
     for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < ffn; i += gridDim.x * blockDim.x) {
         float g, u;
@@ -169,6 +175,8 @@ __global__ void __launch_bounds__(256) k_argmax_part(const float* __restrict__ l
                                                      int32_t* __restrict__ tmp_i, float* __restrict__ logits_copy) {
     __shared__ float s_v[8];
     __shared__ int s_i[8];
+    pdl_launch_dependents();
+    pdl_wait();
     const int r = blockIdx.y, nsl = gridDim.x;
     const int per = ceil_div(vocab, nsl);
     const int lo = blockIdx.x * per, hi = min(vocab, lo + per);
@@ -204,6 +212,8 @@ __global__ void __launch_bounds__(kArgmaxSlices) k_argmax_final(const float* __r
                                                                 int nsl, int32_t* __restrict__ out, DevState* st, int bump_inflight) {
     __shared__ float s_v[kArgmaxSlices / 32];
     __shared__ int s_i[kArgmaxSlices / 32];
+    pdl_launch_dependents();
+    pdl_wait();
     const int r = blockIdx.x;
     float best = -INFINITY;
     int best_i = 0x7fffffff;
@@ -226,6 +236,8 @@ __global__ void __launch_bounds__(kArgmaxSlices) k_argmax_final(const float* __r
 // Greedy acceptance: a = min({i-1 : draft_i != target_{i-1}} U {g}); emit draft_1..draft_a and target_a.
 __global__ void k_accept(DevState* st, const int32_t* __restrict__ draft, const int32_t* __restrict__ target, int g,
                          int32_t* n_acc, int32_t* out_tokens, int32_t* next_tok) {
+    pdl_launch_dependents();
+    pdl_wait();
     if (threadIdx.x != 0 || blockIdx.x != 0) return;
     int a = 0;
     while (a < g && draft[a] == target[a]) ++a;
@@ -240,6 +252,8 @@ __global__ void k_accept(DevState* st, const int32_t* __restrict__ draft, const 
 
 __global__ void k_calib_accum(const uint16_t* __restrict__ x, int rows, int cols, float* __restrict__ sumsq,
                               const DevState* __restrict__ st) {
+    pdl_launch_dependents();
+    pdl_wait();
     if (!st->calib_on) return;
     int c = blockIdx.x * blockDim.x + threadIdx.x;
     if (c >= cols) return;
@@ -264,8 +278,7 @@ int launch_rope_table(float* cos_t, float* sin_t, int max_seq, int d, float thet
 }
 
 int launch_embed(const int32_t* toks, const uint16_t* embed, uint16_t* h, int rows, int hidden, cudaStream_t s) {
-    k_embed<<<rows, 256, 0, s>>>(toks, embed, h, hidden);
-    CASS_LAUNCH_CHECK();
+    CASS_PDL_LAUNCH(k_embed, dim3(rows), dim3(256), 0, s, toks, embed, h, hidden);
     return CASS_OK;
 }
 
@@ -276,8 +289,8 @@ static int norm_threads(int hidden) {
 
 int launch_rmsnorm(const uint16_t* h, const uint16_t* gain, uint16_t* out, int rows, int hidden, float eps, cudaStream_t s) {
     if (hidden % 4 || hidden > kNormMaxIter * 4 * 1024) return CASS_ERR_UNSUPPORTED;
-    k_residual_rmsnorm<<<rows, norm_threads(hidden), 0, s>>>(const_cast<uint16_t*>(h), nullptr, nullptr, 0, 0, gain, out, hidden, eps);
-    CASS_LAUNCH_CHECK();
+    CASS_PDL_LAUNCH(k_residual_rmsnorm, dim3(rows), dim3(norm_threads(hidden)), 0, s, const_cast<uint16_t*>(h), (const uint16_t*)nullptr,
+                    (const float*)nullptr, 0, 0, gain, out, hidden, eps);
     return CASS_OK;
 }
 
@@ -285,8 +298,7 @@ int launch_residual_rmsnorm(uint16_t* h, const uint16_t* y_bf16, const float* pa
                             const uint16_t* gain, uint16_t* out, int rows, int hidden, float eps, cudaStream_t s) {
     if (partial && rows != 1) return CASS_ERR_INVALID_ARG;
     if (hidden % 4 || hidden > kNormMaxIter * 4 * 1024) return CASS_ERR_UNSUPPORTED;
-    k_residual_rmsnorm<<<rows, norm_threads(hidden), 0, s>>>(h, y_bf16, partial, n_seg, n_pad, gain, out, hidden, eps);
-    CASS_LAUNCH_CHECK();
+    CASS_PDL_LAUNCH(k_residual_rmsnorm, dim3(rows), dim3(norm_threads(hidden)), 0, s, h, y_bf16, partial, n_seg, n_pad, gain, out, hidden, eps);
     return CASS_OK;
 }
 
@@ -295,8 +307,7 @@ int launch_qkv_rope(uint16_t* qkv, const float* partial, int n_seg, int n_pad, c
     if (partial && rows != 1) return CASS_ERR_INVALID_ARG;
     int items = (n_q + n_kv) * (d / 2) + n_kv * d;
     dim3 grid(ceil_div(items, 256), rows);
-    k_qkv_rope<<<grid, 256, 0, s>>>(qkv, partial, n_seg, n_pad, cos_t, sin_t, st, use_inflight, n_q, n_kv, d);
-    CASS_LAUNCH_CHECK();
+    CASS_PDL_LAUNCH(k_qkv_rope, grid, dim3(256), 0, s, qkv, partial, n_seg, n_pad, cos_t, sin_t, st, use_inflight, n_q, n_kv, d);
     return CASS_OK;
 }
 
@@ -304,8 +315,7 @@ int launch_swiglu(const uint16_t* gu_bf16, const float* partial, int n_seg, int 
                   cudaStream_t s) {
     if (partial && rows != 1) return CASS_ERR_INVALID_ARG;
     dim3 grid(ceil_div(ffn, 256), rows);
-    k_swiglu<<<grid, 256, 0, s>>>(gu_bf16, partial, n_seg, n_pad, act, ffn);
-    CASS_LAUNCH_CHECK();
+    CASS_PDL_LAUNCH(k_swiglu, grid, dim3(256), 0, s, gu_bf16, partial, n_seg, n_pad, act, ffn);
     return CASS_OK;
 }
 
@@ -315,23 +325,19 @@ int launch_argmax(const float* logits, const float* partial, int n_seg, int n_pa
     int nsl = ceil_div(vocab, 1024);
     if (nsl > kArgmaxSlices) nsl = kArgmaxSlices;
     dim3 grid(nsl, rows);
-    k_argmax_part<<<grid, 256, 0, s>>>(logits, partial, n_seg, n_pad, vocab, tmp_v, tmp_i, logits_copy);
-    CASS_LAUNCH_CHECK();
-    k_argmax_final<<<rows, kArgmaxSlices, 0, s>>>(tmp_v, tmp_i, nsl, out, st, bump_inflight);
-    CASS_LAUNCH_CHECK();
+    CASS_PDL_LAUNCH(k_argmax_part, grid, dim3(256), 0, s, logits, partial, n_seg, n_pad, vocab, tmp_v, tmp_i, logits_copy);
+    CASS_PDL_LAUNCH(k_argmax_final, dim3(rows), dim3(kArgmaxSlices), 0, s, (const float*)tmp_v, (const int32_t*)tmp_i, nsl, out, st, bump_inflight);
     return CASS_OK;
 }
 
 int launch_accept(DevState* st, const int32_t* draft, const int32_t* target, int g, int32_t* n_acc, int32_t* out_tokens,
                   int32_t* next_tok, cudaStream_t s) {
-    k_accept<<<1, 32, 0, s>>>(st, draft, target, g, n_acc, out_tokens, next_tok);
-    CASS_LAUNCH_CHECK();
+    CASS_PDL_LAUNCH(k_accept, dim3(1), dim3(32), 0, s, st, draft, target, g, n_acc, out_tokens, next_tok);
     return CASS_OK;
 }
 
 int launch_calib_accum(const uint16_t* x, int rows, int cols, float* sumsq, const DevState* st, cudaStream_t s) {
-    k_calib_accum<<<ceil_div(cols, 256), 256, 0, s>>>(x, rows, cols, sumsq, st);
-    CASS_LAUNCH_CHECK();
+    CASS_PDL_LAUNCH(k_calib_accum, dim3(ceil_div(cols, 256)), dim3(256), 0, s, x, rows, cols, sumsq, st);
     return CASS_OK;
 }
 

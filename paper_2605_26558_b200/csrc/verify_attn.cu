@@ -18,6 +18,8 @@ __global__ void __launch_bounds__(kVaThreads) k_verify_attn(KvGeom g, const uint
                                                             int rows, int n_q, const DevState* __restrict__ st, AttnScratch sc,
                                                             int n_chunks_alloc) {
     extern __shared__ __align__(16) uint8_t smem[];
+    pdl_launch_dependents();
+    pdl_wait();
     const int chunk = blockIdx.x, head = blockIdx.y;
     const int len = st->len;
     const int t0 = chunk * kAttnChunk;
@@ -140,8 +142,7 @@ int launch_verify_attn(const KvGeom& g, const uint16_t* k_cache, const uint16_t*
         attr = smem;
     }
     dim3 grid(n_chunks, g.n_kv);
-    k_verify_attn<<<grid, kVaThreads, smem, s>>>(g, k_cache, v_cache, qkv, rows, n_q, st, sc, n_chunks);
-    CASS_LAUNCH_CHECK();
+    CASS_PDL_LAUNCH(k_verify_attn, grid, dim3(kVaThreads), smem, s, g, k_cache, v_cache, qkv, rows, n_q, st, sc, n_chunks);
     return launch_attn_merge(sc, n_chunks, kAttnChunk, rows, n_q, g.d, st, 0, out, s);
 }
 

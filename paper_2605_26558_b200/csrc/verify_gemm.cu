@@ -122,6 +122,9 @@ __global__ void __launch_bounds__(kTcThreads) k_verify_gemm_tc(const __grid_cons
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+    // barriers and tensor memory are set up; the activations and the scratch belong to the preceding kernels
+    pdl_launch_dependents();
+    pdl_wait();
 
     if (warp == 0 && lane == 0) {
         // ---- producer: TMA loads into the ring ----
@@ -181,6 +184,8 @@ __global__ void __launch_bounds__(kTcThreads) k_verify_gemm_tc(const __grid_cons
 
 __global__ void k_verify_gemm_finish(const float* __restrict__ partial, int rows, int n, int n_split,
                                      uint16_t* __restrict__ y_bf16, float* __restrict__ y_f32) {
+    pdl_launch_dependents();
+    pdl_wait();
     const int j = blockIdx.x * blockDim.x + threadIdx.x, r = blockIdx.y;
     if (j >= n || r >= rows) return;
     float acc = 0.f;
@@ -224,11 +229,9 @@ int launch_verify_gemm(const uint16_t* W, const uint16_t* X, int rows, int n, in
         attr = true;
     }
     dim3 grid(ceil_div(n, kTcBM), ns);
-    k_verify_gemm_tc<<<grid, kTcThreads, kTcSmem, s>>>(mw, mx, partial, rows, n, kbt, kbs, d_status);
-    CASS_LAUNCH_CHECK();
+    CASS_PDL_LAUNCH(k_verify_gemm_tc, grid, dim3(kTcThreads), (size_t)kTcSmem, s, mw, mx, partial, rows, n, kbt, kbs, d_status);
     dim3 g2(ceil_div(n, 256), rows);
-    k_verify_gemm_finish<<<g2, 256, 0, s>>>(partial, rows, n, ns, y_bf16, y_f32);
-    CASS_LAUNCH_CHECK();
+    CASS_PDL_LAUNCH(k_verify_gemm_finish, g2, dim3(256), 0, s, (const float*)partial, rows, n, ns, y_bf16, y_f32);
     return CASS_OK;
 }
 
