@@ -29,6 +29,14 @@ struct KvGeom {
     int n_kv, d, max_seq, n_blocks, wpt, bm_words, f_words, kept, n_prune, t, arena_words;
 };
 
+// fp32 split-K partial sums of a projection: element (row r, feature i) of part s sits at p[s * seg_stride + r * row_stride + i];
+// consumers add the parts in order and round to bf16 where the projection output is a bf16 activation.
+struct Partials {
+    const float* p;
+    int n_seg;
+    size_t seg_stride, row_stride;
+};
+
 constexpr int kAttnChunk = 64;       // split-K granularity over the sequence (fixed absolute boundaries)
 
 size_t gemv_smem_bytes(const cass_blob_info& bi);
@@ -43,18 +51,18 @@ int launch_rmsnorm(const uint16_t* h, const uint16_t* gain, uint16_t* out, int r
                    cudaStream_t s);
 // h = bf16(h + y); out = rmsnorm(h) * gain.  y comes either as bf16 [rows][hidden] or (rows == 1) as fp32 split-K
 // partials [n_seg][n_pad] that are summed in segment order and rounded to bf16 first.
-int launch_residual_rmsnorm(uint16_t* h, const uint16_t* y_bf16, const float* partial, int n_seg, int n_pad,
+int launch_residual_rmsnorm(uint16_t* h, const uint16_t* y_bf16, Partials pp,
                             const uint16_t* gain, uint16_t* out, int rows, int hidden, float eps, cudaStream_t s);
 // q and k of qkv (bf16 [rows][qkv_dim]) rotated in place at position base + row (base from state: len, or
 // len + inflight when use_inflight).  With partial != NULL (rows == 1) qkv is first formed from the partials.
-int launch_qkv_rope(uint16_t* qkv, const float* partial, int n_seg, int n_pad, const float* cos_t, const float* sin_t,
+int launch_qkv_rope(uint16_t* qkv, Partials pp, const float* cos_t, const float* sin_t,
                     const DevState* st, int use_inflight, int rows, int n_q, int n_kv, int d, cudaStream_t s);
-int launch_swiglu(const uint16_t* gu_bf16, const float* partial, int n_seg, int n_pad, uint16_t* act, int rows,
+int launch_swiglu(const uint16_t* gu_bf16, Partials pp, uint16_t* act, int rows,
                   int ffn, cudaStream_t s);
 // logits (fp32 [rows][vocab], or formed from partials when rows == 1) -> lowest-index argmax per row; optional copy
 // of the logits; bump_inflight adds 1 to the draft counter afterwards.
 // tmp_v / tmp_i: scratch of 16 x 128 entries each.
-int launch_argmax(const float* logits, const float* partial, int n_seg, int n_pad, int rows, int vocab, int32_t* out,
+int launch_argmax(const float* logits, Partials pp, int rows, int vocab, int32_t* out,
                   float* logits_copy, float* tmp_v, int32_t* tmp_i, DevState* st, int bump_inflight, cudaStream_t s);
 int launch_accept(DevState* st, const int32_t* draft, const int32_t* target, int g, int32_t* n_acc,
                   int32_t* out_tokens, int32_t* next_tok, cudaStream_t s);
@@ -85,7 +93,9 @@ int launch_verify_attn(const KvGeom& g, const uint16_t* k_cache, const uint16_t*
 
 // ---- verification GEMM (verify_gemm.cu): Y[r][n] = sum_k W[n][k] X[r][k], bf16 in, fp32 accumulate (tcgen05) ----
 // X is a buffer of 16 rows of k values (the first `rows` are used); partial: fp32 scratch of verify_gemm_partial_floats.
+// With both outputs null only the partial sums are produced: [splits][16][n], see verify_gemm_partials().
 size_t verify_gemm_partial_floats(int n, int k);
+Partials verify_gemm_partials(const float* partial, int n, int k);
 int launch_verify_gemm(const uint16_t* W, const uint16_t* X, int rows, int n, int k, float* partial, uint16_t* y_bf16,
                        float* y_f32, int32_t* d_status, cudaStream_t s);
 

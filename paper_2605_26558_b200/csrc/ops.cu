@@ -40,7 +40,7 @@ __device__ __forceinline__ float block_sum(float v, float* s_red) {
 constexpr int kNormMaxIter = 8;          // hidden <= 8 * 4 * blockDim.x
 
 __global__ void __launch_bounds__(1024) k_residual_rmsnorm(uint16_t* __restrict__ h, const uint16_t* __restrict__ y_bf16,
-                                                           const float* __restrict__ partial, int n_seg, int n_pad,
+                                                           Partials pp,
                                                            const uint16_t* __restrict__ gain, uint16_t* __restrict__ out,
                                                            int hidden, float eps) {
     __shared__ float s_red[32];
@@ -58,12 +58,12 @@ __global__ void __launch_bounds__(1024) k_residual_rmsnorm(uint16_t* __restrict_
             const uint2 hv = *reinterpret_cast<const uint2*>(hr + i);
             float v[4] = {__uint_as_float(hv.x << 16), __uint_as_float(hv.x & 0xFFFF0000u), __uint_as_float(hv.y << 16),
                           __uint_as_float(hv.y & 0xFFFF0000u)};
-            if (y_bf16 || partial) {
+            if (y_bf16 || pp.p) {
                 float y[4];
-                if (partial) {
+                if (pp.p) {
                     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-                    for (int s = 0; s < n_seg; ++s) {
-                        const float4 p = *reinterpret_cast<const float4*>(partial + (size_t)s * n_pad + i);
+                    for (int s = 0; s < pp.n_seg; ++s) {
+                        const float4 p = *reinterpret_cast<const float4*>(pp.p + (size_t)s * pp.seg_stride + (size_t)r * pp.row_stride + i);
                         acc.x += p.x; acc.y += p.y; acc.z += p.z; acc.w += p.w;
                     }
                     y[0] = round_bf16(acc.x); y[1] = round_bf16(acc.y); y[2] = round_bf16(acc.z); y[3] = round_bf16(acc.w);
@@ -105,7 +105,7 @@ __global__ void __launch_bounds__(1024) k_residual_rmsnorm(uint16_t* __restrict_
     }
 }
 
-__global__ void k_qkv_rope(uint16_t* __restrict__ qkv, const float* __restrict__ partial, int n_seg, int n_pad,
+__global__ void k_qkv_rope(uint16_t* __restrict__ qkv, Partials pp,
                            const float* __restrict__ cos_t, const float* __restrict__ sin_t,
                            const DevState* __restrict__ st, int use_inflight, int n_q, int n_kv, int d) {
     pdl_launch_dependents();
@@ -117,9 +117,9 @@ __global__ void k_qkv_rope(uint16_t* __restrict__ qkv, const float* __restrict__
     const int n_rot = (n_q + n_kv) * half;             // rotated pairs
     const int n_items = n_rot + n_kv * d;              // + plain v elements
     auto load = [&](int i) -> float {
-        if (partial) {
+        if (pp.p) {
             float acc = 0.f;
-            for (int s = 0; s < n_seg; ++s) acc += partial[(size_t)s * n_pad + i];
+            for (int s = 0; s < pp.n_seg; ++s) acc += pp.p[(size_t)s * pp.seg_stride + (size_t)r * pp.row_stride + i];
             return round_bf16(acc);
         }
         return bf16_bits_to_float(row[i]);
@@ -132,25 +132,26 @@ __global__ void k_qkv_rope(uint16_t* __restrict__ qkv, const float* __restrict__
             float c = cos_t[(size_t)pos * half + j], s = sin_t[(size_t)pos * half + j];
             row[ia] = float_to_bf16_bits(a * c - b * s);
             row[ib] = float_to_bf16_bits(b * c + a * s);
-        } else if (partial) {
+        } else if (pp.p) {
             int i = (n_q + n_kv) * d + (it - n_rot);
             row[i] = float_to_bf16_bits(load(i));
         }
     }
 }
 
-__global__ void k_swiglu(const uint16_t* __restrict__ gu, const float* __restrict__ partial, int n_seg, int n_pad,
+__global__ void k_swiglu(const uint16_t* __restrict__ gu, Partials pp,
                          uint16_t* __restrict__ act, int ffn) {
     pdl_launch_dependents();
     pdl_wait();
     const int r = blockIdx.y;
     for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < ffn; i += gridDim.x * blockDim.x) {
         float g, u;
-        if (partial) {
+        if (pp.p) {
             float ag = 0.f, au = 0.f;
-            for (int s = 0; s < n_seg; ++s) {
-                ag += partial[(size_t)s * n_pad + i];
-                au += partial[(size_t)s * n_pad + ffn + i];
+            for (int s = 0; s < pp.n_seg; ++s) {
+                const float* q = pp.p + (size_t)s * pp.seg_stride + (size_t)r * pp.row_stride;
+                ag += q[i];
+                au += q[ffn + i];
             }
             g = round_bf16(ag);
             u = round_bf16(au);
@@ -170,8 +171,7 @@ __device__ __forceinline__ void argmax_combine(float& best, int& best_i, float o
     if (ov > best || (ov == best && oi < best_i)) { best = ov; best_i = oi; }
 }
 
-__global__ void __launch_bounds__(256) k_argmax_part(const float* __restrict__ logits, const float* __restrict__ partial,
-                                                     int n_seg, int n_pad, int vocab, float* __restrict__ tmp_v,
+__global__ void __launch_bounds__(256) k_argmax_part(const float* __restrict__ logits, Partials pp, int vocab, float* __restrict__ tmp_v,
                                                      int32_t* __restrict__ tmp_i, float* __restrict__ logits_copy) {
     __shared__ float s_v[8];
     __shared__ int s_i[8];
@@ -184,9 +184,9 @@ __global__ void __launch_bounds__(256) k_argmax_part(const float* __restrict__ l
     int best_i = 0x7fffffff;
     for (int i = lo + threadIdx.x; i < hi; i += blockDim.x) {
         float v;
-        if (partial) {
+        if (pp.p) {
             v = 0.f;
-            for (int s = 0; s < n_seg; ++s) v += partial[(size_t)s * n_pad + i];
+            for (int s = 0; s < pp.n_seg; ++s) v += pp.p[(size_t)s * pp.seg_stride + (size_t)r * pp.row_stride + i];
         } else {
             v = logits[(size_t)r * vocab + i];
         }
@@ -290,42 +290,38 @@ static int norm_threads(int hidden) {
 int launch_rmsnorm(const uint16_t* h, const uint16_t* gain, uint16_t* out, int rows, int hidden, float eps, cudaStream_t s) {
     if (hidden % 4 || hidden > kNormMaxIter * 4 * 1024) return CASS_ERR_UNSUPPORTED;
     CASS_PDL_LAUNCH(k_residual_rmsnorm, dim3(rows), dim3(norm_threads(hidden)), 0, s, const_cast<uint16_t*>(h), (const uint16_t*)nullptr,
-                    (const float*)nullptr, 0, 0, gain, out, hidden, eps);
+                    Partials{nullptr, 0, 0, 0}, gain, out, hidden, eps);
     return CASS_OK;
 }
 
-int launch_residual_rmsnorm(uint16_t* h, const uint16_t* y_bf16, const float* partial, int n_seg, int n_pad,
+int launch_residual_rmsnorm(uint16_t* h, const uint16_t* y_bf16, Partials pp,
                             const uint16_t* gain, uint16_t* out, int rows, int hidden, float eps, cudaStream_t s) {
-    if (partial && rows != 1) return CASS_ERR_INVALID_ARG;
     if (hidden % 4 || hidden > kNormMaxIter * 4 * 1024) return CASS_ERR_UNSUPPORTED;
-    CASS_PDL_LAUNCH(k_residual_rmsnorm, dim3(rows), dim3(norm_threads(hidden)), 0, s, h, y_bf16, partial, n_seg, n_pad, gain, out, hidden, eps);
+    CASS_PDL_LAUNCH(k_residual_rmsnorm, dim3(rows), dim3(norm_threads(hidden)), 0, s, h, y_bf16, pp, gain, out, hidden, eps);
     return CASS_OK;
 }
 
-int launch_qkv_rope(uint16_t* qkv, const float* partial, int n_seg, int n_pad, const float* cos_t, const float* sin_t,
+int launch_qkv_rope(uint16_t* qkv, Partials pp, const float* cos_t, const float* sin_t,
                     const DevState* st, int use_inflight, int rows, int n_q, int n_kv, int d, cudaStream_t s) {
-    if (partial && rows != 1) return CASS_ERR_INVALID_ARG;
     int items = (n_q + n_kv) * (d / 2) + n_kv * d;
     dim3 grid(ceil_div(items, 256), rows);
-    CASS_PDL_LAUNCH(k_qkv_rope, grid, dim3(256), 0, s, qkv, partial, n_seg, n_pad, cos_t, sin_t, st, use_inflight, n_q, n_kv, d);
+    CASS_PDL_LAUNCH(k_qkv_rope, grid, dim3(256), 0, s, qkv, pp, cos_t, sin_t, st, use_inflight, n_q, n_kv, d);
     return CASS_OK;
 }
 
-int launch_swiglu(const uint16_t* gu_bf16, const float* partial, int n_seg, int n_pad, uint16_t* act, int rows, int ffn,
+int launch_swiglu(const uint16_t* gu_bf16, Partials pp, uint16_t* act, int rows, int ffn,
                   cudaStream_t s) {
-    if (partial && rows != 1) return CASS_ERR_INVALID_ARG;
     dim3 grid(ceil_div(ffn, 256), rows);
-    CASS_PDL_LAUNCH(k_swiglu, grid, dim3(256), 0, s, gu_bf16, partial, n_seg, n_pad, act, ffn);
+    CASS_PDL_LAUNCH(k_swiglu, grid, dim3(256), 0, s, gu_bf16, pp, act, ffn);
     return CASS_OK;
 }
 
-int launch_argmax(const float* logits, const float* partial, int n_seg, int n_pad, int rows, int vocab, int32_t* out,
+int launch_argmax(const float* logits, Partials pp, int rows, int vocab, int32_t* out,
                   float* logits_copy, float* tmp_v, int32_t* tmp_i, DevState* st, int bump_inflight, cudaStream_t s) {
-    if (partial && rows != 1) return CASS_ERR_INVALID_ARG;
     int nsl = ceil_div(vocab, 1024);
     if (nsl > kArgmaxSlices) nsl = kArgmaxSlices;
     dim3 grid(nsl, rows);
-    CASS_PDL_LAUNCH(k_argmax_part, grid, dim3(256), 0, s, logits, partial, n_seg, n_pad, vocab, tmp_v, tmp_i, logits_copy);
+    CASS_PDL_LAUNCH(k_argmax_part, grid, dim3(256), 0, s, logits, pp, vocab, tmp_v, tmp_i, logits_copy);
     CASS_PDL_LAUNCH(k_argmax_final, dim3(rows), dim3(kArgmaxSlices), 0, s, (const float*)tmp_v, (const int32_t*)tmp_i, nsl, out, st, bump_inflight);
     return CASS_OK;
 }

@@ -39,7 +39,7 @@ struct Session {
     AttnScratch asc;
     int32_t* argmax_tmp;
     float* argmax_val;
-    bool have_blobs, codebooks_ready;
+    bool have_blobs, codebooks_ready, calib_host;
     int qkv_dim, kmax;
 };
 
@@ -267,6 +267,7 @@ extern "C" int cass_calib_enable(void* session, int on, void* stream_) {
     int32_t v = on ? 1 : 0;
     CASS_CUDA_CHECK(cudaMemcpyAsync(&s->st->calib_on, &v, 4, cudaMemcpyHostToDevice, (cudaStream_t)stream_));
     CASS_CUDA_CHECK(cudaStreamSynchronize((cudaStream_t)stream_));
+    s->calib_host = on != 0;
     return CASS_OK;
 }
 
@@ -374,28 +375,35 @@ extern "C" int cass_verify(void* session, const int32_t* toks, int g, int32_t* t
     RC(launch_embed(toks, (const uint16_t*)s->embed, s->h, rows, d.hidden, st));
     RC(launch_rmsnorm(s->h, (const uint16_t*)s->layers[0].w.norm_attn, s->xn, rows, d.hidden, d.rms_eps, st));
     const int kv_flags = CASS_KV_BF16 | (s->codebooks_ready ? CASS_KV_COMPRESSED : 0);
+    const bool calib = s->calib_host;           // the accumulation kernels are only launched while calibration is on
+    int32_t* status = &s->st->status;
+    // every projection leaves fp32 split-K parts in vg_partial; the kernel that consumes the projection adds them
     for (int l = 0; l < d.n_layers; ++l) {
         LayerDev& L = s->layers[l];
-        RC(launch_calib_accum(s->xn, rows, d.hidden, L.calib[0], s->st, st));
-        RC(launch_verify_gemm((const uint16_t*)L.w.wqkv, s->xn, rows, s->qkv_dim, d.hidden, s->vg_partial, s->qkv, nullptr, &s->st->status, st));
-        RC(launch_qkv_rope(s->qkv, nullptr, 0, 0, s->cos_t, s->sin_t, s->st, 0, rows, d.n_q_heads, d.n_kv_heads, d.head_dim, st));
+        if (calib) RC(launch_calib_accum(s->xn, rows, d.hidden, L.calib[0], s->st, st));
+        RC(launch_verify_gemm((const uint16_t*)L.w.wqkv, s->xn, rows, s->qkv_dim, d.hidden, s->vg_partial, nullptr, nullptr, status, st));
+        RC(launch_qkv_rope(s->qkv, verify_gemm_partials(s->vg_partial, s->qkv_dim, d.hidden), s->cos_t, s->sin_t, s->st, 0, rows,
+                           d.n_q_heads, d.n_kv_heads, d.head_dim, st));
         RC(launch_kv_append(s->kg, L.ck, L.cv, L.kc, L.vc, s->qkv + qd, s->qkv + qd + d.n_kv_heads * d.head_dim, s->qkv_dim,
                             -1, 0, rows, kv_flags, s->st, st));
         RC(launch_verify_attn(s->kg, L.kc, L.vc, s->qkv, rows, d.n_q_heads, s->st, s->asc, s->attn, st));
-        RC(launch_calib_accum(s->attn, rows, qd, L.calib[1], s->st, st));
-        RC(launch_verify_gemm((const uint16_t*)L.w.wo, s->attn, rows, d.hidden, qd, s->vg_partial, s->y, nullptr, &s->st->status, st));
-        RC(launch_residual_rmsnorm(s->h, s->y, nullptr, 0, 0, (const uint16_t*)L.w.norm_ffn, s->xn, rows, d.hidden, d.rms_eps, st));
-        RC(launch_calib_accum(s->xn, rows, d.hidden, L.calib[2], s->st, st));
-        RC(launch_verify_gemm((const uint16_t*)L.w.wgu, s->xn, rows, 2 * d.ffn, d.hidden, s->vg_partial, s->gu, nullptr, &s->st->status, st));
-        RC(launch_swiglu(s->gu, nullptr, 0, 0, s->act, rows, d.ffn, st));
-        RC(launch_calib_accum(s->act, rows, d.ffn, L.calib[3], s->st, st));
-        RC(launch_verify_gemm((const uint16_t*)L.w.wd, s->act, rows, d.hidden, d.ffn, s->vg_partial, s->y, nullptr, &s->st->status, st));
+        if (calib) RC(launch_calib_accum(s->attn, rows, qd, L.calib[1], s->st, st));
+        RC(launch_verify_gemm((const uint16_t*)L.w.wo, s->attn, rows, d.hidden, qd, s->vg_partial, nullptr, nullptr, status, st));
+        RC(launch_residual_rmsnorm(s->h, nullptr, verify_gemm_partials(s->vg_partial, d.hidden, qd), (const uint16_t*)L.w.norm_ffn, s->xn,
+                                   rows, d.hidden, d.rms_eps, st));
+        if (calib) RC(launch_calib_accum(s->xn, rows, d.hidden, L.calib[2], s->st, st));
+        RC(launch_verify_gemm((const uint16_t*)L.w.wgu, s->xn, rows, 2 * d.ffn, d.hidden, s->vg_partial, nullptr, nullptr, status, st));
+        RC(launch_swiglu(nullptr, verify_gemm_partials(s->vg_partial, 2 * d.ffn, d.hidden), s->act, rows, d.ffn, st));
+        if (calib) RC(launch_calib_accum(s->act, rows, d.ffn, L.calib[3], s->st, st));
+        RC(launch_verify_gemm((const uint16_t*)L.w.wd, s->act, rows, d.hidden, d.ffn, s->vg_partial, nullptr, nullptr, status, st));
         const uint16_t* next_gain = (const uint16_t*)(l + 1 < d.n_layers ? s->layers[l + 1].w.norm_attn : s->norm_final);
-        RC(launch_residual_rmsnorm(s->h, s->y, nullptr, 0, 0, next_gain, s->xn, rows, d.hidden, d.rms_eps, st));
+        RC(launch_residual_rmsnorm(s->h, nullptr, verify_gemm_partials(s->vg_partial, d.hidden, d.ffn), next_gain, s->xn, rows, d.hidden,
+                                   d.rms_eps, st));
     }
-    RC(launch_calib_accum(s->xn, rows, d.hidden, s->calib_lm, s->st, st));
-    RC(launch_verify_gemm((const uint16_t*)s->lm_head, s->xn, rows, d.vocab, d.hidden, s->vg_partial, nullptr, s->logits, &s->st->status, st));
-    RC(launch_argmax(s->logits, nullptr, 0, 0, rows, d.vocab, target_argmax, logits_opt, s->argmax_val, s->argmax_tmp, s->st, 0, st));
+    if (calib) RC(launch_calib_accum(s->xn, rows, d.hidden, s->calib_lm, s->st, st));
+    RC(launch_verify_gemm((const uint16_t*)s->lm_head, s->xn, rows, d.vocab, d.hidden, s->vg_partial, nullptr, nullptr, status, st));
+    RC(launch_argmax(nullptr, verify_gemm_partials(s->vg_partial, d.vocab, d.hidden), rows, d.vocab, target_argmax, logits_opt,
+                     s->argmax_val, s->argmax_tmp, s->st, 0, st));
     return CASS_OK;
 }
 
@@ -407,29 +415,26 @@ extern "C" int cass_draft_step(void* session, const int32_t* tok_in, int32_t* to
     const cass_model_desc& d = s->d;
     const int qd = d.n_q_heads * d.head_dim;
     int32_t* status = &s->st->status;
+    auto draftp = [&](const cass_blob_info& b) { return Partials{s->partial, b.n_seg, (size_t)b.n_rowblocks * 32, 0}; };
     RC(launch_embed(tok_in, (const uint16_t*)s->embed, s->h, 1, d.hidden, st));
     RC(launch_rmsnorm(s->h, (const uint16_t*)s->layers[0].w.norm_attn, s->xn, 1, d.hidden, d.rms_eps, st));
     for (int l = 0; l < d.n_layers; ++l) {
         LayerDev& L = s->layers[l];
-        auto npad = [](const cass_blob_info& b) { return b.n_rowblocks * 32; };
         RC(launch_draft_gemv(L.blob[0], L.bi[0], s->xn, s->partial, status, st));
-        RC(launch_qkv_rope(s->qkv, s->partial, L.bi[0].n_seg, npad(L.bi[0]), s->cos_t, s->sin_t, s->st, 1, 1, d.n_q_heads,
-                           d.n_kv_heads, d.head_dim, st));
+        RC(launch_qkv_rope(s->qkv, draftp(L.bi[0]), s->cos_t, s->sin_t, s->st, 1, 1, d.n_q_heads, d.n_kv_heads, d.head_dim, st));
         RC(launch_kv_append(s->kg, L.ck, L.cv, L.kc, L.vc, s->qkv + qd, s->qkv + qd + d.n_kv_heads * d.head_dim, s->qkv_dim,
                             -1, 1, 1, CASS_KV_COMPRESSED, s->st, st));
         RC(launch_draft_attn(s->kg, L.ck, L.cv, s->qkv, d.n_q_heads, s->st, s->asc, s->attn, st));
         RC(launch_draft_gemv(L.blob[1], L.bi[1], s->attn, s->partial, status, st));
-        RC(launch_residual_rmsnorm(s->h, nullptr, s->partial, L.bi[1].n_seg, npad(L.bi[1]), (const uint16_t*)L.w.norm_ffn,
-                                   s->xn, 1, d.hidden, d.rms_eps, st));
+        RC(launch_residual_rmsnorm(s->h, nullptr, draftp(L.bi[1]), (const uint16_t*)L.w.norm_ffn, s->xn, 1, d.hidden, d.rms_eps, st));
         RC(launch_draft_gemv(L.blob[2], L.bi[2], s->xn, s->partial, status, st));
-        RC(launch_swiglu(nullptr, s->partial, L.bi[2].n_seg, npad(L.bi[2]), s->act, 1, d.ffn, st));
+        RC(launch_swiglu(nullptr, draftp(L.bi[2]), s->act, 1, d.ffn, st));
         RC(launch_draft_gemv(L.blob[3], L.bi[3], s->act, s->partial, status, st));
         const uint16_t* next_gain = (const uint16_t*)(l + 1 < d.n_layers ? s->layers[l + 1].w.norm_attn : s->norm_final);
-        RC(launch_residual_rmsnorm(s->h, nullptr, s->partial, L.bi[3].n_seg, npad(L.bi[3]), next_gain, s->xn, 1, d.hidden,
-                                   d.rms_eps, st));
+        RC(launch_residual_rmsnorm(s->h, nullptr, draftp(L.bi[3]), next_gain, s->xn, 1, d.hidden, d.rms_eps, st));
     }
     RC(launch_draft_gemv(s->lm_blob, s->lm_bi, s->xn, s->partial, status, st));
-    RC(launch_argmax(nullptr, s->partial, s->lm_bi.n_seg, s->lm_bi.n_rowblocks * 32, 1, d.vocab, tok_out, logits_opt, s->argmax_val, s->argmax_tmp, s->st, 1, st));
+    RC(launch_argmax(nullptr, draftp(s->lm_bi), 1, d.vocab, tok_out, logits_opt, s->argmax_val, s->argmax_tmp, s->st, 1, st));
     return CASS_OK;
 }
 

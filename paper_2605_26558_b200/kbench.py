@@ -177,7 +177,7 @@ def step_breakdown(gamma=4, n_prompt=512, steps=3):
     gw = {"layers": [engine.fuse_layer_weights(lw) for lw in wt["layers"]], "embed": wt["embed"], "lm_head": wt["lm_head"],
           "norm_final": wt["norm_final"]}
     del wt
-    eng = engine.Engine(shape, gw, max_seq=n_prompt + 256, gamma_max=gamma)
+    eng = engine.Engine(shape, gw, max_seq=n_prompt + 256, gamma_max=max(gamma, 1))
     eng.prefill(synth.random_prompt(n_prompt, shape.vocab, 0), calibrate=True)
     eng.encode_weights(eng.calib_norms())
     eng.build_kv_codebook()
@@ -208,6 +208,7 @@ def main():
     ap.add_argument("--copies", type=int, default=0, help="distinct operand copies (0: enough to exceed 2x L2)")
     ap.add_argument("--iters", type=int, default=5)
     ap.add_argument("--positions", type=int, default=0)
+    ap.add_argument("--gamma", type=int, default=4)
     ap.add_argument("--chunk", type=int, default=0, help="columns per decode chunk of the weight format (0 = default 256)")
     ap.add_argument("--seg", type=int, default=0, help="columns per superblock of the weight format (0 = default 2048)")
     ap.add_argument("--p", type=int, default=400)
@@ -226,7 +227,7 @@ def main():
             copies = args.copies or max(2, int(300e6 / (n * k * 2)) + 1)
             out.append(bench_verify_gemm(name, copies, args.iters))
     if args.kernel == "step":
-        out.extend(step_breakdown())
+        out.extend(step_breakdown(gamma=args.gamma))
     if args.kernel in ("attn", "all"):
         for n_pos in ([args.positions] if args.positions else [4096, 32768]):
             out.extend(bench_draft_attn(n_pos, max(2, int(3.0e5 / n_pos) + 1), args.iters))
