@@ -199,7 +199,7 @@ def run_cass(args):
     from paper_2605_26558_b200 import engine
     import synth
 
-    shape = synth.TINY if args.config == "tiny" else synth.LLAMA3_8B
+    shape = {"tiny": synth.TINY, "llama8b": synth.LLAMA3_8B, "qwen": synth.QWEN_LARGE}[args.config]
     gamma, n_prompt = args.gamma, (64 if args.config == "tiny" else args.prompt)
     dev = torch.device("cuda", local)
     t_setup = time.perf_counter()
@@ -345,9 +345,10 @@ def run_cass(args):
             "metric": METRIC, "value": emitted_all / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": ("tiny (config 1)" if args.config == "tiny" else
-                                    "llama3-8b-shape full model (config 3): 32 layers, vocab 128256, batch 1, "
-                                    f"prompt {n_prompt}, positions {n_prompt}..{n_prompt + args.steps * per_step}"),
+            "config": {"workload": {"tiny": "tiny (config 1)",
+                                    "llama8b": "llama3-8b-shape full model (config 3): 32 layers, vocab 128256, batch 1",
+                                    "qwen": "qwen-style shape (config 5): 48 layers, hidden 5120, vocab 152064, batch 1"}[args.config]
+                                   + f", prompt {n_prompt}, positions {n_prompt}..{n_prompt + args.steps * per_step}",
                        "gamma": gamma, "format": "cassandra-1 p=40% t=4 (weights and KV)",
                        "l2": "inputs larger than L2 (16 GB bf16 weights + speculation data per step)",
                        "parallelism": "replicas only" if world > 1 else "1 gpu",
@@ -380,7 +381,7 @@ def main():
     ap.add_argument("--impl", default="cass", choices=["cass", "reference"])
     ap.add_argument("--gamma", type=int, default=4)
     ap.add_argument("--prompt", type=int, default=512)
-    ap.add_argument("--config", default="llama8b", choices=["llama8b", "tiny"])
+    ap.add_argument("--config", default="llama8b", choices=["llama8b", "tiny", "qwen"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.warmup < 3:

@@ -118,3 +118,36 @@ def test_long_gaps_and_long_codewords(cass):
     got_y = y32.cpu().numpy().astype(np.float64)
     scale = np.abs(codec.bf16_bits_to_f64(dec)) @ np.abs(codec.bf16_bits_to_f64(_bits(x)))
     assert (np.abs(got_y - ref) <= 1e-5 * scale + 1e-30).all()
+
+
+def test_full_size_down_projection(cass):
+    """Llama-3-8B down projection (4096 x 14336: seven column segments, the launch configuration the benchmark
+    times): sampled superblocks bit-exact against the oracle, every GEMV output against the oracle's fp64 product."""
+    rows, cols = 4096, 14336
+    w = synth.student_t_weight(rows, cols, 21, "gpu/full_wd")
+    rng = np.random.default_rng(5)
+    act = (np.abs(rng.standard_normal(cols)) + 0.05).astype(np.float32)
+    wb = _bits(w)
+    fmt = cass.default_format()
+    blob, info, status = _encode_gpu(cass, w, act, fmt)
+    sample = [0, 1, 63, 127]
+    bodies, oinfo = layout.encode_weight_blob(wb, act, 400, 4, rowblocks=sample)
+    got = blob[: info.total_bytes].cpu().numpy().view(np.uint32)
+    assert np.array_equal(got[32:96].view(np.uint8), oinfo["codebook"])
+    n_sb = info.n_rowblocks * info.n_seg
+    directory = got[96: 96 + 4 * n_sb].reshape(n_sb, 4)
+    for sb, (body, w_f, w_u, w3) in bodies.items():
+        off = int(directory[sb][0]) * 4
+        assert tuple(int(x) for x in directory[sb][1:]) == (w_f, w_u, w3), sb
+        assert np.array_equal(got[off: off + body.size], body), sb
+    x = synth.activation_vector(cols, 3, "gpu/full_x")[0]
+    partial = torch.zeros(info.n_seg * info.n_rowblocks * 32, dtype=torch.float32, device="cuda")
+    y32 = torch.zeros(rows, dtype=torch.float32, device="cuda")
+    cass.cass_draft_gemv(blob, info, x.cuda(), partial, None, y32, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    dec = codec.draft_bits(wb, oinfo["keep"], 4)
+    ref = codec.bf16_bits_to_f64(dec) @ codec.bf16_bits_to_f64(_bits(x))
+    rms = float(np.sqrt(np.mean(ref ** 2)))
+    err = np.abs(y32.cpu().numpy().astype(np.float64) - ref).max()
+    assert err <= 2e-2 * rms and err <= 1e-4 * rms + 1e-6, (err, rms)
