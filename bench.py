@@ -114,7 +114,7 @@ def oracle_prepare():
     return dict(shape=shape, W=W, Wd=Wd, prompt=prompt, cores=int(cores))
 
 
-def oracle_sample(prep: dict, gamma: int, budget_s: float = 15.0, max_steps: int = 60) -> dict:
+def oracle_sample(prep: dict, gamma: int, budget_s: float = 15.0, max_steps: int = 150) -> dict:
     """Times the CPU oracle, as it stands, on a bounded sample of the workload: speculative steps (gamma drafts +
     gamma+1 verification rows + greedy accept) of the one-layer sample after a 64-token prefill.  The per-step time is
     multiplied by 32 layers to give tokens/s of the full model (lm_head, 3 % of the weights, is not counted)."""

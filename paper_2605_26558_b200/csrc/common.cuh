@@ -27,12 +27,24 @@
         _cfg.gridDim = (grid_); _cfg.blockDim = (block_); _cfg.dynamicSmemBytes = (smem_); _cfg.stream = (stream_); \
         cudaLaunchAttribute _at[1];                                                                         \
         _at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;                                     \
-        _at[0].val.programmaticStreamSerializationAllowed = 1;                                              \
+        _at[0].val.programmaticStreamSerializationAllowed = cass::pdl_enabled();                            \
         _cfg.attrs = _at; _cfg.numAttrs = 1;                                                                \
         if (cudaLaunchKernelEx(&_cfg, kernel_, __VA_ARGS__) != cudaSuccess) return CASS_ERR_CUDA;            \
     } while (0)
 
+#include <cstdlib>
+
 namespace cass {
+
+// CASS_NO_PDL=1 in the environment turns the overlap off (plain stream order), e.g. to read per-kernel times from a trace.
+inline int pdl_enabled() {
+    static int v = -1;
+    if (v < 0) {
+        const char* e = std::getenv("CASS_NO_PDL");
+        v = (e && e[0] == '1') ? 0 : 1;
+    }
+    return v;
+}
 
 constexpr int kRowsPerBlock = 32;          // rows (or tokens) interleaved in one superblock
 constexpr int kGroupCols = 8;              // kept columns per bitmap-walk group

@@ -339,7 +339,7 @@ int launch_draft_gemv(const void* blob, const cass_blob_info& bi, const void* x_
         cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = stream;            \
         cudaLaunchAttribute at[1];                                                                             \
         at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   /* prologue may overlap the predecessor */ \
-        at[0].val.programmaticStreamSerializationAllowed = 1;                                                  \
+        at[0].val.programmaticStreamSerializationAllowed = pdl_enabled();                                                  \
         cfg.attrs = at; cfg.numAttrs = 1;                                                                      \
         CASS_CUDA_CHECK(cudaLaunchKernelEx(&cfg, k_draft_gemv<TT>, b, x, partial, d_status, stage,             \
                                            (int)bi.max_superblock_bytes, (int)bi.seg_cols));                   \
