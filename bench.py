@@ -29,6 +29,10 @@ if ROOT not in sys.path:
 METRIC = "batch-1 decode tokens/s (8B-shape) + accepted len; draft-kernel HBM GB/s vs peak"
 UNIT = "tokens/s"
 FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum of one k_draft_gemv launch divided by the blob's bytes, from the ncu
+# capture of the 28672 x 4096 matrix (profiles/draft_gemv_wgu_28672x4096.txt: 71.54 MB for a 70.6 MB blob); a launch
+# reads its blob once plus x and writes the partial sums, so traffic scales with the blob bytes.
+DRAM_BYTES_PER_BLOB_BYTE = 1.013
 
 
 def _peaks():
@@ -363,7 +367,10 @@ def run_cass(args):
             "gpu_launches": launches_per_step(shape.n_layers, gamma) * args.steps,
             "roofline": {"kernel": "k_draft_gemv", "bound": "hbm", "achieved": achieved, "peak": hbm_peak,
                          "unit": "GB/s", "frac": achieved / hbm_peak, "peak_kind": f"of {peak_kind}",
-                         "traffic": None, "launches": len(jobs), "avg_launch_us": gemv_ms * 1e3 / len(jobs),
+                         "traffic": int(DRAM_BYTES_PER_BLOB_BYTE * blob_bits / 8 / len(jobs)),
+                         "traffic_note": "bytes per launch (average over the model's blobs), scaled from one ncu capture by blob bytes",
+                         "achieved_note": "algorithmic bytes of all launches / time of all launches",
+                         "launches": len(jobs), "avg_launch_us": gemv_ms * 1e3 / len(jobs),
                          "algorithmic_bytes_per_pass": alg_bits // 8, "blob_bytes_per_pass": blob_bits // 8},
             "cpu_baseline": cpu,
         }

@@ -50,7 +50,7 @@ typedef struct cass_format {
 
 typedef struct cass_model_desc {
     int n_layers, hidden, n_q_heads, n_kv_heads, head_dim, ffn, vocab;
-    int max_seq;             /* KV positions per sequence */
+    int max_seq;             /* KV positions per sequence (>= 32); the committed length stays <= max_seq - 16 */
     int max_batch;           /* sequences (this build: 1) */
     int gamma_max;           /* largest draft length; verification takes up to 16 rows per call */
     float rope_theta, rms_eps;
@@ -185,7 +185,8 @@ int cass_kv_append(void* session, int layer, const void* K_bf16, const void* V_b
  * n_tokens positions of the bf16 cache, freezes them, and encodes those positions into the compressed cache. */
 int cass_kv_build_codebook(void* session, int n_tokens, void* stream);
 
-/* Sets the committed length of sequence 0 (after prefill through cass_verify, or to roll back). */
+/* Sets the committed length of sequence 0 (after prefill through cass_verify, or to roll back).
+ * len + 16 <= max_seq, so that the rows of the next call still fit. */
 int cass_set_len(void* session, int len, void* stream);
 
 /* One draft token (Sec. 4.1 draft inference).  Reads the token id at tok_in, runs the draft model at position
@@ -217,7 +218,9 @@ int cass_verify_gemm(const void* W_bf16, const void* X_bf16, int rows, int n, in
 
 /* Greedy acceptance (Sec. 2.2; Eq. 1 with p/q in {0,1}): a = min({i-1 : draft[i-1] != target_argmax[i-1]} U {g});
  * out_tokens[0..a] = draft[0..a-1], target_argmax[a]; len += a + 1 (both caches are trimmed by that);
- * the draft-in-flight counter returns to 0; *next_tok = target_argmax[a].  n_accepted, next_tok: device. */
+ * the draft-in-flight counter returns to 0; *next_tok = target_argmax[a].  n_accepted, next_tok: device.
+ * A sequence that would come within 16 positions of max_seq keeps its length and the status word is set to
+ * CASS_ERR_CAPACITY (tokens are still reported). */
 int cass_accept(void* session, const int32_t* draft, const int32_t* target_argmax, int g, int32_t* n_accepted,
                 int32_t* out_tokens, int32_t* next_tok, void* stream);
 

@@ -12,6 +12,7 @@ struct DevState {
     int32_t inflight;   // draft tokens appended since the last accept
     int32_t status;     // first device-side error (CASS_ERR_*), 0 if none
     int32_t calib_on;
+    int32_t max_seq;    // KV positions per sequence; len never moves past max_seq - kMaxVerifyRows
 };
 
 // Compressed KV cache of one (layer, K|V): per head a fixed part (bitmap + fields, 32-token blocks interleaved

@@ -11,25 +11,26 @@ constexpr int kKvWarps = 8;
 constexpr int kKvFixMax = 72;        // head_dim 256, no truncation: 8 bitmap + 64 field words
 
 // Per-token selection: lane holds elements c = lane + 32 j.  keep[j] is set for the d - n_prune largest
-// |x| (ties: the lower channel is pruned first).  Key = (|x| bits << 8) | channel is unique.
+// |x| (ties: the lower channel is pruned first).  Key = (|x| bits << 8) | channel is unique, so the kept set is
+// {key >= T} where T is the largest value with at most n_prune keys below it; T is found bit by bit.
 __device__ __forceinline__ void kv_select(const uint32_t (&bits)[kKvMaxPerLane], int nj, int n_prune, int lane,
                                           bool (&keep)[kKvMaxPerLane]) {
     uint32_t key[kKvMaxPerLane];
-    int below[kKvMaxPerLane];
 #pragma unroll
-    for (int j = 0; j < kKvMaxPerLane; ++j) {
+    for (int j = 0; j < kKvMaxPerLane; ++j)
         key[j] = j < nj ? (((bits[j] & 0x7FFFu) << 8) | (uint32_t)(lane + 32 * j)) : 0xFFFFFFFFu;
-        below[j] = 0;
-    }
-    for (int jj = 0; jj < nj; ++jj) {
-        for (int src = 0; src < 32; ++src) {
-            uint32_t other = __shfl_sync(0xffffffffu, key[jj], src);
+    uint32_t thr = 0;
+    if (n_prune > 0) {
+        for (int bit = 22; bit >= 0; --bit) {
+            const uint32_t cand = thr | (1u << bit);
+            int c = 0;
 #pragma unroll
-            for (int j = 0; j < kKvMaxPerLane; ++j) below[j] += other < key[j];
+            for (int j = 0; j < kKvMaxPerLane; ++j) c += key[j] < cand;
+            if (__reduce_add_sync(0xffffffffu, c) <= n_prune) thr = cand;
         }
     }
 #pragma unroll
-    for (int j = 0; j < kKvMaxPerLane; ++j) keep[j] = j < nj && below[j] >= n_prune;
+    for (int j = 0; j < kKvMaxPerLane; ++j) keep[j] = j < nj && key[j] >= thr;
 }
 
 __global__ void __launch_bounds__(256) k_kv_hist(KvGeom g, KvComp ck, KvComp cv, const uint16_t* __restrict__ k_cache,

@@ -246,7 +246,10 @@ __global__ void k_accept(DevState* st, const int32_t* __restrict__ draft, const 
     for (int i = a + 1; i <= g; ++i) out_tokens[i] = -1;
     *n_acc = a;
     if (next_tok) *next_tok = target[a];
-    st->len += a + 1;
+    // Every later call touches positions up to len + 15 at most; a sequence that would come closer than that to
+    // the end of its cache stops growing and the status word says so.
+    if (st->len + a + 1 + kMaxVerifyRows > st->max_seq) atomicCAS(&st->status, 0, CASS_ERR_CAPACITY);
+    else st->len += a + 1;
     st->inflight = 0;
 }
 

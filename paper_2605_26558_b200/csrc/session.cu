@@ -53,7 +53,7 @@ static int check_desc(const cass_model_desc* d, const cass_format* f) {
     if (f->mode != 1) return CASS_ERR_UNSUPPORTED;
     if (d->max_batch != 1) return CASS_ERR_UNSUPPORTED;
     if (d->n_layers <= 0 || d->hidden <= 0 || d->n_q_heads <= 0 || d->n_kv_heads <= 0 || d->head_dim <= 0 ||
-        d->ffn <= 0 || d->vocab <= 0 || d->max_seq <= 0)
+        d->ffn <= 0 || d->vocab <= 0 || d->max_seq < 2 * kMaxVerifyRows)
         return CASS_ERR_INVALID_ARG;
     if (d->n_q_heads % d->n_kv_heads || d->head_dim % 32 || d->head_dim > 256 || d->n_q_heads / d->n_kv_heads > 8)
         return CASS_ERR_UNSUPPORTED;
@@ -215,6 +215,7 @@ extern "C" int cass_session_init(void* mem, size_t bytes, const cass_model_desc*
     for (int l = 0; l < desc->n_layers; ++l) s->layers[l].w = weights->h_layers[l];
     s->embed = weights->embed; s->lm_head = weights->lm_head; s->norm_final = weights->norm_final;
     if (cudaMemsetAsync(mem, 0, need, stream) != cudaSuccess) { delete s; return CASS_ERR_CUDA; }
+    if (cudaMemcpyAsync(&s->st->max_seq, &s->d.max_seq, 4, cudaMemcpyHostToDevice, stream) != cudaSuccess) { delete s; return CASS_ERR_CUDA; }
     rc = launch_rope_table(s->cos_t, s->sin_t, desc->max_seq, desc->head_dim, desc->rope_theta, stream);
     if (!rc && blobs) rc = read_blob_infos(s, blobs, stream);
     if (!rc && cudaStreamSynchronize(stream) != cudaSuccess) rc = CASS_ERR_CUDA;
@@ -239,6 +240,7 @@ extern "C" int cass_session_reset(void* session, void* stream_) {
     Session* s = (Session*)session;
     cudaStream_t stream = (cudaStream_t)stream_;
     CASS_CUDA_CHECK(cudaMemsetAsync(s->st, 0, sizeof(DevState), stream));
+    CASS_CUDA_CHECK(cudaMemcpyAsync(&s->st->max_seq, &s->d.max_seq, 4, cudaMemcpyHostToDevice, stream));
     CASS_CUDA_CHECK(cudaMemsetAsync(s->calib_all, 0, s->calib_count * 4, stream));
     for (auto& L : s->layers)
         for (int kind = 0; kind < 2; ++kind) {
@@ -288,7 +290,7 @@ extern "C" int cass_calib_norms(void* session, float* norms_out, void* stream_) 
 extern "C" int cass_set_len(void* session, int len, void* stream_) {
     if (!session) return CASS_ERR_INVALID_ARG;
     Session* s = (Session*)session;
-    if (len < 0 || len > s->d.max_seq) return CASS_ERR_INVALID_ARG;
+    if (len < 0 || len + kMaxVerifyRows > s->d.max_seq) return CASS_ERR_INVALID_ARG;      // room for one more call's rows
     int32_t v[2] = {len, 0};
     CASS_CUDA_CHECK(cudaMemcpyAsync(&s->st->len, v, 8, cudaMemcpyHostToDevice, (cudaStream_t)stream_));
     CASS_CUDA_CHECK(cudaStreamSynchronize((cudaStream_t)stream_));
