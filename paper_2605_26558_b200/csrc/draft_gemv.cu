@@ -183,11 +183,14 @@ __device__ __forceinline__ float chunk_dot_fast(const uint32_t* __restrict__ sb,
 template <int T>
 __global__ void __launch_bounds__(1024) k_draft_gemv(const uint32_t* __restrict__ blob, const uint16_t* __restrict__ x,
                                                      float* __restrict__ partial, int32_t* __restrict__ d_status,
-                                                     int stage_bytes, int max_sb, int seg_cols_host) {
+                                                     int stage_bytes, int max_sb, int n, int k, int t, int seg_cols,
+                                                     int chunk_cols, int n_seg, int n_rb) {
     extern __shared__ __align__(128) uint8_t smem_raw[];
+    // The geometry comes from the host's copy of the header (the launch sized shared memory from it); the header
+    // itself is fetched now and compared once it has arrived, so that its latency is off the critical path.
     const uint32_t* h = blob;
-    const int n = h[H_ROWS], k = h[H_COLS], t = h[H_T], seg_cols = h[H_SEG], chunk_cols = h[H_CHUNK];
-    const int n_seg = h[H_NSEG], n_rb = h[H_NRB];
+    const uint32_t h_n = h[H_ROWS], h_k = h[H_COLS], h_t = h[H_T], h_seg = h[H_SEG], h_chunk = h[H_CHUNK], h_nseg = h[H_NSEG],
+                   h_nrb = h[H_NRB], h_magic = h[H_MAGIC];
     const int k_pad = ceil_div(k, 32) * 32;
     const int seg = blockIdx.x, rb0 = blockIdx.y, rb_step = gridDim.y;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, n_warps = blockDim.x >> 5;
@@ -202,7 +205,7 @@ __global__ void __launch_bounds__(1024) k_draft_gemv(const uint32_t* __restrict_
     const int n_ch = ceil_div(scols, chunk_cols);
     // The launch sized shared memory from the host's copy of the header; a blob that does not match it is
     // refused instead of overrunning the buffers.
-    if (seg >= n_seg || (int)blockDim.x < 32 * n_ch || seg_cols != seg_cols_host || n_ch > 32) {
+    if (seg >= n_seg || (int)blockDim.x < 32 * n_ch || n_ch > 32) {
         if (tid == 0 && d_status) atomicExch(d_status, CASS_ERR_INVALID_ARG);
         return;
     }
@@ -249,6 +252,13 @@ __global__ void __launch_bounds__(1024) k_draft_gemv(const uint32_t* __restrict_
         xs[i] = (i < scols && c < k) ? bf16_bits_to_float(x[c]) : 0.f;
     }
     __syncthreads();
+    if (h_magic != kBlobMagic || (int)h_n != n || (int)h_k != k || (int)h_t != t || (int)h_seg != seg_cols ||
+        (int)h_chunk != chunk_cols || (int)h_nseg != n_seg || (int)h_nrb != n_rb) {
+        // not the blob the caller described: flag it, let the copies already started land, produce nothing
+        if (tid == 0 && d_status) atomicExch(d_status, CASS_ERR_INVALID_ARG);
+        for (int j = 0; j < n_tiles && j < kGemvStages; ++j) mbar_wait_bounded(&bar[j % kGemvStages], 0u);
+        return;
+    }
 
     for (int i = 0; i < n_tiles; ++i) {
         const int s = i % kGemvStages;
@@ -342,7 +352,9 @@ int launch_draft_gemv(const void* blob, const cass_blob_info& bi, const void* x_
         at[0].val.programmaticStreamSerializationAllowed = pdl_enabled();                                                  \
         cfg.attrs = at; cfg.numAttrs = 1;                                                                      \
         CASS_CUDA_CHECK(cudaLaunchKernelEx(&cfg, k_draft_gemv<TT>, b, x, partial, d_status, stage,             \
-                                           (int)bi.max_superblock_bytes, (int)bi.seg_cols));                   \
+                                           (int)bi.max_superblock_bytes, (int)bi.rows, (int)bi.cols,           \
+                                           (int)bi.trunc_bits, (int)bi.seg_cols, (int)bi.chunk_cols,           \
+                                           (int)bi.n_seg, (int)bi.n_rowblocks));                               \
     } while (0)
     if (bi.trunc_bits == 4) CASS_GEMV_LAUNCH(4);
     else if (bi.trunc_bits == 0) CASS_GEMV_LAUNCH(0);
