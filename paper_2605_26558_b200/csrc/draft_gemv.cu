@@ -247,9 +247,23 @@ __global__ void __launch_bounds__(1024) k_draft_gemv(const uint32_t* __restrict_
     pdl_wait();
     // x of this segment (fp32), zero beyond the matrix
     const int c0 = seg * seg_cols;
-    for (int i = tid; i < seg_cols + kXSlack; i += blockDim.x) {
-        int c = c0 + i;
-        xs[i] = (i < scols && c < k) ? bf16_bits_to_float(x[c]) : 0.f;
+    if ((k & 7) == 0 && ((uintptr_t)x & 15) == 0) {
+        // eight values per 16-byte load: one round trip to L2 for the whole slice
+        for (int i = tid * 8; i < seg_cols + kXSlack; i += blockDim.x * 8) {
+            uint4 v = make_uint4(0u, 0u, 0u, 0u);
+            if (i < scols && c0 + i < k) v = *reinterpret_cast<const uint4*>(x + c0 + i);
+            float4 lo = make_float4(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xFFFF0000u), __uint_as_float(v.y << 16),
+                                    __uint_as_float(v.y & 0xFFFF0000u));
+            float4 hi = make_float4(__uint_as_float(v.z << 16), __uint_as_float(v.z & 0xFFFF0000u), __uint_as_float(v.w << 16),
+                                    __uint_as_float(v.w & 0xFFFF0000u));
+            *reinterpret_cast<float4*>(xs + i) = lo;
+            *reinterpret_cast<float4*>(xs + i + 4) = hi;
+        }
+    } else {
+        for (int i = tid; i < seg_cols + kXSlack; i += blockDim.x) {
+            int c = c0 + i;
+            xs[i] = (i < scols && c < k) ? bf16_bits_to_float(x[c]) : 0.f;
+        }
     }
     __syncthreads();
     if (h_magic != kBlobMagic || (int)h_n != n || (int)h_k != k || (int)h_t != t || (int)h_seg != seg_cols ||
