@@ -61,12 +61,14 @@ def test_verify_gemm_rows_do_not_depend_on_the_batch(cass):
     assert torch.equal(alone[0], full[0])
 
 
-@pytest.mark.parametrize("n_pos", [1, 63, 64, 65, 700, 4096])
-def test_draft_attention_llama_layer_shape(cass, n_pos):
-    """Draft attention of one Llama-3-8B-shaped layer (32 q / 8 kv heads of 128) over synthetic KV (N(0,1), outlier
-    channels in K) against the oracle: softmax(q . K_hat / sqrt(d)) V_hat on the zero-padded reconstruction."""
+@pytest.mark.parametrize("n_pos,n_q", [(1, 32), (63, 32), (64, 32), (65, 32), (700, 32), (4096, 32), (300, 40), (130, 64)])
+def test_draft_attention_llama_layer_shape(cass, n_pos, n_q):
+    """Draft attention of one Llama-3-8B-shaped layer (32 q / 8 kv heads of 128; also 5 and 8 query heads per KV head,
+    the Qwen-style grouping) over synthetic KV (N(0,1), outlier channels in K) against the oracle:
+    softmax(q . K_hat / sqrt(d)) V_hat on the zero-padded reconstruction."""
     from paper_2605_26558_b200 import engine
-    shape = synth.ModelShape(n_layers=1, hidden=256, n_q_heads=32, n_kv_heads=8, head_dim=128, ffn=256, vocab=256)
+    G = n_q // 8
+    shape = synth.ModelShape(n_layers=1, hidden=256, n_q_heads=n_q, n_kv_heads=8, head_dim=128, ffn=256, vocab=256)
     wt = synth.model_weights(shape, 0, device="cuda")
     gw = {"layers": [engine.fuse_layer_weights(lw) for lw in wt["layers"]], "embed": wt["embed"], "lm_head": wt["lm_head"],
           "norm_final": wt["norm_final"]}
@@ -79,8 +81,8 @@ def test_draft_attention_llama_layer_shape(cass, n_pos):
         cass.cass_kv_append(eng.session, 0, k[n0:].cuda().contiguous(), v[n0:].cuda().contiguous(), n0, n_pos - n0,
                             cass.KV_BF16 | cass.KV_COMPRESSED)
     cass.cass_set_len(eng.session, n_pos - 1)
-    q = synth.activation_vector(128, 2, "ka/q", rows=32)
-    out = torch.zeros(32, 128, dtype=torch.bfloat16, device="cuda")
+    q = synth.activation_vector(128, 2, "ka/q", rows=n_q)
+    out = torch.zeros(n_q, 128, dtype=torch.bfloat16, device="cuda")
     cass.cass_draft_attention(eng.session, 0, q.cuda().contiguous(), out)
     torch.cuda.synchronize()
     assert eng.status()[0] == 0
@@ -88,11 +90,11 @@ def test_draft_attention_llama_layer_shape(cass, n_pos):
     kd = codec.bf16_bits_to_f64(codec.draft_bits(kb, codec.keep_mask_kv(kb, 400), 4))
     vd = codec.bf16_bits_to_f64(codec.draft_bits(vb, codec.keep_mask_kv(vb, 400), 4))
     qf = codec.bf16_bits_to_f64(_bits(q))
-    want = np.zeros((32, 128))
-    for hq in range(32):
-        sc = kd[:, hq // 4, :] @ qf[hq] / np.sqrt(128.0)
+    want = np.zeros((n_q, 128))
+    for hq in range(n_q):
+        sc = kd[:, hq // G, :] @ qf[hq] / np.sqrt(128.0)
         p = np.exp(sc - sc.max())
-        want[hq] = (p / p.sum()) @ vd[:, hq // 4, :]
+        want[hq] = (p / p.sum()) @ vd[:, hq // G, :]
     got = codec.bf16_bits_to_f64(_bits(out))
     rms = float(np.sqrt(np.mean(want ** 2)))
     # The output is rounded to bf16, so each element may be off by half an ulp (<= 2^-8 |value|) on top of the

@@ -269,3 +269,46 @@ def test_kv_encoder_records_bit_exact(cass, tiny):
             cache = eng.mem.view(torch.int16)[cache_off: cache_off + (n0 + n1) * shape.n_kv_heads * d]
             assert np.array_equal(cache.cpu().numpy().astype(np.uint16).reshape(n0 + n1, shape.n_kv_heads, d), xb)
     eng.close()
+
+
+def test_five_query_heads_per_kv_head(cass):
+    """The Qwen-style grouping (5 query heads per KV head) on a small model: prefill logits against the oracle and the
+    speculative stream against the same kernels' plain greedy stream."""
+    shape = synth.ModelShape(n_layers=2, hidden=192, n_q_heads=10, n_kv_heads=2, head_dim=32, ffn=320, vocab=512)
+    wt = synth.model_weights(shape, 7)
+    wb = {"layers": [{k: _bits(v) for k, v in lw.items()} for lw in wt["layers"]],
+          "embed": _bits(wt["embed"]), "lm_head": _bits(wt["lm_head"]), "norm_final": _bits(wt["norm_final"])}
+    prompt = synth.random_prompt(40, shape.vocab, 7)
+    W = model.Weights(shape, wb)
+    kv = model.KVCache(shape, 64)
+    ref = np.stack([model.forward_token(W, kv, int(t), p, False, 400, 4) for p, t in enumerate(prompt.numpy())])
+    with model.accumulate_in(np.float32):
+        W32 = model.Weights(shape, wb)
+        kv32 = model.KVCache(shape, 64)
+        l32 = np.stack([model.forward_token(W32, kv32, int(t), p, False, 400, 4) for p, t in enumerate(prompt.numpy())])
+    floor = float((np.abs(l32 - ref).max(axis=1) / np.sqrt(np.mean(ref ** 2, axis=1))).max())
+
+    def make():
+        eng = cass.engine.Engine(shape, _gpu_weights(cass, wt), max_seq=160, gamma_max=6)
+        first = eng.prefill(prompt, calibrate=True)
+        eng.encode_weights(eng.calib_norms())
+        eng.build_kv_codebook()
+        return eng, first
+
+    eng = cass.engine.Engine(shape, _gpu_weights(cass, wt), max_seq=160, gamma_max=6)
+    logits = torch.zeros(16, shape.vocab, dtype=torch.float32, device="cuda")
+    errs = []
+    for pos in (0, 16):
+        cass.cass_set_len(eng.session, pos)
+        cass.cass_verify(eng.session, prompt[pos: pos + 16].cuda(), 15, eng.targ, logits)
+        got = logits.cpu().numpy()
+        errs += [_rel_err(got[r], ref[pos + r]) for r in range(16)]
+    _check_logit_errors(errs, floor)
+    eng.close()
+    e0, f0 = make()
+    plain, _ = e0.generate(24, 0)
+    e1, f1 = make()
+    spec, stats = e1.generate(24, 5)
+    assert f0 == f1 and spec[:24] == plain[:24]
+    assert e1.status()[0] == 0 and stats.emitted == stats.accepted + stats.steps
+    e0.close(); e1.close()
