@@ -214,18 +214,19 @@ def run_cass(args):
     per_step = gamma + 1
     max_seq = n_prompt + (max(args.steps, args.warmup) + 2) * per_step + 64
     max_seq = (max_seq + 255) // 256 * 256
-    eng = engine.Engine(shape, gw, max_seq=max_seq, gamma_max=max(gamma, 1), device=dev)
-    prompt = synth.random_prompt(n_prompt, shape.vocab, seed=rank)
+    nb = args.batch
+    eng = engine.Engine(shape, gw, max_seq=max_seq, gamma_max=max(gamma, 1), device=dev, batch=nb)
+    prompt = torch.stack([synth.random_prompt(n_prompt, shape.vocab, seed=rank * 8 + b) for b in range(nb)])
     eng.prefill(prompt, calibrate=True)
     eng.encode_weights(eng.calib_norms())
     eng.build_kv_codebook()
     torch.cuda.synchronize()
-    first_tok = eng.toks[0:1].clone()
+    first_tok = eng.next_tokens()
     setup_s = time.perf_counter() - t_setup
 
     def rewind():
         cass.cass_set_len(eng.session, n_prompt)
-        eng.toks[0:1] = first_tok
+        eng.set_next_tokens(first_tok)
 
     # CUDA graph of one speculative step (all state, positions included, lives on the device)
     eng.step(gamma)
@@ -245,7 +246,7 @@ def run_cass(args):
         for _ in range(n):
             graph.replay()
             if count:
-                emitted_acc.add_(eng.n_acc.to(torch.int64) + 1)
+                emitted_acc.add_((eng.n_acc[:nb].to(torch.int64) + 1).sum())
 
     # ---- device-resident timing ----
     rewind()
@@ -266,23 +267,24 @@ def run_cass(args):
 
     # ---- end to end: host buffers in, host buffers out, every step ----
     rewind()
-    h_in = torch.zeros(1, dtype=torch.int32).pin_memory()
-    h_out = torch.zeros(gamma + 2, dtype=torch.int32).pin_memory()
-    h_in[0] = int(first_tok.item())
-    d_out = torch.zeros(gamma + 2, dtype=torch.int32, device=dev)
+    h_in = torch.zeros(nb, dtype=torch.int32).pin_memory()
+    h_out = torch.zeros(nb * (gamma + 2), dtype=torch.int32).pin_memory()
+    h_in.copy_(first_tok)
+    d_out = torch.zeros(nb * (gamma + 2), dtype=torch.int32, device=dev)
     e2e_emitted = 0
     barrier()
     e2, e3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e2.record()
     for _ in range(args.steps):
-        eng.toks[0:1].copy_(h_in, non_blocking=True)                       # host -> device: the step's input token
+        eng.set_next_tokens(h_in, non_blocking=True)                       # host -> device: the step's input tokens
         graph.replay()
-        d_out[0:1].copy_(eng.n_acc); d_out[1:].copy_(eng.out_tokens[: gamma + 1])
-        h_out.copy_(d_out, non_blocking=True)                              # device -> host: accepted count + tokens
+        d_out[:nb].copy_(eng.n_acc[:nb]); d_out[nb:].copy_(eng.out_tokens[: nb * (gamma + 1)])
+        h_out.copy_(d_out, non_blocking=True)                              # device -> host: accepted counts + tokens
         torch.cuda.current_stream().synchronize()
-        a = int(h_out[0])
-        e2e_emitted += a + 1
-        h_in[0] = int(h_out[1 + a])
+        for b in range(nb):
+            a = int(h_out[b])
+            e2e_emitted += a + 1
+            h_in[b] = int(h_out[nb + b * (gamma + 1) + a])
     e3.record()
     barrier()
     ms_e2e = e2.elapsed_time(e3)
@@ -304,7 +306,7 @@ def run_cass(args):
         g0.replay()
     p1.record()
     torch.cuda.synchronize()
-    plain_tok_s = n0 / (p0.elapsed_time(p1) * 1e-3)
+    plain_tok_s = n0 * nb / (p0.elapsed_time(p1) * 1e-3)
 
     # ---- dominant kernel: draft GEMV over every blob of the model, back to back (4.8 GB: larger than L2) ----
     hbm_peak, peak_kind = _peaks()
@@ -343,27 +345,28 @@ def run_cass(args):
     if rank == 0:
         cpu = None
         if world == 1 and not args.no_cpu_baseline:
-            cpu = oracle_sample(oracle_prepare(), gamma)
+            cpu = oracle_sample(oracle_prepare(), gamma)       # one sequence: the oracle has no batched form
             cpu = {k: cpu[k] for k in ("value", "unit", "cores", "kind", "sample")}
         line = {
             "metric": METRIC, "value": emitted_all / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": {"tiny": "tiny (config 1)",
-                                    "llama8b": "llama3-8b-shape full model (config 3): 32 layers, vocab 128256, batch 1",
-                                    "qwen": "qwen-style shape (config 5): 48 layers, hidden 5120, vocab 152064, batch 1"}[args.config]
-                                   + f", prompt {n_prompt}, positions {n_prompt}..{n_prompt + args.steps * per_step}",
+                                    "llama8b": "llama3-8b-shape full model (config 3): 32 layers, vocab 128256",
+                                    "qwen": "qwen-style shape (config 5): 48 layers, hidden 5120, vocab 152064"}[args.config]
+                                   + f", batch {nb}, prompt {n_prompt}, positions {n_prompt}..{n_prompt + args.steps * per_step}",
+                       "batch": nb,
                        "gamma": gamma, "format": "cassandra-1 p=40% t=4 (weights and KV)",
                        "l2": "inputs larger than L2 (16 GB bf16 weights + speculation data per step)",
                        "parallelism": "replicas only" if world > 1 else "1 gpu",
-                       "mean_accepted_len": emitted_all / (args.steps * world) - 1.0,
+                       "mean_accepted_len": emitted_all / (args.steps * world * nb) - 1.0,
                        "tokens_per_step": emitted_all / (args.steps * world),
                        "plain_bf16_greedy_tokens_per_s": plain_tok_s,
                        "speedup_vs_plain_bf16": emitted / (ms * 1e-3) / plain_tok_s if world == 1 else None,
                        "speculation_data_bytes": eng.blob_bytes(), "setup_s": setup_s, "status": st_code},
             "clocks": clocks,
-            "e2e": {"value": e2e_all / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": 4,
-                    "d2h_bytes_per_step": 4 * (gamma + 2)},
+            "e2e": {"value": e2e_all / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": 4 * nb,
+                    "d2h_bytes_per_step": 4 * nb * (gamma + 2)},
             "gpu_launches": launches_per_step(shape.n_layers, gamma) * args.steps,
             "roofline": {"kernel": "k_draft_gemv", "bound": "hbm", "achieved": achieved, "peak": hbm_peak,
                          "unit": "GB/s", "frac": achieved / hbm_peak, "peak_kind": f"of {peak_kind}",
@@ -388,6 +391,7 @@ def main():
     ap.add_argument("--impl", default="cass", choices=["cass", "reference"])
     ap.add_argument("--gamma", type=int, default=4)
     ap.add_argument("--prompt", type=int, default=512)
+    ap.add_argument("--batch", type=int, default=1, choices=[1, 2, 4, 8], help="sequences decoded together (config 4 sweeps this)")
     ap.add_argument("--config", default="llama8b", choices=["llama8b", "tiny", "qwen"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

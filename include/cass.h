@@ -51,8 +51,8 @@ typedef struct cass_format {
 typedef struct cass_model_desc {
     int n_layers, hidden, n_q_heads, n_kv_heads, head_dim, ffn, vocab;
     int max_seq;             /* KV positions per sequence (>= 32); the committed length stays <= max_seq - 16 */
-    int max_batch;           /* sequences (this build: 1) */
-    int gamma_max;           /* largest draft length; verification takes up to 16 rows per call */
+    int max_batch;           /* sequences decoded together: 1, 2, 4 or 8; every step-level call handles all of them */
+    int gamma_max;           /* largest draft length (<= 15); max_batch * (gamma_max + 1) <= 64 */
     float rope_theta, rms_eps;
 } cass_model_desc;
 
@@ -126,6 +126,12 @@ int cass_decode_weights(const void* blob, const cass_blob_info* h_info, void* W_
 int cass_draft_gemv(const void* blob, const cass_blob_info* h_info, const void* x_bf16, float* partial,
                     void* y_bf16, float* y_f32, int32_t* d_status, void* stream);
 
+/* The same for n_vec = 1, 2, 4 or 8 vectors (the low-batch regime of Sec. 2.1: one pass over the speculation data,
+ * every decoded weight used n_vec times).  x: bf16 [n_vec][cols]; partial: fp32 scratch [n_vec][n_seg][n_rowblocks*32];
+ * outputs [n_vec][rows].  Vector b's result equals what cass_draft_gemv gives for x[b] alone, bit for bit. */
+int cass_draft_gemv_batch(const void* blob, const cass_blob_info* h_info, const void* x_bf16, int n_vec, float* partial,
+                          void* y_bf16, float* y_f32, int32_t* d_status, void* stream);
+
 /* Draft GEMV without a scratch argument (the paper has no counterpart; this is a convenience of this library).
  * Some callers cannot obtain device memory at the point where they call: code running between the capture-safe
  * parts of an inference server, plug-ins that are handed only their input and output tensors, or hosts whose
@@ -163,6 +169,11 @@ int cass_session_reset(void* session, void* stream);
 
 /* Reads the device status word and the committed length of sequence 0.  SYNCHRONISES `stream`. */
 int cass_session_status(void* session, int32_t* h_status, int32_t* h_len, void* stream);
+/* Committed lengths of all sequences: h_lens[max_batch].  SYNCHRONISES `stream`. */
+int cass_session_lens(void* session, int32_t* h_lens, void* stream);
+/* Rows (over all sequences) one cass_verify call can take for this description: 16, 32 or 64; negative on a bad
+ * description.  Prefill feeds max_batch * (g+1) <= that many rows per call.  Host-only arithmetic. */
+int cass_session_rows(const cass_model_desc* desc);
 
 /* Wanda calibration (Sec. 4.2, Sec. 7.2 "Pre-Computation Cost"): while enabled, cass_verify accumulates the
  * per-input-channel sums of squares of the activations entering each projection.  cass_calib_norms writes
@@ -173,65 +184,78 @@ int cass_calib_norms(void* session, float* norms_out, void* stream);
 size_t cass_calib_norms_count(const cass_model_desc* desc);
 
 /* Online KV encoder (Sec. 4.2 per-token magnitude pruning; Sec. 5.1 encoder).  Writes n_new tokens of one
- * layer, starting at position start_pos of sequence 0, into the bf16 cache and/or the compressed cache
+ * layer, starting at position start_pos of sequence `seq`, into the bf16 cache and/or the compressed cache
  * (flags).  K, V: bf16 [n_new][n_kv_heads][head_dim]; K is expected post-RoPE.  Per token and head the
  * floor(d*p/1000) smallest |x| are pruned (ties: lower channel first).  Positions must be appended in
  * order: start_pos may not exceed the number of positions already in the compressed cache of that layer.
  * The compressed cache uses the layer's frozen codebooks (cass_kv_build_codebook). */
-int cass_kv_append(void* session, int layer, const void* K_bf16, const void* V_bf16, int start_pos, int n_new,
+int cass_kv_append(void* session, int seq, int layer, const void* K_bf16, const void* V_bf16, int start_pos, int n_new,
                    int flags, void* stream);
 
-/* Builds the exponent codebooks of every layer (one for K, one for V) from the kept values of the first
- * n_tokens positions of the bf16 cache, freezes them, and encodes those positions into the compressed cache. */
+/* Builds the exponent codebooks of every sequence and layer (one for K, one for V) from the kept values of the
+ * first n_tokens positions of that sequence's bf16 cache, freezes them, and encodes those positions into the
+ * compressed cache. */
 int cass_kv_build_codebook(void* session, int n_tokens, void* stream);
 
-/* Sets the committed length of sequence 0 (after prefill through cass_verify, or to roll back).
- * len + 16 <= max_seq, so that the rows of the next call still fit. */
+/* Sets the committed length of every sequence to len (after prefill through cass_verify, or to roll back);
+ * cass_set_lens gives each sequence its own (h_lens: HOST [max_batch]).  len + 16 <= max_seq, so that the rows of
+ * the next call still fit.  Both clear the drafts in flight and SYNCHRONISE `stream`. */
 int cass_set_len(void* session, int len, void* stream);
+int cass_set_lens(void* session, const int32_t* h_lens, void* stream);
 
-/* One draft token (Sec. 4.1 draft inference).  Reads the token id at tok_in, runs the draft model at position
- * len + (tokens drafted since the last accept), appends that position's K/V to the compressed cache only,
- * and writes the greedy next token to tok_out (lowest index on ties).  logits_opt: fp32 [vocab] or NULL. */
-int cass_draft_step(void* session, const int32_t* tok_in, int32_t* tok_out, float* logits_opt, void* stream);
+/* One draft token per sequence (Sec. 4.1 draft inference).  Reads the token id tok_in[b * tok_stride] of each
+ * sequence b, runs the draft model for it at position len_b + (tokens drafted since the last accept), appends that
+ * position's K/V to the sequence's compressed cache only, and writes the greedy next token to
+ * tok_out[b * tok_stride] (lowest index on ties).  tok_stride = 1 for packed arrays, g+1 when the tokens sit in the
+ * [max_batch][g+1] array that cass_verify reads.  The weights' speculation data is read and decoded once for all
+ * sequences.  logits_opt: fp32 [max_batch][vocab] or NULL. */
+int cass_draft_step(void* session, const int32_t* tok_in, int32_t* tok_out, int tok_stride, float* logits_opt,
+                    void* stream);
 
-/* Target pass over g+1 rows (Sec. 2.2 verification; Sec. 4.1 target inference): toks[i] sits at position
- * len + i; causal among the rows; K/V of those positions are (over)written in both caches; row i's greedy
- * token goes to target_argmax[i].  g+1 <= 16.  g = 0 is plain autoregressive decoding.  Does not move len.
- * logits_opt: fp32 [g+1][vocab] or NULL.  Row results do not depend on how many rows the call has. */
+/* Target pass over g+1 rows of every sequence (Sec. 2.2 verification; Sec. 4.1 target inference):
+ * toks[b][i] sits at position len_b + i of sequence b; causal among a sequence's rows; K/V of those positions are
+ * (over)written in both caches; the greedy token of row (b, i) goes to target_argmax[b][i].  g+1 <= 16 and
+ * max_batch * (g+1) <= cass_session_rows().  g = 0 is plain autoregressive decoding.  Does not move len.
+ * logits_opt: fp32 [max_batch][g+1][vocab] or NULL.  Row results do not depend on how many rows the call has. */
 int cass_verify(void* session, const int32_t* toks, int g, int32_t* target_argmax, float* logits_opt,
                 void* stream);
 
 /* Stand-alone draft attention of one layer (Sec. 4.1 draft inference over the KV speculation data of Sec. 4.2):
- * q: bf16 [n_q_heads][head_dim] (post-RoPE); the query sees the first len + 1 positions of the layer's compressed
- * cache (len = committed length, see cass_set_len; no draft in flight); out: bf16 [n_q_heads][head_dim]. */
+ * q: bf16 [max_batch][n_q_heads][head_dim] (post-RoPE); sequence b's query sees the first len_b + 1 positions of its
+ * compressed cache of that layer (len = committed length, see cass_set_len; no draft in flight);
+ * out: bf16 [max_batch][n_q_heads][head_dim]. */
 int cass_draft_attention(void* session, int layer, const void* q_bf16, void* out_bf16, void* stream);
 
 /* Stand-alone verification projection (Sec. 2.2: the gamma+1 rows are processed as one small batch, bound by
- * the bf16 weight bytes): Y[r][j] = sum_c W[j][c] X[r][c] for r < rows <= 16, fp32 accumulation on the tensor
- * cores.  W: bf16 [n][k] row-major, 16-byte aligned, k a multiple of 8.  X: bf16 buffer of 16 rows of k values,
- * 16-byte aligned (rows beyond `rows` are read but do not influence the result).  scratch: device memory of
+ * the bf16 weight bytes): Y[r][j] = sum_c W[j][c] X[r][c] for r < rows <= 64, fp32 accumulation on the tensor
+ * cores.  W: bf16 [n][k] row-major, 16-byte aligned, k a multiple of 8.  X: bf16 buffer of 16, 32 or 64 rows (the
+ * smallest of these >= rows) of k values, 16-byte aligned (rows beyond `rows` are read but do not influence the
+ * result).  scratch: device memory of
  * cass_verify_gemm_scratch_bytes(n, k).  Outputs [rows][n]; either may be NULL.  A row's result does not depend
  * on `rows`.  d_status (required) receives CASS_ERR_TIMEOUT if a bounded device wait runs out. */
 size_t cass_verify_gemm_scratch_bytes(int n, int k);
 int cass_verify_gemm(const void* W_bf16, const void* X_bf16, int rows, int n, int k, void* scratch, size_t scratch_bytes,
                      void* y_bf16, float* y_f32, int32_t* d_status, void* stream);
 
-/* Greedy acceptance (Sec. 2.2; Eq. 1 with p/q in {0,1}): a = min({i-1 : draft[i-1] != target_argmax[i-1]} U {g});
- * out_tokens[0..a] = draft[0..a-1], target_argmax[a]; len += a + 1 (both caches are trimmed by that);
- * the draft-in-flight counter returns to 0; *next_tok = target_argmax[a].  n_accepted, next_tok: device.
+/* Greedy acceptance (Sec. 2.2; Eq. 1 with p/q in {0,1}), per sequence b, with draft_b[i] = draft[b * draft_stride + i]:
+ * a = min({i-1 : draft_b[i-1] != target_argmax[b][i-1]} U {g});
+ * out_tokens[b][0..a] = draft_b[0..a-1], target_argmax[b][a] (the rest -1); len_b += a + 1 (both caches are trimmed
+ * by that); the draft-in-flight counter returns to 0; next_tok[b * next_stride] = target_argmax[b][a].
+ * draft_stride >= g (g for a packed [max_batch][g] array; g+1 with draft = toks + 1 of the verification array);
+ * target_argmax and out_tokens: [max_batch][g+1]; n_accepted: [max_batch]; all device.
  * A sequence that would come within 16 positions of max_seq keeps its length and the status word is set to
  * CASS_ERR_CAPACITY (tokens are still reported). */
-int cass_accept(void* session, const int32_t* draft, const int32_t* target_argmax, int g, int32_t* n_accepted,
-                int32_t* out_tokens, int32_t* next_tok, void* stream);
+int cass_accept(void* session, const int32_t* draft, int draft_stride, const int32_t* target_argmax, int g,
+                int32_t* n_accepted, int32_t* out_tokens, int32_t* next_tok, int next_stride, void* stream);
 
-/* Geometry of the compressed KV cache of (layer, kind 0=K 1=V, head) for tests: device pointers to the
+/* Geometry of the compressed KV cache of (sequence, layer, kind 0=K 1=V, head) for tests: device pointers to the
  * fixed-part blocks, the unary arena and the per-token word offsets, plus words per token in the fixed part. */
 typedef struct cass_kv_view {
     const uint32_t* fixed; const uint32_t* arena; const uint32_t* offsets; const uint8_t* codebook;
     const void* k_or_v_bf16;
     int fixed_words_per_token, bitmap_words, arena_words;
 } cass_kv_view;
-int cass_kv_query(void* session, int layer, int kind, int head, cass_kv_view* h_view);
+int cass_kv_query(void* session, int seq, int layer, int kind, int head, cass_kv_view* h_view);
 
 /* Standalone draft attention / verify kernels are reached through cass_draft_step / cass_verify; the
  * activations of the last call can be inspected for tests: which = 0 hidden state after the last layer

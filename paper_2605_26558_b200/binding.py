@@ -148,6 +148,11 @@ def cass_draft_gemv(blob, info: BlobInfo, x_bf16, partial, y_bf16, y_f32, d_stat
                                                   _ptr(y_f32), _ptr(d_status), _stream(stream)))
 
 
+def cass_draft_gemv_batch(blob, info: BlobInfo, x_bf16, n_vec: int, partial, y_bf16, y_f32, d_status, stream=None):
+    _check("cass_draft_gemv_batch", lib.cass_draft_gemv_batch(_ptr(blob), C.byref(info), _ptr(x_bf16), n_vec, _ptr(partial),
+                                                              _ptr(y_bf16), _ptr(y_f32), _ptr(d_status), _stream(stream)))
+
+
 def cass_draft_gemv_static(blob, info: BlobInfo, x_bf16, y_bf16, y_f32, d_status, stream=None):
     """cass_draft_gemv with the partial sums in the library's built-in scratch: nothing is allocated, here or there."""
     _check("cass_draft_gemv_static", lib.cass_draft_gemv_static(_ptr(blob), C.byref(info), _ptr(x_bf16), _ptr(y_bf16),
@@ -186,6 +191,19 @@ def cass_session_status(session, stream=None) -> tuple[int, int]:
     return st.value, ln.value
 
 
+def cass_session_lens(session, batch: int, stream=None) -> list[int]:
+    buf = (C.c_int32 * max(batch, 8))()
+    _check("cass_session_lens", lib.cass_session_lens(session, buf, _stream(stream)))
+    return [int(buf[i]) for i in range(batch)]
+
+
+def cass_session_rows(desc: ModelDesc) -> int:
+    r = int(lib.cass_session_rows(C.byref(desc)))
+    if r < 0:
+        raise CassError("cass_session_rows", r)
+    return r
+
+
 def cass_calib_enable(session, on: bool, stream=None):
     _check("cass_calib_enable", lib.cass_calib_enable(session, int(on), _stream(stream)))
 
@@ -198,8 +216,8 @@ def cass_calib_norms(session, norms_out, stream=None):
     _check("cass_calib_norms", lib.cass_calib_norms(session, _ptr(norms_out), _stream(stream)))
 
 
-def cass_kv_append(session, layer: int, k_bf16, v_bf16, start_pos: int, n_new: int, flags: int, stream=None):
-    _check("cass_kv_append", lib.cass_kv_append(session, layer, _ptr(k_bf16), _ptr(v_bf16), start_pos, n_new, flags,
+def cass_kv_append(session, layer: int, k_bf16, v_bf16, start_pos: int, n_new: int, flags: int, stream=None, seq: int = 0):
+    _check("cass_kv_append", lib.cass_kv_append(session, seq, layer, _ptr(k_bf16), _ptr(v_bf16), start_pos, n_new, flags,
                                                 _stream(stream)))
 
 
@@ -211,8 +229,14 @@ def cass_set_len(session, n: int, stream=None):
     _check("cass_set_len", lib.cass_set_len(session, n, _stream(stream)))
 
 
-def cass_draft_step(session, tok_in, tok_out, logits_opt=None, stream=None):
-    _check("cass_draft_step", lib.cass_draft_step(session, _ptr(tok_in), _ptr(tok_out), _ptr(logits_opt), _stream(stream)))
+def cass_set_lens(session, lens, stream=None):
+    buf = (C.c_int32 * 8)(*[int(v) for v in lens])
+    _check("cass_set_lens", lib.cass_set_lens(session, buf, _stream(stream)))
+
+
+def cass_draft_step(session, tok_in, tok_out, logits_opt=None, stream=None, tok_stride: int = 1):
+    _check("cass_draft_step", lib.cass_draft_step(session, _ptr(tok_in), _ptr(tok_out), tok_stride, _ptr(logits_opt),
+                                                  _stream(stream)))
 
 
 def cass_verify(session, toks, g: int, target_argmax, logits_opt=None, stream=None):
@@ -229,20 +253,22 @@ def cass_verify_gemm_scratch_bytes(n: int, k: int) -> int:
 
 def cass_verify_gemm(w_bf16, x_bf16, rows: int, scratch, y_bf16, y_f32, d_status, stream=None):
     n, k = w_bf16.shape
-    assert x_bf16.shape[0] == 16 and x_bf16.shape[1] == k
+    assert x_bf16.shape[0] == (16 if rows <= 16 else 32 if rows <= 32 else 64) and x_bf16.shape[1] == k
     _check("cass_verify_gemm", lib.cass_verify_gemm(_ptr(w_bf16), _ptr(x_bf16), rows, n, k, _ptr(scratch),
                                                     C.c_size_t(scratch.numel() * scratch.element_size()), _ptr(y_bf16),
                                                     _ptr(y_f32), _ptr(d_status), _stream(stream)))
 
 
-def cass_accept(session, draft, target_argmax, g: int, n_accepted, out_tokens, next_tok, stream=None):
-    _check("cass_accept", lib.cass_accept(session, _ptr(draft), _ptr(target_argmax), g, _ptr(n_accepted),
-                                          _ptr(out_tokens), _ptr(next_tok), _stream(stream)))
+def cass_accept(session, draft, target_argmax, g: int, n_accepted, out_tokens, next_tok, stream=None,
+                draft_stride: int | None = None, next_stride: int = 1):
+    _check("cass_accept", lib.cass_accept(session, _ptr(draft), g if draft_stride is None else draft_stride,
+                                          _ptr(target_argmax), g, _ptr(n_accepted), _ptr(out_tokens), _ptr(next_tok),
+                                          next_stride, _stream(stream)))
 
 
-def cass_kv_query(session, layer: int, kind: int, head: int) -> KVView:
+def cass_kv_query(session, layer: int, kind: int, head: int, seq: int = 0) -> KVView:
     v = KVView()
-    _check("cass_kv_query", lib.cass_kv_query(session, layer, kind, head, C.byref(v)))
+    _check("cass_kv_query", lib.cass_kv_query(session, seq, layer, kind, head, C.byref(v)))
     return v
 
 

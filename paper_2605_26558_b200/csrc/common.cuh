@@ -49,7 +49,9 @@ inline int pdl_enabled() {
 constexpr int kRowsPerBlock = 32;          // rows (or tokens) interleaved in one superblock
 constexpr int kGroupCols = 8;              // kept columns per bitmap-walk group
 constexpr int kGroupCodes = 4;             // codewords per unary-walk group
-constexpr int kMaxVerifyRows = 16;
+constexpr int kMaxVerifyRows = 16;         // rows of one sequence in one verification call; also the margin kept at the end of a cache
+constexpr int kMaxBatch = 8;               // sequences per session
+constexpr int kMaxRows = 64;               // rows of all sequences in one call
 
 __host__ __device__ inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 __host__ __device__ inline size_t align_up(size_t a, size_t b) { return (a + b - 1) / b * b; }

@@ -181,18 +181,20 @@ __device__ __forceinline__ void kv_record_walk(const uint32_t* bmP, const uint32
 }
 
 template <int T>
-__global__ void __launch_bounds__(kDaThreads) k_draft_attn(KvGeom g, KvComp ck, KvComp cv, const uint16_t* __restrict__ qkv,
-                                                           int n_q, const DevState* __restrict__ st, AttnScratch sc,
+__global__ void __launch_bounds__(kDaThreads) k_draft_attn(KvGeom g, KvComp ck0, KvComp cv0, const uint16_t* __restrict__ qkv,
+                                                           int qkv_stride, int n_q, const DevState* __restrict__ st, AttnScratch sc,
                                                            int n_chunks_alloc) {
     extern __shared__ __align__(16) uint8_t smem[];
     pdl_launch_dependents();
     pdl_wait();
-    const int chunk = blockIdx.x, head = blockIdx.y;
-    const int cur_len = st->len + st->inflight + 1;            // positions visible to the drafted token
+    const int chunk = blockIdx.x, head = blockIdx.y, seq = blockIdx.z;
+    const int cur_len = st->len[seq] + st->inflight[seq] + 1;  // positions visible to the drafted token
     const int t0 = chunk * kDaTok;
     if (t0 >= cur_len) return;
     const int G = n_q / g.n_kv, d = g.d;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const KvComp ck = of_seq(ck0, seq, g.seq_stride), cv = of_seq(cv0, seq, g.seq_stride);
+    qkv += (size_t)seq * qkv_stride;
 
     float* q_s = reinterpret_cast<float*>(smem);                              // [d][8]
     float* sc_s = q_s + d * kMaxGroup;                                        // [8][64] scores -> probabilities
@@ -290,19 +292,20 @@ __global__ void __launch_bounds__(kDaThreads) k_draft_attn(KvGeom g, KvComp ck, 
         }
 #pragma unroll
         for (int gi = 0; gi < kMaxGroup; ++gi)
-            if (gi < G) sc.o[((size_t)(head * G + gi) * n_chunks_alloc + chunk) * d + dim] = acc[gi];
+            if (gi < G) sc.o[(((size_t)seq * n_q + head * G + gi) * n_chunks_alloc + chunk) * d + dim] = acc[gi];
     }
     if (tid < G) {
-        int hq = head * G + tid;
-        sc.m[(size_t)hq * n_chunks_alloc + chunk] = ml_s[tid * 2];
-        sc.l[(size_t)hq * n_chunks_alloc + chunk] = ml_s[tid * 2 + 1];
+        const size_t pair = (size_t)seq * n_q + head * G + tid;
+        sc.m[pair * n_chunks_alloc + chunk] = ml_s[tid * 2];
+        sc.l[pair * n_chunks_alloc + chunk] = ml_s[tid * 2 + 1];
     }
 }
 
 // Merge the chunk partials of every (row, query head): out = sum_c e^{m_c - M} o_c / sum_c e^{m_c - M} l_c.
-// Row r sees positions < len + (draft: inflight + 1 | verify: r + 1); chunks hold `chunk_tokens` positions.
+// Row r (the (r % rps)-th of sequence r / rps) sees positions < len + (draft: inflight + 1 | verify: r % rps + 1);
+// chunks hold `chunk_tokens` positions.
 // The reductions run in a fixed order that depends on the number of visible chunks only.
-__global__ void __launch_bounds__(128) k_attn_merge(AttnScratch sc, int n_chunks_alloc, int chunk_tokens, int n_q, int d,
+__global__ void __launch_bounds__(128) k_attn_merge(AttnScratch sc, int n_chunks_alloc, int chunk_tokens, int rps, int n_q, int d,
                                                     const DevState* __restrict__ st, int draft_mode, uint16_t* __restrict__ out) {
     extern __shared__ float w_s[];                  // [n_chunks_alloc] weights e^{m_c - M}
     __shared__ float s_red[4];
@@ -310,7 +313,8 @@ __global__ void __launch_bounds__(128) k_attn_merge(AttnScratch sc, int n_chunks
     pdl_wait();
     const int hq = blockIdx.x, r = blockIdx.y;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int vis = st->len + (draft_mode ? st->inflight + 1 : r + 1);
+    const int seq = r / rps;
+    const int vis = st->len[seq] + (draft_mode ? st->inflight[seq] + 1 : r % rps + 1);
     const int n_ch = ceil_div(vis, chunk_tokens);
     const size_t pair = (size_t)r * n_q + hq;
     const float* mp = sc.m + pair * n_chunks_alloc;
@@ -340,7 +344,7 @@ __global__ void __launch_bounds__(128) k_attn_merge(AttnScratch sc, int n_chunks
     }
 }
 
-int launch_attn_merge(const AttnScratch& sc, int n_chunks_alloc, int chunk_tokens, int rows, int n_q, int d,
+int launch_attn_merge(const AttnScratch& sc, int n_chunks_alloc, int chunk_tokens, int rows, int rps, int n_q, int d,
                       const DevState* st, int draft_mode, uint16_t* out, cudaStream_t s) {
     dim3 grid(n_q, rows);
     const size_t smem = (size_t)n_chunks_alloc * 4;
@@ -350,7 +354,7 @@ int launch_attn_merge(const AttnScratch& sc, int n_chunks_alloc, int chunk_token
         CASS_CUDA_CHECK(cudaFuncSetAttribute(k_attn_merge, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         attr = smem;
     }
-    CASS_PDL_LAUNCH(k_attn_merge, grid, dim3(128), smem, s, sc, n_chunks_alloc, chunk_tokens, n_q, d, st, draft_mode, out);
+    CASS_PDL_LAUNCH(k_attn_merge, grid, dim3(128), smem, s, sc, n_chunks_alloc, chunk_tokens, rps, n_q, d, st, draft_mode, out);
     return CASS_OK;
 }
 
@@ -359,13 +363,13 @@ size_t draft_attn_smem_bytes(const KvGeom& g) {
            (size_t)4 * (g.wpt + 1) * 32 * 4 + (size_t)4 * (kDaUnaStage + 2) * 32 * 4 + (size_t)kDaTok * g.d * 2 + 64;
 }
 
-int launch_draft_attn(const KvGeom& g, const KvComp& ck, const KvComp& cv, const uint16_t* qkv, int n_q,
-                      const DevState* st, const AttnScratch& sc, uint16_t* out, cudaStream_t s) {
+int launch_draft_attn(const KvGeom& g, const KvComp& ck, const KvComp& cv, const uint16_t* qkv, int qkv_stride, int n_q,
+                      int n_seq, const DevState* st, const AttnScratch& sc, uint16_t* out, cudaStream_t s) {
     const int G = n_q / g.n_kv;
     if (G > kMaxGroup || g.d > 256 || g.d % 32) return CASS_ERR_UNSUPPORTED;
     const int n_chunks = ceil_div(g.max_seq, kDaTok);
     const size_t smem = draft_attn_smem_bytes(g);
-    dim3 grid(n_chunks, g.n_kv);
+    dim3 grid(n_chunks, g.n_kv, n_seq);
 #define CASS_DA_LAUNCH(TT)                                                                                           \
     do {                                                                                                             \
         static size_t attr = 0;                                                                                      \
@@ -373,14 +377,14 @@ int launch_draft_attn(const KvGeom& g, const KvComp& ck, const KvComp& cv, const
             CASS_CUDA_CHECK(cudaFuncSetAttribute(k_draft_attn<TT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
             attr = smem;                                                                                             \
         }                                                                                                            \
-        CASS_PDL_LAUNCH(k_draft_attn<TT>, grid, dim3(kDaThreads), smem, s, g, ck, cv, qkv, n_q, st, sc, n_chunks);     \
+        CASS_PDL_LAUNCH(k_draft_attn<TT>, grid, dim3(kDaThreads), smem, s, g, ck, cv, qkv, qkv_stride, n_q, st, sc, n_chunks);     \
     } while (0)
     if (g.t == 4) CASS_DA_LAUNCH(4);
     else if (g.t == 0) CASS_DA_LAUNCH(0);
     else return CASS_ERR_UNSUPPORTED;
 #undef CASS_DA_LAUNCH
     CASS_LAUNCH_CHECK();
-    return launch_attn_merge(sc, n_chunks, kDaTok, 1, n_q, g.d, st, 1, out, s);
+    return launch_attn_merge(sc, n_chunks, kDaTok, n_seq, 1, n_q, g.d, st, 1, out, s);
 }
 
 }  // namespace cass

@@ -20,9 +20,13 @@ constexpr int kXSlack = 288;           // readable floats after the x slice: a w
 
 static size_t gemv_stage_bytes(const cass_blob_info& bi) { return align_up((size_t)bi.max_superblock_bytes + 256, 128); }
 
-size_t gemv_smem_bytes(const cass_blob_info& bi) {
+// Bytes per column of the x slice in shared memory: one vector is kept as fp32, several as packed bf16 [col][nb].
+__host__ __device__ constexpr int x_col_bytes(int nb) { return nb == 1 ? 4 : 2 * nb; }
+
+size_t gemv_smem_bytes(const cass_blob_info& bi, int nb) {
     const int n_ch = ceil_div(bi.seg_cols, bi.chunk_cols);
-    return kGemvStages * gemv_stage_bytes(bi) + (size_t)(bi.seg_cols + kXSlack) * 4 + 256 * 4 + (size_t)2 * n_ch * 32 * 4 + 64;
+    return kGemvStages * gemv_stage_bytes(bi) + (size_t)(bi.seg_cols + kXSlack) * x_col_bytes(nb) + 256 * 4 +
+           (size_t)(nb < 2 ? 2 : nb) * n_ch * 32 * 4 + 64;
 }
 
 __device__ __forceinline__ uint32_t shl_sat(uint32_t v, uint32_t s) {      // shift counts >= 32 give 0
@@ -42,17 +46,45 @@ __device__ __forceinline__ uint32_t mad_lo(uint32_t a, uint32_t b, uint32_t c) {
     return r;
 }
 
+template <int NB>
 struct WalkState {
-    float acc;
+    float acc[NB];
     uint32_t bpos, upos;
 };
 
+// The NB values of x at one column: raw words as they sit in shared memory, and their use in the accumulators.
+template <int NB>
+struct XRaw { uint32_t w[NB == 1 ? 1 : NB / 2]; };
+
+template <int NB>
+__device__ __forceinline__ XRaw<NB> x_load(uint32_t addr) {
+    XRaw<NB> r;
+    if constexpr (NB <= 2) asm volatile("ld.shared.u32 %0, [%1];" : "=r"(r.w[0]) : "r"(addr));
+    else if constexpr (NB == 4) asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(r.w[0]), "=r"(r.w[1]) : "r"(addr));
+    else asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r.w[0]), "=r"(r.w[1]), "=r"(r.w[2]), "=r"(r.w[3]) : "r"(addr));
+    return r;
+}
+
+template <int NB>
+__device__ __forceinline__ void x_fma(const XRaw<NB>& r, uint32_t wb, float (&acc)[NB]) {
+    const float w = __uint_as_float(wb);
+    if constexpr (NB == 1) {
+        acc[0] = fmaf(w, __uint_as_float(r.w[0]), acc[0]);
+    } else {
+#pragma unroll
+        for (int i = 0; i < NB / 2; ++i) {
+            acc[2 * i] = fmaf(w, __uint_as_float(r.w[i] << 16), acc[2 * i]);
+            acc[2 * i + 1] = fmaf(w, __uint_as_float(r.w[i] & 0xFFFF0000u), acc[2 * i + 1]);
+        }
+    }
+}
+
 // Careful walk of `count` (<= 8) kept values of one row from column bpos / code bit upos on: any gap between
 // kept columns, any codeword length.  Used for the rare groups that do not fit the 32-bit windows.
-template <int T>
-__device__ __noinline__ WalkState group_slow(const uint32_t* bmS, const uint32_t* unS, const uint32_t* flG, int count,
-                                             WalkState st, uint32_t bpos_lim, uint32_t upos_lim, const float* xs,
-                                             const uint32_t* lut) {
+template <int T, int NB>
+__device__ __noinline__ WalkState<NB> group_slow(const uint32_t* bmS, const uint32_t* unS, const uint32_t* flG, int count,
+                                                 WalkState<NB> st, uint32_t bpos_lim, uint32_t upos_lim, const float* xs,
+                                                 const uint32_t* lut) {
     constexpr int F = 8 - T, PER = 32 / F;
     constexpr uint32_t MASK = 0x80000000u | (((1u << (7 - T)) - 1u) << (16 + T));
     for (int e = 0; e < count; ++e) {
@@ -63,12 +95,12 @@ __device__ __noinline__ WalkState group_slow(const uint32_t* bmS, const uint32_t
             st.bpos = (st.bpos | 31u) + 1u;
         }
         if (!found) break;                                   // corrupt stream: stop inside the buffers
-        const float xv = xs[st.bpos];
+        const XRaw<NB> xv = x_load<NB>(smem_u32(xs) + st.bpos * (uint32_t)x_col_bytes(NB));
         st.bpos += 1;
         const int rank = read_unary(unS, st.upos, upos_lim);
         const uint32_t fword = flG[(e / PER) * 32];
         const uint32_t a = __funnelshift_l(fword, fword, (F * (e % PER)) & 31);
-        st.acc = fmaf(__uint_as_float((a & MASK) | lut[rank & 255]), xv, st.acc);
+        x_fma<NB>(xv, (a & MASK) | lut[rank & 255], st.acc);
     }
     return st;
 }
@@ -90,13 +122,14 @@ __device__ __forceinline__ uint32_t lds_u32_off(uint32_t addr) {
 // codewords.  A group whose 8 kept columns span more than 32 columns, or whose 4 codewords take more than 32 bits,
 // shows up as a window that ran dry (no bit left to find); that lane then redoes the group with the careful
 // walk while the others wait.  The walk addresses shared memory through 32-bit shared-space addresses.
-template <int T>
-__device__ __forceinline__ float chunk_dot_fast(const uint32_t* __restrict__ sb, const SbGeom& g, int ch, int lane,
-                                                int chunk_elems, const float* __restrict__ xs,
-                                                const uint32_t* __restrict__ lut) {
+template <int T, int NB>
+__device__ __forceinline__ void chunk_dot_fast(const uint32_t* __restrict__ sb, const SbGeom& g, int ch, int lane,
+                                               int chunk_elems, const float* __restrict__ xs,
+                                               const uint32_t* __restrict__ lut, float (&acc)[NB]) {
     constexpr int F = 8 - T, PER = 32 / F, NFW = kGroupCols / PER;       // field words per group of 8
     constexpr uint32_t MASK = 0x80000000u | (((1u << (7 - T)) - 1u) << (16 + T));   // sign + kept mantissa of a binary32
     static_assert(32 % F == 0 && (PER == 4 || PER == 8), "fast path: rotated fields, 4 or 8 per word");
+    constexpr uint32_t XS = (uint32_t)x_col_bytes(NB);            // bytes per column of the x slice
     const uint32_t e0 = sb[g.tab + ch * 32 + lane];            // where this row's value ch * chunk_elems sits
     const uint32_t fw = (uint32_t)(ch * chunk_elems) / PER;    // its field word (chunk_elems is a multiple of 8)
     uint32_t upos = e0 & 0xFFFFFu;
@@ -112,7 +145,6 @@ __device__ __forceinline__ float chunk_dot_fast(const uint32_t* __restrict__ sb,
     const int n_groups = ceil_div(__reduce_max_sync(0xffffffffu, m), kGroupCols);
     uint32_t bpos = e0 >> 20;
     const uint32_t bpos_lim = (uint32_t)(g.bm_words * 32), upos_lim = (uint32_t)(g.w_u * 32);
-    float acc = 0.f;
 
     // Bit positions are counted from the least significant end (bfind): a window keeps its place and the bit
     // just used is cleared, so a kept column is x[bpos + 31 - p] and a codeword's rank is the distance between two
@@ -120,10 +152,13 @@ __device__ __forceinline__ float chunk_dot_fast(const uint32_t* __restrict__ sb,
     // position of each window tells whether the whole group fitted.
     auto group = [&](int grp, auto tail_c) {
         constexpr bool tail = decltype(tail_c)::value;         // two specialisations: full groups carry no per-value tests
-        const WalkState st0 = {acc, bpos, upos};
+        WalkState<NB> st0;
+#pragma unroll
+        for (int b = 0; b < NB; ++b) st0.acc[b] = acc[b];
+        st0.bpos = bpos; st0.upos = upos;
         const uint32_t ba = bm_a + (bpos >> 5) * 128u;
         uint32_t bv = __funnelshift_l(lds_u32_off<128>(ba), lds_u32(ba), bpos);    // 32 columns from bpos on
-        const uint32_t xg = xs_a + bpos * 4u + 124u;                               // address of x[bpos + 31]
+        const uint32_t xg = xs_a + bpos * XS + 31u * XS;                           // address of x[bpos + 31]
         uint32_t fwd[NFW];
         fwd[0] = lds_u32(fl_a);
         if (NFW > 1) fwd[NFW - 1] = lds_u32_off<128>(fl_a);
@@ -140,8 +175,7 @@ __device__ __forceinline__ float chunk_dot_fast(const uint32_t* __restrict__ sb,
             for (int j = 0; j < kGroupCodes; ++j) {
                 const int e = half * kGroupCodes + j;
                 p = bfind_u32(bv);                                   // next kept column
-                float xv;
-                asm volatile("ld.shared.f32 %0, [%1];" : "=f"(xv) : "r"(mad_lo(p, 0xFFFFFFFCu, xg)));
+                const XRaw<NB> xv = x_load<NB>(mad_lo(p, 0u - XS, xg));
                 bv &= ~shl_sat(1u, p);
                 q = bfind_u32(uv);                                   // next terminator
                 const uint32_t eb = lds_u32(mad_lo(q, 0xFFFFFFFCu, la));          // lut[previous - q - 1]
@@ -151,9 +185,9 @@ __device__ __forceinline__ float chunk_dot_fast(const uint32_t* __restrict__ sb,
                 const uint32_t a = __funnelshift_l(fword, fword, (F * (e % PER)) & 31);
                 const uint32_t wb = (a & MASK) | eb;
                 if (!tail) {
-                    acc = fmaf(__uint_as_float(wb), xv, acc);
+                    x_fma<NB>(xv, wb, acc);
                 } else if (e < rem) {
-                    acc = fmaf(__uint_as_float(wb), xv, acc);
+                    x_fma<NB>(xv, wb, acc);
                     dry |= p | q;
                 }
             }
@@ -165,9 +199,11 @@ __device__ __forceinline__ float chunk_dot_fast(const uint32_t* __restrict__ sb,
         if (tail) bpos = min(bpos, bpos_lim);
         else dry |= p;
         if ((int32_t)dry < 0) {
-            const WalkState r = group_slow<T>(bmS, unS, flS + (fw + grp * NFW) * 32, min(rem, kGroupCols), st0, bpos_lim,
-                                              upos_lim, xs, lut);
-            acc = r.acc; bpos = r.bpos; upos = r.upos;
+            const WalkState<NB> r = group_slow<T, NB>(bmS, unS, flS + (fw + grp * NFW) * 32, min(rem, kGroupCols), st0, bpos_lim,
+                                                      upos_lim, xs, lut);
+#pragma unroll
+            for (int b = 0; b < NB; ++b) acc[b] = r.acc[b];
+            bpos = r.bpos; upos = r.upos;
         }
         fl_a += NFW * 128u;
     };
@@ -175,12 +211,13 @@ __device__ __forceinline__ float chunk_dot_fast(const uint32_t* __restrict__ sb,
     int grp = 0;
     for (; grp < n_full; ++grp) group(grp, std::false_type{});
     for (; grp < n_groups; ++grp) group(grp, std::true_type{});
-    return acc;
 }
 
 // T >= 0: fast path for regular chunks, generic path otherwise.  T = -1: generic path only (any t).
 // grid = (n_seg, G): CTA (seg, j) handles the superblocks (rb, seg) for rb = j, j + G, ...
-template <int T>
+// NB vectors x[b] (bf16 [NB][k]) are multiplied in the same pass: every decoded weight is used NB times, and each
+// vector's sums are formed in the same order as with NB = 1.
+template <int T, int NB>
 __global__ void __launch_bounds__(1024) k_draft_gemv(const uint32_t* __restrict__ blob, const uint16_t* __restrict__ x,
                                                      float* __restrict__ partial, int32_t* __restrict__ d_status,
                                                      int stage_bytes, int max_sb, int n, int k, int t, int seg_cols,
@@ -196,9 +233,9 @@ __global__ void __launch_bounds__(1024) k_draft_gemv(const uint32_t* __restrict_
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, n_warps = blockDim.x >> 5;
 
     float* xs = reinterpret_cast<float*>(smem_raw + (size_t)kGemvStages * stage_bytes);
-    uint32_t* lut = reinterpret_cast<uint32_t*>(xs + seg_cols + kXSlack);
-    float* red = reinterpret_cast<float*>(lut + 256);                       // [2][n_warps][32]
-    uint64_t* bar = reinterpret_cast<uint64_t*>(red + 2 * n_warps * 32);    // [kGemvStages]
+    uint32_t* lut = reinterpret_cast<uint32_t*>(reinterpret_cast<uint8_t*>(xs) + (size_t)(seg_cols + kXSlack) * x_col_bytes(NB));
+    float* red = reinterpret_cast<float*>(lut + 256);                       // NB = 1: [2][n_warps][32], else [NB][n_warps][32]
+    uint64_t* bar = reinterpret_cast<uint64_t*>(red + (NB < 2 ? 2 : NB) * n_warps * 32);    // [kGemvStages]
     __shared__ int s_skip[kGemvStages];
 
     const int scols = seg_cols_of(k_pad, seg_cols, seg);
@@ -247,7 +284,29 @@ __global__ void __launch_bounds__(1024) k_draft_gemv(const uint32_t* __restrict_
     pdl_wait();
     // x of this segment (fp32), zero beyond the matrix
     const int c0 = seg * seg_cols;
-    if ((k & 7) == 0 && ((uintptr_t)x & 15) == 0) {
+    if constexpr (NB > 1) {
+        // packed bf16 [col][NB]: all vectors' values of one column side by side
+        uint16_t* xs16 = reinterpret_cast<uint16_t*>(xs);
+        if ((k & 7) == 0 && ((uintptr_t)x & 15) == 0) {
+            const int n_oct = (seg_cols + kXSlack) / 8;
+            for (int it = tid; it < n_oct * NB; it += blockDim.x) {
+                const int i = (it / NB) * 8, b = it % NB;
+                uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                if (i < scols && c0 + i < k) v = *reinterpret_cast<const uint4*>(x + (size_t)b * k + c0 + i);
+                const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    xs16[(size_t)(i + 2 * q) * NB + b] = (uint16_t)(w[q] & 0xFFFFu);
+                    xs16[(size_t)(i + 2 * q + 1) * NB + b] = (uint16_t)(w[q] >> 16);
+                }
+            }
+        } else {
+            for (int it = tid; it < (seg_cols + kXSlack) * NB; it += blockDim.x) {
+                const int i = it / NB, b = it % NB, c = c0 + i;
+                xs16[it] = (i < scols && c < k) ? x[(size_t)b * k + c] : (uint16_t)0;
+            }
+        }
+    } else if ((k & 7) == 0 && ((uintptr_t)x & 15) == 0) {
         // eight values per 16-byte load: one round trip to L2 for the whole slice
         for (int i = tid * 8; i < seg_cols + kXSlack; i += blockDim.x * 8) {
             uint4 v = make_uint4(0u, 0u, 0u, 0u);
@@ -285,43 +344,66 @@ __global__ void __launch_bounds__(1024) k_draft_gemv(const uint32_t* __restrict_
             return;
         }
         const uint32_t* sb = reinterpret_cast<const uint32_t*>(smem_raw + (size_t)s * stage_bytes);
-        float acc = 0.f;
+        float acc[NB];
+#pragma unroll
+        for (int b = 0; b < NB; ++b) acc[b] = 0.f;
         if (warp < n_ch && !s_skip[s]) {
             const uint32_t* dir = blob + kBlobDirOffset / 4 + (rb * n_seg + seg) * 4;
             const SbGeom g = SbGeom::make(n_ch, scols, (int)dir[1], (int)dir[2]);
             if (T >= 0) {
-                acc = chunk_dot_fast<(T >= 0 ? T : 0)>(sb, g, warp, lane, dir_chunk_elems(dir[3]), xs, lut);
+                chunk_dot_fast<(T >= 0 ? T : 0), NB>(sb, g, warp, lane, dir_chunk_elems(dir[3]), xs, lut, acc);
             } else {
+                const uint32_t xs_a = smem_u32(xs);
                 decode_chunk_generic(sb, g, dir_chunk_elems(dir[3]), warp, lane, t, cb, [&](int col, uint16_t bits) {
-                    acc = fmaf(bf16_bits_to_float(bits), xs[col], acc);
+                    x_fma<NB>(x_load<NB>(xs_a + (uint32_t)col * (uint32_t)x_col_bytes(NB)), (uint32_t)bits << 16, acc);
                 });
             }
         }
-        float* red_i = red + (i & 1) * n_warps * 32;
-        red_i[warp * 32 + lane] = acc;
-        __syncthreads();                              // all reads of stage s are done; partial sums are visible
-        if (tid == 0 && i + kGemvStages < n_tiles) {
-            fence_proxy_async();
-            issue(i + kGemvStages);
-        }
-        if (warp == 0) {
-            float sum = 0.f;
-            for (int w = 0; w < n_ch; ++w) sum += red_i[w * 32 + lane];
-            int row = rb * kRowsPerBlock + lane;
-            if (row < n) partial[(size_t)seg * (n_rb * kRowsPerBlock) + row] = sum;
+        const size_t n_pad = (size_t)n_rb * kRowsPerBlock;
+        const int row = rb * kRowsPerBlock + lane;
+        if constexpr (NB == 1) {
+            float* red_i = red + (i & 1) * n_warps * 32;
+            red_i[warp * 32 + lane] = acc[0];
+            __syncthreads();                              // all reads of stage s are done; partial sums are visible
+            if (tid == 0 && i + kGemvStages < n_tiles) {
+                fence_proxy_async();
+                issue(i + kGemvStages);
+            }
+            if (warp == 0) {
+                float sum = 0.f;
+                for (int w = 0; w < n_ch; ++w) sum += red_i[w * 32 + lane];
+                if (row < n) partial[(size_t)seg * n_pad + row] = sum;
+            }
+        } else {
+#pragma unroll
+            for (int b = 0; b < NB; ++b) red[(b * n_warps + warp) * 32 + lane] = acc[b];
+            __syncthreads();
+            if (tid == 0 && i + kGemvStages < n_tiles) {
+                fence_proxy_async();
+                issue(i + kGemvStages);
+            }
+            for (int b = warp; b < NB; b += n_warps) {    // vector b's chunk sums, added in chunk order as with NB = 1
+                float sum = 0.f;
+                for (int w = 0; w < n_ch; ++w) sum += red[(b * n_warps + w) * 32 + lane];
+                if (row < n) partial[((size_t)b * n_seg + seg) * n_pad + row] = sum;
+            }
+            __syncthreads();                              // the sums are read before the next tile overwrites them
         }
     }
 }
 
+// grid.y = vector b: partial [b][n_seg][n_pad] -> y [b][n]
 __global__ void k_gemv_finish(const float* __restrict__ partial, int n, int n_pad, int n_seg,
                               uint16_t* __restrict__ y_bf16, float* __restrict__ y_f32) {
     pdl_wait();
     int r = blockIdx.x * blockDim.x + threadIdx.x;
     if (r >= n) return;
+    const int b = blockIdx.y;
+    partial += (size_t)b * n_seg * n_pad;
     float acc = 0.f;
     for (int s = 0; s < n_seg; ++s) acc += partial[(size_t)s * n_pad + r];
-    if (y_f32) y_f32[r] = acc;
-    if (y_bf16) y_bf16[r] = float_to_bf16_bits(acc);
+    if (y_f32) y_f32[(size_t)b * n + r] = acc;
+    if (y_bf16) y_bf16[(size_t)b * n + r] = float_to_bf16_bits(acc);
 }
 
 static int sm_count() {
@@ -334,11 +416,12 @@ static int sm_count() {
     return n;
 }
 
-int launch_draft_gemv(const void* blob, const cass_blob_info& bi, const void* x_bf16, float* partial,
+int launch_draft_gemv(const void* blob, const cass_blob_info& bi, const void* x_bf16, int nb, float* partial,
                       int32_t* d_status, cudaStream_t stream) {
     const int n_ch = ceil_div(bi.seg_cols, bi.chunk_cols);
     if (n_ch > 32) return CASS_ERR_UNSUPPORTED;
-    const size_t smem = gemv_smem_bytes(bi);
+    if (nb != 1 && nb != 2 && nb != 4 && nb != 8) return CASS_ERR_UNSUPPORTED;
+    const size_t smem = gemv_smem_bytes(bi, nb);
     if (smem > 227 * 1024) return CASS_ERR_CAPACITY;
     const int threads = 32 * n_ch;
     int per_sm = (int)((228 * 1024) / (smem + 1024));
@@ -351,11 +434,11 @@ int launch_draft_gemv(const void* blob, const cass_blob_info& bi, const void* x_
     const uint32_t* b = (const uint32_t*)blob;
     const uint16_t* x = (const uint16_t*)x_bf16;
     const int stage = (int)gemv_stage_bytes(bi);
-#define CASS_GEMV_LAUNCH(TT)                                                                                   \
+#define CASS_GEMV_LAUNCH(TT, NN)                                                                               \
     do {                                                                                                       \
         static int attr_smem = 0;      /* largest size already granted to this instantiation */              \
         if ((int)smem > attr_smem) {                                                                           \
-            CASS_CUDA_CHECK(cudaFuncSetAttribute(k_draft_gemv<TT>, cudaFuncAttributeMaxDynamicSharedMemorySize,\
+            CASS_CUDA_CHECK(cudaFuncSetAttribute(k_draft_gemv<TT, NN>, cudaFuncAttributeMaxDynamicSharedMemorySize,\
                                                  (int)smem));                                                  \
             attr_smem = (int)smem;                                                                             \
         }                                                                                                      \
@@ -365,14 +448,22 @@ int launch_draft_gemv(const void* blob, const cass_blob_info& bi, const void* x_
         at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   /* prologue may overlap the predecessor */ \
         at[0].val.programmaticStreamSerializationAllowed = pdl_enabled();                                                  \
         cfg.attrs = at; cfg.numAttrs = 1;                                                                      \
-        CASS_CUDA_CHECK(cudaLaunchKernelEx(&cfg, k_draft_gemv<TT>, b, x, partial, d_status, stage,             \
+        CASS_CUDA_CHECK(cudaLaunchKernelEx(&cfg, k_draft_gemv<TT, NN>, b, x, partial, d_status, stage,         \
                                            (int)bi.max_superblock_bytes, (int)bi.rows, (int)bi.cols,           \
                                            (int)bi.trunc_bits, (int)bi.seg_cols, (int)bi.chunk_cols,           \
                                            (int)bi.n_seg, (int)bi.n_rowblocks));                               \
     } while (0)
-    if (bi.trunc_bits == 4) CASS_GEMV_LAUNCH(4);
-    else if (bi.trunc_bits == 0) CASS_GEMV_LAUNCH(0);
-    else CASS_GEMV_LAUNCH(-1);
+#define CASS_GEMV_LAUNCH_NB(TT)                                                                                \
+    do {                                                                                                       \
+        if (nb == 1) CASS_GEMV_LAUNCH(TT, 1);                                                                  \
+        else if (nb == 2) CASS_GEMV_LAUNCH(TT, 2);                                                             \
+        else if (nb == 4) CASS_GEMV_LAUNCH(TT, 4);                                                             \
+        else CASS_GEMV_LAUNCH(TT, 8);                                                                          \
+    } while (0)
+    if (bi.trunc_bits == 4) CASS_GEMV_LAUNCH_NB(4);
+    else if (bi.trunc_bits == 0) CASS_GEMV_LAUNCH_NB(0);
+    else CASS_GEMV_LAUNCH_NB(-1);
+#undef CASS_GEMV_LAUNCH_NB
 #undef CASS_GEMV_LAUNCH
     CASS_LAUNCH_CHECK();
     return CASS_OK;
@@ -386,12 +477,27 @@ extern "C" int cass_draft_gemv(const void* blob, const cass_blob_info* h_info, c
                                void* y_bf16, float* y_f32, int32_t* d_status, void* stream_) {
     if (!blob || !h_info || !x_bf16 || !partial) return CASS_ERR_INVALID_ARG;
     cudaStream_t stream = (cudaStream_t)stream_;
-    int rc = launch_draft_gemv(blob, *h_info, x_bf16, partial, d_status, stream);
+    int rc = launch_draft_gemv(blob, *h_info, x_bf16, 1, partial, d_status, stream);
     if (rc) return rc;
     if (!y_bf16 && !y_f32) return CASS_OK;
     int n_pad = h_info->n_rowblocks * kRowsPerBlock;
     k_gemv_finish<<<ceil_div(h_info->rows, 256), 256, 0, stream>>>(partial, h_info->rows, n_pad, h_info->n_seg,
                                                                     (uint16_t*)y_bf16, y_f32);
+    CASS_LAUNCH_CHECK();
+    return CASS_OK;
+}
+
+extern "C" int cass_draft_gemv_batch(const void* blob, const cass_blob_info* h_info, const void* x_bf16, int n_vec,
+                                     float* partial, void* y_bf16, float* y_f32, int32_t* d_status, void* stream_) {
+    if (!blob || !h_info || !x_bf16 || !partial) return CASS_ERR_INVALID_ARG;
+    if (n_vec != 1 && n_vec != 2 && n_vec != 4 && n_vec != 8) return CASS_ERR_INVALID_ARG;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    int rc = launch_draft_gemv(blob, *h_info, x_bf16, n_vec, partial, d_status, stream);
+    if (rc) return rc;
+    if (!y_bf16 && !y_f32) return CASS_OK;
+    int n_pad = h_info->n_rowblocks * kRowsPerBlock;
+    k_gemv_finish<<<dim3(ceil_div(h_info->rows, 256), n_vec), 256, 0, stream>>>(partial, h_info->rows, n_pad, h_info->n_seg,
+                                                                                 (uint16_t*)y_bf16, y_f32);
     CASS_LAUNCH_CHECK();
     return CASS_OK;
 }
@@ -421,7 +527,7 @@ extern "C" int cass_draft_gemv_static(const void* blob, const cass_blob_info* h_
     }
     float* partial = s_scratch[dev];
     cudaStream_t stream = (cudaStream_t)stream_;
-    int rc = launch_draft_gemv(blob, *h_info, x_bf16, partial, d_status, stream);
+    int rc = launch_draft_gemv(blob, *h_info, x_bf16, 1, partial, d_status, stream);
     if (rc) return rc;
     const int n_pad = h_info->n_rowblocks * kRowsPerBlock;
     k_gemv_finish<<<ceil_div(h_info->rows, 256), 256, 0, stream>>>(partial, h_info->rows, n_pad, h_info->n_seg,

@@ -5,15 +5,17 @@
 
 namespace cass {
 
-// Device-resident step state of one sequence; kernels read positions from here so that a captured graph of
-// launches can be replayed without host-side position arguments.
+// Device-resident step state of the session's sequences; kernels read positions from here so that a captured
+// graph of launches can be replayed without host-side position arguments.
 struct DevState {
-    int32_t len;        // committed KV positions
-    int32_t inflight;   // draft tokens appended since the last accept
+    int32_t len[kMaxBatch];        // committed KV positions of each sequence
+    int32_t inflight[kMaxBatch];   // draft tokens appended since the last accept
     int32_t status;     // first device-side error (CASS_ERR_*), 0 if none
     int32_t calib_on;
     int32_t max_seq;    // KV positions per sequence; len never moves past max_seq - kMaxVerifyRows
 };
+
+// Row r of a call with `rps` rows per sequence belongs to sequence r / rps and is its (r % rps)-th new row.
 
 // Compressed KV cache of one (layer, K|V): per head a fixed part (bitmap + fields, 32-token blocks interleaved
 // word by word), an append-only arena of unary words and per-token word offsets.
@@ -28,7 +30,21 @@ struct KvComp {
 
 struct KvGeom {
     int n_kv, d, max_seq, n_blocks, wpt, bm_words, f_words, kept, n_prune, t, arena_words;
+    size_t seq_stride;      // bytes between the KV storage (both caches, all layers) of consecutive sequences
 };
+
+// The same object of sequence b: every sequence's KV storage has the same internal layout.
+template <class P>
+__host__ __device__ __forceinline__ P* of_seq(P* p, int b, size_t seq_stride) {
+    return reinterpret_cast<P*>(reinterpret_cast<uintptr_t>(p) + (size_t)b * seq_stride);
+}
+__host__ __device__ __forceinline__ KvComp of_seq(const KvComp& c, int b, size_t seq_stride) {
+    KvComp r;
+    r.fixed = of_seq(c.fixed, b, seq_stride); r.arena = of_seq(c.arena, b, seq_stride); r.off = of_seq(c.off, b, seq_stride);
+    r.rank_to_exp = of_seq(c.rank_to_exp, b, seq_stride); r.exp_to_rank = of_seq(c.exp_to_rank, b, seq_stride);
+    r.hist = of_seq(c.hist, b, seq_stride);
+    return r;
+}
 
 // fp32 split-K partial sums of a projection: element (row r, feature i) of part s sits at p[s * seg_stride + r * row_stride + i];
 // consumers add the parts in order and round to bf16 where the projection output is a bf16 activation.
@@ -40,42 +56,51 @@ struct Partials {
 
 constexpr int kAttnChunk = 64;       // split-K granularity over the sequence (fixed absolute boundaries)
 
-size_t gemv_smem_bytes(const cass_blob_info& bi);
-// partial: fp32 [n_seg][n_rowblocks*32]; the caller sums the segments (fixed order) afterwards.
-int launch_draft_gemv(const void* blob, const cass_blob_info& bi, const void* x_bf16, float* partial,
+size_t gemv_smem_bytes(const cass_blob_info& bi, int nb);
+// x: bf16 [nb][cols], nb in {1, 2, 4, 8} vectors multiplied in one pass over the blob.
+// partial: fp32 [nb][n_seg][n_rowblocks*32]; the caller sums the segments (fixed order) afterwards.
+int launch_draft_gemv(const void* blob, const cass_blob_info& bi, const void* x_bf16, int nb, float* partial,
                       int32_t* d_status, cudaStream_t stream);
+inline Partials draft_gemv_partials(const float* partial, const cass_blob_info& bi) {
+    const size_t n_pad = (size_t)bi.n_rowblocks * kRowsPerBlock;
+    return Partials{partial, bi.n_seg, n_pad, (size_t)bi.n_seg * n_pad};
+}
 
 // ---- small ops (ops.cu) -------------------------------------------------------------------------------
 int launch_rope_table(float* cos_t, float* sin_t, int max_seq, int d, float theta, cudaStream_t s);
-int launch_embed(const int32_t* toks, const uint16_t* embed, uint16_t* h, int rows, int hidden, cudaStream_t s);
+// row r takes token toks[r * tok_stride]
+int launch_embed(const int32_t* toks, int tok_stride, const uint16_t* embed, uint16_t* h, int rows, int hidden, cudaStream_t s);
 int launch_rmsnorm(const uint16_t* h, const uint16_t* gain, uint16_t* out, int rows, int hidden, float eps,
                    cudaStream_t s);
 // h = bf16(h + y); out = rmsnorm(h) * gain.  y comes either as bf16 [rows][hidden] or (rows == 1) as fp32 split-K
 // partials [n_seg][n_pad] that are summed in segment order and rounded to bf16 first.
 int launch_residual_rmsnorm(uint16_t* h, const uint16_t* y_bf16, Partials pp,
                             const uint16_t* gain, uint16_t* out, int rows, int hidden, float eps, cudaStream_t s);
-// q and k of qkv (bf16 [rows][qkv_dim]) rotated in place at position base + row (base from state: len, or
-// len + inflight when use_inflight).  With partial != NULL (rows == 1) qkv is first formed from the partials.
+// q and k of qkv (bf16 [rows][qkv_dim]) rotated in place at the row's position: len (+ inflight when use_inflight)
+// of its sequence + its index among the sequence's rps rows.  With partials, qkv is first formed from them.
 int launch_qkv_rope(uint16_t* qkv, Partials pp, const float* cos_t, const float* sin_t,
-                    const DevState* st, int use_inflight, int rows, int n_q, int n_kv, int d, cudaStream_t s);
+                    const DevState* st, int use_inflight, int rows, int rps, int n_q, int n_kv, int d, cudaStream_t s);
 int launch_swiglu(const uint16_t* gu_bf16, Partials pp, uint16_t* act, int rows,
                   int ffn, cudaStream_t s);
-// logits (fp32 [rows][vocab], or formed from partials when rows == 1) -> lowest-index argmax per row; optional copy
-// of the logits; bump_inflight adds 1 to the draft counter afterwards.
-// tmp_v / tmp_i: scratch of 16 x 128 entries each.
-int launch_argmax(const float* logits, Partials pp, int rows, int vocab, int32_t* out,
+// logits (fp32 [rows][vocab], or formed from partials) -> lowest-index argmax per row; optional copy
+// of the logits; bump_inflight adds 1 to the draft counter of sequence r (one row per sequence) afterwards.
+// tmp_v / tmp_i: scratch of kMaxRows x 128 entries each.
+// Row r's token goes to out[r * out_stride].
+int launch_argmax(const float* logits, Partials pp, int rows, int vocab, int32_t* out, int out_stride,
                   float* logits_copy, float* tmp_v, int32_t* tmp_i, DevState* st, int bump_inflight, cudaStream_t s);
-int launch_accept(DevState* st, const int32_t* draft, const int32_t* target, int g, int32_t* n_acc,
-                  int32_t* out_tokens, int32_t* next_tok, cudaStream_t s);
+int launch_accept(DevState* st, int n_seq, const int32_t* draft, int draft_stride, const int32_t* target, int g, int32_t* n_acc,
+                  int32_t* out_tokens, int32_t* next_tok, int next_stride, cudaStream_t s);
 int launch_calib_accum(const uint16_t* x, int rows, int cols, float* sumsq, const DevState* st, cudaStream_t s);
 int launch_sqrt(const float* in, float* out, size_t n, cudaStream_t s);
 
 // ---- KV encoder (kv.cu) -------------------------------------------------------------------------------
-// src_k/src_v: bf16 rows with `row_stride` elements between tokens and n_kv*d contiguous per token.
+// Appends n_new tokens to each of the n_seq sequences seq0 .. seq0 + n_seq - 1 (caches given for sequence 0).
+// src_k/src_v: bf16 rows with `row_stride` elements between tokens and n_kv*d contiguous per token; the rows of the
+// i-th sequence of the call start at row i * n_new.
 // start_pos < 0: take the position from the state (len, or len + inflight when use_inflight).
 int launch_kv_append(const KvGeom& g, const KvComp& ck, const KvComp& cv, uint16_t* k_cache, uint16_t* v_cache,
                      const uint16_t* src_k, const uint16_t* src_v, int row_stride, int start_pos, int use_inflight,
-                     int n_new, int flags, DevState* st, cudaStream_t s);
+                     int n_new, int flags, DevState* st, int seq0, int n_seq, cudaStream_t s);
 int launch_kv_codebook(const KvGeom& g, const KvComp& ck, const KvComp& cv, const uint16_t* k_cache,
                        const uint16_t* v_cache, int n_tokens, cudaStream_t s);
 
@@ -85,19 +110,22 @@ struct AttnScratch {
     float* m;     // [rows*n_q][n_chunks]
     float* l;     // [rows*n_q][n_chunks]
 };
-// Draft: one query row at position len + inflight over the compressed cache.
-int launch_draft_attn(const KvGeom& g, const KvComp& ck, const KvComp& cv, const uint16_t* qkv, int n_q,
-                      const DevState* st, const AttnScratch& sc, uint16_t* out, cudaStream_t s);
-// Verify: rows at positions len + r over the bf16 cache, causal.
+// Draft: one query row per sequence (qkv row b, `qkv_stride` elements apart) at position len + inflight over that
+// sequence's compressed cache (caches given for sequence 0).
+int launch_draft_attn(const KvGeom& g, const KvComp& ck, const KvComp& cv, const uint16_t* qkv, int qkv_stride, int n_q,
+                      int n_seq, const DevState* st, const AttnScratch& sc, uint16_t* out, cudaStream_t s);
+// Verify: rps rows per sequence at positions len + i over that sequence's bf16 cache, causal.
 int launch_verify_attn(const KvGeom& g, const uint16_t* k_cache, const uint16_t* v_cache, const uint16_t* qkv,
-                       int rows, int n_q, const DevState* st, const AttnScratch& sc, uint16_t* out, cudaStream_t s);
+                       int n_seq, int rps, int n_q, const DevState* st, const AttnScratch& sc, uint16_t* out, cudaStream_t s);
 
 // ---- verification GEMM (verify_gemm.cu): Y[r][n] = sum_k W[n][k] X[r][k], bf16 in, fp32 accumulate (tcgen05) ----
-// X is a buffer of 16 rows of k values (the first `rows` are used); partial: fp32 scratch of verify_gemm_partial_floats.
-// With both outputs null only the partial sums are produced: [splits][16][n], see verify_gemm_partials().
-size_t verify_gemm_partial_floats(int n, int k);
-Partials verify_gemm_partials(const float* partial, int n, int k);
-int launch_verify_gemm(const uint16_t* W, const uint16_t* X, int rows, int n, int k, float* partial, uint16_t* y_bf16,
+// X is a buffer of `bn` rows of k values (bn = 16, 32 or 64 token columns of the MMA; the first `rows` are used);
+// partial: fp32 scratch of verify_gemm_partial_floats.
+// With both outputs null only the partial sums are produced: [splits][bn][n], see verify_gemm_partials().
+inline int verify_gemm_bn(int rows) { return rows <= 16 ? 16 : rows <= 32 ? 32 : 64; }
+size_t verify_gemm_partial_floats(int n, int k, int bn);
+Partials verify_gemm_partials(const float* partial, int n, int k, int bn);
+int launch_verify_gemm(const uint16_t* W, const uint16_t* X, int rows, int bn, int n, int k, float* partial, uint16_t* y_bf16,
                        float* y_f32, int32_t* d_status, cudaStream_t s);
 
 }  // namespace cass

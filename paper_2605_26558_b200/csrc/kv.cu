@@ -73,21 +73,22 @@ __global__ void k_kv_rank(KvComp ck, KvComp cv) {
 
 // grid (n_kv, 2): block of 8 warps walks the n_new tokens in batches of 8; offsets into the unary arena are
 // assigned sequentially by one thread per batch, so records stay densely packed in token order.
+// grid.z = sequence of the call; its rows start at row blockIdx.z * n_new of the source.
 __global__ void __launch_bounds__(256) k_kv_append(KvGeom g, KvComp ck, KvComp cv, uint16_t* __restrict__ k_cache,
                                                    uint16_t* __restrict__ v_cache, const uint16_t* __restrict__ src_k,
                                                    const uint16_t* __restrict__ src_v, int row_stride, int start_pos_arg,
-                                                   int use_inflight, int n_new, int flags, DevState* st) {
+                                                   int use_inflight, int n_new, int flags, DevState* st, int seq0) {
     __shared__ uint32_t s_fix[kKvWarps][kKvFixMax];          // bitmap (<= 8) + field words (<= 64)
     __shared__ uint32_t s_una[kKvWarps][kKvStageWords];
     __shared__ uint32_t s_nw[kKvWarps], s_off[kKvWarps];
     pdl_launch_dependents();
     pdl_wait();
-    const int head = blockIdx.x, kind = blockIdx.y;
+    const int head = blockIdx.x, kind = blockIdx.y, seq = seq0 + blockIdx.z;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const KvComp c = kind ? cv : ck;
-    const uint16_t* src = kind ? src_v : src_k;
-    uint16_t* cache = kind ? v_cache : k_cache;
-    const int start_pos = start_pos_arg >= 0 ? start_pos_arg : st->len + (use_inflight ? st->inflight : 0);
+    const KvComp c = of_seq(kind ? cv : ck, seq, g.seq_stride);
+    const uint16_t* src = (kind ? src_v : src_k) + (size_t)blockIdx.z * n_new * row_stride;
+    uint16_t* cache = of_seq(kind ? v_cache : k_cache, seq, g.seq_stride);
+    const int start_pos = start_pos_arg >= 0 ? start_pos_arg : st->len[seq] + (use_inflight ? st->inflight[seq] : 0);
     const int nj = g.d / 32, t_bits = g.t, F = 8 - t_bits, per = 32 / F;
     uint32_t* off = c.off + (size_t)head * (g.max_seq + 1);
     uint32_t* arena = c.arena + (size_t)head * g.arena_words;
@@ -179,11 +180,11 @@ __global__ void __launch_bounds__(256) k_kv_append(KvGeom g, KvComp ck, KvComp c
 
 int launch_kv_append(const KvGeom& g, const KvComp& ck, const KvComp& cv, uint16_t* k_cache, uint16_t* v_cache,
                      const uint16_t* src_k, const uint16_t* src_v, int row_stride, int start_pos, int use_inflight,
-                     int n_new, int flags, DevState* st, cudaStream_t s) {
-    if (n_new <= 0) return CASS_OK;
-    dim3 grid(g.n_kv, 2);
+                     int n_new, int flags, DevState* st, int seq0, int n_seq, cudaStream_t s) {
+    if (n_new <= 0 || n_seq <= 0) return CASS_OK;
+    dim3 grid(g.n_kv, 2, n_seq);
     CASS_PDL_LAUNCH(k_kv_append, grid, dim3(256), 0, s, g, ck, cv, k_cache, v_cache, src_k, src_v, row_stride, start_pos,
-                    use_inflight, n_new, flags, st);
+                    use_inflight, n_new, flags, st, seq0);
     return CASS_OK;
 }
 

@@ -15,12 +15,12 @@ __global__ void k_rope_table(float* __restrict__ cos_t, float* __restrict__ sin_
     sin_t[i] = (float)sin(ang);
 }
 
-__global__ void k_embed(const int32_t* __restrict__ toks, const uint16_t* __restrict__ embed, uint16_t* __restrict__ h,
-                        int hidden) {
+__global__ void k_embed(const int32_t* __restrict__ toks, int tok_stride, const uint16_t* __restrict__ embed,
+                        uint16_t* __restrict__ h, int hidden) {
     pdl_launch_dependents();
     pdl_wait();
     int r = blockIdx.x;
-    const uint16_t* src = embed + (size_t)toks[r] * hidden;
+    const uint16_t* src = embed + (size_t)toks[(size_t)r * tok_stride] * hidden;
     for (int i = threadIdx.x; i < hidden; i += blockDim.x) h[(size_t)r * hidden + i] = src[i];
 }
 
@@ -107,12 +107,13 @@ __global__ void __launch_bounds__(1024) k_residual_rmsnorm(uint16_t* __restrict_
 
 __global__ void k_qkv_rope(uint16_t* __restrict__ qkv, Partials pp,
                            const float* __restrict__ cos_t, const float* __restrict__ sin_t,
-                           const DevState* __restrict__ st, int use_inflight, int n_q, int n_kv, int d) {
+                           const DevState* __restrict__ st, int use_inflight, int rps, int n_q, int n_kv, int d) {
     pdl_launch_dependents();
     pdl_wait();
     const int r = blockIdx.y, half = d / 2;
     const int qkv_dim = (n_q + 2 * n_kv) * d;
-    const int pos = st->len + (use_inflight ? st->inflight : 0) + r;
+    const int b = r / rps;
+    const int pos = st->len[b] + (use_inflight ? st->inflight[b] : 0) + r % rps;
     uint16_t* row = qkv + (size_t)r * qkv_dim;
     const int n_rot = (n_q + n_kv) * half;             // rotated pairs
     const int n_items = n_rot + n_kv * d;              // + plain v elements
@@ -209,7 +210,8 @@ __global__ void __launch_bounds__(256) k_argmax_part(const float* __restrict__ l
 }
 
 __global__ void __launch_bounds__(kArgmaxSlices) k_argmax_final(const float* __restrict__ tmp_v, const int32_t* __restrict__ tmp_i,
-                                                                int nsl, int32_t* __restrict__ out, DevState* st, int bump_inflight) {
+                                                                int nsl, int32_t* __restrict__ out, int out_stride, DevState* st,
+                                                                int bump_inflight) {
     __shared__ float s_v[kArgmaxSlices / 32];
     __shared__ int s_i[kArgmaxSlices / 32];
     pdl_launch_dependents();
@@ -228,17 +230,25 @@ __global__ void __launch_bounds__(kArgmaxSlices) k_argmax_final(const float* __r
     __syncthreads();
     if (threadIdx.x == 0) {
         for (int w = 1; w < kArgmaxSlices / 32; ++w) argmax_combine(best, best_i, s_v[w], s_i[w]);
-        out[r] = best_i == 0x7fffffff ? 0 : best_i;
-        if (bump_inflight && r == 0) st->inflight += 1;
+        out[(size_t)r * out_stride] = best_i == 0x7fffffff ? 0 : best_i;
+        if (bump_inflight && r < kMaxBatch) st->inflight[r] += 1;
     }
 }
 
 // Greedy acceptance: a = min({i-1 : draft_i != target_{i-1}} U {g}); emit draft_1..draft_a and target_a.
-__global__ void k_accept(DevState* st, const int32_t* __restrict__ draft, const int32_t* __restrict__ target, int g,
-                         int32_t* n_acc, int32_t* out_tokens, int32_t* next_tok) {
+// One block per sequence b: draft[b * draft_stride + i], target[b][g+1] -> n_acc[b], out_tokens[b][g+1],
+// next_tok[b * next_stride].
+__global__ void k_accept(DevState* st, const int32_t* __restrict__ draft, int draft_stride, const int32_t* __restrict__ target, int g,
+                         int32_t* n_acc, int32_t* out_tokens, int32_t* next_tok, int next_stride) {
     pdl_launch_dependents();
     pdl_wait();
-    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    if (threadIdx.x != 0) return;
+    const int b = blockIdx.x;
+    draft += (size_t)b * draft_stride;
+    target += (size_t)b * (g + 1);
+    out_tokens += (size_t)b * (g + 1);
+    n_acc += b;
+    if (next_tok) next_tok += (size_t)b * next_stride;
     int a = 0;
     while (a < g && draft[a] == target[a]) ++a;
     for (int i = 0; i < a; ++i) out_tokens[i] = draft[i];
@@ -248,9 +258,9 @@ __global__ void k_accept(DevState* st, const int32_t* __restrict__ draft, const 
     if (next_tok) *next_tok = target[a];
     // Every later call touches positions up to len + 15 at most; a sequence that would come closer than that to
     // the end of its cache stops growing and the status word says so.
-    if (st->len + a + 1 + kMaxVerifyRows > st->max_seq) atomicCAS(&st->status, 0, CASS_ERR_CAPACITY);
-    else st->len += a + 1;
-    st->inflight = 0;
+    if (st->len[b] + a + 1 + kMaxVerifyRows > st->max_seq) atomicCAS(&st->status, 0, CASS_ERR_CAPACITY);
+    else st->len[b] += a + 1;
+    st->inflight[b] = 0;
 }
 
 __global__ void k_calib_accum(const uint16_t* __restrict__ x, int rows, int cols, float* __restrict__ sumsq,
@@ -280,8 +290,8 @@ int launch_rope_table(float* cos_t, float* sin_t, int max_seq, int d, float thet
     return CASS_OK;
 }
 
-int launch_embed(const int32_t* toks, const uint16_t* embed, uint16_t* h, int rows, int hidden, cudaStream_t s) {
-    CASS_PDL_LAUNCH(k_embed, dim3(rows), dim3(256), 0, s, toks, embed, h, hidden);
+int launch_embed(const int32_t* toks, int tok_stride, const uint16_t* embed, uint16_t* h, int rows, int hidden, cudaStream_t s) {
+    CASS_PDL_LAUNCH(k_embed, dim3(rows), dim3(256), 0, s, toks, tok_stride, embed, h, hidden);
     return CASS_OK;
 }
 
@@ -305,10 +315,10 @@ int launch_residual_rmsnorm(uint16_t* h, const uint16_t* y_bf16, Partials pp,
 }
 
 int launch_qkv_rope(uint16_t* qkv, Partials pp, const float* cos_t, const float* sin_t,
-                    const DevState* st, int use_inflight, int rows, int n_q, int n_kv, int d, cudaStream_t s) {
+                    const DevState* st, int use_inflight, int rows, int rps, int n_q, int n_kv, int d, cudaStream_t s) {
     int items = (n_q + n_kv) * (d / 2) + n_kv * d;
     dim3 grid(ceil_div(items, 256), rows);
-    CASS_PDL_LAUNCH(k_qkv_rope, grid, dim3(256), 0, s, qkv, pp, cos_t, sin_t, st, use_inflight, n_q, n_kv, d);
+    CASS_PDL_LAUNCH(k_qkv_rope, grid, dim3(256), 0, s, qkv, pp, cos_t, sin_t, st, use_inflight, rps, n_q, n_kv, d);
     return CASS_OK;
 }
 
@@ -319,19 +329,19 @@ int launch_swiglu(const uint16_t* gu_bf16, Partials pp, uint16_t* act, int rows,
     return CASS_OK;
 }
 
-int launch_argmax(const float* logits, Partials pp, int rows, int vocab, int32_t* out,
+int launch_argmax(const float* logits, Partials pp, int rows, int vocab, int32_t* out, int out_stride,
                   float* logits_copy, float* tmp_v, int32_t* tmp_i, DevState* st, int bump_inflight, cudaStream_t s) {
     int nsl = ceil_div(vocab, 1024);
     if (nsl > kArgmaxSlices) nsl = kArgmaxSlices;
     dim3 grid(nsl, rows);
     CASS_PDL_LAUNCH(k_argmax_part, grid, dim3(256), 0, s, logits, pp, vocab, tmp_v, tmp_i, logits_copy);
-    CASS_PDL_LAUNCH(k_argmax_final, dim3(rows), dim3(kArgmaxSlices), 0, s, (const float*)tmp_v, (const int32_t*)tmp_i, nsl, out, st, bump_inflight);
+    CASS_PDL_LAUNCH(k_argmax_final, dim3(rows), dim3(kArgmaxSlices), 0, s, (const float*)tmp_v, (const int32_t*)tmp_i, nsl, out, out_stride, st, bump_inflight);
     return CASS_OK;
 }
 
-int launch_accept(DevState* st, const int32_t* draft, const int32_t* target, int g, int32_t* n_acc, int32_t* out_tokens,
-                  int32_t* next_tok, cudaStream_t s) {
-    CASS_PDL_LAUNCH(k_accept, dim3(1), dim3(32), 0, s, st, draft, target, g, n_acc, out_tokens, next_tok);
+int launch_accept(DevState* st, int n_seq, const int32_t* draft, int draft_stride, const int32_t* target, int g, int32_t* n_acc,
+                  int32_t* out_tokens, int32_t* next_tok, int next_stride, cudaStream_t s) {
+    CASS_PDL_LAUNCH(k_accept, dim3(n_seq), dim3(32), 0, s, st, draft, draft_stride, target, g, n_acc, out_tokens, next_tok, next_stride);
     return CASS_OK;
 }
 

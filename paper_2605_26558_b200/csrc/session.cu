@@ -1,5 +1,6 @@
 // Session: device memory plan, model pointers, and the three step-level entry points
 // (draft step, verification pass, greedy accept) built from the library's kernels.
+#include <cstddef>
 #include <new>
 #include <vector>
 
@@ -32,7 +33,8 @@ struct Session {
     float* calib_all;        // start of the calibration block
     size_t calib_count;
     int calib_kmax;
-    // activations (rows <= 16)
+    int B, R;                // sequences; row capacity of one call (16, 32 or 64 = token columns of the verification MMA)
+    // activations (R rows)
     uint16_t *h, *xn, *qkv, *attn, *y, *gu, *act;
     float *logits, *partial, *vg_partial;
     size_t partial_floats;
@@ -51,7 +53,7 @@ struct Plan {
 static int check_desc(const cass_model_desc* d, const cass_format* f) {
     if (!d || !f) return CASS_ERR_INVALID_ARG;
     if (f->mode != 1) return CASS_ERR_UNSUPPORTED;
-    if (d->max_batch != 1) return CASS_ERR_UNSUPPORTED;
+    if (d->max_batch != 1 && d->max_batch != 2 && d->max_batch != 4 && d->max_batch != 8) return CASS_ERR_UNSUPPORTED;
     if (d->n_layers <= 0 || d->hidden <= 0 || d->n_q_heads <= 0 || d->n_kv_heads <= 0 || d->head_dim <= 0 ||
         d->ffn <= 0 || d->vocab <= 0 || d->max_seq < 2 * kMaxVerifyRows)
         return CASS_ERR_INVALID_ARG;
@@ -59,6 +61,7 @@ static int check_desc(const cass_model_desc* d, const cass_format* f) {
         return CASS_ERR_UNSUPPORTED;
     if (d->hidden % 8 || d->ffn % 8 || (d->n_q_heads * d->head_dim) % 8) return CASS_ERR_UNSUPPORTED;
     if (d->gamma_max < 0 || d->gamma_max + 1 > kMaxVerifyRows) return CASS_ERR_INVALID_ARG;
+    if (d->max_batch * (d->gamma_max + 1) > kMaxRows) return CASS_ERR_INVALID_ARG;
     if (f->kv_prune_permille < 0 || f->kv_prune_permille > 999 || f->kv_trunc_bits < 0 || f->kv_trunc_bits > 7)
         return CASS_ERR_INVALID_ARG;
     if (f->kv_trunc_bits != 0 && f->kv_trunc_bits != 4) return CASS_ERR_UNSUPPORTED;    // draft attention walks t = 0 or 4 records
@@ -83,9 +86,16 @@ static KvGeom make_kv_geom(const cass_model_desc& d, const cass_format& f) {
 }
 
 // Lays the session out in `base` (base may be null: sizes only).
+static int row_capacity(const cass_model_desc& d) {
+    int r = d.max_batch * (d.gamma_max + 1);
+    return verify_gemm_bn(r < kMaxVerifyRows ? kMaxVerifyRows : r);
+}
+
 static size_t layout(Session* s, uint8_t* base) {
     const cass_model_desc& d = s->d;
-    const KvGeom& g = s->kg;
+    KvGeom& g = s->kg;
+    s->B = d.max_batch;
+    s->R = row_capacity(d);
     Plan p;
     auto at = [&](size_t o) { return base ? base + o : nullptr; };
     s->st = (DevState*)at(p.take(sizeof(DevState)));
@@ -100,7 +110,7 @@ static size_t layout(Session* s, uint8_t* base) {
     s->calib_count = (size_t)d.n_layers * 4 * s->kmax + d.hidden;
     s->calib_all = (float*)at(p.take(s->calib_count * 4));
     s->calib_lm = s->calib_all ? s->calib_all + (size_t)d.n_layers * 4 * s->kmax : nullptr;
-    const int R = kMaxVerifyRows;
+    const int R = s->R;
     s->h = (uint16_t*)at(p.take((size_t)R * d.hidden * 2));
     s->xn = (uint16_t*)at(p.take((size_t)R * d.hidden * 2));
     s->qkv = (uint16_t*)at(p.take((size_t)R * s->qkv_dim * 2));
@@ -122,12 +132,12 @@ static size_t layout(Session* s, uint8_t* base) {
         for (size_t v : c) if (v > pf) pf = v;
     }
     (void)segmax; (void)nmax;
-    s->partial_floats = pf;
-    s->partial = (float*)at(p.take(pf * 4));
+    s->partial_floats = pf;                                   // per vector of a draft GEMV
+    s->partial = (float*)at(p.take(pf * 4 * s->B));
     {   // split-K scratch of the verification GEMMs
-        size_t c[5] = {verify_gemm_partial_floats(s->qkv_dim, d.hidden), verify_gemm_partial_floats(d.hidden, d.n_q_heads * d.head_dim),
-                       verify_gemm_partial_floats(2 * d.ffn, d.hidden), verify_gemm_partial_floats(d.hidden, d.ffn),
-                       verify_gemm_partial_floats(d.vocab, d.hidden)};
+        size_t c[5] = {verify_gemm_partial_floats(s->qkv_dim, d.hidden, R), verify_gemm_partial_floats(d.hidden, d.n_q_heads * d.head_dim, R),
+                       verify_gemm_partial_floats(2 * d.ffn, d.hidden, R), verify_gemm_partial_floats(d.hidden, d.ffn, R),
+                       verify_gemm_partial_floats(d.vocab, d.hidden, R)};
         size_t m = 0;
         for (size_t v : c) if (v > m) m = v;
         s->vg_partial = (float*)at(p.take(m * 4));
@@ -137,9 +147,11 @@ static size_t layout(Session* s, uint8_t* base) {
     s->asc.o = (float*)at(p.take(pairs * n_chunks * d.head_dim * 4));
     s->asc.m = (float*)at(p.take(pairs * n_chunks * 4));
     s->asc.l = (float*)at(p.take(pairs * n_chunks * 4));
-    s->argmax_tmp = (int32_t*)at(p.take(kMaxVerifyRows * 128 * 4));
-    s->argmax_val = (float*)at(p.take(kMaxVerifyRows * 128 * 4));
+    s->argmax_tmp = (int32_t*)at(p.take((size_t)R * 128 * 4));
+    s->argmax_val = (float*)at(p.take((size_t)R * 128 * 4));
     s->layers.resize(d.n_layers);
+    // KV storage: the block of sequence 0 (all layers, both caches), then identical blocks for the other sequences
+    const size_t kv_begin = p.off;
     for (int l = 0; l < d.n_layers; ++l) {
         LayerDev& L = s->layers[l];
         size_t kvb = (size_t)d.max_seq * g.n_kv * g.d * 2;
@@ -156,6 +168,8 @@ static size_t layout(Session* s, uint8_t* base) {
         }
         for (int i = 0; i < 4; ++i) L.calib[i] = s->calib_all ? s->calib_all + ((size_t)l * 4 + i) * s->kmax : nullptr;
     }
+    g.seq_stride = p.off - kv_begin;
+    p.off += g.seq_stride * (size_t)(s->B - 1);
     return p.off;
 }
 
@@ -170,7 +184,7 @@ static int read_blob_infos(Session* s, const cass_model_blobs* blobs, cudaStream
             int rc = cass_weight_blob_info(ptr[i], &s->layers[l].bi[i], stream);
             if (rc) return rc;
             if (s->layers[l].bi[i].rows != rows[i] || s->layers[l].bi[i].cols != cols[i]) return CASS_ERR_INVALID_ARG;
-            if (gemv_smem_bytes(s->layers[l].bi[i]) > 227 * 1024) return CASS_ERR_CAPACITY;
+            if (gemv_smem_bytes(s->layers[l].bi[i], s->B) > 227 * 1024) return CASS_ERR_CAPACITY;
             if ((size_t)s->layers[l].bi[i].n_seg * s->layers[l].bi[i].n_rowblocks * 32 > s->partial_floats) return CASS_ERR_CAPACITY;
             s->layers[l].blob[i] = ptr[i];
         }
@@ -243,10 +257,11 @@ extern "C" int cass_session_reset(void* session, void* stream_) {
     CASS_CUDA_CHECK(cudaMemcpyAsync(&s->st->max_seq, &s->d.max_seq, 4, cudaMemcpyHostToDevice, stream));
     CASS_CUDA_CHECK(cudaMemsetAsync(s->calib_all, 0, s->calib_count * 4, stream));
     for (auto& L : s->layers)
-        for (int kind = 0; kind < 2; ++kind) {
-            KvComp& c = kind ? L.cv : L.ck;
-            CASS_CUDA_CHECK(cudaMemsetAsync(c.off, 0, (size_t)s->kg.n_kv * (s->kg.max_seq + 1) * 4, stream));
-        }
+        for (int kind = 0; kind < 2; ++kind)
+            for (int b = 0; b < s->B; ++b) {
+                KvComp c = of_seq(kind ? L.cv : L.ck, b, s->kg.seq_stride);
+                CASS_CUDA_CHECK(cudaMemsetAsync(c.off, 0, (size_t)s->kg.n_kv * (s->kg.max_seq + 1) * 4, stream));
+            }
     s->codebooks_ready = false;
     return CASS_OK;
 }
@@ -259,8 +274,25 @@ extern "C" int cass_session_status(void* session, int32_t* h_status, int32_t* h_
     CASS_CUDA_CHECK(cudaMemcpyAsync(&st, s->st, sizeof(st), cudaMemcpyDeviceToHost, stream));
     CASS_CUDA_CHECK(cudaStreamSynchronize(stream));
     if (h_status) *h_status = st.status;
-    if (h_len) *h_len = st.len;
+    if (h_len) *h_len = st.len[0];
     return CASS_OK;
+}
+
+extern "C" int cass_session_lens(void* session, int32_t* h_lens, void* stream_) {
+    if (!session || !h_lens) return CASS_ERR_INVALID_ARG;
+    Session* s = (Session*)session;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    DevState st;
+    CASS_CUDA_CHECK(cudaMemcpyAsync(&st, s->st, sizeof(st), cudaMemcpyDeviceToHost, stream));
+    CASS_CUDA_CHECK(cudaStreamSynchronize(stream));
+    for (int b = 0; b < s->B; ++b) h_lens[b] = st.len[b];
+    return CASS_OK;
+}
+
+extern "C" int cass_session_rows(const cass_model_desc* desc) {
+    if (!desc || desc->max_batch < 1 || desc->gamma_max < 0) return CASS_ERR_INVALID_ARG;
+    if (desc->max_batch * (desc->gamma_max + 1) > kMaxRows) return CASS_ERR_INVALID_ARG;
+    return row_capacity(*desc);
 }
 
 extern "C" int cass_calib_enable(void* session, int on, void* stream_) {
@@ -291,22 +323,38 @@ extern "C" int cass_set_len(void* session, int len, void* stream_) {
     if (!session) return CASS_ERR_INVALID_ARG;
     Session* s = (Session*)session;
     if (len < 0 || len + kMaxVerifyRows > s->d.max_seq) return CASS_ERR_INVALID_ARG;      // room for one more call's rows
-    int32_t v[2] = {len, 0};
-    CASS_CUDA_CHECK(cudaMemcpyAsync(&s->st->len, v, 8, cudaMemcpyHostToDevice, (cudaStream_t)stream_));
+    int32_t v[2 * kMaxBatch];
+    for (int b = 0; b < kMaxBatch; ++b) { v[b] = len; v[kMaxBatch + b] = 0; }
+    static_assert(offsetof(DevState, inflight) == sizeof(int32_t) * kMaxBatch, "len[] then inflight[]");
+    CASS_CUDA_CHECK(cudaMemcpyAsync(s->st->len, v, sizeof(v), cudaMemcpyHostToDevice, (cudaStream_t)stream_));
     CASS_CUDA_CHECK(cudaStreamSynchronize((cudaStream_t)stream_));
     return CASS_OK;
 }
 
-extern "C" int cass_kv_append(void* session, int layer, const void* K_bf16, const void* V_bf16, int start_pos, int n_new,
-                              int flags, void* stream_) {
+extern "C" int cass_set_lens(void* session, const int32_t* h_lens, void* stream_) {
+    if (!session || !h_lens) return CASS_ERR_INVALID_ARG;
+    Session* s = (Session*)session;
+    int32_t v[2 * kMaxBatch] = {0};
+    for (int b = 0; b < s->B; ++b) {
+        if (h_lens[b] < 0 || h_lens[b] + kMaxVerifyRows > s->d.max_seq) return CASS_ERR_INVALID_ARG;
+        v[b] = h_lens[b];
+    }
+    CASS_CUDA_CHECK(cudaMemcpyAsync(s->st->len, v, sizeof(v), cudaMemcpyHostToDevice, (cudaStream_t)stream_));
+    CASS_CUDA_CHECK(cudaStreamSynchronize((cudaStream_t)stream_));
+    return CASS_OK;
+}
+
+extern "C" int cass_kv_append(void* session, int seq, int layer, const void* K_bf16, const void* V_bf16, int start_pos,
+                              int n_new, int flags, void* stream_) {
     if (!session || !K_bf16 || !V_bf16) return CASS_ERR_INVALID_ARG;
     Session* s = (Session*)session;
-    if (layer < 0 || layer >= s->d.n_layers || start_pos < 0 || n_new < 0 || start_pos + n_new > s->d.max_seq)
+    if (seq < 0 || seq >= s->B || layer < 0 || layer >= s->d.n_layers || start_pos < 0 || n_new < 0 ||
+        start_pos + n_new > s->d.max_seq)
         return CASS_ERR_INVALID_ARG;
     if (!(flags & (CASS_KV_BF16 | CASS_KV_COMPRESSED))) return CASS_ERR_INVALID_ARG;
     LayerDev& L = s->layers[layer];
     return launch_kv_append(s->kg, L.ck, L.cv, L.kc, L.vc, (const uint16_t*)K_bf16, (const uint16_t*)V_bf16,
-                            s->kg.n_kv * s->kg.d, start_pos, 0, n_new, flags, s->st, (cudaStream_t)stream_);
+                            s->kg.n_kv * s->kg.d, start_pos, 0, n_new, flags, s->st, seq, 1, (cudaStream_t)stream_);
 }
 
 extern "C" int cass_kv_build_codebook(void* session, int n_tokens, void* stream_) {
@@ -314,29 +362,33 @@ extern "C" int cass_kv_build_codebook(void* session, int n_tokens, void* stream_
     Session* s = (Session*)session;
     if (n_tokens < 0 || n_tokens > s->d.max_seq) return CASS_ERR_INVALID_ARG;
     cudaStream_t stream = (cudaStream_t)stream_;
-    for (auto& L : s->layers) {
-        int rc = launch_kv_codebook(s->kg, L.ck, L.cv, L.kc, L.vc, n_tokens, stream);
-        if (rc) return rc;
-        rc = launch_kv_append(s->kg, L.ck, L.cv, L.kc, L.vc, L.kc, L.vc, s->kg.n_kv * s->kg.d, 0, 0, n_tokens,
-                              CASS_KV_COMPRESSED, s->st, stream);
-        if (rc) return rc;
-    }
+    const size_t ss = s->kg.seq_stride;
+    for (auto& L : s->layers)
+        for (int b = 0; b < s->B; ++b) {       // every sequence has its own codebooks, built from its own prompt
+            const uint16_t *kc = of_seq(L.kc, b, ss), *vc = of_seq(L.vc, b, ss);
+            int rc = launch_kv_codebook(s->kg, of_seq(L.ck, b, ss), of_seq(L.cv, b, ss), kc, vc, n_tokens, stream);
+            if (rc) return rc;
+            rc = launch_kv_append(s->kg, L.ck, L.cv, L.kc, L.vc, kc, vc, s->kg.n_kv * s->kg.d, 0, 0, n_tokens,
+                                  CASS_KV_COMPRESSED, s->st, b, 1, stream);
+            if (rc) return rc;
+        }
     s->codebooks_ready = true;
     return CASS_OK;
 }
 
-extern "C" int cass_kv_query(void* session, int layer, int kind, int head, cass_kv_view* v) {
+extern "C" int cass_kv_query(void* session, int seq, int layer, int kind, int head, cass_kv_view* v) {
     if (!session || !v) return CASS_ERR_INVALID_ARG;
     Session* s = (Session*)session;
-    if (layer < 0 || layer >= s->d.n_layers || kind < 0 || kind > 1 || head < 0 || head >= s->kg.n_kv) return CASS_ERR_INVALID_ARG;
+    if (seq < 0 || seq >= s->B || layer < 0 || layer >= s->d.n_layers || kind < 0 || kind > 1 || head < 0 || head >= s->kg.n_kv)
+        return CASS_ERR_INVALID_ARG;
     const KvGeom& g = s->kg;
     LayerDev& L = s->layers[layer];
-    const KvComp& c = kind ? L.cv : L.ck;
+    const KvComp c = of_seq(kind ? L.cv : L.ck, seq, g.seq_stride);
     v->fixed = c.fixed + (size_t)head * g.n_blocks * g.wpt * 32;
     v->arena = c.arena + (size_t)head * g.arena_words;
     v->offsets = c.off + (size_t)head * (g.max_seq + 1);
     v->codebook = c.rank_to_exp;
-    v->k_or_v_bf16 = kind ? L.vc : L.kc;
+    v->k_or_v_bf16 = of_seq(kind ? L.vc : L.kc, seq, g.seq_stride);
     v->fixed_words_per_token = g.wpt;
     v->bitmap_words = g.bm_words;
     v->arena_words = g.arena_words;
@@ -348,8 +400,8 @@ extern "C" int cass_draft_attention(void* session, int layer, const void* q_bf16
     Session* s = (Session*)session;
     if (layer < 0 || layer >= s->d.n_layers) return CASS_ERR_INVALID_ARG;
     LayerDev& L = s->layers[layer];
-    return launch_draft_attn(s->kg, L.ck, L.cv, (const uint16_t*)q_bf16, s->d.n_q_heads, s->st, s->asc, (uint16_t*)out_bf16,
-                             (cudaStream_t)stream_);
+    return launch_draft_attn(s->kg, L.ck, L.cv, (const uint16_t*)q_bf16, s->d.n_q_heads * s->d.head_dim, s->d.n_q_heads, s->B,
+                             s->st, s->asc, (uint16_t*)out_bf16, (cudaStream_t)stream_);
 }
 
 extern "C" int cass_debug_activation(void* session, int which, const void** d_ptr, int* h_rows, int* h_cols) {
@@ -359,7 +411,7 @@ extern "C" int cass_debug_activation(void* session, int which, const void** d_pt
     else if (which == 1) { *d_ptr = s->attn; if (h_cols) *h_cols = s->d.n_q_heads * s->d.head_dim; }
     else if (which == 2) { *d_ptr = s->qkv; if (h_cols) *h_cols = s->qkv_dim; }
     else return CASS_ERR_INVALID_ARG;
-    if (h_rows) *h_rows = kMaxVerifyRows;
+    if (h_rows) *h_rows = s->R;
     return CASS_OK;
 }
 
@@ -369,12 +421,14 @@ extern "C" int cass_verify(void* session, const int32_t* toks, int g, int32_t* t
                            void* stream_) {
     if (!session || !toks || !target_argmax) return CASS_ERR_INVALID_ARG;
     Session* s = (Session*)session;
-    const int rows = g + 1;
-    if (g < 0 || rows > kMaxVerifyRows) return CASS_ERR_INVALID_ARG;
+    const int rps = g + 1, B = s->B, bn = s->R;      // rows per sequence; the MMA's token columns are fixed per session
+    const int rows = B * rps;
+    if (g < 0 || rps > kMaxVerifyRows || rows > s->R) return CASS_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)stream_;
     const cass_model_desc& d = s->d;
+    auto vparts = [&](int n, int k) { return verify_gemm_partials(s->vg_partial, n, k, bn); };
     const int qd = d.n_q_heads * d.head_dim;
-    RC(launch_embed(toks, (const uint16_t*)s->embed, s->h, rows, d.hidden, st));
+    RC(launch_embed(toks, 1, (const uint16_t*)s->embed, s->h, rows, d.hidden, st));
     RC(launch_rmsnorm(s->h, (const uint16_t*)s->layers[0].w.norm_attn, s->xn, rows, d.hidden, d.rms_eps, st));
     const int kv_flags = CASS_KV_BF16 | (s->codebooks_ready ? CASS_KV_COMPRESSED : 0);
     const bool calib = s->calib_host;           // the accumulation kernels are only launched while calibration is on
@@ -383,67 +437,71 @@ extern "C" int cass_verify(void* session, const int32_t* toks, int g, int32_t* t
     for (int l = 0; l < d.n_layers; ++l) {
         LayerDev& L = s->layers[l];
         if (calib) RC(launch_calib_accum(s->xn, rows, d.hidden, L.calib[0], s->st, st));
-        RC(launch_verify_gemm((const uint16_t*)L.w.wqkv, s->xn, rows, s->qkv_dim, d.hidden, s->vg_partial, nullptr, nullptr, status, st));
-        RC(launch_qkv_rope(s->qkv, verify_gemm_partials(s->vg_partial, s->qkv_dim, d.hidden), s->cos_t, s->sin_t, s->st, 0, rows,
+        RC(launch_verify_gemm((const uint16_t*)L.w.wqkv, s->xn, rows, bn, s->qkv_dim, d.hidden, s->vg_partial, nullptr, nullptr, status, st));
+        RC(launch_qkv_rope(s->qkv, vparts(s->qkv_dim, d.hidden), s->cos_t, s->sin_t, s->st, 0, rows, rps,
                            d.n_q_heads, d.n_kv_heads, d.head_dim, st));
         RC(launch_kv_append(s->kg, L.ck, L.cv, L.kc, L.vc, s->qkv + qd, s->qkv + qd + d.n_kv_heads * d.head_dim, s->qkv_dim,
-                            -1, 0, rows, kv_flags, s->st, st));
-        RC(launch_verify_attn(s->kg, L.kc, L.vc, s->qkv, rows, d.n_q_heads, s->st, s->asc, s->attn, st));
+                            -1, 0, rps, kv_flags, s->st, 0, B, st));
+        RC(launch_verify_attn(s->kg, L.kc, L.vc, s->qkv, B, rps, d.n_q_heads, s->st, s->asc, s->attn, st));
         if (calib) RC(launch_calib_accum(s->attn, rows, qd, L.calib[1], s->st, st));
-        RC(launch_verify_gemm((const uint16_t*)L.w.wo, s->attn, rows, d.hidden, qd, s->vg_partial, nullptr, nullptr, status, st));
-        RC(launch_residual_rmsnorm(s->h, nullptr, verify_gemm_partials(s->vg_partial, d.hidden, qd), (const uint16_t*)L.w.norm_ffn, s->xn,
+        RC(launch_verify_gemm((const uint16_t*)L.w.wo, s->attn, rows, bn, d.hidden, qd, s->vg_partial, nullptr, nullptr, status, st));
+        RC(launch_residual_rmsnorm(s->h, nullptr, vparts(d.hidden, qd), (const uint16_t*)L.w.norm_ffn, s->xn,
                                    rows, d.hidden, d.rms_eps, st));
         if (calib) RC(launch_calib_accum(s->xn, rows, d.hidden, L.calib[2], s->st, st));
-        RC(launch_verify_gemm((const uint16_t*)L.w.wgu, s->xn, rows, 2 * d.ffn, d.hidden, s->vg_partial, nullptr, nullptr, status, st));
-        RC(launch_swiglu(nullptr, verify_gemm_partials(s->vg_partial, 2 * d.ffn, d.hidden), s->act, rows, d.ffn, st));
+        RC(launch_verify_gemm((const uint16_t*)L.w.wgu, s->xn, rows, bn, 2 * d.ffn, d.hidden, s->vg_partial, nullptr, nullptr, status, st));
+        RC(launch_swiglu(nullptr, vparts(2 * d.ffn, d.hidden), s->act, rows, d.ffn, st));
         if (calib) RC(launch_calib_accum(s->act, rows, d.ffn, L.calib[3], s->st, st));
-        RC(launch_verify_gemm((const uint16_t*)L.w.wd, s->act, rows, d.hidden, d.ffn, s->vg_partial, nullptr, nullptr, status, st));
+        RC(launch_verify_gemm((const uint16_t*)L.w.wd, s->act, rows, bn, d.hidden, d.ffn, s->vg_partial, nullptr, nullptr, status, st));
         const uint16_t* next_gain = (const uint16_t*)(l + 1 < d.n_layers ? s->layers[l + 1].w.norm_attn : s->norm_final);
-        RC(launch_residual_rmsnorm(s->h, nullptr, verify_gemm_partials(s->vg_partial, d.hidden, d.ffn), next_gain, s->xn, rows, d.hidden,
+        RC(launch_residual_rmsnorm(s->h, nullptr, vparts(d.hidden, d.ffn), next_gain, s->xn, rows, d.hidden,
                                    d.rms_eps, st));
     }
     if (calib) RC(launch_calib_accum(s->xn, rows, d.hidden, s->calib_lm, s->st, st));
-    RC(launch_verify_gemm((const uint16_t*)s->lm_head, s->xn, rows, d.vocab, d.hidden, s->vg_partial, nullptr, nullptr, status, st));
-    RC(launch_argmax(nullptr, verify_gemm_partials(s->vg_partial, d.vocab, d.hidden), rows, d.vocab, target_argmax, logits_opt,
+    RC(launch_verify_gemm((const uint16_t*)s->lm_head, s->xn, rows, bn, d.vocab, d.hidden, s->vg_partial, nullptr, nullptr, status, st));
+    RC(launch_argmax(nullptr, vparts(d.vocab, d.hidden), rows, d.vocab, target_argmax, 1, logits_opt,
                      s->argmax_val, s->argmax_tmp, s->st, 0, st));
     return CASS_OK;
 }
 
-extern "C" int cass_draft_step(void* session, const int32_t* tok_in, int32_t* tok_out, float* logits_opt, void* stream_) {
-    if (!session || !tok_in || !tok_out) return CASS_ERR_INVALID_ARG;
+extern "C" int cass_draft_step(void* session, const int32_t* tok_in, int32_t* tok_out, int tok_stride, float* logits_opt,
+                               void* stream_) {
+    if (!session || !tok_in || !tok_out || tok_stride < 1) return CASS_ERR_INVALID_ARG;
     Session* s = (Session*)session;
     if (!s->have_blobs || !s->codebooks_ready) return CASS_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)stream_;
     const cass_model_desc& d = s->d;
     const int qd = d.n_q_heads * d.head_dim;
     int32_t* status = &s->st->status;
-    auto draftp = [&](const cass_blob_info& b) { return Partials{s->partial, b.n_seg, (size_t)b.n_rowblocks * 32, 0}; };
-    RC(launch_embed(tok_in, (const uint16_t*)s->embed, s->h, 1, d.hidden, st));
-    RC(launch_rmsnorm(s->h, (const uint16_t*)s->layers[0].w.norm_attn, s->xn, 1, d.hidden, d.rms_eps, st));
+    const int B = s->B;
+    auto draftp = [&](const cass_blob_info& b) { return draft_gemv_partials(s->partial, b); };
+    RC(launch_embed(tok_in, tok_stride, (const uint16_t*)s->embed, s->h, B, d.hidden, st));
+    RC(launch_rmsnorm(s->h, (const uint16_t*)s->layers[0].w.norm_attn, s->xn, B, d.hidden, d.rms_eps, st));
     for (int l = 0; l < d.n_layers; ++l) {
         LayerDev& L = s->layers[l];
-        RC(launch_draft_gemv(L.blob[0], L.bi[0], s->xn, s->partial, status, st));
-        RC(launch_qkv_rope(s->qkv, draftp(L.bi[0]), s->cos_t, s->sin_t, s->st, 1, 1, d.n_q_heads, d.n_kv_heads, d.head_dim, st));
+        RC(launch_draft_gemv(L.blob[0], L.bi[0], s->xn, B, s->partial, status, st));
+        RC(launch_qkv_rope(s->qkv, draftp(L.bi[0]), s->cos_t, s->sin_t, s->st, 1, B, 1, d.n_q_heads, d.n_kv_heads, d.head_dim, st));
         RC(launch_kv_append(s->kg, L.ck, L.cv, L.kc, L.vc, s->qkv + qd, s->qkv + qd + d.n_kv_heads * d.head_dim, s->qkv_dim,
-                            -1, 1, 1, CASS_KV_COMPRESSED, s->st, st));
-        RC(launch_draft_attn(s->kg, L.ck, L.cv, s->qkv, d.n_q_heads, s->st, s->asc, s->attn, st));
-        RC(launch_draft_gemv(L.blob[1], L.bi[1], s->attn, s->partial, status, st));
-        RC(launch_residual_rmsnorm(s->h, nullptr, draftp(L.bi[1]), (const uint16_t*)L.w.norm_ffn, s->xn, 1, d.hidden, d.rms_eps, st));
-        RC(launch_draft_gemv(L.blob[2], L.bi[2], s->xn, s->partial, status, st));
-        RC(launch_swiglu(nullptr, draftp(L.bi[2]), s->act, 1, d.ffn, st));
-        RC(launch_draft_gemv(L.blob[3], L.bi[3], s->act, s->partial, status, st));
+                            -1, 1, 1, CASS_KV_COMPRESSED, s->st, 0, B, st));
+        RC(launch_draft_attn(s->kg, L.ck, L.cv, s->qkv, s->qkv_dim, d.n_q_heads, B, s->st, s->asc, s->attn, st));
+        RC(launch_draft_gemv(L.blob[1], L.bi[1], s->attn, B, s->partial, status, st));
+        RC(launch_residual_rmsnorm(s->h, nullptr, draftp(L.bi[1]), (const uint16_t*)L.w.norm_ffn, s->xn, B, d.hidden, d.rms_eps, st));
+        RC(launch_draft_gemv(L.blob[2], L.bi[2], s->xn, B, s->partial, status, st));
+        RC(launch_swiglu(nullptr, draftp(L.bi[2]), s->act, B, d.ffn, st));
+        RC(launch_draft_gemv(L.blob[3], L.bi[3], s->act, B, s->partial, status, st));
         const uint16_t* next_gain = (const uint16_t*)(l + 1 < d.n_layers ? s->layers[l + 1].w.norm_attn : s->norm_final);
-        RC(launch_residual_rmsnorm(s->h, nullptr, draftp(L.bi[3]), next_gain, s->xn, 1, d.hidden, d.rms_eps, st));
+        RC(launch_residual_rmsnorm(s->h, nullptr, draftp(L.bi[3]), next_gain, s->xn, B, d.hidden, d.rms_eps, st));
     }
-    RC(launch_draft_gemv(s->lm_blob, s->lm_bi, s->xn, s->partial, status, st));
-    RC(launch_argmax(nullptr, draftp(s->lm_bi), 1, d.vocab, tok_out, logits_opt, s->argmax_val, s->argmax_tmp, s->st, 1, st));
+    RC(launch_draft_gemv(s->lm_blob, s->lm_bi, s->xn, B, s->partial, status, st));
+    RC(launch_argmax(nullptr, draftp(s->lm_bi), B, d.vocab, tok_out, tok_stride, logits_opt, s->argmax_val, s->argmax_tmp, s->st, 1, st));
     return CASS_OK;
 }
 
-extern "C" int cass_accept(void* session, const int32_t* draft, const int32_t* target_argmax, int g, int32_t* n_accepted,
-                           int32_t* out_tokens, int32_t* next_tok, void* stream_) {
+extern "C" int cass_accept(void* session, const int32_t* draft, int draft_stride, const int32_t* target_argmax, int g,
+                           int32_t* n_accepted, int32_t* out_tokens, int32_t* next_tok, int next_stride, void* stream_) {
     if (!session || !target_argmax || !n_accepted || !out_tokens || (g > 0 && !draft)) return CASS_ERR_INVALID_ARG;
+    if (draft_stride < g || next_stride < 1) return CASS_ERR_INVALID_ARG;
     Session* s = (Session*)session;
     if (g < 0 || g + 1 > kMaxVerifyRows) return CASS_ERR_INVALID_ARG;
-    return launch_accept(s->st, draft, target_argmax, g, n_accepted, out_tokens, next_tok, (cudaStream_t)stream_);
+    return launch_accept(s->st, s->B, draft, draft_stride, target_argmax, g, n_accepted, out_tokens, next_tok, next_stride,
+                         (cudaStream_t)stream_);
 }

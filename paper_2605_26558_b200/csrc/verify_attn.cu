@@ -13,6 +13,7 @@ constexpr int kVaMaxGroup = 8;
 constexpr int kVaMaxPairs = kVaRowBatch * kVaMaxGroup;      // (row, query head) pairs handled at a time
 constexpr int kVaHalfPairs = kVaMaxPairs / 2;
 
+// grid (chunk, KV head, sequence); `rows` = rows of each sequence in this call.
 __global__ void __launch_bounds__(kVaThreads) k_verify_attn(KvGeom g, const uint16_t* __restrict__ k_cache,
                                                             const uint16_t* __restrict__ v_cache, const uint16_t* __restrict__ qkv,
                                                             int rows, int n_q, const DevState* __restrict__ st, AttnScratch sc,
@@ -20,13 +21,16 @@ __global__ void __launch_bounds__(kVaThreads) k_verify_attn(KvGeom g, const uint
     extern __shared__ __align__(16) uint8_t smem[];
     pdl_launch_dependents();
     pdl_wait();
-    const int chunk = blockIdx.x, head = blockIdx.y;
-    const int len = st->len;
+    const int chunk = blockIdx.x, head = blockIdx.y, seq = blockIdx.z;
+    const int len = st->len[seq];
+    k_cache = of_seq(k_cache, seq, g.seq_stride);
+    v_cache = of_seq(v_cache, seq, g.seq_stride);
     const int t0 = chunk * kAttnChunk;
     if (t0 >= len + rows) return;
     const int d = g.d, G = n_q / g.n_kv, ks = d + 8;                  // padded K row stride (elements)
     const int qkv_dim = (n_q + 2 * g.n_kv) * d;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    qkv += (size_t)seq * rows * qkv_dim;                                 // this sequence's rows
     uint16_t* k_s = reinterpret_cast<uint16_t*>(smem);                         // [64][d+8]
     uint16_t* v_s = k_s + kAttnChunk * ks;                                      // [64][d]
     float* q_s = reinterpret_cast<float*>(v_s + kAttnChunk * d);                // [pairs][d]
@@ -103,7 +107,7 @@ __global__ void __launch_bounds__(kVaThreads) k_verify_attn(KvGeom g, const uint
             s_s[p * kAttnChunk + 32 + lane] = b;
             const float l = warp_sum(a + b);
             __syncwarp();
-            const size_t pair = (size_t)r * n_q + head * G + gi;
+            const size_t pair = ((size_t)seq * rows + r) * n_q + head * G + gi;
             for (int dim = lane * 4; dim < d; dim += 128) {             // four dims per lane, tokens in order
                 float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll 4
@@ -125,11 +129,11 @@ __global__ void __launch_bounds__(kVaThreads) k_verify_attn(KvGeom g, const uint
     }
 }
 
-int launch_attn_merge(const AttnScratch& sc, int n_chunks_alloc, int chunk_tokens, int rows, int n_q, int d,
+int launch_attn_merge(const AttnScratch& sc, int n_chunks_alloc, int chunk_tokens, int rows, int rps, int n_q, int d,
                       const DevState* st, int draft_mode, uint16_t* out, cudaStream_t s);
 
-int launch_verify_attn(const KvGeom& g, const uint16_t* k_cache, const uint16_t* v_cache, const uint16_t* qkv, int rows,
-                       int n_q, const DevState* st, const AttnScratch& sc, uint16_t* out, cudaStream_t s) {
+int launch_verify_attn(const KvGeom& g, const uint16_t* k_cache, const uint16_t* v_cache, const uint16_t* qkv, int n_seq,
+                       int rps, int n_q, const DevState* st, const AttnScratch& sc, uint16_t* out, cudaStream_t s) {
     const int G = n_q / g.n_kv;
     if (G > kVaMaxGroup || g.d % 8) return CASS_ERR_UNSUPPORTED;
     static_assert(kAttnChunk == 64 && kVaThreads == 2 * kAttnChunk, "thread = (token, half of the pairs)");
@@ -141,9 +145,9 @@ int launch_verify_attn(const KvGeom& g, const uint16_t* k_cache, const uint16_t*
         CASS_CUDA_CHECK(cudaFuncSetAttribute(k_verify_attn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         attr = smem;
     }
-    dim3 grid(n_chunks, g.n_kv);
-    CASS_PDL_LAUNCH(k_verify_attn, grid, dim3(kVaThreads), smem, s, g, k_cache, v_cache, qkv, rows, n_q, st, sc, n_chunks);
-    return launch_attn_merge(sc, n_chunks, kAttnChunk, rows, n_q, g.d, st, 0, out, s);
+    dim3 grid(n_chunks, g.n_kv, n_seq);
+    CASS_PDL_LAUNCH(k_verify_attn, grid, dim3(kVaThreads), smem, s, g, k_cache, v_cache, qkv, rps, n_q, st, sc, n_chunks);
+    return launch_attn_merge(sc, n_chunks, kAttnChunk, n_seq * rps, rps, n_q, g.d, st, 0, out, s);
 }
 
 }  // namespace cass

@@ -2,9 +2,9 @@
 // memory-bound on the bf16 weights): Y[r][n] = sum_k W[n][k] X[r][k], bf16 operands, fp32 accumulation.
 //
 // tcgen05 version, "swap-AB": the weights are the M operand (128 output features per CTA), the token rows the N
-// operand (always padded to 16 columns), the accumulator lives in tensor memory.  One CTA = one 128-feature tile x
+// operand (padded to BN = 16, 32 or 64 columns), the accumulator lives in tensor memory.  One CTA = one 128-feature tile x
 // one K range (split-K so that small matrices still fill the GPU); warp 0 streams 128x64 weight tiles and the
-// 16x64 activation tile through a ring of TMA loads (128-byte swizzle), warp 1 issues the MMAs, warps 2-5 read the
+// BNx64 activation tile through a ring of TMA loads (128-byte swizzle), warp 1 issues the MMAs, warps 2-5 read the
 // accumulator back and store fp32 partial sums; a second kernel adds the K ranges in fixed order.
 //
 // Row-count invariance: an accumulator column belongs to one token row, the tile shape, the K ranges and the order
@@ -15,11 +15,13 @@
 
 namespace cass {
 
-constexpr int kTcBM = 128, kTcBN = 16, kTcBK = 64, kTcStages = 6;
-constexpr int kTcABytes = kTcBM * kTcBK * 2, kTcBBytes = kTcBN * kTcBK * 2;
+constexpr int kTcBM = 128, kTcBK = 64;
+constexpr int tc_stages(int bn) { return bn <= 16 ? 6 : bn <= 32 ? 5 : 4; }      // two CTAs per SM at every bn
+constexpr int kTcABytes = kTcBM * kTcBK * 2;
 constexpr int kTcThreads = 192;
-constexpr int kTcSmem = kTcStages * (kTcABytes + kTcBBytes) + 256 + 1024;     // + barriers + alignment slack
-constexpr int kTcTmemCols = 32;
+constexpr int tc_b_bytes(int bn) { return bn * kTcBK * 2; }
+constexpr int tc_smem(int bn) { return tc_stages(bn) * (kTcABytes + tc_b_bytes(bn)) + 256 + 1024; }     // + barriers + alignment slack
+constexpr int tc_tmem_cols(int bn) { return bn <= 32 ? 32 : 64; }                                   // a power of two >= 32
 
 // ---- tensor maps ------------------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -79,18 +81,21 @@ __device__ __forceinline__ uint64_t tc_smem_desc(const void* p) {
     return d;
 }
 
-// Instruction descriptor of kind::f16: D fp32, A and B bf16, both K-major, M = 128, N = 16.
-constexpr uint32_t kTcIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kTcBN >> 3) << 17) | ((uint32_t)(kTcBM >> 4) << 24);
+// Instruction descriptor of kind::f16: D fp32, A and B bf16, both K-major, M = 128, N = bn.
+constexpr uint32_t tc_idesc(int bn) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(kTcBM >> 4) << 24);
+}
 
-__device__ __forceinline__ void tc_mma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t accumulate) {
+__device__ __forceinline__ void tc_mma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
     asm volatile(
         "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
-        "l"(adesc), "l"(bdesc), "r"(kTcIdesc), "r"(accumulate)
+        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
 
-// grid (m tiles, k splits).  partial: fp32 [k splits][16][n].
+// grid (m tiles, k splits).  partial: fp32 [k splits][BN][n].
+template <int BN>
 __global__ void __launch_bounds__(kTcThreads) k_verify_gemm_tc(const __grid_constant__ CUtensorMap map_w,
                                                                 const __grid_constant__ CUtensorMap map_x,
                                                                 float* __restrict__ partial, int rows, int n,
@@ -98,6 +103,8 @@ __global__ void __launch_bounds__(kTcThreads) k_verify_gemm_tc(const __grid_cons
     extern __shared__ uint8_t smem_dyn[];
     uint8_t* base = reinterpret_cast<uint8_t*>(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);     // swizzled tiles: 1024-byte aligned
     uint8_t* sA = base;
+    constexpr int kTcBBytes = tc_b_bytes(BN), kTcTmemCols = tc_tmem_cols(BN), kTcStages = tc_stages(BN);
+    constexpr uint32_t kIdesc = tc_idesc(BN);
     uint8_t* sB = base + kTcStages * kTcABytes;
     uint64_t* full = reinterpret_cast<uint64_t*>(sB + kTcStages * kTcBBytes);
     uint64_t* empty = full + kTcStages;
@@ -147,7 +154,7 @@ __global__ void __launch_bounds__(kTcThreads) k_verify_gemm_tc(const __grid_cons
             const uint64_t ad = tc_smem_desc(sA + s * kTcABytes), bd = tc_smem_desc(sB + s * kTcBBytes);
 #pragma unroll
             for (int kk = 0; kk < kTcBK / 16; ++kk)      // 16 bf16 = 32 bytes along K inside the swizzle row: +2 in the address field
-                tc_mma(tmem, ad + (uint64_t)(kk * 2), bd + (uint64_t)(kk * 2), (uint32_t)((kb | kk) != 0));
+                tc_mma(tmem, ad + (uint64_t)(kk * 2), bd + (uint64_t)(kk * 2), kIdesc, (uint32_t)((kb | kk) != 0));
             tc_commit(&empty[s]);                        // frees the stage once these MMAs have read it
         }
         tc_commit(acc_ready);                            // accumulator complete (or abandoned after a time-out)
@@ -157,18 +164,21 @@ __global__ void __launch_bounds__(kTcThreads) k_verify_gemm_tc(const __grid_cons
             __syncwarp();
             tc_fence_after();
             const int q = warp & 3;
-            uint32_t v[16];
-            asm volatile(
-                "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-                : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
-                  "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
-                : "r"(tmem + ((uint32_t)(q * 32) << 16)));
-            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
             const int feat = m0 + q * 32 + lane;
-            if (feat < n && nkb > 0) {
 #pragma unroll
-                for (int r = 0; r < kTcBN; ++r)
-                    if (r < rows) partial[((size_t)ks * kTcBN + r) * n + feat] = __uint_as_float(v[r]);
+            for (int c0 = 0; c0 < BN; c0 += 16) {          // 16 accumulator columns (token rows) at a time
+                uint32_t v[16];
+                asm volatile(
+                    "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+                    : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+                      "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+                    : "r"(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)c0));
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                if (feat < n && nkb > 0) {
+#pragma unroll
+                    for (int r = 0; r < 16; ++r)
+                        if (c0 + r < rows) partial[((size_t)ks * BN + c0 + r) * n + feat] = __uint_as_float(v[r]);
+                }
             }
         } else {
             atomicExch(d_status, CASS_ERR_TIMEOUT);
@@ -182,14 +192,14 @@ __global__ void __launch_bounds__(kTcThreads) k_verify_gemm_tc(const __grid_cons
     }
 }
 
-__global__ void k_verify_gemm_finish(const float* __restrict__ partial, int rows, int n, int n_split,
+__global__ void k_verify_gemm_finish(const float* __restrict__ partial, int rows, int bn, int n, int n_split,
                                      uint16_t* __restrict__ y_bf16, float* __restrict__ y_f32) {
     pdl_launch_dependents();
     pdl_wait();
     const int j = blockIdx.x * blockDim.x + threadIdx.x, r = blockIdx.y;
     if (j >= n || r >= rows) return;
     float acc = 0.f;
-    for (int s = 0; s < n_split; ++s) acc += partial[((size_t)s * kTcBN + r) * n + j];
+    for (int s = 0; s < n_split; ++s) acc += partial[((size_t)s * bn + r) * n + j];
     if (y_f32) y_f32[(size_t)r * n + j] = acc;
     if (y_bf16) y_bf16[(size_t)r * n + j] = float_to_bf16_bits(acc);
 }
@@ -206,39 +216,50 @@ static void split_plan(int n, int k, int* kb_total, int* kb_per_split, int* n_sp
     *n_split = ceil_div(*kb_total, *kb_per_split);
 }
 
-Partials verify_gemm_partials(const float* partial, int n, int k) {
+Partials verify_gemm_partials(const float* partial, int n, int k, int bn) {
     int kbt, kbs, ns;
     split_plan(n, k, &kbt, &kbs, &ns);
-    return Partials{partial, ns, (size_t)kTcBN * n, (size_t)n};
+    return Partials{partial, ns, (size_t)bn * n, (size_t)n};
 }
 
-size_t verify_gemm_partial_floats(int n, int k) {
+size_t verify_gemm_partial_floats(int n, int k, int bn) {
     int kbt, kbs, ns;
     split_plan(n, k, &kbt, &kbs, &ns);
-    return (size_t)ns * kTcBN * n;
+    return (size_t)ns * bn * n;
 }
 
-int launch_verify_gemm(const uint16_t* W, const uint16_t* X, int rows, int n, int k, float* partial, uint16_t* y_bf16,
+template <int BN>
+static int launch_tc(const CUtensorMap& mw, const CUtensorMap& mx, float* partial, int rows, int n, int kbt, int kbs, int ns,
+                     int32_t* d_status, cudaStream_t s) {
+    static bool attr = false;
+    if (!attr) {
+        CASS_CUDA_CHECK(cudaFuncSetAttribute(k_verify_gemm_tc<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc_smem(BN)));
+        attr = true;
+    }
+    dim3 grid(ceil_div(n, kTcBM), ns);
+    CASS_PDL_LAUNCH(k_verify_gemm_tc<BN>, grid, dim3(kTcThreads), (size_t)tc_smem(BN), s, mw, mx, partial, rows, n, kbt, kbs, d_status);
+    return CASS_OK;
+}
+
+int launch_verify_gemm(const uint16_t* W, const uint16_t* X, int rows, int bn, int n, int k, float* partial, uint16_t* y_bf16,
                        float* y_f32, int32_t* d_status, cudaStream_t s) {
-    if (rows < 1 || rows > kMaxVerifyRows || (k % 8) || n < 1 || !partial || !d_status) return CASS_ERR_INVALID_ARG;
+    if (rows < 1 || rows > bn || (bn != 16 && bn != 32 && bn != 64) || (k % 8) || n < 1 || !partial || !d_status)
+        return CASS_ERR_INVALID_ARG;
     if (((uintptr_t)W & 15) || ((uintptr_t)X & 15)) return CASS_ERR_INVALID_ARG;
     CUtensorMap mw, mx;
     int rc = make_map(&mw, W, n, k, kTcBM);
     if (rc) return rc;
-    rc = make_map(&mx, X, kMaxVerifyRows, k, kTcBN);      // the activation buffer always has 16 rows
+    rc = make_map(&mx, X, bn, k, bn);      // the activation buffer always has bn rows
     if (rc) return rc;
     int kbt, kbs, ns;
     split_plan(n, k, &kbt, &kbs, &ns);
-    static bool attr = false;
-    if (!attr) {
-        CASS_CUDA_CHECK(cudaFuncSetAttribute(k_verify_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmem));
-        attr = true;
-    }
-    dim3 grid(ceil_div(n, kTcBM), ns);
-    CASS_PDL_LAUNCH(k_verify_gemm_tc, grid, dim3(kTcThreads), (size_t)kTcSmem, s, mw, mx, partial, rows, n, kbt, kbs, d_status);
+    if (bn == 16) rc = launch_tc<16>(mw, mx, partial, rows, n, kbt, kbs, ns, d_status, s);
+    else if (bn == 32) rc = launch_tc<32>(mw, mx, partial, rows, n, kbt, kbs, ns, d_status, s);
+    else rc = launch_tc<64>(mw, mx, partial, rows, n, kbt, kbs, ns, d_status, s);
+    if (rc) return rc;
     if (!y_bf16 && !y_f32) return CASS_OK;          // the caller's next kernel adds the parts itself
     dim3 g2(ceil_div(n, 256), rows);
-    CASS_PDL_LAUNCH(k_verify_gemm_finish, g2, dim3(256), 0, s, (const float*)partial, rows, n, ns, y_bf16, y_f32);
+    CASS_PDL_LAUNCH(k_verify_gemm_finish, g2, dim3(256), 0, s, (const float*)partial, rows, bn, n, ns, y_bf16, y_f32);
     return CASS_OK;
 }
 
@@ -248,13 +269,14 @@ using namespace cass;
 
 extern "C" size_t cass_verify_gemm_scratch_bytes(int n, int k) {
     if (n < 1 || k < 1) return 0;
-    return verify_gemm_partial_floats(n, k) * sizeof(float);
+    return verify_gemm_partial_floats(n, k, kMaxRows) * sizeof(float);
 }
 
 extern "C" int cass_verify_gemm(const void* W_bf16, const void* X_bf16, int rows, int n, int k, void* scratch,
                                 size_t scratch_bytes, void* y_bf16, float* y_f32, int32_t* d_status, void* stream) {
     if (!W_bf16 || !X_bf16 || !scratch || (!y_bf16 && !y_f32)) return CASS_ERR_INVALID_ARG;
     if (n < 1 || k < 1 || scratch_bytes < cass_verify_gemm_scratch_bytes(n, k)) return CASS_ERR_CAPACITY;
-    return launch_verify_gemm((const uint16_t*)W_bf16, (const uint16_t*)X_bf16, rows, n, k, (float*)scratch, (uint16_t*)y_bf16,
-                              y_f32, d_status, (cudaStream_t)stream);
+    if (rows < 1 || rows > kMaxRows) return CASS_ERR_INVALID_ARG;
+    return launch_verify_gemm((const uint16_t*)W_bf16, (const uint16_t*)X_bf16, rows, verify_gemm_bn(rows), n, k, (float*)scratch,
+                              (uint16_t*)y_bf16, y_f32, d_status, (cudaStream_t)stream);
 }

@@ -37,15 +37,18 @@ def fuse_layer_weights(lw: dict) -> dict:
 
 
 class Engine:
-    """One sequence on one GPU.  `weights` = {"layers": [fused layer dicts], "embed", "lm_head", "norm_final"}
-    of bf16 CUDA tensors (see fuse_layer_weights)."""
+    """`batch` sequences (1, 2, 4 or 8) decoded together on one GPU.  `weights` = {"layers": [fused layer dicts],
+    "embed", "lm_head", "norm_final"} of bf16 CUDA tensors (see fuse_layer_weights).  With batch = 1 the token-level
+    results (prefill's return, generate's list) are plain ints; with more they are per-sequence lists."""
 
     def __init__(self, shape, weights: dict, fmt: B.Format | None = None, max_seq: int = 1024, gamma_max: int = 8,
-                 device="cuda"):
+                 device="cuda", batch: int = 1):
         self.shape, self.w, self.device = shape, weights, torch.device(device)
         self.fmt = fmt if fmt is not None else B.default_format()
+        self.batch = batch
         self.desc = B.ModelDesc(shape.n_layers, shape.hidden, shape.n_q_heads, shape.n_kv_heads, shape.head_dim,
-                                shape.ffn, shape.vocab, max_seq, 1, gamma_max, shape.rope_theta, shape.rms_eps)
+                                shape.ffn, shape.vocab, max_seq, batch, gamma_max, shape.rope_theta, shape.rms_eps)
+        self.max_rows = B.cass_session_rows(self.desc)
         nbytes = B.cass_session_bytes(self.desc, self.fmt)
         self.mem = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
         self._lw = (B.LayerWeights * shape.n_layers)()
@@ -58,11 +61,13 @@ class Engine:
         self.session = B.cass_session_init(self.mem, self.desc, self.fmt, self._mw, None)
         self.blobs = None
         self.n_prompt = 0
-        # step buffers: toks[0] = last emitted token, toks[1..g] = drafted tokens
-        self.toks = torch.zeros(32, dtype=torch.int32, device=self.device)
-        self.targ = torch.zeros(32, dtype=torch.int32, device=self.device)
-        self.out_tokens = torch.zeros(32, dtype=torch.int32, device=self.device)
-        self.n_acc = torch.zeros(1, dtype=torch.int32, device=self.device)
+        # step buffers, [batch][gamma + 1] for the gamma in use: toks[b][0] = last emitted token of sequence b,
+        # toks[b][1..g] = its drafted tokens
+        self.toks = torch.zeros(64, dtype=torch.int32, device=self.device)
+        self.targ = torch.zeros(64, dtype=torch.int32, device=self.device)
+        self.out_tokens = torch.zeros(64, dtype=torch.int32, device=self.device)
+        self.n_acc = torch.zeros(8, dtype=torch.int32, device=self.device)
+        self._stride = 1              # gamma + 1 of the layout the token buffers are in
         self._graphs = {}
 
     def close(self):
@@ -75,24 +80,27 @@ class Engine:
         B.cass_session_reset(self.session)
         self.n_prompt = 0
 
-    def prefill(self, prompt: torch.Tensor, calibrate: bool = False) -> int:
-        """Target pass over the prompt in chunks of up to 16 rows (bf16 cache only); returns the first generated
-        token.  With calibrate, the Wanda activation statistics are accumulated on the way."""
-        prompt = prompt.to(self.device, torch.int32).contiguous()
-        n = int(prompt.numel())
+    def prefill(self, prompt: torch.Tensor, calibrate: bool = False):
+        """Target pass over the prompt(s) ([n] or [batch][n] token ids, equal lengths) in chunks of up to 16 rows per
+        sequence (bf16 cache only); returns the first generated token (per sequence).  With calibrate, the Wanda
+        activation statistics are accumulated on the way."""
+        prompt = prompt.to(self.device, torch.int32).reshape(self.batch, -1).contiguous()
+        n = int(prompt.shape[1])
+        chunk = min(16, self.max_rows // self.batch)
         B.cass_calib_enable(self.session, calibrate)
-        pos = 0
+        pos, rows = 0, 0
         while pos < n:
-            rows = min(16, n - pos)
+            rows = min(chunk, n - pos)
             B.cass_set_len(self.session, pos)
-            B.cass_verify(self.session, prompt[pos: pos + rows], rows - 1, self.targ)
+            B.cass_verify(self.session, prompt[:, pos: pos + rows].contiguous(), rows - 1, self.targ)
             pos += rows
         B.cass_calib_enable(self.session, False)
         B.cass_set_len(self.session, n)
         self.n_prompt = n
-        first = self.targ[(n - 1) % 16: (n - 1) % 16 + 1]
-        self.toks[0:1] = first
-        return int(first.item())
+        first = self.targ[: self.batch * rows].view(self.batch, rows)[:, rows - 1].clone()
+        self._stride = 1
+        self.toks[: self.batch] = first
+        return int(first[0].item()) if self.batch == 1 else first.tolist()
 
     def calib_norms(self) -> dict:
         cnt = B.cass_calib_norms_count(self.desc)
@@ -152,21 +160,41 @@ class Engine:
         B.cass_kv_build_codebook(self.session, self.n_prompt)
 
     # ------------------------------------------------------------------ decoding
+    def next_tokens(self) -> torch.Tensor:
+        """The token every sequence feeds into its next step ([batch], a copy)."""
+        return self.toks[: self.batch * self._stride: self._stride].clone()
+
+    def set_next_tokens(self, toks: torch.Tensor, non_blocking: bool = False):
+        self.toks[: self.batch * self._stride: self._stride].copy_(toks, non_blocking=non_blocking)
+
+    def _layout(self, gamma: int):
+        """Moves the next input tokens to where a step with this gamma expects them: toks[b * (gamma + 1)]."""
+        if self._stride != gamma + 1:
+            nxt = self.toks[: self.batch * self._stride: self._stride].clone()
+            self._stride = gamma + 1
+            self.toks[: self.batch * self._stride: self._stride] = nxt
+
     def _spec_step(self, gamma: int):
+        s = gamma + 1
         for i in range(gamma):
-            B.cass_draft_step(self.session, self.toks[i: i + 1], self.toks[i + 1: i + 2])
+            B.cass_draft_step(self.session, self.toks[i:], self.toks[i + 1:], tok_stride=s)
         B.cass_verify(self.session, self.toks, gamma, self.targ)
-        B.cass_accept(self.session, self.toks[1:], self.targ, gamma, self.n_acc, self.out_tokens, self.toks)
+        B.cass_accept(self.session, self.toks[1:], self.targ, gamma, self.n_acc, self.out_tokens, self.toks,
+                      draft_stride=s, next_stride=s)
 
     def step(self, gamma: int):
-        """One speculative step (gamma = 0: one plain autoregressive step).  Results stay on the device:
-        n_acc[0] accepted drafts, out_tokens[0..n_acc] emitted tokens, toks[0] the next input."""
+        """One speculative step (gamma = 0: one plain autoregressive step) of every sequence.  Results stay on the
+        device: n_acc[b] accepted drafts, out_tokens[b][0..n_acc[b]] emitted tokens, toks[b][0] the next input
+        (arrays of gamma + 1 entries per sequence)."""
+        self._layout(gamma)
         self._spec_step(gamma)
 
     def generate(self, n_tokens: int, gamma: int, use_graph: bool = False, sync_every: int = 1):
-        """Emits at least n_tokens tokens after the prefill token.  Returns (tokens list, StepStats)."""
-        out: list[int] = []
+        """Emits at least n_tokens tokens per sequence after the prefill token.  Returns (tokens, StepStats): tokens
+        is a list (batch 1) or a list of per-sequence lists."""
+        out: list[list[int]] = [[] for _ in range(self.batch)]
         stats = StepStats()
+        self._layout(gamma)
         if use_graph and gamma not in self._graphs:
             # capture needs a warm step and the captured step also executes nothing by itself: do both here
             self._spec_step(gamma)
@@ -175,21 +203,26 @@ class Engine:
             with torch.cuda.graph(graph):
                 self._spec_step(gamma)
             self._graphs[gamma] = graph
-        while len(out) < n_tokens:
+        while min(len(o) for o in out) < n_tokens:
             if use_graph:
                 self._graphs[gamma].replay()
             else:
                 self._spec_step(gamma)
             self._collect(out, stats)
-        return out, stats
+        return (out[0] if self.batch == 1 else out), stats
 
     def _collect(self, out, stats):
-        a = int(self.n_acc.item())
-        toks = self.out_tokens[: a + 1].tolist()
-        out.extend(toks)
+        s = self._stride
+        acc = self.n_acc[: self.batch].tolist()
+        toks = self.out_tokens[: self.batch * s].view(self.batch, s).tolist()
+        for b, a in enumerate(acc):
+            out[b].extend(toks[b][: a + 1])
+            stats.accepted += a
+            stats.emitted += a + 1
         stats.steps += 1
-        stats.accepted += a
-        stats.emitted += a + 1
 
     def status(self) -> tuple[int, int]:
         return B.cass_session_status(self.session)
+
+    def lens(self) -> list[int]:
+        return B.cass_session_lens(self.session, self.batch)

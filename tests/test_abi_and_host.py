@@ -41,10 +41,21 @@ def test_host_only_queries_and_argument_checks():
     assert e.value.code == cass.ERR_INVALID_ARG
     desc = cass.ModelDesc(2, 256, 4, 2, 64, 688, 1024, 256, 1, 4, 1.0e4, 1.0e-5)
     assert cass.cass_session_bytes(desc, fmt) > 0
-    desc2 = cass.ModelDesc(2, 256, 4, 2, 64, 688, 1024, 256, 2, 4, 1.0e4, 1.0e-5)      # batch 2 is not supported
+    desc2 = cass.ModelDesc(2, 256, 4, 2, 64, 688, 1024, 256, 2, 4, 1.0e4, 1.0e-5)      # two sequences: twice the KV storage
+    desc8 = cass.ModelDesc(2, 256, 4, 2, 64, 688, 1024, 256, 8, 4, 1.0e4, 1.0e-5)
+    b1, b2, b8 = (cass.cass_session_bytes(d, fmt) for d in (desc, desc2, desc8))
+    assert b1 < b2 < b8
+    kv_seq = 2 * 2 * 256 * 2 * 64 * 2                    # layers x (K, V) x positions x heads x dim x bf16: the dense caches alone
+    assert b2 - b1 >= kv_seq and b8 - b2 >= 6 * kv_seq
+    assert [cass.cass_session_rows(d) for d in (desc, desc2, desc8)] == [16, 16, 64]
+    desc3 = cass.ModelDesc(2, 256, 4, 2, 64, 688, 1024, 256, 3, 4, 1.0e4, 1.0e-5)      # 3 sequences: not a supported count
     with pytest.raises(cass.CassError) as e:
-        cass.cass_session_bytes(desc2, fmt)
+        cass.cass_session_bytes(desc3, fmt)
     assert e.value.code == cass.ERR_UNSUPPORTED
+    wide = cass.ModelDesc(2, 256, 4, 2, 64, 688, 1024, 256, 8, 8, 1.0e4, 1.0e-5)       # 8 x 9 rows exceed one call
+    with pytest.raises(cass.CassError) as e:
+        cass.cass_session_bytes(wide, fmt)
+    assert e.value.code == cass.ERR_INVALID_ARG
     assert cass.cass_calib_norms_count(desc) == 2 * 4 * 688 + 256
 
 
