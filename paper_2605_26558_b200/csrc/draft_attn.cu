@@ -193,7 +193,6 @@ __global__ void __launch_bounds__(kDaThreads) k_draft_attn(KvGeom g, KvComp ck0,
     if (t0 >= cur_len) return;
     const int G = n_q / g.n_kv, d = g.d;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const KvComp ck = of_seq(ck0, seq, g.seq_stride), cv = of_seq(cv0, seq, g.seq_stride);
     qkv += (size_t)seq * qkv_stride;
 
     float* q_s = reinterpret_cast<float*>(smem);                              // [d][8]
@@ -209,23 +208,26 @@ __global__ void __launch_bounds__(kDaThreads) k_draft_attn(KvGeom g, KvComp ck0,
         int col = i / kMaxGroup, gi = i % kMaxGroup;
         q_s[i] = gi < G ? bf16_bits_to_float(qkv[(size_t)(head * G + gi) * d + col]) : 0.f;
     }
-    for (int i = tid; i < 512; i += kDaThreads) lut_s[i] = (uint32_t)(i < 256 ? ck.rank_to_exp[i] : cv.rank_to_exp[i - 256]) << 23;
+    {
+        const uint8_t *rk = of_seq(ck0.rank_to_exp, seq, g.seq_stride), *rv = of_seq(cv0.rank_to_exp, seq, g.seq_stride);
+        for (int i = tid; i < 512; i += kDaThreads) lut_s[i] = (uint32_t)(i < 256 ? rk[i] : rv[i - 256]) << 23;
+    }
     for (int i = tid; i < kDaTok * d / 2; i += kDaThreads) reinterpret_cast<uint32_t*>(v_s)[i] = 0u;
 
     // stage this warp's 32 records: warps 0,1 -> K of tokens t0 + 32 w .., warps 2,3 -> V of the same tokens
     const int kind = warp >> 1, tw = warp & 1;
     const int tok = t0 + tw * 32 + lane;
     const bool valid = tok < cur_len;
-    const KvComp& c = kind ? cv : ck;
+    const KvComp& c = kind ? cv0 : ck0;                      // sequence 0's; shifted to this sequence where used
     uint32_t* my_fix = fix_s + warp * (g.wpt + 1) * 32;
     uint32_t* my_una = una_s + warp * (kDaUnaStage + 2) * 32;
     {
-        const uint32_t* fixed = c.fixed + ((size_t)head * g.n_blocks + tok / 32) * g.wpt * 32;
+        const uint32_t* fixed = of_seq(c.fixed, seq, g.seq_stride) + ((size_t)head * g.n_blocks + tok / 32) * g.wpt * 32;
         for (int w = 0; w < g.wpt; ++w) my_fix[w * 32 + lane] = fixed[w * 32 + lane];          // coalesced block copy
         my_fix[g.wpt * 32 + lane] = 0u;
     }
-    const uint32_t* off = c.off + (size_t)head * (g.max_seq + 1);
-    const uint32_t* arena = c.arena + (size_t)head * g.arena_words;
+    const uint32_t* off = of_seq(c.off, seq, g.seq_stride) + (size_t)head * (g.max_seq + 1);
+    const uint32_t* arena = of_seq(c.arena, seq, g.seq_stride) + (size_t)head * g.arena_words;
     uint32_t o0 = 0, n_una = 0;
     if (valid) { o0 = off[tok]; n_una = off[tok + 1] - o0; }
     const bool staged = n_una <= (uint32_t)kDaUnaStage;

@@ -1,6 +1,8 @@
 // Internal launchers shared between the translation units of the library.
 #pragma once
 
+#include <type_traits>
+
 #include "common.cuh"
 
 namespace cass {
@@ -36,7 +38,8 @@ struct KvGeom {
 // The same object of sequence b: every sequence's KV storage has the same internal layout.
 template <class P>
 __host__ __device__ __forceinline__ P* of_seq(P* p, int b, size_t seq_stride) {
-    return reinterpret_cast<P*>(reinterpret_cast<uintptr_t>(p) + (size_t)b * seq_stride);
+    using Byte = typename std::conditional<std::is_const<P>::value, const char, char>::type;
+    return reinterpret_cast<P*>(reinterpret_cast<Byte*>(p) + (size_t)b * seq_stride);     // pointer arithmetic: stays a global-memory pointer
 }
 __host__ __device__ __forceinline__ KvComp of_seq(const KvComp& c, int b, size_t seq_stride) {
     KvComp r;

@@ -85,14 +85,15 @@ __global__ void __launch_bounds__(256) k_kv_append(KvGeom g, KvComp ck, KvComp c
     pdl_wait();
     const int head = blockIdx.x, kind = blockIdx.y, seq = seq0 + blockIdx.z;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const KvComp c = of_seq(kind ? cv : ck, seq, g.seq_stride);
+    const KvComp& c0 = kind ? cv : ck;                       // sequence 0's; shifted to this sequence below
+    const uint8_t* exp_to_rank = of_seq(c0.exp_to_rank, seq, g.seq_stride);
     const uint16_t* src = (kind ? src_v : src_k) + (size_t)blockIdx.z * n_new * row_stride;
     uint16_t* cache = of_seq(kind ? v_cache : k_cache, seq, g.seq_stride);
     const int start_pos = start_pos_arg >= 0 ? start_pos_arg : st->len[seq] + (use_inflight ? st->inflight[seq] : 0);
     const int nj = g.d / 32, t_bits = g.t, F = 8 - t_bits, per = 32 / F;
-    uint32_t* off = c.off + (size_t)head * (g.max_seq + 1);
-    uint32_t* arena = c.arena + (size_t)head * g.arena_words;
-    uint32_t* fixed = c.fixed + (size_t)head * g.n_blocks * g.wpt * 32;
+    uint32_t* off = of_seq(c0.off, seq, g.seq_stride) + (size_t)head * (g.max_seq + 1);
+    uint32_t* arena = of_seq(c0.arena, seq, g.seq_stride) + (size_t)head * g.arena_words;
+    uint32_t* fixed = of_seq(c0.fixed, seq, g.seq_stride) + (size_t)head * g.n_blocks * g.wpt * 32;
 
     for (int base = 0; base < n_new; base += kKvWarps) {
         const int i = base + warp;
@@ -124,7 +125,7 @@ __global__ void __launch_bounds__(256) k_kv_append(KvGeom g, KvComp ck, KvComp c
                     if (j < nj) {
                         uint32_t bm = __brev(__ballot_sync(0xffffffffu, keep[j]));   // channel c at bit 31 - c%32
                         if (lane == 0) s_fix[warp][j] = bm;
-                        uint32_t len = keep[j] ? (uint32_t)c.exp_to_rank[(bits[j] >> 7) & 0xFF] + 1u : 0u;
+                        uint32_t len = keep[j] ? (uint32_t)exp_to_rank[(bits[j] >> 7) & 0xFF] + 1u : 0u;
                         uint32_t incl = len;
 #pragma unroll
                         for (int o = 1; o < 32; o <<= 1) {

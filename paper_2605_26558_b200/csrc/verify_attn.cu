@@ -14,8 +14,8 @@ constexpr int kVaMaxPairs = kVaRowBatch * kVaMaxGroup;      // (row, query head)
 constexpr int kVaHalfPairs = kVaMaxPairs / 2;
 
 // grid (chunk, KV head, sequence); `rows` = rows of each sequence in this call.
-__global__ void __launch_bounds__(kVaThreads) k_verify_attn(KvGeom g, const uint16_t* __restrict__ k_cache,
-                                                            const uint16_t* __restrict__ v_cache, const uint16_t* __restrict__ qkv,
+__global__ void __launch_bounds__(kVaThreads) k_verify_attn(KvGeom g, const uint16_t* __restrict__ k_cache0,
+                                                            const uint16_t* __restrict__ v_cache0, const uint16_t* __restrict__ qkv0,
                                                             int rows, int n_q, const DevState* __restrict__ st, AttnScratch sc,
                                                             int n_chunks_alloc) {
     extern __shared__ __align__(16) uint8_t smem[];
@@ -23,14 +23,14 @@ __global__ void __launch_bounds__(kVaThreads) k_verify_attn(KvGeom g, const uint
     pdl_wait();
     const int chunk = blockIdx.x, head = blockIdx.y, seq = blockIdx.z;
     const int len = st->len[seq];
-    k_cache = of_seq(k_cache, seq, g.seq_stride);
-    v_cache = of_seq(v_cache, seq, g.seq_stride);
+    const uint16_t* __restrict__ k_cache = of_seq(k_cache0, seq, g.seq_stride);
+    const uint16_t* __restrict__ v_cache = of_seq(v_cache0, seq, g.seq_stride);
     const int t0 = chunk * kAttnChunk;
     if (t0 >= len + rows) return;
     const int d = g.d, G = n_q / g.n_kv, ks = d + 8;                  // padded K row stride (elements)
     const int qkv_dim = (n_q + 2 * g.n_kv) * d;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    qkv += (size_t)seq * rows * qkv_dim;                                 // this sequence's rows
+    const uint16_t* __restrict__ qkv = qkv0 + (size_t)seq * rows * qkv_dim;     // this sequence's rows
     uint16_t* k_s = reinterpret_cast<uint16_t*>(smem);                         // [64][d+8]
     uint16_t* v_s = k_s + kAttnChunk * ks;                                      // [64][d]
     float* q_s = reinterpret_cast<float*>(v_s + kAttnChunk * d);                // [pairs][d]

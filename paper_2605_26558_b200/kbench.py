@@ -163,7 +163,7 @@ def bench_draft_attn(n_pos, layers, iters):
     return res
 
 
-def step_breakdown(gamma=4, n_prompt=512, steps=3):
+def step_breakdown(gamma=4, n_prompt=512, steps=3, batch=1):
     """Per-kernel device time of the speculative step on the full Llama-3-8B shape, from the CUPTI kernel trace of a
     few eager steps (warm, not under ncu)."""
     import re
@@ -177,8 +177,8 @@ def step_breakdown(gamma=4, n_prompt=512, steps=3):
     gw = {"layers": [engine.fuse_layer_weights(lw) for lw in wt["layers"]], "embed": wt["embed"], "lm_head": wt["lm_head"],
           "norm_final": wt["norm_final"]}
     del wt
-    eng = engine.Engine(shape, gw, max_seq=n_prompt + 256, gamma_max=max(gamma, 1))
-    eng.prefill(synth.random_prompt(n_prompt, shape.vocab, 0), calibrate=True)
+    eng = engine.Engine(shape, gw, max_seq=n_prompt + 256, gamma_max=max(gamma, 1), batch=batch)
+    eng.prefill(torch.stack([synth.random_prompt(n_prompt, shape.vocab, b) for b in range(batch)]), calibrate=True)
     eng.encode_weights(eng.calib_norms())
     eng.build_kv_codebook()
     for _ in range(2):
@@ -198,7 +198,7 @@ def step_breakdown(gamma=4, n_prompt=512, steps=3):
     rows = [{"kernel": k, "launches_per_step": v[0] / steps, "us_per_step": v[1] / steps, "share": v[1] / tot,
              "avg_us": v[1] / v[0]} for k, v in sorted(agg.items(), key=lambda kv: -kv[1][1])]
     eng.close()
-    return [{"kernel": "step_breakdown", "gamma": gamma, "kernel_us_per_step": tot / steps}] + rows
+    return [{"kernel": "step_breakdown", "gamma": gamma, "batch": batch, "kernel_us_per_step": tot / steps}] + rows
 
 
 def main():
@@ -211,6 +211,7 @@ def main():
     ap.add_argument("--gamma", type=int, default=4)
     ap.add_argument("--chunk", type=int, default=0, help="columns per decode chunk of the weight format (0 = default 256)")
     ap.add_argument("--seg", type=int, default=0, help="columns per superblock of the weight format (0 = default 2048)")
+    ap.add_argument("--batch", type=int, default=1, help="sequences decoded together (step breakdown)")
     ap.add_argument("--p", type=int, default=400)
     ap.add_argument("--t", type=int, default=4)
     args = ap.parse_args()
@@ -227,7 +228,7 @@ def main():
             copies = args.copies or max(2, int(300e6 / (n * k * 2)) + 1)
             out.append(bench_verify_gemm(name, copies, args.iters))
     if args.kernel == "step":
-        out.extend(step_breakdown(gamma=args.gamma))
+        out.extend(step_breakdown(gamma=args.gamma, batch=args.batch))
     if args.kernel in ("attn", "all"):
         for n_pos in ([args.positions] if args.positions else [4096, 32768]):
             out.extend(bench_draft_attn(n_pos, max(2, int(3.0e5 / n_pos) + 1), args.iters))
