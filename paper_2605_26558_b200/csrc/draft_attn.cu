@@ -13,9 +13,8 @@ namespace cass {
 
 constexpr int kDaTok = kAttnChunk;            // tokens per CTA
 constexpr int kDaThreads = 128;
-constexpr int kDaUnaStage = 32;               // staged unary words per token; longer records are read in place
+constexpr int kDaUnaStage = 12;               // staged unary words per token (a typical record has 5-8); longer records are read in place
 constexpr int kMaxGroup = 8;                  // query heads per KV head
-constexpr int kQStride = kMaxGroup * 4;       // bytes per column of the query tile q_s[col][8]
 
 __device__ __forceinline__ uint32_t da_shl(uint32_t v, uint32_t s) {
     uint32_t r;
@@ -29,20 +28,22 @@ __device__ __forceinline__ uint32_t da_lds(uint32_t a) {
 }
 
 // What happens to a decoded value.  K: multiply with the query tile; V: store into the token's dense row.
+// GQ = query heads the tile has room for (4 or 8): q_s[col][GQ] floats.
+template <int GQ>
 struct EmitK {
-    float acc[kMaxGroup], g[kMaxGroup];
+    float acc[GQ], g[GQ];
     uint32_t q_a;
-    int G;
     __device__ __forceinline__ void reset() {
 #pragma unroll
-        for (int i = 0; i < kMaxGroup; ++i) g[i] = 0.f;
+        for (int i = 0; i < GQ; ++i) g[i] = 0.f;
     }
-    __device__ __forceinline__ void fma_into(float (&dst)[kMaxGroup], uint32_t off, uint32_t wb) {
+    __device__ __forceinline__ void fma_into(float (&dst)[GQ], uint32_t off, uint32_t wb) {
         const float w = __uint_as_float(wb);
-        float4 a, b = make_float4(0.f, 0.f, 0.f, 0.f);
+        float4 a;
         asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(a.x), "=f"(a.y), "=f"(a.z), "=f"(a.w) : "r"(q_a + off));
         dst[0] = fmaf(w, a.x, dst[0]); dst[1] = fmaf(w, a.y, dst[1]); dst[2] = fmaf(w, a.z, dst[2]); dst[3] = fmaf(w, a.w, dst[3]);
-        if (G > 4) {
+        if constexpr (GQ > 4) {
+            float4 b;
             asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4+16];" : "=f"(b.x), "=f"(b.y), "=f"(b.z), "=f"(b.w) : "r"(q_a + off));
             dst[4] = fmaf(w, b.x, dst[4]); dst[5] = fmaf(w, b.y, dst[5]); dst[6] = fmaf(w, b.z, dst[6]); dst[7] = fmaf(w, b.w, dst[7]);
         }
@@ -51,12 +52,12 @@ struct EmitK {
     __device__ __forceinline__ void elem(uint32_t off, uint32_t wb, bool valid) { if (valid) fma_into(g, off, wb); }
     __device__ __forceinline__ void commit(int) {
 #pragma unroll
-        for (int i = 0; i < kMaxGroup; ++i) acc[i] += g[i];
+        for (int i = 0; i < GQ; ++i) acc[i] += g[i];
     }
     __device__ __forceinline__ void direct(uint32_t off, uint32_t wb) { fma_into(acc, off, wb); }
     __device__ __forceinline__ void restart() {
 #pragma unroll
-        for (int i = 0; i < kMaxGroup; ++i) acc[i] = 0.f;
+        for (int i = 0; i < GQ; ++i) acc[i] = 0.f;
     }
 };
 
@@ -180,7 +181,7 @@ __device__ __forceinline__ void kv_record_walk(const uint32_t* bmP, const uint32
     }
 }
 
-template <int T>
+template <int T, int GQ>
 __global__ void __launch_bounds__(kDaThreads) k_draft_attn(KvGeom g, KvComp ck0, KvComp cv0, const uint16_t* __restrict__ qkv,
                                                            int qkv_stride, int n_q, const DevState* __restrict__ st, AttnScratch sc,
                                                            int n_chunks_alloc) {
@@ -195,17 +196,18 @@ __global__ void __launch_bounds__(kDaThreads) k_draft_attn(KvGeom g, KvComp ck0,
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     qkv += (size_t)seq * qkv_stride;
 
-    float* q_s = reinterpret_cast<float*>(smem);                              // [d][8]
-    float* sc_s = q_s + d * kMaxGroup;                                        // [8][64] scores -> probabilities
-    float* ml_s = sc_s + kMaxGroup * kDaTok;                                  // [8][2]
-    uint32_t* lut_s = reinterpret_cast<uint32_t*>(ml_s + 2 * kMaxGroup);      // [2][256] rank -> exponent << 23
+    constexpr int kQStride = GQ * 4;                                          // bytes per column of the query tile
+    float* q_s = reinterpret_cast<float*>(smem);                              // [d][GQ]
+    float* sc_s = q_s + d * GQ;                                               // [GQ][64] scores -> probabilities
+    float* ml_s = sc_s + GQ * kDaTok;                                         // [GQ][2]
+    uint32_t* lut_s = reinterpret_cast<uint32_t*>(ml_s + 2 * GQ);             // [2][256] rank -> exponent << 23
     uint32_t* fix_s = lut_s + 512;                                            // [4 warps][wpt + 1][32]
     uint32_t* una_s = fix_s + 4 * (g.wpt + 1) * 32;                           // [4 warps][kDaUnaStage + 2][32]
     uint16_t* v_s = reinterpret_cast<uint16_t*>(una_s + 4 * (kDaUnaStage + 2) * 32);   // [64][d] bf16
 
     const float scale = rsqrtf((float)d);
-    for (int i = tid; i < d * kMaxGroup; i += kDaThreads) {
-        int col = i / kMaxGroup, gi = i % kMaxGroup;
+    for (int i = tid; i < d * GQ; i += kDaThreads) {
+        int col = i / GQ, gi = i % GQ;
         q_s[i] = gi < G ? bf16_bits_to_float(qkv[(size_t)(head * G + gi) * d + col]) : 0.f;
     }
     {
@@ -236,9 +238,8 @@ __global__ void __launch_bounds__(kDaThreads) k_draft_attn(KvGeom g, KvComp ck0,
 
     const uint32_t* lutP = lut_s + kind * 256;
     if (kind == 0) {
-        EmitK em;
+        EmitK<GQ> em;
         em.q_a = smem_u32(q_s);
-        em.G = G;
         em.restart();
         kv_record_walk<T, kQStride>(my_fix + lane, my_fix + g.bm_words * 32 + lane, my_una + lane, smem_u32(lutP), lutP, g.kept, d,
                                     n_una * 32u, valid && staged, em);
@@ -251,7 +252,7 @@ __global__ void __launch_bounds__(kDaThreads) k_draft_attn(KvGeom g, KvComp ck0,
                                            n_una * 32u, lutP, em);
         }
 #pragma unroll
-        for (int gi = 0; gi < kMaxGroup; ++gi)
+        for (int gi = 0; gi < GQ; ++gi)
             if (gi < G) sc_s[gi * kDaTok + tw * 32 + lane] = valid ? em.acc[gi] * scale : -INFINITY;
     } else {
         EmitV em;
@@ -282,18 +283,18 @@ __global__ void __launch_bounds__(kDaThreads) k_draft_attn(KvGeom g, KvComp ck0,
     // o[gi][dim] = sum_t p[gi][t] * v[t][dim]
     const int n_tok = min(kDaTok, cur_len - t0);
     for (int dim = tid; dim < d; dim += kDaThreads) {
-        float acc[kMaxGroup];
+        float acc[GQ];
 #pragma unroll
-        for (int gi = 0; gi < kMaxGroup; ++gi) acc[gi] = 0.f;
+        for (int gi = 0; gi < GQ; ++gi) acc[gi] = 0.f;
 #pragma unroll 4
         for (int t = 0; t < n_tok; ++t) {
             const float v = bf16_bits_to_float(v_s[(size_t)t * d + dim]);
 #pragma unroll
-            for (int gi = 0; gi < kMaxGroup; ++gi)
+            for (int gi = 0; gi < GQ; ++gi)
                 if (gi < G) acc[gi] = fmaf(sc_s[gi * kDaTok + t], v, acc[gi]);
         }
 #pragma unroll
-        for (int gi = 0; gi < kMaxGroup; ++gi)
+        for (int gi = 0; gi < GQ; ++gi)
             if (gi < G) sc.o[(((size_t)seq * n_q + head * G + gi) * n_chunks_alloc + chunk) * d + dim] = acc[gi];
     }
     if (tid < G) {
@@ -360,8 +361,8 @@ int launch_attn_merge(const AttnScratch& sc, int n_chunks_alloc, int chunk_token
     return CASS_OK;
 }
 
-size_t draft_attn_smem_bytes(const KvGeom& g) {
-    return (size_t)g.d * kMaxGroup * 4 + (size_t)kMaxGroup * kDaTok * 4 + 2 * kMaxGroup * 4 + 512 * 4 +
+size_t draft_attn_smem_bytes(const KvGeom& g, int gq) {
+    return (size_t)g.d * gq * 4 + (size_t)gq * kDaTok * 4 + 2 * gq * 4 + 512 * 4 +
            (size_t)4 * (g.wpt + 1) * 32 * 4 + (size_t)4 * (kDaUnaStage + 2) * 32 * 4 + (size_t)kDaTok * g.d * 2 + 64;
 }
 
@@ -370,19 +371,22 @@ int launch_draft_attn(const KvGeom& g, const KvComp& ck, const KvComp& cv, const
     const int G = n_q / g.n_kv;
     if (G > kMaxGroup || g.d > 256 || g.d % 32) return CASS_ERR_UNSUPPORTED;
     const int n_chunks = ceil_div(g.max_seq, kDaTok);
-    const size_t smem = draft_attn_smem_bytes(g);
+    const int gq = G <= 4 ? 4 : 8;
+    const size_t smem = draft_attn_smem_bytes(g, gq);
     dim3 grid(n_chunks, g.n_kv, n_seq);
-#define CASS_DA_LAUNCH(TT)                                                                                           \
+#define CASS_DA_LAUNCH(TT, GG)                                                                                         \
     do {                                                                                                             \
         static size_t attr = 0;                                                                                      \
         if (smem > attr) {                                                                                           \
-            CASS_CUDA_CHECK(cudaFuncSetAttribute(k_draft_attn<TT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
+            CASS_CUDA_CHECK(cudaFuncSetAttribute((k_draft_attn<TT, GG>), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
             attr = smem;                                                                                             \
         }                                                                                                            \
-        CASS_PDL_LAUNCH(k_draft_attn<TT>, grid, dim3(kDaThreads), smem, s, g, ck, cv, qkv, qkv_stride, n_q, st, sc, n_chunks);     \
+        CASS_PDL_LAUNCH((k_draft_attn<TT, GG>), grid, dim3(kDaThreads), smem, s, g, ck, cv, qkv, qkv_stride, n_q, st, sc, n_chunks);     \
     } while (0)
-    if (g.t == 4) CASS_DA_LAUNCH(4);
-    else if (g.t == 0) CASS_DA_LAUNCH(0);
+    if (g.t == 4 && gq == 4) CASS_DA_LAUNCH(4, 4);
+    else if (g.t == 4) CASS_DA_LAUNCH(4, 8);
+    else if (g.t == 0 && gq == 4) CASS_DA_LAUNCH(0, 4);
+    else if (g.t == 0) CASS_DA_LAUNCH(0, 8);
     else return CASS_ERR_UNSUPPORTED;
 #undef CASS_DA_LAUNCH
     CASS_LAUNCH_CHECK();

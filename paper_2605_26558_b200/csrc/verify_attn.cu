@@ -51,8 +51,9 @@ __global__ void __launch_bounds__(kVaThreads) k_verify_attn(KvGeom g, const uint
     }
     const float scale = rsqrtf((float)d);
 
-    for (int r0 = 0; r0 < rows; r0 += kVaRowBatch) {
-        const int nr = min(kVaRowBatch, rows - r0);
+    const int row_batch = kVaMaxPairs / G;                            // rows whose (row, query head) pairs fit one pass
+    for (int r0 = 0; r0 < rows; r0 += row_batch) {
+        const int nr = min(row_batch, rows - r0);
         if (t0 >= len + r0 + nr) continue;                              // no row of this batch sees the chunk (later rows may)
         const int P = nr * G;
         __syncthreads();

@@ -201,6 +201,58 @@ def step_breakdown(gamma=4, n_prompt=512, steps=3, batch=1):
     return [{"kernel": "step_breakdown", "gamma": gamma, "batch": batch, "kernel_us_per_step": tot / steps}] + rows
 
 
+def long_decode(gamma=4, n_tokens=8192, n_prompt=512, config="llama8b"):
+    """Decodes n_tokens greedy tokens after the prompt twice on the full model -- plain bf16 greedy (gamma = 0) and
+    speculatively -- with CUDA-graph steps, compares the two streams token by token and reports tokens/s of both,
+    overall and over the first and last 10 % of the speculative steps (the context grows from n_prompt to
+    n_prompt + n_tokens)."""
+    import time
+    import synth
+    from . import engine
+    dev = torch.device("cuda")
+    shape = {"llama8b": synth.LLAMA3_8B, "qwen": synth.QWEN_LARGE, "tiny": synth.TINY}[config]
+    wt = synth.model_weights(shape, 0, device=dev)
+    gw = {"layers": [engine.fuse_layer_weights(lw) for lw in wt["layers"]], "embed": wt["embed"], "lm_head": wt["lm_head"],
+          "norm_final": wt["norm_final"]}
+    del wt
+    max_seq = (n_prompt + n_tokens + 2 * (gamma + 1) + 32 + 255) // 256 * 256
+    eng = engine.Engine(shape, gw, max_seq=max_seq, gamma_max=max(gamma, 1))
+    eng.prefill(synth.random_prompt(n_prompt, shape.vocab, 0), calibrate=True)
+    eng.encode_weights(eng.calib_norms())
+    eng.build_kv_codebook()
+    first = eng.next_tokens()
+
+    def timed(g):
+        eng.generate(0, g, use_graph=True)            # lays the token buffers out for this gamma and captures the step
+        B.cass_set_len(eng.session, n_prompt)
+        eng.set_next_tokens(first)
+        out, marks = [], []
+        stats = engine.StepStats()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        while len(out) < n_tokens:
+            eng._graphs[g].replay()
+            eng._collect([out], stats)
+            marks.append((time.perf_counter() - t0, len(out)))
+        return out, stats, marks
+
+    def tail_rate(m):
+        k = max(1, len(m) // 10)
+        return (m[-1][1] - m[-k - 1][1]) / (m[-1][0] - m[-k - 1][0])
+
+    plain, _, pm = timed(0)
+    spec, st, sm = timed(gamma)
+    n = min(len(plain), len(spec), n_tokens)
+    k = max(1, len(sm) // 10)
+    status, ln = eng.status()
+    eng.close()
+    return [{"kernel": "long_decode", "config": config, "gamma": gamma, "prompt": n_prompt, "tokens": n,
+             "streams_identical": spec[:n] == plain[:n], "final_len": ln, "status": status,
+             "spec_tokens_per_s": sm[-1][1] / sm[-1][0], "spec_tokens_per_s_first_10pct": sm[k - 1][1] / sm[k - 1][0],
+             "spec_tokens_per_s_last_10pct": tail_rate(sm), "steps": st.steps, "mean_accepted": st.mean_accepted,
+             "plain_tokens_per_s": pm[-1][1] / pm[-1][0], "plain_tokens_per_s_last_10pct": tail_rate(pm)}]
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--kernel", default="gemv")
@@ -212,6 +264,9 @@ def main():
     ap.add_argument("--chunk", type=int, default=0, help="columns per decode chunk of the weight format (0 = default 256)")
     ap.add_argument("--seg", type=int, default=0, help="columns per superblock of the weight format (0 = default 2048)")
     ap.add_argument("--batch", type=int, default=1, help="sequences decoded together (step breakdown)")
+    ap.add_argument("--tokens", type=int, default=8192, help="tokens to decode (--kernel decode)")
+    ap.add_argument("--prompt", type=int, default=512)
+    ap.add_argument("--config", default="llama8b")
     ap.add_argument("--p", type=int, default=400)
     ap.add_argument("--t", type=int, default=4)
     args = ap.parse_args()
@@ -227,6 +282,8 @@ def main():
             n, k = SHAPES[name]
             copies = args.copies or max(2, int(300e6 / (n * k * 2)) + 1)
             out.append(bench_verify_gemm(name, copies, args.iters))
+    if args.kernel == "decode":
+        out.extend(long_decode(args.gamma, args.tokens, args.prompt, args.config))
     if args.kernel == "step":
         out.extend(step_breakdown(gamma=args.gamma, batch=args.batch))
     if args.kernel in ("attn", "all"):

@@ -312,3 +312,27 @@ def test_five_query_heads_per_kv_head(cass):
     assert f0 == f1 and spec[:24] == plain[:24]
     assert e1.status()[0] == 0 and stats.emitted == stats.accepted + stats.steps
     e0.close(); e1.close()
+
+
+def test_full_llama_8b_shape_stream_identity(cass):
+    """The whole Llama-3-8B-shaped model (32 layers, vocab 128256) in the launch configuration the benchmark times
+    (CUDA-graph steps, gamma = 4): the speculative stream equals the plain bf16 greedy stream of the same kernels."""
+    shape = synth.LLAMA3_8B
+    wt = synth.model_weights(shape, 0, device="cuda")
+    gw = {"layers": [cass.engine.fuse_layer_weights(lw) for lw in wt["layers"]], "embed": wt["embed"],
+          "lm_head": wt["lm_head"], "norm_final": wt["norm_final"]}
+    del wt
+    eng = cass.engine.Engine(shape, gw, max_seq=768, gamma_max=4)
+    eng.prefill(synth.random_prompt(256, shape.vocab, 0), calibrate=True)
+    eng.encode_weights(eng.calib_norms())
+    eng.build_kv_codebook()
+    first = eng.next_tokens()
+    plain, _ = eng.generate(120, 0, use_graph=True)
+    eng.generate(0, 4, use_graph=True)            # token buffers into the gamma = 4 layout, step captured
+    cass.cass_set_len(eng.session, 256)
+    eng.set_next_tokens(first)
+    spec, stats = eng.generate(120, 4, use_graph=True)
+    assert eng.status()[0] == 0
+    assert spec[:120] == plain[:120]
+    assert stats.emitted == stats.accepted + stats.steps
+    eng.close()
