@@ -169,8 +169,8 @@ def run_reference(args):
 # ----------------------------------------------------------------------------------------------------------
 
 def launches_per_step(n_layers: int, gamma: int) -> int:
-    draft = 2 + n_layers * 11 + 3            # embed, norm | per layer: 4 gemv, rope, kv, attn, merge, 2 norm, swiglu | lm gemv, 2 argmax
-    verify = 2 + n_layers * 11 + 3           # per layer: 4 gemm, rope, kv, attn, merge, 2 norm, swiglu | lm gemm, 2 argmax
+    draft = 2 + n_layers * 10 + 3            # embed, norm | per layer: 4 gemv, rope+kv, attn, merge, 2 norm, swiglu | lm gemv, 2 argmax
+    verify = 2 + n_layers * 10 + 3           # per layer: 4 gemm, rope+kv, attn, merge, 2 norm, swiglu | lm gemm, 2 argmax
     return gamma * draft + verify + 1
 
 

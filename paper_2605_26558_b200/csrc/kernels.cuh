@@ -104,6 +104,14 @@ int launch_sqrt(const float* in, float* out, size_t n, cudaStream_t s);
 int launch_kv_append(const KvGeom& g, const KvComp& ck, const KvComp& cv, uint16_t* k_cache, uint16_t* v_cache,
                      const uint16_t* src_k, const uint16_t* src_v, int row_stride, int start_pos, int use_inflight,
                      int n_new, int flags, DevState* st, int seq0, int n_seq, cudaStream_t s);
+// The same fused with what precedes it in a layer: adds the qkv projection's split-K parts, rounds to bf16, applies
+// RoPE to q and k at each row's position, writes the bf16 qkv rows (rps per sequence) and appends the K/V of those
+// rows at the positions the state gives.  Needs head_dim % 64 == 0 (rope_kv_fusable); otherwise the caller runs
+// launch_qkv_rope + launch_kv_append.
+bool rope_kv_fusable(const KvGeom& g);
+int launch_rope_kv_append(const KvGeom& g, const KvComp& ck, const KvComp& cv, uint16_t* k_cache, uint16_t* v_cache,
+                          Partials pp, const float* cos_t, const float* sin_t, uint16_t* qkv, int n_q, int use_inflight,
+                          int rps, int flags, DevState* st, int n_seq, cudaStream_t s);
 int launch_kv_codebook(const KvGeom& g, const KvComp& ck, const KvComp& cv, const uint16_t* k_cache,
                        const uint16_t* v_cache, int n_tokens, cudaStream_t s);
 

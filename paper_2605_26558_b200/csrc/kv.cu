@@ -73,11 +73,25 @@ __global__ void k_kv_rank(KvComp ck, KvComp cv) {
 
 // grid (n_kv, 2): block of 8 warps walks the n_new tokens in batches of 8; offsets into the unary arena are
 // assigned sequentially by one thread per batch, so records stay densely packed in token order.
+// What the fused form of the encoder needs on top: the projection's fp32 split-K parts (the q, k, v features of every
+// row), the rotary tables and the bf16 qkv rows to write.
+struct RopeSrc {
+    Partials pp;
+    const float *cos_t, *sin_t;
+    uint16_t* qkv;          // [rows][(n_q + 2 n_kv) d]
+    int n_q;
+};
+
 // grid.z = sequence of the call; its rows start at row blockIdx.z * n_new of the source.
+// FUSED: the source is the qkv projection's split-K parts: this kernel adds them, rounds to bf16, rotates q and k
+// (RoPE, Sec. 2.1) and writes the qkv rows; the K and V records are then formed from the rotated values as in the
+// plain form.  Blocks with blockIdx.x >= n_kv rotate the query heads; head_dim must be a multiple of 64 so that a
+// rotation pair (c, c + d/2) sits in one lane.
+template <bool FUSED>
 __global__ void __launch_bounds__(256) k_kv_append(KvGeom g, KvComp ck, KvComp cv, uint16_t* __restrict__ k_cache,
                                                    uint16_t* __restrict__ v_cache, const uint16_t* __restrict__ src_k,
                                                    const uint16_t* __restrict__ src_v, int row_stride, int start_pos_arg,
-                                                   int use_inflight, int n_new, int flags, DevState* st, int seq0) {
+                                                   int use_inflight, int n_new, int flags, DevState* st, int seq0, RopeSrc rs) {
     __shared__ uint32_t s_fix[kKvWarps][kKvFixMax];          // bitmap (<= 8) + field words (<= 64)
     __shared__ uint32_t s_una[kKvWarps][kKvStageWords];
     __shared__ uint32_t s_nw[kKvWarps], s_off[kKvWarps];
@@ -85,6 +99,32 @@ __global__ void __launch_bounds__(256) k_kv_append(KvGeom g, KvComp ck, KvComp c
     pdl_wait();
     const int head = blockIdx.x, kind = blockIdx.y, seq = seq0 + blockIdx.z;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (FUSED && head >= g.n_kv) {
+        // ---- query heads: q[r][h][j], q[r][h][j + d/2] rotated by the row's position ----
+        if (kind != 0) return;
+        const int start = st->len[seq] + (use_inflight ? st->inflight[seq] : 0);
+        const int half = g.d / 2, qkv_dim = (rs.n_q + 2 * g.n_kv) * g.d;
+        const int per_row = rs.n_q * half, n_items = n_new * per_row;
+        const Partials& pp = rs.pp;
+        for (int it = (head - g.n_kv) * blockDim.x + threadIdx.x; it < n_items; it += (gridDim.x - g.n_kv) * blockDim.x) {
+            const int i = it / per_row, e = it % per_row, hq = e / half, j = e % half;
+            const size_t r = (size_t)blockIdx.z * n_new + i;
+            const int ia = hq * g.d + j, ib = ia + half;
+            float a = 0.f, b = 0.f;
+            for (int sgm = 0; sgm < pp.n_seg; ++sgm) {
+                const float* q = pp.p + (size_t)sgm * pp.seg_stride + r * pp.row_stride;
+                a += q[ia];
+                b += q[ib];
+            }
+            a = round_bf16(a);
+            b = round_bf16(b);
+            const size_t ti = (size_t)(start + i) * half + j;
+            const float c = rs.cos_t[ti], sn = rs.sin_t[ti];
+            rs.qkv[r * qkv_dim + ia] = float_to_bf16_bits(a * c - b * sn);
+            rs.qkv[r * qkv_dim + ib] = float_to_bf16_bits(b * c + a * sn);
+        }
+        return;
+    }
     const KvComp& c0 = kind ? cv : ck;                       // sequence 0's; shifted to this sequence below
     const uint8_t* exp_to_rank = of_seq(c0.exp_to_rank, seq, g.seq_stride);
     const uint16_t* src = (kind ? src_v : src_k) + (size_t)blockIdx.z * n_new * row_stride;
@@ -103,9 +143,43 @@ __global__ void __launch_bounds__(256) k_kv_append(KvGeom g, KvComp ck, KvComp c
         bool keep[kKvMaxPerLane];
         uint32_t n_words = 0;
         if (active) {
-            const uint16_t* row = src + (size_t)i * row_stride + (size_t)head * g.d;
+            if (FUSED) {
+                const int qkv_dim = (rs.n_q + 2 * g.n_kv) * g.d, half = g.d / 2, hj = nj / 2;
+                const size_t r = (size_t)blockIdx.z * n_new + i;
+                const int base = (rs.n_q + (kind ? g.n_kv : 0) + head) * g.d;
+                const Partials& pp = rs.pp;
+                float val[kKvMaxPerLane];
 #pragma unroll
-            for (int j = 0; j < kKvMaxPerLane; ++j) bits[j] = j < nj ? row[lane + 32 * j] : 0;
+                for (int j = 0; j < kKvMaxPerLane; ++j) {
+                    val[j] = 0.f;
+                    if (j < nj) {
+                        for (int sgm = 0; sgm < pp.n_seg; ++sgm)
+                            val[j] += pp.p[(size_t)sgm * pp.seg_stride + r * pp.row_stride + base + lane + 32 * j];
+                        val[j] = round_bf16(val[j]);
+                    }
+                }
+                if (kind == 0) {                         // K: rotate the pairs (c, c + d/2), both held by this lane
+#pragma unroll
+                    for (int j = 0; j < kKvMaxPerLane / 2; ++j) {
+                        if (j < hj) {
+                            const size_t ti = (size_t)pos * half + lane + 32 * j;
+                            const float c = rs.cos_t[ti], sn = rs.sin_t[ti];
+                            const float a = val[j], b = val[j + hj];
+                            val[j] = bf16_bits_to_float(float_to_bf16_bits(a * c - b * sn));
+                            val[j + hj] = bf16_bits_to_float(float_to_bf16_bits(b * c + a * sn));
+                        }
+                    }
+                }
+#pragma unroll
+                for (int j = 0; j < kKvMaxPerLane; ++j) {
+                    bits[j] = j < nj ? float_to_bf16_bits(val[j]) : 0;
+                    if (j < nj) rs.qkv[r * qkv_dim + base + lane + 32 * j] = (uint16_t)bits[j];
+                }
+            } else {
+                const uint16_t* row = src + (size_t)i * row_stride + (size_t)head * g.d;
+#pragma unroll
+                for (int j = 0; j < kKvMaxPerLane; ++j) bits[j] = j < nj ? row[lane + 32 * j] : 0;
+            }
             if (flags & CASS_KV_BF16) {
                 uint16_t* dst = cache + ((size_t)pos * g.n_kv + head) * g.d;
 #pragma unroll
@@ -184,8 +258,22 @@ int launch_kv_append(const KvGeom& g, const KvComp& ck, const KvComp& cv, uint16
                      int n_new, int flags, DevState* st, int seq0, int n_seq, cudaStream_t s) {
     if (n_new <= 0 || n_seq <= 0) return CASS_OK;
     dim3 grid(g.n_kv, 2, n_seq);
-    CASS_PDL_LAUNCH(k_kv_append, grid, dim3(256), 0, s, g, ck, cv, k_cache, v_cache, src_k, src_v, row_stride, start_pos,
-                    use_inflight, n_new, flags, st, seq0);
+    CASS_PDL_LAUNCH(k_kv_append<false>, grid, dim3(256), 0, s, g, ck, cv, k_cache, v_cache, src_k, src_v, row_stride, start_pos,
+                    use_inflight, n_new, flags, st, seq0, RopeSrc{});
+    return CASS_OK;
+}
+
+bool rope_kv_fusable(const KvGeom& g) { return g.d % 64 == 0; }
+
+int launch_rope_kv_append(const KvGeom& g, const KvComp& ck, const KvComp& cv, uint16_t* k_cache, uint16_t* v_cache,
+                          Partials pp, const float* cos_t, const float* sin_t, uint16_t* qkv, int n_q, int use_inflight,
+                          int rps, int flags, DevState* st, int n_seq, cudaStream_t s) {
+    if (rps <= 0 || n_seq <= 0) return CASS_OK;
+    if (!rope_kv_fusable(g) || !pp.p) return CASS_ERR_UNSUPPORTED;
+    const int q_blocks = ceil_div(n_q * (g.d / 2), 256);
+    dim3 grid(g.n_kv + q_blocks, 2, n_seq);
+    CASS_PDL_LAUNCH(k_kv_append<true>, grid, dim3(256), 0, s, g, ck, cv, k_cache, v_cache, (const uint16_t*)nullptr,
+                    (const uint16_t*)nullptr, 0, -1, use_inflight, rps, flags, st, 0, RopeSrc{pp, cos_t, sin_t, qkv, n_q});
     return CASS_OK;
 }
 

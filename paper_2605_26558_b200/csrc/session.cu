@@ -427,6 +427,7 @@ extern "C" int cass_verify(void* session, const int32_t* toks, int g, int32_t* t
     cudaStream_t st = (cudaStream_t)stream_;
     const cass_model_desc& d = s->d;
     auto vparts = [&](int n, int k) { return verify_gemm_partials(s->vg_partial, n, k, bn); };
+    const bool fused = rope_kv_fusable(s->kg);       // RoPE and the KV append in one kernel
     const int qd = d.n_q_heads * d.head_dim;
     RC(launch_embed(toks, 1, (const uint16_t*)s->embed, s->h, rows, d.hidden, st));
     RC(launch_rmsnorm(s->h, (const uint16_t*)s->layers[0].w.norm_attn, s->xn, rows, d.hidden, d.rms_eps, st));
@@ -438,10 +439,15 @@ extern "C" int cass_verify(void* session, const int32_t* toks, int g, int32_t* t
         LayerDev& L = s->layers[l];
         if (calib) RC(launch_calib_accum(s->xn, rows, d.hidden, L.calib[0], s->st, st));
         RC(launch_verify_gemm((const uint16_t*)L.w.wqkv, s->xn, rows, bn, s->qkv_dim, d.hidden, s->vg_partial, nullptr, nullptr, status, st));
-        RC(launch_qkv_rope(s->qkv, vparts(s->qkv_dim, d.hidden), s->cos_t, s->sin_t, s->st, 0, rows, rps,
-                           d.n_q_heads, d.n_kv_heads, d.head_dim, st));
-        RC(launch_kv_append(s->kg, L.ck, L.cv, L.kc, L.vc, s->qkv + qd, s->qkv + qd + d.n_kv_heads * d.head_dim, s->qkv_dim,
-                            -1, 0, rps, kv_flags, s->st, 0, B, st));
+        if (fused) {
+            RC(launch_rope_kv_append(s->kg, L.ck, L.cv, L.kc, L.vc, vparts(s->qkv_dim, d.hidden), s->cos_t, s->sin_t, s->qkv,
+                                     d.n_q_heads, 0, rps, kv_flags, s->st, B, st));
+        } else {
+            RC(launch_qkv_rope(s->qkv, vparts(s->qkv_dim, d.hidden), s->cos_t, s->sin_t, s->st, 0, rows, rps,
+                               d.n_q_heads, d.n_kv_heads, d.head_dim, st));
+            RC(launch_kv_append(s->kg, L.ck, L.cv, L.kc, L.vc, s->qkv + qd, s->qkv + qd + d.n_kv_heads * d.head_dim, s->qkv_dim,
+                                -1, 0, rps, kv_flags, s->st, 0, B, st));
+        }
         RC(launch_verify_attn(s->kg, L.kc, L.vc, s->qkv, B, rps, d.n_q_heads, s->st, s->asc, s->attn, st));
         if (calib) RC(launch_calib_accum(s->attn, rows, qd, L.calib[1], s->st, st));
         RC(launch_verify_gemm((const uint16_t*)L.w.wo, s->attn, rows, bn, d.hidden, qd, s->vg_partial, nullptr, nullptr, status, st));
@@ -474,14 +480,20 @@ extern "C" int cass_draft_step(void* session, const int32_t* tok_in, int32_t* to
     int32_t* status = &s->st->status;
     const int B = s->B;
     auto draftp = [&](const cass_blob_info& b) { return draft_gemv_partials(s->partial, b); };
+    const bool fused = rope_kv_fusable(s->kg);
     RC(launch_embed(tok_in, tok_stride, (const uint16_t*)s->embed, s->h, B, d.hidden, st));
     RC(launch_rmsnorm(s->h, (const uint16_t*)s->layers[0].w.norm_attn, s->xn, B, d.hidden, d.rms_eps, st));
     for (int l = 0; l < d.n_layers; ++l) {
         LayerDev& L = s->layers[l];
         RC(launch_draft_gemv(L.blob[0], L.bi[0], s->xn, B, s->partial, status, st));
-        RC(launch_qkv_rope(s->qkv, draftp(L.bi[0]), s->cos_t, s->sin_t, s->st, 1, B, 1, d.n_q_heads, d.n_kv_heads, d.head_dim, st));
-        RC(launch_kv_append(s->kg, L.ck, L.cv, L.kc, L.vc, s->qkv + qd, s->qkv + qd + d.n_kv_heads * d.head_dim, s->qkv_dim,
-                            -1, 1, 1, CASS_KV_COMPRESSED, s->st, 0, B, st));
+        if (fused) {
+            RC(launch_rope_kv_append(s->kg, L.ck, L.cv, L.kc, L.vc, draftp(L.bi[0]), s->cos_t, s->sin_t, s->qkv, d.n_q_heads, 1, 1,
+                                     CASS_KV_COMPRESSED, s->st, B, st));
+        } else {
+            RC(launch_qkv_rope(s->qkv, draftp(L.bi[0]), s->cos_t, s->sin_t, s->st, 1, B, 1, d.n_q_heads, d.n_kv_heads, d.head_dim, st));
+            RC(launch_kv_append(s->kg, L.ck, L.cv, L.kc, L.vc, s->qkv + qd, s->qkv + qd + d.n_kv_heads * d.head_dim, s->qkv_dim,
+                                -1, 1, 1, CASS_KV_COMPRESSED, s->st, 0, B, st));
+        }
         RC(launch_draft_attn(s->kg, L.ck, L.cv, s->qkv, s->qkv_dim, d.n_q_heads, B, s->st, s->asc, s->attn, st));
         RC(launch_draft_gemv(L.blob[1], L.bi[1], s->attn, B, s->partial, status, st));
         RC(launch_residual_rmsnorm(s->h, nullptr, draftp(L.bi[1]), (const uint16_t*)L.w.norm_ffn, s->xn, B, d.hidden, d.rms_eps, st));

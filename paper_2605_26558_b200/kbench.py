@@ -158,6 +158,13 @@ def bench_draft_attn(n_pos, layers, iters):
     ms = _time(lambda: [B.cass_kv_append(eng.session, l, kvs[l][0][n_pos:], kvs[l][1][n_pos:], n_pos, 1,
                                          B.KV_BF16 | B.KV_COMPRESSED) for l in range(layers)], iters)
     res.append({"kernel": "kv_append (1 token, bf16 + compressed)", "positions": n_pos, "us_per_layer": ms * 1e3 / layers})
+    # verification pass of 5 rows over the same caches: per layer RoPE + KV append, k_verify_attn over n_pos positions,
+    # merge, and the (small, hidden 256) projections of this cut-down layer
+    toks = torch.zeros(8, dtype=torch.int32, device=dev)
+    targ = torch.zeros(8, dtype=torch.int32, device=dev)
+    ms = _time(lambda: B.cass_verify(eng.session, toks, 4, targ), iters)
+    res.append({"kernel": "verify pass, 5 rows (verify_attn + small ops of a hidden-256 layer)", "positions": n_pos,
+                "us_per_layer": ms * 1e3 / layers, "bf16_kv_bytes_per_layer": n_pos * 8 * 128 * 2 * 2})
     assert eng.status()[0] == 0
     eng.close()
     return res

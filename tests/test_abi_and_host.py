@@ -88,4 +88,4 @@ def test_replica_reduction_world_size_2():
 def test_launch_count_formula():
     sys.path.insert(0, ROOT)
     import bench
-    assert bench.launches_per_step(32, 4) == 4 * (2 + 32 * 11 + 3) + (2 + 32 * 11 + 3) + 1
+    assert bench.launches_per_step(32, 4) == 4 * (2 + 32 * 10 + 3) + (2 + 32 * 10 + 3) + 1
