@@ -308,10 +308,13 @@ __global__ void __launch_bounds__(kDaThreads) k_draft_attn(KvGeom g, KvComp ck0,
 // Row r (the (r % rps)-th of sequence r / rps) sees positions < len + (draft: inflight + 1 | verify: r % rps + 1);
 // chunks hold `chunk_tokens` positions.
 // The reductions run in a fixed order that depends on the number of visible chunks only.
-__global__ void __launch_bounds__(128) k_attn_merge(AttnScratch sc, int n_chunks_alloc, int chunk_tokens, int rps, int n_q, int d,
-                                                    const DevState* __restrict__ st, int draft_mode, uint16_t* __restrict__ out) {
-    extern __shared__ float w_s[];                  // [n_chunks_alloc] weights e^{m_c - M}
-    __shared__ float s_red[4];
+constexpr int kMergeThreads = 256;
+constexpr int kMergeWarps = kMergeThreads / 32;
+
+__global__ void __launch_bounds__(kMergeThreads) k_attn_merge(AttnScratch sc, int n_chunks_alloc, int chunk_tokens, int rps, int n_q, int d,
+                                                              const DevState* __restrict__ st, int draft_mode, uint16_t* __restrict__ out) {
+    extern __shared__ __align__(16) float w_s[];    // [n_chunks_alloc] weights e^{m_c - M}, then [kMergeWarps][d] partial outputs
+    __shared__ float s_red[kMergeWarps];
     pdl_launch_dependents();
     pdl_wait();
     const int hq = blockIdx.x, r = blockIdx.y;
@@ -322,15 +325,18 @@ __global__ void __launch_bounds__(128) k_attn_merge(AttnScratch sc, int n_chunks
     const size_t pair = (size_t)r * n_q + hq;
     const float* mp = sc.m + pair * n_chunks_alloc;
     const float* lp = sc.l + pair * n_chunks_alloc;
+    float* part_s = w_s + ((n_chunks_alloc + 3) & ~3);
     float M = -INFINITY;
-    for (int c = tid; c < n_ch; c += 128) M = fmaxf(M, mp[c]);
+    for (int c = tid; c < n_ch; c += kMergeThreads) M = fmaxf(M, mp[c]);
     M = warp_max(M);
     if (lane == 0) s_red[warp] = M;
     __syncthreads();
-    M = fmaxf(fmaxf(s_red[0], s_red[1]), fmaxf(s_red[2], s_red[3]));
+    M = s_red[0];
+#pragma unroll
+    for (int w = 1; w < kMergeWarps; ++w) M = fmaxf(M, s_red[w]);
     __syncthreads();
     float L = 0.f;
-    for (int c = tid; c < n_ch; c += 128) {
+    for (int c = tid; c < n_ch; c += kMergeThreads) {
         const float w = expf(mp[c] - M);
         w_s[c] = w;
         L += w * lp[c];
@@ -338,26 +344,43 @@ __global__ void __launch_bounds__(128) k_attn_merge(AttnScratch sc, int n_chunks
     L = warp_sum(L);
     if (lane == 0) s_red[warp] = L;
     __syncthreads();
-    L = (s_red[0] + s_red[1]) + (s_red[2] + s_red[3]);
+    L = s_red[0];
+#pragma unroll
+    for (int w = 1; w < kMergeWarps; ++w) L += s_red[w];
+    // warp w adds the chunks w, w + 8, ... (four dims per lane, 16-byte loads); the warps' sums are then added in warp
+    // order: the order of every addition depends on the number of visible chunks only
     const float* op = sc.o + pair * n_chunks_alloc * d;
-    for (int dim = tid; dim < d; dim += 128) {
-        float acc = 0.f;
-        for (int c = 0; c < n_ch; ++c) acc = fmaf(w_s[c], op[(size_t)c * d + dim], acc);
+    for (int dim = lane * 4; dim < d; dim += 128) {
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 4
+        for (int c = warp; c < n_ch; c += kMergeWarps) {
+            const float w = w_s[c];
+            const float4 o = *reinterpret_cast<const float4*>(op + (size_t)c * d + dim);
+            acc.x = fmaf(w, o.x, acc.x); acc.y = fmaf(w, o.y, acc.y); acc.z = fmaf(w, o.z, acc.z); acc.w = fmaf(w, o.w, acc.w);
+        }
+        *reinterpret_cast<float4*>(part_s + warp * d + dim) = acc;
+    }
+    __syncthreads();
+    for (int dim = tid; dim < d; dim += kMergeThreads) {
+        float acc = part_s[dim];
+#pragma unroll
+        for (int w = 1; w < kMergeWarps; ++w) acc += part_s[w * d + dim];
         out[((size_t)r * n_q + hq) * d + dim] = float_to_bf16_bits(acc / L);
     }
 }
 
 int launch_attn_merge(const AttnScratch& sc, int n_chunks_alloc, int chunk_tokens, int rows, int rps, int n_q, int d,
                       const DevState* st, int draft_mode, uint16_t* out, cudaStream_t s) {
+    if (d % 4) return CASS_ERR_UNSUPPORTED;
     dim3 grid(n_q, rows);
-    const size_t smem = (size_t)n_chunks_alloc * 4;
+    const size_t smem = ((size_t)((n_chunks_alloc + 3) & ~3) + (size_t)kMergeWarps * d) * 4;
     if (smem > 200 * 1024) return CASS_ERR_CAPACITY;
     static size_t attr = 48 * 1024;
     if (smem > attr) {
         CASS_CUDA_CHECK(cudaFuncSetAttribute(k_attn_merge, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         attr = smem;
     }
-    CASS_PDL_LAUNCH(k_attn_merge, grid, dim3(128), smem, s, sc, n_chunks_alloc, chunk_tokens, rps, n_q, d, st, draft_mode, out);
+    CASS_PDL_LAUNCH(k_attn_merge, grid, dim3(kMergeThreads), smem, s, sc, n_chunks_alloc, chunk_tokens, rps, n_q, d, st, draft_mode, out);
     return CASS_OK;
 }
 
