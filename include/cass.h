@@ -42,7 +42,9 @@ enum { CASS_KV_BF16 = 1, CASS_KV_COMPRESSED = 2 };
  * speculation data (Eq. 2's w_t / kv_t; 7 - t mantissa bits remain).  Paper default: 400 / 4 (Sec. 6.1, 7.2).
  * w_seg_cols / w_chunk_cols: columns per superblock and per decode chunk (0 = 2048 / 256). */
 typedef struct cass_format {
-    int mode;                /* 1 = Cassandra-1 (unary exponent code) */
+    int mode;                /* weights: 1 = Cassandra-1 (unary exponent code, lossless for the kept bits),
+                              * 2 = Cassandra-2 (Sec. 4.2: MX, blocks of 32 kept values share an exponent, MXINT
+                              * elements; see cass_encode_weights).  The KV cache is Cassandra-1 in both modes. */
     int w_prune_permille, w_trunc_bits;
     int kv_prune_permille, kv_trunc_bits;
     int w_seg_cols, w_chunk_cols;
@@ -98,6 +100,7 @@ int cass_encode_weights(const cass_format* fmt, const void* W_bf16, const float*
 typedef struct cass_blob_info {
     int rows, cols, prune_permille, trunc_bits, seg_cols, chunk_cols, n_seg, n_rowblocks, kept_per_row;
     int max_superblock_bytes;
+    int mode, reserved;      /* 1 = Cassandra-1 (unary exponent code), 2 = Cassandra-2 (shared MX exponents) */
     uint64_t total_bytes;
 } cass_blob_info;
 

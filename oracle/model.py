@@ -76,8 +76,14 @@ class Weights:
         self.norm_final = np.asarray(w_bits["norm_final"], dtype=np.uint16)
 
 
-def draft_weight_bits(w_bits: dict, act_norms: dict, p: int, t: int) -> dict:
-    """Speculation-data view of every projection and of lm_head (embeddings and norm gains stay bf16)."""
+def draft_weight_bits(w_bits: dict, act_norms: dict, p: int, t: int, mode: int = 1) -> dict:
+    """Speculation-data view of every projection and of lm_head (embeddings and norm gains stay bf16).
+    mode 1: Cassandra-1 (exponents kept exactly); mode 2: Cassandra-2 (MX shared exponents, `mx.py`)."""
+    if mode == 2:
+        from . import mx
+        view = lambda v, keep: mx.draft_bits(v, keep, t)
+    else:
+        view = lambda v, keep: codec.draft_bits(v, keep, t)
     out = {"layers": []}
     for li, lw in enumerate(w_bits["layers"]):
         d = {}
@@ -85,12 +91,12 @@ def draft_weight_bits(w_bits: dict, act_norms: dict, p: int, t: int) -> dict:
             if k.startswith("w"):
                 v = np.asarray(v, dtype=np.uint16)
                 keep = codec.keep_mask_weights(v, act_norms["layers"][li][k], p)
-                d[k] = codec.draft_bits(v, keep, t)
+                d[k] = view(v, keep)
             else:
                 d[k] = v
         out["layers"].append(d)
     lm = np.asarray(w_bits["lm_head"], dtype=np.uint16)
-    out["lm_head"] = codec.draft_bits(lm, codec.keep_mask_weights(lm, act_norms["lm_head"], p), t)
+    out["lm_head"] = view(lm, codec.keep_mask_weights(lm, act_norms["lm_head"], p))
     out["embed"] = w_bits["embed"]
     out["norm_final"] = w_bits["norm_final"]
     return out

@@ -32,8 +32,8 @@ class Format(C.Structure):
                 ("w_chunk_cols", C.c_int)]
 
 
-def default_format(w_p=400, w_t=4, kv_p=400, kv_t=4, seg_cols=0, chunk_cols=0) -> Format:
-    return Format(1, w_p, w_t, kv_p, kv_t, seg_cols, chunk_cols)
+def default_format(w_p=400, w_t=4, kv_p=400, kv_t=4, seg_cols=0, chunk_cols=0, mode=1) -> Format:
+    return Format(mode, w_p, w_t, kv_p, kv_t, seg_cols, chunk_cols)
 
 
 class ModelDesc(C.Structure):
@@ -62,7 +62,8 @@ class ModelBlobs(C.Structure):
 class BlobInfo(C.Structure):
     _fields_ = [("rows", C.c_int), ("cols", C.c_int), ("prune_permille", C.c_int), ("trunc_bits", C.c_int),
                 ("seg_cols", C.c_int), ("chunk_cols", C.c_int), ("n_seg", C.c_int), ("n_rowblocks", C.c_int),
-                ("kept_per_row", C.c_int), ("max_superblock_bytes", C.c_int), ("total_bytes", C.c_uint64)]
+                ("kept_per_row", C.c_int), ("max_superblock_bytes", C.c_int), ("mode", C.c_int), ("reserved", C.c_int),
+                ("total_bytes", C.c_uint64)]
 
 
 class BlobStats(C.Structure):

@@ -213,7 +213,100 @@ __device__ __forceinline__ void chunk_dot_fast(const uint32_t* __restrict__ sb, 
     for (; grp < n_groups; ++grp) group(grp, std::true_type{});
 }
 
+// ---- Cassandra-2 (MX) chunk: 4-bit fields (sign + 3 magnitude bits, t = 4), one exponent byte per 32 values ------
+// Same bitmap walk as above; the unary parse is replaced by a 16-entry table look-up of the signed magnitude, and a
+// block's 32 products are summed first and scaled by the block's power of two once (Sec. 5.1, MX decoder: the shared
+// exponent is broadcast to the elements of its block).
+template <int NB>
+__device__ __noinline__ WalkState<NB> group_slow_mx(const uint32_t* bmS, uint32_t fword, int count, WalkState<NB> st,
+                                                    uint32_t bpos_lim, const float* xs, const float* nlut) {
+    for (int e = 0; e < count; ++e) {
+        bool found = false;
+        while (st.bpos < bpos_lim) {
+            uint32_t w = bmS[(st.bpos >> 5) * 32] << (st.bpos & 31);
+            if (w) { st.bpos += __clz(w); found = true; break; }
+            st.bpos = (st.bpos | 31u) + 1u;
+        }
+        if (!found) break;
+        const XRaw<NB> xv = x_load<NB>(smem_u32(xs) + st.bpos * (uint32_t)x_col_bytes(NB));
+        st.bpos += 1;
+        x_fma<NB>(xv, __float_as_uint(nlut[(fword >> (28 - 4 * e)) & 15u]), st.acc);
+    }
+    return st;
+}
+
+template <int NB>
+__device__ __forceinline__ void chunk_dot_mx4(const uint32_t* __restrict__ sb, const SbGeom& g, int ch, int lane,
+                                              int chunk_elems, const float* __restrict__ xs,
+                                              const float* __restrict__ nlut, float (&acc)[NB]) {
+    constexpr uint32_t XS = (uint32_t)x_col_bytes(NB);
+    const uint32_t e0 = sb[g.tab + ch * 32 + lane];
+    const uint32_t* bmS = sb + g.bm + lane;
+    const uint32_t bm_a = smem_u32(bmS), xs_a = smem_u32(xs), nl_a = smem_u32(nlut);      // nlut is 64-byte aligned
+    uint32_t fl_a = smem_u32(sb + g.fl + lane) + (uint32_t)(ch * chunk_elems / 8) * 128u;
+    const uint32_t ex_a = smem_u32(sb + g.un + lane);
+    const int kept = (int)(sb[g.tab + g.n_ch * 32 + lane] >> 20);
+    const int m = max(0, min(chunk_elems, kept - ch * chunk_elems));
+    const int n_full = __reduce_min_sync(0xffffffffu, m) / kGroupCols;
+    const int n_groups = ceil_div(__reduce_max_sync(0xffffffffu, m), kGroupCols);
+    uint32_t bpos = e0 >> 20;
+    const uint32_t blk0 = (e0 & 0xFFFFFu) >> 3;                 // index of the chunk's first exponent byte
+    const uint32_t bpos_lim = (uint32_t)(g.bm_words * 32);
+    float blk[NB];
+#pragma unroll
+    for (int b = 0; b < NB; ++b) blk[b] = 0.f;
+
+    auto group = [&](int grp, auto tail_c) {
+        constexpr bool tail = decltype(tail_c)::value;
+        WalkState<NB> st0;
+#pragma unroll
+        for (int b = 0; b < NB; ++b) st0.acc[b] = blk[b];
+        st0.bpos = bpos; st0.upos = 0;
+        const uint32_t ba = bm_a + (bpos >> 5) * 128u;
+        uint32_t bv = __funnelshift_l(lds_u32_off<128>(ba), lds_u32(ba), bpos);
+        const uint32_t xg = xs_a + bpos * XS + 31u * XS;
+        const uint32_t fword = lds_u32(fl_a);
+        const int rem = m - grp * kGroupCols;
+        uint32_t dry = 0, p = 0;
+#pragma unroll
+        for (int e = 0; e < kGroupCols; ++e) {
+            p = bfind_u32(bv);
+            const XRaw<NB> xv = x_load<NB>(mad_lo(p, 0u - XS, xg));
+            bv &= ~shl_sat(1u, p);
+            const uint32_t off = e < 7 ? (fword >> (26 - 4 * e)) : (fword << 2);
+            const uint32_t wb = lds_u32((off & 0x3Cu) | nl_a);                         // +-(magnitude << 4) as a float
+            if (!tail) {
+                x_fma<NB>(xv, wb, blk);
+            } else if (e < rem) {
+                x_fma<NB>(xv, wb, blk);
+                dry |= p;
+            }
+        }
+        bpos += 32u - p;
+        if (tail) bpos = min(bpos, bpos_lim);
+        else dry |= p;
+        if ((int32_t)dry < 0) {
+            const WalkState<NB> r = group_slow_mx<NB>(bmS, fword, min(rem, kGroupCols), st0, bpos_lim, xs, nlut);
+#pragma unroll
+            for (int b = 0; b < NB; ++b) blk[b] = r.acc[b];
+            bpos = r.bpos;
+        }
+        fl_a += 128u;
+        if ((grp & 3) == 3 || grp == n_groups - 1) {              // a block of 32 values is complete: apply its scale
+            const uint32_t bi = blk0 + (uint32_t)(grp >> 2);
+            const uint32_t eb = (lds_u32(ex_a + (bi >> 2) * 128u) >> (24u - 8u * (bi & 3u))) & 0xFFu;
+            const float scale = __uint_as_float(eb >= 7u ? (eb - 6u) << 23 : 0u);     // 2^(E - 133)
+#pragma unroll
+            for (int b = 0; b < NB; ++b) { acc[b] = fmaf(blk[b], scale, acc[b]); blk[b] = 0.f; }
+        }
+    };
+    int grp = 0;
+    for (; grp < n_full; ++grp) group(grp, std::false_type{});
+    for (; grp < n_groups; ++grp) group(grp, std::true_type{});
+}
+
 // T >= 0: fast path for regular chunks, generic path otherwise.  T = -1: generic path only (any t).
+// T = 104: Cassandra-2 blob with t = 4 (fast path); T = -2: Cassandra-2 blob, generic path (any t).
 // grid = (n_seg, G): CTA (seg, j) handles the superblocks (rb, seg) for rb = j, j + G, ...
 // NB vectors x[b] (bf16 [NB][k]) are multiplied in the same pass: every decoded weight is used NB times, and each
 // vector's sums are formed in the same order as with NB = 1.
@@ -242,7 +335,7 @@ __global__ void __launch_bounds__(1024) k_draft_gemv(const uint32_t* __restrict_
     const int n_ch = ceil_div(scols, chunk_cols);
     // The launch sized shared memory from the host's copy of the header; a blob that does not match it is
     // refused instead of overrunning the buffers.
-    if (seg >= n_seg || (int)blockDim.x < 32 * n_ch || n_ch > 32) {
+    if (seg >= n_seg || (int)blockDim.x < 32 * n_ch || n_ch > 32 || (T == 104 && (smem_u32(lut) & 63u))) {
         if (tid == 0 && d_status) atomicExch(d_status, CASS_ERR_INVALID_ARG);
         return;
     }
@@ -278,7 +371,12 @@ __global__ void __launch_bounds__(1024) k_draft_gemv(const uint32_t* __restrict_
     }
     // the rank -> exponent table, pre-shifted into place
     const uint8_t* cb = reinterpret_cast<const uint8_t*>(blob) + kBlobHeaderBytes;
-    for (int i = tid; i < 256; i += blockDim.x) lut[i] = (uint32_t)cb[i] << 23;
+    if (T == 104) {
+        // signed magnitudes of the 16 field values, as floats: (+-) (m << 4)
+        if (tid < 16) reinterpret_cast<float*>(lut)[tid] = (tid & 8 ? -16.f : 16.f) * (float)(tid & 7);
+    } else {
+        for (int i = tid; i < 256; i += blockDim.x) lut[i] = (uint32_t)cb[i] << 23;
+    }
     // Everything above touches only the blob, which no kernel writes.  When the launch allows this grid to start
     // before its predecessor in the stream has finished, wait here: x and the scratch `partial` are the predecessor's.
     pdl_wait();
@@ -325,7 +423,7 @@ __global__ void __launch_bounds__(1024) k_draft_gemv(const uint32_t* __restrict_
         }
     }
     __syncthreads();
-    if (h_magic != kBlobMagic || (int)h_n != n || (int)h_k != k || (int)h_t != t || (int)h_seg != seg_cols ||
+    if (h[H_MODE] != ((T == 104 || T == -2) ? kBlobModeMx : kBlobModeUnary) || h_magic != kBlobMagic || (int)h_n != n || (int)h_k != k || (int)h_t != t || (int)h_seg != seg_cols ||
         (int)h_chunk != chunk_cols || (int)h_nseg != n_seg || (int)h_nrb != n_rb) {
         // not the blob the caller described: flag it, let the copies already started land, produce nothing
         if (tid == 0 && d_status) atomicExch(d_status, CASS_ERR_INVALID_ARG);
@@ -350,8 +448,15 @@ __global__ void __launch_bounds__(1024) k_draft_gemv(const uint32_t* __restrict_
         if (warp < n_ch && !s_skip[s]) {
             const uint32_t* dir = blob + kBlobDirOffset / 4 + (rb * n_seg + seg) * 4;
             const SbGeom g = SbGeom::make(n_ch, scols, (int)dir[1], (int)dir[2]);
-            if (T >= 0) {
-                chunk_dot_fast<(T >= 0 ? T : 0), NB>(sb, g, warp, lane, dir_chunk_elems(dir[3]), xs, lut, acc);
+            if (T == 104) {
+                chunk_dot_mx4<NB>(sb, g, warp, lane, dir_chunk_elems(dir[3]), xs, reinterpret_cast<const float*>(lut), acc);
+            } else if (T == -2) {
+                const uint32_t xs_a = smem_u32(xs);
+                decode_chunk_generic_mx(sb, g, dir_chunk_elems(dir[3]), warp, lane, t, [&](int col, uint16_t bits) {
+                    x_fma<NB>(x_load<NB>(xs_a + (uint32_t)col * (uint32_t)x_col_bytes(NB)), (uint32_t)bits << 16, acc);
+                });
+            } else if (T >= 0) {
+                chunk_dot_fast<(T >= 0 && T < 8 ? T : 0), NB>(sb, g, warp, lane, dir_chunk_elems(dir[3]), xs, lut, acc);
             } else {
                 const uint32_t xs_a = smem_u32(xs);
                 decode_chunk_generic(sb, g, dir_chunk_elems(dir[3]), warp, lane, t, cb, [&](int col, uint16_t bits) {
@@ -460,7 +565,9 @@ int launch_draft_gemv(const void* blob, const cass_blob_info& bi, const void* x_
         else if (nb == 4) CASS_GEMV_LAUNCH(TT, 4);                                                             \
         else CASS_GEMV_LAUNCH(TT, 8);                                                                          \
     } while (0)
-    if (bi.trunc_bits == 4) CASS_GEMV_LAUNCH_NB(4);
+    if (bi.mode == 2 && bi.trunc_bits == 4) CASS_GEMV_LAUNCH_NB(104);
+    else if (bi.mode == 2) CASS_GEMV_LAUNCH_NB(-2);
+    else if (bi.trunc_bits == 4) CASS_GEMV_LAUNCH_NB(4);
     else if (bi.trunc_bits == 0) CASS_GEMV_LAUNCH_NB(0);
     else CASS_GEMV_LAUNCH_NB(-1);
 #undef CASS_GEMV_LAUNCH_NB

@@ -31,11 +31,13 @@ static EncWs carve(void* base, int n_pad, int k_pad, int n_seg) {
 
 struct EncGeom {
     int n, k, k_pad, n_pad, n_rb, n_seg, seg_cols, chunk_cols, p, t, n_prune;
+    int mx;          // 1: Cassandra-2 (shared exponents), 0: Cassandra-1 (unary code)
 };
 
 static int make_geom(const cass_format* fmt, int rows, int cols, EncGeom* g) {
     if (!fmt || rows <= 0 || cols <= 0) return CASS_ERR_INVALID_ARG;
-    if (fmt->mode != 1) return CASS_ERR_UNSUPPORTED;
+    if (fmt->mode != 1 && fmt->mode != 2) return CASS_ERR_UNSUPPORTED;
+    g->mx = fmt->mode == 2;
     int p = fmt->w_prune_permille, t = fmt->w_trunc_bits;
     if (p < 0 || p > 999 || t < 0 || t > 7) return CASS_ERR_INVALID_ARG;
     int chunk = fmt->w_chunk_cols ? fmt->w_chunk_cols : 256;
@@ -143,6 +145,7 @@ __global__ void k_sizes(const uint16_t* __restrict__ W, EncGeom g, const uint32_
             kept_n += __popc(bm);
         }
     }
+    if (g.mx) ub = 8u * ((kept_n + kMxBlock - 1) / kMxBlock);        // one exponent byte per block of 32 kept values
     if (lane == 0) { cnt_kept[gw] = kept_n; ubits[gw] = ub; }
 }
 
@@ -190,7 +193,8 @@ __global__ void __launch_bounds__(1024) k_directory(EncGeom g, const uint32_t* _
             dir[sb * 4 + 0] = (uint32_t)(excl / 16);
             dir[sb * 4 + 1] = wf;
             dir[sb * 4 + 2] = wu;
-            dir[sb * 4 + 3] = (uint32_t)n_ch | ((uint32_t)chunk_elems_for((int)max_kept, n_ch) << 8);
+            const int e_chunk = g.mx ? mx_chunk_elems_for((int)max_kept, n_ch) : chunk_elems_for((int)max_kept, n_ch);
+            dir[sb * 4 + 3] = (uint32_t)n_ch | ((uint32_t)e_chunk << 8);
         }
         __syncthreads();
         if (tid == 1023) s_carry += s_scan[1023];
@@ -204,6 +208,7 @@ __global__ void __launch_bounds__(1024) k_directory(EncGeom g, const uint32_t* _
         h[H_SEG] = g.seg_cols; h[H_CHUNK] = g.chunk_cols; h[H_NSEG] = g.n_seg; h[H_NRB] = g.n_rb;
         h[H_KEPT] = g.k - g.n_prune; h[H_DIROFF] = kBlobDirOffset; h[H_BODYOFF] = (uint32_t)body_off;
         h[H_TOTLO] = (uint32_t)total; h[H_TOTHI] = (uint32_t)(total >> 32); h[H_MAXSB] = s_maxsb;
+        h[H_MODE] = g.mx ? kBlobModeMx : kBlobModeUnary;
         // zero the padding between directory and first body
         for (unsigned long long o = kBlobDirOffset + 16ull * n_sb; o < body_off; o += 4) blob[o / 4] = 0;
         if (total > blob_cap) {
@@ -270,6 +275,65 @@ __global__ void __launch_bounds__(1024) k_pack(const uint16_t* __restrict__ W, E
     }
 }
 
+// ---- E6 for Cassandra-2: the same superblock with shared exponents (Sec. 4.2, MX) --------------------------
+// Pass 1 finds the largest exponent of every block of 32 kept values of every row (shared memory), pass 2 writes the
+// bitmap, the magnitudes relative to their block's exponent, the exponent bytes and the chunk table.
+__global__ void __launch_bounds__(1024) k_pack_mx(const uint16_t* __restrict__ W, EncGeom g,
+                                                  const uint32_t* __restrict__ keepbm, uint32_t* __restrict__ blob,
+                                                  const uint32_t* __restrict__ abort_flag) {
+    __shared__ uint32_t s_exp[kRowsPerBlock][2048 / kMxBlock];
+    if (*abort_flag) return;
+    const int sb = blockIdx.x, rb = sb / g.n_seg, seg = sb % g.n_seg;
+    const int tid = threadIdx.x, lane = tid & 31, r = tid >> 5;
+    const uint32_t* dir = blob + kBlobDirOffset / 4 + sb * 4;
+    const int scols = seg_cols_of(g.k_pad, g.seg_cols, seg);
+    const int n_ch = dir_n_ch(dir[3]);
+    const uint32_t E = (uint32_t)dir_chunk_elems(dir[3]);
+    const SbGeom sg = SbGeom::make(n_ch, scols, (int)dir[1], (int)dir[2]);
+    uint32_t* body = blob + (size_t)dir[0] * 4;
+    for (int i = tid; i < sg.total / 4; i += 1024) reinterpret_cast<uint4*>(body)[i] = make_uint4(0, 0, 0, 0);
+    for (int i = lane; i < 2048 / kMxBlock; i += 32) s_exp[r][i] = 0;
+    __syncthreads();
+
+    const int row = rb * kRowsPerBlock + r;
+    const int t = g.t, F = 8 - t, per = 32 / F;
+    const int words = g.k_pad / 32;
+    const int w0 = seg * (g.seg_cols / 32);
+    uint32_t k_base = 0;
+    for (int j = 0; j < sg.bm_words; ++j) {                      // pass 1: block maxima
+        uint32_t bm = row < g.n ? keepbm[(size_t)row * words + w0 + j] : 0u;
+        if ((bm >> (31 - lane)) & 1u) {
+            uint32_t k = k_base + (lane ? __popc(bm >> (32 - lane)) : 0u);
+            atomicMax(&s_exp[r][k / kMxBlock], ((uint32_t)W[(size_t)row * g.k + (w0 + j) * 32 + lane] >> 7) & 0xFFu);
+        }
+        k_base += __popc(bm);
+    }
+    __syncwarp();
+    const uint32_t n_blk = (k_base + kMxBlock - 1) / kMxBlock;
+    for (uint32_t b = lane; b < n_blk; b += 32) atomicOr(&body[sg.un + (b / 4) * 32 + r], s_exp[r][b] << (24 - 8 * (b % 4)));
+    k_base = 0;
+    for (int j = 0; j < sg.bm_words; ++j) {                      // pass 2: bitmap, fields, table
+        uint32_t bm = row < g.n ? keepbm[(size_t)row * words + w0 + j] : 0u;
+        if (lane == 0) body[sg.bm + j * 32 + r] = bm;
+        if ((bm >> (31 - lane)) & 1u) {
+            const uint32_t b = W[(size_t)row * g.k + (w0 + j) * 32 + lane];
+            const uint32_t k = k_base + (lane ? __popc(bm >> (32 - lane)) : 0u);
+            const uint32_t e = (b >> 7) & 0xFFu, e_blk = s_exp[r][k / kMxBlock];
+            const uint32_t shift = 1u + e_blk - e;
+            const uint32_t m7 = (shift < 8u && e > 0u && e_blk >= 7u) ? (0x80u | (b & 0x7Fu)) >> shift : 0u;
+            const uint32_t field = ((b >> 15) << (7 - t)) | (m7 >> t);
+            atomicOr(&body[sg.fl + (k / per) * 32 + r], field << (32 - F * (k % per + 1)));
+            if (k % E == 0 && k / E < (uint32_t)n_ch)
+                body[sg.tab + (k / E) * 32 + r] = ((uint32_t)(j * 32 + lane) << 20) | (8u * (k / kMxBlock));
+        }
+        k_base += __popc(bm);
+    }
+    for (int c = lane; c <= n_ch; c += 32) {
+        if (c == n_ch) body[sg.tab + c * 32 + r] = (k_base << 20) | (8u * n_blk);
+        else if ((uint32_t)c * E >= k_base) body[sg.tab + c * 32 + r] = ((uint32_t)scols << 20) | (8u * n_blk);
+    }
+}
+
 // ---- test hook: zero-padded reconstruction of the whole blob ---------------------------------------------
 __global__ void k_decode(const uint32_t* __restrict__ blob, uint16_t* __restrict__ out) {
     const uint32_t* h = blob;
@@ -284,10 +348,12 @@ __global__ void k_decode(const uint32_t* __restrict__ blob, uint16_t* __restrict
     for (int item = threadIdx.x; item < sg.n_ch * 32; item += blockDim.x) {
         int ch = item >> 5, r = item & 31, row = rb * kRowsPerBlock + r;
         if (row >= n) continue;
-        decode_chunk_generic(body, sg, chunk_elems, ch, r, t, cb, [&](int col, uint16_t bits) {
+        auto emit = [&](int col, uint16_t bits) {
             int c = seg * seg_cols + col;
             if (c < k) out[(size_t)row * k + c] = bits;
-        });
+        };
+        if (h[H_MODE] == kBlobModeMx) decode_chunk_generic_mx(body, sg, chunk_elems, ch, r, t, emit);
+        else decode_chunk_generic(body, sg, chunk_elems, ch, r, t, cb, emit);
     }
 }
 
@@ -366,14 +432,19 @@ extern "C" int cass_encode_weights(const cass_format* fmt, const void* W_bf16, c
     CASS_CUDA_CHECK(cudaFuncSetAttribute(k_select, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     k_select<<<g.n, 256, smem, stream>>>(W, act_norm, g, ws.keepbm, ws.hist);
     CASS_LAUNCH_CHECK();
-    k_codebook<<<1, 256, 0, stream>>>(ws.hist, (uint8_t*)blob + kBlobHeaderBytes, ws.exp_to_rank);
-    CASS_LAUNCH_CHECK();
+    if (g.mx) {
+        CASS_CUDA_CHECK(cudaMemsetAsync((uint8_t*)blob + kBlobHeaderBytes, 0, kBlobCodebookBytes, stream));    // no codebook
+    } else {
+        k_codebook<<<1, 256, 0, stream>>>(ws.hist, (uint8_t*)blob + kBlobHeaderBytes, ws.exp_to_rank);
+        CASS_LAUNCH_CHECK();
+    }
     int warps = g.n_pad * g.n_seg;
     k_sizes<<<ceil_div(warps, 8), 256, 0, stream>>>(W, g, ws.keepbm, ws.exp_to_rank, ws.cnt_fw, ws.ubits);
     CASS_LAUNCH_CHECK();
     k_directory<<<1, 1024, 0, stream>>>(g, ws.cnt_fw, ws.ubits, b32, (unsigned long long)blob_cap, ws.abort_flag, d_status);
     CASS_LAUNCH_CHECK();
-    k_pack<<<(unsigned)n_sb, 1024, 0, stream>>>(W, g, ws.keepbm, ws.exp_to_rank, b32, ws.abort_flag);
+    if (g.mx) k_pack_mx<<<(unsigned)n_sb, 1024, 0, stream>>>(W, g, ws.keepbm, b32, ws.abort_flag);
+    else k_pack<<<(unsigned)n_sb, 1024, 0, stream>>>(W, g, ws.keepbm, ws.exp_to_rank, b32, ws.abort_flag);
     CASS_LAUNCH_CHECK();
     return CASS_OK;
 }
@@ -388,6 +459,7 @@ extern "C" int cass_weight_blob_info(const void* blob, cass_blob_info* h_info, v
     h_info->rows = h[H_ROWS]; h_info->cols = h[H_COLS]; h_info->prune_permille = h[H_P]; h_info->trunc_bits = h[H_T];
     h_info->seg_cols = h[H_SEG]; h_info->chunk_cols = h[H_CHUNK]; h_info->n_seg = h[H_NSEG]; h_info->n_rowblocks = h[H_NRB];
     h_info->kept_per_row = h[H_KEPT]; h_info->max_superblock_bytes = h[H_MAXSB];
+    h_info->mode = h[H_MODE] == kBlobModeMx ? 2 : 1; h_info->reserved = 0;
     h_info->total_bytes = (uint64_t)h[H_TOTLO] | ((uint64_t)h[H_TOTHI] << 32);
     return CASS_OK;
 }

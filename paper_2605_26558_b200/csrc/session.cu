@@ -52,7 +52,7 @@ struct Plan {
 
 static int check_desc(const cass_model_desc* d, const cass_format* f) {
     if (!d || !f) return CASS_ERR_INVALID_ARG;
-    if (f->mode != 1) return CASS_ERR_UNSUPPORTED;
+    if (f->mode != 1 && f->mode != 2) return CASS_ERR_UNSUPPORTED;     // weights: Cassandra-1 or Cassandra-2; KV: Cassandra-1
     if (d->max_batch != 1 && d->max_batch != 2 && d->max_batch != 4 && d->max_batch != 8) return CASS_ERR_UNSUPPORTED;
     if (d->n_layers <= 0 || d->hidden <= 0 || d->n_q_heads <= 0 || d->n_kv_heads <= 0 || d->head_dim <= 0 ||
         d->ffn <= 0 || d->vocab <= 0 || d->max_seq < 2 * kMaxVerifyRows)

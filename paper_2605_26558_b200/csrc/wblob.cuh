@@ -15,8 +15,14 @@ namespace cass {
 
 enum BlobHeaderWord {
     H_MAGIC = 0, H_VERSION, H_ROWS, H_COLS, H_P, H_T, H_SEG, H_CHUNK, H_NSEG, H_NRB, H_KEPT,
-    H_DIROFF, H_BODYOFF, H_TOTLO, H_TOTHI, H_MAXSB
+    H_DIROFF, H_BODYOFF, H_TOTLO, H_TOTHI, H_MAXSB, H_MODE
 };
+// H_MODE: 0 = Cassandra-1 (unary exponent code, the layout described above), 2 = Cassandra-2 (MX: the kept values of
+// a row are cut into blocks of 32 that share one exponent byte; fields hold sign + the high 7-t bits of a 7-bit
+// magnitude, packed from the most significant end; the fourth section holds the exponent bytes, four per word from
+// the most significant end; a table entry's low 20 bits are 8 x the index of the chunk's first block).
+constexpr uint32_t kBlobModeUnary = 0, kBlobModeMx = 2;
+constexpr int kMxBlock = 32;
 constexpr uint32_t kBlobMagic = 0x57534143u;
 constexpr uint32_t kBlobVersion = 3;
 constexpr int kBlobHeaderBytes = 128;
@@ -51,6 +57,25 @@ __host__ __device__ inline int chunk_elems_for(int max_kept, int n_ch) {       /
     int per_chunk = ceil_div(max_kept, n_ch);
     int e = ceil_div(per_chunk, 8) * 8;
     return e < 8 ? 8 : e;
+}
+
+__host__ __device__ inline int mx_chunk_elems_for(int max_kept, int n_ch) {    // smallest multiple of 32 with n_ch * E >= max_kept
+    int per_chunk = ceil_div(max_kept, n_ch);
+    int e = ceil_div(per_chunk, kMxBlock) * kMxBlock;
+    return e < kMxBlock ? kMxBlock : e;
+}
+
+// Cassandra-2 element -> bf16 bits: field = sign, magnitude >> t (8-t bits); value = (-1)^s (mag << t) 2^(E-133);
+// the leading-zero count of the magnitude gives the shift and the exponent correction; zero magnitude -> +0.
+__device__ __forceinline__ uint16_t mx_value_bf16(uint32_t field, uint32_t e_blk, int t) {
+    const uint32_t mag = (field & ((1u << (7 - t)) - 1u)) << t;
+    if (mag == 0) return 0;
+    const int top = 31 - __clz(mag);
+    return (uint16_t)(((field >> (7 - t)) << 15) | ((e_blk - 6u + (uint32_t)top) << 7) | ((mag << (7 - top)) & 0x7Fu));
+}
+__device__ __forceinline__ uint32_t mx_field_of(uint32_t fword, int j, int t) {        // field j of a word
+    const int w = 8 - t;
+    return (fword >> (32 - w * (j + 1))) & ((1u << w) - 1u);
 }
 
 __host__ __device__ inline int seg_cols_of(int k_pad, int seg_cols, int seg) {
@@ -105,6 +130,36 @@ __device__ inline void decode_chunk_generic(const uint32_t* sb, const SbGeom& g,
         int rank = read_unary(un_row, ub, limit);
         uint32_t e = rank_to_exp[rank & 255];
         emit((int)col, (uint16_t)(field_sign_mant_bf16(fword, k % per, t) | (e << 7)));
+        col += 1;
+    }
+}
+
+// The same for a Cassandra-2 blob (shared exponent per block of 32 kept values instead of a codeword per value).
+template <class Emit>
+__device__ inline void decode_chunk_generic_mx(const uint32_t* sb, const SbGeom& g, int chunk_elems, int ch, int row,
+                                               int t, Emit&& emit) {
+    const int per = 32 / (8 - t);
+    const uint32_t e0 = sb[g.tab + ch * 32 + row];
+    const int kept = (int)(sb[g.tab + g.n_ch * 32 + row] >> 20);
+    const int k0 = ch * chunk_elems;
+    const int cnt = min(chunk_elems, kept - k0);
+    if (cnt <= 0) return;
+    uint32_t col = e0 >> 20;
+    const uint32_t* fl_row = sb + g.fl + row;
+    const uint32_t* ex_row = sb + g.un + row;
+    const uint32_t col_lim = (uint32_t)g.bm_words * 32u;
+    for (int k = k0; k < k0 + cnt; ++k) {
+        bool found = false;
+        while (col < col_lim) {
+            uint32_t bm = sb[g.bm + (col >> 5) * 32 + row] << (col & 31);
+            if (bm) { col += __clz(bm); found = true; break; }
+            col = (col | 31u) + 1u;
+        }
+        if (!found) return;
+        const int b = k / kMxBlock;
+        if (b / 4 >= g.w_u) return;                           // corrupt geometry: stay inside the buffers
+        const uint32_t e_blk = (ex_row[(b / 4) * 32] >> (24 - 8 * (b % 4))) & 0xFFu;
+        emit((int)col, mx_value_bf16(mx_field_of(fl_row[(k / per) * 32], k % per, t), e_blk, t));
         col += 1;
     }
 }
