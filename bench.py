@@ -215,7 +215,8 @@ def run_cass(args):
     max_seq = n_prompt + (max(args.steps, args.warmup) + 2) * per_step + 64
     max_seq = (max_seq + 255) // 256 * 256
     nb = args.batch
-    eng = engine.Engine(shape, gw, max_seq=max_seq, gamma_max=max(gamma, 1), device=dev, batch=nb)
+    eng = engine.Engine(shape, gw, fmt=cass.default_format(mode=args.mode), max_seq=max_seq, gamma_max=max(gamma, 1),
+                        device=dev, batch=nb)
     prompt = torch.stack([synth.random_prompt(n_prompt, shape.vocab, seed=rank * 8 + b) for b in range(nb)])
     eng.prefill(prompt, calibrate=True)
     eng.encode_weights(eng.calib_norms())
@@ -356,7 +357,9 @@ def run_cass(args):
                                     "qwen": "qwen-style shape (config 5): 48 layers, hidden 5120, vocab 152064"}[args.config]
                                    + f", batch {nb}, prompt {n_prompt}, positions {n_prompt}..{n_prompt + args.steps * per_step}",
                        "batch": nb,
-                       "gamma": gamma, "format": "cassandra-1 p=40% t=4 (weights and KV)",
+                       "gamma": gamma,
+                       "format": "cassandra-1 p=40% t=4 (weights and KV)" if args.mode == 1 else
+                                 "cassandra-2 (MX, blocks of 32) p=40% t=4 weights, cassandra-1 KV",
                        "l2": "inputs larger than L2 (16 GB bf16 weights + speculation data per step)",
                        "parallelism": "replicas only" if world > 1 else "1 gpu",
                        "mean_accepted_len": emitted_all / (args.steps * world * nb) - 1.0,
@@ -393,6 +396,8 @@ def main():
     ap.add_argument("--prompt", type=int, default=512)
     ap.add_argument("--batch", type=int, default=1, choices=[1, 2, 4, 8], help="sequences decoded together (config 4 sweeps this)")
     ap.add_argument("--config", default="llama8b", choices=["llama8b", "tiny", "qwen"])
+    ap.add_argument("--mode", type=int, default=1, choices=[1, 2],
+                    help="weight format of the draft: 1 = Cassandra-1 (unary exponents), 2 = Cassandra-2 (MX exponents)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.warmup < 3:

@@ -104,6 +104,17 @@ typedef struct cass_blob_info {
     uint64_t total_bytes;
 } cass_blob_info;
 
+/* With fmt->mode = 2 the same call produces Cassandra-2 speculation data (Sec. 4.2, exponent compression by the MX
+ * format; Sec. 5.1, MX decoder): pruning, bitmap and truncation as above, but instead of a unary codeword per value
+ * every block of 32 consecutive kept values of a row (within one column segment) shares one exponent byte E = the
+ * largest exponent of the block, and a field holds the sign and the high 7-t bits of the 7-bit magnitude
+ * (0x80 | mantissa) >> (1 + E - e) (an MXINT8 element in sign-magnitude form, truncated toward zero; 0 when the value
+ * lies 7 or more binades below the block maximum, when it is zero or denormal, or when E < 7).  The draft value is
+ * (-1)^s (magnitude >> t << t) 2^(E-133).  Unlike mode 1 this loses exponent information (the paper's "minor
+ * accuracy loss"); verification stays bf16, so the token stream stays lossless.  cass_draft_gemv,
+ * cass_draft_gemv_batch, cass_decode_weights, cass_weight_blob_stats (code_bits = exponent bits) and the session
+ * take blobs of either mode. */
+
 /* Reads the blob header back to the host.  SYNCHRONISES `stream`. */
 int cass_weight_blob_info(const void* blob, cass_blob_info* h_info, void* stream);
 

@@ -274,10 +274,11 @@ def main():
     ap.add_argument("--tokens", type=int, default=8192, help="tokens to decode (--kernel decode)")
     ap.add_argument("--prompt", type=int, default=512)
     ap.add_argument("--config", default="llama8b")
+    ap.add_argument("--mode", type=int, default=1, help="weight format: 1 = Cassandra-1 (unary), 2 = Cassandra-2 (MX)")
     ap.add_argument("--p", type=int, default=400)
     ap.add_argument("--t", type=int, default=4)
     args = ap.parse_args()
-    fmt = B.default_format(w_p=args.p, w_t=args.t, chunk_cols=args.chunk, seg_cols=args.seg)
+    fmt = B.default_format(w_p=args.p, w_t=args.t, chunk_cols=args.chunk, seg_cols=args.seg, mode=args.mode)
     out = []
     if args.kernel in ("gemv", "all"):
         for name in (SHAPES if args.shape == "all" else [args.shape]):
