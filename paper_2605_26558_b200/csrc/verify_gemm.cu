@@ -9,8 +9,7 @@
 //
 // Row-count invariance: an accumulator column belongs to one token row, the tile shape, the K ranges and the order
 // of the MMAs depend on (n, k) only, so a row gives the same bits whether it is verified alone or with others.
-#include <cuda.h>
-
+#include "tc.cuh"
 #include "kernels.cuh"
 
 namespace cass {
@@ -22,25 +21,6 @@ constexpr int kTcThreads = 192;
 constexpr int tc_b_bytes(int bn) { return bn * kTcBK * 2; }
 constexpr int tc_smem(int bn) { return tc_stages(bn) * (kTcABytes + tc_b_bytes(bn)) + 256 + 1024; }     // + barriers + alignment slack
 constexpr int tc_tmem_cols(int bn) { return bn <= 32 ? 32 : 64; }                                   // a power of two >= 32
-
-// ---- tensor maps ------------------------------------------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-static EncodeTiledFn encode_fn() {
-    static EncodeTiledFn fn = nullptr;
-    static bool tried = false;
-    if (!tried) {
-        tried = true;
-        void* p = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-            q == cudaDriverEntryPointSuccess)
-            fn = (EncodeTiledFn)p;
-    }
-    return fn;
-}
 
 // bf16 matrix [rows][cols] row-major -> map with a (box_rows x 64)-element box, 128-byte swizzle, zero fill outside.
 static int make_map(CUtensorMap* m, const void* ptr, int rows, int cols, int box_rows) {
@@ -56,43 +36,8 @@ static int make_map(CUtensorMap* m, const void* ptr, int rows, int cols, int box
     return r == CUDA_SUCCESS ? CASS_OK : CASS_ERR_INVALID_ARG;
 }
 
-// ---- PTX wrappers -----------------------------------------------------------------------------------------
-__device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
-    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(
-                     smem_u32(smem_dst)),
-                 "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y)
-                 : "memory");
-}
-
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-__device__ __forceinline__ void tc_commit(uint64_t* bar) {      // arrives on `bar` when all MMAs issued so far are done
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-
-// Shared-memory operand descriptor: K-major tile, rows of 64 bf16 (128 bytes), 128-byte swizzle, groups of 8 rows
-// 1024 bytes apart.
-__device__ __forceinline__ uint64_t tc_smem_desc(const void* p) {
-    uint64_t d = (uint64_t)((smem_u32(p) & 0x3FFFFu) >> 4);
-    d |= (uint64_t)(1024 >> 4) << 32;      // stride between 8-row groups
-    d |= 1ull << 46;                       // descriptor version of this architecture
-    d |= 2ull << 61;                       // 128-byte swizzle
-    return d;
-}
-
 // Instruction descriptor of kind::f16: D fp32, A and B bf16, both K-major, M = 128, N = bn.
-constexpr uint32_t tc_idesc(int bn) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(kTcBM >> 4) << 24);
-}
-
-__device__ __forceinline__ void tc_mma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
-        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
+constexpr uint32_t tc_idesc(int bn) { return tc_idesc_mn(kTcBM, bn, false); }
 
 // grid (m tiles, k splits).  partial: fp32 [k splits][BN][n].
 template <int BN>

@@ -103,3 +103,52 @@ def test_draft_attention_llama_layer_shape(cass, n_pos, n_q):
     assert (err <= 2.0 ** -8 * np.abs(want) + 0.05 * TOL * rms).all(), (err.max(), rms)
     assert np.median(err) <= 0.1 * TOL * rms
     eng.close()
+
+
+@pytest.mark.parametrize("n_pos,g,n_q", [(3, 4, 32), (127, 0, 32), (128, 4, 32), (300, 7, 32), (4096, 4, 32), (200, 3, 64)])
+def test_verify_attention_llama_head_geometry(cass, n_pos, g, n_q):
+    """Verification attention with heads of 128 (the tensor-core kernel where rows x group <= 32): g+1 new rows over
+    n_pos cached positions of synthetic KV, against the oracle's causal softmax(q K^T / sqrt(d)) V computed in fp64 from
+    the rotated q rows and the bf16 caches the call leaves behind."""
+    from paper_2605_26558_b200 import engine
+    G = n_q // 8
+    shape = synth.ModelShape(n_layers=1, hidden=256, n_q_heads=n_q, n_kv_heads=8, head_dim=128, ffn=256, vocab=256)
+    wt = synth.model_weights(shape, 0, device="cuda")
+    gw = {"layers": [engine.fuse_layer_weights(lw) for lw in wt["layers"]], "embed": wt["embed"], "lm_head": wt["lm_head"],
+          "norm_final": wt["norm_final"]}
+    eng = engine.Engine(shape, gw, max_seq=4096 + 64, gamma_max=max(g, 1))
+    k, v = synth.kv_fill(n_pos, 8, 128, 3, "va/kv", device="cuda")
+    cass.cass_kv_append(eng.session, 0, k.contiguous(), v.contiguous(), 0, n_pos, cass.KV_BF16)
+    cass.cass_set_len(eng.session, n_pos)
+    rows = g + 1
+    toks = torch.arange(7, 7 + rows, dtype=torch.int32, device="cuda")
+    cass.cass_verify(eng.session, toks, g, eng.targ)
+    torch.cuda.synchronize()
+    assert eng.status()[0] == 0
+    base = eng.mem.data_ptr()
+    m16 = eng.mem.view(torch.bfloat16)
+
+    def grab(which):
+        p, r, c = cass.cass_debug_activation(eng.session, which)
+        off = (p - base) // 2
+        return m16[off: off + rows * c].view(rows, c).float().cpu().numpy().astype(np.float64)
+
+    qkv, got = grab(2), grab(1)
+    kc = cass.cass_kv_query(eng.session, 0, 0, 0).k_or_v_bf16
+    vc = cass.cass_kv_query(eng.session, 0, 1, 0).k_or_v_bf16
+    n_all = n_pos + rows
+    kd = m16[(kc - base) // 2: (kc - base) // 2 + n_all * 1024].view(n_all, 8, 128).float().cpu().numpy().astype(np.float64)
+    vd = m16[(vc - base) // 2: (vc - base) // 2 + n_all * 1024].view(n_all, 8, 128).float().cpu().numpy().astype(np.float64)
+    want = np.zeros((rows, n_q * 128))
+    for r in range(rows):
+        vis = n_pos + r + 1
+        for hq in range(n_q):
+            q = qkv[r, hq * 128: (hq + 1) * 128]
+            sc = kd[:vis, hq // G, :] @ q / np.sqrt(128.0)
+            p = np.exp(sc - sc.max())
+            want[r, hq * 128: (hq + 1) * 128] = (p / p.sum()) @ vd[:vis, hq // G, :]
+    rms = float(np.sqrt(np.mean(want ** 2)))
+    err = np.abs(got - want)
+    assert np.all(err <= 2.0 ** -7 * np.abs(want) + TOL * rms), float(err.max() / rms)
+    assert np.median(err) <= 0.25 * TOL * rms
+    eng.close()
