@@ -168,6 +168,21 @@ __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.
 
 // Programmatic dependent launch: let the next kernel start / wait for the previous kernel's memory.
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// Which kernel classes release their successor (griddepcontrol.launch_dependents) before they finish (bit per class:
+// 0 small operators, 1 KV encoder, 2 draft attention, 3 attention merge, 4 verification attention, 5 verification
+// GEMM).  A kernel outside the mask releases its successor when it exits; every kernel still starts with
+// griddepcontrol.wait, and the draft GEMV does its set-up (barriers, table, first weight copy) before that wait.
+// Measured on the full model (ms per speculative step / plain tokens per s): none 25.5 / 249, small operators + GEMM
+// 25.7 / 252, all but the KV encoder about the same, with the KV encoder 26.6 / 224, all 27.1 / 226: an early release
+// mostly lets the successor's CTAs take SM resources while they wait, so the default releases nothing early.
+#ifndef CASS_PDL_EARLY_MASK
+#define CASS_PDL_EARLY_MASK 0x00
+#endif
+template <int CLS>
+__device__ __forceinline__ void pdl_early() {
+    if constexpr ((CASS_PDL_EARLY_MASK >> CLS) & 1) pdl_launch_dependents();
+}
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 }  // namespace cass

@@ -186,7 +186,7 @@ __global__ void __launch_bounds__(kDaThreads) k_draft_attn(KvGeom g, KvComp ck0,
                                                            int qkv_stride, int n_q, const DevState* __restrict__ st, AttnScratch sc,
                                                            int n_chunks_alloc) {
     extern __shared__ __align__(16) uint8_t smem[];
-    pdl_launch_dependents();
+    pdl_early<2>();
     pdl_wait();
     const int chunk = blockIdx.x, head = blockIdx.y, seq = blockIdx.z;
     const int cur_len = st->len[seq] + st->inflight[seq] + 1;  // positions visible to the drafted token
@@ -315,7 +315,7 @@ __global__ void __launch_bounds__(kMergeThreads) k_attn_merge(AttnScratch sc, in
                                                               const DevState* __restrict__ st, int draft_mode, uint16_t* __restrict__ out) {
     extern __shared__ __align__(16) float w_s[];    // [n_chunks_alloc] weights e^{m_c - M}, then [kMergeWarps][d] partial outputs
     __shared__ float s_red[kMergeWarps];
-    pdl_launch_dependents();
+    pdl_early<3>();
     pdl_wait();
     const int hq = blockIdx.x, r = blockIdx.y;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;

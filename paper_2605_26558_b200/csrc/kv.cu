@@ -95,7 +95,7 @@ __global__ void __launch_bounds__(256) k_kv_append(KvGeom g, KvComp ck, KvComp c
     __shared__ uint32_t s_fix[kKvWarps][kKvFixMax];          // bitmap (<= 8) + field words (<= 64)
     __shared__ uint32_t s_una[kKvWarps][kKvStageWords];
     __shared__ uint32_t s_nw[kKvWarps], s_off[kKvWarps];
-    pdl_launch_dependents();
+    pdl_early<1>();
     pdl_wait();
     const int head = blockIdx.x, kind = blockIdx.y, seq = seq0 + blockIdx.z;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;

@@ -17,7 +17,7 @@ __global__ void k_rope_table(float* __restrict__ cos_t, float* __restrict__ sin_
 
 __global__ void k_embed(const int32_t* __restrict__ toks, int tok_stride, const uint16_t* __restrict__ embed,
                         uint16_t* __restrict__ h, int hidden) {
-    pdl_launch_dependents();
+    pdl_early<0>();
     pdl_wait();
     int r = blockIdx.x;
     const uint16_t* src = embed + (size_t)toks[(size_t)r * tok_stride] * hidden;
@@ -44,7 +44,7 @@ __global__ void __launch_bounds__(1024) k_residual_rmsnorm(uint16_t* __restrict_
                                                            const uint16_t* __restrict__ gain, uint16_t* __restrict__ out,
                                                            int hidden, float eps) {
     __shared__ float s_red[32];
-    pdl_launch_dependents();            // a following draft GEMV may start fetching its weights now
+    pdl_early<0>();
     pdl_wait();
     const int r = blockIdx.x;
     uint16_t* hr = h + (size_t)r * hidden;
@@ -108,7 +108,7 @@ __global__ void __launch_bounds__(1024) k_residual_rmsnorm(uint16_t* __restrict_
 __global__ void k_qkv_rope(uint16_t* __restrict__ qkv, Partials pp,
                            const float* __restrict__ cos_t, const float* __restrict__ sin_t,
                            const DevState* __restrict__ st, int use_inflight, int rps, int n_q, int n_kv, int d) {
-    pdl_launch_dependents();
+    pdl_early<0>();
     pdl_wait();
     const int r = blockIdx.y, half = d / 2;
     const int qkv_dim = (n_q + 2 * n_kv) * d;
@@ -142,7 +142,7 @@ __global__ void k_qkv_rope(uint16_t* __restrict__ qkv, Partials pp,
 
 __global__ void k_swiglu(const uint16_t* __restrict__ gu, Partials pp,
                          uint16_t* __restrict__ act, int ffn) {
-    pdl_launch_dependents();
+    pdl_early<0>();
     pdl_wait();
     const int r = blockIdx.y;
     for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < ffn; i += gridDim.x * blockDim.x) {
@@ -176,7 +176,7 @@ __global__ void __launch_bounds__(256) k_argmax_part(const float* __restrict__ l
                                                      int32_t* __restrict__ tmp_i, float* __restrict__ logits_copy) {
     __shared__ float s_v[8];
     __shared__ int s_i[8];
-    pdl_launch_dependents();
+    pdl_early<0>();
     pdl_wait();
     const int r = blockIdx.y, nsl = gridDim.x;
     const int per = ceil_div(vocab, nsl);
@@ -214,7 +214,7 @@ __global__ void __launch_bounds__(kArgmaxSlices) k_argmax_final(const float* __r
                                                                 int bump_inflight) {
     __shared__ float s_v[kArgmaxSlices / 32];
     __shared__ int s_i[kArgmaxSlices / 32];
-    pdl_launch_dependents();
+    pdl_early<0>();
     pdl_wait();
     const int r = blockIdx.x;
     float best = -INFINITY;
@@ -240,7 +240,7 @@ __global__ void __launch_bounds__(kArgmaxSlices) k_argmax_final(const float* __r
 // next_tok[b * next_stride].
 __global__ void k_accept(DevState* st, const int32_t* __restrict__ draft, int draft_stride, const int32_t* __restrict__ target, int g,
                          int32_t* n_acc, int32_t* out_tokens, int32_t* next_tok, int next_stride) {
-    pdl_launch_dependents();
+    pdl_early<0>();
     pdl_wait();
     if (threadIdx.x != 0) return;
     const int b = blockIdx.x;
@@ -265,7 +265,7 @@ __global__ void k_accept(DevState* st, const int32_t* __restrict__ draft, int dr
 
 __global__ void k_calib_accum(const uint16_t* __restrict__ x, int rows, int cols, float* __restrict__ sumsq,
                               const DevState* __restrict__ st) {
-    pdl_launch_dependents();
+    pdl_early<0>();
     pdl_wait();
     if (!st->calib_on) return;
     int c = blockIdx.x * blockDim.x + threadIdx.x;

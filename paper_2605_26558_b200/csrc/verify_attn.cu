@@ -19,7 +19,7 @@ __global__ void __launch_bounds__(kVaThreads) k_verify_attn(KvGeom g, const uint
                                                             int rows, int n_q, const DevState* __restrict__ st, AttnScratch sc,
                                                             int n_chunks_alloc) {
     extern __shared__ __align__(16) uint8_t smem[];
-    pdl_launch_dependents();
+    pdl_early<4>();
     pdl_wait();
     const int chunk = blockIdx.x, head = blockIdx.y, seq = blockIdx.z;
     const int len = st->len[seq];

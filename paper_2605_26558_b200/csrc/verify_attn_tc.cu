@@ -35,7 +35,7 @@ __global__ void __launch_bounds__(kVtThreads) k_verify_attn_tc(const __grid_cons
                                                                 const DevState* __restrict__ st, AttnScratch sc, int n_chunks_alloc,
                                                                 int32_t* __restrict__ d_status) {
     extern __shared__ uint8_t smem_dyn[];
-    pdl_launch_dependents();
+    pdl_early<4>();
     pdl_wait();
     const int chunk = blockIdx.x, head = blockIdx.y, seq = blockIdx.z;
     const int len = st->len[seq];

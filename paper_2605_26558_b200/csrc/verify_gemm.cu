@@ -75,7 +75,7 @@ __global__ void __launch_bounds__(kTcThreads) k_verify_gemm_tc(const __grid_cons
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
     // barriers and tensor memory are set up; the activations and the scratch belong to the preceding kernels
-    pdl_launch_dependents();
+    pdl_early<5>();
     pdl_wait();
 
     if (warp == 0 && lane == 0) {
@@ -139,7 +139,7 @@ __global__ void __launch_bounds__(kTcThreads) k_verify_gemm_tc(const __grid_cons
 
 __global__ void k_verify_gemm_finish(const float* __restrict__ partial, int rows, int bn, int n, int n_split,
                                      uint16_t* __restrict__ y_bf16, float* __restrict__ y_f32) {
-    pdl_launch_dependents();
+    pdl_early<5>();
     pdl_wait();
     const int j = blockIdx.x * blockDim.x + threadIdx.x, r = blockIdx.y;
     if (j >= n || r >= rows) return;
