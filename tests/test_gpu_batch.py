@@ -145,6 +145,24 @@ def test_batched_streams_equal_the_sequences_decoded_alone(cass, batch, gamma):
     eng.close()
 
 
+def test_batched_streams_with_heads_of_128(cass):
+    """The same comparison on a model with heads of 128 (tensor-core verification attention, whose K/V tiles of
+    sequence b are fetched through the sequence dimension of its tensor maps) and 4 query heads per KV head."""
+    shape = synth.ModelShape(n_layers=2, hidden=256, n_q_heads=8, n_kv_heads=2, head_dim=128, ffn=512, vocab=512)
+    gw = _weights(cass, shape, 3)
+    n_prompt, n_tok, batch, gamma = 150, 20, 4, 4
+    prompts = torch.stack([synth.random_prompt(n_prompt, shape.vocab, 300 + b) for b in range(batch)])
+    eng, first = _ready(cass, shape, gw, prompts, batch, gamma, max_seq=320)
+    out, stats = eng.generate(n_tok, gamma)
+    assert eng.status()[0] == 0
+    for b in range(batch):
+        alone, f1 = _ready(cass, shape, gw, prompts[b], 1, gamma, max_seq=320)
+        want, _ = alone.generate(len(out[b]), 0)
+        alone.close()
+        assert f1 == first[b] and out[b] == want[: len(out[b])], b
+    eng.close()
+
+
 def test_batched_graph_replay_and_gamma_switch(cass):
     """A captured batched step replays to the same streams as eager stepping, also after the draft length changes."""
     shape = synth.TINY
