@@ -2,12 +2,14 @@
 """Benchmark of the Cassandra self-speculative decode step on B200.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl cass|reference] [--gamma G]
+                    [--config llama8b|qwen|tiny] [--batch 1|2|4|8] [--mode 1|2] [--prompt P]
 
 A step is one pass of the whole hot path over one batch-1 sequence: gamma draft tokens (draft GEMVs and draft
 attention on the speculation data, the KV encoder appending each drafted token), one bf16 verification pass over
 gamma+1 rows, and greedy accept/rollback.  The workload is the full Llama-3-8B-shaped model (32 layers, vocab
 128256, random init, prompt of 512 random ids); weights (16 GB bf16 + about 5 GB of speculation data) are far larger
-than L2, so no flush is needed between steps.  With N > 1 every rank runs an independent replica (the path does
+than L2, so no flush is needed between steps.  --batch decodes several sequences together (independent prompts,
+per-sequence acceptance), --mode 2 drafts from Cassandra-2 (MX) weights, --config picks another model shape.  With N > 1 every rank runs an independent replica (the path does
 not shard); the time is the maximum over ranks.
 
 `--impl reference` times the CPU oracle (test infrastructure, never tuned) on a bounded sample of the same workload.
