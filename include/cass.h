@@ -131,6 +131,19 @@ int cass_weight_blob_stats(const void* blob, const cass_blob_info* h_info, void*
 /* Test hook: zero-padded reconstruction (Sec. 4.1, draft inference) of a whole blob into bf16 [rows][cols]. */
 int cass_decode_weights(const void* blob, const cass_blob_info* h_info, void* W_bf16_out, void* stream);
 
+/* Verification data of a Cassandra-1 blob (Sec. 4.1 target inference: the target model reads speculation and
+ * verification data and concatenates them; Sec. 5.1 encoder: the verification group is stored without transformation):
+ * the low t mantissa bits of every kept value and the pruned values as they are.  Layout: 8 header words {'CASV', 1,
+ * rows, cols, kept per row, t, words per row, 0}; per row ceil(kept*t/32) words of t-bit groups (column order, MSB
+ * first), then the pruned values (column order) as 16-bit little-endian halfwords, padded to a word.  The bitmap is the
+ * blob's.  cass_decode_full rebuilds the bf16 matrix from the two parts, bit for bit.  This library's verification
+ * pass reads a bf16 copy instead; these calls exist to check the exactness of the split and to weigh its parts.
+ * Mode 1 blobs only (CASS_ERR_UNSUPPORTED otherwise).  h_bytes: host; vdata: device, 4-byte aligned. */
+int cass_verification_data_bytes(const cass_blob_info* h_info, size_t* h_bytes);
+int cass_encode_verification_data(const void* blob, const cass_blob_info* h_info, const void* W_bf16, void* vdata,
+                                  size_t vdata_bytes, void* stream);
+int cass_decode_full(const void* blob, const cass_blob_info* h_info, const void* vdata, void* W_bf16_out, void* stream);
+
 /* ------------------------------------------------------------------------------------------------------
  * Draft GEMV on speculation data (Sec. 4.1 draft inference; decoder dataflow of Sec. 5.1 / Algorithm 1).
  *   y[r] = sum_c decode(blob)[r][c] * x[c], fp32 accumulation, y rounded to bf16 (y_bf16) and/or kept fp32.

@@ -412,3 +412,61 @@ def kv_codebook(x_bits: np.ndarray, p: int) -> np.ndarray:
     heads (x_bits [..., d])."""
     keep = codec.keep_mask_kv(x_bits, p)
     return codec.codebook_from_counts(codec.exponent_counts(x_bits, keep))
+
+
+# ---- verification data (Sec. 4.1 target inference, Sec. 5.1 encoder) ------------------------------------------------
+# What the speculation data leaves out: the low t mantissa bits of every kept value and the pruned values as they
+# are.  Together with the speculation data (which holds the bitmap) it gives the bf16 matrix back exactly.
+# Layout of this build: header of 8 words {magic 'CASV', 1, rows, cols, kept per row, t, words per row, 0}, then per
+# row (all rows have the same kept count, so rows have one fixed size): ceil(kept*t/32) words with the t-bit groups of
+# the kept values in column order, filled MSB first, then the pruned values in column order as 16-bit little-endian
+# halfwords (padded to a whole word).
+VDATA_MAGIC = 0x56534143
+VDATA_HEADER_WORDS = 8
+
+
+def verification_row_words(cols: int, p: int, t: int) -> int:
+    kept = cols - codec.n_pruned(cols, p)
+    return (kept * t + 31) // 32 + (cols - kept + 1) // 2
+
+
+def encode_verification_data(w_bits: np.ndarray, keep: np.ndarray, p: int, t: int) -> np.ndarray:
+    w_bits = np.asarray(w_bits, dtype=np.uint16)
+    n, k = w_bits.shape
+    kept = k - codec.n_pruned(k, p)
+    lo_words = (kept * t + 31) // 32
+    row_words = verification_row_words(k, p, t)
+    out = np.zeros((n, row_words), dtype=np.uint32)
+    for r in range(n):
+        idx = np.flatnonzero(keep[r])
+        assert idx.size == kept
+        if t:
+            lo = (w_bits[r, idx] & ((1 << t) - 1)).astype(np.uint8)
+            bits = ((lo[:, None] >> np.arange(t - 1, -1, -1)[None, :]) & 1).reshape(-1)
+            out[r, :lo_words] = bits_to_words(bits)
+        raw = w_bits[r, ~keep[r]].astype(np.uint32)
+        if raw.size % 2:
+            raw = np.concatenate([raw, np.zeros(1, np.uint32)])
+        out[r, lo_words:] = raw[0::2] | (raw[1::2] << 16)
+    header = np.array([VDATA_MAGIC, 1, n, k, kept, t, row_words, 0], dtype=np.uint32)
+    return np.concatenate([header, out.reshape(-1)])
+
+
+def decode_full(draft_bits: np.ndarray, keep: np.ndarray, vdata: np.ndarray) -> np.ndarray:
+    """Speculation data (as its zero-padded reconstruction and its bitmap) + verification data -> the bf16 matrix."""
+    vdata = np.asarray(vdata, dtype=np.uint32)
+    assert int(vdata[0]) == VDATA_MAGIC and int(vdata[1]) == 1
+    n, k, kept, t, row_words = (int(x) for x in vdata[2:7])
+    lo_words = (kept * t + 31) // 32
+    body = vdata[VDATA_HEADER_WORDS:].reshape(n, row_words)
+    out = np.array(draft_bits, dtype=np.uint16, copy=True)
+    for r in range(n):
+        idx = np.flatnonzero(keep[r])
+        if t:
+            bits = words_to_bits(body[r, :lo_words])[: kept * t].reshape(kept, t)
+            lo = (bits.astype(np.uint16) << np.arange(t - 1, -1, -1, dtype=np.uint16)[None, :]).sum(axis=1).astype(np.uint16)
+            out[r, idx] |= lo
+        raw = body[r, lo_words:]
+        half = np.stack([raw & 0xFFFF, raw >> 16], axis=1).reshape(-1)[: k - kept].astype(np.uint16)
+        out[r, ~keep[r]] = half
+    return out

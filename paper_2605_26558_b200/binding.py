@@ -144,6 +144,21 @@ def cass_decode_weights(blob, info: BlobInfo, out_bf16, stream=None):
     _check("cass_decode_weights", lib.cass_decode_weights(_ptr(blob), C.byref(info), _ptr(out_bf16), _stream(stream)))
 
 
+def cass_verification_data_bytes(info: BlobInfo) -> int:
+    n = C.c_size_t(0)
+    _check("cass_verification_data_bytes", lib.cass_verification_data_bytes(C.byref(info), C.byref(n)))
+    return n.value
+
+
+def cass_encode_verification_data(blob, info: BlobInfo, w_bf16, vdata, stream=None):
+    _check("cass_encode_verification_data", lib.cass_encode_verification_data(
+        _ptr(blob), C.byref(info), _ptr(w_bf16), _ptr(vdata), C.c_size_t(vdata.numel() * vdata.element_size()), _stream(stream)))
+
+
+def cass_decode_full(blob, info: BlobInfo, vdata, out_bf16, stream=None):
+    _check("cass_decode_full", lib.cass_decode_full(_ptr(blob), C.byref(info), _ptr(vdata), _ptr(out_bf16), _stream(stream)))
+
+
 def cass_draft_gemv(blob, info: BlobInfo, x_bf16, partial, y_bf16, y_f32, d_status, stream=None):
     _check("cass_draft_gemv", lib.cass_draft_gemv(_ptr(blob), C.byref(info), _ptr(x_bf16), _ptr(partial), _ptr(y_bf16),
                                                   _ptr(y_f32), _ptr(d_status), _stream(stream)))

@@ -151,3 +151,33 @@ def test_full_size_down_projection(cass):
     rms = float(np.sqrt(np.mean(ref ** 2)))
     err = np.abs(y32.cpu().numpy().astype(np.float64) - ref).max()
     assert err <= 2e-2 * rms and err <= 1e-4 * rms + 1e-6, (err, rms)
+
+
+@pytest.mark.parametrize("rows,cols,p,t,seg,chunk", [(70, 688, 400, 4, 512, 128), (33, 1000, 300, 5, 256, 64),
+                                                      (40, 704, 0, 0, 0, 0), (64, 4096, 400, 4, 0, 0)])
+def test_verification_data_and_exact_reconstruction(cass, rows, cols, p, t, seg, chunk):
+    """Verification data (low mantissa bits of kept values, raw pruned values) bit-exact against the oracle's, and
+    speculation data + verification data decoded back to the original bf16 matrix bit for bit (Sec. 4.1)."""
+    w = synth.student_t_weight(rows, cols, 4, f"gpu/vd{rows}x{cols}")
+    rng = np.random.default_rng(rows + cols)
+    act = (np.abs(rng.standard_normal(cols)) + 0.05).astype(np.float32)
+    wb = _bits(w)
+    fmt = cass.default_format(w_p=p, w_t=t, seg_cols=seg, chunk_cols=chunk)
+    blob, info, _ = _encode_gpu(cass, w, act, fmt)
+    nbytes = cass.cass_verification_data_bytes(info)
+    keep = codec.keep_mask_weights(wb, act, p)
+    want = layout.encode_verification_data(wb, keep, p, t)
+    assert nbytes == want.size * 4
+    vdata = torch.full((nbytes // 4,), -1, dtype=torch.int32, device="cuda")
+    cass.cass_encode_verification_data(blob, info, w.cuda(), vdata)
+    assert np.array_equal(vdata.cpu().numpy().view(np.uint32), want)
+    full = torch.zeros(rows, cols, dtype=torch.bfloat16, device="cuda")
+    cass.cass_decode_full(blob, info, vdata, full)
+    torch.cuda.synchronize()
+    assert np.array_equal(_bits(full), wb)
+    # both parts together hold fewer bits than the bf16 matrix (the memory claim of Sec. 7.2): the exponent code saves
+    # more than the bitmap costs
+    st = cass.cass_weight_blob_stats(blob, info, torch.zeros(8, dtype=torch.uint8, device="cuda"))
+    kept = info.kept_per_row
+    content = st.bitmap_bits + st.field_bits + st.code_bits + rows * (kept * t + (cols - kept) * 16)
+    assert content < 16 * rows * cols

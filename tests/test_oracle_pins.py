@@ -402,3 +402,26 @@ def test_greedy_accept_is_eq1_special_case():
     assert model.greedy_accept([5, 6, 7], [5, 6, 7, 8]) == 3
     assert model.greedy_accept([5, 6, 7], [4, 6, 7, 8]) == 0
     assert model.greedy_accept([5, 6, 7], [5, 6, 9, 8]) == 2
+
+
+@pytest.mark.parametrize("rows,cols,p,t", [(5, 64, 400, 4), (3, 100, 333, 0), (4, 96, 0, 7), (2, 70, 999, 3)])
+def test_verification_data_restores_the_matrix_exactly(rows, cols, p, t):
+    """Sec. 4.1 / 5.1: speculation data + verification data give the original bf16 matrix back bit for bit (the target
+    model loses nothing); the verification side holds exactly t bits per kept value and 16 bits per pruned value,
+    plus less than two words of padding per row."""
+    rng = np.random.default_rng(rows * cols + t)
+    w = rng.integers(0, 1 << 16, (rows, cols)).astype(np.uint16)
+    w &= 0xBFFF                                                    # magnitudes below 2: no inf / NaN, no overflow of the scores
+    act = (np.abs(rng.standard_normal(cols)) + 0.1).astype(np.float32)
+    keep = codec.keep_mask_weights(w, act, p)
+    vdata = layout.encode_verification_data(w, keep, p, t)
+    kept = cols - codec.n_pruned(cols, p)
+    assert vdata.size == layout.VDATA_HEADER_WORDS + rows * layout.verification_row_words(cols, p, t)
+    assert layout.verification_row_words(cols, p, t) * 32 - (kept * t + (cols - kept) * 16) < 32 + 16
+    full = layout.decode_full(codec.draft_bits(w, keep, t), keep, vdata)
+    assert np.array_equal(full, w)
+    # a flipped bit in either part is seen: the two parts do not overlap
+    v2 = vdata.copy()
+    v2[layout.VDATA_HEADER_WORDS] ^= 0x80000000
+    if kept * t > 0 or cols - kept > 0:
+        assert not np.array_equal(layout.decode_full(codec.draft_bits(w, keep, t), keep, v2), w)
