@@ -129,11 +129,13 @@ int launch_draft_attn(const KvGeom& g, const KvComp& ck, const KvComp& cv, const
 int launch_verify_attn(const KvGeom& g, const uint16_t* k_cache, const uint16_t* v_cache, const uint16_t* qkv,
                        int n_seq, int rps, int n_q, const DevState* st, const AttnScratch& sc, uint16_t* out, cudaStream_t s);
 
-// Tensor-core version (verify_attn_tc.cu) for head_dim 128 and rps * (n_q / n_kv) <= 32.
+// Tensor-core version (verify_attn_tc.cu) for head_dim 128 and rps * (n_q / n_kv) <= 64.  np_cols = 32 or 64: the
+// MMA's pair columns (>= rps * group); a pair's result does not depend on it, but a session keeps one value for
+// all its decode calls.
 bool verify_attn_tc_usable(const KvGeom& g, int rps, int n_q);
 int launch_verify_attn_tc(const KvGeom& g, const uint16_t* k_cache, const uint16_t* v_cache, const uint16_t* qkv, int n_seq,
-                          int rps, int n_q, const DevState* st, const AttnScratch& sc, uint16_t* out, int32_t* d_status,
-                          cudaStream_t s);
+                          int rps, int n_q, int np_cols, const DevState* st, const AttnScratch& sc, uint16_t* out,
+                          int32_t* d_status, cudaStream_t s);
 
 // ---- verification GEMM (verify_gemm.cu): Y[r][n] = sum_k W[n][k] X[r][k], bf16 in, fp32 accumulate (tcgen05) ----
 // X is a buffer of `bn` rows of k values (bn = 16, 32 or 64 token columns of the MMA; the first `rows` are used);

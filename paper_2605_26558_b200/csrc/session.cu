@@ -429,11 +429,14 @@ extern "C" int cass_verify(void* session, const int32_t* toks, int g, int32_t* t
     const cass_model_desc& d = s->d;
     auto vparts = [&](int n, int k) { return verify_gemm_partials(s->vg_partial, n, k, bn); };
     const bool fused = rope_kv_fusable(s->kg);       // RoPE and the KV append in one kernel
-    // tensor-core attention where the shape allows.  The choice depends on the session's gamma_max only, so that plain
-    // and speculative decoding of a session run the same kernel; calls with more rows per sequence (prefill chunks) and
-    // CASS_SIMT_VERIFY_ATTN=1 use the fp32-pipe kernel.
+    // tensor-core attention where the shape allows (head_dim 128, rows x group <= 64); CASS_SIMT_VERIFY_ATTN=1 keeps
+    // the fp32-pipe kernel.  For a given model shape every decode call of a session takes the same path.
     static const bool simt_env = [] { const char* e = std::getenv("CASS_SIMT_VERIFY_ATTN"); return e && e[0] == '1'; }();
-    const bool attn_tc = !simt_env && rps <= d.gamma_max + 1 && verify_attn_tc_usable(s->kg, d.gamma_max + 1, d.n_q_heads);
+    const int grp = d.n_q_heads / d.n_kv_heads;
+    // decode calls (rps <= gamma_max + 1) are classed by gamma_max, so that plain and speculative decoding agree
+    const bool attn_tc = !simt_env && verify_attn_tc_usable(s->kg, rps <= d.gamma_max + 1 ? d.gamma_max + 1 : rps, d.n_q_heads);
+    // decode calls (rps <= gamma_max + 1) all use the column count the session's gamma_max needs; longer prefill chunks 64
+    const int np_cols = (rps <= d.gamma_max + 1 && (d.gamma_max + 1) * grp <= 32) ? 32 : 64;
     const int qd = d.n_q_heads * d.head_dim;
     RC(launch_embed(toks, 1, (const uint16_t*)s->embed, s->h, rows, d.hidden, st));
     RC(launch_rmsnorm(s->h, (const uint16_t*)s->layers[0].w.norm_attn, s->xn, rows, d.hidden, d.rms_eps, st));
@@ -454,7 +457,7 @@ extern "C" int cass_verify(void* session, const int32_t* toks, int g, int32_t* t
             RC(launch_kv_append(s->kg, L.ck, L.cv, L.kc, L.vc, s->qkv + qd, s->qkv + qd + d.n_kv_heads * d.head_dim, s->qkv_dim,
                                 -1, 0, rps, kv_flags, s->st, 0, B, st));
         }
-        if (attn_tc) RC(launch_verify_attn_tc(s->kg, L.kc, L.vc, s->qkv, B, rps, d.n_q_heads, s->st, s->asc, s->attn, status, st));
+        if (attn_tc) RC(launch_verify_attn_tc(s->kg, L.kc, L.vc, s->qkv, B, rps, d.n_q_heads, np_cols, s->st, s->asc, s->attn, status, st));
         else RC(launch_verify_attn(s->kg, L.kc, L.vc, s->qkv, B, rps, d.n_q_heads, s->st, s->asc, s->attn, st));
         if (calib) RC(launch_calib_accum(s->attn, rows, qd, L.calib[1], s->st, st));
         RC(launch_verify_gemm((const uint16_t*)L.w.wo, s->attn, rows, bn, d.hidden, qd, s->vg_partial, nullptr, nullptr, status, st));

@@ -1,26 +1,27 @@
 // Verification attention on the tensor cores (Sec. 2.2: the gamma+1 rows are verified in one pass; bf16 KV cache).
 // One CTA = one (128-token chunk, KV head, sequence).  Both products of the chunk run as tcgen05 MMAs with the
 // accumulators in tensor memory:
-//   scores^T [128 tokens x 32 pairs] = K tile [128 x d] . Q^T          (pairs = (row, query head of the group), padded)
-//   out^T    [d x 32 pairs]          = V tile^T [d x 128 tokens] . P^T  (P = chunk-local softmax numerators, bf16)
+//   scores^T [128 tokens x NP pairs] = K tile [128 x d] . Q^T          (pairs = (row, query head of the group), padded
+//   out^T    [d x NP pairs]          = V tile^T [d x 128 tokens] . P^T   to NP = 32 or 64; P = chunk-local softmax
+//                                                                        numerators, bf16)
 // K and V tiles arrive by TMA (128-byte swizzle); Q and P are written to shared memory by threads in the same
 // swizzled layout.  The V tile is used as it lies in memory (rows = tokens), i.e. as an M-contiguous A operand.
 // Chunk results (o, running maximum m, sum l) go to the split-K scratch and k_attn_merge combines the chunks, as for
 // the SIMT kernel.  A (row, head) pair is one accumulator column, so its result does not depend on the other rows.
-// Needs head_dim = 128 and rows x group <= 32; other shapes use k_verify_attn.
+// Needs head_dim = 128 and rows x group <= 64; other shapes use k_verify_attn.
 #include "tc.cuh"
 #include "kernels.cuh"
 
 namespace cass {
 
 constexpr int kVtTok = 128;            // tokens per CTA: M of the score product, K of the output product
-constexpr int kVtPairs = 32;           // N of both products
+constexpr int kVtMaxPairs = 64;        // largest N of both products (template NP = 32 or 64)
 constexpr int kVtD = 128;              // head_dim
 constexpr int kVtThreads = 192;        // warp 0: TMA; warp 1: MMA issue and tensor-memory allocation; warps 2-5: softmax, epilogue
 constexpr int kVtTileBytes = kVtTok * 64 * 2;          // one TMA box: 128 tokens x 64 dims
-constexpr int kVtQBytes = kVtPairs * 64 * 2;           // one K-block of the Q or P operand: 32 rows x 64 elements
-constexpr int kVtSmem = 4 * kVtTileBytes + 4 * kVtQBytes + kVtPairs * kVtTok * 4 + 256 + 1024;
-constexpr int kVtTmemCols = 64;        // scores^T in columns 0..31, out^T in columns 32..63
+constexpr int vt_q_bytes(int np) { return np * 64 * 2; }               // one K-block of the Q or P operand: NP rows x 64 elements
+constexpr int vt_smem(int np) { return 4 * kVtTileBytes + 4 * vt_q_bytes(np) + np * kVtTok * 4 + 256 + 1024; }
+constexpr int vt_tmem_cols(int np) { return 2 * np; }                  // scores^T in columns 0..NP-1, out^T in columns NP..2NP-1
 
 // Byte offset of element (row, col) in a K-major operand block of rows x 64 bf16 with 128-byte swizzle.
 __device__ __forceinline__ uint32_t swz_off(int row, int col) {
@@ -29,6 +30,20 @@ __device__ __forceinline__ uint32_t swz_off(int row, int col) {
 
 __device__ __forceinline__ void named_sync_128() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
+// 32 consecutive fp32 columns of this warp's 32 tensor-memory lanes: v[i] = column i of the thread's lane.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,"
+        "%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+          "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+          "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+template <int NP>
 __global__ void __launch_bounds__(kVtThreads) k_verify_attn_tc(const __grid_constant__ CUtensorMap map_k,
                                                                 const __grid_constant__ CUtensorMap map_v,
                                                                 const uint16_t* __restrict__ qkv, int rows, int n_q, int n_kv,
@@ -41,6 +56,7 @@ __global__ void __launch_bounds__(kVtThreads) k_verify_attn_tc(const __grid_cons
     const int len = st->len[seq];
     const int t0 = chunk * kVtTok;
     if (t0 >= len + rows) return;                              // no row of this call sees the chunk
+    constexpr int kVtPairs = NP, kVtQBytes = vt_q_bytes(NP), kVtTmemCols = vt_tmem_cols(NP);
     uint8_t* base = reinterpret_cast<uint8_t*>(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);
     uint8_t* sK = base;                                        // 2 boxes [128 tok][64 d]
     uint8_t* sV = sK + 2 * kVtTileBytes;                       // 2 boxes [128 tok][64 d]
@@ -117,7 +133,7 @@ __global__ void __launch_bounds__(kVtThreads) k_verify_attn_tc(const __grid_cons
                 const uint64_t ad = tc_smem_desc(sV + kk * 2048, kVtTileBytes);
                 // B: block kk / 4 of P (64 tokens each), 32 bytes per 16 tokens inside the swizzled row
                 const uint64_t bd = tc_smem_desc(sP + (kk >> 2) * kVtQBytes) + (uint64_t)((kk & 3) * 2);
-                tc_mma(tmem + 32u, ad, bd, idesc2, (uint32_t)(kk != 0));
+                tc_mma(tmem + (uint32_t)NP, ad, bd, idesc2, (uint32_t)(kk != 0));
             }
         } else if (ok) {
             atomicExch(d_status, CASS_ERR_TIMEOUT);
@@ -129,27 +145,19 @@ __global__ void __launch_bounds__(kVtThreads) k_verify_attn_tc(const __grid_cons
         const int et = q * 32 + lane;                 // this thread's token (scores) and dim (output)
         const float scale = rsqrtf((float)kVtD);
         uint32_t v[32];
-        bool have = mbar_wait_bounded(bar_s, 0);
-        if (have) {
-            __syncwarp();
-            tc_fence_after();
-            asm volatile(
-                "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,"
-                "%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-                : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
-                  "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
-                  "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
-                  "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-                : "r"(tmem + ((uint32_t)(q * 32) << 16)));
-            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-        } else {
-            atomicExch(d_status, CASS_ERR_TIMEOUT);
-        }
+        const bool have = mbar_wait_bounded(bar_s, 0);
+        if (have) { __syncwarp(); tc_fence_after(); }
+        else atomicExch(d_status, CASS_ERR_TIMEOUT);
         // scores^T -> sS[pair][token], scaled, causal: row r of the call sits at position len + r
 #pragma unroll
-        for (int p = 0; p < kVtPairs; ++p) {
-            const bool vis = have && p < P && (t0 + et) <= len + p / G;
-            sS[p * kVtTok + et] = vis ? __uint_as_float(v[p]) * scale : -INFINITY;
+        for (int c0 = 0; c0 < NP; c0 += 32) {
+            if (have) tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                const int p = c0 + i;
+                const bool vis = have && p < P && (t0 + et) <= len + p / G;
+                sS[p * kVtTok + et] = vis ? __uint_as_float(v[i]) * scale : -INFINITY;
+            }
         }
         named_sync_128();
         // chunk softmax of every pair (warp q: pairs q, q + 4, ...), numerators rounded to bf16 into the P operand
@@ -179,20 +187,16 @@ __global__ void __launch_bounds__(kVtThreads) k_verify_attn_tc(const __grid_cons
         if (mbar_wait_bounded(bar_o, 0)) {
             __syncwarp();
             tc_fence_after();
-            asm volatile(
-                "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,"
-                "%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-                : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
-                  "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
-                  "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
-                  "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-                : "r"(tmem + ((uint32_t)(q * 32) << 16) + 32u));
-            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
-            for (int p = 0; p < kVtPairs; ++p) {
-                if (p < P && t0 <= len + p / G) {
-                    const size_t pair = ((size_t)seq * rows + p / G) * n_q + head * G + p % G;
-                    sc.o[(pair * n_chunks_alloc + chunk) * kVtD + et] = __uint_as_float(v[p]);
+            for (int c0 = 0; c0 < NP; c0 += 32) {
+                tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(NP + c0), v);
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    const int p = c0 + i;
+                    if (p < P && t0 <= len + p / G) {
+                        const size_t pair = ((size_t)seq * rows + p / G) * n_q + head * G + p % G;
+                        sc.o[(pair * n_chunks_alloc + chunk) * kVtD + et] = __uint_as_float(v[i]);
+                    }
                 }
             }
         } else {
@@ -211,14 +215,15 @@ int launch_attn_merge(const AttnScratch& sc, int n_chunks_alloc, int chunk_token
                       const DevState* st, int draft_mode, uint16_t* out, cudaStream_t s);
 
 bool verify_attn_tc_usable(const KvGeom& g, int rps, int n_q) {
-    return g.d == kVtD && rps * (n_q / g.n_kv) <= kVtPairs && (g.seq_stride % 16) == 0;
+    return g.d == kVtD && rps * (n_q / g.n_kv) <= kVtMaxPairs && (g.seq_stride % 16) == 0;
 }
 
 // caches: sequence 0's bf16 K and V of one layer ([max_seq][n_kv][128]); the other sequences lie seq_stride bytes apart.
 int launch_verify_attn_tc(const KvGeom& g, const uint16_t* k_cache, const uint16_t* v_cache, const uint16_t* qkv, int n_seq,
-                          int rps, int n_q, const DevState* st, const AttnScratch& sc, uint16_t* out, int32_t* d_status,
-                          cudaStream_t s) {
-    if (!verify_attn_tc_usable(g, rps, n_q)) return CASS_ERR_UNSUPPORTED;
+                          int rps, int n_q, int np_cols, const DevState* st, const AttnScratch& sc, uint16_t* out,
+                          int32_t* d_status, cudaStream_t s) {
+    if (!verify_attn_tc_usable(g, rps, n_q) || (np_cols != 32 && np_cols != 64) || rps * (n_q / g.n_kv) > np_cols)
+        return CASS_ERR_UNSUPPORTED;
     EncodeTiledFn fn = encode_fn();
     if (!fn) return CASS_ERR_CUDA;
     CUtensorMap mk, mv;
@@ -232,14 +237,25 @@ int launch_verify_attn_tc(const KvGeom& g, const uint16_t* k_cache, const uint16
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) return CASS_ERR_INVALID_ARG;
     }
-    static bool attr = false;
-    if (!attr) {
-        CASS_CUDA_CHECK(cudaFuncSetAttribute(k_verify_attn_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kVtSmem));
-        attr = true;
-    }
     const int n_chunks = ceil_div(g.max_seq, kVtTok);
     dim3 grid(n_chunks, g.n_kv, n_seq);
-    CASS_PDL_LAUNCH(k_verify_attn_tc, grid, dim3(kVtThreads), (size_t)kVtSmem, s, mk, mv, qkv, rps, n_q, g.n_kv, st, sc, n_chunks, d_status);
+    if (np_cols == 32) {
+        static bool attr = false;
+        if (!attr) {
+            CASS_CUDA_CHECK(cudaFuncSetAttribute(k_verify_attn_tc<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, vt_smem(32)));
+            attr = true;
+        }
+        CASS_PDL_LAUNCH(k_verify_attn_tc<32>, grid, dim3(kVtThreads), (size_t)vt_smem(32), s, mk, mv, qkv, rps, n_q, g.n_kv, st, sc,
+                        n_chunks, d_status);
+    } else {
+        static bool attr = false;
+        if (!attr) {
+            CASS_CUDA_CHECK(cudaFuncSetAttribute(k_verify_attn_tc<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, vt_smem(64)));
+            attr = true;
+        }
+        CASS_PDL_LAUNCH(k_verify_attn_tc<64>, grid, dim3(kVtThreads), (size_t)vt_smem(64), s, mk, mv, qkv, rps, n_q, g.n_kv, st, sc,
+                        n_chunks, d_status);
+    }
     return launch_attn_merge(sc, n_chunks, kVtTok, n_seq * rps, rps, n_q, g.d, st, 0, out, s);
 }
 

@@ -105,9 +105,10 @@ def test_draft_attention_llama_layer_shape(cass, n_pos, n_q):
     eng.close()
 
 
-@pytest.mark.parametrize("n_pos,g,n_q", [(3, 4, 32), (127, 0, 32), (128, 4, 32), (300, 7, 32), (4096, 4, 32), (200, 3, 64)])
+@pytest.mark.parametrize("n_pos,g,n_q", [(3, 4, 32), (127, 0, 32), (128, 4, 32), (300, 7, 32), (4096, 4, 32), (200, 3, 64),
+                                         (100, 8, 32), (300, 15, 32), (70, 7, 64)])
 def test_verify_attention_llama_head_geometry(cass, n_pos, g, n_q):
-    """Verification attention with heads of 128 (the tensor-core kernel where rows x group <= 32): g+1 new rows over
+    """Verification attention with heads of 128 (the tensor-core kernel, 32 or 64 pair columns): g+1 new rows over
     n_pos cached positions of synthetic KV, against the oracle's causal softmax(q K^T / sqrt(d)) V computed in fp64 from
     the rotated q rows and the bf16 caches the call leaves behind."""
     from paper_2605_26558_b200 import engine
