@@ -208,7 +208,7 @@ def step_breakdown(gamma=4, n_prompt=512, steps=3, batch=1):
     return [{"kernel": "step_breakdown", "gamma": gamma, "batch": batch, "kernel_us_per_step": tot / steps}] + rows
 
 
-def long_decode(gamma=4, n_tokens=8192, n_prompt=512, config="llama8b"):
+def long_decode(gamma=4, n_tokens=8192, n_prompt=512, config="llama8b", batch=1):
     """Decodes n_tokens greedy tokens after the prompt twice on the full model -- plain bf16 greedy (gamma = 0) and
     speculatively -- with CUDA-graph steps, compares the two streams token by token and reports tokens/s of both,
     overall and over the first and last 10 % of the speculative steps (the context grows from n_prompt to
@@ -223,8 +223,8 @@ def long_decode(gamma=4, n_tokens=8192, n_prompt=512, config="llama8b"):
           "norm_final": wt["norm_final"]}
     del wt
     max_seq = (n_prompt + n_tokens + 2 * (gamma + 1) + 32 + 255) // 256 * 256
-    eng = engine.Engine(shape, gw, max_seq=max_seq, gamma_max=max(gamma, 1))
-    eng.prefill(synth.random_prompt(n_prompt, shape.vocab, 0), calibrate=True)
+    eng = engine.Engine(shape, gw, max_seq=max_seq, gamma_max=max(gamma, 1), batch=batch)
+    eng.prefill(torch.stack([synth.random_prompt(n_prompt, shape.vocab, b) for b in range(batch)]), calibrate=True)
     eng.encode_weights(eng.calib_norms())
     eng.build_kv_codebook()
     first = eng.next_tokens()
@@ -233,14 +233,14 @@ def long_decode(gamma=4, n_tokens=8192, n_prompt=512, config="llama8b"):
         eng.generate(0, g, use_graph=True)            # lays the token buffers out for this gamma and captures the step
         B.cass_set_len(eng.session, n_prompt)
         eng.set_next_tokens(first)
-        out, marks = [], []
+        out, marks = [[] for _ in range(batch)], []
         stats = engine.StepStats()
         torch.cuda.synchronize()
         t0 = time.perf_counter()
-        while len(out) < n_tokens:
+        while min(len(o) for o in out) < n_tokens:
             eng._graphs[g].replay()
-            eng._collect([out], stats)
-            marks.append((time.perf_counter() - t0, len(out)))
+            eng._collect(out, stats)
+            marks.append((time.perf_counter() - t0, sum(len(o) for o in out)))
         return out, stats, marks
 
     def tail_rate(m):
@@ -249,14 +249,16 @@ def long_decode(gamma=4, n_tokens=8192, n_prompt=512, config="llama8b"):
 
     plain, _, pm = timed(0)
     spec, st, sm = timed(gamma)
-    n = min(len(plain), len(spec), n_tokens)
+    n = min(min(len(o) for o in plain), min(len(o) for o in spec), n_tokens)
     k = max(1, len(sm) // 10)
     status, ln = eng.status()
+    lens = eng.lens()
     eng.close()
-    return [{"kernel": "long_decode", "config": config, "gamma": gamma, "prompt": n_prompt, "tokens": n,
-             "streams_identical": spec[:n] == plain[:n], "final_len": ln, "status": status,
+    return [{"kernel": "long_decode", "config": config, "gamma": gamma, "batch": batch, "prompt": n_prompt, "tokens": n,
+             "streams_identical": all(spec[b][:n] == plain[b][:n] for b in range(batch)), "final_len": ln, "final_lens": lens,
+             "status": status,
              "spec_tokens_per_s": sm[-1][1] / sm[-1][0], "spec_tokens_per_s_first_10pct": sm[k - 1][1] / sm[k - 1][0],
-             "spec_tokens_per_s_last_10pct": tail_rate(sm), "steps": st.steps, "mean_accepted": st.mean_accepted,
+             "spec_tokens_per_s_last_10pct": tail_rate(sm), "steps": st.steps, "mean_accepted": st.mean_accepted / batch,
              "plain_tokens_per_s": pm[-1][1] / pm[-1][0], "plain_tokens_per_s_last_10pct": tail_rate(pm)}]
 
 
@@ -291,7 +293,7 @@ def main():
             copies = args.copies or max(2, int(300e6 / (n * k * 2)) + 1)
             out.append(bench_verify_gemm(name, copies, args.iters))
     if args.kernel == "decode":
-        out.extend(long_decode(args.gamma, args.tokens, args.prompt, args.config))
+        out.extend(long_decode(args.gamma, args.tokens, args.prompt, args.config, args.batch))
     if args.kernel == "step":
         out.extend(step_breakdown(gamma=args.gamma, batch=args.batch))
     if args.kernel in ("attn", "all"):
