@@ -20,7 +20,11 @@ constexpr int kVtD = 128;              // head_dim
 constexpr int kVtThreads = 192;        // warp 0: TMA; warp 1: MMA issue and tensor-memory allocation; warps 2-5: softmax, epilogue
 constexpr int kVtTileBytes = kVtTok * 64 * 2;          // one TMA box: 128 tokens x 64 dims
 constexpr int vt_q_bytes(int np) { return np * 64 * 2; }               // one K-block of the Q or P operand: NP rows x 64 elements
-constexpr int vt_smem(int np) { return 4 * kVtTileBytes + 4 * vt_q_bytes(np) + np * kVtTok * 4 + 256 + 1024; }
+// K tiles (32 KB) | V tiles (32 KB) | Q (2 blocks) | [P (2 blocks) when np = 64] | barriers.  The scores (np x 128
+// floats) reuse the K tiles' memory, and with np = 32 so does P: both are written only after the first product has
+// finished reading K.
+constexpr int vt_smem(int np) { return 4 * kVtTileBytes + (np == 32 ? 2 : 4) * vt_q_bytes(np) + 256 + 1024; }
+static_assert(32 * kVtTok * 4 + 2 * vt_q_bytes(32) <= 2 * kVtTileBytes && 64 * kVtTok * 4 <= 2 * kVtTileBytes, "scores (and P) fit the K tiles");
 constexpr int vt_tmem_cols(int np) { return 2 * np; }                  // scores^T in columns 0..NP-1, out^T in columns NP..2NP-1
 
 // Byte offset of element (row, col) in a K-major operand block of rows x 64 bf16 with 128-byte swizzle.
@@ -60,10 +64,10 @@ __global__ void __launch_bounds__(kVtThreads) k_verify_attn_tc(const __grid_cons
     uint8_t* base = reinterpret_cast<uint8_t*>(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);
     uint8_t* sK = base;                                        // 2 boxes [128 tok][64 d]
     uint8_t* sV = sK + 2 * kVtTileBytes;                       // 2 boxes [128 tok][64 d]
-    uint8_t* sQ = sV + 2 * kVtTileBytes;                       // 2 blocks [32 pairs][64 d]
-    uint8_t* sP = sQ + 2 * kVtQBytes;                          // 2 blocks [32 pairs][64 tok]
-    float* sS = reinterpret_cast<float*>(sP + 2 * kVtQBytes);  // [32 pairs][128 tok] scores, then probabilities
-    uint64_t* bar_k = reinterpret_cast<uint64_t*>(sS + kVtPairs * kVtTok);
+    uint8_t* sQ = sV + 2 * kVtTileBytes;                       // 2 blocks [NP pairs][64 d]
+    float* sS = reinterpret_cast<float*>(sK);                  // [NP pairs][128 tok] scores: over the K tiles, once consumed
+    uint8_t* sP = NP == 32 ? sK + NP * kVtTok * 4 : sQ + 2 * kVtQBytes;      // 2 blocks [NP pairs][64 tok], 1024-aligned
+    uint64_t* bar_k = reinterpret_cast<uint64_t*>(sQ + (NP == 32 ? 2 : 4) * kVtQBytes);
     uint64_t* bar_v = bar_k + 1;
     uint64_t* bar_s = bar_k + 2;       // scores complete in tensor memory
     uint64_t* bar_p = bar_k + 3;       // P written to shared memory (128 arrivals)
