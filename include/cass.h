@@ -1,10 +1,11 @@
 /*
  * cass.h -- C boundary of the B200-native Cassandra self-speculative decode step.
  *
- * One draft pass reads only the speculation data (pruned, mantissa-truncated, unary-exponent-coded
- * weights and KV cache; Sec. 4.1-4.2 of the paper), decodes it in registers and runs batch-1 GEMV and
- * grouped-query decode attention on it; a bf16 verification pass over the gamma+1 drafted rows and a
- * greedy accept/rollback close each step (Sec. 2.2).
+ * One draft pass reads only the speculation data (pruned, mantissa-truncated weights and KV cache with
+ * compressed exponents: unary-coded, or MX-shared for the weights; Sec. 4.1-4.2 of the paper), decodes it in
+ * registers and runs low-batch (1 to 8 sequences) GEMV and grouped-query decode attention on it; a bf16
+ * verification pass over the gamma+1 drafted rows of every sequence (tensor cores) and a greedy accept/rollback
+ * per sequence close each step (Sec. 2.2).
  *
  * Conventions
  *   - Every entry point returns 0 (CASS_OK) or a negative CASS_ERR_* code; nothing throws.
