@@ -122,7 +122,7 @@ __device__ __forceinline__ uint32_t lanemask_lt() {
     return m;
 }
 
-// ---- mbarrier + bulk async copy (TMA, no multicast) --------------------------------------------------
+// ---- mbarrier + bulk async copy (TMA, one destination CTA) --------------------------------------------------
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
