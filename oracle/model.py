@@ -113,63 +113,99 @@ class KVCache:
         self.n = 0                           # committed length
 
 
-def forward_token(W: Weights, kv: KVCache, tok: int, pos: int, draft: bool, kv_p: int, kv_t: int,
-                  calib: dict | None = None):
-    """One token at position `pos`.  Target mode writes K/V in both forms at `pos`; draft mode
-    writes only the draft view.  Returns the fp64 logits."""
-    s = W.shape
+def attention(q_bits: np.ndarray, k_bits: np.ndarray, v_bits: np.ndarray) -> np.ndarray:
+    """Grouped-query softmax attention of one query position over the visible positions (Sec. 2.1).
+
+    q [n_q, d], k and v [n_pos, n_kv, d] as bf16 bit patterns (every position in k/v is visible: the caller
+    passes the causal range).  Query head hq reads KV head hq // (n_q / n_kv); scores are q.k / sqrt(d);
+    returns the unrounded output [n_q, d] in the accumulation type."""
+    qf, kc, vc = _f(q_bits), _f(k_bits), _f(v_bits)
+    n_q, d = qf.shape
+    g = n_q // kc.shape[1]
+    o = np.zeros((n_q, d), dtype=_ACC)
+    for hq in range(n_q):
+        hk = hq // g
+        sc = (kc[:, hk, :] @ qf[hq]) / _ACC(np.sqrt(float(d)))
+        sc = sc - sc.max()
+        pr = np.exp(sc)
+        pr = pr / pr.sum()
+        o[hq] = pr @ vc[:, hk, :]
+    return o
+
+
+def swiglu(gate_bits: np.ndarray, up_bits: np.ndarray) -> np.ndarray:
+    """SwiGLU activation silu(gate) * up = gate / (1 + exp(-gate)) * up on bf16 inputs, rounded to bf16."""
+    gate, up = _f(gate_bits), _f(up_bits)
+    return _r(gate / (_ACC(1.0) + np.exp(-gate)) * up)
+
+
+def layer(lw: dict, shape, h_bits: np.ndarray, pos: int, k_cache: np.ndarray, v_cache: np.ndarray,
+          kd_cache: np.ndarray, vd_cache: np.ndarray, draft: bool, kv_p: int, kv_t: int, note=None) -> np.ndarray:
+    """One decoder layer for the token at `pos` (pre-norm residual blocks: attention, then SwiGLU FFN).
+
+    lw: the layer's matrices (accumulation type) and norm gains (bf16 bits); h_bits: bf16 hidden state;
+    k_cache/v_cache [max_seq, n_kv, d]: the target's bf16 cache of this layer, kd_cache/vd_cache: the draft's view.
+    The draft view of the new K/V is written at `pos` in both modes, the bf16 cache only in target mode.
+    `note(names, x_bits)` sees the input of each projection (Wanda calibration).  Returns the new hidden state."""
+    s = shape
     d = s.head_dim
-    g = s.n_q_heads // s.n_kv_heads
-    h = W.embed_bits[tok].copy()
+    xn = rmsnorm(h_bits, lw["norm_attn"], s.rms_eps)
+    if note:
+        note(("wq", "wk", "wv"), xn)
+    x = _f(xn)
+    q = _r(lw["wq"] @ x).reshape(s.n_q_heads, d)
+    k = _r(lw["wk"] @ x).reshape(s.n_kv_heads, d)
+    v = _r(lw["wv"] @ x).reshape(s.n_kv_heads, d)
+    q = rope(q, pos, s.rope_theta)
+    k = rope(k, pos, s.rope_theta)
+    kd_cache[pos] = codec.draft_bits(k, codec.keep_mask_kv(k, kv_p), kv_t)
+    vd_cache[pos] = codec.draft_bits(v, codec.keep_mask_kv(v, kv_p), kv_t)
+    if not draft:
+        k_cache[pos], v_cache[pos] = k, v
+    o = attention(q, (kd_cache if draft else k_cache)[: pos + 1], (vd_cache if draft else v_cache)[: pos + 1])
+    ob = _r(o.reshape(-1))
+    if note:
+        note(("wo",), ob)
+    attn = _r(lw["wo"] @ _f(ob))
+    h = _r(_f(h_bits) + _f(attn))
+    xn = rmsnorm(h, lw["norm_ffn"], s.rms_eps)
+    if note:
+        note(("wg", "wu"), xn)
+    x = _f(xn)
+    act = swiglu(_r(lw["wg"] @ x), _r(lw["wu"] @ x))
+    if note:
+        note(("wd",), act)
+    down = _r(lw["wd"] @ _f(act))
+    return _r(_f(h) + _f(down))
 
-    def note(li, names, x_bits):
-        if calib is not None:
-            x = _f(x_bits)
-            for nm in names:
-                calib["layers"][li][nm] += x * x
 
-    for li, lw in enumerate(W.layers):
-        xn = rmsnorm(h, lw["norm_attn"], s.rms_eps)
-        note(li, ("wq", "wk", "wv"), xn)
-        x = _f(xn)
-        q = _r(lw["wq"] @ x).reshape(s.n_q_heads, d)
-        k = _r(lw["wk"] @ x).reshape(s.n_kv_heads, d)
-        v = _r(lw["wv"] @ x).reshape(s.n_kv_heads, d)
-        q = rope(q, pos, s.rope_theta)
-        k = rope(k, pos, s.rope_theta)
-        kd = codec.draft_bits(k, codec.keep_mask_kv(k, kv_p), kv_t)
-        vd = codec.draft_bits(v, codec.keep_mask_kv(v, kv_p), kv_t)
-        kv.kd[li, pos], kv.vd[li, pos] = kd, vd
-        if not draft:
-            kv.k[li, pos], kv.v[li, pos] = k, v
-        kc = _f((kv.kd if draft else kv.k)[li, : pos + 1])          # [pos+1, n_kv, d]
-        vc = _f((kv.vd if draft else kv.v)[li, : pos + 1])
-        qf = _f(q)
-        o = np.zeros((s.n_q_heads, d), dtype=_ACC)
-        for hq in range(s.n_q_heads):
-            hk = hq // g
-            sc = (kc[:, hk, :] @ qf[hq]) / _ACC(np.sqrt(float(d)))
-            sc = sc - sc.max()
-            pr = np.exp(sc)
-            pr = pr / pr.sum()
-            o[hq] = pr @ vc[:, hk, :]
-        ob = _r(o.reshape(-1))
-        note(li, ("wo",), ob)
-        attn = _r(lw["wo"] @ _f(ob))
-        h = _r(_f(h) + _f(attn))
-        xn = rmsnorm(h, lw["norm_ffn"], s.rms_eps)
-        note(li, ("wg", "wu"), xn)
-        x = _f(xn)
-        gate = _f(_r(lw["wg"] @ x))
-        up = _f(_r(lw["wu"] @ x))
-        act = _r(gate / (_ACC(1.0) + np.exp(-gate)) * up)
-        note(li, ("wd",), act)
-        down = _r(lw["wd"] @ _f(act))
-        h = _r(_f(h) + _f(down))
-    xn = rmsnorm(h, W.norm_final, s.rms_eps)
+def lm_logits(W: Weights, h_bits: np.ndarray, calib: dict | None = None) -> np.ndarray:
+    """Final RMSNorm and the output projection; logits stay in the accumulation type."""
+    xn = rmsnorm(h_bits, W.norm_final, W.shape.rms_eps)
     if calib is not None:
         calib["lm_head"] += _f(xn) ** 2
     return W.lm_head @ _f(xn)
+
+
+def forward_token(W: Weights, kv: KVCache, tok: int, pos: int, draft: bool, kv_p: int, kv_t: int,
+                  calib: dict | None = None, hidden_out: list | None = None):
+    """One token at position `pos`.  Target mode writes K/V in both forms at `pos`; draft mode
+    writes only the draft view.  Returns the fp64 logits.  `hidden_out`, when given, receives the bf16 hidden
+    state entering every layer and the one entering the final norm."""
+    h = W.embed_bits[tok].copy()
+    for li, lw in enumerate(W.layers):
+        if hidden_out is not None:
+            hidden_out.append(h.copy())
+        note = None
+        if calib is not None:
+            def note(names, x_bits, li=li):
+                x = _f(x_bits)
+                for nm in names:
+                    calib["layers"][li][nm] += x * x
+        h = layer(lw, W.shape, h, pos, kv.k[li], kv.v[li], kv.kd[li], kv.vd[li], draft, kv_p, kv_t, note)
+    if hidden_out is not None:
+        hidden_out.append(h.copy())
+    return lm_logits(W, h, calib)
 
 
 def new_calib(shape) -> dict:

@@ -134,10 +134,12 @@ class Engine:
         for l, lw in enumerate(self.w["layers"]):
             d = {}
             for nm in ("wqkv", "wo", "wgu", "wd"):
-                a = None if norms is None else norms["layers"][l][nm].to(self.device, torch.float32).contiguous()
+                a = None if norms is None or norms["layers"][l].get(nm) is None else \
+                    norms["layers"][l][nm].to(self.device, torch.float32).contiguous()
                 d[nm], blobs["infos"][(l, nm)] = enc(lw[nm], a)
             blobs["layers"].append(d)
-        a = None if norms is None else norms["lm_head"].to(self.device, torch.float32).contiguous()
+        a = None if norms is None or norms.get("lm_head") is None else \
+            norms["lm_head"].to(self.device, torch.float32).contiguous()
         blobs["lm_head"], blobs["infos"]["lm_head"] = enc(self.w["lm_head"], a)
         if int(status.item()) != 0:
             raise B.CassError("cass_encode_weights(status)", int(status.item()))

@@ -4,7 +4,7 @@ import pytest
 import torch
 
 import synth
-from oracle import codec, layout
+from oracle import codec, layout, model
 
 pytestmark = pytest.mark.gpu
 TOL = 2e-2
@@ -87,14 +87,9 @@ def test_draft_attention_llama_layer_shape(cass, n_pos, n_q):
     torch.cuda.synchronize()
     assert eng.status()[0] == 0
     kb, vb = _bits(k), _bits(v)
-    kd = codec.bf16_bits_to_f64(codec.draft_bits(kb, codec.keep_mask_kv(kb, 400), 4))
-    vd = codec.bf16_bits_to_f64(codec.draft_bits(vb, codec.keep_mask_kv(vb, 400), 4))
-    qf = codec.bf16_bits_to_f64(_bits(q))
-    want = np.zeros((n_q, 128))
-    for hq in range(n_q):
-        sc = kd[:, hq // G, :] @ qf[hq] / np.sqrt(128.0)
-        p = np.exp(sc - sc.max())
-        want[hq] = (p / p.sum()) @ vd[:, hq // G, :]
+    kd = codec.draft_bits(kb, codec.keep_mask_kv(kb, 400), 4)
+    vd = codec.draft_bits(vb, codec.keep_mask_kv(vb, 400), 4)
+    want = model.attention(_bits(q), kd, vd)                 # the oracle's own attention, pinned on the CPU
     got = codec.bf16_bits_to_f64(_bits(out))
     rms = float(np.sqrt(np.mean(want ** 2)))
     # The output is rounded to bf16, so each element may be off by half an ulp (<= 2^-8 |value|) on top of the
@@ -129,25 +124,21 @@ def test_verify_attention_llama_head_geometry(cass, n_pos, g, n_q):
     base = eng.mem.data_ptr()
     m16 = eng.mem.view(torch.bfloat16)
 
-    def grab(which):
+    def grab_bits(which):
         p, r, c = cass.cass_debug_activation(eng.session, which)
         off = (p - base) // 2
-        return m16[off: off + rows * c].view(rows, c).float().cpu().numpy().astype(np.float64)
+        return _bits(m16[off: off + rows * c].view(rows, c))
 
-    qkv, got = grab(2), grab(1)
+    qbits, got = grab_bits(2), codec.bf16_bits_to_f64(grab_bits(1))
     kc = cass.cass_kv_query(eng.session, 0, 0, 0).k_or_v_bf16
     vc = cass.cass_kv_query(eng.session, 0, 1, 0).k_or_v_bf16
     n_all = n_pos + rows
-    kd = m16[(kc - base) // 2: (kc - base) // 2 + n_all * 1024].view(n_all, 8, 128).float().cpu().numpy().astype(np.float64)
-    vd = m16[(vc - base) // 2: (vc - base) // 2 + n_all * 1024].view(n_all, 8, 128).float().cpu().numpy().astype(np.float64)
+    kd = _bits(m16[(kc - base) // 2: (kc - base) // 2 + n_all * 1024].view(n_all, 8, 128))
+    vd = _bits(m16[(vc - base) // 2: (vc - base) // 2 + n_all * 1024].view(n_all, 8, 128))
     want = np.zeros((rows, n_q * 128))
-    for r in range(rows):
+    for r in range(rows):                                    # causal: row r sees the cache and the new rows up to itself
         vis = n_pos + r + 1
-        for hq in range(n_q):
-            q = qkv[r, hq * 128: (hq + 1) * 128]
-            sc = kd[:vis, hq // G, :] @ q / np.sqrt(128.0)
-            p = np.exp(sc - sc.max())
-            want[r, hq * 128: (hq + 1) * 128] = (p / p.sum()) @ vd[:vis, hq // G, :]
+        want[r] = model.attention(qbits[r, : n_q * 128].reshape(n_q, 128), kd[:vis], vd[:vis]).reshape(-1)
     rms = float(np.sqrt(np.mean(want ** 2)))
     err = np.abs(got - want)
     assert np.all(err <= 2.0 ** -7 * np.abs(want) + TOL * rms), float(err.max() / rms)

@@ -1,0 +1,216 @@
+"""Teacher-forced per-layer parity of the step-level entry points against the oracle (Sec. 2.1 architecture, Sec. 4.1
+draft = the same graph on the zero-padded speculation data).
+
+Layer l of the oracle's model is run on the GPU as a ONE-layer session whose embedding table holds, row by row, the
+oracle's own bf16 inputs of layer l (prompt positions, forced draft steps, verification rows), so the layer sees
+exactly the oracle's input and only that layer's arithmetic is compared: its output hidden state must lie within
+2e-2 of the output's RMS at every element, outright.  A session whose output projections are zero passes its input
+through unchanged; it compares the final norm + lm_head logits given the oracle's final hidden state.
+"""
+import numpy as np
+import pytest
+import torch
+
+import synth
+from oracle import codec, model
+
+pytestmark = pytest.mark.gpu
+TOL = 2e-2
+
+
+def _bits(t: torch.Tensor) -> np.ndarray:
+    return t.detach().cpu().contiguous().view(torch.int16).numpy().astype(np.uint16)
+
+
+def _from_bits(bits: np.ndarray) -> torch.Tensor:
+    return torch.from_numpy(np.ascontiguousarray(bits).astype(np.uint16).view(np.int16)).view(torch.bfloat16)
+
+
+@pytest.fixture(scope="module")
+def cass():
+    import paper_2605_26558_b200 as m
+    from paper_2605_26558_b200 import engine
+    m.engine = engine
+    return m
+
+
+def _oracle_trace(shape, wt, prompt, forced, p=400, t=4):
+    """Runs the oracle over the prompt, `len(forced) - 1` forced draft steps and the verification of the forced rows.
+    Returns the bf16 hidden state entering every layer (and the final norm) for each of those tokens, the logits,
+    and the calibration norms."""
+    wb = {"layers": [{k: _bits(v) for k, v in lw.items()} for lw in wt["layers"]],
+          "embed": _bits(wt["embed"]), "lm_head": _bits(wt["lm_head"]), "norm_final": _bits(wt["norm_final"])}
+    W = model.Weights(shape, wb)
+    n = len(prompt)
+    kv = model.KVCache(shape, n + len(forced) + 4)
+    calib = model.new_calib(shape)
+    pre_h, pre_logits = [], []
+    for pos, tok in enumerate(prompt):
+        hs = []
+        pre_logits.append(model.forward_token(W, kv, int(tok), pos, False, p, t, calib, hidden_out=hs))
+        pre_h.append(hs)
+    kv.n = n
+    norms = model.calib_to_norms(calib)
+    Wd = model.Weights(shape, model.draft_weight_bits(wb, norms, p, t))
+    dr_h, dr_logits = [], []
+    for i, tok in enumerate(forced[:-1]):
+        hs = []
+        dr_logits.append(model.forward_token(Wd, kv, tok, n + i, True, p, t, hidden_out=hs))
+        dr_h.append(hs)
+    ve_h, ve_logits = [], []
+    for i, tok in enumerate(forced):
+        hs = []
+        ve_logits.append(model.forward_token(W, kv, tok, n + i, False, p, t, hidden_out=hs))
+        ve_h.append(hs)
+    return dict(wb=wb, norms=norms, pre_h=pre_h, dr_h=dr_h, ve_h=ve_h, pre_logits=pre_logits, dr_logits=dr_logits,
+                ve_logits=ve_logits)
+
+
+def _layer_session(cass, shape, lw, rows_bits, lm_head, norm_final, norms_l, norms_lm, n_prompt, max_seq):
+    """One-layer session: layer weights lw (torch bf16, CPU), embedding rows = rows_bits."""
+    one = synth.ModelShape(n_layers=1, hidden=shape.hidden, n_q_heads=shape.n_q_heads, n_kv_heads=shape.n_kv_heads,
+                           head_dim=shape.head_dim, ffn=shape.ffn, vocab=lm_head.shape[0],
+                           rope_theta=shape.rope_theta, rms_eps=shape.rms_eps)
+    embed = torch.zeros(one.vocab, shape.hidden, dtype=torch.bfloat16)
+    embed[: rows_bits.shape[0]] = _from_bits(rows_bits)
+    gw = {"layers": [cass.engine.fuse_layer_weights({k: v.cuda() for k, v in lw.items()})], "embed": embed.cuda(),
+          "lm_head": lm_head.cuda(), "norm_final": norm_final.cuda()}
+    eng = cass.engine.Engine(one, gw, max_seq=max_seq, gamma_max=8)
+    eng.prefill(torch.arange(n_prompt, dtype=torch.int32))
+    fused = {"layers": [{"wqkv": torch.from_numpy(norms_l["wq"]), "wo": torch.from_numpy(norms_l["wo"]),
+                         "wgu": torch.from_numpy(norms_l["wg"]), "wd": torch.from_numpy(norms_l["wd"])}],
+             "lm_head": torch.from_numpy(norms_lm)}
+    eng.encode_weights(fused)
+    eng.build_kv_codebook()
+    return eng
+
+
+def _hidden(cass, eng, rows):
+    p, r, c = cass.cass_debug_activation(eng.session, 0)
+    off = (p - eng.mem.data_ptr()) // 2
+    return codec.bf16_bits_to_f64(_bits(eng.mem.view(torch.bfloat16)[off: off + rows * c].view(rows, c)))
+
+
+def _assert_close(got, want_bits, what):
+    """Every element within TOL of the RMS of the oracle's vector, outright."""
+    want = codec.bf16_bits_to_f64(want_bits)
+    rms = float(np.sqrt(np.mean(want ** 2)))
+    err = float(np.abs(got - want).max())
+    assert err <= TOL * rms, (what, err / rms)
+    return err / rms
+
+
+def _run_layer(cass, shape, wt, tr, li, prompt, forced):
+    """Layer li teacher-forced: prefill chunks, forced draft steps, verification rows."""
+    n, g = len(prompt), len(forced) - 1
+    rows_bits = np.stack([tr["pre_h"][pos][li] for pos in range(n)] + [tr["dr_h"][i][li] for i in range(g)] +
+                         [tr["ve_h"][i][li] for i in range(g + 1)])
+    vocab = max(256, (rows_bits.shape[0] + 255) // 256 * 256)
+    lm = synth.student_t_weight(vocab, shape.hidden, 11, "lp/lm")
+    eng = _layer_session(cass, shape, wt["layers"][li], rows_bits, lm, wt["norm_final"], tr["norms"]["layers"][li],
+                         tr["norms"]["lm_head"], n, n + 64)
+    worst = 0.0
+    # the last prefill chunk is still in the activation buffer
+    chunk = 16
+    last0 = (n - 1) // chunk * chunk
+    got = _hidden(cass, eng, n - last0)
+    for r in range(n - last0):
+        worst = max(worst, _assert_close(got[r], tr["pre_h"][last0 + r][li + 1], ("prefill", li, last0 + r)))
+    scratch = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for i in range(g):
+        tok = torch.tensor([n + i], dtype=torch.int32, device="cuda")
+        cass.cass_draft_step(eng.session, tok, scratch)
+        worst = max(worst, _assert_close(_hidden(cass, eng, 1)[0], tr["dr_h"][i][li + 1], ("draft", li, i)))
+    toks = torch.arange(n + g, n + 2 * g + 1, dtype=torch.int32, device="cuda")
+    cass.cass_verify(eng.session, toks, g, eng.targ)
+    got = _hidden(cass, eng, g + 1)
+    for i in range(g + 1):
+        worst = max(worst, _assert_close(got[i], tr["ve_h"][i][li + 1], ("verify", li, i)))
+    assert eng.status()[0] == 0
+    eng.close()
+    return worst
+
+
+def _run_logits(cass, shape, wt, tr, prompt, forced):
+    """Final norm + output projection given the oracle's final hidden states (a layer with zero wo / wd is the identity)."""
+    n, g, L = len(prompt), len(forced) - 1, shape.n_layers
+    n_pre = 16
+    rows_bits = np.stack([tr["pre_h"][pos][L] for pos in range(n - n_pre, n)] + [tr["dr_h"][i][L] for i in range(g)] +
+                         [tr["ve_h"][i][L] for i in range(g + 1)])
+    lw = {k: v.clone() for k, v in wt["layers"][0].items()}
+    lw["wo"].zero_()
+    lw["wd"].zero_()
+    one = synth.ModelShape(n_layers=1, hidden=shape.hidden, n_q_heads=shape.n_q_heads, n_kv_heads=shape.n_kv_heads,
+                           head_dim=shape.head_dim, ffn=shape.ffn, vocab=shape.vocab, rope_theta=shape.rope_theta,
+                           rms_eps=shape.rms_eps)
+    embed = torch.zeros(one.vocab, shape.hidden, dtype=torch.bfloat16)
+    embed[: rows_bits.shape[0]] = _from_bits(rows_bits)
+    gw = {"layers": [cass.engine.fuse_layer_weights({k: v.cuda() for k, v in lw.items()})], "embed": embed.cuda(),
+          "lm_head": wt["lm_head"].cuda(), "norm_final": wt["norm_final"].cuda()}
+    eng = cass.engine.Engine(one, gw, max_seq=96, gamma_max=8)
+    eng.prefill(torch.arange(n_pre, dtype=torch.int32))
+    # the layer's own matrices play no part in the result (their outputs are multiplied by zero); lm_head is encoded
+    # with the oracle's calibration norms so that the draft logits use the oracle's speculation data
+    eng.encode_weights({"layers": [{"wqkv": None, "wo": None, "wgu": None, "wd": None}],
+                        "lm_head": torch.from_numpy(tr["norms"]["lm_head"])})
+    eng.build_kv_codebook()
+    logits = torch.zeros(shape.vocab, dtype=torch.float32, device="cuda")
+    scratch = torch.zeros(1, dtype=torch.int32, device="cuda")
+    worst = 0.0
+
+    def close(got, want, what):
+        rms = float(np.sqrt(np.mean(want ** 2)))
+        err = float(np.abs(got.astype(np.float64) - want).max())
+        assert err <= TOL * rms, (what, err / rms)
+        return err / rms
+
+    for i in range(g):
+        tok = torch.tensor([n_pre + i], dtype=torch.int32, device="cuda")
+        cass.cass_draft_step(eng.session, tok, scratch, logits)
+        worst = max(worst, close(logits.cpu().numpy(), tr["dr_logits"][i], ("draft logits", i)))
+    vlog = torch.zeros(g + 1, shape.vocab, dtype=torch.float32, device="cuda")
+    toks = torch.arange(n_pre + g, n_pre + 2 * g + 1, dtype=torch.int32, device="cuda")
+    cass.cass_verify(eng.session, toks, g, eng.targ, vlog)
+    got = vlog.cpu().numpy()
+    for i in range(g + 1):
+        worst = max(worst, close(got[i], tr["ve_logits"][i], ("verify logits", i)))
+    assert eng.status()[0] == 0
+    eng.close()
+    return worst
+
+
+def test_tiny_model_every_layer_and_the_logits(cass):
+    """Config 1 (2 layers, hidden 256, 4 q / 2 kv heads of 64, FFN 688, vocab 1024): prompt of 64, gamma = 4."""
+    shape = synth.TINY
+    wt = synth.model_weights(shape, 0)
+    prompt = synth.random_prompt(64, shape.vocab, 0).numpy()
+    forced = [int(t) for t in (901, 17, 333, 5, 640)]
+    tr = _oracle_trace(shape, wt, prompt, forced)
+    for li in range(shape.n_layers):
+        _run_layer(cass, shape, wt, tr, li, prompt, forced)
+    _run_logits(cass, shape, wt, tr, prompt, forced)
+
+
+def test_five_query_heads_per_kv_head_layers(cass):
+    """The Qwen-style grouping (5 query heads per KV head, heads of 32)."""
+    shape = synth.ModelShape(n_layers=2, hidden=192, n_q_heads=10, n_kv_heads=2, head_dim=32, ffn=320, vocab=512)
+    wt = synth.model_weights(shape, 7)
+    prompt = synth.random_prompt(40, shape.vocab, 7).numpy()
+    forced = [3, 400, 77, 12, 250, 9]
+    tr = _oracle_trace(shape, wt, prompt, forced)
+    for li in range(shape.n_layers):
+        _run_layer(cass, shape, wt, tr, li, prompt, forced)
+    _run_logits(cass, shape, wt, tr, prompt, forced)
+
+
+def test_llama_8b_layer_geometry(cass):
+    """One layer of the Llama-3-8B geometry (hidden 4096, 32 q / 8 kv heads of 128, FFN 14336; vocabulary cut to 1024):
+    the tensor-core attention, the fused RoPE + KV encoder and the draft GEMV chain together.  Prompt of 40, four forced
+    draft steps and a five-row verification; layer output and logits against the oracle."""
+    shape = synth.ModelShape(n_layers=1, hidden=4096, n_q_heads=32, n_kv_heads=8, head_dim=128, ffn=14336, vocab=1024)
+    wt = synth.model_weights(shape, 0)
+    prompt = synth.random_prompt(40, shape.vocab, 0).numpy()
+    forced = [101, 7, 993, 512, 64]
+    tr = _oracle_trace(shape, wt, prompt, forced)
+    _run_layer(cass, shape, wt, tr, 0, prompt, forced)
+    _run_logits(cass, shape, wt, tr, prompt, forced)

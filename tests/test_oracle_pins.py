@@ -314,12 +314,7 @@ def test_draft_gemv_and_attention_reduce_to_library_routines():
         qf[None, :, None, :], kd.permute(1, 0, 2).repeat_interleave(2, 0)[None],
         vd.permute(1, 0, 2).repeat_interleave(2, 0)[None])[0, :, 0, :]
     # the oracle's own attention for the same inputs
-    d = 16
-    o2 = np.zeros((4, d))
-    for hq in range(4):
-        sc = (kd[:, hq // 2, :].numpy() @ qf[hq].numpy()) / np.sqrt(d)
-        pr = np.exp(sc - sc.max()); pr /= pr.sum()
-        o2[hq] = pr @ vd[:, hq // 2, :].numpy()
+    o2 = model.attention(qb, kv.kd[0, : kv.n + 1], kv.vd[0, : kv.n + 1])
     assert np.allclose(o.numpy(), o2, rtol=1e-12, atol=1e-14)
     assert np.isfinite(logits).all()
     # the draft view of the cache is the truncated, pruned target cache
