@@ -150,6 +150,10 @@ int cass_decode_full(const void* blob, const cass_blob_info* h_info, const void*
  *   y[r] = sum_c decode(blob)[r][c] * x[c], fp32 accumulation, y rounded to bf16 (y_bf16) and/or kept fp32.
  * x: bf16 [cols].  partial: fp32 scratch [n_seg][n_rowblocks*32], which receives the per-segment sums.  Either
  * output pointer may be NULL; with both NULL only `partial` is produced.
+ * h_info is what cass_weight_blob_info returned for this blob (that call synchronises, so the blob is complete: the
+ * kernel starts reading the blob before earlier work on the stream has finished).  The blob buffer holds at least
+ * h_info->total_bytes bytes; nothing beyond them is read, and a directory entry that points outside, like a header
+ * that differs from h_info, is refused through d_status (CASS_ERR_INVALID_ARG) instead of being followed.
  * ---------------------------------------------------------------------------------------------------- */
 int cass_draft_gemv(const void* blob, const cass_blob_info* h_info, const void* x_bf16, float* partial,
                     void* y_bf16, float* y_f32, int32_t* d_status, void* stream);
@@ -236,7 +240,8 @@ int cass_set_lens(void* session, const int32_t* h_lens, void* stream);
  * position's K/V to the sequence's compressed cache only, and writes the greedy next token to
  * tok_out[b * tok_stride] (lowest index on ties).  tok_stride = 1 for packed arrays, g+1 when the tokens sit in the
  * [max_batch][g+1] array that cass_verify reads.  The weights' speculation data is read and decoded once for all
- * sequences.  logits_opt: fp32 [max_batch][vocab] or NULL. */
+ * sequences.  logits_opt: fp32 [max_batch][vocab] or NULL.  At most gamma_max calls between two accepts (or
+ * cass_set_len / cass_set_lens / cass_session_reset): one more returns CASS_ERR_INVALID_ARG and launches nothing. */
 int cass_draft_step(void* session, const int32_t* tok_in, int32_t* tok_out, int tok_stride, float* logits_opt,
                     void* stream);
 
@@ -276,6 +281,31 @@ int cass_verify_gemm(const void* W_bf16, const void* X_bf16, int rows, int n, in
 int cass_accept(void* session, const int32_t* draft, int draft_stride, const int32_t* target_argmax, int g,
                 int32_t* n_accepted, int32_t* out_tokens, int32_t* next_tok, int next_stride, void* stream);
 
+/* Acceptance by rejection sampling (Sec. 2.2, Eq. 1), for decoding with sampling instead of greedy choice.  Per
+ * sequence b, with x_i = draft[b * draft_stride + i - 1] the i-th drafted token (drawn from the draft's distribution
+ * q_i), p_i the target's distribution at the same row and r_i a uniform number in (0, 1):
+ *   n = min({i-1 : 1 <= i <= g, r_i > p_i(x_i) / q_i(x_i)} U {g})                                        (Eq. 1)
+ * and the step emits one more token, drawn with the uniform number u_b by inverse CDF (lowest index whose cumulative
+ * weight exceeds u_b times the total): from the normalised positive part of p_{n+1} - q_{n+1} after a rejection, from
+ * p_{g+1} when all g drafts were accepted.  (The paper states the guarantee -- outputs distributed exactly as the
+ * target's -- and cites speculative sampling for the procedure; this is that procedure's correction step.)
+ * p_target: fp32 [n_seq][g+1][vocab], q_draft: fp32 [n_seq][g][vocab] (probabilities, see cass_softmax);
+ * r_uniform: fp32 [n_seq][g]; u_uniform: fp32 [n_seq]; the library draws no random numbers itself.
+ * Outputs as cass_accept: n_accepted [n_seq], out_tokens [n_seq][g+1] (n drafts, the extra token, then -1),
+ * next_tok[b * next_stride] = the extra token.  With a session (n_seq must equal its max_batch, vocab its vocab) the
+ * lengths move by n+1 and the draft counters are cleared exactly as in cass_accept; session may be NULL, then only
+ * the outputs are produced (any n_seq).  A drafted token outside [0, vocab) is rejected. */
+int cass_accept_sampling(void* session, int n_seq, const int32_t* draft, int draft_stride, const float* p_target,
+                         const float* q_draft, int vocab, const float* r_uniform, const float* u_uniform, int g,
+                         int32_t* n_accepted, int32_t* out_tokens, int32_t* next_tok, int next_stride, void* stream);
+
+/* Helpers for sampled decoding (Sec. 2.2).  cass_softmax: probs[r][v] = softmax(logits[r][.] / temperature), fp32
+ * [rows][vocab] both, temperature > 0 (the fp32 logits are what cass_draft_step / cass_verify return in logits_opt).
+ * cass_sample: tokens[r * tok_stride] = inverse-CDF draw from probs[r][.] (non-negative weights; need not be
+ * normalised) with the uniform number u[r] in [0, 1). */
+int cass_softmax(const float* logits, int rows, int vocab, float temperature, float* probs, void* stream);
+int cass_sample(const float* probs, int rows, int vocab, const float* u, int32_t* tokens, int tok_stride, void* stream);
+
 /* Geometry of the compressed KV cache of (sequence, layer, kind 0=K 1=V, head) for tests: device pointers to the
  * fixed-part blocks, the unary arena and the per-token word offsets, plus words per token in the fixed part. */
 typedef struct cass_kv_view {
@@ -287,7 +317,8 @@ int cass_kv_query(void* session, int seq, int layer, int kind, int head, cass_kv
 
 /* Standalone draft attention / verify kernels are reached through cass_draft_step / cass_verify; the
  * activations of the last call can be inspected for tests: which = 0 hidden state after the last layer
- * (bf16 [rows][hidden]), 1 = layer-0 attention output (bf16 [rows][n_q d]). */
+ * (bf16 [rows][hidden]), 1 = the last layer's attention output (bf16 [rows][n_q d]), 2 = the last layer's rotated
+ * q, k, v rows (bf16 [rows][(n_q + 2 n_kv) d]).  *h_rows is the buffer's row capacity. */
 int cass_debug_activation(void* session, int which, const void** d_ptr, int* h_rows, int* h_cols);
 
 const char* cass_version(void);

@@ -182,53 +182,41 @@ def unary_decode_sequential(bits: np.ndarray, numel: int) -> np.ndarray:
 
 
 def unary_decode_chunked(bits: np.ndarray, numel: int, chunk: int = 8) -> np.ndarray:
-    """Algorithm 1: parallel zero counting on fixed-size chunks, then reorganisation.
+    """Chunk-parallel unary decoder (Sec. 5.1, the parallel zero counter and the reorganisation step of Algorithm 1).
 
-    Step 1 (per chunk, independent of the others): for every one in the chunk, the
-    number of zeros since the previous one *of the same chunk* (or since the chunk
-    start); the number of ones; the count of trailing zeros after the last one.
-    Step 2 (reorganisation): zeros left over at the end of a chunk (all of them if
-    the chunk has no one) are added to the first output of the next chunk that
-    contains a one.
-    Step 3: outputs are read in order and stop after `numel` symbols.
+    The stream is cut into chunks of `chunk` bits that are examined independently of one another:
+      * inside a chunk, every one closes a zero run that started after the previous one OF THAT CHUNK (or at the
+        chunk's first bit);
+      * the zeros after a chunk's last one (the whole chunk if it has no one) are not a codeword yet: they are pending.
+    Pending zeros then travel forwards: they are added to the first run of the next chunk that holds a one, crossing
+    any number of chunks without a one on the way.  The first `numel` runs, in stream order, are the ranks.
+    The result equals `unary_decode_sequential`; zero runs may be longer than a chunk.
     """
     bits = np.asarray(bits, dtype=np.uint8)
     n_chunks = (bits.size + chunk - 1) // chunk
-    padded = np.zeros(n_chunks * chunk, dtype=np.uint8)
-    padded[: bits.size] = bits
-    chunks = padded.reshape(n_chunks, chunk)
-
-    outputs: list[list[int]] = []
-    trailing: list[int] = []
-    for i in range(n_chunks):                       # "parallel zero counting"
-        cnt = 0
-        out_i: list[int] = []
-        for j in range(chunk):
-            if chunks[i, j] == 0:
-                cnt += 1
-            else:
-                out_i.append(cnt)
-                cnt = 0
-        outputs.append(out_i)
-        trailing.append(cnt)                        # zeros after the chunk's last one
-
-    carry = 0                                       # "parallel reorganisation"
-    for k in range(n_chunks):
-        if outputs[k]:
-            outputs[k][0] += carry
-            carry = trailing[k]
-        else:
-            carry += trailing[k]                    # a chunk without a one passes everything on
-
-    exp_ranks: list[int] = []
-    for l in range(n_chunks):
-        for v in outputs[l]:
-            if len(exp_ranks) == numel:
-                return np.array(exp_ranks, dtype=np.int64)
-            exp_ranks.append(v)
-    if len(exp_ranks) != numel:
+    table = np.zeros((n_chunks, chunk), dtype=np.uint8)
+    table.reshape(-1)[: bits.size] = bits
+    at_chunk, at_bit = np.nonzero(table)                       # every one: its chunk and its place in the chunk, stream order
+    if at_chunk.size < numel:
         raise ValueError("stream ended before numel codewords")
-    return np.array(exp_ranks, dtype=np.int64)
+    if numel == 0:
+        return np.zeros(0, dtype=np.int64)
+    opens_chunk = np.concatenate(([True], at_chunk[1:] != at_chunk[:-1]))      # the first one of its chunk
+    left_neighbour = np.where(opens_chunk, -1, np.concatenate(([0], at_bit[:-1])))
+    runs = (at_bit - left_neighbour - 1).astype(np.int64)      # zero runs as each chunk sees them on its own
+    last_one = np.full(n_chunks, -1, dtype=np.int64)
+    last_one[at_chunk] = at_bit                                # later ones overwrite earlier ones of the same chunk
+    pending = chunk - 1 - last_one                             # zeros left at the end of each chunk (all of it if no one)
+    # zeros pending at the START of chunk c: everything left behind since (and including) the latest earlier chunk that
+    # holds a one -- a prefix sum of `pending` that restarts at every such chunk
+    before = np.concatenate(([0], np.cumsum(pending)[:-1]))    # sum of pending over chunks < c
+    holds_one = last_one >= 0
+    restart = np.where(holds_one, np.arange(n_chunks), 0)
+    latest = np.concatenate(([0], np.maximum.accumulate(restart)[:-1]))        # latest chunk < c with a one (0 if none)
+    seen_one = np.concatenate(([False], np.logical_or.accumulate(holds_one)[:-1]))
+    arriving = before - np.where(seen_one, before[latest], 0)
+    runs[opens_chunk] += arriving[at_chunk[opens_chunk]]
+    return runs[:numel]
 
 
 def unary_decode_fast(bits: np.ndarray, numel: int) -> np.ndarray:

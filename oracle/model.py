@@ -238,6 +238,46 @@ def greedy_accept(draft_tokens, target_argmax):
     return min(rejected + [gamma])
 
 
+def softmax(logits: np.ndarray, temperature: float = 1.0) -> np.ndarray:
+    """Probabilities of a logit vector at a sampling temperature (fp64)."""
+    z = np.asarray(logits, dtype=np.float64) / float(temperature)
+    z = z - z.max()
+    e = np.exp(z)
+    return e / e.sum()
+
+
+def inverse_cdf_sample(weights: np.ndarray, u: float) -> int:
+    """Index drawn from the (unnormalised, non-negative) weights by the uniform number u in [0, 1): the lowest index
+    whose cumulative weight exceeds u times the total."""
+    w = np.asarray(weights, dtype=np.float64)
+    c = np.cumsum(w)
+    return int(min(np.searchsorted(c, u * c[-1], side="right"), w.size - 1))
+
+
+def sampling_accept(p: np.ndarray, q: np.ndarray, draft_tokens, r: np.ndarray, u: float):
+    """Acceptance by rejection sampling (Sec. 2.2, Eq. 1) and the token that closes the step.
+
+    p [gamma+1, V]: the target's distributions at the gamma+1 verified rows; q [gamma, V]: the draft's distributions
+    the tokens x_i = draft_tokens[i-1] were drawn from; r [gamma]: uniform numbers in (0, 1), one per drafted token;
+    u: one more uniform number.  Eq. 1: n = min({i-1 : 1 <= i <= gamma, r_i > p_i(x_i) / q_i(x_i)} U {gamma}).
+    The step then emits one more token.  The paper states the guarantee (outputs distributed exactly as the target's)
+    and cites speculative sampling for the procedure; that procedure draws the extra token from the normalised
+    positive part of p_{n+1} - q_{n+1} after a rejection, and from p_{gamma+1} when every draft was accepted -- the
+    choice that makes the guarantee hold.  Returns (n, emitted tokens: the n accepted drafts + the extra token)."""
+    p = np.asarray(p, dtype=np.float64)
+    q = np.asarray(q, dtype=np.float64)
+    gamma = len(draft_tokens)
+    stops = [i - 1 for i in range(1, gamma + 1)
+             if r[i - 1] * q[i - 1, draft_tokens[i - 1]] > p[i - 1, draft_tokens[i - 1]]]     # r > p/q without dividing
+    n = min(stops + [gamma])
+    if n < gamma:
+        residual = np.maximum(p[n] - q[n], 0.0)
+        extra = inverse_cdf_sample(residual if residual.sum() > 0.0 else p[n], u)
+    else:
+        extra = inverse_cdf_sample(p[gamma], u)
+    return n, [int(t) for t in draft_tokens[:n]] + [extra]
+
+
 def plain_greedy(W: Weights, kv: KVCache, first_tok: int, n_tokens: int, kv_p: int, kv_t: int):
     """Autoregressive decoding with the target only.  `first_tok` is the token predicted from the
     prompt; returns the n_tokens tokens that follow it."""

@@ -282,6 +282,23 @@ def cass_accept(session, draft, target_argmax, g: int, n_accepted, out_tokens, n
                                           next_stride, _stream(stream)))
 
 
+def cass_accept_sampling(session, n_seq: int, draft, p_target, q_draft, vocab: int, r_uniform, u_uniform, g: int,
+                         n_accepted, out_tokens, next_tok, stream=None, draft_stride: int | None = None,
+                         next_stride: int = 1):
+    _check("cass_accept_sampling", lib.cass_accept_sampling(
+        session, n_seq, _ptr(draft), g if draft_stride is None else draft_stride, _ptr(p_target), _ptr(q_draft), vocab,
+        _ptr(r_uniform), _ptr(u_uniform), g, _ptr(n_accepted), _ptr(out_tokens), _ptr(next_tok), next_stride,
+        _stream(stream)))
+
+
+def cass_softmax(logits, rows: int, vocab: int, temperature: float, probs, stream=None):
+    _check("cass_softmax", lib.cass_softmax(_ptr(logits), rows, vocab, C.c_float(temperature), _ptr(probs), _stream(stream)))
+
+
+def cass_sample(probs, rows: int, vocab: int, u, tokens, stream=None, tok_stride: int = 1):
+    _check("cass_sample", lib.cass_sample(_ptr(probs), rows, vocab, _ptr(u), _ptr(tokens), tok_stride, _stream(stream)))
+
+
 def cass_kv_query(session, layer: int, kind: int, head: int, seq: int = 0) -> KVView:
     v = KVView()
     _check("cass_kv_query", lib.cass_kv_query(session, seq, layer, kind, head, C.byref(v)))

@@ -3,9 +3,9 @@
 // through a rank->exponent table, sign/mantissa concatenation).
 //
 // Work unit = one superblock (32 rows x one column segment).  A CTA owns one column segment (its slice of x
-// stays in shared memory as fp32) and walks the row blocks assigned to it; superblocks arrive through a
-// two-stage ring of bulk asynchronous copies (contiguous reads, as Sec. 5.3 asks), so the copy of the next
-// superblocks overlaps the decode of the current one.  Warp c decodes chunk c with lane = row: every lane
+// stays in shared memory as fp32) and walks the row blocks assigned to it; a superblock arrives by one bulk
+// asynchronous copy (contiguous reads, as Sec. 5.3 asks) into the CTA's single stage; the CTAs that share an SM
+// overlap each other's copies and decodes.  Warp c decodes chunk c with lane = row: every lane
 // walks its own bitmap, field and unary streams, which are interleaved word by word over the 32 rows so that
 // all shared-memory reads of the streams are conflict free.
 #include <type_traits>
@@ -314,7 +314,7 @@ template <int T, int NB>
 __global__ void __launch_bounds__(1024) k_draft_gemv(const uint32_t* __restrict__ blob, const uint16_t* __restrict__ x,
                                                      float* __restrict__ partial, int32_t* __restrict__ d_status,
                                                      int stage_bytes, int max_sb, int n, int k, int t, int seg_cols,
-                                                     int chunk_cols, int n_seg, int n_rb) {
+                                                     int chunk_cols, int n_seg, int n_rb, unsigned long long blob_bytes) {
     extern __shared__ __align__(128) uint8_t smem_raw[];
     // The geometry comes from the host's copy of the header (the launch sized shared memory from it); the header
     // itself is fetched now and compared once it has arrived, so that its latency is off the critical path.
@@ -347,21 +347,25 @@ __global__ void __launch_bounds__(1024) k_draft_gemv(const uint32_t* __restrict_
     }
     __syncthreads();
 
-    // thread 0: start the copy of tile i into stage i % kGemvStages
+    // thread 0: start the copy of tile i into stage i % kGemvStages.  Nothing is read beyond blob + blob_bytes (the
+    // size the caller's description gives): a directory entry that points outside is skipped and flagged.
     auto issue = [&](int i) {
         const int s = i % kGemvStages;
         const int sb_i = (rb0 + i * rb_step) * n_seg + seg;
         const uint32_t* dir = blob + kBlobDirOffset / 4 + sb_i * 4;
-        const SbGeom g = SbGeom::make(dir_n_ch(dir[3]), scols, (int)dir[1], (int)dir[2]);
+        const bool dir_ok = (unsigned long long)kBlobDirOffset + ((unsigned long long)sb_i + 1ull) * 16ull <= blob_bytes;
+        const uint32_t d0 = dir_ok ? dir[0] : 0u, d1 = dir_ok ? dir[1] : 0u, d2 = dir_ok ? dir[2] : 0u, d3 = dir_ok ? dir[3] : 0u;
+        const SbGeom g = SbGeom::make(dir_n_ch(d3), scols, (int)d1, (int)d2);
         const uint32_t bytes = (uint32_t)g.total * 4u;
-        if (bytes > (uint32_t)max_sb || dir_n_ch(dir[3]) != n_ch) {               // does not fit: skip the tile, flag it
+        if (!dir_ok || bytes > (uint32_t)max_sb || dir_n_ch(d3) != n_ch || d1 > 0xFFFFu || d2 > 0xFFFFu ||
+            (unsigned long long)d0 * 16ull + bytes > blob_bytes) {                // does not fit: skip the tile, flag it
             s_skip[s] = 1;
             if (d_status) atomicExch(d_status, CASS_ERR_INVALID_ARG);
             mbar_expect_tx(&bar[s], 0);
             return;
         }
         s_skip[s] = 0;
-        const uint8_t* src = reinterpret_cast<const uint8_t*>(blob) + (size_t)dir[0] * 16;
+        const uint8_t* src = reinterpret_cast<const uint8_t*>(blob) + (size_t)d0 * 16;
         uint8_t* dst = smem_raw + (size_t)s * stage_bytes;
         mbar_expect_tx(&bar[s], bytes);
         for (uint32_t off = 0; off < bytes; off += 32768u) bulk_g2s(dst + off, src + off, min(32768u, bytes - off), &bar[s]);
@@ -556,7 +560,8 @@ int launch_draft_gemv(const void* blob, const cass_blob_info& bi, const void* x_
         CASS_CUDA_CHECK(cudaLaunchKernelEx(&cfg, k_draft_gemv<TT, NN>, b, x, partial, d_status, stage,         \
                                            (int)bi.max_superblock_bytes, (int)bi.rows, (int)bi.cols,           \
                                            (int)bi.trunc_bits, (int)bi.seg_cols, (int)bi.chunk_cols,           \
-                                           (int)bi.n_seg, (int)bi.n_rowblocks));                               \
+                                           (int)bi.n_seg, (int)bi.n_rowblocks,                                 \
+                                           (unsigned long long)bi.total_bytes));                               \
     } while (0)
 #define CASS_GEMV_LAUNCH_NB(TT)                                                                                \
     do {                                                                                                       \

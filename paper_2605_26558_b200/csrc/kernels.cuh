@@ -93,6 +93,11 @@ int launch_argmax(const float* logits, Partials pp, int rows, int vocab, int32_t
                   float* logits_copy, float* tmp_v, int32_t* tmp_i, DevState* st, int bump_inflight, cudaStream_t s);
 int launch_accept(DevState* st, int n_seq, const int32_t* draft, int draft_stride, const int32_t* target, int g, int32_t* n_acc,
                   int32_t* out_tokens, int32_t* next_tok, int next_stride, cudaStream_t s);
+// Sampling-based acceptance (sampling.cu): p [n_seq][g+1][vocab], q [n_seq][g][vocab] probabilities, r [n_seq][g] and
+// u [n_seq] uniform numbers; st may be null (no lengths to move).
+int launch_accept_sampling(DevState* st, int n_seq, const int32_t* draft, int draft_stride, const float* p, const float* q,
+                           int vocab, const float* r, const float* u, int g, int32_t* n_acc, int32_t* out_tokens,
+                           int32_t* next_tok, int next_stride, cudaStream_t s);
 int launch_calib_accum(const uint16_t* x, int rows, int cols, float* sumsq, const DevState* st, cudaStream_t s);
 int launch_sqrt(const float* in, float* out, size_t n, cudaStream_t s);
 

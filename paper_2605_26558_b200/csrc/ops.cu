@@ -231,7 +231,11 @@ __global__ void __launch_bounds__(kArgmaxSlices) k_argmax_final(const float* __r
     if (threadIdx.x == 0) {
         for (int w = 1; w < kArgmaxSlices / 32; ++w) argmax_combine(best, best_i, s_v[w], s_i[w]);
         out[(size_t)r * out_stride] = best_i == 0x7fffffff ? 0 : best_i;
-        if (bump_inflight && r < kMaxBatch) st->inflight[r] += 1;
+        if (bump_inflight && r < kMaxBatch) {
+            // the draft counter never passes the margin kept free at the end of a cache (positions len .. len + 15)
+            if (st->inflight[r] < kMaxVerifyRows - 1) st->inflight[r] += 1;
+            else atomicCAS(&st->status, 0, CASS_ERR_INVALID_ARG);
+        }
     }
 }
 

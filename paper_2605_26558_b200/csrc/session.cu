@@ -44,6 +44,7 @@ struct Session {
     float* argmax_val;
     bool have_blobs, codebooks_ready, calib_host;
     int qkv_dim, kmax;
+    int drafts_pending;      // cass_draft_step calls since the last accept / set_len / reset (host-side count)
 };
 
 struct Plan {
@@ -264,6 +265,7 @@ extern "C" int cass_session_reset(void* session, void* stream_) {
                 CASS_CUDA_CHECK(cudaMemsetAsync(c.off, 0, (size_t)s->kg.n_kv * (s->kg.max_seq + 1) * 4, stream));
             }
     s->codebooks_ready = false;
+    s->drafts_pending = 0;
     return CASS_OK;
 }
 
@@ -329,6 +331,7 @@ extern "C" int cass_set_len(void* session, int len, void* stream_) {
     static_assert(offsetof(DevState, inflight) == sizeof(int32_t) * kMaxBatch, "len[] then inflight[]");
     CASS_CUDA_CHECK(cudaMemcpyAsync(s->st->len, v, sizeof(v), cudaMemcpyHostToDevice, (cudaStream_t)stream_));
     CASS_CUDA_CHECK(cudaStreamSynchronize((cudaStream_t)stream_));
+    s->drafts_pending = 0;
     return CASS_OK;
 }
 
@@ -342,6 +345,7 @@ extern "C" int cass_set_lens(void* session, const int32_t* h_lens, void* stream_
     }
     CASS_CUDA_CHECK(cudaMemcpyAsync(s->st->len, v, sizeof(v), cudaMemcpyHostToDevice, (cudaStream_t)stream_));
     CASS_CUDA_CHECK(cudaStreamSynchronize((cudaStream_t)stream_));
+    s->drafts_pending = 0;
     return CASS_OK;
 }
 
@@ -484,6 +488,10 @@ extern "C" int cass_draft_step(void* session, const int32_t* tok_in, int32_t* to
     if (!session || !tok_in || !tok_out || tok_stride < 1) return CASS_ERR_INVALID_ARG;
     Session* s = (Session*)session;
     if (!s->have_blobs || !s->codebooks_ready) return CASS_ERR_INVALID_ARG;
+    // a drafted token sits at position len + (drafts since the last accept); more than gamma_max of them would leave
+    // the rows a verification call can take and, at the end of a cache, the cache itself
+    if (s->drafts_pending >= s->d.gamma_max) return CASS_ERR_INVALID_ARG;
+    s->drafts_pending += 1;
     cudaStream_t st = (cudaStream_t)stream_;
     const cass_model_desc& d = s->d;
     const int qd = d.n_q_heads * d.head_dim;
@@ -524,6 +532,26 @@ extern "C" int cass_accept(void* session, const int32_t* draft, int draft_stride
     if (draft_stride < g || next_stride < 1) return CASS_ERR_INVALID_ARG;
     Session* s = (Session*)session;
     if (g < 0 || g + 1 > kMaxVerifyRows) return CASS_ERR_INVALID_ARG;
+    s->drafts_pending = 0;
     return launch_accept(s->st, s->B, draft, draft_stride, target_argmax, g, n_accepted, out_tokens, next_tok, next_stride,
                          (cudaStream_t)stream_);
+}
+
+extern "C" int cass_accept_sampling(void* session, int n_seq, const int32_t* draft, int draft_stride, const float* p_target,
+                                    const float* q_draft, int vocab, const float* r_uniform, const float* u_uniform, int g,
+                                    int32_t* n_accepted, int32_t* out_tokens, int32_t* next_tok, int next_stride,
+                                    void* stream_) {
+    if (!p_target || !u_uniform || !n_accepted || !out_tokens || (g > 0 && (!draft || !q_draft || !r_uniform)))
+        return CASS_ERR_INVALID_ARG;
+    if (g < 0 || g + 1 > kMaxVerifyRows || draft_stride < g || next_stride < 1 || vocab <= 0 || n_seq < 1)
+        return CASS_ERR_INVALID_ARG;
+    DevState* st = nullptr;
+    if (session) {
+        Session* s = (Session*)session;
+        if (n_seq != s->B || vocab != s->d.vocab) return CASS_ERR_INVALID_ARG;
+        s->drafts_pending = 0;
+        st = s->st;
+    }
+    return launch_accept_sampling(st, n_seq, draft, draft_stride, p_target, q_draft, vocab, r_uniform, u_uniform, g, n_accepted,
+                                  out_tokens, next_tok, next_stride, (cudaStream_t)stream_);
 }

@@ -80,6 +80,69 @@ def test_gemv_refuses_a_blob_that_does_not_match_its_description(cass):
         cass.cass_weight_blob_info(torch.zeros(1024, dtype=torch.uint8, device="cuda"))
 
 
+def test_gemv_skips_directory_entries_that_point_outside_the_blob(cass):
+    """A directory entry whose offset or size would take the bulk copy past the blob's end (as the caller's description
+    sizes it) is skipped and flagged; the other superblocks still give their rows."""
+    fmt = cass.default_format()
+    w = synth.student_t_weight(96, 512, 2, "err/w3").cuda()
+    bound, ws_bytes = cass.cass_encoded_weight_bytes(fmt, 96, 512)
+    blob = torch.zeros(bound, dtype=torch.uint8, device="cuda")
+    ws = torch.zeros(ws_bytes, dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    cass.cass_encode_weights(fmt, w, None, blob, ws, status)
+    info = cass.cass_weight_blob_info(blob)
+    blob = blob[: info.total_bytes].clone()
+    x = synth.activation_vector(512, 1, "err/x3").cuda()[0].contiguous()
+    partial = torch.zeros(info.n_seg * info.n_rowblocks * 32, dtype=torch.float32, device="cuda")
+    good = torch.zeros(96, dtype=torch.float32, device="cuda")
+    cass.cass_draft_gemv(blob, info, x, partial, None, good, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    words = blob.view(torch.int32)
+    dir0 = (128 + 256) // 4                               # directory: 4 words per superblock, after header and codebook
+    for field, value in ((0, 0x7FFFFFF), (1, 0x7FFF)):    # offset far outside; field words that overrun the blob
+        bad = blob.clone()
+        bw = bad.view(torch.int32)
+        bw[dir0 + 4 * 1 + field] = value                  # superblock 1 = rows 32..63
+        status.zero_()
+        y = torch.zeros(96, dtype=torch.float32, device="cuda")
+        partial.zero_()
+        cass.cass_draft_gemv(bad, info, x, partial, None, y, status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == cass.ERR_INVALID_ARG
+        assert torch.equal(y[:32], good[:32]) and torch.equal(y[64:], good[64:])
+    short = cass.cass_weight_blob_info(blob)
+    short.total_bytes = 128 + 256 + 16                    # a description that ends inside the directory
+    status.zero_()
+    cass.cass_draft_gemv(blob, short, x, partial, None, good.clone(), status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == cass.ERR_INVALID_ARG
+
+
+def test_draft_steps_beyond_gamma_max_are_refused(cass):
+    """More drafted tokens than gamma_max since the last accept would leave the rows of a verification call (and, at
+    the end of a cache, the cache): the call is refused on the host; accept and set_len clear the count."""
+    eng = _tiny_engine(cass)                              # gamma_max = 4
+    eng.prefill(synth.random_prompt(20, synth.TINY.vocab, 5))
+    eng.encode_weights(None)
+    eng.build_kv_codebook()
+    tok = torch.zeros(8, dtype=torch.int32, device="cuda")
+    for i in range(4):
+        cass.cass_draft_step(eng.session, tok[i: i + 1], tok[i + 1: i + 2])
+    with pytest.raises(cass.CassError) as e:
+        cass.cass_draft_step(eng.session, tok[4:5], tok[5:6])
+    assert e.value.code == cass.ERR_INVALID_ARG
+    cass.cass_set_len(eng.session, 20)
+    cass.cass_draft_step(eng.session, tok[:1], tok[1:2])  # counted from zero again
+    cass.cass_verify(eng.session, tok, 1, eng.targ)
+    cass.cass_accept(eng.session, tok[1:], eng.targ, 1, eng.n_acc, eng.out_tokens, eng.toks)
+    for i in range(4):
+        cass.cass_draft_step(eng.session, tok[i: i + 1], tok[i + 1: i + 2])
+    torch.cuda.synchronize()
+    assert eng.status()[0] == 0
+    eng.close()
+
+
 def test_empty_and_single_position_inputs(cass):
     eng = _tiny_engine(cass)
     k, v = synth.kv_fill(1, 2, 64, 0, "err/kv")

@@ -92,12 +92,22 @@ def _hidden(cass, eng, rows):
 
 
 def _assert_close(got, want_bits, what):
-    """Every element within TOL of the RMS of the oracle's vector, outright."""
+    """A layer's output hidden state against the oracle's.  Both sides are bf16-ROUNDED and a layer rounds its residual
+    stream twice (after the attention block and after the FFN block): where the fp32 and the fp64 sums fall on different
+    sides of a rounding boundary the results are neighbouring bf16 values.  On the elements fed by this workload's x20
+    outlier channels, several times the vector's RMS, one bf16 ulp (2^-7 of the element) is more than TOL * RMS by
+    itself.  So: every element within TOL * RMS, except that an element may instead be within two bf16 ulps of the
+    oracle's value (one per rounded residual add); at most 1 % of a vector's elements may need the exception."""
     want = codec.bf16_bits_to_f64(want_bits)
+    got_bits = codec.f64_to_bf16_bits(got)
     rms = float(np.sqrt(np.mean(want ** 2)))
-    err = float(np.abs(got - want).max())
-    assert err <= TOL * rms, (what, err / rms)
-    return err / rms
+    err = np.abs(got - want)
+    key = lambda b: np.where(b & 0x8000, -(b & 0x7FFF).astype(np.int64), (b & 0x7FFF).astype(np.int64))
+    ulps = np.abs(key(got_bits) - key(np.asarray(want_bits, dtype=np.uint16)))
+    over = err > TOL * rms
+    assert not (over & (ulps > 2)).any(), (what, float(err.max()) / rms, int(ulps[over].max()))
+    assert over.mean() <= 0.01, (what, float(over.mean()))
+    return float(err.max()) / rms
 
 
 def _run_layer(cass, shape, wt, tr, li, prompt, forced):
@@ -179,38 +189,54 @@ def _run_logits(cass, shape, wt, tr, prompt, forced):
     return worst
 
 
-def test_tiny_model_every_layer_and_the_logits(cass):
-    """Config 1 (2 layers, hidden 256, 4 q / 2 kv heads of 64, FFN 688, vocab 1024): prompt of 64, gamma = 4."""
+def _tiny_case():
     shape = synth.TINY
     wt = synth.model_weights(shape, 0)
     prompt = synth.random_prompt(64, shape.vocab, 0).numpy()
-    forced = [int(t) for t in (901, 17, 333, 5, 640)]
-    tr = _oracle_trace(shape, wt, prompt, forced)
-    for li in range(shape.n_layers):
-        _run_layer(cass, shape, wt, tr, li, prompt, forced)
-    _run_logits(cass, shape, wt, tr, prompt, forced)
+    return shape, wt, prompt, [int(t) for t in (901, 17, 333, 5, 640)]
 
 
-def test_five_query_heads_per_kv_head_layers(cass):
-    """The Qwen-style grouping (5 query heads per KV head, heads of 32)."""
+def _group5_case():
     shape = synth.ModelShape(n_layers=2, hidden=192, n_q_heads=10, n_kv_heads=2, head_dim=32, ffn=320, vocab=512)
     wt = synth.model_weights(shape, 7)
     prompt = synth.random_prompt(40, shape.vocab, 7).numpy()
-    forced = [3, 400, 77, 12, 250, 9]
-    tr = _oracle_trace(shape, wt, prompt, forced)
-    for li in range(shape.n_layers):
-        _run_layer(cass, shape, wt, tr, li, prompt, forced)
-    _run_logits(cass, shape, wt, tr, prompt, forced)
+    return shape, wt, prompt, [3, 400, 77, 12, 250, 9]
 
 
-def test_llama_8b_layer_geometry(cass):
-    """One layer of the Llama-3-8B geometry (hidden 4096, 32 q / 8 kv heads of 128, FFN 14336; vocabulary cut to 1024):
-    the tensor-core attention, the fused RoPE + KV encoder and the draft GEMV chain together.  Prompt of 40, four forced
-    draft steps and a five-row verification; layer output and logits against the oracle."""
+def _llama_layer_case():
     shape = synth.ModelShape(n_layers=1, hidden=4096, n_q_heads=32, n_kv_heads=8, head_dim=128, ffn=14336, vocab=1024)
     wt = synth.model_weights(shape, 0)
     prompt = synth.random_prompt(40, shape.vocab, 0).numpy()
-    forced = [101, 7, 993, 512, 64]
-    tr = _oracle_trace(shape, wt, prompt, forced)
-    _run_layer(cass, shape, wt, tr, 0, prompt, forced)
-    _run_logits(cass, shape, wt, tr, prompt, forced)
+    return shape, wt, prompt, [101, 7, 993, 512, 64]
+
+
+_CASES = {"tiny": _tiny_case, "group5": _group5_case, "llama8b_layer": _llama_layer_case}
+_TRACES = {}
+
+
+def _case(name):
+    """config 1 (2 layers, hidden 256, 4 q / 2 kv heads of 64, FFN 688, vocab 1024; prompt 64, gamma 4); the Qwen-style
+    grouping (5 query heads per KV head, heads of 32; gamma 5); one layer of the Llama-3-8B geometry (hidden 4096,
+    32 q / 8 kv heads of 128, FFN 14336, vocabulary cut to 1024): tensor-core attention, fused RoPE + KV encoder and
+    the draft GEMV chain together."""
+    if name not in _TRACES:
+        shape, wt, prompt, forced = _CASES[name]()
+        _TRACES[name] = (shape, wt, prompt, forced, _oracle_trace(shape, wt, prompt, forced))
+    return _TRACES[name]
+
+
+@pytest.mark.parametrize("name", ["tiny", "group5", "llama8b_layer"])
+def test_every_layer_teacher_forced(cass, name):
+    """Prefill chunk, forced draft steps and the verification rows of every layer, each fed the oracle's own input."""
+    shape, wt, prompt, forced, tr = _case(name)
+    worst = [_run_layer(cass, shape, wt, tr, li, prompt, forced) for li in range(shape.n_layers)]
+    print(f"{name}: worst layer-output error / RMS per layer: {worst}")
+
+
+@pytest.mark.parametrize("name", ["tiny", "group5", "llama8b_layer"])
+def test_logits_given_the_final_hidden_state(cass, name):
+    """Draft and verification logits (fp32, unrounded) given the oracle's final hidden states: max |delta| <= 2e-2 of
+    the logit RMS, outright."""
+    shape, wt, prompt, forced, tr = _case(name)
+    worst = _run_logits(cass, shape, wt, tr, prompt, forced)
+    print(f"{name}: worst logit error / RMS: {worst}")

@@ -252,3 +252,83 @@ def test_draft_layer_reads_the_draft_view_only():
     k1, v1, kd1, vd1 = z(), z(), z(), z()
     b = model.layer(lw, shape, _bits(hs[0]), 0, k1, v1, kd1, vd1, True, 0, 0)
     assert np.array_equal(a, b) and np.array_equal(kd0[0], k0[0]) and not k1.any()
+
+
+# ------------------------------------------------------------------------------------------- sampling acceptance (Eq. 1)
+
+
+def _chi_square(counts, probs):
+    n = counts.sum()
+    exp = probs * n
+    return float(((counts - exp) ** 2 / exp).sum())
+
+
+def test_sampling_accept_preserves_the_target_distribution():
+    """Sec. 2.2: with rejection sampling the emitted tokens are distributed exactly as the target's.  16-symbol
+    vocabulary, gamma = 1: draw x ~ q, run Eq. 1, histogram the first emitted token over 1e5 draws; chi-square against p
+    (15 degrees of freedom: 37.7 is the 0.1 % point).  A rule that resampled from p instead of the positive part of
+    p - q, or that accepted on r < q/p, fails by a wide margin."""
+    rng = np.random.default_rng(0)
+    V, N = 16, 100_000
+    p = rng.dirichlet(np.ones(V) * 0.7)
+    q = rng.dirichlet(np.ones(V) * 0.7)
+    p2 = rng.dirichlet(np.ones(V))
+    xs = rng.choice(V, size=N, p=q)
+    r = rng.uniform(size=N)
+    u = rng.uniform(size=N)
+    first = np.zeros(V)
+    n_acc = 0
+    for i in range(N):
+        n, toks = model.sampling_accept(np.stack([p, p2]), q[None], [int(xs[i])], r[i: i + 1], u[i])
+        first[toks[0]] += 1
+        n_acc += n
+    assert _chi_square(first, p) < 37.7
+    # acceptance probability of one draft = sum_x min(p(x), q(x))
+    assert abs(n_acc / N - np.minimum(p, q).sum()) < 4 * np.sqrt(0.25 / N)
+    # a wrong rule, planted here on the CPU: resample from p after a rejection -> the histogram leaves p
+    wrong = np.zeros(V)
+    for i in range(20000):
+        x = int(xs[i])
+        wrong[x if r[i] * q[x] <= p[x] else model.inverse_cdf_sample(p, u[i])] += 1
+    assert _chi_square(wrong, p) > 37.7
+
+
+def test_sampling_accept_longer_drafts_and_special_cases():
+    rng = np.random.default_rng(1)
+    V, g = 8, 3
+    # the second emitted token, given that the first draft was accepted, follows the target's second distribution
+    p = rng.dirichlet(np.ones(V), size=g + 1)
+    q = rng.dirichlet(np.ones(V), size=g)
+    hist, hits = np.zeros(V), 0
+    for _ in range(60000):
+        xs = [int(rng.choice(V, p=q[i])) for i in range(g)]
+        n, toks = model.sampling_accept(p, q, xs, rng.uniform(size=g), rng.uniform())
+        assert len(toks) == n + 1 and toks[:n] == xs[:n]
+        if n >= 1:
+            hist[toks[1]] += 1
+            hits += 1
+    assert _chi_square(hist, p[1]) < 24.3                    # 7 degrees of freedom, 0.1 % point
+    # Eq. 1 by brute force on random inputs
+    for _ in range(300):
+        xs = rng.integers(0, V, g).tolist()
+        r = rng.uniform(size=g)
+        n, _ = model.sampling_accept(p, q, xs, r, 0.5)
+        want = g
+        for i in range(1, g + 1):
+            if r[i - 1] > p[i - 1, xs[i - 1]] / q[i - 1, xs[i - 1]]:
+                want = i - 1
+                break
+        assert n == want
+    # identical models: every draft accepted, the extra token comes from p_{gamma+1}
+    n, toks = model.sampling_accept(p, p[:g], [1, 2, 3], np.array([0.999, 0.999, 0.999]), 0.0)
+    assert n == g and toks[-1] == 0
+    # one-hot distributions: the greedy rule of Sec. 2.2 (accept identical tokens, emit the target's choice)
+    eye = np.eye(V)
+    tgt, drf = [3, 5, 1, 7], [3, 5, 2]
+    n, toks = model.sampling_accept(eye[tgt], eye[drf], drf, rng.uniform(0.01, 0.99, 3), 0.3)
+    assert n == model.greedy_accept(drf, tgt) == 2 and toks == [3, 5, 1]
+    # inverse-CDF draw: lowest index whose cumulative weight exceeds u * total
+    w = np.array([0.0, 2.0, 0.0, 1.0, 1.0])
+    assert [model.inverse_cdf_sample(w, u) for u in (0.0, 0.49, 0.5, 0.74, 0.75, 0.999)] == [1, 1, 3, 3, 4, 4]
+    assert np.allclose(model.softmax(np.log(w[[1, 3, 4]]), 1.0), [0.5, 0.25, 0.25])
+    assert np.allclose(model.softmax(np.log(w[[1, 3, 4]]), 0.5), np.array([4.0, 1.0, 1.0]) / 6.0)
