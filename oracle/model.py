@@ -140,13 +140,15 @@ def swiglu(gate_bits: np.ndarray, up_bits: np.ndarray) -> np.ndarray:
 
 
 def layer(lw: dict, shape, h_bits: np.ndarray, pos: int, k_cache: np.ndarray, v_cache: np.ndarray,
-          kd_cache: np.ndarray, vd_cache: np.ndarray, draft: bool, kv_p: int, kv_t: int, note=None) -> np.ndarray:
+          kd_cache: np.ndarray, vd_cache: np.ndarray, draft: bool, kv_p: int, kv_t: int, note=None,
+          probe: dict | None = None) -> np.ndarray:
     """One decoder layer for the token at `pos` (pre-norm residual blocks: attention, then SwiGLU FFN).
 
     lw: the layer's matrices (accumulation type) and norm gains (bf16 bits); h_bits: bf16 hidden state;
     k_cache/v_cache [max_seq, n_kv, d]: the target's bf16 cache of this layer, kd_cache/vd_cache: the draft's view.
     The draft view of the new K/V is written at `pos` in both modes, the bf16 cache only in target mode.
-    `note(names, x_bits)` sees the input of each projection (Wanda calibration).  Returns the new hidden state."""
+    `note(names, x_bits)` sees the input of each projection (Wanda calibration); `probe`, when given, receives the
+    bf16 attention output and SwiGLU output (the inputs of wo and wd).  Returns the new hidden state."""
     s = shape
     d = s.head_dim
     xn = rmsnorm(h_bits, lw["norm_attn"], s.rms_eps)
@@ -175,6 +177,8 @@ def layer(lw: dict, shape, h_bits: np.ndarray, pos: int, k_cache: np.ndarray, v_
     act = swiglu(_r(lw["wg"] @ x), _r(lw["wu"] @ x))
     if note:
         note(("wd",), act)
+    if probe is not None:
+        probe["attn_out"], probe["act"] = ob, act
     down = _r(lw["wd"] @ _f(act))
     return _r(_f(h) + _f(down))
 
@@ -188,10 +192,10 @@ def lm_logits(W: Weights, h_bits: np.ndarray, calib: dict | None = None) -> np.n
 
 
 def forward_token(W: Weights, kv: KVCache, tok: int, pos: int, draft: bool, kv_p: int, kv_t: int,
-                  calib: dict | None = None, hidden_out: list | None = None):
+                  calib: dict | None = None, hidden_out: list | None = None, probes: list | None = None):
     """One token at position `pos`.  Target mode writes K/V in both forms at `pos`; draft mode
     writes only the draft view.  Returns the fp64 logits.  `hidden_out`, when given, receives the bf16 hidden
-    state entering every layer and the one entering the final norm."""
+    state entering every layer and the one entering the final norm; `probes` one dict per layer (see `layer`)."""
     h = W.embed_bits[tok].copy()
     for li, lw in enumerate(W.layers):
         if hidden_out is not None:
@@ -202,7 +206,11 @@ def forward_token(W: Weights, kv: KVCache, tok: int, pos: int, draft: bool, kv_p
                 x = _f(x_bits)
                 for nm in names:
                     calib["layers"][li][nm] += x * x
-        h = layer(lw, W.shape, h, pos, kv.k[li], kv.v[li], kv.kd[li], kv.vd[li], draft, kv_p, kv_t, note)
+        probe = None
+        if probes is not None:
+            probe = {}
+            probes.append(probe)
+        h = layer(lw, W.shape, h, pos, kv.k[li], kv.v[li], kv.kd[li], kv.vd[li], draft, kv_p, kv_t, note, probe)
     if hidden_out is not None:
         hidden_out.append(h.copy())
     return lm_logits(W, h, calib)
