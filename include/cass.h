@@ -45,10 +45,13 @@ enum { CASS_KV_BF16 = 1, CASS_KV_COMPRESSED = 2 };
 typedef struct cass_format {
     int mode;                /* weights: 1 = Cassandra-1 (unary exponent code, lossless for the kept bits),
                               * 2 = Cassandra-2 (Sec. 4.2: MX, blocks of 32 kept values share an exponent, MXINT
-                              * elements; see cass_encode_weights).  The KV cache is Cassandra-1 in both modes. */
+                              * elements; see cass_encode_weights). */
     int w_prune_permille, w_trunc_bits;
     int kv_prune_permille, kv_trunc_bits;
     int w_seg_cols, w_chunk_cols;
+    int kv_mode;             /* compressed KV cache: 0 or 1 = Cassandra-1 records (unary exponent code), 2 = Cassandra-2
+                              * records (Sec. 4.2: the kept values among 32 consecutive channels of a head share one
+                              * exponent byte; elements as for the weights); see cass_kv_append */
 } cass_format;
 
 typedef struct cass_model_desc {
@@ -220,7 +223,14 @@ size_t cass_calib_norms_count(const cass_model_desc* desc);
  * (flags).  K, V: bf16 [n_new][n_kv_heads][head_dim]; K is expected post-RoPE.  Per token and head the
  * floor(d*p/1000) smallest |x| are pruned (ties: lower channel first).  Positions must be appended in
  * order: start_pos may not exceed the number of positions already in the compressed cache of that layer.
- * The compressed cache uses the layer's frozen codebooks (cass_kv_build_codebook). */
+ * The compressed cache uses the layer's frozen codebooks (cass_kv_build_codebook).
+ * Record of one (token, head, K|V) in the compressed cache, kv_mode 1: entry words (a 10-bit code-bit offset for every
+ * 32-channel slice after the first, three per word from bit 29 down: the d/32 slices of a record decode side by side;
+ * bit 31 of the first word = raw flag), bitmap, sign+mantissa fields, and in the arena the unary exponent stream -- or,
+ * when that stream would take more than min(8 * kept, 1023) bits, the kept exponents as raw bytes, so that a record
+ * never takes more than ceil(8 * kept / 32) arena words and the arena is sized for that: a codebook that fits the later
+ * tokens badly costs bytes, never capacity.  kv_mode 2: bitmap, fields (sign + high 7-t bits of the MXINT magnitude)
+ * and one shared exponent byte per 32-channel slice; fixed size, no arena use, no codebook. */
 int cass_kv_append(void* session, int seq, int layer, const void* K_bf16, const void* V_bf16, int start_pos, int n_new,
                    int flags, void* stream);
 

@@ -44,7 +44,11 @@ Weight blob  (rows N x cols K, row-major source)
       unary        W_u words/row  (max over the 32 rows)
 
 KV record (one token, one KV head, K or V; d = head_dim)
-  bitmap d/32 words, fields W_f = ceil(kept/per_word) words, unary: variable word count.
+  fixed part: entry words (see kv_entry_words: a 10-bit code-bit offset for every 32-channel slice after the first,
+  so that d/32 decoders can work on one record side by side; bit 31 of the first word = raw-exponent flag),
+  bitmap d/32 words, fields W_f = ceil(kept/per_word) words;
+  exponent part (variable word count): the unary stream, or -- when that stream would be longer than 8 bits per
+  kept value or than 1023 bits -- the kept values' exponents as raw bytes, four per word from the top.
 """
 from __future__ import annotations
 
@@ -375,35 +379,99 @@ def blob_section_bits(blob: np.ndarray) -> dict:
 # --------------------------------------------------------------------------------------
 
 
+KV_RAW_FLAG = 0x80000000
+
+
+def kv_entry_words(d: int) -> int:
+    """Words holding the entry points of a record: one 10-bit code offset for each 32-channel slice after the first,
+    three per word (from bit 29 downwards); bit 31 of the first word flags a record with raw exponents."""
+    return max(1, (d // 32 - 1 + 2) // 3)
+
+
 def kv_fixed_words(d: int, p: int, t: int) -> int:
     kept = d - codec.n_pruned(d, p)
-    return d // 32 + (kept + fields_per_word(t) - 1) // fields_per_word(t)
+    return kv_entry_words(d) + d // 32 + (kept + fields_per_word(t) - 1) // fields_per_word(t)
+
+
+def kv_code_budget(kept: int) -> int:
+    """A record keeps its unary codewords as long as they take no more bits than raw 8-bit exponents would and its
+    slice offsets fit their 10-bit entries; beyond that the exponents are stored raw (one byte per kept value)."""
+    return min(8 * kept, 1023)
+
+
+def kv_arena_words_max(d: int, p: int) -> int:
+    kept = d - codec.n_pruned(d, p)
+    return (8 * kept + 31) // 32
+
+
+def pack_bytes_msb(b: np.ndarray) -> np.ndarray:
+    """Bytes -> words, four per word from the most significant end."""
+    b = np.asarray(b, dtype=np.uint32)
+    n_words = (b.size + 3) // 4
+    padded = np.zeros(n_words * 4, dtype=np.uint32)
+    padded[: b.size] = b
+    padded = padded.reshape(n_words, 4)
+    return (padded[:, 0] << 24) | (padded[:, 1] << 16) | (padded[:, 2] << 8) | padded[:, 3]
 
 
 def encode_kv_token(x_bits: np.ndarray, p: int, t: int, exp_to_rank: np.ndarray):
-    """One token, one head: returns (bitmap words, field words, unary words)."""
+    """One token, one head: returns (fixed part: entry words | bitmap words | field words, exponent words of the
+    arena: the unary stream, or raw exponent bytes when the stream would exceed its budget).
+
+    The entry words make a record decodable by d/32 parallel decoders, one per 32-channel slice (the software form
+    of the per-section cursors of Sec. 5.3): slice s > 0 starts at the record's kept value number popcount(bitmap
+    words < s), whose codeword starts at the bit offset stored for it."""
     x_bits = np.asarray(x_bits, dtype=np.uint16)
+    d = x_bits.size
     keep = codec.keep_mask_kv(x_bits, p)
     idx = np.flatnonzero(keep)
     _, e, _ = codec.split_fields(x_bits[idx])
-    ranks = np.asarray(exp_to_rank)[e]
-    return (bits_to_words(keep.astype(np.uint8)),
-            _pack_fields_fast(codec.spec_field(x_bits[idx], t), t),
-            bits_to_words(codec.unary_encode_fast(ranks)) if idx.size else np.zeros(0, np.uint32))
+    ranks = np.asarray(exp_to_rank)[e].astype(np.int64)
+    entry = np.zeros(kv_entry_words(d), dtype=np.uint32)
+    total = int((ranks + 1).sum())
+    if total <= kv_code_budget(idx.size):
+        cum = np.concatenate(([0], np.cumsum(ranks + 1)))
+        for s in range(1, d // 32):
+            first = int(np.searchsorted(idx, 32 * s))          # kept values in channels below 32 s
+            entry[(s - 1) // 3] |= np.uint32(int(cum[first]) << (20 - 10 * ((s - 1) % 3)))
+        arena = bits_to_words(codec.unary_encode_fast(ranks)) if idx.size else np.zeros(0, np.uint32)
+    else:
+        entry[0] |= np.uint32(KV_RAW_FLAG)
+        arena = pack_bytes_msb(e)
+    fixed = np.concatenate([entry, bits_to_words(keep.astype(np.uint8)), _pack_fields_fast(codec.spec_field(x_bits[idx], t), t)])
+    return fixed.astype(np.uint32), arena.astype(np.uint32)
 
 
-def decode_kv_token(bm_words, field_words, unary_words, d: int, t: int, rank_to_exp: np.ndarray) -> np.ndarray:
+def decode_kv_token(fixed, arena, d: int, p: int, t: int, rank_to_exp: np.ndarray, by_slices: bool = False) -> np.ndarray:
+    """Zero-padded reconstruction of a record.  by_slices: decode every 32-channel slice on its own, entering the
+    exponent stream at the slice's stored offset (what parallel decoders do); the result is the same."""
+    fixed = np.asarray(fixed, dtype=np.uint32)
+    n_e, n_b = kv_entry_words(d), d // 32
+    entry, bm_words, field_words = fixed[:n_e], fixed[n_e: n_e + n_b], fixed[n_e + n_b:]
     keep = words_to_bits(bm_words)[:d].astype(bool)
     idx = np.flatnonzero(keep)
     out = np.zeros(d, dtype=np.uint16)
     if idx.size == 0:
         return out
     fields = unpack_fields(field_words, idx.size, t)
-    ranks = codec.unary_decode_fast(words_to_bits(unary_words), idx.size)
-    e = np.asarray(rank_to_exp)[ranks].astype(np.uint16)
-    s = (fields >> (7 - t)).astype(np.uint16) & 1
+    raw = bool(int(entry[0]) & KV_RAW_FLAG)
+    if raw:
+        by = words_to_bits(arena).reshape(-1, 8)
+        e = (by.astype(np.uint16) << np.arange(7, -1, -1, dtype=np.uint16)[None, :]).sum(axis=1)[: idx.size].astype(np.uint16)
+    elif not by_slices:
+        e = np.asarray(rank_to_exp)[codec.unary_decode_fast(words_to_bits(arena), idx.size)].astype(np.uint16)
+    else:
+        bits = words_to_bits(arena)
+        e = np.zeros(idx.size, dtype=np.uint16)
+        for s in range(n_b):
+            first = int(np.searchsorted(idx, 32 * s))
+            cnt = int(np.searchsorted(idx, 32 * (s + 1))) - first
+            off = 0 if s == 0 else (int(entry[(s - 1) // 3]) >> (20 - 10 * ((s - 1) % 3))) & 0x3FF
+            if cnt:
+                e[first: first + cnt] = np.asarray(rank_to_exp)[codec.unary_decode_fast(bits[off:], cnt)]
+    s_ = (fields >> (7 - t)).astype(np.uint16) & 1
     m_hi = (fields & ((1 << (7 - t)) - 1)).astype(np.uint16)
-    out[idx] = (s << 15) | (e << 7) | (m_hi << t)
+    out[idx] = (s_ << 15) | (e << 7) | (m_hi << t)
     return out
 
 

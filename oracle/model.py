@@ -139,9 +139,19 @@ def swiglu(gate_bits: np.ndarray, up_bits: np.ndarray) -> np.ndarray:
     return _r(gate / (_ACC(1.0) + np.exp(-gate)) * up)
 
 
+def kv_draft_view(x_bits: np.ndarray, kv_p: int, kv_t: int, kv_mode: int = 1) -> np.ndarray:
+    """What the draft model sees of K or V [..., d]: pruned per token and head by magnitude, mantissas truncated;
+    exponents exact (kv_mode 1, Cassandra-1) or shared per 32 channels (kv_mode 2, Cassandra-2: `mx.kv_draft_bits`)."""
+    keep = codec.keep_mask_kv(x_bits, kv_p)
+    if kv_mode == 2:
+        from . import mx
+        return mx.kv_draft_bits(x_bits, keep, kv_t)
+    return codec.draft_bits(x_bits, keep, kv_t)
+
+
 def layer(lw: dict, shape, h_bits: np.ndarray, pos: int, k_cache: np.ndarray, v_cache: np.ndarray,
           kd_cache: np.ndarray, vd_cache: np.ndarray, draft: bool, kv_p: int, kv_t: int, note=None,
-          probe: dict | None = None) -> np.ndarray:
+          probe: dict | None = None, kv_mode: int = 1) -> np.ndarray:
     """One decoder layer for the token at `pos` (pre-norm residual blocks: attention, then SwiGLU FFN).
 
     lw: the layer's matrices (accumulation type) and norm gains (bf16 bits); h_bits: bf16 hidden state;
@@ -160,8 +170,8 @@ def layer(lw: dict, shape, h_bits: np.ndarray, pos: int, k_cache: np.ndarray, v_
     v = _r(lw["wv"] @ x).reshape(s.n_kv_heads, d)
     q = rope(q, pos, s.rope_theta)
     k = rope(k, pos, s.rope_theta)
-    kd_cache[pos] = codec.draft_bits(k, codec.keep_mask_kv(k, kv_p), kv_t)
-    vd_cache[pos] = codec.draft_bits(v, codec.keep_mask_kv(v, kv_p), kv_t)
+    kd_cache[pos] = kv_draft_view(k, kv_p, kv_t, kv_mode)
+    vd_cache[pos] = kv_draft_view(v, kv_p, kv_t, kv_mode)
     if not draft:
         k_cache[pos], v_cache[pos] = k, v
     o = attention(q, (kd_cache if draft else k_cache)[: pos + 1], (vd_cache if draft else v_cache)[: pos + 1])
@@ -192,7 +202,8 @@ def lm_logits(W: Weights, h_bits: np.ndarray, calib: dict | None = None) -> np.n
 
 
 def forward_token(W: Weights, kv: KVCache, tok: int, pos: int, draft: bool, kv_p: int, kv_t: int,
-                  calib: dict | None = None, hidden_out: list | None = None, probes: list | None = None):
+                  calib: dict | None = None, hidden_out: list | None = None, probes: list | None = None,
+                  kv_mode: int = 1):
     """One token at position `pos`.  Target mode writes K/V in both forms at `pos`; draft mode
     writes only the draft view.  Returns the fp64 logits.  `hidden_out`, when given, receives the bf16 hidden
     state entering every layer and the one entering the final norm; `probes` one dict per layer (see `layer`)."""
@@ -210,7 +221,7 @@ def forward_token(W: Weights, kv: KVCache, tok: int, pos: int, draft: bool, kv_p
         if probes is not None:
             probe = {}
             probes.append(probe)
-        h = layer(lw, W.shape, h, pos, kv.k[li], kv.v[li], kv.kd[li], kv.vd[li], draft, kv_p, kv_t, note, probe)
+        h = layer(lw, W.shape, h, pos, kv.k[li], kv.v[li], kv.kd[li], kv.vd[li], draft, kv_p, kv_t, note, probe, kv_mode)
     if hidden_out is not None:
         hidden_out.append(h.copy())
     return lm_logits(W, h, calib)
@@ -229,11 +240,11 @@ def calib_to_norms(calib: dict) -> dict:
             "lm_head": np.sqrt(calib["lm_head"]).astype(np.float32)}
 
 
-def prefill(W: Weights, kv: KVCache, prompt, kv_p: int, kv_t: int, calib: dict | None = None):
+def prefill(W: Weights, kv: KVCache, prompt, kv_p: int, kv_t: int, calib: dict | None = None, kv_mode: int = 1):
     """Target pass over the prompt; returns the logits of the last prompt token."""
     logits = None
     for pos, tok in enumerate(prompt):
-        logits = forward_token(W, kv, int(tok), pos, False, kv_p, kv_t, calib)
+        logits = forward_token(W, kv, int(tok), pos, False, kv_p, kv_t, calib, kv_mode=kv_mode)
     kv.n = len(prompt)
     return logits
 
@@ -286,13 +297,13 @@ def sampling_accept(p: np.ndarray, q: np.ndarray, draft_tokens, r: np.ndarray, u
     return n, [int(t) for t in draft_tokens[:n]] + [extra]
 
 
-def plain_greedy(W: Weights, kv: KVCache, first_tok: int, n_tokens: int, kv_p: int, kv_t: int):
+def plain_greedy(W: Weights, kv: KVCache, first_tok: int, n_tokens: int, kv_p: int, kv_t: int, kv_mode: int = 1):
     """Autoregressive decoding with the target only.  `first_tok` is the token predicted from the
     prompt; returns the n_tokens tokens that follow it."""
     out = []
     tok = first_tok
     for _ in range(n_tokens):
-        logits = forward_token(W, kv, tok, kv.n, False, kv_p, kv_t)
+        logits = forward_token(W, kv, tok, kv.n, False, kv_p, kv_t, kv_mode=kv_mode)
         kv.n += 1
         tok = argmax_lowest(logits)
         out.append(tok)
@@ -300,7 +311,7 @@ def plain_greedy(W: Weights, kv: KVCache, first_tok: int, n_tokens: int, kv_p: i
 
 
 def speculative_greedy(W: Weights, Wd, kv: KVCache, first_tok: int, n_tokens: int, gamma: int,
-                       kv_p: int, kv_t: int, draft_fn=None, trace=None):
+                       kv_p: int, kv_t: int, draft_fn=None, trace=None, kv_mode: int = 1):
     """Draft gamma tokens, verify gamma+1 rows with the target, accept the matching prefix,
     emit the target's token at the first mismatch (or its bonus token), roll the cache back.
 
@@ -316,13 +327,13 @@ def speculative_greedy(W: Weights, Wd, kv: KVCache, first_tok: int, n_tokens: in
             if draft_fn is not None:
                 nxt = int(draft_fn(i, tok, n + i))
             else:
-                nxt = argmax_lowest(forward_token(Wd, kv, tok, n + i, True, kv_p, kv_t))
+                nxt = argmax_lowest(forward_token(Wd, kv, tok, n + i, True, kv_p, kv_t, kv_mode=kv_mode))
             drafts.append(nxt)
             tok = nxt
         rows = [last] + drafts
         targ = []
         for i, tk in enumerate(rows):                 # batched verification == row-by-row causal pass
-            targ.append(argmax_lowest(forward_token(W, kv, tk, n + i, False, kv_p, kv_t)))
+            targ.append(argmax_lowest(forward_token(W, kv, tk, n + i, False, kv_p, kv_t, kv_mode=kv_mode)))
         a = greedy_accept(drafts, targ)
         emitted = drafts[:a] + [targ[a]]
         out.extend(emitted)

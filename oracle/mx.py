@@ -241,3 +241,91 @@ def blob_section_bits(info: dict, t: int) -> dict:
     """Content bits of a blob (closed form): bitmap, fields, shared exponents."""
     return {"bitmap": info["rows"] * info["cols"], "fields": info["rows"] * info["kept_per_row"] * (8 - t),
             "exponents": 8 * info["exponent_blocks"]}
+
+
+# ---- Cassandra-2 KV records (Sec. 4.2: the MX exponent compression applies to the KV cache as it does to the weights) ----
+# Pruning (per token and head, by magnitude), bitmap and mantissa truncation as for Cassandra-1 records.  Reading K1
+# (the paper leaves the block open): the values that share an exponent are the KEPT values among 32 consecutive
+# channels of the head -- the 32-element block of the OCP formats laid over the channel axis -- so a record of a head
+# of d channels carries d/32 exponent bytes, and the d/32 slices of a record decode independently of one another.
+# Elements, truncation and the draft value follow M2-M6 above.
+# Record = bitmap d/32 words | fields (8-t bits each, floor(32/(8-t)) per word, from the most significant end) |
+# exponent bytes (four per word from the most significant end); fixed size, no exponent stream.
+
+
+def kv_fields(x_bits: np.ndarray, keep: np.ndarray, t: int):
+    """One token, one head -> (slice exponents uint8 [d/32], fields of the kept values in channel order)."""
+    x_bits = np.asarray(x_bits, dtype=np.uint16)
+    d = x_bits.size
+    s, e, m = (v.astype(np.int64) for v in codec.split_fields(x_bits))
+    exps = np.zeros(d // 32, dtype=np.uint8)
+    fields = []
+    for b in range(d // 32):
+        sl = slice(32 * b, 32 * b + 32)
+        kb = np.asarray(keep[sl], dtype=bool)
+        if not kb.any():
+            continue
+        E = int(e[sl][kb].max())
+        exps[b] = E
+        sh = 1 + E - e[sl][kb]
+        m7 = np.where((sh < 8) & (e[sl][kb] > 0) & (E >= 7), (0x80 | m[sl][kb]) >> np.minimum(sh, 8), 0)
+        fields.append((s[sl][kb] << (7 - t)) | (m7 >> t))
+    fields = np.concatenate(fields).astype(np.uint32) if fields else np.zeros(0, np.uint32)
+    return exps, fields
+
+
+def kv_value_bits(exps: np.ndarray, fields: np.ndarray, keep: np.ndarray, t: int) -> np.ndarray:
+    """Zero-padded draft values of one record as bf16 bit patterns [d]."""
+    keep = np.asarray(keep, dtype=bool)
+    d = keep.size
+    out = np.zeros(d, dtype=np.uint16)
+    k0 = 0
+    for b in range(d // 32):
+        idx = np.flatnonzero(keep[32 * b: 32 * b + 32])
+        if idx.size:
+            f = np.asarray(fields[k0: k0 + idx.size], dtype=np.int64)
+            sign, mag = f >> (7 - t), (f & ((1 << (7 - t)) - 1)) << t
+            for i, c in enumerate(idx):
+                g = int(mag[i])
+                if g:
+                    top = g.bit_length() - 1
+                    out[32 * b + c] = (int(sign[i]) << 15) | ((int(exps[b]) - 6 + top) << 7) | ((g << (7 - top)) & 0x7F)
+            k0 += idx.size
+    return out
+
+
+def kv_draft_bits(x_bits: np.ndarray, keep: np.ndarray, t: int) -> np.ndarray:
+    """Draft view of K or V [..., d] under Cassandra-2 (per record: kv_fields then kv_value_bits)."""
+    x_bits = np.asarray(x_bits, dtype=np.uint16)
+    keep = np.asarray(keep, dtype=bool)
+    flat_x, flat_k = x_bits.reshape(-1, x_bits.shape[-1]), keep.reshape(-1, x_bits.shape[-1])
+    out = np.zeros_like(flat_x)
+    for i in range(flat_x.shape[0]):
+        exps, fields = kv_fields(flat_x[i], flat_k[i], t)
+        out[i] = kv_value_bits(exps, fields, flat_k[i], t)
+    return out.reshape(x_bits.shape)
+
+
+def kv_fixed_words(d: int, p: int, t: int) -> int:
+    kept = d - codec.n_pruned(d, p)
+    per = 32 // (8 - t)
+    return d // 32 + (kept + per - 1) // per + (d // 32 + 3) // 4
+
+
+def encode_kv_token(x_bits: np.ndarray, p: int, t: int) -> np.ndarray:
+    x_bits = np.asarray(x_bits, dtype=np.uint16)
+    keep = codec.keep_mask_kv(x_bits, p)
+    exps, fields = kv_fields(x_bits, keep, t)
+    return np.concatenate([layout.bits_to_words(keep.astype(np.uint8)), pack_fields(fields, t), pack_bytes(exps)]).astype(np.uint32)
+
+
+def decode_kv_token(words: np.ndarray, d: int, p: int, t: int) -> np.ndarray:
+    words = np.asarray(words, dtype=np.uint32)
+    kept = d - codec.n_pruned(d, p)
+    per = 32 // (8 - t)
+    n_b, n_f = d // 32, (kept + per - 1) // per
+    keep = layout.words_to_bits(words[:n_b])[:d].astype(bool)
+    fields = unpack_fields(words[n_b: n_b + n_f], int(keep.sum()), t)
+    ew = words[n_b + n_f:]
+    exps = np.array([(int(ew[b // 4]) >> (24 - 8 * (b % 4))) & 0xFF for b in range(n_b)], dtype=np.uint8)
+    return kv_value_bits(exps, fields, keep, t)

@@ -29,11 +29,11 @@ class CassError(RuntimeError):
 class Format(C.Structure):
     _fields_ = [("mode", C.c_int), ("w_prune_permille", C.c_int), ("w_trunc_bits", C.c_int),
                 ("kv_prune_permille", C.c_int), ("kv_trunc_bits", C.c_int), ("w_seg_cols", C.c_int),
-                ("w_chunk_cols", C.c_int)]
+                ("w_chunk_cols", C.c_int), ("kv_mode", C.c_int)]
 
 
-def default_format(w_p=400, w_t=4, kv_p=400, kv_t=4, seg_cols=0, chunk_cols=0, mode=1) -> Format:
-    return Format(mode, w_p, w_t, kv_p, kv_t, seg_cols, chunk_cols)
+def default_format(w_p=400, w_t=4, kv_p=400, kv_t=4, seg_cols=0, chunk_cols=0, mode=1, kv_mode=1) -> Format:
+    return Format(mode, w_p, w_t, kv_p, kv_t, seg_cols, chunk_cols, kv_mode)
 
 
 class ModelDesc(C.Structure):

@@ -1,24 +1,30 @@
 // Draft decode attention over the compressed KV cache (Sec. 4.1 draft inference; KV speculation data of
-// Sec. 4.2): grouped-query attention of one query row, split over the sequence in fixed 64-token chunks with a
-// log-sum-exp merge.  One CTA = one (KV head, chunk): warps 0-1 decode the K records of 32 tokens each (lane =
-// token) and form q.k for all query heads of the group, warps 2-3 decode the V records of the same tokens into a
-// dense bf16 tile in shared memory; then the chunk's probabilities multiply the tile.  Records are walked like
-// the weight streams: 8 kept values per 32-bit bitmap window, 4 codewords per 32-bit unary window, with a
-// careful walk for the rare group that does not fit its windows.
+// Sec. 4.2): grouped-query attention of one query row per sequence, split over the sequence with a log-sum-exp
+// merge.  One CTA = one (KV head, run of 32..256 tokens); it walks its run in passes of 32 tokens (one block of the
+// cache's fixed part) with a running softmax.  Inside a pass a record (token, K|V) is decoded by d/32 lanes side by
+// side, one per 32-channel slice: warp (kind, slice) has lane = token, so every stream read is conflict free; a
+// slice enters the record through its bitmap word, the popcount of the lower bitmap words (field index) and, for
+// Cassandra-1 records, the code-bit offset its entry word holds -- the software form of the per-section cursors
+// of Sec. 5.3.  K slices leave partial dot products with the group's query heads, V slices a dense bf16 tile; then
+// the pass's probabilities multiply the tile.
 #include <type_traits>
 
 #include "kernels.cuh"
 
 namespace cass {
 
-constexpr int kDaTok = kAttnChunk;            // tokens per CTA
-constexpr int kDaThreads = 128;
-constexpr int kDaUnaStage = 12;               // staged unary words per token (a typical record has 5-8); longer records are read in place
+constexpr int kDaSub = 32;                    // tokens per pass
+constexpr int kDaUnaStageMax = 32;            // staged exponent words per token (records up to 1023 code bits fit)
 constexpr int kMaxGroup = 8;                  // query heads per KV head
 
-__device__ __forceinline__ uint32_t da_shl(uint32_t v, uint32_t s) {
+__device__ __forceinline__ uint32_t da_shl(uint32_t v, uint32_t s) {          // shift counts >= 32 give 0
     uint32_t r;
     asm("shl.b32 %0, %1, %2;" : "=r"(r) : "r"(v), "r"(s));
+    return r;
+}
+__device__ __forceinline__ uint32_t da_bfind(uint32_t v) {                    // most significant set bit, 0xFFFFFFFF if none
+    uint32_t r;
+    asm("bfind.u32 %0, %1;" : "=r"(r) : "r"(v));
     return r;
 }
 __device__ __forceinline__ uint32_t da_lds(uint32_t a) {
@@ -27,280 +33,321 @@ __device__ __forceinline__ uint32_t da_lds(uint32_t a) {
     return v;
 }
 
-// What happens to a decoded value.  K: multiply with the query tile; V: store into the token's dense row.
-// GQ = query heads the tile has room for (4 or 8): q_s[col][GQ] floats.
+// What happens to a decoded value of channel `col` (0..31 inside the slice).
+// K: multiply with the query tile q_s[channel][GQ]; V: store into the token's dense row.
 template <int GQ>
 struct EmitK {
-    float acc[GQ], g[GQ];
-    uint32_t q_a;
-    __device__ __forceinline__ void reset() {
-#pragma unroll
-        for (int i = 0; i < GQ; ++i) g[i] = 0.f;
-    }
-    __device__ __forceinline__ void fma_into(float (&dst)[GQ], uint32_t off, uint32_t wb) {
-        const float w = __uint_as_float(wb);
-        float4 a;
-        asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(a.x), "=f"(a.y), "=f"(a.z), "=f"(a.w) : "r"(q_a + off));
-        dst[0] = fmaf(w, a.x, dst[0]); dst[1] = fmaf(w, a.y, dst[1]); dst[2] = fmaf(w, a.z, dst[2]); dst[3] = fmaf(w, a.w, dst[3]);
-        if constexpr (GQ > 4) {
-            float4 b;
-            asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4+16];" : "=f"(b.x), "=f"(b.y), "=f"(b.z), "=f"(b.w) : "r"(q_a + off));
-            dst[4] = fmaf(w, b.x, dst[4]); dst[5] = fmaf(w, b.y, dst[5]); dst[6] = fmaf(w, b.z, dst[6]); dst[7] = fmaf(w, b.w, dst[7]);
-        }
-    }
-    template <int E>
-    __device__ __forceinline__ void elem(uint32_t off, uint32_t wb, bool valid) { if (valid) fma_into(g, off, wb); }
-    __device__ __forceinline__ void commit(int) {
-#pragma unroll
-        for (int i = 0; i < GQ; ++i) acc[i] += g[i];
-    }
-    __device__ __forceinline__ void direct(uint32_t off, uint32_t wb) { fma_into(acc, off, wb); }
-    __device__ __forceinline__ void restart() {
+    float acc[GQ];
+    uint32_t q_a;                        // shared address of the slice's first channel in the query tile
+    __device__ __forceinline__ void init() {
 #pragma unroll
         for (int i = 0; i < GQ; ++i) acc[i] = 0.f;
+    }
+    __device__ __forceinline__ void put(uint32_t col, float w) {
+        float4 a;
+        asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(a.x), "=f"(a.y), "=f"(a.z), "=f"(a.w) : "r"(q_a + col * (GQ * 4)));
+        acc[0] = fmaf(w, a.x, acc[0]); acc[1] = fmaf(w, a.y, acc[1]); acc[2] = fmaf(w, a.z, acc[2]); acc[3] = fmaf(w, a.w, acc[3]);
+        if constexpr (GQ > 4) {
+            float4 b;
+            asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4+16];" : "=f"(b.x), "=f"(b.y), "=f"(b.z), "=f"(b.w) : "r"(q_a + col * (GQ * 4)));
+            acc[4] = fmaf(w, b.x, acc[4]); acc[5] = fmaf(w, b.y, acc[5]); acc[6] = fmaf(w, b.z, acc[6]); acc[7] = fmaf(w, b.w, acc[7]);
+        }
     }
 };
 
 struct EmitV {
-    uint32_t row_a;                      // shared address of the token's dense row
-    uint32_t off[kGroupCols], wb[kGroupCols];
-    __device__ __forceinline__ void reset() {}
-    template <int E>
-    __device__ __forceinline__ void elem(uint32_t o, uint32_t w, bool) { off[E] = o; wb[E] = w; }
-    __device__ __forceinline__ void commit(int cnt) {
-#pragma unroll
-        for (int e = 0; e < kGroupCols; ++e)
-            if (e < cnt) asm volatile("st.shared.u16 [%0], %1;" ::"r"(row_a + off[e]), "h"((uint16_t)(wb[e] >> 16)));
+    uint32_t row_a;                      // shared address of the slice's first channel in the token's dense row
+    __device__ __forceinline__ void init() {}
+    __device__ __forceinline__ void put(uint32_t col, float w) {
+        asm volatile("st.shared.u16 [%0], %1;" ::"r"(row_a + col * 2u), "h"((uint16_t)(__float_as_uint(w) >> 16)));
     }
-    __device__ __forceinline__ void direct(uint32_t o, uint32_t w) {
-        asm volatile("st.shared.u16 [%0], %1;" ::"r"(row_a + o), "h"((uint16_t)(w >> 16)));
-    }
-    __device__ __forceinline__ void restart() {}
 };
 
-// Careful walk of `count` kept values from column bpos / code bit upos on.  bm/fl: this token's words, `fs` words
-// apart; un: unary words `us` apart.  STRIDE: bytes per column on the emitter's side.
-template <int T, int STRIDE, class Emit>
-__device__ __forceinline__ void kv_group_slow(const uint32_t* bm, const uint32_t* fl, int fs, const uint32_t* un, int us,
-                                           int count, uint32_t& bpos, uint32_t& upos, uint32_t bpos_lim, uint32_t upos_lim,
-                                           const uint32_t* lut, Emit& em) {
+// ---- Cassandra-1 slice -------------------------------------------------------------------------------------------
+// Careful walk of a slice's values [e_from, n): any codeword length, raw exponents too.  `un` points at the record's
+// first exponent word, words `us` apart.
+template <int T, class Emit>
+__device__ __noinline__ void kv_slice_slow(uint32_t bv, const uint32_t* fl, uint32_t fi, const uint32_t* un, int us,
+                                           uint32_t upos, uint32_t upos_lim, bool raw, int n, const uint32_t* lut, Emit& em) {
     constexpr int F = 8 - T, PER = 32 / F;
     constexpr uint32_t MASK = 0x80000000u | (((1u << (7 - T)) - 1u) << (16 + T));
-    for (int e = 0; e < count; ++e) {
-        bool found = false;
-        while (bpos < bpos_lim) {
-            uint32_t w = bm[(bpos >> 5) * fs] << (bpos & 31);
-            if (w) { bpos += __clz(w); found = true; break; }
-            bpos = (bpos | 31u) + 1u;
+    for (int e = 0; e < n && bv; ++e, ++fi) {
+        const uint32_t p = da_bfind(bv);
+        bv &= ~(1u << p);
+        uint32_t eb;
+        if (raw) {
+            eb = ((un[(fi >> 2) * us] >> (24 - 8 * (fi & 3))) & 0xFFu) << 23;
+        } else {
+            int rank = 0;
+            while (upos < upos_lim) {
+                const uint32_t v = un[(upos >> 5) * us] << (upos & 31);
+                const int avail = 32 - (int)(upos & 31);
+                if (v) { const int z = __clz(v); rank += z; upos += z + 1; break; }
+                rank += avail;
+                upos += avail;
+            }
+            eb = lut[rank & 255];
         }
-        if (!found) break;
-        const uint32_t col = bpos;
-        bpos += 1;
-        int rank = 0;
-        while (upos < upos_lim) {
-            uint32_t v = un[(upos >> 5) * us] << (upos & 31);
-            int avail = 32 - (int)(upos & 31);
-            if (v) { int z = __clz(v); rank += z; upos += z + 1; break; }
-            rank += avail;
-            upos += avail;
-        }
-        const uint32_t fword = fl[(e / PER) * fs];
-        const uint32_t a = __funnelshift_l(fword, fword, (F * (e % PER)) & 31);
-        em.direct(col * STRIDE, (a & MASK) | lut[rank & 255]);
+        const uint32_t fword = fl[(fi / PER) * 32];
+        const uint32_t a = __funnelshift_l(fword, fword, (F * (fi % PER)) & 31);
+        em.put(31u - p, __uint_as_float((a & MASK) | eb));
     }
 }
 
-// Walk of one record by one lane; `active` lanes emit, the others only keep the warp in step.
-// bm_a / fl_a / un_a: shared addresses of this lane's first bitmap / field / unary word (words 128 bytes apart).
-template <int T, int STRIDE, class Emit>
-__device__ __forceinline__ void kv_record_walk(const uint32_t* bmP, const uint32_t* flP, const uint32_t* unP, uint32_t lut_a,
-                                               const uint32_t* lutP, int kept, int d, uint32_t una_bits, bool active, Emit& em) {
+// One slice of a Cassandra-1 record per lane.  B: the slice's bitmap word; fi: index of its first field; upos: bit
+// offset of its first codeword in the staged stream (words 128 bytes apart from un_a); n: its kept values (0 for
+// lanes that only keep the warp in step).  Groups of 8 values, 4 codewords per 32-bit window; a window that runs dry
+// sends that lane through the careful walk for the rest of its slice.
+template <int T, class Emit>
+__device__ __forceinline__ void kv_slice_walk(uint32_t B, uint32_t fi, uint32_t upos, int n, uint32_t fl_a, const uint32_t* flP,
+                                              uint32_t un_a, const uint32_t* unP, uint32_t upos_lim, uint32_t lut_a,
+                                              const uint32_t* lutP, Emit& em) {
     constexpr int F = 8 - T, PER = 32 / F, NFW = kGroupCols / PER;
     constexpr uint32_t MASK = 0x80000000u | (((1u << (7 - T)) - 1u) << (16 + T));
-    const uint32_t bm_a = smem_u32(bmP), un_a = smem_u32(unP);
-    uint32_t fl_a = smem_u32(flP);
-    uint32_t bpos = 0, upos = 0;
-    const uint32_t bpos_lim = (uint32_t)d, upos_lim = (uint32_t)kDaUnaStage * 32u;
-    const int n_groups = ceil_div(kept, kGroupCols);
+    const int n_groups = ceil_div(__reduce_max_sync(0xffffffffu, n), kGroupCols);
+    uint32_t bv = B;
+    bool slow = false;
     for (int grp = 0; grp < n_groups; ++grp) {
-        const int cnt = min(kGroupCols, kept - grp * kGroupCols);
-        const bool tail = cnt < kGroupCols;
-        const uint32_t bpos0 = bpos, upos0 = upos;
-        const uint32_t ba = bm_a + (bpos >> 5) * 128u;
-        uint32_t bv = __funnelshift_l(da_lds(ba + 128u), da_lds(ba), bpos);
-        const uint32_t x0 = bpos * STRIDE;
-        uint32_t xa = x0;
-        uint32_t fwd[NFW];
-        fwd[0] = da_lds(fl_a);
-        if (NFW > 1) fwd[NFW - 1] = da_lds(fl_a + 128u);
-        uint32_t dry = 0, umax = 0;
-        em.reset();
+        const int rem = n - grp * kGroupCols;                                 // values this lane still has (may be <= 0)
+        const uint32_t fw_a = fl_a + (fi / PER) * 128u, j0 = fi % PER;
+        uint32_t fwd[NFW + 1];
+#pragma unroll
+        for (int i = 0; i <= NFW; ++i) fwd[i] = da_lds(fw_a + 128u * i);
+        const uint32_t bv0 = bv, upos0 = upos;
+        uint32_t cols[kGroupCols], wbs[kGroupCols];
+        uint32_t dry = 0;
 #pragma unroll
         for (int half = 0; half < kGroupCols / kGroupCodes; ++half) {
             const uint32_t ua = un_a + (upos >> 5) * 128u;
-            uint32_t uv = __funnelshift_l(da_lds(ua + 128u), da_lds(ua), upos);
-            uint32_t usum = 0;
-            auto elem = [&](auto ec) {
-                constexpr int e = decltype(ec)::value;
-                const uint32_t s = __clz(bv);
-                xa += s * STRIDE;
-                bv = da_shl(da_shl(bv, s), 1);
-                const uint32_t tt = __clz(uv);
-                const uint32_t eb = da_lds(lut_a + tt * 4u);
-                uv = da_shl(da_shl(uv, tt), 1);
-                usum += tt;
-                const uint32_t fword = fwd[e / PER];
-                const uint32_t a = __funnelshift_l(fword, fword, (F * (e % PER)) & 31);
-                const bool valid = active && (!tail || e < cnt);
-                em.template elem<e>(xa + e * STRIDE, (a & MASK) | eb, valid);
-                if (tail && e < cnt) dry |= s | tt;
-            };
-            if (half == 0) {
-                elem(std::integral_constant<int, 0>{}); elem(std::integral_constant<int, 1>{});
-                elem(std::integral_constant<int, 2>{}); elem(std::integral_constant<int, 3>{});
-            } else {
-                elem(std::integral_constant<int, 4>{}); elem(std::integral_constant<int, 5>{});
-                elem(std::integral_constant<int, 6>{}); elem(std::integral_constant<int, 7>{});
+            uint32_t uv = __funnelshift_l(da_lds(ua + 128u), da_lds(ua), upos);            // 32 code bits from upos on
+            uint32_t la = lut_a + 124u, q = 0;
+#pragma unroll
+            for (int j = 0; j < kGroupCodes; ++j) {
+                const int e = half * kGroupCodes + j;
+                const uint32_t p = da_bfind(bv);
+                bv &= ~da_shl(1u, p);
+                q = da_bfind(uv);
+                const uint32_t eb = da_lds(la - (q & 31u) * 4u);                           // lut[previous - q - 1]
+                la = lut_a - 4u + (q & 31u) * 4u;
+                uv &= ~da_shl(1u, q);
+                const uint32_t jj = j0 + e;                                                // field jj of the group's words
+                const uint32_t fword = (jj >= (uint32_t)(PER * ((e / PER) + 1))) ? fwd[e / PER + 1] : fwd[e / PER];
+                const uint32_t a = __funnelshift_l(fword, fword, (F * jj) & 31);
+                cols[e] = 31u - (p & 31u);
+                wbs[e] = (a & MASK) | eb;
+                if (e < rem) dry |= q;                                                     // sign bit set: the window ran dry
             }
-            upos = min(upos + usum + kGroupCodes, upos_lim);
-            umax = max(umax, usum);
+            upos = min(upos + 32u - (q & 31u), upos_lim);
         }
-        const uint32_t adv = (xa - x0) / STRIDE;
-        bpos = min(bpos + adv + kGroupCols, bpos_lim);
-        if (!tail) dry = (adv + kGroupCols > 32u || umax + kGroupCodes > 32u) ? 32u : 0u;
-        if (active) {
-            if (dry & 32u) {                           // a window ran dry: redo this group one value at a time
-                bpos = bpos0; upos = upos0;
-                kv_group_slow<T, STRIDE>(bmP, flP + grp * NFW * 32, 32, unP, 32, cnt, bpos, upos, bpos_lim, min(una_bits, upos_lim),
-                                         lutP, em);
+        if (rem > 0 && !slow) {
+            if ((int32_t)dry < 0) {
+                slow = true;                             // finish this slice one value at a time, from the group's start
+                kv_slice_slow<T>(bv0, flP, fi, unP, 32, upos0, upos_lim, false, rem, lutP, em);
             } else {
-                em.commit(cnt);
+#pragma unroll
+                for (int e = 0; e < kGroupCols; ++e)
+                    if (e < rem) em.put(cols[e], __uint_as_float(wbs[e]));
             }
         }
-        fl_a += NFW * 128u;
+        fi += kGroupCols;
     }
 }
 
-template <int T, int GQ>
-__global__ void __launch_bounds__(kDaThreads) k_draft_attn(KvGeom g, KvComp ck0, KvComp cv0, const uint16_t* __restrict__ qkv,
-                                                           int qkv_stride, int n_q, const DevState* __restrict__ st, AttnScratch sc,
-                                                           int n_chunks_alloc) {
+// ---- Cassandra-2 slice: fields = sign + magnitude, one shared exponent per slice ------------------------------------
+// vlut: float value of every field pattern, +-(magnitude << t); scale = 2^(E - 133).
+template <int T, class Emit>
+__device__ __forceinline__ void kv_slice_walk_mx(uint32_t B, uint32_t fi, int n, uint32_t fl_a, uint32_t vlut_a, float scale,
+                                                 Emit& em) {
+    constexpr int F = 8 - T, PER = 32 / F;
+    const int n_groups = ceil_div(__reduce_max_sync(0xffffffffu, n), 4);
+    uint32_t bv = B;
+    for (int grp = 0; grp < n_groups; ++grp) {
+        const int rem = n - grp * 4;
+        const uint32_t fw_a = fl_a + (fi / PER) * 128u;
+        const uint32_t comb = __funnelshift_l(da_lds(fw_a + 128u), da_lds(fw_a), (F * (fi % PER)) & 31);   // 4 fields from the top
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const uint32_t p = da_bfind(bv);
+            bv &= ~da_shl(1u, p);
+            const uint32_t f = (comb >> (32 - F * (e + 1))) & ((1u << F) - 1u);
+            const float v = __uint_as_float(da_lds(vlut_a + f * 4u)) * scale;
+            if (e < rem) em.put(31u - (p & 31u), v);
+        }
+        fi += 4;
+    }
+}
+
+template <int MODE, int T, int GQ>
+__global__ void __launch_bounds__(512) k_draft_attn(KvGeom g, KvComp ck0, KvComp cv0, const uint16_t* __restrict__ qkv,
+                                                    int qkv_stride, int n_q, const DevState* __restrict__ st, AttnScratch sc,
+                                                    int n_chunks_alloc, int stage) {
     extern __shared__ __align__(16) uint8_t smem[];
     pdl_early<2>();
     pdl_wait();
-    const int chunk = blockIdx.x, head = blockIdx.y, seq = blockIdx.z;
+    const int head = blockIdx.y, seq = blockIdx.z;
     const int cur_len = st->len[seq] + st->inflight[seq] + 1;  // positions visible to the drafted token
-    const int t0 = chunk * kDaTok;
-    if (t0 >= cur_len) return;
-    const int G = n_q / g.n_kv, d = g.d;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int tpc = da_tokens_per_cta(cur_len, g.n_kv * (int)gridDim.z);
+    const int t_begin = blockIdx.x * tpc;
+    if (t_begin >= cur_len) return;
+    const int t_end = min(cur_len, t_begin + tpc);
+    const int G = n_q / g.n_kv, d = g.d, S = d / 32;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, n_thr = blockDim.x;
     qkv += (size_t)seq * qkv_stride;
 
-    constexpr int kQStride = GQ * 4;                                          // bytes per column of the query tile
+    const int vrow = d + 2;                                                   // halfwords per row of the V tile (padded)
     float* q_s = reinterpret_cast<float*>(smem);                              // [d][GQ]
-    float* sc_s = q_s + d * GQ;                                               // [GQ][64] scores -> probabilities
-    float* ml_s = sc_s + GQ * kDaTok;                                         // [GQ][2]
-    uint32_t* lut_s = reinterpret_cast<uint32_t*>(ml_s + 2 * GQ);             // [2][256] rank -> exponent << 23
-    uint32_t* fix_s = lut_s + 512;                                            // [4 warps][wpt + 1][32]
-    uint32_t* una_s = fix_s + 4 * (g.wpt + 1) * 32;                           // [4 warps][kDaUnaStage + 2][32]
-    uint16_t* v_s = reinterpret_cast<uint16_t*>(una_s + 4 * (kDaUnaStage + 2) * 32);   // [64][d] bf16
+    float* part_s = q_s + d * GQ;                                             // [S][GQ][32] partial q.k of the slices
+    float* sc_s = part_s + S * GQ * kDaSub;                                   // [GQ][32] probabilities of the pass
+    float* run_s = sc_s + GQ * kDaSub;                                        // [GQ][4]: running max, running sum, rescale factor
+    uint32_t* lut_s = reinterpret_cast<uint32_t*>(run_s + 4 * GQ);            // mode 1: [2][256] rank -> exponent << 23; mode 2: [256] field values
+    uint32_t* meta_s = lut_s + 512;                                           // [2][32] arena offset, [2][32] arena words of the pass's records
+    uint32_t* fix_s = meta_s + 128;                                           // [2][wpt + 2][32]
+    uint32_t* una_s = fix_s + 2 * (g.wpt + 2) * 32;                           // [2][stage + 2][32] (mode 1)
+    uint16_t* v_s = reinterpret_cast<uint16_t*>(una_s + (MODE == 1 ? 2 * (stage + 2) * 32 : 0));   // [32][vrow] bf16
 
     const float scale = rsqrtf((float)d);
-    for (int i = tid; i < d * GQ; i += kDaThreads) {
-        int col = i / GQ, gi = i % GQ;
+    for (int i = tid; i < d * GQ; i += n_thr) {
+        const int col = i / GQ, gi = i % GQ;
         q_s[i] = gi < G ? bf16_bits_to_float(qkv[(size_t)(head * G + gi) * d + col]) : 0.f;
     }
-    {
+    if (MODE == 1) {
         const uint8_t *rk = of_seq(ck0.rank_to_exp, seq, g.seq_stride), *rv = of_seq(cv0.rank_to_exp, seq, g.seq_stride);
-        for (int i = tid; i < 512; i += kDaThreads) lut_s[i] = (uint32_t)(i < 256 ? rk[i] : rv[i - 256]) << 23;
-    }
-    for (int i = tid; i < kDaTok * d / 2; i += kDaThreads) reinterpret_cast<uint32_t*>(v_s)[i] = 0u;
-
-    // stage this warp's 32 records: warps 0,1 -> K of tokens t0 + 32 w .., warps 2,3 -> V of the same tokens
-    const int kind = warp >> 1, tw = warp & 1;
-    const int tok = t0 + tw * 32 + lane;
-    const bool valid = tok < cur_len;
-    const KvComp& c = kind ? cv0 : ck0;                      // sequence 0's; shifted to this sequence where used
-    uint32_t* my_fix = fix_s + warp * (g.wpt + 1) * 32;
-    uint32_t* my_una = una_s + warp * (kDaUnaStage + 2) * 32;
-    {
-        const uint32_t* fixed = of_seq(c.fixed, seq, g.seq_stride) + ((size_t)head * g.n_blocks + tok / 32) * g.wpt * 32;
-        for (int w = 0; w < g.wpt; ++w) my_fix[w * 32 + lane] = fixed[w * 32 + lane];          // coalesced block copy
-        my_fix[g.wpt * 32 + lane] = 0u;
-    }
-    const uint32_t* off = of_seq(c.off, seq, g.seq_stride) + (size_t)head * (g.max_seq + 1);
-    const uint32_t* arena = of_seq(c.arena, seq, g.seq_stride) + (size_t)head * g.arena_words;
-    uint32_t o0 = 0, n_una = 0;
-    if (valid) { o0 = off[tok]; n_una = off[tok + 1] - o0; }
-    const bool staged = n_una <= (uint32_t)kDaUnaStage;
-    for (int w = 0; w < kDaUnaStage + 2; ++w) my_una[w * 32 + lane] = (staged && (uint32_t)w < n_una) ? arena[o0 + w] : 0u;
-    __syncthreads();
-
-    const uint32_t* lutP = lut_s + kind * 256;
-    if (kind == 0) {
-        EmitK<GQ> em;
-        em.q_a = smem_u32(q_s);
-        em.restart();
-        kv_record_walk<T, kQStride>(my_fix + lane, my_fix + g.bm_words * 32 + lane, my_una + lane, smem_u32(lutP), lutP, g.kept, d,
-                                    n_una * 32u, valid && staged, em);
-        if (valid && !staged) {                                               // very long record: walk it in place
-            uint32_t bpos = 0, upos = 0;
-            em.restart();
-            for (int grp = 0; grp * kGroupCols < g.kept; ++grp)
-                kv_group_slow<T, kQStride>(my_fix + lane, my_fix + (g.bm_words + grp * (kGroupCols * (8 - T) / 32)) * 32 + lane, 32,
-                                           arena + o0, 1, min(kGroupCols, g.kept - grp * kGroupCols), bpos, upos, (uint32_t)d,
-                                           n_una * 32u, lutP, em);
-        }
-#pragma unroll
-        for (int gi = 0; gi < GQ; ++gi)
-            if (gi < G) sc_s[gi * kDaTok + tw * 32 + lane] = valid ? em.acc[gi] * scale : -INFINITY;
+        for (int i = tid; i < 512; i += n_thr) lut_s[i] = (uint32_t)(i < 256 ? rk[i] : rv[i - 256]) << 23;
     } else {
-        EmitV em;
-        em.row_a = smem_u32(v_s + (size_t)(tw * 32 + lane) * d);
-        kv_record_walk<T, 2>(my_fix + lane, my_fix + g.bm_words * 32 + lane, my_una + lane, smem_u32(lutP), lutP, g.kept, d,
-                             n_una * 32u, valid && staged, em);
-        if (valid && !staged) {
-            uint32_t bpos = 0, upos = 0;
-            for (int grp = 0; grp * kGroupCols < g.kept; ++grp)
-                kv_group_slow<T, 2>(my_fix + lane, my_fix + (g.bm_words + grp * (kGroupCols * (8 - T) / 32)) * 32 + lane, 32,
-                                    arena + o0, 1, min(kGroupCols, g.kept - grp * kGroupCols), bpos, upos, (uint32_t)d,
-                                    n_una * 32u, lutP, em);
+        constexpr int NF = 1 << (8 - T);
+        for (int i = tid; i < NF; i += n_thr) {
+            const float mag = (float)((i & (NF / 2 - 1)) << T);
+            lut_s[i] = __float_as_uint((i & (NF / 2)) ? -mag : mag);
         }
     }
-    __syncthreads();
-    // chunk softmax statistics: warp w handles query heads w, w + 4
-    for (int gi = warp; gi < G; gi += kDaThreads / 32) {
-        float a = sc_s[gi * kDaTok + lane], b = sc_s[gi * kDaTok + 32 + lane];
-        const float m = warp_max(fmaxf(a, b));
-        a = expf(a - m);                                              // exp(-inf) = 0 for tokens beyond the end
-        b = expf(b - m);
-        sc_s[gi * kDaTok + lane] = a;
-        sc_s[gi * kDaTok + 32 + lane] = b;
-        const float l = warp_sum(a + b);
-        if (lane == 0) { ml_s[gi * 2] = m; ml_s[gi * 2 + 1] = l; }
-    }
-    __syncthreads();
-    // o[gi][dim] = sum_t p[gi][t] * v[t][dim]
-    const int n_tok = min(kDaTok, cur_len - t0);
-    for (int dim = tid; dim < d; dim += kDaThreads) {
-        float acc[GQ];
+    if (tid < 4 * GQ) run_s[tid] = (tid & 3) == 0 ? -INFINITY : 0.f;
+
+    const int kind = warp / S, slice = warp % S;                              // warps 0..S-1: K slices, S..2S-1: V slices
+    const KvComp& c = kind ? cv0 : ck0;                                       // sequence 0's; shifted to this sequence where used
+    const uint32_t* fixed_k = of_seq(ck0.fixed, seq, g.seq_stride) + (size_t)head * g.n_blocks * g.wpt * 32;
+    const uint32_t* fixed_v = of_seq(cv0.fixed, seq, g.seq_stride) + (size_t)head * g.n_blocks * g.wpt * 32;
+    const uint32_t* off_k = of_seq(ck0.off, seq, g.seq_stride) + (size_t)head * (g.max_seq + 1);
+    const uint32_t* off_v = of_seq(cv0.off, seq, g.seq_stride) + (size_t)head * (g.max_seq + 1);
+    const uint32_t* arena_k = of_seq(ck0.arena, seq, g.seq_stride) + (size_t)head * g.arena_words;
+    const uint32_t* arena_v = of_seq(cv0.arena, seq, g.seq_stride) + (size_t)head * g.arena_words;
+    (void)c;
+    const int fsz = (g.wpt + 2) * 32, usz = (stage + 2) * 32;
+    float o_acc[GQ];
 #pragma unroll
-        for (int gi = 0; gi < GQ; ++gi) acc[gi] = 0.f;
+    for (int gi = 0; gi < GQ; ++gi) o_acc[gi] = 0.f;
+
+    for (int t0 = t_begin; t0 < t_end; t0 += kDaSub) {
+        // ---- stage the pass: both fixed-part blocks (coalesced), the V tile cleared, the exponent words of its records ----
+        const int blk = t0 / 32;
+        for (int i = tid; i < 2 * fsz; i += n_thr) {
+            const int kd = i / fsz, w = i % fsz;
+            fix_s[i] = w < g.wpt * 32 ? (kd ? fixed_v : fixed_k)[(size_t)blk * g.wpt * 32 + w] : 0u;
+        }
+        for (int i = tid; i < kDaSub * vrow / 2; i += n_thr) reinterpret_cast<uint32_t*>(v_s)[i] = 0u;
+        if (MODE == 1 && tid < 64) {
+            const int kd = tid >> 5, tok = t0 + (tid & 31);
+            uint32_t o0 = 0, nw = 0;
+            if (tok < cur_len) { const uint32_t* off = kd ? off_v : off_k; o0 = off[tok]; nw = off[tok + 1] - o0; }
+            meta_s[kd * 32 + (tid & 31)] = o0;
+            meta_s[64 + kd * 32 + (tid & 31)] = nw;
+        }
+        __syncthreads();
+        if (MODE == 1) {
+            for (int i = tid; i < 2 * usz; i += n_thr) {
+                const int kd = i / usz, w = (i % usz) / 32, tk = i % 32;
+                const uint32_t nw = meta_s[64 + kd * 32 + tk];
+                una_s[i] = (nw <= (uint32_t)stage && (uint32_t)w < nw) ? (kd ? arena_v : arena_k)[meta_s[kd * 32 + tk] + w] : 0u;
+            }
+            __syncthreads();
+        }
+        // ---- decode: warp (kind, slice), lane = token ----
+        if (warp < 2 * S) {
+            const int tok = t0 + lane;
+            const bool valid = tok < cur_len;
+            const uint32_t* fx = fix_s + kind * fsz + lane;                      // word w of this token at fx[w * 32]
+            const int bm0 = MODE == 1 ? g.e_words : 0;
+            const uint32_t B = fx[(bm0 + slice) * 32];
+            uint32_t fi = 0;
+            for (int s2 = 0; s2 < slice; ++s2) fi += __popc(fx[(bm0 + s2) * 32]);
+            const int n = valid ? __popc(B) : 0;
+            const uint32_t fl_a = smem_u32(fx + (bm0 + g.bm_words) * 32);
+            EmitK<GQ> ek;
+            EmitV ev;
+            ek.q_a = smem_u32(q_s + (size_t)slice * 32 * GQ);
+            ev.row_a = smem_u32(v_s + (size_t)lane * vrow + slice * 32);
+            ek.init();
+            if (MODE == 1) {
+                const uint32_t e0 = fx[0];
+                const bool raw = (e0 & kKvRawFlag) != 0;
+                const uint32_t upos = slice == 0 ? 0u : (fx[((slice - 1) / 3) * 32] >> (20 - 10 * ((slice - 1) % 3))) & 0x3FFu;
+                const uint32_t nw = meta_s[64 + kind * 32 + lane];
+                const bool staged = nw <= (uint32_t)stage;
+                const bool fast = valid && !raw && staged;
+                const uint32_t* lutP = lut_s + kind * 256;
+                const uint32_t* unP = una_s + kind * usz + lane;
+                const uint32_t upos_lim = (uint32_t)stage * 32u;
+                if (kind == 0) kv_slice_walk<T>(B, fi, upos, fast ? n : 0, fl_a, fx + (bm0 + g.bm_words) * 32, smem_u32(unP), unP, upos_lim,
+                                                smem_u32(lutP), lutP, ek);
+                else kv_slice_walk<T>(B, fi, upos, fast ? n : 0, fl_a, fx + (bm0 + g.bm_words) * 32, smem_u32(unP), unP, upos_lim,
+                                      smem_u32(lutP), lutP, ev);
+                if (valid && !fast) {                     // raw exponents, or a record longer than the staging: read it in place
+                    const uint32_t* un = (kind ? arena_v : arena_k) + meta_s[kind * 32 + lane];
+                    if (kind == 0) kv_slice_slow<T>(B, fx + (bm0 + g.bm_words) * 32, fi, un, 1, upos, nw * 32u, raw, n, lutP, ek);
+                    else kv_slice_slow<T>(B, fx + (bm0 + g.bm_words) * 32, fi, un, 1, upos, nw * 32u, raw, n, lutP, ev);
+                }
+            } else {
+                const uint32_t xw = fx[(g.bm_words + g.f_words + slice / 4) * 32];
+                const uint32_t eb = (xw >> (24 - 8 * (slice % 4))) & 0xFFu;
+                const float sc2 = __uint_as_float(eb >= 7u ? (eb - 6u) << 23 : 0u);     // 2^(E - 133)
+                if (kind == 0) kv_slice_walk_mx<T>(B, fi, n, fl_a, smem_u32(lut_s), sc2, ek);
+                else kv_slice_walk_mx<T>(B, fi, n, fl_a, smem_u32(lut_s), sc2, ev);
+            }
+            if (kind == 0) {
+#pragma unroll
+                for (int gi = 0; gi < GQ; ++gi) part_s[(slice * GQ + gi) * kDaSub + lane] = ek.acc[gi];
+            }
+        }
+        __syncthreads();
+        // ---- running softmax: warp gi handles query head gi of the group, lane = token ----
+        for (int gi = warp; gi < G; gi += n_thr / 32) {
+            float sdot = 0.f;
+            for (int s2 = 0; s2 < S; ++s2) sdot += part_s[(s2 * GQ + gi) * kDaSub + lane];
+            const bool valid = t0 + lane < cur_len;
+            const float sv = valid ? sdot * scale : -INFINITY;
+            const float m_old = run_s[gi * 4], l_old = run_s[gi * 4 + 1];
+            const float m_new = fmaxf(m_old, warp_max(sv));                   // finite: the pass has at least one visible token
+            const float pr = valid ? expf(sv - m_new) : 0.f;
+            const float alpha = expf(m_old - m_new);                          // exp(-inf) = 0 on the first pass
+            sc_s[gi * kDaSub + lane] = pr;
+            const float l_new = l_old * alpha + warp_sum(pr);
+            __syncwarp();
+            if (lane == 0) { run_s[gi * 4] = m_new; run_s[gi * 4 + 1] = l_new; run_s[gi * 4 + 2] = alpha; }
+        }
+        __syncthreads();
+        // ---- o[gi][dim] = alpha o + sum_t p[gi][t] v[t][dim]; thread = dim ----
+        if (tid < d) {
+            const int n_tok = min(kDaSub, cur_len - t0);
+#pragma unroll
+            for (int gi = 0; gi < GQ; ++gi) o_acc[gi] *= run_s[gi * 4 + 2];
 #pragma unroll 4
-        for (int t = 0; t < n_tok; ++t) {
-            const float v = bf16_bits_to_float(v_s[(size_t)t * d + dim]);
+            for (int t = 0; t < n_tok; ++t) {
+                const float v = bf16_bits_to_float(v_s[(size_t)t * vrow + tid]);
 #pragma unroll
-            for (int gi = 0; gi < GQ; ++gi)
-                if (gi < G) acc[gi] = fmaf(sc_s[gi * kDaTok + t], v, acc[gi]);
+                for (int gi = 0; gi < GQ; ++gi) o_acc[gi] = fmaf(sc_s[gi * kDaSub + t], v, o_acc[gi]);
+            }
         }
+        __syncthreads();                                                      // the pass's buffers are free again
+    }
+    const int chunk = blockIdx.x;
+    if (tid < d) {
 #pragma unroll
         for (int gi = 0; gi < GQ; ++gi)
-            if (gi < G) sc.o[(((size_t)seq * n_q + head * G + gi) * n_chunks_alloc + chunk) * d + dim] = acc[gi];
+            if (gi < G) sc.o[(((size_t)seq * n_q + head * G + gi) * n_chunks_alloc + chunk) * d + tid] = o_acc[gi];
     }
     if (tid < G) {
         const size_t pair = (size_t)seq * n_q + head * G + tid;
-        sc.m[pair * n_chunks_alloc + chunk] = ml_s[tid * 2];
-        sc.l[pair * n_chunks_alloc + chunk] = ml_s[tid * 2 + 1];
+        sc.m[pair * n_chunks_alloc + chunk] = run_s[tid * 4];
+        sc.l[pair * n_chunks_alloc + chunk] = run_s[tid * 4 + 1];
     }
 }
 
@@ -312,7 +359,8 @@ constexpr int kMergeThreads = 256;
 constexpr int kMergeWarps = kMergeThreads / 32;
 
 __global__ void __launch_bounds__(kMergeThreads) k_attn_merge(AttnScratch sc, int n_chunks_alloc, int chunk_tokens, int rps, int n_q, int d,
-                                                              const DevState* __restrict__ st, int draft_mode, uint16_t* __restrict__ out) {
+                                                              const DevState* __restrict__ st, int draft_mode, int draft_units,
+                                                              uint16_t* __restrict__ out) {
     extern __shared__ __align__(16) float w_s[];    // [n_chunks_alloc] weights e^{m_c - M}, then [kMergeWarps][d] partial outputs
     __shared__ float s_red[kMergeWarps];
     pdl_early<3>();
@@ -321,6 +369,7 @@ __global__ void __launch_bounds__(kMergeThreads) k_attn_merge(AttnScratch sc, in
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int seq = r / rps;
     const int vis = st->len[seq] + (draft_mode ? st->inflight[seq] + 1 : r % rps + 1);
+    if (draft_mode) chunk_tokens = da_tokens_per_cta(vis, draft_units);       // the split the draft attention chose for this length
     const int n_ch = ceil_div(vis, chunk_tokens);
     const size_t pair = (size_t)r * n_q + hq;
     const float* mp = sc.m + pair * n_chunks_alloc;
@@ -370,7 +419,7 @@ __global__ void __launch_bounds__(kMergeThreads) k_attn_merge(AttnScratch sc, in
 }
 
 int launch_attn_merge(const AttnScratch& sc, int n_chunks_alloc, int chunk_tokens, int rows, int rps, int n_q, int d,
-                      const DevState* st, int draft_mode, uint16_t* out, cudaStream_t s) {
+                      const DevState* st, int draft_mode, int draft_units, uint16_t* out, cudaStream_t s) {
     if (d % 4) return CASS_ERR_UNSUPPORTED;
     dim3 grid(n_q, rows);
     const size_t smem = ((size_t)((n_chunks_alloc + 3) & ~3) + (size_t)kMergeWarps * d) * 4;
@@ -380,40 +429,53 @@ int launch_attn_merge(const AttnScratch& sc, int n_chunks_alloc, int chunk_token
         CASS_CUDA_CHECK(cudaFuncSetAttribute(k_attn_merge, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         attr = smem;
     }
-    CASS_PDL_LAUNCH(k_attn_merge, grid, dim3(kMergeThreads), smem, s, sc, n_chunks_alloc, chunk_tokens, rps, n_q, d, st, draft_mode, out);
+    CASS_PDL_LAUNCH(k_attn_merge, grid, dim3(kMergeThreads), smem, s, sc, n_chunks_alloc, chunk_tokens, rps, n_q, d, st, draft_mode,
+                    draft_units, out);
     return CASS_OK;
 }
 
+static int draft_attn_stage(const KvGeom& g) { return g.rec_words_max < kDaUnaStageMax ? g.rec_words_max : kDaUnaStageMax; }
+
 size_t draft_attn_smem_bytes(const KvGeom& g, int gq) {
-    return (size_t)g.d * gq * 4 + (size_t)gq * kDaTok * 4 + 2 * gq * 4 + 512 * 4 +
-           (size_t)4 * (g.wpt + 1) * 32 * 4 + (size_t)4 * (kDaUnaStage + 2) * 32 * 4 + (size_t)kDaTok * g.d * 2 + 64;
+    const int S = g.d / 32, stage = draft_attn_stage(g);
+    return (size_t)g.d * gq * 4 + (size_t)S * gq * kDaSub * 4 + (size_t)gq * kDaSub * 4 + 4 * gq * 4 + 512 * 4 + 128 * 4 +
+           (size_t)2 * (g.wpt + 2) * 32 * 4 + (g.mode == 1 ? (size_t)2 * (stage + 2) * 32 * 4 : 0) +
+           (size_t)kDaSub * (g.d + 2) * 2 + 64;
 }
 
 int launch_draft_attn(const KvGeom& g, const KvComp& ck, const KvComp& cv, const uint16_t* qkv, int qkv_stride, int n_q,
                       int n_seq, const DevState* st, const AttnScratch& sc, uint16_t* out, cudaStream_t s) {
     const int G = n_q / g.n_kv;
     if (G > kMaxGroup || g.d > 256 || g.d % 32) return CASS_ERR_UNSUPPORTED;
-    const int n_chunks = ceil_div(g.max_seq, kDaTok);
+    const int n_chunks = ceil_div(g.max_seq, kDaSub);        // the most CTAs a head can need (32 tokens each); longer runs use fewer
     const int gq = G <= 4 ? 4 : 8;
     const size_t smem = draft_attn_smem_bytes(g, gq);
+    const int stage = draft_attn_stage(g);
+    const int threads = 2 * (g.d / 32) * 32;
     dim3 grid(n_chunks, g.n_kv, n_seq);
-#define CASS_DA_LAUNCH(TT, GG)                                                                                         \
+#define CASS_DA_LAUNCH(MM, TT, GG)                                                                                     \
     do {                                                                                                             \
         static size_t attr = 0;                                                                                      \
         if (smem > attr) {                                                                                           \
-            CASS_CUDA_CHECK(cudaFuncSetAttribute((k_draft_attn<TT, GG>), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
+            CASS_CUDA_CHECK(cudaFuncSetAttribute((k_draft_attn<MM, TT, GG>), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
             attr = smem;                                                                                             \
         }                                                                                                            \
-        CASS_PDL_LAUNCH((k_draft_attn<TT, GG>), grid, dim3(kDaThreads), smem, s, g, ck, cv, qkv, qkv_stride, n_q, st, sc, n_chunks);     \
+        CASS_PDL_LAUNCH((k_draft_attn<MM, TT, GG>), grid, dim3(threads), smem, s, g, ck, cv, qkv, qkv_stride, n_q, st, sc, n_chunks, stage); \
     } while (0)
-    if (g.t == 4 && gq == 4) CASS_DA_LAUNCH(4, 4);
-    else if (g.t == 4) CASS_DA_LAUNCH(4, 8);
-    else if (g.t == 0 && gq == 4) CASS_DA_LAUNCH(0, 4);
-    else if (g.t == 0) CASS_DA_LAUNCH(0, 8);
-    else return CASS_ERR_UNSUPPORTED;
+#define CASS_DA_LAUNCH_T(MM)                                                                                          \
+    do {                                                                                                             \
+        if (g.t == 4 && gq == 4) CASS_DA_LAUNCH(MM, 4, 4);                                                           \
+        else if (g.t == 4) CASS_DA_LAUNCH(MM, 4, 8);                                                                 \
+        else if (g.t == 0 && gq == 4) CASS_DA_LAUNCH(MM, 0, 4);                                                      \
+        else if (g.t == 0) CASS_DA_LAUNCH(MM, 0, 8);                                                                 \
+        else return CASS_ERR_UNSUPPORTED;                                                                            \
+    } while (0)
+    if (g.mode == 2) CASS_DA_LAUNCH_T(2);
+    else CASS_DA_LAUNCH_T(1);
+#undef CASS_DA_LAUNCH_T
 #undef CASS_DA_LAUNCH
     CASS_LAUNCH_CHECK();
-    return launch_attn_merge(sc, n_chunks, kDaTok, n_seq, 1, n_q, g.d, st, 1, out, s);
+    return launch_attn_merge(sc, n_chunks, kDaSub, n_seq, 1, n_q, g.d, st, 1, g.n_kv * n_seq, out, s);
 }
 
 }  // namespace cass

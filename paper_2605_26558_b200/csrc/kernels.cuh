@@ -19,8 +19,15 @@ struct DevState {
 
 // Row r of a call with `rps` rows per sequence belongs to sequence r / rps and is its (r % rps)-th new row.
 
-// Compressed KV cache of one (layer, K|V): per head a fixed part (bitmap + fields, 32-token blocks interleaved
-// word by word), an append-only arena of unary words and per-token word offsets.
+// Compressed KV cache of one (layer, K|V): per head a fixed part (32-token blocks interleaved word by word), an
+// append-only arena of exponent words and per-token word offsets.
+// Cassandra-1 record (mode 1): fixed part = entry words | bitmap | fields (rotated, as in the weight blobs); the arena
+// holds the record's unary exponent stream or, when that would take more than min(8 * kept, 1023) bits, the kept
+// values' exponents as raw bytes (four per word from the top; bit 31 of the first entry word says so).  Entry words:
+// a 10-bit code-bit offset for every 32-channel slice after the first, three per word from bit 29 down, so that the
+// d/32 slices of a record can be decoded side by side.
+// Cassandra-2 record (mode 2): fixed part = bitmap | fields (sign + magnitude, packed from the top) | one shared
+// exponent byte per 32-channel slice (four per word from the top); no arena use.
 struct KvComp {
     uint32_t* fixed;        // [n_kv][n_blocks][wpt][32]
     uint32_t* arena;        // [n_kv][arena_words]
@@ -30,8 +37,13 @@ struct KvComp {
     unsigned long long* hist;   // [256]
 };
 
+constexpr uint32_t kKvRawFlag = 0x80000000u;
 struct KvGeom {
     int n_kv, d, max_seq, n_blocks, wpt, bm_words, f_words, kept, n_prune, t, arena_words;
+    int mode;               // 1 = Cassandra-1 records, 2 = Cassandra-2 (MX) records
+    int e_words;            // entry words in front of the bitmap (mode 1), 0 in mode 2
+    int x_words;            // exponent words behind the fields (mode 2), 0 in mode 1
+    int rec_words_max;      // most arena words one record can take
     size_t seq_stride;      // bytes between the KV storage (both caches, all layers) of consecutive sequences
 };
 
@@ -40,6 +52,15 @@ template <class P>
 __host__ __device__ __forceinline__ P* of_seq(P* p, int b, size_t seq_stride) {
     using Byte = typename std::conditional<std::is_const<P>::value, const char, char>::type;
     return reinterpret_cast<P*>(reinterpret_cast<Byte*>(p) + (size_t)b * seq_stride);     // pointer arithmetic: stays a global-memory pointer
+}
+__host__ __device__ inline int kv_entry_words(int d) { int n = (d / 32 - 1 + 2) / 3; return n < 1 ? 1 : n; }
+__host__ __device__ inline int kv_code_budget(int kept) { return 8 * kept < 1023 ? 8 * kept : 1023; }
+// Tokens one CTA of the draft attention handles: 32, doubled while the grid would exceed about four CTAs per SM.
+// Draft attention and its merge compute it from the same visible length, so they agree without host involvement.
+__host__ __device__ inline int da_tokens_per_cta(int visible, int heads_x_seqs) {
+    int t = 32;
+    while (t < 256 && ceil_div(visible, t) * heads_x_seqs > 592) t *= 2;
+    return t;
 }
 __host__ __device__ __forceinline__ KvComp of_seq(const KvComp& c, int b, size_t seq_stride) {
     KvComp r;

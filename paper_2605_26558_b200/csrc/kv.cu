@@ -6,9 +6,9 @@
 namespace cass {
 
 constexpr int kKvMaxPerLane = 8;       // head_dim <= 256
-constexpr int kKvStageWords = 96;      // unary staging per token: up to 3072 code bits
+constexpr int kKvStageWords = 64;      // exponent staging per token: 2048 bits (a unary stream takes at most 1023, raw bytes 8 per value)
 constexpr int kKvWarps = 8;
-constexpr int kKvFixMax = 72;        // head_dim 256, no truncation: 8 bitmap + 64 field words
+constexpr int kKvFixMax = 76;        // head_dim 256, no truncation: 3 entry + 8 bitmap + 64 field words (+ 2 exponent words in mode 2)
 
 // Per-token selection: lane holds elements c = lane + 32 j.  keep[j] is set for the d - n_prune largest
 // |x| (ties: the lower channel is pruned first).  Key = (|x| bits << 8) | channel is unique, so the kept set is
@@ -193,34 +193,86 @@ __global__ void __launch_bounds__(256) k_kv_append(KvGeom g, KvComp ck, KvComp c
                 for (int w = lane; w < kKvFixMax; w += 32) s_fix[warp][w] = 0;
                 for (int w = lane; w < kKvStageWords; w += 32) s_una[warp][w] = 0;
                 __syncwarp();
-                uint32_t kbase = 0, ubase = 0;
+                if (g.mode == 2) {
+                    // ---- Cassandra-2 record: bitmap | fields (sign, magnitude >> t; packed from the top) | slice exponents ----
+                    uint32_t kbase = 0;
 #pragma unroll
-                for (int j = 0; j < kKvMaxPerLane; ++j) {
-                    if (j < nj) {
-                        uint32_t bm = __brev(__ballot_sync(0xffffffffu, keep[j]));   // channel c at bit 31 - c%32
-                        if (lane == 0) s_fix[warp][j] = bm;
-                        uint32_t len = keep[j] ? (uint32_t)exp_to_rank[(bits[j] >> 7) & 0xFF] + 1u : 0u;
-                        uint32_t incl = len;
-#pragma unroll
-                        for (int o = 1; o < 32; o <<= 1) {
-                            uint32_t v = __shfl_up_sync(0xffffffffu, incl, o);
-                            if (lane >= o) incl += v;
+                    for (int j = 0; j < kKvMaxPerLane; ++j) {
+                        if (j < nj) {
+                            const uint32_t bm = __brev(__ballot_sync(0xffffffffu, keep[j]));
+                            const uint32_t e = (bits[j] >> 7) & 0xFFu;
+                            const uint32_t E = __reduce_max_sync(0xffffffffu, keep[j] ? e : 0u);   // the slice's shared exponent
+                            if (lane == 0) {
+                                s_fix[warp][j] = bm;
+                                atomicOr(&s_fix[warp][g.bm_words + g.f_words + j / 4], E << (24 - 8 * (j % 4)));
+                            }
+                            if (keep[j]) {
+                                const uint32_t sh = 1u + E - e;
+                                const uint32_t m7 = (sh < 8u && e > 0u && E >= 7u) ? ((0x80u | (bits[j] & 0x7Fu)) >> sh) : 0u;
+                                const uint32_t field = ((bits[j] >> 15) << (7 - t_bits)) | (m7 >> t_bits);
+                                const uint32_t k = kbase + (lane ? __popc(bm >> (32 - lane)) : 0u);
+                                atomicOr(&s_fix[warp][g.bm_words + k / per], field << (32 - F * (k % per + 1)));
+                            }
+                            kbase += __popc(bm);
                         }
-                        if (keep[j]) {
-                            uint32_t k = kbase + (lane ? __popc(bm >> (32 - lane)) : 0u);
-                            uint32_t field = ((bits[j] >> 15) << (7 - t_bits)) | ((bits[j] & 0x7Fu) >> t_bits);
-                            atomicOr(&s_fix[warp][nj + k / per], field_bits_in_word(field, k % per, t_bits));
-                            uint32_t p = ubase + incl - 1;
-                            if ((p >> 5) < (uint32_t)kKvStageWords) atomicOr(&s_una[warp][p >> 5], 0x80000000u >> (p & 31));
-                        }
-                        kbase += __popc(bm);
-                        ubase += __shfl_sync(0xffffffffu, incl, 31);
                     }
-                }
-                n_words = (ubase + 31) / 32;
-                if (n_words > (uint32_t)kKvStageWords) {          // record too long for the staging buffer
-                    if (lane == 0) atomicCAS(&st->status, 0, CASS_ERR_CAPACITY);
-                    n_words = kKvStageWords;
+                    n_words = 0;
+                } else {
+                    // ---- Cassandra-1 record: entry words | bitmap | fields; exponent stream staged in s_una ----
+                    const int ew = g.e_words;
+                    uint32_t kbase = 0, ubase = 0;
+#pragma unroll
+                    for (int j = 0; j < kKvMaxPerLane; ++j) {
+                        if (j < nj) {
+                            // entry point of slice j: code bits of all kept values in lower channels
+                            if (j > 0 && lane == 0) s_fix[warp][(j - 1) / 3] |= (ubase & 0x3FFu) << (20 - 10 * ((j - 1) % 3));
+                            uint32_t bm = __brev(__ballot_sync(0xffffffffu, keep[j]));   // channel c at bit 31 - c%32
+                            if (lane == 0) s_fix[warp][ew + j] = bm;
+                            uint32_t len = keep[j] ? (uint32_t)exp_to_rank[(bits[j] >> 7) & 0xFF] + 1u : 0u;
+                            uint32_t incl = len;
+#pragma unroll
+                            for (int o = 1; o < 32; o <<= 1) {
+                                uint32_t v = __shfl_up_sync(0xffffffffu, incl, o);
+                                if (lane >= o) incl += v;
+                            }
+                            if (keep[j]) {
+                                uint32_t k = kbase + (lane ? __popc(bm >> (32 - lane)) : 0u);
+                                uint32_t field = ((bits[j] >> 15) << (7 - t_bits)) | ((bits[j] & 0x7Fu) >> t_bits);
+                                atomicOr(&s_fix[warp][ew + nj + k / per], field_bits_in_word(field, k % per, t_bits));
+                                uint32_t p = ubase + incl - 1;
+                                if ((p >> 5) < (uint32_t)kKvStageWords) atomicOr(&s_una[warp][p >> 5], 0x80000000u >> (p & 31));
+                            }
+                            kbase += __popc(bm);
+                            ubase += __shfl_sync(0xffffffffu, incl, 31);
+                        }
+                    }
+                    n_words = (ubase + 31) / 32;
+                    if (ubase > (uint32_t)kv_code_budget(g.kept)) {
+                        // the codewords take more room than raw exponents would (or their offsets leave the entry
+                        // words): store the kept exponents as bytes instead and flag the record
+                        __syncwarp();
+                        for (int w = lane; w < kKvStageWords; w += 32) s_una[warp][w] = 0;
+                        for (int w = lane; w < ew; w += 32) s_fix[warp][w] = w == 0 ? kKvRawFlag : 0u;
+                        __syncwarp();
+                        uint32_t kb2 = 0;
+#pragma unroll
+                        for (int j = 0; j < kKvMaxPerLane; ++j) {
+                            if (j < nj) {
+                                const uint32_t bm = __brev(__ballot_sync(0xffffffffu, keep[j]));
+                                if (keep[j]) {
+                                    const uint32_t k = kb2 + (lane ? __popc(bm >> (32 - lane)) : 0u);
+                                    if ((k >> 2) < (uint32_t)kKvStageWords)
+                                        atomicOr(&s_una[warp][k >> 2], ((bits[j] >> 7) & 0xFFu) << (24 - 8 * (k & 3)));
+                                }
+                                kb2 += __popc(bm);
+                            }
+                        }
+                        n_words = (uint32_t)ceil_div(g.kept, 4);
+                    }
+                    if (n_words > (uint32_t)kKvStageWords) {          // cannot happen for head_dim <= 256
+                        if (lane == 0) atomicCAS(&st->status, 0, CASS_ERR_CAPACITY);
+                        n_words = kKvStageWords;
+                    }
                 }
             }
             if (lane == 0) s_nw[warp] = active ? n_words : 0u;

@@ -54,7 +54,7 @@ struct Plan {
 
 static int check_desc(const cass_model_desc* d, const cass_format* f) {
     if (!d || !f) return CASS_ERR_INVALID_ARG;
-    if (f->mode != 1 && f->mode != 2) return CASS_ERR_UNSUPPORTED;     // weights: Cassandra-1 or Cassandra-2; KV: Cassandra-1
+    if (f->mode != 1 && f->mode != 2) return CASS_ERR_UNSUPPORTED;     // weights: Cassandra-1 or Cassandra-2; KV: see kv_mode
     if (d->max_batch != 1 && d->max_batch != 2 && d->max_batch != 4 && d->max_batch != 8) return CASS_ERR_UNSUPPORTED;
     if (d->n_layers <= 0 || d->hidden <= 0 || d->n_q_heads <= 0 || d->n_kv_heads <= 0 || d->head_dim <= 0 ||
         d->ffn <= 0 || d->vocab <= 0 || d->max_seq < 2 * kMaxVerifyRows)
@@ -67,6 +67,7 @@ static int check_desc(const cass_model_desc* d, const cass_format* f) {
     if (f->kv_prune_permille < 0 || f->kv_prune_permille > 999 || f->kv_trunc_bits < 0 || f->kv_trunc_bits > 7)
         return CASS_ERR_INVALID_ARG;
     if (f->kv_trunc_bits != 0 && f->kv_trunc_bits != 4) return CASS_ERR_UNSUPPORTED;    // draft attention walks t = 0 or 4 records
+    if (f->kv_mode < 0 || f->kv_mode > 2) return CASS_ERR_INVALID_ARG;
     return CASS_OK;
 }
 
@@ -77,13 +78,17 @@ static KvGeom make_kv_geom(const cass_model_desc& d, const cass_format& f) {
     g.n_prune = (d.head_dim * f.kv_prune_permille) / 1000;
     g.kept = d.head_dim - g.n_prune;
     g.t = f.kv_trunc_bits;
+    g.mode = f.kv_mode == 2 ? 2 : 1;
     int per = 32 / (8 - g.t);
     g.bm_words = d.head_dim / 32;
     g.f_words = ceil_div(g.kept, per);
-    g.wpt = g.bm_words + g.f_words;
-    // arena: room for a mean code length of 6 bits per kept value, at least 2 words per token
-    int wcap = ceil_div(g.kept * 6, 32);
-    g.arena_words = d.max_seq * (wcap < 2 ? 2 : wcap);
+    g.e_words = g.mode == 1 ? kv_entry_words(d.head_dim) : 0;
+    g.x_words = g.mode == 2 ? ceil_div(g.bm_words, 4) : 0;
+    g.wpt = g.e_words + g.bm_words + g.f_words + g.x_words;
+    // arena: the most a record can take (raw exponents: one byte per kept value), so that only the end of the cache
+    // itself can exhaust it; Cassandra-2 records have no variable part
+    g.rec_words_max = g.mode == 1 ? ceil_div(8 * g.kept, 32) : 0;
+    g.arena_words = g.mode == 1 ? d.max_seq * (g.rec_words_max < 1 ? 1 : g.rec_words_max) : 32;
     return g;
 }
 

@@ -131,7 +131,7 @@ __global__ void __launch_bounds__(kVaThreads) k_verify_attn(KvGeom g, const uint
 }
 
 int launch_attn_merge(const AttnScratch& sc, int n_chunks_alloc, int chunk_tokens, int rows, int rps, int n_q, int d,
-                      const DevState* st, int draft_mode, uint16_t* out, cudaStream_t s);
+                      const DevState* st, int draft_mode, int draft_units, uint16_t* out, cudaStream_t s);
 
 int launch_verify_attn(const KvGeom& g, const uint16_t* k_cache, const uint16_t* v_cache, const uint16_t* qkv, int n_seq,
                        int rps, int n_q, const DevState* st, const AttnScratch& sc, uint16_t* out, cudaStream_t s) {
@@ -148,7 +148,7 @@ int launch_verify_attn(const KvGeom& g, const uint16_t* k_cache, const uint16_t*
     }
     dim3 grid(n_chunks, g.n_kv, n_seq);
     CASS_PDL_LAUNCH(k_verify_attn, grid, dim3(kVaThreads), smem, s, g, k_cache, v_cache, qkv, rps, n_q, st, sc, n_chunks);
-    return launch_attn_merge(sc, n_chunks, kAttnChunk, n_seq * rps, rps, n_q, g.d, st, 0, out, s);
+    return launch_attn_merge(sc, n_chunks, kAttnChunk, n_seq * rps, rps, n_q, g.d, st, 0, 0, out, s);
 }
 
 }  // namespace cass

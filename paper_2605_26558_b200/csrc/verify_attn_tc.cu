@@ -216,7 +216,7 @@ __global__ void __launch_bounds__(kVtThreads) k_verify_attn_tc(const __grid_cons
 }
 
 int launch_attn_merge(const AttnScratch& sc, int n_chunks_alloc, int chunk_tokens, int rows, int rps, int n_q, int d,
-                      const DevState* st, int draft_mode, uint16_t* out, cudaStream_t s);
+                      const DevState* st, int draft_mode, int draft_units, uint16_t* out, cudaStream_t s);
 
 bool verify_attn_tc_usable(const KvGeom& g, int rps, int n_q) {
     return g.d == kVtD && rps * (n_q / g.n_kv) <= kVtMaxPairs && (g.seq_stride % 16) == 0;
@@ -260,7 +260,7 @@ int launch_verify_attn_tc(const KvGeom& g, const uint16_t* k_cache, const uint16
         CASS_PDL_LAUNCH(k_verify_attn_tc<64>, grid, dim3(kVtThreads), (size_t)vt_smem(64), s, mk, mv, qkv, rps, n_q, g.n_kv, st, sc,
                         n_chunks, d_status);
     }
-    return launch_attn_merge(sc, n_chunks, kVtTok, n_seq * rps, rps, n_q, g.d, st, 0, out, s);
+    return launch_attn_merge(sc, n_chunks, kVtTok, n_seq * rps, rps, n_q, g.d, st, 0, 0, out, s);
 }
 
 }  // namespace cass

@@ -236,8 +236,8 @@ def test_batched_draft_attention_and_kv_records(cass):
             offs = mem32[oo: oo + n_tok + 1].cpu().numpy().view(np.uint32)
             arena = mem32[ao: ao + int(offs[-1])].cpu().numpy().view(np.uint32)
             for tok in range(n_tok):
-                bm, fl, un = layout.encode_kv_token(xb[tok, 1], 400, 4, inv)
-                assert np.array_equal(fixed[tok // 32, :, tok % 32], np.concatenate([bm, fl])), (b, kind, tok)
+                fx, un = layout.encode_kv_token(xb[tok, 1], 400, 4, inv)
+                assert np.array_equal(fixed[tok // 32, :, tok % 32], fx), (b, kind, tok)
                 assert np.array_equal(arena[offs[tok]: offs[tok + 1]], un), (b, kind, tok)
         one.close()
     both.close()

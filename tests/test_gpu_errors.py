@@ -154,9 +154,9 @@ def test_empty_and_single_position_inputs(cass):
     eng.encode_weights(None)
     eng.build_kv_codebook()
     toks, stats = eng.generate(6, 2)
-    # A codebook frozen after a single position ranks most later exponents badly; their long codewords may fill
-    # the compressed cache's code arena (sized for a mean of 6 bits per kept value), which the status word reports.
-    assert len(toks) >= 6 and eng.status()[0] in (0, cass.ERR_CAPACITY)
+    # A codebook frozen after a single position ranks most later exponents badly; records whose codewords would take
+    # more than 8 bits per kept value store their exponents raw, and the arena is sized for that: no capacity error.
+    assert len(toks) >= 6 and eng.status()[0] == 0
     eng.close()
 
 

@@ -159,7 +159,7 @@ def test_kv_encoder_records_bit_exact_heads_of_128(cass):
     """cass_kv_append with the head geometry every benchmark config uses (8 KV heads of 128, p = 40 %, t = 4; four
     elements per lane): three 32-token blocks of records against the oracle's encoder, bit for bit.  Among the appended
     tokens: one whose magnitudes are all equal (the tie rule: the lower channels are pruned), one whose exponents
-    rank badly in the frozen codebook (codewords that span many words), one of zeros."""
+    rank badly in the frozen codebook (so badly that the record stores them raw), one of zeros."""
     eng = _kv_engine(cass)
     n0, n1, d, p, t = 40, 30, 128, 400, 4
     k, v = synth.kv_fill(n0 + n1, 8, d, 5, "k128/kv")
@@ -180,7 +180,7 @@ def test_kv_encoder_records_bit_exact_heads_of_128(cass):
     torch.cuda.synchronize()
     assert eng.status()[0] == 0
     base, mem32 = eng.mem.data_ptr(), eng.mem.view(torch.int32)
-    longest = 0
+    longest, raw_seen = 0, 0
     for kind, x in ((0, k), (1, v)):
         xb = _bits(x)
         cb = layout.kv_codebook(xb[:n0], p)
@@ -197,11 +197,13 @@ def test_kv_encoder_records_bit_exact_heads_of_128(cass):
             offs = mem32[oo: oo + n0 + n1 + 1].cpu().numpy().view(np.uint32)
             arena = mem32[ao: ao + int(offs[-1])].cpu().numpy().view(np.uint32)
             for tok in range(n0 + n1):
-                bm, fl, un = layout.encode_kv_token(xb[tok, head], p, t, inv)
-                assert np.array_equal(fixed[tok // 32, :, tok % 32], np.concatenate([bm, fl])), (kind, head, tok)
+                fx, un = layout.encode_kv_token(xb[tok, head], p, t, inv)
+                assert np.array_equal(fixed[tok // 32, :, tok % 32], fx), (kind, head, tok)
                 assert np.array_equal(arena[offs[tok]: offs[tok + 1]], un), (kind, head, tok)
                 longest = max(longest, un.size)
-    assert longest > 12                                   # a record beyond the draft attention's staged code words
+                raw_seen += int(fx[0] >> 31)
+    # the spread tokens' codewords would take more than 8 bits per kept value: their exponents are stored raw
+    assert longest == 20 and raw_seen >= 8
     # the tie rule, stated directly: with equal magnitudes the floor(128 * 0.4) = 51 lowest channels go
     keep = codec.keep_mask_kv(_bits(k[n0 + 3]), p)
     assert not keep[:, :51].any() and keep[:, 51:].all()

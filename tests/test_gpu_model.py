@@ -261,8 +261,8 @@ def test_kv_encoder_records_bit_exact(cass, tiny):
             arena = mem32[ao: ao + int(offs[-1])].cpu().numpy().view(np.uint32)
             assert offs[0] == 0
             for tok in range(n0 + n1):
-                bm, fl, un = layout.encode_kv_token(xb[tok, head], p, t, inv)
-                assert np.array_equal(fixed[tok // 32, :, tok % 32], np.concatenate([bm, fl])), (kind, head, tok)
+                fx, un = layout.encode_kv_token(xb[tok, head], p, t, inv)
+                assert np.array_equal(fixed[tok // 32, :, tok % 32], fx), (kind, head, tok)
                 assert offs[tok + 1] - offs[tok] == un.size, (kind, head, tok)
                 assert np.array_equal(arena[offs[tok]: offs[tok + 1]], un), (kind, head, tok)
             cache_off = (view.k_or_v_bf16 - base) // 2

@@ -272,9 +272,9 @@ def test_kv_record_round_trip():
             inv = codec.invert_codebook(cb)
             for tok in range(0, 40, 7):
                 for h in range(2):
-                    bm, fl, un = layout.encode_kv_token(xb[tok, h], p, t, inv)
-                    assert bm.size + fl.size == layout.kv_fixed_words(64, p, t)
-                    dec = layout.decode_kv_token(bm, fl, un, 64, t, cb)
+                    fixed, un = layout.encode_kv_token(xb[tok, h], p, t, inv)
+                    assert fixed.size == layout.kv_fixed_words(64, p, t)
+                    dec = layout.decode_kv_token(fixed, un, 64, p, t, cb)
                     keep = codec.keep_mask_kv(xb[tok, h], p)
                     assert np.array_equal(dec, codec.draft_bits(xb[tok, h], keep, t))
 
