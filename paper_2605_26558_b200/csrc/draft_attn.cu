@@ -66,9 +66,10 @@ struct EmitV {
 // ---- Cassandra-1 slice -------------------------------------------------------------------------------------------
 // Careful walk of a slice's values [e_from, n): any codeword length, raw exponents too.  `un` points at the record's
 // first exponent word, words `us` apart.
+// The emitter travels by value (in registers): a reference would pin it to local memory in the fast path too.
 template <int T, class Emit>
-__device__ __noinline__ void kv_slice_slow(uint32_t bv, const uint32_t* fl, uint32_t fi, const uint32_t* un, int us,
-                                           uint32_t upos, uint32_t upos_lim, bool raw, int n, const uint32_t* lut, Emit& em) {
+__device__ __noinline__ Emit kv_slice_slow(uint32_t bv, const uint32_t* fl, uint32_t fi, const uint32_t* un, int us,
+                                           uint32_t upos, uint32_t upos_lim, bool raw, int n, const uint32_t* lut, Emit em) {
     constexpr int F = 8 - T, PER = 32 / F;
     constexpr uint32_t MASK = 0x80000000u | (((1u << (7 - T)) - 1u) << (16 + T));
     for (int e = 0; e < n && bv; ++e, ++fi) {
@@ -92,64 +93,59 @@ __device__ __noinline__ void kv_slice_slow(uint32_t bv, const uint32_t* fl, uint
         const uint32_t a = __funnelshift_l(fword, fword, (F * (fi % PER)) & 31);
         em.put(31u - p, __uint_as_float((a & MASK) | eb));
     }
+    return em;
 }
 
 // One slice of a Cassandra-1 record per lane.  B: the slice's bitmap word; fi: index of its first field; upos: bit
 // offset of its first codeword in the staged stream (words 128 bytes apart from un_a); n: its kept values (0 for
-// lanes that only keep the warp in step).  Groups of 8 values, 4 codewords per 32-bit window; a window that runs dry
-// sends that lane through the careful walk for the rest of its slice.
+// lanes that only keep the warp in step).  Groups of 4 values = one 32-bit code window; a window that runs dry sends
+// that lane through the careful walk for the rest of its slice.
 template <int T, class Emit>
 __device__ __forceinline__ void kv_slice_walk(uint32_t B, uint32_t fi, uint32_t upos, int n, uint32_t fl_a, const uint32_t* flP,
                                               uint32_t un_a, const uint32_t* unP, uint32_t upos_lim, uint32_t lut_a,
                                               const uint32_t* lutP, Emit& em) {
-    constexpr int F = 8 - T, PER = 32 / F, NFW = kGroupCols / PER;
+    constexpr int F = 8 - T, PER = 32 / F, GS = kGroupCodes;
+    static_assert(GS <= PER, "a group's fields lie in two consecutive words");
     constexpr uint32_t MASK = 0x80000000u | (((1u << (7 - T)) - 1u) << (16 + T));
-    const int n_groups = ceil_div(__reduce_max_sync(0xffffffffu, n), kGroupCols);
+    const int n_groups = ceil_div(__reduce_max_sync(0xffffffffu, n), GS);
     uint32_t bv = B;
     bool slow = false;
     for (int grp = 0; grp < n_groups; ++grp) {
-        const int rem = n - grp * kGroupCols;                                 // values this lane still has (may be <= 0)
+        const int rem = n - grp * GS;                                         // values this lane still has (may be <= 0)
         const uint32_t fw_a = fl_a + (fi / PER) * 128u, j0 = fi % PER;
-        uint32_t fwd[NFW + 1];
-#pragma unroll
-        for (int i = 0; i <= NFW; ++i) fwd[i] = da_lds(fw_a + 128u * i);
+        const uint32_t f0 = da_lds(fw_a), f1 = da_lds(fw_a + 128u);
         const uint32_t bv0 = bv, upos0 = upos;
-        uint32_t cols[kGroupCols], wbs[kGroupCols];
-        uint32_t dry = 0;
+        const uint32_t ua = un_a + (upos >> 5) * 128u;
+        uint32_t uv = __funnelshift_l(da_lds(ua + 128u), da_lds(ua), upos);                // 32 code bits from upos on
+        uint32_t la = lut_a + 124u, q = 0, dry = 0;
+        uint32_t cols[GS], wbs[GS];
 #pragma unroll
-        for (int half = 0; half < kGroupCols / kGroupCodes; ++half) {
-            const uint32_t ua = un_a + (upos >> 5) * 128u;
-            uint32_t uv = __funnelshift_l(da_lds(ua + 128u), da_lds(ua), upos);            // 32 code bits from upos on
-            uint32_t la = lut_a + 124u, q = 0;
-#pragma unroll
-            for (int j = 0; j < kGroupCodes; ++j) {
-                const int e = half * kGroupCodes + j;
-                const uint32_t p = da_bfind(bv);
-                bv &= ~da_shl(1u, p);
-                q = da_bfind(uv);
-                const uint32_t eb = da_lds(la - (q & 31u) * 4u);                           // lut[previous - q - 1]
-                la = lut_a - 4u + (q & 31u) * 4u;
-                uv &= ~da_shl(1u, q);
-                const uint32_t jj = j0 + e;                                                // field jj of the group's words
-                const uint32_t fword = (jj >= (uint32_t)(PER * ((e / PER) + 1))) ? fwd[e / PER + 1] : fwd[e / PER];
-                const uint32_t a = __funnelshift_l(fword, fword, (F * jj) & 31);
-                cols[e] = 31u - (p & 31u);
-                wbs[e] = (a & MASK) | eb;
-                if (e < rem) dry |= q;                                                     // sign bit set: the window ran dry
-            }
-            upos = min(upos + 32u - (q & 31u), upos_lim);
+        for (int e = 0; e < GS; ++e) {
+            const uint32_t p = da_bfind(bv);
+            bv &= ~da_shl(1u, p);
+            q = da_bfind(uv);
+            const uint32_t eb = da_lds(la - (q & 31u) * 4u);                               // lut[previous - q - 1]
+            la = lut_a - 4u + (q & 31u) * 4u;
+            uv &= ~da_shl(1u, q);
+            const uint32_t jj = j0 + e;                                                    // field jj of the two words
+            const uint32_t fword = jj >= (uint32_t)PER ? f1 : f0;
+            const uint32_t a = __funnelshift_l(fword, fword, (F * jj) & 31);
+            cols[e] = 31u - (p & 31u);
+            wbs[e] = (a & MASK) | eb;
+            if (e < rem) dry |= q;                                                         // sign bit set: the window ran dry
         }
+        upos = min(upos + 32u - (q & 31u), upos_lim);
         if (rem > 0 && !slow) {
             if ((int32_t)dry < 0) {
                 slow = true;                             // finish this slice one value at a time, from the group's start
-                kv_slice_slow<T>(bv0, flP, fi, unP, 32, upos0, upos_lim, false, rem, lutP, em);
+                em = kv_slice_slow<T>(bv0, flP, fi, unP, 32, upos0, upos_lim, false, rem, lutP, em);
             } else {
 #pragma unroll
-                for (int e = 0; e < kGroupCols; ++e)
+                for (int e = 0; e < GS; ++e)
                     if (e < rem) em.put(cols[e], __uint_as_float(wbs[e]));
             }
         }
-        fi += kGroupCols;
+        fi += GS;
     }
 }
 
@@ -177,11 +173,19 @@ __device__ __forceinline__ void kv_slice_walk_mx(uint32_t B, uint32_t fi, int n,
     }
 }
 
+// 4-byte asynchronous copy global -> shared; `take` false writes a zero instead (nothing is read).
+__device__ __forceinline__ void da_cp_async4(uint32_t dst, const void* src, bool take) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(src), "r"(take ? 4 : 0) : "memory");
+}
+__device__ __forceinline__ void da_cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void da_cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+
 template <int MODE, int T, int GQ>
-__global__ void __launch_bounds__(512) k_draft_attn(KvGeom g, KvComp ck0, KvComp cv0, const uint16_t* __restrict__ qkv,
-                                                    int qkv_stride, int n_q, const DevState* __restrict__ st, AttnScratch sc,
-                                                    int n_chunks_alloc, int stage) {
+__global__ void __launch_bounds__(512, 2) k_draft_attn(KvGeom g, KvComp ck0, KvComp cv0, const uint16_t* __restrict__ qkv,
+                                                       int qkv_stride, int n_q, const DevState* __restrict__ st, AttnScratch sc,
+                                                       int n_chunks_alloc, int stage, uint16_t* __restrict__ out) {
     extern __shared__ __align__(16) uint8_t smem[];
+    __shared__ int s_last;
     pdl_early<2>();
     pdl_wait();
     const int head = blockIdx.y, seq = blockIdx.z;
@@ -195,15 +199,16 @@ __global__ void __launch_bounds__(512) k_draft_attn(KvGeom g, KvComp ck0, KvComp
     qkv += (size_t)seq * qkv_stride;
 
     const int vrow = d + 2;                                                   // halfwords per row of the V tile (padded)
+    const int fsz = (g.wpt + 2) * 32, usz = (stage + 2) * 32;
     float* q_s = reinterpret_cast<float*>(smem);                              // [d][GQ]
     float* part_s = q_s + d * GQ;                                             // [S][GQ][32] partial q.k of the slices
-    float* sc_s = part_s + S * GQ * kDaSub;                                   // [GQ][32] probabilities of the pass
+    float* sc_s = part_s + S * GQ * kDaSub;                                   // [32][GQ] probabilities of the pass
     float* run_s = sc_s + GQ * kDaSub;                                        // [GQ][4]: running max, running sum, rescale factor
     uint32_t* lut_s = reinterpret_cast<uint32_t*>(run_s + 4 * GQ);            // mode 1: [2][256] rank -> exponent << 23; mode 2: [256] field values
-    uint32_t* meta_s = lut_s + 512;                                           // [2][32] arena offset, [2][32] arena words of the pass's records
-    uint32_t* fix_s = meta_s + 128;                                           // [2][wpt + 2][32]
-    uint32_t* una_s = fix_s + 2 * (g.wpt + 2) * 32;                           // [2][stage + 2][32] (mode 1)
-    uint16_t* v_s = reinterpret_cast<uint16_t*>(una_s + (MODE == 1 ? 2 * (stage + 2) * 32 : 0));   // [32][vrow] bf16
+    uint32_t* meta_s = lut_s + 512;                                           // [2 buffers][2 kinds][34]: arena offsets of 32 tokens + the next
+    uint32_t* fix_s = meta_s + 2 * 2 * 34;                                    // [2 buffers][2 kinds][wpt + 2][32]
+    uint32_t* una_s = fix_s + 2 * 2 * fsz;                                    // [2 buffers][2 kinds][stage + 2][32] (mode 1)
+    uint16_t* v_s = reinterpret_cast<uint16_t*>(una_s + (MODE == 1 ? 2 * 2 * usz : 0));   // [32][vrow] bf16
 
     const float scale = rsqrtf((float)d);
     for (int i = tid; i < d * GQ; i += n_thr) {
@@ -221,50 +226,77 @@ __global__ void __launch_bounds__(512) k_draft_attn(KvGeom g, KvComp ck0, KvComp
         }
     }
     if (tid < 4 * GQ) run_s[tid] = (tid & 3) == 0 ? -INFINITY : 0.f;
+    for (int i = tid; i < 2 * 2 * 2 * 32; i += n_thr) fix_s[(i / 64) * fsz + g.wpt * 32 + (i % 64)] = 0u;   // the two slack rows of every block stay zero
+    if (MODE == 1) for (int i = tid; i < 2 * 2 * 2 * 32; i += n_thr) una_s[(i / 64) * usz + stage * 32 + (i % 64)] = 0u;
 
     const int kind = warp / S, slice = warp % S;                              // warps 0..S-1: K slices, S..2S-1: V slices
-    const KvComp& c = kind ? cv0 : ck0;                                       // sequence 0's; shifted to this sequence where used
-    const uint32_t* fixed_k = of_seq(ck0.fixed, seq, g.seq_stride) + (size_t)head * g.n_blocks * g.wpt * 32;
-    const uint32_t* fixed_v = of_seq(cv0.fixed, seq, g.seq_stride) + (size_t)head * g.n_blocks * g.wpt * 32;
-    const uint32_t* off_k = of_seq(ck0.off, seq, g.seq_stride) + (size_t)head * (g.max_seq + 1);
-    const uint32_t* off_v = of_seq(cv0.off, seq, g.seq_stride) + (size_t)head * (g.max_seq + 1);
-    const uint32_t* arena_k = of_seq(ck0.arena, seq, g.seq_stride) + (size_t)head * g.arena_words;
-    const uint32_t* arena_v = of_seq(cv0.arena, seq, g.seq_stride) + (size_t)head * g.arena_words;
-    (void)c;
-    const int fsz = (g.wpt + 2) * 32, usz = (stage + 2) * 32;
+    const uint32_t* fixed_kv[2] = {of_seq(ck0.fixed, seq, g.seq_stride) + (size_t)head * g.n_blocks * g.wpt * 32,
+                                   of_seq(cv0.fixed, seq, g.seq_stride) + (size_t)head * g.n_blocks * g.wpt * 32};
+    const uint32_t* off_kv[2] = {of_seq(ck0.off, seq, g.seq_stride) + (size_t)head * (g.max_seq + 1),
+                                 of_seq(cv0.off, seq, g.seq_stride) + (size_t)head * (g.max_seq + 1)};
+    const uint32_t* arena_kv[2] = {of_seq(ck0.arena, seq, g.seq_stride) + (size_t)head * g.arena_words,
+                                   of_seq(cv0.arena, seq, g.seq_stride) + (size_t)head * g.arena_words};
+    const int n_warps = n_thr / 32;
+
+    // Staging runs ahead of the decode through asynchronous copies: the arena offsets of a pass two passes early, its
+    // fixed-part blocks and exponent words one pass early, into the buffer the pass before the last has left.  A warp
+    // copies whole rows (word w of the 32 tokens), lane = token.
+    auto stage_meta = [&](int t0, int buf) {               // offsets off[t0 .. t0 + 32] of both kinds
+        if (MODE == 1 && warp < 2) {
+            const bool in_run = t0 < t_end;
+            const bool take = in_run && t0 + lane <= cur_len;
+            da_cp_async4(smem_u32(meta_s + (buf * 2 + warp) * 34 + lane), off_kv[warp] + (take ? t0 + lane : 0), take);
+            if (lane == 0) {
+                const bool take2 = in_run && t0 + 32 <= cur_len;
+                da_cp_async4(smem_u32(meta_s + (buf * 2 + warp) * 34 + 32), off_kv[warp] + (take2 ? t0 + 32 : 0), take2);
+            }
+        }
+    };
+    auto stage_records = [&](int t0, int buf) {
+        if (t0 >= t_end) return;
+        const size_t blk = (size_t)(t0 / 32) * g.wpt * 32;
+        for (int row = warp; row < 2 * g.wpt; row += n_warps) {
+            const int kd = row >= g.wpt, w = row - kd * g.wpt;
+            da_cp_async4(smem_u32(fix_s + (buf * 2 + kd) * fsz + w * 32 + lane), fixed_kv[kd] + blk + w * 32 + lane, true);
+        }
+        if (MODE == 1) {
+            const bool tok_ok = t0 + lane < cur_len;
+            uint32_t o0[2], nw[2];
+#pragma unroll
+            for (int kd = 0; kd < 2; ++kd) {
+                const uint32_t* m = meta_s + (buf * 2 + kd) * 34 + lane;
+                o0[kd] = m[0];
+                nw[kd] = m[1] - m[0];
+                if (!tok_ok || nw[kd] > (uint32_t)stage) nw[kd] = 0;          // longer records are read in place
+            }
+            for (int row = warp; row < 2 * stage; row += n_warps) {
+                const int kd = row >= stage, w = row - kd * stage;
+                const bool take = (uint32_t)w < nw[kd];
+                da_cp_async4(smem_u32(una_s + (buf * 2 + kd) * usz + w * 32 + lane), arena_kv[kd] + (take ? o0[kd] + w : 0), take);
+            }
+        }
+    };
+    stage_meta(t_begin, 0);
+    stage_meta(t_begin + kDaSub, 1);
+    da_cp_async_wait_all();
+    __syncthreads();
+    stage_records(t_begin, 0);
+    da_cp_async_wait_all();
+    __syncthreads();
+
     float o_acc[GQ];
 #pragma unroll
     for (int gi = 0; gi < GQ; ++gi) o_acc[gi] = 0.f;
 
-    for (int t0 = t_begin; t0 < t_end; t0 += kDaSub) {
-        // ---- stage the pass: both fixed-part blocks (coalesced), the V tile cleared, the exponent words of its records ----
-        const int blk = t0 / 32;
-        for (int i = tid; i < 2 * fsz; i += n_thr) {
-            const int kd = i / fsz, w = i % fsz;
-            fix_s[i] = w < g.wpt * 32 ? (kd ? fixed_v : fixed_k)[(size_t)blk * g.wpt * 32 + w] : 0u;
-        }
-        for (int i = tid; i < kDaSub * vrow / 2; i += n_thr) reinterpret_cast<uint32_t*>(v_s)[i] = 0u;
-        if (MODE == 1 && tid < 64) {
-            const int kd = tid >> 5, tok = t0 + (tid & 31);
-            uint32_t o0 = 0, nw = 0;
-            if (tok < cur_len) { const uint32_t* off = kd ? off_v : off_k; o0 = off[tok]; nw = off[tok + 1] - o0; }
-            meta_s[kd * 32 + (tid & 31)] = o0;
-            meta_s[64 + kd * 32 + (tid & 31)] = nw;
-        }
-        __syncthreads();
-        if (MODE == 1) {
-            for (int i = tid; i < 2 * usz; i += n_thr) {
-                const int kd = i / usz, w = (i % usz) / 32, tk = i % 32;
-                const uint32_t nw = meta_s[64 + kd * 32 + tk];
-                una_s[i] = (nw <= (uint32_t)stage && (uint32_t)w < nw) ? (kd ? arena_v : arena_k)[meta_s[kd * 32 + tk] + w] : 0u;
-            }
-            __syncthreads();
-        }
+    int pass = 0;
+    for (int t0 = t_begin; t0 < t_end; t0 += kDaSub, ++pass) {
+        const int buf = pass & 1;
+        stage_records(t0 + kDaSub, buf ^ 1);               // the next pass's records travel while this pass is decoded
         // ---- decode: warp (kind, slice), lane = token ----
         if (warp < 2 * S) {
             const int tok = t0 + lane;
             const bool valid = tok < cur_len;
-            const uint32_t* fx = fix_s + kind * fsz + lane;                      // word w of this token at fx[w * 32]
+            const uint32_t* fx = fix_s + (buf * 2 + kind) * fsz + lane;          // word w of this token at fx[w * 32]
             const int bm0 = MODE == 1 ? g.e_words : 0;
             const uint32_t B = fx[(bm0 + slice) * 32];
             uint32_t fi = 0;
@@ -276,24 +308,29 @@ __global__ void __launch_bounds__(512) k_draft_attn(KvGeom g, KvComp ck0, KvComp
             ek.q_a = smem_u32(q_s + (size_t)slice * 32 * GQ);
             ev.row_a = smem_u32(v_s + (size_t)lane * vrow + slice * 32);
             ek.init();
+            if (kind == 1) {                              // a V lane owns its token's 32 channels of the tile: clear them first
+#pragma unroll
+                for (int i = 0; i < 16; ++i) asm volatile("st.shared.u32 [%0], %1;" ::"r"(ev.row_a + 4u * i), "r"(0u));
+            }
             if (MODE == 1) {
                 const uint32_t e0 = fx[0];
                 const bool raw = (e0 & kKvRawFlag) != 0;
                 const uint32_t upos = slice == 0 ? 0u : (fx[((slice - 1) / 3) * 32] >> (20 - 10 * ((slice - 1) % 3))) & 0x3FFu;
-                const uint32_t nw = meta_s[64 + kind * 32 + lane];
+                const uint32_t* m = meta_s + (buf * 2 + kind) * 34 + lane;
+                const uint32_t o0 = m[0], nw = valid ? m[1] - m[0] : 0u;
                 const bool staged = nw <= (uint32_t)stage;
                 const bool fast = valid && !raw && staged;
                 const uint32_t* lutP = lut_s + kind * 256;
-                const uint32_t* unP = una_s + kind * usz + lane;
+                const uint32_t* unP = una_s + (buf * 2 + kind) * usz + lane;
                 const uint32_t upos_lim = (uint32_t)stage * 32u;
                 if (kind == 0) kv_slice_walk<T>(B, fi, upos, fast ? n : 0, fl_a, fx + (bm0 + g.bm_words) * 32, smem_u32(unP), unP, upos_lim,
                                                 smem_u32(lutP), lutP, ek);
                 else kv_slice_walk<T>(B, fi, upos, fast ? n : 0, fl_a, fx + (bm0 + g.bm_words) * 32, smem_u32(unP), unP, upos_lim,
                                       smem_u32(lutP), lutP, ev);
                 if (valid && !fast) {                     // raw exponents, or a record longer than the staging: read it in place
-                    const uint32_t* un = (kind ? arena_v : arena_k) + meta_s[kind * 32 + lane];
-                    if (kind == 0) kv_slice_slow<T>(B, fx + (bm0 + g.bm_words) * 32, fi, un, 1, upos, nw * 32u, raw, n, lutP, ek);
-                    else kv_slice_slow<T>(B, fx + (bm0 + g.bm_words) * 32, fi, un, 1, upos, nw * 32u, raw, n, lutP, ev);
+                    const uint32_t* un = arena_kv[kind] + o0;
+                    if (kind == 0) ek = kv_slice_slow<T>(B, fx + (bm0 + g.bm_words) * 32, fi, un, 1, upos, nw * 32u, raw, n, lutP, ek);
+                    else ev = kv_slice_slow<T>(B, fx + (bm0 + g.bm_words) * 32, fi, un, 1, upos, nw * 32u, raw, n, lutP, ev);
                 }
             } else {
                 const uint32_t xw = fx[(g.bm_words + g.f_words + slice / 4) * 32];
@@ -308,6 +345,8 @@ __global__ void __launch_bounds__(512) k_draft_attn(KvGeom g, KvComp ck0, KvComp
             }
         }
         __syncthreads();
+        // this pass's offsets are no longer needed: fetch those of the pass after the next into their place
+        stage_meta(t0 + 2 * kDaSub, buf);
         // ---- running softmax: warp gi handles query head gi of the group, lane = token ----
         for (int gi = warp; gi < G; gi += n_thr / 32) {
             float sdot = 0.f;
@@ -318,7 +357,7 @@ __global__ void __launch_bounds__(512) k_draft_attn(KvGeom g, KvComp ck0, KvComp
             const float m_new = fmaxf(m_old, warp_max(sv));                   // finite: the pass has at least one visible token
             const float pr = valid ? expf(sv - m_new) : 0.f;
             const float alpha = expf(m_old - m_new);                          // exp(-inf) = 0 on the first pass
-            sc_s[gi * kDaSub + lane] = pr;
+            sc_s[lane * GQ + gi] = pr;
             const float l_new = l_old * alpha + warp_sum(pr);
             __syncwarp();
             if (lane == 0) { run_s[gi * 4] = m_new; run_s[gi * 4 + 1] = l_new; run_s[gi * 4 + 2] = alpha; }
@@ -332,13 +371,30 @@ __global__ void __launch_bounds__(512) k_draft_attn(KvGeom g, KvComp ck0, KvComp
 #pragma unroll 4
             for (int t = 0; t < n_tok; ++t) {
                 const float v = bf16_bits_to_float(v_s[(size_t)t * vrow + tid]);
-#pragma unroll
-                for (int gi = 0; gi < GQ; ++gi) o_acc[gi] = fmaf(sc_s[gi * kDaSub + t], v, o_acc[gi]);
+                const float4 pa = *reinterpret_cast<const float4*>(sc_s + t * GQ);         // the pass's probabilities [token][GQ]
+                o_acc[0] = fmaf(pa.x, v, o_acc[0]); o_acc[1] = fmaf(pa.y, v, o_acc[1]);
+                o_acc[2] = fmaf(pa.z, v, o_acc[2]); o_acc[3] = fmaf(pa.w, v, o_acc[3]);
+                if constexpr (GQ > 4) {
+                    const float4 pb = *reinterpret_cast<const float4*>(sc_s + t * GQ + 4);
+                    o_acc[4] = fmaf(pb.x, v, o_acc[4]); o_acc[5] = fmaf(pb.y, v, o_acc[5]);
+                    o_acc[6] = fmaf(pb.z, v, o_acc[6]); o_acc[7] = fmaf(pb.w, v, o_acc[7]);
+                }
             }
         }
-        __syncthreads();                                                      // the pass's buffers are free again
+        da_cp_async_wait_all();                            // the next pass's records (and the offsets beyond) have landed
+        __syncthreads();                                   // and the pass's tile and probabilities are free again
     }
     const int chunk = blockIdx.x;
+    const int n_act = ceil_div(cur_len, tpc);                                 // CTAs of this (sequence, head) that have tokens
+    if (n_act == 1) {
+        // the whole visible range in one CTA: normalise and write the output rows directly
+        if (tid < d) {
+#pragma unroll
+            for (int gi = 0; gi < GQ; ++gi)
+                if (gi < G) out[((size_t)seq * n_q + head * G + gi) * d + tid] = float_to_bf16_bits(o_acc[gi] / run_s[gi * 4 + 1]);
+        }
+        return;
+    }
     if (tid < d) {
 #pragma unroll
         for (int gi = 0; gi < GQ; ++gi)
@@ -348,6 +404,46 @@ __global__ void __launch_bounds__(512) k_draft_attn(KvGeom g, KvComp ck0, KvComp
         const size_t pair = (size_t)seq * n_q + head * G + tid;
         sc.m[pair * n_chunks_alloc + chunk] = run_s[tid * 4];
         sc.l[pair * n_chunks_alloc + chunk] = run_s[tid * 4 + 1];
+    }
+    // ---- the CTA that finishes last merges the runs of its (sequence, head): a fixed order, whoever does it ----
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        int* cnt = sc.cnt + seq * g.n_kv + head;
+        const int done = atomicAdd(cnt, 1);
+        s_last = done == n_act - 1;
+        if (s_last) *cnt = 0;                                                 // ready for the next launch
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    // warp gi: weights of query head gi's runs (lane-parallel over the runs); then thread (gi, dim) adds the runs in order
+    float* w_s = reinterpret_cast<float*>(fix_s);                             // [G][n_act] weights e^{m_c - M} (the record buffers are free; size checked at launch)
+    float* L_s = sc_s;                                                        // [GQ]
+    for (int gi = warp; gi < G; gi += n_thr / 32) {
+        const size_t pair = (size_t)seq * n_q + head * G + gi;
+        const float* mp = sc.m + pair * n_chunks_alloc;
+        const float* lp = sc.l + pair * n_chunks_alloc;
+        float M = -INFINITY;
+        for (int c = lane; c < n_act; c += 32) M = fmaxf(M, __ldcg(mp + c));
+        M = warp_max(M);
+        float L = 0.f;
+        for (int c0 = 0; c0 < n_act; c0 += 32) {          // sums of 32 runs at a time, in run order
+            const int c = c0 + lane;
+            float w = 0.f, wl = 0.f;
+            if (c < n_act) { w = expf(__ldcg(mp + c) - M); wl = w * __ldcg(lp + c); w_s[gi * n_act + c] = w; }
+            L += warp_sum(wl);
+        }
+        if (lane == 0) L_s[gi] = L;
+    }
+    __syncthreads();
+    for (int i = tid; i < G * d; i += n_thr) {
+        const int gi = i / d, dim = i % d;
+        const float* op = sc.o + ((size_t)seq * n_q + head * G + gi) * n_chunks_alloc * d + dim;
+        float acc = 0.f;
+#pragma unroll 4
+        for (int c = 0; c < n_act; ++c) acc = fmaf(w_s[gi * n_act + c], __ldcg(op + (size_t)c * d), acc);
+        out[((size_t)seq * n_q + head * G + gi) * d + dim] = float_to_bf16_bits(acc / L_s[gi]);
     }
 }
 
@@ -369,7 +465,7 @@ __global__ void __launch_bounds__(kMergeThreads) k_attn_merge(AttnScratch sc, in
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int seq = r / rps;
     const int vis = st->len[seq] + (draft_mode ? st->inflight[seq] + 1 : r % rps + 1);
-    if (draft_mode) chunk_tokens = da_tokens_per_cta(vis, draft_units);       // the split the draft attention chose for this length
+    if (draft_units > 0) chunk_tokens = da_tokens_per_cta(vis, draft_units);  // runs whose length follows the visible length
     const int n_ch = ceil_div(vis, chunk_tokens);
     const size_t pair = (size_t)r * n_q + hq;
     const float* mp = sc.m + pair * n_chunks_alloc;
@@ -438,17 +534,29 @@ static int draft_attn_stage(const KvGeom& g) { return g.rec_words_max < kDaUnaSt
 
 size_t draft_attn_smem_bytes(const KvGeom& g, int gq) {
     const int S = g.d / 32, stage = draft_attn_stage(g);
-    return (size_t)g.d * gq * 4 + (size_t)S * gq * kDaSub * 4 + (size_t)gq * kDaSub * 4 + 4 * gq * 4 + 512 * 4 + 128 * 4 +
-           (size_t)2 * (g.wpt + 2) * 32 * 4 + (g.mode == 1 ? (size_t)2 * (stage + 2) * 32 * 4 : 0) +
+    return (size_t)g.d * gq * 4 + (size_t)S * gq * kDaSub * 4 + (size_t)gq * kDaSub * 4 + 4 * gq * 4 + 512 * 4 + 2 * 2 * 34 * 4 +
+           (size_t)4 * (g.wpt + 2) * 32 * 4 + (g.mode == 1 ? (size_t)4 * (stage + 2) * 32 * 4 : 0) +
            (size_t)kDaSub * (g.d + 2) * 2 + 64;
 }
 
+int launch_draft_attn_rec(const KvGeom& g, const KvComp& ck, const KvComp& cv, const uint16_t* qkv, int qkv_stride, int n_q,
+                          int n_seq, const DevState* st, const AttnScratch& sc, uint16_t* out, cudaStream_t s);
+
+// Sessions with long caches (more than kDaSliceMaxSeq positions) and Cassandra-1 records use the whole-record kernel,
+// which needs about half the instructions per value; the slice-parallel kernel is the faster one while the grid is small.
+constexpr int kDaSliceMaxSeq = 2048;
+
 int launch_draft_attn(const KvGeom& g, const KvComp& ck, const KvComp& cv, const uint16_t* qkv, int qkv_stride, int n_q,
                       int n_seq, const DevState* st, const AttnScratch& sc, uint16_t* out, cudaStream_t s) {
+    if (g.mode == 1 && g.max_seq > kDaSliceMaxSeq) return launch_draft_attn_rec(g, ck, cv, qkv, qkv_stride, n_q, n_seq, st, sc, out, s);
     const int G = n_q / g.n_kv;
     if (G > kMaxGroup || g.d > 256 || g.d % 32) return CASS_ERR_UNSUPPORTED;
-    const int n_chunks = ceil_div(g.max_seq, kDaSub);        // the most CTAs a head can need (32 tokens each); longer runs use fewer
     const int gq = G <= 4 ? 4 : 8;
+    // the most CTAs a head can need: runs of 32 tokens while that keeps the grid below the target, of 256 at most
+    int n_chunks = 592 / (g.n_kv * n_seq) + 1;
+    if (ceil_div(g.max_seq, 256) > n_chunks) n_chunks = ceil_div(g.max_seq, 256);
+    if (ceil_div(g.max_seq, kDaSub) < n_chunks) n_chunks = ceil_div(g.max_seq, kDaSub);
+    if (G * n_chunks > 4 * (g.wpt + 2) * 32) return CASS_ERR_UNSUPPORTED;        // the merge keeps one weight per (query head, run) in shared memory
     const size_t smem = draft_attn_smem_bytes(g, gq);
     const int stage = draft_attn_stage(g);
     const int threads = 2 * (g.d / 32) * 32;
@@ -460,7 +568,7 @@ int launch_draft_attn(const KvGeom& g, const KvComp& ck, const KvComp& cv, const
             CASS_CUDA_CHECK(cudaFuncSetAttribute((k_draft_attn<MM, TT, GG>), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
             attr = smem;                                                                                             \
         }                                                                                                            \
-        CASS_PDL_LAUNCH((k_draft_attn<MM, TT, GG>), grid, dim3(threads), smem, s, g, ck, cv, qkv, qkv_stride, n_q, st, sc, n_chunks, stage); \
+        CASS_PDL_LAUNCH((k_draft_attn<MM, TT, GG>), grid, dim3(threads), smem, s, g, ck, cv, qkv, qkv_stride, n_q, st, sc, n_chunks, stage, out); \
     } while (0)
 #define CASS_DA_LAUNCH_T(MM)                                                                                          \
     do {                                                                                                             \
@@ -475,7 +583,7 @@ int launch_draft_attn(const KvGeom& g, const KvComp& ck, const KvComp& cv, const
 #undef CASS_DA_LAUNCH_T
 #undef CASS_DA_LAUNCH
     CASS_LAUNCH_CHECK();
-    return launch_attn_merge(sc, n_chunks, kDaSub, n_seq, 1, n_q, g.d, st, 1, g.n_kv * n_seq, out, s);
+    return CASS_OK;                                       // the last CTA of every (sequence, head) has merged its runs
 }
 
 }  // namespace cass

@@ -146,6 +146,7 @@ struct AttnScratch {
     float* o;     // [rows*n_q][n_chunks][d]
     float* m;     // [rows*n_q][n_chunks]
     float* l;     // [rows*n_q][n_chunks]
+    int* cnt;     // [kMaxBatch * n_kv] arrival counters of the draft attention's CTAs, zero between launches
 };
 // Draft: one query row per sequence (qkv row b, `qkv_stride` elements apart) at position len + inflight over that
 // sequence's compressed cache (caches given for sequence 0).

@@ -115,7 +115,7 @@ def bench_verify_gemm(name, copies, iters, rows=5):
             "peak": f"{peak} GB/s ({kind})", "tflops": 2.0 * rows * n * k * copies / (ms * 1e-3) / 1e12}
 
 
-def bench_draft_attn(n_pos, layers, iters):
+def bench_draft_attn(n_pos, layers, iters, kv_mode=1):
     """Draft attention and the KV encoder on `layers` Llama-3-8B-shaped layers (32 q / 8 kv heads of 128) holding
     n_pos synthetic positions each; the layers' compressed caches together exceed L2 for layers * n_pos >= 2.6e5."""
     import synth
@@ -125,7 +125,7 @@ def bench_draft_attn(n_pos, layers, iters):
     wt = synth.model_weights(shape, 0, device=dev, layers=[0])
     lw = engine.fuse_layer_weights(wt["layers"][0])
     gw = {"layers": [lw] * layers, "embed": wt["embed"], "lm_head": wt["lm_head"], "norm_final": wt["norm_final"]}
-    eng = engine.Engine(shape, gw, max_seq=(n_pos + 64 + 255) // 256 * 256, gamma_max=4)
+    eng = engine.Engine(shape, gw, fmt=B.default_format(kv_mode=kv_mode), max_seq=(n_pos + 64 + 255) // 256 * 256, gamma_max=4)
     n0 = min(n_pos, 512)
     kvs = []
     for l in range(layers):
@@ -151,7 +151,7 @@ def bench_draft_attn(n_pos, layers, iters):
     ms = _time(lambda: [B.cass_draft_attention(eng.session, l, q, out) for l in range(layers)], iters)
     peak, kind_ = _peak()
     gbs = bytes_layer * layers / (ms * 1e-3) / 1e9
-    res = [{"kernel": "draft_attn (+merge)", "positions": n_pos, "layers": layers, "us_per_layer": ms * 1e3 / layers,
+    res = [{"kernel": "draft_attn (+merge)", "kv_mode": kv_mode, "positions": n_pos, "layers": layers, "us_per_layer": ms * 1e3 / layers,
             "compressed_kv_bytes_per_layer": bytes_layer, "bf16_kv_bytes_per_layer": n_pos * 8 * 128 * 2 * 2,
             "algorithmic_GBps": gbs, "frac_of_hbm_peak": gbs / peak, "peak": f"{peak} GB/s ({kind_})"}]
     # KV encoder: one new token per layer, both caches
@@ -277,6 +277,8 @@ def main():
     ap.add_argument("--prompt", type=int, default=512)
     ap.add_argument("--config", default="llama8b")
     ap.add_argument("--mode", type=int, default=1, help="weight format: 1 = Cassandra-1 (unary), 2 = Cassandra-2 (MX)")
+    ap.add_argument("--layers", type=int, default=0, help="layers of the attention benchmark (0: enough to exceed L2)")
+    ap.add_argument("--kv-mode", type=int, default=1, help="KV cache format: 1 = Cassandra-1 records, 2 = Cassandra-2 (MX) records")
     ap.add_argument("--p", type=int, default=400)
     ap.add_argument("--t", type=int, default=4)
     args = ap.parse_args()
@@ -298,7 +300,7 @@ def main():
         out.extend(step_breakdown(gamma=args.gamma, batch=args.batch))
     if args.kernel in ("attn", "all"):
         for n_pos in ([args.positions] if args.positions else [4096, 32768]):
-            out.extend(bench_draft_attn(n_pos, max(2, int(3.0e5 / n_pos) + 1), args.iters))
+            out.extend(bench_draft_attn(n_pos, args.layers or max(2, int(3.0e5 / n_pos) + 1), args.iters, args.kv_mode))
     for r in out:
         print(json.dumps(r))
 

@@ -155,12 +155,13 @@ def _kv_engine(cass, n_q=32, max_seq=512):
     return engine.Engine(shape, gw, max_seq=max_seq, gamma_max=4)
 
 
-def test_kv_encoder_records_bit_exact_heads_of_128(cass):
+@pytest.mark.parametrize("max_seq", [512, 2304])           # the slice-parallel and the whole-record draft attention
+def test_kv_encoder_records_bit_exact_heads_of_128(cass, max_seq):
     """cass_kv_append with the head geometry every benchmark config uses (8 KV heads of 128, p = 40 %, t = 4; four
     elements per lane): three 32-token blocks of records against the oracle's encoder, bit for bit.  Among the appended
     tokens: one whose magnitudes are all equal (the tie rule: the lower channels are pruned), one whose exponents
     rank badly in the frozen codebook (so badly that the record stores them raw), one of zeros."""
-    eng = _kv_engine(cass)
+    eng = _kv_engine(cass, max_seq=max_seq)
     n0, n1, d, p, t = 40, 30, 128, 400, 4
     k, v = synth.kv_fill(n0 + n1, 8, d, 5, "k128/kv")
     g = torch.Generator().manual_seed(9)
