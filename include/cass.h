@@ -140,8 +140,8 @@ int cass_decode_weights(const void* blob, const cass_blob_info* h_info, void* W_
  * the low t mantissa bits of every kept value and the pruned values as they are.  Layout: 8 header words {'CASV', 1,
  * rows, cols, kept per row, t, words per row, 0}; per row ceil(kept*t/32) words of t-bit groups (column order, MSB
  * first), then the pruned values (column order) as 16-bit little-endian halfwords, padded to a word.  The bitmap is the
- * blob's.  cass_decode_full rebuilds the bf16 matrix from the two parts, bit for bit.  This library's verification
- * pass reads a bf16 copy instead; these calls exist to check the exactness of the split and to weigh its parts.
+ * blob's.  cass_decode_full rebuilds the bf16 matrix from the two parts, bit for bit (one pass, every value written
+ * once).  By default the verification pass reads a bf16 copy; cass_session_verify_from_parts makes it read the two parts.
  * Mode 1 blobs only (CASS_ERR_UNSUPPORTED otherwise).  h_bytes: host; vdata: device, 4-byte aligned. */
 int cass_verification_data_bytes(const cass_blob_info* h_info, size_t* h_bytes);
 int cass_encode_verification_data(const void* blob, const cass_blob_info* h_info, const void* W_bf16, void* vdata,
@@ -198,6 +198,22 @@ int cass_session_init(void* mem, size_t bytes, const cass_model_desc* desc, cons
                       void* stream);
 int cass_session_set_blobs(void* session, const cass_model_blobs* blobs, void* stream);   /* SYNCHRONISES */
 int cass_session_destroy(void* session);
+
+/* Verification from the two parts (Sec. 4.1 target inference: "both the speculation and verification data are loaded and
+ * fully reconstructed"; Sec. 7.2: no bf16 copy has to stay resident).  vdata: device pointers to the verification data
+ * (cass_encode_verification_data) of the matrices whose speculation data the session already has (Cassandra-1 blobs).
+ * From then on cass_verify rebuilds each matrix -- kept values with their low mantissa bits appended, pruned values as
+ * stored, bit for bit the original -- into `scratch_bf16` right before the projection that reads it, and never touches
+ * the bf16 matrices given at cass_session_init again (the caller may free them; embeddings and norm gains are still
+ * read).  Results are bit-identical to verification from the bf16 copy.  scratch_bf16: device, 16-byte aligned, at
+ * least cass_verify_from_parts_scratch_bytes (the largest matrix).  vdata = NULL switches back to the bf16 copy. */
+typedef struct cass_layer_vdata { const void *wqkv, *wo, *wgu, *wd; } cass_layer_vdata;
+typedef struct cass_model_vdata {
+    const cass_layer_vdata* h_layers;     /* HOST array [n_layers] */
+    const void* lm_head;
+} cass_model_vdata;
+size_t cass_verify_from_parts_scratch_bytes(const cass_model_desc* desc);
+int cass_session_verify_from_parts(void* session, const cass_model_vdata* vdata, void* scratch_bf16, size_t scratch_bytes);
 
 /* Forget all sequences: committed length 0, no draft in flight, KV codebooks cleared. */
 int cass_session_reset(void* session, void* stream);

@@ -59,6 +59,14 @@ class ModelBlobs(C.Structure):
     _fields_ = [("h_layers", C.POINTER(LayerBlobs)), ("lm_head", C.c_void_p)]
 
 
+class LayerVdata(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("wqkv", "wo", "wgu", "wd")]
+
+
+class ModelVdata(C.Structure):
+    _fields_ = [("h_layers", C.POINTER(LayerVdata)), ("lm_head", C.c_void_p)]
+
+
 class BlobInfo(C.Structure):
     _fields_ = [("rows", C.c_int), ("cols", C.c_int), ("prune_permille", C.c_int), ("trunc_bits", C.c_int),
                 ("seg_cols", C.c_int), ("chunk_cols", C.c_int), ("n_seg", C.c_int), ("n_rowblocks", C.c_int),
@@ -87,6 +95,7 @@ def _load() -> C.CDLL:
 lib = _load()
 lib.cass_version.restype = C.c_char_p
 lib.cass_verify_gemm_scratch_bytes.restype = C.c_size_t
+lib.cass_verify_from_parts_scratch_bytes.restype = C.c_size_t
 if hasattr(lib, "cass_calib_norms_count"):
     lib.cass_calib_norms_count.restype = C.c_size_t
 
@@ -191,6 +200,18 @@ def cass_session_init(mem, desc: ModelDesc, fmt: Format, weights: ModelWeights, 
 
 def cass_session_set_blobs(session, blobs: ModelBlobs, stream=None):
     _check("cass_session_set_blobs", lib.cass_session_set_blobs(session, C.byref(blobs), _stream(stream)))
+
+
+def cass_verify_from_parts_scratch_bytes(desc: ModelDesc) -> int:
+    return int(lib.cass_verify_from_parts_scratch_bytes(C.byref(desc)))
+
+
+def cass_session_verify_from_parts(session, vdata, scratch_bf16):
+    if vdata is None:
+        _check("cass_session_verify_from_parts", lib.cass_session_verify_from_parts(session, None, None, C.c_size_t(0)))
+        return
+    _check("cass_session_verify_from_parts", lib.cass_session_verify_from_parts(
+        session, C.byref(vdata), _ptr(scratch_bf16), C.c_size_t(scratch_bf16.numel() * scratch_bf16.element_size())))
 
 
 def cass_session_destroy(session):

@@ -11,6 +11,7 @@ namespace cass {
 
 struct LayerDev {
     cass_layer_weights w;
+    const void* vdata[4];    // verification data of wqkv, wo, wgu, wd (only when verifying from the two parts)
     const void* blob[4];
     cass_blob_info bi[4];
     uint16_t *kc, *vc;       // bf16 caches [max_seq][n_kv][d]
@@ -45,6 +46,9 @@ struct Session {
     bool have_blobs, codebooks_ready, calib_host;
     int qkv_dim, kmax;
     int drafts_pending;      // cass_draft_step calls since the last accept / set_len / reset (host-side count)
+    bool from_parts;         // verification rebuilds each matrix from speculation + verification data into vscratch
+    const void* lm_vdata;
+    uint16_t* vscratch;
 };
 
 struct Plan {
@@ -448,6 +452,15 @@ extern "C" int cass_verify(void* session, const int32_t* toks, int g, int32_t* t
     // decode calls (rps <= gamma_max + 1) all use the column count the session's gamma_max needs; longer prefill chunks 64
     const int np_cols = (rps <= d.gamma_max + 1 && (d.gamma_max + 1) * grp <= 32) ? 32 : 64;
     const int qd = d.n_q_heads * d.head_dim;
+    // The matrix a projection multiplies with: the caller's bf16 copy, or -- Sec. 4.1 target inference -- the exact
+    // reconstruction from speculation + verification data, rebuilt into the session's scratch right before its use.
+    int w_rc = CASS_OK;
+    auto weight = [&](const void* bf16, const void* blob, const cass_blob_info& bi, const void* vd) -> const uint16_t* {
+        if (!s->from_parts) return (const uint16_t*)bf16;
+        const int rc = cass_decode_full(blob, &bi, vd, s->vscratch, stream_);
+        if (rc) w_rc = rc;
+        return s->vscratch;
+    };
     RC(launch_embed(toks, 1, (const uint16_t*)s->embed, s->h, rows, d.hidden, st));
     RC(launch_rmsnorm(s->h, (const uint16_t*)s->layers[0].w.norm_attn, s->xn, rows, d.hidden, d.rms_eps, st));
     const int kv_flags = CASS_KV_BF16 | (s->codebooks_ready ? CASS_KV_COMPRESSED : 0);
@@ -457,7 +470,7 @@ extern "C" int cass_verify(void* session, const int32_t* toks, int g, int32_t* t
     for (int l = 0; l < d.n_layers; ++l) {
         LayerDev& L = s->layers[l];
         if (calib) RC(launch_calib_accum(s->xn, rows, d.hidden, L.calib[0], s->st, st));
-        RC(launch_verify_gemm((const uint16_t*)L.w.wqkv, s->xn, rows, bn, s->qkv_dim, d.hidden, s->vg_partial, nullptr, nullptr, status, st));
+        RC(launch_verify_gemm(weight(L.w.wqkv, L.blob[0], L.bi[0], L.vdata[0]), s->xn, rows, bn, s->qkv_dim, d.hidden, s->vg_partial, nullptr, nullptr, status, st));
         if (fused) {
             RC(launch_rope_kv_append(s->kg, L.ck, L.cv, L.kc, L.vc, vparts(s->qkv_dim, d.hidden), s->cos_t, s->sin_t, s->qkv,
                                      d.n_q_heads, 0, rps, kv_flags, s->st, B, st));
@@ -470,23 +483,23 @@ extern "C" int cass_verify(void* session, const int32_t* toks, int g, int32_t* t
         if (attn_tc) RC(launch_verify_attn_tc(s->kg, L.kc, L.vc, s->qkv, B, rps, d.n_q_heads, np_cols, s->st, s->asc, s->attn, status, st));
         else RC(launch_verify_attn(s->kg, L.kc, L.vc, s->qkv, B, rps, d.n_q_heads, s->st, s->asc, s->attn, st));
         if (calib) RC(launch_calib_accum(s->attn, rows, qd, L.calib[1], s->st, st));
-        RC(launch_verify_gemm((const uint16_t*)L.w.wo, s->attn, rows, bn, d.hidden, qd, s->vg_partial, nullptr, nullptr, status, st));
+        RC(launch_verify_gemm(weight(L.w.wo, L.blob[1], L.bi[1], L.vdata[1]), s->attn, rows, bn, d.hidden, qd, s->vg_partial, nullptr, nullptr, status, st));
         RC(launch_residual_rmsnorm(s->h, nullptr, vparts(d.hidden, qd), (const uint16_t*)L.w.norm_ffn, s->xn,
                                    rows, d.hidden, d.rms_eps, st));
         if (calib) RC(launch_calib_accum(s->xn, rows, d.hidden, L.calib[2], s->st, st));
-        RC(launch_verify_gemm((const uint16_t*)L.w.wgu, s->xn, rows, bn, 2 * d.ffn, d.hidden, s->vg_partial, nullptr, nullptr, status, st));
+        RC(launch_verify_gemm(weight(L.w.wgu, L.blob[2], L.bi[2], L.vdata[2]), s->xn, rows, bn, 2 * d.ffn, d.hidden, s->vg_partial, nullptr, nullptr, status, st));
         RC(launch_swiglu(nullptr, vparts(2 * d.ffn, d.hidden), s->act, rows, d.ffn, st));
         if (calib) RC(launch_calib_accum(s->act, rows, d.ffn, L.calib[3], s->st, st));
-        RC(launch_verify_gemm((const uint16_t*)L.w.wd, s->act, rows, bn, d.hidden, d.ffn, s->vg_partial, nullptr, nullptr, status, st));
+        RC(launch_verify_gemm(weight(L.w.wd, L.blob[3], L.bi[3], L.vdata[3]), s->act, rows, bn, d.hidden, d.ffn, s->vg_partial, nullptr, nullptr, status, st));
         const uint16_t* next_gain = (const uint16_t*)(l + 1 < d.n_layers ? s->layers[l + 1].w.norm_attn : s->norm_final);
         RC(launch_residual_rmsnorm(s->h, nullptr, vparts(d.hidden, d.ffn), next_gain, s->xn, rows, d.hidden,
                                    d.rms_eps, st));
     }
     if (calib) RC(launch_calib_accum(s->xn, rows, d.hidden, s->calib_lm, s->st, st));
-    RC(launch_verify_gemm((const uint16_t*)s->lm_head, s->xn, rows, bn, d.vocab, d.hidden, s->vg_partial, nullptr, nullptr, status, st));
+    RC(launch_verify_gemm(weight(s->lm_head, s->lm_blob, s->lm_bi, s->lm_vdata), s->xn, rows, bn, d.vocab, d.hidden, s->vg_partial, nullptr, nullptr, status, st));
     RC(launch_argmax(nullptr, vparts(d.vocab, d.hidden), rows, d.vocab, target_argmax, 1, logits_opt,
                      s->argmax_val, s->argmax_tmp, s->st, 0, st));
-    return CASS_OK;
+    return w_rc;
 }
 
 extern "C" int cass_draft_step(void* session, const int32_t* tok_in, int32_t* tok_out, int tok_stride, float* logits_opt,
@@ -560,4 +573,37 @@ extern "C" int cass_accept_sampling(void* session, int n_seq, const int32_t* dra
     }
     return launch_accept_sampling(st, n_seq, draft, draft_stride, p_target, q_draft, vocab, r_uniform, u_uniform, g, n_accepted,
                                   out_tokens, next_tok, next_stride, (cudaStream_t)stream_);
+}
+
+extern "C" size_t cass_verify_from_parts_scratch_bytes(const cass_model_desc* d) {
+    if (!d) return 0;
+    const size_t qkv = (size_t)(d->n_q_heads + 2 * d->n_kv_heads) * d->head_dim;
+    size_t m = qkv * d->hidden;
+    const size_t c[4] = {(size_t)d->hidden * d->n_q_heads * d->head_dim, (size_t)2 * d->ffn * d->hidden, (size_t)d->hidden * d->ffn,
+                         (size_t)d->vocab * d->hidden};
+    for (size_t v : c) if (v > m) m = v;
+    return m * 2;
+}
+
+extern "C" int cass_session_verify_from_parts(void* session, const cass_model_vdata* vdata, void* scratch_bf16, size_t scratch_bytes) {
+    if (!session) return CASS_ERR_INVALID_ARG;
+    Session* s = (Session*)session;
+    if (!vdata) { s->from_parts = false; return CASS_OK; }                 // back to the caller's bf16 matrices
+    if (!vdata->h_layers || !vdata->lm_head || !scratch_bf16 || ((uintptr_t)scratch_bf16 & 15)) return CASS_ERR_INVALID_ARG;
+    if (!s->have_blobs) return CASS_ERR_INVALID_ARG;                       // the speculation data comes first
+    if (scratch_bytes < cass_verify_from_parts_scratch_bytes(&s->d)) return CASS_ERR_CAPACITY;
+    if (s->lm_bi.mode != 1) return CASS_ERR_UNSUPPORTED;                   // Cassandra-2 speculation data has no exact complement here
+    for (int l = 0; l < s->d.n_layers; ++l) {
+        const cass_layer_vdata& v = vdata->h_layers[l];
+        const void* p[4] = {v.wqkv, v.wo, v.wgu, v.wd};
+        for (int i = 0; i < 4; ++i) {
+            if (!p[i]) return CASS_ERR_INVALID_ARG;
+            if (s->layers[l].bi[i].mode != 1) return CASS_ERR_UNSUPPORTED;
+            s->layers[l].vdata[i] = p[i];
+        }
+    }
+    s->lm_vdata = vdata->lm_head;
+    s->vscratch = (uint16_t*)scratch_bf16;
+    s->from_parts = true;
+    return CASS_OK;
 }

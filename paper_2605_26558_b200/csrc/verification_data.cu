@@ -1,7 +1,7 @@
 // Verification data (Sec. 4.1 target inference, Sec. 5.1 encoder): what the Cassandra-1 speculation data leaves out
 // -- the low t mantissa bits of the kept values and the pruned values as they are -- and the exact reconstruction
-// of the bf16 matrix from the two parts.  Not on the decode path of this library (verification reads a bf16 copy);
-// it shows that the format is a strict split of the original bits and what the two parts weigh.
+// of the bf16 matrix from the two parts (k_decode_full).  A session told to verify from the two parts
+// (cass_session_verify_from_parts) rebuilds every matrix with it right before the verification GEMM reads it.
 //
 // Layout: header of 8 words {magic 'CASV', 1, rows, cols, kept per row, t, words per row, 0}; per row
 // ceil(kept*t/32) words of t-bit groups (kept values in column order, MSB first), then the pruned values in column
@@ -75,6 +75,66 @@ __global__ void __launch_bounds__(256) k_vdata(const uint32_t* __restrict__ blob
     }
 }
 
+// Exact reconstruction in one pass (Sec. 4.1 target inference: speculation and verification data are loaded and the
+// original values rebuilt; Sec. 5.1 mantissa concatenator).  One CTA per superblock, warp = chunk, lane = row: the lane
+// walks its chunk's kept values in column order (the blob's streams are interleaved over the 32 rows, so the warp's
+// reads are contiguous), appends each value's low t bits from the row's verification data, and fills the columns
+// between kept values with the raw pruned values.  Chunk c owns the columns from its first kept value up to the next
+// chunk's first kept value (chunk 0 also the columns before its first value).
+__global__ void __launch_bounds__(1024) k_decode_full(const uint32_t* __restrict__ blob, const uint32_t* __restrict__ vdata,
+                                                      uint16_t* __restrict__ out) {
+    const uint32_t* h = blob;
+    const int n = h[H_ROWS], k = h[H_COLS], t = h[H_T], seg_cols = h[H_SEG], n_seg = h[H_NSEG], kept = h[H_KEPT];
+    const int k_pad = ceil_div(k, 32) * 32;
+    const int sb = blockIdx.x, rb = sb / n_seg, seg = sb % n_seg;
+    const uint32_t* dir = blob + kBlobDirOffset / 4 + sb * 4;
+    const int scols = seg_cols_of(k_pad, seg_cols, seg);
+    const SbGeom sg = SbGeom::make(dir_n_ch(dir[3]), scols, (int)dir[1], (int)dir[2]);
+    const int chunk_elems = dir_chunk_elems(dir[3]);
+    const uint32_t* body = blob + (size_t)dir[0] * 4;
+    const uint8_t* cb = reinterpret_cast<const uint8_t*>(blob) + kBlobHeaderBytes;
+    const int lo_words = vdata_lo_words(kept, t), row_words = vdata_row_words(k, kept, t);
+    const int ch = threadIdx.x >> 5, r = threadIdx.x & 31, row = rb * kRowsPerBlock + r;
+    if (ch >= sg.n_ch || row >= n) return;
+    // kept values of this row in the segments before this one (their chunk tables end with the segment's kept count)
+    uint32_t kept_before = 0;
+    for (int s2 = 0; s2 < seg; ++s2) {
+        const uint32_t* d2 = blob + kBlobDirOffset / 4 + (rb * n_seg + s2) * 4;
+        const SbGeom g2 = SbGeom::make(dir_n_ch(d2[3]), seg_cols_of(k_pad, seg_cols, s2), (int)d2[1], (int)d2[2]);
+        kept_before += blob[(size_t)d2[0] * 4 + g2.tab + g2.n_ch * 32 + r] >> 20;
+    }
+    const uint32_t* lo = vdata + kVdataHeaderWords + (size_t)row * row_words;
+    const uint16_t* raw = reinterpret_cast<const uint16_t*>(lo + lo_words);
+    uint16_t* orow = out + (size_t)row * k;
+    const int c_base = seg * seg_cols;
+    const int kept_seg = (int)(body[sg.tab + sg.n_ch * 32 + r] >> 20);
+    const int k0 = ch * chunk_elems;                                    // this chunk's first kept value (index inside the segment)
+    if (k0 >= kept_seg && ch > 0) return;                               // no values: an earlier chunk owns the rest of the row
+    const int col_first = k0 < kept_seg ? (int)(body[sg.tab + ch * 32 + r] >> 20) : scols;
+    const int col_end = (ch + 1 < sg.n_ch && (ch + 1) * chunk_elems < kept_seg) ? (int)(body[sg.tab + (ch + 1) * 32 + r] >> 20) : scols;
+    int next_col = ch == 0 ? 0 : col_first;                             // first column not yet written
+    uint32_t kk = kept_before + (uint32_t)k0;                           // row-wide index of the next kept value
+    auto fill_pruned = [&](int from, int to) {                          // columns [from, to) of the segment are pruned
+        for (int c = from; c < to; ++c) {
+            const int cc = c_base + c;
+            if (cc < k) orow[cc] = raw[(uint32_t)cc - kk];              // pruned columns before cc = cc - kept values before cc
+        }
+    };
+    auto emit = [&](int col, uint16_t bits) {
+        fill_pruned(next_col, col);
+        if (t > 0) {
+            const uint32_t bit0 = kk * (uint32_t)t, sh = bit0 & 31u, wi = bit0 >> 5;
+            const uint64_t two = ((uint64_t)lo[wi] << 32) | (sh + t > 32 ? lo[wi + 1] : 0u);
+            bits |= (uint16_t)((two >> (64 - t - sh)) & ((1u << t) - 1u));
+        }
+        if (c_base + col < k) orow[c_base + col] = bits;
+        ++kk;
+        next_col = col + 1;
+    };
+    if (k0 < kept_seg) decode_chunk_generic(body, sg, chunk_elems, ch, r, t, cb, emit);
+    fill_pruned(next_col, col_end);
+}
+
 }  // namespace cass
 
 using namespace cass;
@@ -102,10 +162,10 @@ extern "C" int cass_encode_verification_data(const void* blob, const cass_blob_i
 extern "C" int cass_decode_full(const void* blob, const cass_blob_info* bi, const void* vdata, void* W_bf16_out, void* stream_) {
     if (!blob || !bi || !vdata || !W_bf16_out) return CASS_ERR_INVALID_ARG;
     if (bi->mode != 1) return CASS_ERR_UNSUPPORTED;
-    int rc = cass_decode_weights(blob, bi, W_bf16_out, stream_);           // kept values without their low bits, zeros elsewhere
-    if (rc) return rc;
-    k_vdata<false><<<ceil_div(bi->rows, 8), 256, 0, (cudaStream_t)stream_>>>((const uint32_t*)blob, nullptr,
-                                                                             (uint32_t*)const_cast<void*>(vdata), (uint16_t*)W_bf16_out);
+    const int n_ch = ceil_div(bi->seg_cols, bi->chunk_cols);
+    if (n_ch > 32) return CASS_ERR_UNSUPPORTED;
+    k_decode_full<<<bi->n_rowblocks * bi->n_seg, 32 * n_ch, 0, (cudaStream_t)stream_>>>((const uint32_t*)blob, (const uint32_t*)vdata,
+                                                                                         (uint16_t*)W_bf16_out);
     CASS_LAUNCH_CHECK();
     return CASS_OK;
 }

@@ -155,6 +155,40 @@ class Engine:
         self._mb = B.ModelBlobs(self._lb, blobs["lm_head"].data_ptr())
         B.cass_session_set_blobs(self.session, self._mb)
 
+    def verify_from_parts(self, drop_bf16: bool = False) -> int:
+        """Encodes the verification data of every matrix and makes the session verify from speculation + verification
+        data instead of the bf16 copy (needs encode_weights first).  With drop_bf16 the engine lets go of the bf16
+        projection matrices (embeddings and norm gains stay).  Returns the bytes of verification data."""
+        assert self.blobs is not None
+        self.vdata = {"layers": []}
+        total = 0
+
+        def enc(blob, info, w):
+            nonlocal total
+            buf = torch.empty(B.cass_verification_data_bytes(info), dtype=torch.uint8, device=self.device)
+            B.cass_encode_verification_data(blob, info, w, buf)
+            total += buf.numel()
+            return buf
+
+        for l, lw in enumerate(self.w["layers"]):
+            self.vdata["layers"].append({nm: enc(self.blobs["layers"][l][nm], self.blobs["infos"][(l, nm)], lw[nm])
+                                         for nm in ("wqkv", "wo", "wgu", "wd")})
+        self.vdata["lm_head"] = enc(self.blobs["lm_head"], self.blobs["infos"]["lm_head"], self.w["lm_head"])
+        self._lv = (B.LayerVdata * self.shape.n_layers)()
+        for i, d in enumerate(self.vdata["layers"]):
+            for nm in ("wqkv", "wo", "wgu", "wd"):
+                setattr(self._lv[i], nm, d[nm].data_ptr())
+        self._mv = B.ModelVdata(self._lv, self.vdata["lm_head"].data_ptr())
+        self.vscratch = torch.empty(B.cass_verify_from_parts_scratch_bytes(self.desc), dtype=torch.uint8, device=self.device)
+        torch.cuda.synchronize(self.device)
+        B.cass_session_verify_from_parts(self.session, self._mv, self.vscratch)
+        if drop_bf16:
+            for lw in self.w["layers"]:
+                for nm in ("wqkv", "wo", "wgu", "wd"):
+                    lw[nm] = None
+            self.w["lm_head"] = None
+        return total
+
     def blob_bytes(self) -> int:
         return sum(sum(t.numel() for t in d.values()) for d in self.blobs["layers"]) + self.blobs["lm_head"].numel()
 
