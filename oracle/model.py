@@ -297,6 +297,14 @@ def sampling_accept(p: np.ndarray, q: np.ndarray, draft_tokens, r: np.ndarray, u
     return n, [int(t) for t in draft_tokens[:n]] + [extra]
 
 
+def design_objective(alpha: float, s_w: float, w_p: float, w_t: int, s_kv: float, kv_p: float, kv_t: int, bits: int = 16) -> float:
+    """Objective of the format search (Sec. 7.2, Eq. 2): acceptance rate per bit the draft model has to move,
+    J = alpha / (S_w (1 - w_p)(B - w_t) + S_kv (1 - kv_p)(B - kv_t)); sizes in values, pruning ratios as fractions,
+    B the target model's bits per value."""
+    moved = s_w * (1.0 - w_p) * (bits - w_t) + s_kv * (1.0 - kv_p) * (bits - kv_t)
+    return alpha / moved
+
+
 def plain_greedy(W: Weights, kv: KVCache, first_tok: int, n_tokens: int, kv_p: int, kv_t: int, kv_mode: int = 1):
     """Autoregressive decoding with the target only.  `first_tok` is the token predicted from the
     prompt; returns the n_tokens tokens that follow it."""

@@ -46,6 +46,15 @@ __device__ __forceinline__ uint32_t mad_lo(uint32_t a, uint32_t b, uint32_t c) {
     return r;
 }
 
+// Sign and kept mantissa bits of a field at their binary32 positions, for truncations whose fields do not tile a
+// word (8 - t = 7, 6, 5, 3): the field is packed from the most significant end, floor(32 / (8 - t)) per word.
+template <int T>
+__device__ __forceinline__ uint32_t packed_field_f32(uint32_t word, uint32_t j) {
+    constexpr int F = 8 - T;
+    const uint32_t f = (word >> (32u - (uint32_t)F * (j + 1u))) & ((1u << F) - 1u);
+    return ((f >> (F - 1)) << 31) | ((f & ((1u << (F - 1)) - 1u)) << (16 + T));
+}
+
 template <int NB>
 struct WalkState {
     float acc[NB];
@@ -81,8 +90,9 @@ __device__ __forceinline__ void x_fma(const XRaw<NB>& r, uint32_t wb, float (&ac
 
 // Careful walk of `count` (<= 8) kept values of one row from column bpos / code bit upos on: any gap between
 // kept columns, any codeword length.  Used for the rare groups that do not fit the 32-bit windows.
+// flC: the segment's first field word of this row; k0: index (inside the segment) of the group's first value.
 template <int T, int NB>
-__device__ __noinline__ WalkState<NB> group_slow(const uint32_t* bmS, const uint32_t* unS, const uint32_t* flG, int count,
+__device__ __noinline__ WalkState<NB> group_slow(const uint32_t* bmS, const uint32_t* unS, const uint32_t* flC, uint32_t k0, int count,
                                                  WalkState<NB> st, uint32_t bpos_lim, uint32_t upos_lim, const float* xs,
                                                  const uint32_t* lut) {
     constexpr int F = 8 - T, PER = 32 / F;
@@ -98,9 +108,12 @@ __device__ __noinline__ WalkState<NB> group_slow(const uint32_t* bmS, const uint
         const XRaw<NB> xv = x_load<NB>(smem_u32(xs) + st.bpos * (uint32_t)x_col_bytes(NB));
         st.bpos += 1;
         const int rank = read_unary(unS, st.upos, upos_lim);
-        const uint32_t fword = flG[(e / PER) * 32];
-        const uint32_t a = __funnelshift_l(fword, fword, (F * (e % PER)) & 31);
-        x_fma<NB>(xv, (a & MASK) | lut[rank & 255], st.acc);
+        const uint32_t k = k0 + (uint32_t)e;
+        const uint32_t fword = flC[(k / PER) * 32];
+        uint32_t a;
+        if constexpr (32 % F == 0) a = __funnelshift_l(fword, fword, (F * (k % PER)) & 31) & MASK;
+        else a = packed_field_f32<T>(fword, k % PER);
+        x_fma<NB>(xv, a | lut[rank & 255], st.acc);
     }
     return st;
 }
@@ -126,18 +139,21 @@ template <int T, int NB>
 __device__ __forceinline__ void chunk_dot_fast(const uint32_t* __restrict__ sb, const SbGeom& g, int ch, int lane,
                                                int chunk_elems, const float* __restrict__ xs,
                                                const uint32_t* __restrict__ lut, float (&acc)[NB]) {
-    constexpr int F = 8 - T, PER = 32 / F, NFW = kGroupCols / PER;       // field words per group of 8
+    constexpr int F = 8 - T, PER = 32 / F;
+    constexpr bool ROT = 32 % F == 0;                                    // fields tile a word: float-aligned and rotated
+    constexpr int NFW = ROT ? kGroupCols / PER : 3;                      // field words a group of 8 can touch
     constexpr uint32_t MASK = 0x80000000u | (((1u << (7 - T)) - 1u) << (16 + T));   // sign + kept mantissa of a binary32
-    static_assert(32 % F == 0 && (PER == 4 || PER == 8), "fast path: rotated fields, 4 or 8 per word");
+    static_assert(ROT ? (PER == 4 || PER == 8) : (PER >= 4 && PER <= 10), "fast path: 4 to 10 fields per word");
     constexpr uint32_t XS = (uint32_t)x_col_bytes(NB);            // bytes per column of the x slice
     const uint32_t e0 = sb[g.tab + ch * 32 + lane];            // where this row's value ch * chunk_elems sits
-    const uint32_t fw = (uint32_t)(ch * chunk_elems) / PER;    // its field word (chunk_elems is a multiple of 8)
+    const uint32_t fw = (uint32_t)(ch * chunk_elems) / PER;    // the word of the chunk's first field (fields are numbered through the segment)
     uint32_t upos = e0 & 0xFFFFFu;
     const uint32_t* bmS = sb + g.bm + lane;
     const uint32_t* flS = sb + g.fl + lane;
     const uint32_t* unS = sb + g.un + lane;
     const uint32_t bm_a = smem_u32(bmS), un_a = smem_u32(unS), xs_a = smem_u32(xs), lut_a = smem_u32(lut);
     uint32_t fl_a = smem_u32(flS + fw * 32);
+    uint32_t j0 = (uint32_t)(ch * chunk_elems) % PER;           // packed fields: place of the group's first field in its word
     // every row has chunk_elems values in each chunk except its last ones, so the lanes of a warp stay in step
     const int kept = (int)(sb[g.tab + g.n_ch * 32 + lane] >> 20);
     const int m = max(0, min(chunk_elems, kept - ch * chunk_elems));
@@ -161,7 +177,8 @@ __device__ __forceinline__ void chunk_dot_fast(const uint32_t* __restrict__ sb, 
         const uint32_t xg = xs_a + bpos * XS + 31u * XS;                           // address of x[bpos + 31]
         uint32_t fwd[NFW];
         fwd[0] = lds_u32(fl_a);
-        if (NFW > 1) fwd[NFW - 1] = lds_u32_off<128>(fl_a);
+        if (NFW > 1) fwd[1] = lds_u32_off<128>(fl_a);
+        if (NFW > 2) fwd[2] = lds_u32_off<256>(fl_a);
         const int rem = m - grp * kGroupCols;
         uint32_t dry = 0;                           // sign bit set: a window ran dry under a value that counts
         uint32_t p = 0;
@@ -181,9 +198,17 @@ __device__ __forceinline__ void chunk_dot_fast(const uint32_t* __restrict__ sb, 
                 const uint32_t eb = lds_u32(mad_lo(q, 0xFFFFFFFCu, la));          // lut[previous - q - 1]
                 la = mad_lo(q, 4u, lut_a - 4u);
                 uv &= ~shl_sat(1u, q);
-                const uint32_t fword = fwd[e / PER];
-                const uint32_t a = __funnelshift_l(fword, fword, (F * (e % PER)) & 31);
-                const uint32_t wb = (a & MASK) | eb;
+                uint32_t wb;
+                if constexpr (ROT) {
+                    const uint32_t fword = fwd[e / PER];
+                    const uint32_t a = __funnelshift_l(fword, fword, (F * (e % PER)) & 31);
+                    wb = (a & MASK) | eb;
+                } else {
+                    const uint32_t jj = j0 + (uint32_t)e;                 // field jj of the group's (up to three) words
+                    const uint32_t wsel = jj >= 2u * PER ? 2u : (jj >= (uint32_t)PER ? 1u : 0u);
+                    const uint32_t fword = wsel == 2u ? fwd[NFW - 1] : (wsel == 1u ? fwd[1] : fwd[0]);
+                    wb = packed_field_f32<T>(fword, jj - wsel * PER) | eb;
+                }
                 if (!tail) {
                     x_fma<NB>(xv, wb, acc);
                 } else if (e < rem) {
@@ -199,13 +224,20 @@ __device__ __forceinline__ void chunk_dot_fast(const uint32_t* __restrict__ sb, 
         if (tail) bpos = min(bpos, bpos_lim);
         else dry |= p;
         if ((int32_t)dry < 0) {
-            const WalkState<NB> r = group_slow<T, NB>(bmS, unS, flS + (fw + grp * NFW) * 32, min(rem, kGroupCols), st0, bpos_lim,
-                                                      upos_lim, xs, lut);
+            const WalkState<NB> r = group_slow<T, NB>(bmS, unS, flS, (uint32_t)(ch * chunk_elems + grp * kGroupCols), min(rem, kGroupCols),
+                                                      st0, bpos_lim, upos_lim, xs, lut);
 #pragma unroll
             for (int b = 0; b < NB; ++b) acc[b] = r.acc[b];
             bpos = r.bpos; upos = r.upos;
         }
-        fl_a += NFW * 128u;
+        if constexpr (ROT) {
+            fl_a += NFW * 128u;
+        } else {
+            const uint32_t jn = j0 + (uint32_t)kGroupCols;
+            const uint32_t adv = jn >= 2u * PER ? 2u : (jn >= (uint32_t)PER ? 1u : 0u);
+            fl_a += adv * 128u;
+            j0 = jn - adv * PER;
+        }
     };
 
     int grp = 0;
@@ -460,7 +492,7 @@ __global__ void __launch_bounds__(1024) k_draft_gemv(const uint32_t* __restrict_
                     x_fma<NB>(x_load<NB>(xs_a + (uint32_t)col * (uint32_t)x_col_bytes(NB)), (uint32_t)bits << 16, acc);
                 });
             } else if (T >= 0) {
-                chunk_dot_fast<(T >= 0 && T < 8 ? T : 0), NB>(sb, g, warp, lane, dir_chunk_elems(dir[3]), xs, lut, acc);
+                chunk_dot_fast<(T >= 0 && T <= 5 ? T : 0), NB>(sb, g, warp, lane, dir_chunk_elems(dir[3]), xs, lut, acc);
             } else {
                 const uint32_t xs_a = smem_u32(xs);
                 decode_chunk_generic(sb, g, dir_chunk_elems(dir[3]), warp, lane, t, cb, [&](int col, uint16_t bits) {
@@ -574,6 +606,10 @@ int launch_draft_gemv(const void* blob, const cass_blob_info& bi, const void* x_
     else if (bi.mode == 2) CASS_GEMV_LAUNCH_NB(-2);
     else if (bi.trunc_bits == 4) CASS_GEMV_LAUNCH_NB(4);
     else if (bi.trunc_bits == 0) CASS_GEMV_LAUNCH_NB(0);
+    else if (bi.trunc_bits == 1) CASS_GEMV_LAUNCH_NB(1);          // fields that do not tile a word: the design-space sweep of Sec. 7.2
+    else if (bi.trunc_bits == 2) CASS_GEMV_LAUNCH_NB(2);
+    else if (bi.trunc_bits == 3) CASS_GEMV_LAUNCH_NB(3);
+    else if (bi.trunc_bits == 5) CASS_GEMV_LAUNCH_NB(5);
     else CASS_GEMV_LAUNCH_NB(-1);
 #undef CASS_GEMV_LAUNCH_NB
 #undef CASS_GEMV_LAUNCH

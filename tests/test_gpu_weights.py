@@ -42,7 +42,11 @@ CASES = [
     (96, 1024, 400, 4, 0, 0),
     (64, 256, 400, 4, 0, 0),
     (33, 704, 0, 0, 0, 0),                # identity format
-    (40, 512, 300, 5, 256, 64),           # a truncation the fast path does not cover
+    (40, 512, 300, 5, 256, 64),           # 3-bit fields: ten per word, packed (not rotated)
+    (96, 2048, 400, 1, 0, 0),             # 7-bit fields: four per word, chunks that start inside a field word
+    (70, 1376, 500, 2, 1024, 128),        # 6-bit fields: five per word
+    (64, 4096, 300, 3, 0, 0),             # 5-bit fields: six per word, two full segments
+    (32, 4096, 600, 5, 2048, 64),         # 3-bit fields, 60 % pruned: long gaps between kept columns
     (128, 4096, 400, 4, 0, 0),            # Llama-3-8B hidden size: two full segments
     (64, 4096, 500, 0, 1024, 256),
 ]

@@ -332,3 +332,24 @@ def test_sampling_accept_longer_drafts_and_special_cases():
     assert [model.inverse_cdf_sample(w, u) for u in (0.0, 0.49, 0.5, 0.74, 0.75, 0.999)] == [1, 1, 3, 3, 4, 4]
     assert np.allclose(model.softmax(np.log(w[[1, 3, 4]]), 1.0), [0.5, 0.25, 0.25])
     assert np.allclose(model.softmax(np.log(w[[1, 3, 4]]), 0.5), np.array([4.0, 1.0, 1.0]) / 6.0)
+
+
+def test_design_objective_of_eq_2():
+    """Hand-worked: alpha = 0.6, S_w = 1000 values at 40 % / 4 bits -> 1000 * 0.6 * 12 = 7200 bits; S_kv = 100 values at
+    50 % / 2 bits -> 100 * 0.5 * 14 = 700 bits; J = 0.6 / 7900.  The search script's bookkeeping uses the same formula."""
+    assert abs(model.design_objective(0.6, 1000, 0.4, 4, 100, 0.5, 2) - 0.6 / 7900.0) < 1e-18
+    assert model.design_objective(0.5, 10, 0.0, 0, 0, 0.0, 0) == 0.5 / 160.0          # nothing removed: 16 bits per value
+    # more pruning or more truncation at equal acceptance raises J; lower acceptance lowers it
+    base = model.design_objective(0.5, 1e6, 0.4, 4, 1e4, 0.4, 4)
+    assert model.design_objective(0.5, 1e6, 0.5, 4, 1e4, 0.4, 4) > base < model.design_objective(0.5, 1e6, 0.4, 5, 1e4, 0.4, 4)
+    assert model.design_objective(0.4, 1e6, 0.4, 4, 1e4, 0.4, 4) < base
+    import importlib.util, os
+    path = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "paper_2605_26558_b200", "sweep.py")
+    src = open(path).read()
+    ns = {}
+    exec(src[src.index("def objective("):src.index("def _shape(")], {"TARGET_BITS": 16}, ns)   # the formula alone, no library import
+    rng = np.random.default_rng(0)
+    for _ in range(50):
+        a, sw, skv = rng.uniform(0, 1), rng.uniform(1e3, 1e9), rng.uniform(1e3, 1e9)
+        wp, kp, wt, kt = rng.uniform(0, 0.9), rng.uniform(0, 0.9), int(rng.integers(0, 8)), int(rng.integers(0, 8))
+        assert np.isclose(ns["objective"](a, sw, wp, wt, skv, kp, kt), model.design_objective(a, sw, wp, wt, skv, kp, kt), rtol=1e-14)
