@@ -2,7 +2,7 @@
 """Benchmark of the Cassandra self-speculative decode step on B200.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl cass|reference] [--gamma G]
-                    [--config llama8b|qwen|tiny] [--batch 1|2|4|8] [--mode 1|2] [--prompt P]
+                    [--config llama8b|qwen|tiny] [--batch 1|2|4|8] [--mode 1|2] [--kv-mode 1|2] [--from-parts] [--prompt P]
 
 A step is one pass of the whole hot path over one batch-1 sequence: gamma draft tokens (draft GEMVs and draft
 attention on the speculation data, the KV encoder appending each drafted token), one bf16 verification pass over
@@ -170,9 +170,11 @@ def run_reference(args):
 # CUDA path
 # ----------------------------------------------------------------------------------------------------------
 
-def launches_per_step(n_layers: int, gamma: int) -> int:
-    draft = 2 + n_layers * 10 + 3            # embed, norm | per layer: 4 gemv, rope+kv, attn, merge, 2 norm, swiglu | lm gemv, 2 argmax
-    verify = 2 + n_layers * 10 + 3           # per layer: 4 gemm, rope+kv, attn, merge, 2 norm, swiglu | lm gemm, 2 argmax
+def launches_per_step(n_layers: int, gamma: int, max_seq: int = 0, kv_mode: int = 1, from_parts: bool = False) -> int:
+    # draft, per layer: 4 gemv, rope+kv, attention (its last CTA merges; long Cassandra-1 caches add a merge kernel), 2 norm, swiglu
+    draft = 2 + n_layers * (9 + (1 if kv_mode == 1 and max_seq > 2048 else 0)) + 3     # + embed, norm | lm gemv, 2 argmax
+    # verify, per layer: 4 gemm (each preceded by a reconstruction kernel when verifying from the two parts), rope+kv, attn, merge, 2 norm, swiglu
+    verify = 2 + n_layers * (10 + (4 if from_parts else 0)) + 3 + (1 if from_parts else 0)
     return gamma * draft + verify + 1
 
 
@@ -217,12 +219,18 @@ def run_cass(args):
     max_seq = n_prompt + (max(args.steps, args.warmup) + 2) * per_step + 64
     max_seq = (max_seq + 255) // 256 * 256
     nb = args.batch
-    eng = engine.Engine(shape, gw, fmt=cass.default_format(mode=args.mode), max_seq=max_seq, gamma_max=max(gamma, 1),
-                        device=dev, batch=nb)
+    eng = engine.Engine(shape, gw, fmt=cass.default_format(mode=args.mode, kv_mode=args.kv_mode), max_seq=max_seq,
+                        gamma_max=max(gamma, 1), device=dev, batch=nb)
     prompt = torch.stack([synth.random_prompt(n_prompt, shape.vocab, seed=rank * 8 + b) for b in range(nb)])
     eng.prefill(prompt, calibrate=True)
-    eng.encode_weights(eng.calib_norms())
+    norms = eng.calib_norms()
+    eng.encode_weights(norms)
     eng.build_kv_codebook()
+    bf16_matrix_bytes = sum(lw[nm].numel() * 2 for lw in gw["layers"] for nm in ("wqkv", "wo", "wgu", "wd")) + gw["lm_head"].numel() * 2
+    vdata_bytes = 0
+    if args.from_parts:
+        # Sec. 4.1 / 7.2: verification rebuilds every matrix from speculation + verification data; no bf16 matrix stays resident
+        vdata_bytes = eng.verify_from_parts(drop_bf16=(args.context_points == 0))
     torch.cuda.synchronize()
     first_tok = eng.next_tokens()
     setup_s = time.perf_counter() - t_setup
@@ -345,6 +353,48 @@ def run_cass(args):
     # ---- gather over ranks ----
     ms, ms_e2e, emitted_all, e2e_all = combine_replicas(ms, ms_e2e, emitted, e2e_emitted, world, dev)
 
+    # ---- context points (not the headline): the identity format, whose draft equals the target (every draft accepted:
+    # the upper bound of tokens per step), and the KV cache truncated but not pruned (the Sec. 6.1 reading of the default) ----
+    context = {}
+    if world == 1 and args.context_points > 0 and args.mode == 1 and args.kv_mode == 1:
+        def spec_rate(e, n_steps):
+            e.step(gamma); torch.cuda.synchronize()
+            cass.cass_set_len(e.session, n_prompt); e.set_next_tokens(first_tok)
+            g2 = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g2):
+                e.step(gamma)
+            for _ in range(3):
+                g2.replay()
+            cass.cass_set_len(e.session, n_prompt); e.set_next_tokens(first_tok)
+            acc = torch.zeros(1, dtype=torch.int64, device=dev)
+            torch.cuda.synchronize()
+            c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            c0.record()
+            for _ in range(n_steps):
+                g2.replay()
+                acc.add_((e.n_acc[:nb].to(torch.int64) + 1).sum())
+            c1.record()
+            torch.cuda.synchronize()
+            t_ms = c0.elapsed_time(c1)
+            return {"tokens_per_s": int(acc.item()) / (t_ms * 1e-3), "ms_per_step": t_ms / n_steps,
+                    "mean_accepted_len": int(acc.item()) / (n_steps * nb) - 1.0, "status": e.status()[0]}
+
+        n_ctx = min(args.steps, args.context_points)
+        blobs_default = eng.blobs
+        for name, fmt_kw in (("kv_truncated_not_pruned", dict(kv_p=0, kv_t=4)), ("identity_format", dict(w_p=0, w_t=0, kv_p=0, kv_t=0))):
+            e2 = engine.Engine(shape, gw, fmt=cass.default_format(**fmt_kw), max_seq=max_seq, gamma_max=max(gamma, 1), device=dev, batch=nb)
+            e2.prefill(prompt)
+            if name == "identity_format":
+                e2.encode_weights(None)
+            else:
+                e2.set_blobs(blobs_default)               # the same speculation data of the weights
+            e2.build_kv_codebook()
+            context[name] = spec_rate(e2, n_ctx)
+            context[name]["format"] = fmt_kw
+            e2.close()
+            del e2
+            torch.cuda.empty_cache()
+
     if rank == 0:
         cpu = None
         if world == 1 and not args.no_cpu_baseline:
@@ -360,8 +410,12 @@ def run_cass(args):
                                    + f", batch {nb}, prompt {n_prompt}, positions {n_prompt}..{n_prompt + args.steps * per_step}",
                        "batch": nb,
                        "gamma": gamma,
-                       "format": "cassandra-1 p=40% t=4 (weights and KV)" if args.mode == 1 else
-                                 "cassandra-2 (MX, blocks of 32) p=40% t=4 weights, cassandra-1 KV",
+                       "format": ("cassandra-1 p=40% t=4 weights" if args.mode == 1 else "cassandra-2 (MX, blocks of 32 kept values) p=40% t=4 weights")
+                                 + (", cassandra-1 KV p=40% t=4" if args.kv_mode == 1 else ", cassandra-2 KV (MX per 32 channels) p=40% t=4"),
+                       "verification": "from speculation + verification data (no bf16 matrices resident)" if args.from_parts else "bf16 copy",
+                       "resident_weight_bits_per_value": (eng.blob_bytes() + vdata_bytes) * 8.0 / (bf16_matrix_bytes / 2) if args.from_parts
+                                                         else (eng.blob_bytes() + bf16_matrix_bytes) * 8.0 / (bf16_matrix_bytes / 2),
+                       "context_points": context,
                        "l2": "inputs larger than L2 (16 GB bf16 weights + speculation data per step)",
                        "parallelism": "replicas only" if world > 1 else "1 gpu",
                        "mean_accepted_len": emitted_all / (args.steps * world * nb) - 1.0,
@@ -372,7 +426,7 @@ def run_cass(args):
             "clocks": clocks,
             "e2e": {"value": e2e_all / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": 4 * nb,
                     "d2h_bytes_per_step": 4 * nb * (gamma + 2)},
-            "gpu_launches": launches_per_step(shape.n_layers, gamma) * args.steps,
+            "gpu_launches": launches_per_step(shape.n_layers, gamma, max_seq, args.kv_mode, args.from_parts) * args.steps,
             "roofline": {"kernel": "k_draft_gemv", "bound": "hbm", "achieved": achieved, "peak": hbm_peak,
                          "unit": "GB/s", "frac": achieved / hbm_peak, "peak_kind": f"of {peak_kind}",
                          "traffic": int(DRAM_BYTES_PER_BLOB_BYTE * blob_bits / 8 / len(jobs)),
@@ -400,6 +454,12 @@ def main():
     ap.add_argument("--config", default="llama8b", choices=["llama8b", "tiny", "qwen"])
     ap.add_argument("--mode", type=int, default=1, choices=[1, 2],
                     help="weight format of the draft: 1 = Cassandra-1 (unary exponents), 2 = Cassandra-2 (MX exponents)")
+    ap.add_argument("--kv-mode", type=int, default=1, choices=[1, 2],
+                    help="KV cache format of the draft: 1 = Cassandra-1 records, 2 = Cassandra-2 (MX) records")
+    ap.add_argument("--from-parts", action="store_true",
+                    help="verify from speculation + verification data instead of the bf16 copy (Sec. 4.1, 7.2)")
+    ap.add_argument("--context-points", type=int, default=30,
+                    help="steps of each context run (identity format; KV not pruned) reported in config; 0 = skip them")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.warmup < 3:

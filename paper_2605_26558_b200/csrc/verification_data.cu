@@ -75,64 +75,100 @@ __global__ void __launch_bounds__(256) k_vdata(const uint32_t* __restrict__ blob
     }
 }
 
-// Exact reconstruction in one pass (Sec. 4.1 target inference: speculation and verification data are loaded and the
-// original values rebuilt; Sec. 5.1 mantissa concatenator).  One CTA per superblock, warp = chunk, lane = row: the lane
-// walks its chunk's kept values in column order (the blob's streams are interleaved over the 32 rows, so the warp's
-// reads are contiguous), appends each value's low t bits from the row's verification data, and fills the columns
-// between kept values with the raw pruned values.  Chunk c owns the columns from its first kept value up to the next
-// chunk's first kept value (chunk 0 also the columns before its first value).
-__global__ void __launch_bounds__(1024) k_decode_full(const uint32_t* __restrict__ blob, const uint32_t* __restrict__ vdata,
-                                                      uint16_t* __restrict__ out) {
+// Exact reconstruction (Sec. 4.1 target inference: speculation and verification data are loaded and the original values
+// rebuilt; Sec. 5.1 mantissa concatenator), in two light kernels that keep many warps per SM in flight:
+//   k_decode_kept<T>: one CTA per superblock, warp = chunk, lane = row.  The lane walks its chunk's kept values (the
+//     blob's streams are interleaved over the 32 rows, so the warp's reads are contiguous) and stores their speculation
+//     bits (sign, exponent, high mantissa bits) at their columns of the output.
+//   k_merge_vdata: one warp per row, lane = column.  For every 32 columns the kept values get their low t bits from the
+//     row's verification data and the pruned columns their raw values; kept and pruned counts before a column are
+//     popcounts of the bitmap (prefix sums over the row's bitmap words first, so that the words are then independent
+//     and their loads overlap), neighbouring lanes read neighbouring verification data and the row leaves as
+//     contiguous stores.
+template <int TT>                                                       // truncated bits (0..5), or -1: read from the header
+__global__ void __launch_bounds__(1024) k_decode_kept(const uint32_t* __restrict__ blob, uint16_t* __restrict__ out) {
+    __shared__ uint16_t lut_s[256];                                     // rank -> exponent at its bf16 position
     const uint32_t* h = blob;
-    const int n = h[H_ROWS], k = h[H_COLS], t = h[H_T], seg_cols = h[H_SEG], n_seg = h[H_NSEG], kept = h[H_KEPT];
+    const int n = h[H_ROWS], k = h[H_COLS], t = TT >= 0 ? TT : (int)h[H_T], seg_cols = h[H_SEG], n_seg = h[H_NSEG];
     const int k_pad = ceil_div(k, 32) * 32;
     const int sb = blockIdx.x, rb = sb / n_seg, seg = sb % n_seg;
     const uint32_t* dir = blob + kBlobDirOffset / 4 + sb * 4;
-    const int scols = seg_cols_of(k_pad, seg_cols, seg);
-    const SbGeom sg = SbGeom::make(dir_n_ch(dir[3]), scols, (int)dir[1], (int)dir[2]);
+    const SbGeom sg = SbGeom::make(dir_n_ch(dir[3]), seg_cols_of(k_pad, seg_cols, seg), (int)dir[1], (int)dir[2]);
     const int chunk_elems = dir_chunk_elems(dir[3]);
     const uint32_t* body = blob + (size_t)dir[0] * 4;
     const uint8_t* cb = reinterpret_cast<const uint8_t*>(blob) + kBlobHeaderBytes;
-    const int lo_words = vdata_lo_words(kept, t), row_words = vdata_row_words(k, kept, t);
+    if ((int)h[H_T] != t) return;                                       // not the blob the launch was told about
+    for (int i = threadIdx.x; i < 256; i += blockDim.x) lut_s[i] = (uint16_t)cb[i] << 7;
+    __syncthreads();
     const int ch = threadIdx.x >> 5, r = threadIdx.x & 31, row = rb * kRowsPerBlock + r;
     if (ch >= sg.n_ch || row >= n) return;
-    // kept values of this row in the segments before this one (their chunk tables end with the segment's kept count)
-    uint32_t kept_before = 0;
-    for (int s2 = 0; s2 < seg; ++s2) {
-        const uint32_t* d2 = blob + kBlobDirOffset / 4 + (rb * n_seg + s2) * 4;
-        const SbGeom g2 = SbGeom::make(dir_n_ch(d2[3]), seg_cols_of(k_pad, seg_cols, s2), (int)d2[1], (int)d2[2]);
-        kept_before += blob[(size_t)d2[0] * 4 + g2.tab + g2.n_ch * 32 + r] >> 20;
-    }
+    uint16_t* orow = out + (size_t)row * k + seg * seg_cols;
+    const int cols_here = k - seg * seg_cols;
+    auto put = [&](int col, uint16_t bits) { if (col < cols_here) orow[col] = bits; };
+    if constexpr (TT >= 0) decode_chunk_fixed<(TT >= 0 ? TT : 0)>(body, sg, chunk_elems, ch, r, lut_s, put);
+    else decode_chunk_generic(body, sg, chunk_elems, ch, r, t, cb, put);
+}
+
+constexpr int kMergeRowWarps = 8;
+__global__ void __launch_bounds__(32 * kMergeRowWarps) k_merge_vdata(const uint32_t* __restrict__ blob, const uint32_t* __restrict__ vdata,
+                                                                     uint16_t* __restrict__ out) {
+    __shared__ uint32_t kb_s[kMergeRowWarps][64];                       // kept values before each 32-column word of the segment in hand
+    const uint32_t* h = blob;
+    const int n = h[H_ROWS], k = h[H_COLS], t = h[H_T], seg_cols = h[H_SEG], n_seg = h[H_NSEG], kept = h[H_KEPT];
+    const int k_pad = ceil_div(k, 32) * 32;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int row = blockIdx.x * kMergeRowWarps + warp;
+    if (row >= n) return;
+    const int rb = row / kRowsPerBlock, rr = row % kRowsPerBlock;
+    const int lo_words = vdata_lo_words(kept, t), row_words = vdata_row_words(k, kept, t);
     const uint32_t* lo = vdata + kVdataHeaderWords + (size_t)row * row_words;
     const uint16_t* raw = reinterpret_cast<const uint16_t*>(lo + lo_words);
-    uint16_t* orow = out + (size_t)row * k;
-    const int c_base = seg * seg_cols;
-    const int kept_seg = (int)(body[sg.tab + sg.n_ch * 32 + r] >> 20);
-    const int k0 = ch * chunk_elems;                                    // this chunk's first kept value (index inside the segment)
-    if (k0 >= kept_seg && ch > 0) return;                               // no values: an earlier chunk owns the rest of the row
-    const int col_first = k0 < kept_seg ? (int)(body[sg.tab + ch * 32 + r] >> 20) : scols;
-    const int col_end = (ch + 1 < sg.n_ch && (ch + 1) * chunk_elems < kept_seg) ? (int)(body[sg.tab + (ch + 1) * 32 + r] >> 20) : scols;
-    int next_col = ch == 0 ? 0 : col_first;                             // first column not yet written
-    uint32_t kk = kept_before + (uint32_t)k0;                           // row-wide index of the next kept value
-    auto fill_pruned = [&](int from, int to) {                          // columns [from, to) of the segment are pruned
-        for (int c = from; c < to; ++c) {
-            const int cc = c_base + c;
-            if (cc < k) orow[cc] = raw[(uint32_t)cc - kk];              // pruned columns before cc = cc - kept values before cc
+    uint32_t k_base = 0;                                                // kept values of the row in the segments already done
+    for (int seg = 0; seg < n_seg; ++seg) {
+        const uint32_t* dir = blob + kBlobDirOffset / 4 + (rb * n_seg + seg) * 4;
+        const int scols = seg_cols_of(k_pad, seg_cols, seg), n_words = scols / 32;       // <= 64 words
+        const SbGeom sg = SbGeom::make(dir_n_ch(dir[3]), scols, (int)dir[1], (int)dir[2]);
+        const uint32_t* bmw = blob + (size_t)dir[0] * 4 + sg.bm + rr;  // bitmap word j of this row at bmw[j * 32]
+        const int c_base = seg * seg_cols;
+        uint16_t* orow = out + (size_t)row * k + c_base;
+        __syncwarp();
+        uint32_t c0 = 0, c1 = 0;
+        if (lane < n_words) c0 = __popc(bmw[lane * 32]);
+        if (lane + 32 < n_words) c1 = __popc(bmw[(lane + 32) * 32]);
+        uint32_t i0 = c0, i1 = c1;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t a = __shfl_up_sync(0xffffffffu, i0, o), b2 = __shfl_up_sync(0xffffffffu, i1, o);
+            if (lane >= o) { i0 += a; i1 += b2; }
         }
-    };
-    auto emit = [&](int col, uint16_t bits) {
-        fill_pruned(next_col, col);
-        if (t > 0) {
-            const uint32_t bit0 = kk * (uint32_t)t, sh = bit0 & 31u, wi = bit0 >> 5;
-            const uint64_t two = ((uint64_t)lo[wi] << 32) | (sh + t > 32 ? lo[wi + 1] : 0u);
-            bits |= (uint16_t)((two >> (64 - t - sh)) & ((1u << t) - 1u));
+        const uint32_t tot0 = __shfl_sync(0xffffffffu, i0, 31), tot1 = __shfl_sync(0xffffffffu, i1, 31);
+        kb_s[warp][lane] = k_base + i0 - c0;
+        kb_s[warp][lane + 32] = k_base + tot0 + i1 - c1;
+        __syncwarp();
+#pragma unroll 4
+        for (int j = 0; j < n_words; ++j) {
+            const uint32_t bm = bmw[j * 32];
+            const int c = j * 32 + lane;
+            const uint32_t kb = kb_s[warp][j];
+            const bool in = c_base + c < k, is_kept = (bm >> (31 - lane)) & 1u;
+            const uint32_t before = lane ? __popc(bm >> (32 - lane)) : 0u;          // kept columns of this word before mine
+            if (in) {
+                uint16_t v;
+                if (is_kept) {
+                    v = orow[c];                                                    // the speculation bits k_decode_kept left here
+                    if (t > 0) {
+                        const uint32_t bit0 = (kb + before) * (uint32_t)t, sh = bit0 & 31u, wi = bit0 >> 5;
+                        const uint64_t two = ((uint64_t)lo[wi] << 32) | (sh + t > 32 ? lo[wi + 1] : 0u);
+                        v |= (uint16_t)((two >> (64 - t - sh)) & ((1u << t) - 1u));
+                    }
+                } else {
+                    v = raw[(uint32_t)(c_base + c) - kb - before];                   // pruned columns before mine = columns - kept before
+                }
+                orow[c] = v;
+            }
         }
-        if (c_base + col < k) orow[c_base + col] = bits;
-        ++kk;
-        next_col = col + 1;
-    };
-    if (k0 < kept_seg) decode_chunk_generic(body, sg, chunk_elems, ch, r, t, cb, emit);
-    fill_pruned(next_col, col_end);
+        k_base += tot0 + tot1;
+    }
 }
 
 }  // namespace cass
@@ -164,8 +200,22 @@ extern "C" int cass_decode_full(const void* blob, const cass_blob_info* bi, cons
     if (bi->mode != 1) return CASS_ERR_UNSUPPORTED;
     const int n_ch = ceil_div(bi->seg_cols, bi->chunk_cols);
     if (n_ch > 32) return CASS_ERR_UNSUPPORTED;
-    k_decode_full<<<bi->n_rowblocks * bi->n_seg, 32 * n_ch, 0, (cudaStream_t)stream_>>>((const uint32_t*)blob, (const uint32_t*)vdata,
-                                                                                         (uint16_t*)W_bf16_out);
+    const int threads = 32 * n_ch;
+    const int grid = bi->n_rowblocks * bi->n_seg;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    const uint32_t* b32 = (const uint32_t*)blob;
+    uint16_t* o16 = (uint16_t*)W_bf16_out;
+    switch (bi->trunc_bits) {
+        case 0: k_decode_kept<0><<<grid, threads, 0, stream>>>(b32, o16); break;
+        case 1: k_decode_kept<1><<<grid, threads, 0, stream>>>(b32, o16); break;
+        case 2: k_decode_kept<2><<<grid, threads, 0, stream>>>(b32, o16); break;
+        case 3: k_decode_kept<3><<<grid, threads, 0, stream>>>(b32, o16); break;
+        case 4: k_decode_kept<4><<<grid, threads, 0, stream>>>(b32, o16); break;
+        case 5: k_decode_kept<5><<<grid, threads, 0, stream>>>(b32, o16); break;
+        default: k_decode_kept<-1><<<grid, threads, 0, stream>>>(b32, o16); break;
+    }
+    CASS_LAUNCH_CHECK();
+    k_merge_vdata<<<ceil_div(bi->rows, kMergeRowWarps), 32 * kMergeRowWarps, 0, stream>>>(b32, (const uint32_t*)vdata, o16);
     CASS_LAUNCH_CHECK();
     return CASS_OK;
 }

@@ -134,6 +134,47 @@ __device__ inline void decode_chunk_generic(const uint32_t* sb, const SbGeom& g,
     }
 }
 
+// The same with the truncation known at compile time (no run-time divisions in the field arithmetic): what a kernel
+// that decodes whole matrices uses.  `lut`: rank -> exponent << 7 (bf16 position), 256 entries.
+template <int T, class Emit>
+__device__ __forceinline__ void decode_chunk_fixed(const uint32_t* sb, const SbGeom& g, int chunk_elems, int ch, int row,
+                                                   const uint16_t* lut, Emit&& emit) {
+    constexpr int F = 8 - T, PER = 32 / F;
+    constexpr uint32_t KEEP = 0x8000u | (0x7Fu & ~((1u << T) - 1u));    // sign + kept mantissa bits of a bf16
+    const uint32_t e0 = sb[g.tab + ch * 32 + row];
+    const int kept = (int)(sb[g.tab + g.n_ch * 32 + row] >> 20);
+    const int k0 = ch * chunk_elems;
+    const int cnt = min(chunk_elems, kept - k0);
+    if (cnt <= 0) return;
+    uint32_t col = e0 >> 20, ub = e0 & 0xFFFFFu;
+    const uint32_t* bm_row = sb + g.bm + row;
+    const uint32_t* fl_row = sb + g.fl + row;
+    const uint32_t* un_row = sb + g.un + row;
+    const uint32_t limit = (uint32_t)g.w_u * 32u, col_lim = (uint32_t)g.bm_words * 32u;
+    uint32_t bw = col < col_lim ? bm_row[(col >> 5) * 32] << (col & 31) : 0u;      // bitmap bits from `col` on, left-aligned
+    for (uint32_t k = (uint32_t)k0; k < (uint32_t)(k0 + cnt); ++k) {
+        while (!bw) {                                                              // nothing kept up to the word's end: next bitmap word
+            col = (col + 31u) & ~31u;                                              // the next word boundary (col itself when on one)
+            if (col >= col_lim) return;                                            // corrupt stream: stop inside the buffers
+            bw = bm_row[(col >> 5) * 32];
+            if (!bw) col += 1u;                                                    // an empty word: the next round moves past it
+        }
+        const uint32_t z = __clz(bw);
+        col += z;
+        const int rank = read_unary(un_row, ub, limit);
+        const uint32_t fword = fl_row[(k / PER) * 32], j = k % PER;
+        uint32_t sm;
+        if constexpr (32 % F == 0) sm = (__funnelshift_l(fword, fword, (F * j) & 31) >> 16) & KEEP;
+        else {
+            const uint32_t f = (fword >> (32u - (uint32_t)F * (j + 1u))) & ((1u << F) - 1u);
+            sm = ((f >> (F - 1)) << 15) | ((f & ((1u << (F - 1)) - 1u)) << T);
+        }
+        emit((int)col, (uint16_t)(sm | lut[rank & 255]));
+        col += 1;
+        bw = z >= 31u ? 0u : (bw << (z + 1u));                                     // bit 31 is column `col` again; 0 once the word is used up
+    }
+}
+
 // The same for a Cassandra-2 blob (shared exponent per block of 32 kept values instead of a codeword per value).
 template <class Emit>
 __device__ inline void decode_chunk_generic_mx(const uint32_t* sb, const SbGeom& g, int chunk_elems, int ch, int row,
