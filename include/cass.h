@@ -17,6 +17,11 @@
  *     returns CASS_ERR_CUDA (there is no fallback path).
  *   - Device-side problems (capacity exceeded, bounded wait ran out) are recorded in the session's
  *     status word, readable with cass_session_status().
+ *   - Two environment variables, read once per process, are debugging aids:
+ *     CASS_NO_PDL=1 launches every kernel in plain stream order (no programmatic dependent launch), so that
+ *     a trace shows per-kernel times without overlap; CASS_SIMT_VERIFY_ATTN=1 makes cass_verify keep its
+ *     fp32-pipe attention kernel where the tensor-core one would run (results then differ by the bf16
+ *     rounding of the attention probabilities that the tensor-core kernel applies).
  */
 #ifndef CASS_H_
 #define CASS_H_

@@ -19,6 +19,16 @@ Pins (tests that tie the oracle to the paper / to mathematics, not to itself):
   * greedy speculative stream == plain greedy stream for any draft  (Sec. 2.2)
   * greedy acceptance == Eq. 1 with p/q in {0, 1}
   * draft GEMV / attention on decoded operands == library matmul / softmax
+  * attention == the library's scaled-dot-product attention, a brute-force
+    double loop, and its one-key / equal-keys special cases          (Sec. 2.1)
+  * RMSNorm on a hand-computed vector; SwiGLU against its closed form
+  * a whole decoder layer == an independent restatement with library ops
+  * sampling acceptance: emitted token distributed as the target's
+    (chi-square), acceptance probability sum(min(p, q)), Eq. 1 by brute
+    force, one-hot distributions reduce to the greedy rule           (Eq. 1)
+  * KV records: entry words, raw-exponent escape, per-slice decode
+    round trips; Cassandra-2 KV values against the MX definition     (Sec. 4.1-4.3)
+  * design objective on hand-computed points                         (Eq. 2)
 
 Parity unpinned (this build's own readings, fixed only by agreement between the
 oracle and the CUDA path): the physical superblock layout, the per-row pruning

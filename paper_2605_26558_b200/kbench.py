@@ -196,9 +196,18 @@ def step_breakdown(gamma=4, n_prompt=512, steps=3, batch=1):
             eng.step(gamma)
         torch.cuda.synchronize()
     agg = collections.defaultdict(lambda: [0, 0.0])
-    for ev in prof.events():
-        if ev.device_type is not None and "cuda" in str(ev.device_type).lower() and ev.name.find("Memcpy") < 0 and ev.name.find("Memset") < 0:
+    evs = [ev for ev in prof.events() if ev.device_type is not None and "cuda" in str(ev.device_type).lower()
+           and ev.name.find("Memcpy") < 0 and ev.name.find("Memset") < 0]
+    evs.sort(key=lambda ev: ev.time_range.start)
+    per_pass = 4 * shape.n_layers + 1              # draft projections of one pass, in launch order: (wqkv, wo, wgu, wd) per layer, lm_head
+    n_gemv = 0
+    for ev in evs:
+        if True:
             name = re.sub(r"<.*|\(.*", "", ev.name).replace("void ", "").replace("cass::", "")
+            if name == "k_draft_gemv":
+                c = n_gemv % per_pass
+                name += "[" + ("lm_head" if c == per_pass - 1 else ("wqkv", "wo", "wgu", "wd")[c % 4]) + "]"
+                n_gemv += 1
             agg[name][0] += 1
             agg[name][1] += ev.device_time_total if hasattr(ev, "device_time_total") else ev.cuda_time_total
     tot = sum(v[1] for v in agg.values())
