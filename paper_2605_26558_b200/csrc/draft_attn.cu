@@ -466,6 +466,7 @@ __global__ void __launch_bounds__(kMergeThreads) k_attn_merge(AttnScratch sc, in
     const int seq = r / rps;
     const int vis = st->len[seq] + (draft_mode ? st->inflight[seq] + 1 : r % rps + 1);
     if (draft_units > 0) chunk_tokens = da_tokens_per_cta(vis, draft_units);  // runs whose length follows the visible length
+    if (draft_units < 0) chunk_tokens = tc_run_tokens(vis, -draft_units);     // the same for the dense-tile kernel
     const int n_ch = ceil_div(vis, chunk_tokens);
     const size_t pair = (size_t)r * n_q + hq;
     const float* mp = sc.m + pair * n_chunks_alloc;
@@ -546,9 +547,16 @@ int launch_draft_attn_rec(const KvGeom& g, const KvComp& ck, const KvComp& cv, c
 // which needs about half the instructions per value; the slice-parallel kernel is the faster one while the grid is small.
 constexpr int kDaSliceMaxSeq = 2048;
 
+bool draft_attn_tc_supported(const KvGeom& g, int n_q);
+int launch_draft_attn_tc(const KvGeom& g, const KvComp& ck, const KvComp& cv, const uint16_t* qkv, int qkv_stride, int n_q,
+                         int n_seq, const DevState* st, const AttnScratch& sc, uint16_t* out, cudaStream_t s);
+
 int launch_draft_attn(const KvGeom& g, const KvComp& ck, const KvComp& cv, const uint16_t* qkv, int qkv_stride, int n_q,
                       int n_seq, const DevState* st, const AttnScratch& sc, uint16_t* out, cudaStream_t s) {
-    if (g.mode == 1 && g.max_seq > kDaSliceMaxSeq) return launch_draft_attn_rec(g, ck, cv, qkv, qkv_stride, n_q, n_seq, st, sc, out, s);
+    if (g.mode == 1 && g.max_seq > kDaSliceMaxSeq) {
+        if (draft_attn_tc_supported(g, n_q)) return launch_draft_attn_tc(g, ck, cv, qkv, qkv_stride, n_q, n_seq, st, sc, out, s);
+        return launch_draft_attn_rec(g, ck, cv, qkv, qkv_stride, n_q, n_seq, st, sc, out, s);
+    }
     const int G = n_q / g.n_kv;
     if (G > kMaxGroup || g.d > 256 || g.d % 32) return CASS_ERR_UNSUPPORTED;
     const int gq = G <= 4 ? 4 : 8;

@@ -62,6 +62,13 @@ __host__ __device__ inline int da_tokens_per_cta(int visible, int heads_x_seqs) 
     while (t < 256 && ceil_div(visible, t) * heads_x_seqs > 592) t *= 2;
     return t;
 }
+// Positions one CTA of the dense-tile draft attention (long caches) handles: one 64-token chunk, doubled while the grid
+// would exceed about four CTAs per SM.  The kernel and its merge compute it from the same visible length.
+__host__ __device__ inline int tc_run_tokens(int visible, int heads_x_seqs) {
+    int t = 64;
+    while (t < 2048 && ceil_div(visible, t) * heads_x_seqs > 592) t *= 2;
+    return t;
+}
 __host__ __device__ __forceinline__ KvComp of_seq(const KvComp& c, int b, size_t seq_stride) {
     KvComp r;
     r.fixed = of_seq(c.fixed, b, seq_stride); r.arena = of_seq(c.arena, b, seq_stride); r.off = of_seq(c.off, b, seq_stride);
