@@ -540,22 +540,17 @@ size_t draft_attn_smem_bytes(const KvGeom& g, int gq) {
            (size_t)kDaSub * (g.d + 2) * 2 + 64;
 }
 
-int launch_draft_attn_rec(const KvGeom& g, const KvComp& ck, const KvComp& cv, const uint16_t* qkv, int qkv_stride, int n_q,
-                          int n_seq, const DevState* st, const AttnScratch& sc, uint16_t* out, cudaStream_t s);
-
-// Sessions with long caches (more than kDaSliceMaxSeq positions) and Cassandra-1 records use the whole-record kernel,
-// which needs about half the instructions per value; the slice-parallel kernel is the faster one while the grid is small.
-constexpr int kDaSliceMaxSeq = 2048;
-
+// Cassandra-1 records go to the dense-tile kernel (draft_attn_tc.cu: whole record per lane, products on mma.sync) where
+// its shape limits hold; Cassandra-2 records, and the shapes it leaves out, take the slice-parallel kernel below.
 bool draft_attn_tc_supported(const KvGeom& g, int n_q);
 int launch_draft_attn_tc(const KvGeom& g, const KvComp& ck, const KvComp& cv, const uint16_t* qkv, int qkv_stride, int n_q,
                          int n_seq, const DevState* st, const AttnScratch& sc, uint16_t* out, cudaStream_t s);
 
 int launch_draft_attn(const KvGeom& g, const KvComp& ck, const KvComp& cv, const uint16_t* qkv, int qkv_stride, int n_q,
                       int n_seq, const DevState* st, const AttnScratch& sc, uint16_t* out, cudaStream_t s) {
-    if (g.mode == 1 && g.max_seq > kDaSliceMaxSeq) {
-        if (draft_attn_tc_supported(g, n_q)) return launch_draft_attn_tc(g, ck, cv, qkv, qkv_stride, n_q, n_seq, st, sc, out, s);
-        return launch_draft_attn_rec(g, ck, cv, qkv, qkv_stride, n_q, n_seq, st, sc, out, s);
+    if (draft_attn_tc_supported(g, n_q)) {
+        const int rc = launch_draft_attn_tc(g, ck, cv, qkv, qkv_stride, n_q, n_seq, st, sc, out, s);
+        if (rc != CASS_ERR_UNSUPPORTED) return rc;
     }
     const int G = n_q / g.n_kv;
     if (G > kMaxGroup || g.d > 256 || g.d % 32) return CASS_ERR_UNSUPPORTED;

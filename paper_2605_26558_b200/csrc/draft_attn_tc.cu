@@ -435,12 +435,15 @@ int launch_draft_attn_tc(const KvGeom& g, const KvComp& ck, const KvComp& cv, co
             CASS_CUDA_CHECK(cudaFuncSetAttribute((k_draft_attn_tc<TT>), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
             attr = smem;                                                                                             \
         }                                                                                                            \
-        CASS_PDL_LAUNCH((k_draft_attn_tc<TT>), grid, dim3(kTcThreads), smem, s, g, ck, cv, qkv, qkv_stride, n_q, st, sc, n_chunks);     \
+        CASS_PDL_LAUNCH((k_draft_attn_tc<TT>), grid, dim3(kTcThreads), smem, s, g, ck, cv, qkv, qkv_stride, n_q, st, sc, n_chunks);      \
     } while (0)
     if (g.t == 4) CASS_TC_LAUNCH(4);
     else CASS_TC_LAUNCH(0);
 #undef CASS_TC_LAUNCH
     CASS_LAUNCH_CHECK();
+    // the runs of every (sequence, query head) are merged by a kernel of their own: one CTA per head with the runs spread
+    // over its warps (a merge by the last CTA of a KV head, as the slice-parallel kernel does it, is one CTA adding up to
+    // 74 runs for the whole group in sequence: measured 32.6 instead of 16.7 us at 4096 positions)
     return launch_attn_merge(sc, n_chunks, kTcTok, n_seq, 1, n_q, g.d, st, 1, -g.n_kv * n_seq, out, s);
 }
 

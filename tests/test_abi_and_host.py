@@ -88,10 +88,10 @@ def test_replica_reduction_world_size_2():
 def test_launch_count_formula():
     sys.path.insert(0, ROOT)
     import bench
-    # draft attention merges in its last CTA: 9 launches per draft layer, 10 per verification layer
-    assert bench.launches_per_step(32, 4) == 4 * (2 + 32 * 9 + 3) + (2 + 32 * 10 + 3) + 1
-    # long Cassandra-1 caches use the whole-record kernel with a merge launch of its own
-    assert bench.launches_per_step(32, 4, max_seq=4096) == 4 * (2 + 32 * 10 + 3) + (2 + 32 * 10 + 3) + 1
-    assert bench.launches_per_step(32, 4, max_seq=4096, kv_mode=2) == bench.launches_per_step(32, 4)
+    # 10 launches per draft layer (4 projections, RoPE + KV append, attention, merge, 2 norms, SwiGLU) and per verification layer
+    assert bench.launches_per_step(32, 4) == 4 * (2 + 32 * 10 + 3) + (2 + 32 * 10 + 3) + 1
+    # the count does not depend on the cache length; a Cassandra-2 cache merges inside the attention kernel
+    assert bench.launches_per_step(32, 4, max_seq=4096) == bench.launches_per_step(32, 4)
+    assert bench.launches_per_step(32, 4, kv_mode=2) == bench.launches_per_step(32, 4) - 4 * 32
     # verification from the two parts: two reconstruction launches per matrix
     assert bench.launches_per_step(2, 1, from_parts=True) - bench.launches_per_step(2, 1) == 2 * (2 * 4 + 1)

@@ -155,7 +155,7 @@ def _kv_engine(cass, n_q=32, max_seq=512):
     return engine.Engine(shape, gw, max_seq=max_seq, gamma_max=4)
 
 
-@pytest.mark.parametrize("max_seq", [512, 2304])           # the slice-parallel and the whole-record draft attention
+@pytest.mark.parametrize("max_seq", [512, 2304])           # a cache of one run per head and a longer one
 def test_kv_encoder_records_bit_exact_heads_of_128(cass, max_seq):
     """cass_kv_append with the head geometry every benchmark config uses (8 KV heads of 128, p = 40 %, t = 4; four
     elements per lane): three 32-token blocks of records against the oracle's encoder, bit for bit.  Among the appended
