@@ -85,6 +85,58 @@ struct Partials {
     size_t seg_stride, row_stride;
 };
 
+// Sum of the parts at element offset `off` (row and feature already applied), added in part order.  The loads of up to
+// eight parts are issued before the first addition, so that a sum costs one round trip to L2 instead of one per part.
+constexpr int kPartBatch = 8;
+__device__ __forceinline__ float parts_sum(const Partials& pp, size_t off) {
+    float acc = 0.f;
+    const float* p = pp.p + off;
+    for (int s0 = 0; s0 < pp.n_seg; s0 += kPartBatch) {
+        float v[kPartBatch];
+#pragma unroll
+        for (int i = 0; i < kPartBatch; ++i) v[i] = s0 + i < pp.n_seg ? __ldcg(p + (size_t)(s0 + i) * pp.seg_stride) : 0.f;
+#pragma unroll
+        for (int i = 0; i < kPartBatch; ++i)
+            if (s0 + i < pp.n_seg) acc += v[i];
+    }
+    return acc;
+}
+// Four consecutive elements (16-byte loads; `off` a multiple of 4 elements, strides too), four parts per batch.
+__device__ __forceinline__ float4 parts_sum4(const Partials& pp, size_t off) {
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    const float* p = pp.p + off;
+    for (int s0 = 0; s0 < pp.n_seg; s0 += 4) {
+        float4 v[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            v[i] = s0 + i < pp.n_seg ? __ldcg(reinterpret_cast<const float4*>(p + (size_t)(s0 + i) * pp.seg_stride)) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            if (s0 + i < pp.n_seg) { acc.x += v[i].x; acc.y += v[i].y; acc.z += v[i].z; acc.w += v[i].w; }
+    }
+    return acc;
+}
+// The same for N offsets at once: all loads of a batch of parts travel together.
+template <int N>
+__device__ __forceinline__ void parts_sum_n(const Partials& pp, const size_t (&off)[N], const bool (&on)[N], float (&acc)[N]) {
+    constexpr int B = N >= 8 ? 2 : (N >= 4 ? 4 : 8);                  // parts per batch: at most 16-32 loads in flight per thread
+#pragma unroll
+    for (int j = 0; j < N; ++j) acc[j] = 0.f;
+    for (int s0 = 0; s0 < pp.n_seg; s0 += B) {
+        float v[N][B];
+#pragma unroll
+        for (int j = 0; j < N; ++j)
+#pragma unroll
+            for (int i = 0; i < B; ++i)
+                v[j][i] = (on[j] && s0 + i < pp.n_seg) ? __ldcg(pp.p + (size_t)(s0 + i) * pp.seg_stride + off[j]) : 0.f;
+#pragma unroll
+        for (int j = 0; j < N; ++j)
+#pragma unroll
+            for (int i = 0; i < B; ++i)
+                if (on[j] && s0 + i < pp.n_seg) acc[j] += v[j][i];
+    }
+}
+
 constexpr int kAttnChunk = 64;       // split-K granularity over the sequence (fixed absolute boundaries)
 
 size_t gemv_smem_bytes(const cass_blob_info& bi, int nb);

@@ -110,14 +110,11 @@ __global__ void __launch_bounds__(256) k_kv_append(KvGeom g, KvComp ck, KvComp c
             const int i = it / per_row, e = it % per_row, hq = e / half, j = e % half;
             const size_t r = (size_t)blockIdx.z * n_new + i;
             const int ia = hq * g.d + j, ib = ia + half;
-            float a = 0.f, b = 0.f;
-            for (int sgm = 0; sgm < pp.n_seg; ++sgm) {
-                const float* q = pp.p + (size_t)sgm * pp.seg_stride + r * pp.row_stride;
-                a += q[ia];
-                b += q[ib];
-            }
-            a = round_bf16(a);
-            b = round_bf16(b);
+            const size_t offs[2] = {r * pp.row_stride + ia, r * pp.row_stride + ib};
+            const bool on2[2] = {true, true};
+            float ab[2];
+            parts_sum_n<2>(pp, offs, on2, ab);
+            const float a = round_bf16(ab[0]), b = round_bf16(ab[1]);
             const size_t ti = (size_t)(start + i) * half + j;
             const float c = rs.cos_t[ti], sn = rs.sin_t[ti];
             rs.qkv[r * qkv_dim + ia] = float_to_bf16_bits(a * c - b * sn);
@@ -149,14 +146,14 @@ __global__ void __launch_bounds__(256) k_kv_append(KvGeom g, KvComp ck, KvComp c
                 const int base = (rs.n_q + (kind ? g.n_kv : 0) + head) * g.d;
                 const Partials& pp = rs.pp;
                 float val[kKvMaxPerLane];
+                {
+                    size_t offs[kKvMaxPerLane];
+                    bool on[kKvMaxPerLane];
 #pragma unroll
-                for (int j = 0; j < kKvMaxPerLane; ++j) {
-                    val[j] = 0.f;
-                    if (j < nj) {
-                        for (int sgm = 0; sgm < pp.n_seg; ++sgm)
-                            val[j] += pp.p[(size_t)sgm * pp.seg_stride + r * pp.row_stride + base + lane + 32 * j];
-                        val[j] = round_bf16(val[j]);
-                    }
+                    for (int j = 0; j < kKvMaxPerLane; ++j) { offs[j] = r * pp.row_stride + base + lane + 32 * j; on[j] = j < nj; }
+                    parts_sum_n<kKvMaxPerLane>(pp, offs, on, val);
+#pragma unroll
+                    for (int j = 0; j < kKvMaxPerLane; ++j) val[j] = j < nj ? round_bf16(val[j]) : 0.f;
                 }
                 if (kind == 0) {                         // K: rotate the pairs (c, c + d/2), both held by this lane
 #pragma unroll

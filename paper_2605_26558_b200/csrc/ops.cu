@@ -61,11 +61,7 @@ __global__ void __launch_bounds__(1024) k_residual_rmsnorm(uint16_t* __restrict_
             if (y_bf16 || pp.p) {
                 float y[4];
                 if (pp.p) {
-                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-                    for (int s = 0; s < pp.n_seg; ++s) {
-                        const float4 p = *reinterpret_cast<const float4*>(pp.p + (size_t)s * pp.seg_stride + (size_t)r * pp.row_stride + i);
-                        acc.x += p.x; acc.y += p.y; acc.z += p.z; acc.w += p.w;
-                    }
+                    const float4 acc = parts_sum4(pp, (size_t)r * pp.row_stride + i);
                     y[0] = round_bf16(acc.x); y[1] = round_bf16(acc.y); y[2] = round_bf16(acc.z); y[3] = round_bf16(acc.w);
                 } else {
                     const uint2 yv = *reinterpret_cast<const uint2*>(y_bf16 + (size_t)r * hidden + i);
@@ -119,9 +115,7 @@ __global__ void k_qkv_rope(uint16_t* __restrict__ qkv, Partials pp,
     const int n_items = n_rot + n_kv * d;              // + plain v elements
     auto load = [&](int i) -> float {
         if (pp.p) {
-            float acc = 0.f;
-            for (int s = 0; s < pp.n_seg; ++s) acc += pp.p[(size_t)s * pp.seg_stride + (size_t)r * pp.row_stride + i];
-            return round_bf16(acc);
+            return round_bf16(parts_sum(pp, (size_t)r * pp.row_stride + i));
         }
         return bf16_bits_to_float(row[i]);
     };
@@ -148,14 +142,12 @@ __global__ void k_swiglu(const uint16_t* __restrict__ gu, Partials pp,
     for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < ffn; i += gridDim.x * blockDim.x) {
         float g, u;
         if (pp.p) {
-            float ag = 0.f, au = 0.f;
-            for (int s = 0; s < pp.n_seg; ++s) {
-                const float* q = pp.p + (size_t)s * pp.seg_stride + (size_t)r * pp.row_stride;
-                ag += q[i];
-                au += q[ffn + i];
-            }
-            g = round_bf16(ag);
-            u = round_bf16(au);
+            const size_t offs[2] = {(size_t)r * pp.row_stride + i, (size_t)r * pp.row_stride + ffn + i};
+            const bool on2[2] = {true, true};
+            float gu2[2];
+            parts_sum_n<2>(pp, offs, on2, gu2);
+            g = round_bf16(gu2[0]);
+            u = round_bf16(gu2[1]);
         } else {
             g = bf16_bits_to_float(gu[(size_t)r * 2 * ffn + i]);
             u = bf16_bits_to_float(gu[(size_t)r * 2 * ffn + ffn + i]);
@@ -186,8 +178,7 @@ __global__ void __launch_bounds__(256) k_argmax_part(const float* __restrict__ l
     for (int i = lo + threadIdx.x; i < hi; i += blockDim.x) {
         float v;
         if (pp.p) {
-            v = 0.f;
-            for (int s = 0; s < pp.n_seg; ++s) v += pp.p[(size_t)s * pp.seg_stride + (size_t)r * pp.row_stride + i];
+            v = parts_sum(pp, (size_t)r * pp.row_stride + i);
         } else {
             v = logits[(size_t)r * vocab + i];
         }
