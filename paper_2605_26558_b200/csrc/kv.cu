@@ -12,7 +12,9 @@ constexpr int kKvFixMax = 76;        // head_dim 256, no truncation: 3 entry + 8
 
 // Per-token selection: lane holds elements c = lane + 32 j.  keep[j] is set for the d - n_prune largest
 // |x| (ties: the lower channel is pruned first).  Key = (|x| bits << 8) | channel is unique, so the kept set is
-// {key >= T} where T is the largest value with at most n_prune keys below it; T is found bit by bit.
+// {key >= T} where T is the largest value with at most n_prune keys below it; T is found two bits at a time: the three
+// candidates of a step are counted in one packed word, so a step costs one warp reduction and the chain of dependent
+// reductions is half that of a bit-by-bit search.
 __device__ __forceinline__ void kv_select(const uint32_t (&bits)[kKvMaxPerLane], int nj, int n_prune, int lane,
                                           bool (&keep)[kKvMaxPerLane]) {
     uint32_t key[kKvMaxPerLane];
@@ -21,12 +23,22 @@ __device__ __forceinline__ void kv_select(const uint32_t (&bits)[kKvMaxPerLane],
         key[j] = j < nj ? (((bits[j] & 0x7FFFu) << 8) | (uint32_t)(lane + 32 * j)) : 0xFFFFFFFFu;
     uint32_t thr = 0;
     if (n_prune > 0) {
-        for (int bit = 22; bit >= 0; --bit) {
-            const uint32_t cand = thr | (1u << bit);
+        {                                                                        // 23 key bits: the top one alone
             int c = 0;
 #pragma unroll
-            for (int j = 0; j < kKvMaxPerLane; ++j) c += key[j] < cand;
-            if (__reduce_add_sync(0xffffffffu, c) <= n_prune) thr = cand;
+            for (int j = 0; j < kKvMaxPerLane; ++j) c += key[j] < (1u << 22);
+            if ((int)__reduce_add_sync(0xffffffffu, c) <= n_prune) thr = 1u << 22;
+        }
+#pragma unroll 1
+        for (int bit = 20; bit >= 0; bit -= 2) {
+            const uint32_t c1 = thr | (1u << bit), c2 = thr | (2u << bit), c3 = thr | (3u << bit);
+            uint32_t c = 0;                                   // three counts of at most 256 each in one word: one reduction per step
+#pragma unroll
+            for (int j = 0; j < kKvMaxPerLane; ++j)
+                c += (uint32_t)(key[j] < c1) + ((uint32_t)(key[j] < c2) << 10) + ((uint32_t)(key[j] < c3) << 20);
+            c = __reduce_add_sync(0xffffffffu, c);
+            const int n1 = (int)(c & 1023u), n2 = (int)((c >> 10) & 1023u), n3 = (int)(c >> 20);      // n1 <= n2 <= n3
+            thr = n3 <= n_prune ? c3 : (n2 <= n_prune ? c2 : (n1 <= n_prune ? c1 : thr));
         }
     }
 #pragma unroll
@@ -95,10 +107,16 @@ __global__ void __launch_bounds__(256) k_kv_append(KvGeom g, KvComp ck, KvComp c
     __shared__ uint32_t s_fix[kKvWarps][kKvFixMax];          // bitmap (<= 8) + field words (<= 64)
     __shared__ uint32_t s_una[kKvWarps][kKvStageWords];
     __shared__ uint32_t s_nw[kKvWarps], s_off[kKvWarps];
-    pdl_early<1>();
-    pdl_wait();
+    __shared__ uint8_t s_e2r[256];                           // exponent -> rank of this (head, K|V): frozen with the codebook
     const int head = blockIdx.x, kind = blockIdx.y, seq = seq0 + blockIdx.z;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    // The codebook tables were written when the codebook was frozen, long before this launch's predecessor: they may be
+    // read ahead of the wait, which hides their latency.
+    if ((flags & CASS_KV_COMPRESSED) && (!FUSED || head < g.n_kv) && threadIdx.x < 256)
+        s_e2r[threadIdx.x] = of_seq((kind ? cv : ck).exp_to_rank, seq, g.seq_stride)[threadIdx.x];
+    pdl_early<1>();
+    pdl_wait();
+    __syncthreads();
     if (FUSED && head >= g.n_kv) {
         // ---- query heads: q[r][h][j], q[r][h][j + d/2] rotated by the row's position ----
         if (kind != 0) return;
@@ -110,13 +128,13 @@ __global__ void __launch_bounds__(256) k_kv_append(KvGeom g, KvComp ck, KvComp c
             const int i = it / per_row, e = it % per_row, hq = e / half, j = e % half;
             const size_t r = (size_t)blockIdx.z * n_new + i;
             const int ia = hq * g.d + j, ib = ia + half;
+            const size_t ti = (size_t)(start + i) * half + j;
+            const float c = __ldg(rs.cos_t + ti), sn = __ldg(rs.sin_t + ti);      // travel together with the parts
             const size_t offs[2] = {r * pp.row_stride + ia, r * pp.row_stride + ib};
             const bool on2[2] = {true, true};
             float ab[2];
             parts_sum_n<2>(pp, offs, on2, ab);
             const float a = round_bf16(ab[0]), b = round_bf16(ab[1]);
-            const size_t ti = (size_t)(start + i) * half + j;
-            const float c = rs.cos_t[ti], sn = rs.sin_t[ti];
             rs.qkv[r * qkv_dim + ia] = float_to_bf16_bits(a * c - b * sn);
             rs.qkv[r * qkv_dim + ib] = float_to_bf16_bits(b * c + a * sn);
         }
@@ -146,6 +164,14 @@ __global__ void __launch_bounds__(256) k_kv_append(KvGeom g, KvComp ck, KvComp c
                 const int base = (rs.n_q + (kind ? g.n_kv : 0) + head) * g.d;
                 const Partials& pp = rs.pp;
                 float val[kKvMaxPerLane];
+                float rc[kKvMaxPerLane / 2], rsn[kKvMaxPerLane / 2];      // the position's rotation, fetched while the parts travel
+#pragma unroll
+                for (int j = 0; j < kKvMaxPerLane / 2; ++j) {
+                    const bool rot = kind == 0 && j < hj;
+                    const size_t ti = (size_t)pos * half + lane + 32 * j;
+                    rc[j] = rot ? __ldg(rs.cos_t + ti) : 1.f;
+                    rsn[j] = rot ? __ldg(rs.sin_t + ti) : 0.f;
+                }
                 {
                     size_t offs[kKvMaxPerLane];
                     bool on[kKvMaxPerLane];
@@ -159,8 +185,7 @@ __global__ void __launch_bounds__(256) k_kv_append(KvGeom g, KvComp ck, KvComp c
 #pragma unroll
                     for (int j = 0; j < kKvMaxPerLane / 2; ++j) {
                         if (j < hj) {
-                            const size_t ti = (size_t)pos * half + lane + 32 * j;
-                            const float c = rs.cos_t[ti], sn = rs.sin_t[ti];
+                            const float c = rc[j], sn = rsn[j];
                             const float a = val[j], b = val[j + hj];
                             val[j] = bf16_bits_to_float(float_to_bf16_bits(a * c - b * sn));
                             val[j + hj] = bf16_bits_to_float(float_to_bf16_bits(b * c + a * sn));
@@ -185,6 +210,8 @@ __global__ void __launch_bounds__(256) k_kv_append(KvGeom g, KvComp ck, KvComp c
             }
         }
         if (flags & CASS_KV_COMPRESSED) {
+            uint32_t off_first = 0;                          // arena offset of this round's first token: fetched while the record is formed
+            if (threadIdx.x == 0 && start_pos + base < g.max_seq) off_first = off[start_pos + base];
             if (active) {
                 kv_select(bits, nj, g.n_prune, lane, keep);
                 for (int w = lane; w < kKvFixMax; w += 32) s_fix[warp][w] = 0;
@@ -225,7 +252,7 @@ __global__ void __launch_bounds__(256) k_kv_append(KvGeom g, KvComp ck, KvComp c
                             if (j > 0 && lane == 0) s_fix[warp][(j - 1) / 3] |= (ubase & 0x3FFu) << (20 - 10 * ((j - 1) % 3));
                             uint32_t bm = __brev(__ballot_sync(0xffffffffu, keep[j]));   // channel c at bit 31 - c%32
                             if (lane == 0) s_fix[warp][ew + j] = bm;
-                            uint32_t len = keep[j] ? (uint32_t)exp_to_rank[(bits[j] >> 7) & 0xFF] + 1u : 0u;
+                            uint32_t len = keep[j] ? (uint32_t)s_e2r[(bits[j] >> 7) & 0xFF] + 1u : 0u;
                             uint32_t incl = len;
 #pragma unroll
                             for (int o = 1; o < 32; o <<= 1) {
@@ -275,7 +302,7 @@ __global__ void __launch_bounds__(256) k_kv_append(KvGeom g, KvComp ck, KvComp c
             if (lane == 0) s_nw[warp] = active ? n_words : 0u;
             __syncthreads();
             if (threadIdx.x == 0) {
-                uint32_t o = off[start_pos + base];
+                uint32_t o = off_first;
                 for (int w = 0; w < kKvWarps; ++w) {
                     int p = start_pos + base + w;
                     if (base + w >= n_new || p >= g.max_seq) break;
