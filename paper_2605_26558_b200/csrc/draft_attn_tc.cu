@@ -21,8 +21,14 @@ namespace cass {
 
 constexpr int kTcTok = kAttnChunk;            // tokens per CTA
 constexpr int kTcThreads = 128;
-constexpr int kTcUnaStage = 12;               // staged unary words per token (a typical record has 5-8)
-constexpr int kTcUnaRows = kTcUnaStage + 2;   // rows of a warp's unary staging: a window reads the word of its cursor and the next
+// Staged exponent words per token: room for 5 code bits per kept value (a typical record takes 2-3), the whole code
+// budget at most; longer records and records with raw exponents are read in place.  A warp's staging has two rows more:
+// a window reads the word of its cursor and the next.
+__host__ __device__ inline int tc_una_stage(const KvGeom& g) {
+    int w = ceil_div(5 * g.kept, 32);
+    if (w > g.rec_words_max) w = g.rec_words_max;
+    return w < 4 ? 4 : w;
+}
 constexpr int kTcHeads = 8;                   // query heads per KV head the N = 8 operand holds
 constexpr int kTcPad = 8;                     // halfwords of padding per tile row: rows 16 bytes apart modulo 128
 
@@ -119,7 +125,7 @@ __device__ __noinline__ void tc_walk_slow(const uint32_t* bm, const uint32_t* fl
 // the group and redoes it with the careful walk.  `emit` = false: the lane only keeps the warp in step.
 template <int T>
 __device__ __forceinline__ void tc_walk(const uint32_t* bmP, const uint32_t* flP, const uint32_t* unP, const uint32_t* lutP, const uint8_t* r2e,
-                                        int kept, int d, uint32_t una_bits, uint32_t row_a, bool emit) {
+                                        int kept, int d, uint32_t una_bits, uint32_t row_a, bool emit, int stage) {
     constexpr int F = 8 - T, PER = 32 / F, NFW = kGroupCols / PER;
     constexpr uint32_t MASK16 = 0x8000u | (((1u << (7 - T)) - 1u) << T);
     static_assert(PER == 4 || PER == 8, "fields tile a word");
@@ -188,7 +194,7 @@ __device__ __forceinline__ void tc_walk(const uint32_t* bmP, const uint32_t* flP
             bpos = b; upos = u;
         }
         bpos = min(bpos, (uint32_t)d);                                // a walk that lost its way stays inside the staging
-        upos = min(upos, (uint32_t)kTcUnaStage * 32u);
+        upos = min(upos, (uint32_t)stage * 32u);
         fl_a += NFW * 128u;
     };
     for (int grp = 0; grp < n_full; ++grp) group(grp, std::false_type{});
@@ -235,15 +241,16 @@ __global__ void __launch_bounds__(kTcThreads) k_draft_attn_tc(KvGeom g, KvComp c
     uint32_t* fix_s = reinterpret_cast<uint32_t*>(q_s + kTcHeads * ks);       // [4 warps][wpt + 1][32] records; after the walk:
     uint16_t* p_s = reinterpret_cast<uint16_t*>(fix_s);                       //   [2][8][64 + 8] probabilities, high and low bf16 term
     float* sc_s = reinterpret_cast<float*>(p_s + 2 * kTcHeads * (kTcTok + kTcPad));   //   [8][64] scores
-    uint32_t* una_s = fix_s + tc_fix_words(g);                                // [4 warps][kTcUnaRows][32]
-    uint32_t* lut_s = una_s + 4 * kTcUnaRows * 32;                            // [2][32] rank -> exponent << 7 (a window holds ranks < 32)
+    const int stage = tc_una_stage(g), una_rows = stage + 2;
+    uint32_t* una_s = fix_s + tc_fix_words(g);                                // [4 warps][una_rows][32]
+    uint32_t* lut_s = una_s + 4 * una_rows * 32;                            // [2][32] rank -> exponent << 7 (a window holds ranks < 32)
     float* run_s = reinterpret_cast<float*>(lut_s + 64);                      // [8][3]: running max, running sum, rescale factor of the chunk
 
     // warps 0,1 -> K records of tokens t0 + 32 w .., warps 2,3 -> V records of the same tokens
     const int kind = warp >> 1, tw = warp & 1;
     const KvComp& c = kind ? cv0 : ck0;                                       // sequence 0's; shifted to this sequence where used
     uint32_t* my_fix = fix_s + warp * (g.wpt + 1) * 32;
-    uint32_t* my_una = una_s + warp * kTcUnaRows * 32;
+    uint32_t* my_una = una_s + warp * una_rows * 32;
     const uint32_t* fixed_h = of_seq(c.fixed, seq, g.seq_stride) + (size_t)head * g.n_blocks * g.wpt * 32;
     const uint32_t* off_h = of_seq(c.off, seq, g.seq_stride) + (size_t)head * (g.max_seq + 1);
     const uint32_t* arena = of_seq(c.arena, seq, g.seq_stride) + (size_t)head * g.arena_words;
@@ -292,9 +299,9 @@ __global__ void __launch_bounds__(kTcThreads) k_draft_attn_tc(KvGeom g, KvComp c
             for (int w = 0; w < g.wpt; ++w) tc_cp_async4(fa + w * 128, fixed + w * 32 + src_lane, true);      // coalesced block copy
             my_fix[g.wpt * 32 + lane] = 0u;
             const uint32_t ua = smem_u32(my_una + lane);
-            const bool fits = n_una <= (uint32_t)kTcUnaStage;
-#pragma unroll
-            for (int w = 0; w < kTcUnaRows; ++w) {
+            const bool fits = n_una <= (uint32_t)stage;
+#pragma unroll 4
+            for (int w = 0; w < una_rows; ++w) {
                 const bool take = fits && (uint32_t)w < n_una;
                 tc_cp_async4(ua + w * 128, arena + (take ? o0 + w : 0), take);
             }
@@ -309,12 +316,12 @@ __global__ void __launch_bounds__(kTcThreads) k_draft_attn_tc(KvGeom g, KvComp c
         __syncthreads();
         if (n_here > 0) {
             const bool raw = (my_fix[lane] & kKvRawFlag) != 0;                // entry word 0 of this token's record
-            const bool staged = n_una <= (uint32_t)kTcUnaStage && !raw;
+            const bool staged = n_una <= (uint32_t)stage && !raw;
             const uint32_t* lutP = lut_s + kind * 32;
             const uint32_t row_a = smem_u32((kind ? vt_s : kt_s) + (size_t)(tw * 32 + lane) * ks);
             const uint32_t* bmP = my_fix + g.e_words * 32 + lane;
             const uint32_t* flP = bmP + g.bm_words * 32;
-            tc_walk<T>(bmP, flP, my_una + lane, lutP, r2e, g.kept, d, n_una * 32u, row_a, staged);
+            tc_walk<T>(bmP, flP, my_una + lane, lutP, r2e, g.kept, d, n_una * 32u, row_a, staged, stage);
             if (!staged)                                                      // raw exponents or a very long record: read it in place
                 tc_walk_slow<T>(bmP, flP, arena + o0, 1, raw, 0, g.kept, 0u, 0u, (uint32_t)d, n_una * 32u, r2e, row_a);
         }
@@ -416,7 +423,7 @@ int launch_attn_merge(const AttnScratch& sc, int n_chunks_alloc, int chunk_token
 
 size_t draft_attn_tc_smem_bytes(const KvGeom& g) {
     const size_t ks = (size_t)g.d + kTcPad;
-    return (2 * kTcTok + kTcHeads) * ks * 2 + (size_t)tc_fix_words(g) * 4 + (size_t)4 * kTcUnaRows * 32 * 4 + 64 * 4 + 3 * kTcHeads * 4 + 64;
+    return (2 * kTcTok + kTcHeads) * ks * 2 + (size_t)tc_fix_words(g) * 4 + (size_t)4 * (tc_una_stage(g) + 2) * 32 * 4 + 64 * 4 + 3 * kTcHeads * 4 + 64;
 }
 
 bool draft_attn_tc_supported(const KvGeom& g, int n_q) {
