@@ -266,19 +266,34 @@ __global__ void __launch_bounds__(kTcThreads) k_draft_attn_tc(KvGeom g, KvComp c
         }
     };
 
+    // Everything the first chunk needs from global memory is requested before any of it is used: the first records'
+    // arena offsets, the rank tables and the query rows share one round trip.
+    uint32_t o0, n_una, o0_next, nu_next;
+    load_off(t_begin, o0_next, nu_next);
+    uint32_t lut_v = 0;
     if (tid < 64) {
         const uint8_t *rk = of_seq(ck0.rank_to_exp, seq, g.seq_stride), *rv = of_seq(cv0.rank_to_exp, seq, g.seq_stride);
-        lut_s[tid] = (uint32_t)(tid < 32 ? rk[tid] : rv[tid - 32]) << 7;
+        lut_v = tid < 32 ? rk[tid] : rv[tid - 32];
     }
+    constexpr int kQIter = 4;                                                 // query words per thread and batch
+    const int n_qw = G * d / 2;
+    for (int i = tid; i < kTcHeads * ks / 2; i += kTcThreads) reinterpret_cast<uint32_t*>(q_s)[i] = 0u;   // unused heads stay zero
     if (tid < 3 * kTcHeads) run_s[tid] = tid % 3 == 0 ? -INFINITY : 0.f;
-    {   // the query heads of the group, bf16 as they are; unused heads zero
-        for (int i = tid; i < kTcHeads * ks / 2; i += kTcThreads) reinterpret_cast<uint32_t*>(q_s)[i] = 0u;
-        __syncthreads();
-        for (int i = tid; i < G * d / 2; i += kTcThreads) {
-            const int gi = i / (d / 2), c2 = i % (d / 2);
-            reinterpret_cast<uint32_t*>(q_s + gi * ks)[c2] = reinterpret_cast<const uint32_t*>(qkv + (size_t)(head * G + gi) * d)[c2];
+    __syncthreads();
+    for (int i0 = tid; i0 < n_qw; i0 += kTcThreads * kQIter) {                // the query heads of the group, bf16 as they are
+        uint32_t qv[kQIter];
+#pragma unroll
+        for (int u = 0; u < kQIter; ++u) {
+            const int i = i0 + u * kTcThreads;
+            qv[u] = i < n_qw ? __ldg(reinterpret_cast<const uint32_t*>(qkv + (size_t)(head * G + i / (d / 2)) * d) + i % (d / 2)) : 0u;
+        }
+#pragma unroll
+        for (int u = 0; u < kQIter; ++u) {
+            const int i = i0 + u * kTcThreads;
+            if (i < n_qw) reinterpret_cast<uint32_t*>(q_s + (i / (d / 2)) * ks)[i % (d / 2)] = qv[u];
         }
     }
+    if (tid < 64) lut_s[tid] = lut_v << 7;
     constexpr int kMaxMt = 4;                                                 // 16-channel tiles of the output per warp (head_dim <= 256)
     float o_acc[kMaxMt][4];
 #pragma unroll
@@ -286,8 +301,6 @@ __global__ void __launch_bounds__(kTcThreads) k_draft_attn_tc(KvGeom g, KvComp c
 #pragma unroll
         for (int i = 0; i < 4; ++i) o_acc[j][i] = 0.f;
     const float scale = rsqrtf((float)d);
-    uint32_t o0, n_una, o0_next, nu_next;
-    load_off(t_begin, o0_next, nu_next);
 
     for (int t0 = t_begin; t0 < t_end; t0 += kTcTok) {
         o0 = o0_next; n_una = nu_next;

@@ -39,6 +39,7 @@ __device__ __forceinline__ float block_sum(float v, float* s_red) {
 // and iteration (16-byte loads of the fp32 partial sums); the updated values stay in registers for the second pass.
 constexpr int kNormMaxIter = 8;          // hidden <= 8 * 4 * blockDim.x
 
+template <int ITERS>          // rounds of 4 x blockDim.x values: hidden <= ITERS * 4 * blockDim.x
 __global__ void __launch_bounds__(1024) k_residual_rmsnorm(uint16_t* __restrict__ h, const uint16_t* __restrict__ y_bf16,
                                                            Partials pp,
                                                            const uint16_t* __restrict__ gain, uint16_t* __restrict__ out,
@@ -48,20 +49,21 @@ __global__ void __launch_bounds__(1024) k_residual_rmsnorm(uint16_t* __restrict_
     pdl_wait();
     const int r = blockIdx.x;
     uint16_t* hr = h + (size_t)r * hidden;
-    float vals[kNormMaxIter][4];
+    float vals[ITERS][4];
     float ss = 0.f;
     const int step = blockDim.x * 4;
 #pragma unroll
-    for (int it = 0; it < kNormMaxIter; ++it) {
+    for (int it = 0; it < ITERS; ++it) {
         const int i = threadIdx.x * 4 + it * step;
         if (i < hidden) {
             const uint2 hv = *reinterpret_cast<const uint2*>(hr + i);
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (pp.p) acc = parts_sum4(pp, (size_t)r * pp.row_stride + i);       // requested before hv is first used: one round trip for both
             float v[4] = {__uint_as_float(hv.x << 16), __uint_as_float(hv.x & 0xFFFF0000u), __uint_as_float(hv.y << 16),
                           __uint_as_float(hv.y & 0xFFFF0000u)};
             if (y_bf16 || pp.p) {
                 float y[4];
                 if (pp.p) {
-                    const float4 acc = parts_sum4(pp, (size_t)r * pp.row_stride + i);
                     y[0] = round_bf16(acc.x); y[1] = round_bf16(acc.y); y[2] = round_bf16(acc.z); y[3] = round_bf16(acc.w);
                 } else {
                     const uint2 yv = *reinterpret_cast<const uint2*>(y_bf16 + (size_t)r * hidden + i);
@@ -83,7 +85,7 @@ __global__ void __launch_bounds__(1024) k_residual_rmsnorm(uint16_t* __restrict_
     const float inv = 1.0f / sqrtf(ss / (float)hidden + eps);
     if (out) {
 #pragma unroll
-        for (int it = 0; it < kNormMaxIter; ++it) {
+        for (int it = 0; it < ITERS; ++it) {
             const int i = threadIdx.x * 4 + it * step;
             if (i < hidden) {
                 const uint2 gv = *reinterpret_cast<const uint2*>(gain + i);
@@ -295,18 +297,26 @@ static int norm_threads(int hidden) {
     return t > 1024 ? 1024 : t;
 }
 
-int launch_rmsnorm(const uint16_t* h, const uint16_t* gain, uint16_t* out, int rows, int hidden, float eps, cudaStream_t s) {
-    if (hidden % 4 || hidden > kNormMaxIter * 4 * 1024) return CASS_ERR_UNSUPPORTED;
-    CASS_PDL_LAUNCH(k_residual_rmsnorm, dim3(rows), dim3(norm_threads(hidden)), 0, s, const_cast<uint16_t*>(h), (const uint16_t*)nullptr,
-                    Partials{nullptr, 0, 0, 0}, gain, out, hidden, eps);
-    return CASS_OK;
+static int norm_iters(int hidden, int threads) {
+    const int it = ceil_div(hidden, 4 * threads);
+    return it <= 1 ? 1 : (it <= 2 ? 2 : (it <= 4 ? 4 : 8));
 }
 
 int launch_residual_rmsnorm(uint16_t* h, const uint16_t* y_bf16, Partials pp,
                             const uint16_t* gain, uint16_t* out, int rows, int hidden, float eps, cudaStream_t s) {
     if (hidden % 4 || hidden > kNormMaxIter * 4 * 1024) return CASS_ERR_UNSUPPORTED;
-    CASS_PDL_LAUNCH(k_residual_rmsnorm, dim3(rows), dim3(norm_threads(hidden)), 0, s, h, y_bf16, pp, gain, out, hidden, eps);
+    const int threads = norm_threads(hidden);
+    switch (norm_iters(hidden, threads)) {
+        case 1: CASS_PDL_LAUNCH(k_residual_rmsnorm<1>, dim3(rows), dim3(threads), 0, s, h, y_bf16, pp, gain, out, hidden, eps); break;
+        case 2: CASS_PDL_LAUNCH(k_residual_rmsnorm<2>, dim3(rows), dim3(threads), 0, s, h, y_bf16, pp, gain, out, hidden, eps); break;
+        case 4: CASS_PDL_LAUNCH(k_residual_rmsnorm<4>, dim3(rows), dim3(threads), 0, s, h, y_bf16, pp, gain, out, hidden, eps); break;
+        default: CASS_PDL_LAUNCH(k_residual_rmsnorm<8>, dim3(rows), dim3(threads), 0, s, h, y_bf16, pp, gain, out, hidden, eps); break;
+    }
     return CASS_OK;
+}
+
+int launch_rmsnorm(const uint16_t* h, const uint16_t* gain, uint16_t* out, int rows, int hidden, float eps, cudaStream_t s) {
+    return launch_residual_rmsnorm(const_cast<uint16_t*>(h), nullptr, Partials{nullptr, 0, 0, 0}, gain, out, rows, hidden, eps, s);
 }
 
 int launch_qkv_rope(uint16_t* qkv, Partials pp, const float* cos_t, const float* sin_t,
