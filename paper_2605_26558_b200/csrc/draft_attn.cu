@@ -472,8 +472,20 @@ __global__ void __launch_bounds__(kMergeThreads) k_attn_merge(AttnScratch sc, in
     const float* mp = sc.m + pair * n_chunks_alloc;
     const float* lp = sc.l + pair * n_chunks_alloc;
     float* part_s = w_s + ((n_chunks_alloc + 3) & ~3);
-    float M = -INFINITY;
-    for (int c = tid; c < n_ch; c += kMergeThreads) M = fmaxf(M, mp[c]);
+    // What the first round of every loop below needs is requested here, before any of it is used: the statistics of
+    // chunk tid and the partial outputs of this warp's first two chunks share one round trip to L2.
+    const float* op = sc.o + pair * n_chunks_alloc * d;
+    const bool has0 = tid < n_ch;
+    const float m_first = has0 ? __ldcg(mp + tid) : -INFINITY, l_first = has0 ? __ldcg(lp + tid) : 0.f;
+    const int dim0 = lane * 4;
+    float4 o_first[2];
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+        const int c = warp + k * kMergeWarps;
+        o_first[k] = (c < n_ch && dim0 < d) ? __ldcg(reinterpret_cast<const float4*>(op + (size_t)c * d + dim0)) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    float M = m_first;
+    for (int c = tid + kMergeThreads; c < n_ch; c += kMergeThreads) M = fmaxf(M, mp[c]);
     M = warp_max(M);
     if (lane == 0) s_red[warp] = M;
     __syncthreads();
@@ -482,7 +494,12 @@ __global__ void __launch_bounds__(kMergeThreads) k_attn_merge(AttnScratch sc, in
     for (int w = 1; w < kMergeWarps; ++w) M = fmaxf(M, s_red[w]);
     __syncthreads();
     float L = 0.f;
-    for (int c = tid; c < n_ch; c += kMergeThreads) {
+    if (has0) {
+        const float w = expf(m_first - M);
+        w_s[tid] = w;
+        L += w * l_first;
+    }
+    for (int c = tid + kMergeThreads; c < n_ch; c += kMergeThreads) {
         const float w = expf(mp[c] - M);
         w_s[c] = w;
         L += w * lp[c];
@@ -495,11 +512,21 @@ __global__ void __launch_bounds__(kMergeThreads) k_attn_merge(AttnScratch sc, in
     for (int w = 1; w < kMergeWarps; ++w) L += s_red[w];
     // warp w adds the chunks w, w + 8, ... (four dims per lane, 16-byte loads); the warps' sums are then added in warp
     // order: the order of every addition depends on the number of visible chunks only
-    const float* op = sc.o + pair * n_chunks_alloc * d;
-    for (int dim = lane * 4; dim < d; dim += 128) {
+    for (int dim = dim0; dim < d; dim += 128) {
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        int c = warp;
+        if (dim == dim0) {
+#pragma unroll
+            for (int k = 0; k < 2; ++k, c += kMergeWarps) {
+                if (c < n_ch) {
+                    const float w = w_s[c];
+                    const float4 o = o_first[k];
+                    acc.x = fmaf(w, o.x, acc.x); acc.y = fmaf(w, o.y, acc.y); acc.z = fmaf(w, o.z, acc.z); acc.w = fmaf(w, o.w, acc.w);
+                }
+            }
+        }
 #pragma unroll 4
-        for (int c = warp; c < n_ch; c += kMergeWarps) {
+        for (; c < n_ch; c += kMergeWarps) {
             const float w = w_s[c];
             const float4 o = *reinterpret_cast<const float4*>(op + (size_t)c * d + dim);
             acc.x = fmaf(w, o.x, acc.x); acc.y = fmaf(w, o.y, acc.y); acc.z = fmaf(w, o.z, acc.z); acc.w = fmaf(w, o.w, acc.w);
