@@ -230,7 +230,9 @@ int launch_verify_attn_tc(const KvGeom& g, const uint16_t* k_cache, const uint16
 inline int verify_gemm_bn(int rows) { return rows <= 16 ? 16 : rows <= 32 ? 32 : 64; }
 size_t verify_gemm_partial_floats(int n, int k, int bn);
 Partials verify_gemm_partials(const float* partial, int n, int k, int bn);
+// w_static: W is not the output of a kernel that may still be running when this one is scheduled (the bf16 matrices of
+// a session); its first tiles are then requested before the wait for the predecessor.
 int launch_verify_gemm(const uint16_t* W, const uint16_t* X, int rows, int bn, int n, int k, float* partial, uint16_t* y_bf16,
-                       float* y_f32, int32_t* d_status, cudaStream_t s);
+                       float* y_f32, int32_t* d_status, cudaStream_t s, int w_static = 0);
 
 }  // namespace cass

@@ -470,7 +470,7 @@ extern "C" int cass_verify(void* session, const int32_t* toks, int g, int32_t* t
     for (int l = 0; l < d.n_layers; ++l) {
         LayerDev& L = s->layers[l];
         if (calib) RC(launch_calib_accum(s->xn, rows, d.hidden, L.calib[0], s->st, st));
-        RC(launch_verify_gemm(weight(L.w.wqkv, L.blob[0], L.bi[0], L.vdata[0]), s->xn, rows, bn, s->qkv_dim, d.hidden, s->vg_partial, nullptr, nullptr, status, st));
+        RC(launch_verify_gemm(weight(L.w.wqkv, L.blob[0], L.bi[0], L.vdata[0]), s->xn, rows, bn, s->qkv_dim, d.hidden, s->vg_partial, nullptr, nullptr, status, st, s->from_parts ? 0 : 1));
         if (fused) {
             RC(launch_rope_kv_append(s->kg, L.ck, L.cv, L.kc, L.vc, vparts(s->qkv_dim, d.hidden), s->cos_t, s->sin_t, s->qkv,
                                      d.n_q_heads, 0, rps, kv_flags, s->st, B, st));
@@ -483,20 +483,20 @@ extern "C" int cass_verify(void* session, const int32_t* toks, int g, int32_t* t
         if (attn_tc) RC(launch_verify_attn_tc(s->kg, L.kc, L.vc, s->qkv, B, rps, d.n_q_heads, np_cols, s->st, s->asc, s->attn, status, st));
         else RC(launch_verify_attn(s->kg, L.kc, L.vc, s->qkv, B, rps, d.n_q_heads, s->st, s->asc, s->attn, st));
         if (calib) RC(launch_calib_accum(s->attn, rows, qd, L.calib[1], s->st, st));
-        RC(launch_verify_gemm(weight(L.w.wo, L.blob[1], L.bi[1], L.vdata[1]), s->attn, rows, bn, d.hidden, qd, s->vg_partial, nullptr, nullptr, status, st));
+        RC(launch_verify_gemm(weight(L.w.wo, L.blob[1], L.bi[1], L.vdata[1]), s->attn, rows, bn, d.hidden, qd, s->vg_partial, nullptr, nullptr, status, st, s->from_parts ? 0 : 1));
         RC(launch_residual_rmsnorm(s->h, nullptr, vparts(d.hidden, qd), (const uint16_t*)L.w.norm_ffn, s->xn,
                                    rows, d.hidden, d.rms_eps, st));
         if (calib) RC(launch_calib_accum(s->xn, rows, d.hidden, L.calib[2], s->st, st));
-        RC(launch_verify_gemm(weight(L.w.wgu, L.blob[2], L.bi[2], L.vdata[2]), s->xn, rows, bn, 2 * d.ffn, d.hidden, s->vg_partial, nullptr, nullptr, status, st));
+        RC(launch_verify_gemm(weight(L.w.wgu, L.blob[2], L.bi[2], L.vdata[2]), s->xn, rows, bn, 2 * d.ffn, d.hidden, s->vg_partial, nullptr, nullptr, status, st, s->from_parts ? 0 : 1));
         RC(launch_swiglu(nullptr, vparts(2 * d.ffn, d.hidden), s->act, rows, d.ffn, st));
         if (calib) RC(launch_calib_accum(s->act, rows, d.ffn, L.calib[3], s->st, st));
-        RC(launch_verify_gemm(weight(L.w.wd, L.blob[3], L.bi[3], L.vdata[3]), s->act, rows, bn, d.hidden, d.ffn, s->vg_partial, nullptr, nullptr, status, st));
+        RC(launch_verify_gemm(weight(L.w.wd, L.blob[3], L.bi[3], L.vdata[3]), s->act, rows, bn, d.hidden, d.ffn, s->vg_partial, nullptr, nullptr, status, st, s->from_parts ? 0 : 1));
         const uint16_t* next_gain = (const uint16_t*)(l + 1 < d.n_layers ? s->layers[l + 1].w.norm_attn : s->norm_final);
         RC(launch_residual_rmsnorm(s->h, nullptr, vparts(d.hidden, d.ffn), next_gain, s->xn, rows, d.hidden,
                                    d.rms_eps, st));
     }
     if (calib) RC(launch_calib_accum(s->xn, rows, d.hidden, s->calib_lm, s->st, st));
-    RC(launch_verify_gemm(weight(s->lm_head, s->lm_blob, s->lm_bi, s->lm_vdata), s->xn, rows, bn, d.vocab, d.hidden, s->vg_partial, nullptr, nullptr, status, st));
+    RC(launch_verify_gemm(weight(s->lm_head, s->lm_blob, s->lm_bi, s->lm_vdata), s->xn, rows, bn, d.vocab, d.hidden, s->vg_partial, nullptr, nullptr, status, st, s->from_parts ? 0 : 1));
     RC(launch_argmax(nullptr, vparts(d.vocab, d.hidden), rows, d.vocab, target_argmax, 1, logits_opt,
                      s->argmax_val, s->argmax_tmp, s->st, 0, st));
     return w_rc;

@@ -44,7 +44,8 @@ template <int BN>
 __global__ void __launch_bounds__(kTcThreads) k_verify_gemm_tc(const __grid_constant__ CUtensorMap map_w,
                                                                 const __grid_constant__ CUtensorMap map_x,
                                                                 float* __restrict__ partial, int rows, int n,
-                                                                int kb_total, int kb_per_split, int32_t* __restrict__ d_status) {
+                                                                int kb_total, int kb_per_split, int32_t* __restrict__ d_status,
+                                                                int w_static) {
     extern __shared__ uint8_t smem_dyn[];
     uint8_t* base = reinterpret_cast<uint8_t*>(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);     // swizzled tiles: 1024-byte aligned
     uint8_t* sA = base;
@@ -74,13 +75,29 @@ __global__ void __launch_bounds__(kTcThreads) k_verify_gemm_tc(const __grid_cons
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
-    // barriers and tensor memory are set up; the activations and the scratch belong to the preceding kernels
+    // Barriers and tensor memory are set up.  The weights are nobody's output: the first ring of weight tiles is
+    // requested ahead of the wait for the preceding kernels, whose results are the activations and the scratch.
+    // (w_static = 0: the weights too come from a preceding kernel, e.g. rebuilt from their two parts: nothing is early)
+    const int n_pre = nkb < kTcStages ? nkb : kTcStages;
+    if (warp == 0 && lane == 0 && w_static) {
+        for (int kb = 0; kb < n_pre; ++kb) {                 // stages are empty at the start: nothing to wait for
+            mbar_expect_tx(&full[kb], kTcABytes + kTcBBytes);
+            tma_load_2d(sA + kb * kTcABytes, &map_w, (kb0 + kb) * kTcBK, m0, &full[kb]);
+        }
+    }
     pdl_early<5>();
     pdl_wait();
 
     if (warp == 0 && lane == 0) {
         // ---- producer: TMA loads into the ring ----
-        for (int kb = 0; kb < nkb; ++kb) {
+        for (int kb = 0; kb < n_pre; ++kb) {
+            if (!w_static) {
+                mbar_expect_tx(&full[kb], kTcABytes + kTcBBytes);
+                tma_load_2d(sA + kb * kTcABytes, &map_w, (kb0 + kb) * kTcBK, m0, &full[kb]);
+            }
+            tma_load_2d(sB + kb * kTcBBytes, &map_x, (kb0 + kb) * kTcBK, 0, &full[kb]);
+        }
+        for (int kb = n_pre; kb < nkb; ++kb) {
             const int s = kb % kTcStages;
             const uint32_t ph = (uint32_t)(kb / kTcStages) & 1u;
             if (!mbar_wait_bounded(&empty[s], ph ^ 1u)) { atomicExch(d_status, CASS_ERR_TIMEOUT); break; }
@@ -175,19 +192,19 @@ size_t verify_gemm_partial_floats(int n, int k, int bn) {
 
 template <int BN>
 static int launch_tc(const CUtensorMap& mw, const CUtensorMap& mx, float* partial, int rows, int n, int kbt, int kbs, int ns,
-                     int32_t* d_status, cudaStream_t s) {
+                     int32_t* d_status, int w_static, cudaStream_t s) {
     static bool attr = false;
     if (!attr) {
         CASS_CUDA_CHECK(cudaFuncSetAttribute(k_verify_gemm_tc<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc_smem(BN)));
         attr = true;
     }
     dim3 grid(ceil_div(n, kTcBM), ns);
-    CASS_PDL_LAUNCH(k_verify_gemm_tc<BN>, grid, dim3(kTcThreads), (size_t)tc_smem(BN), s, mw, mx, partial, rows, n, kbt, kbs, d_status);
+    CASS_PDL_LAUNCH(k_verify_gemm_tc<BN>, grid, dim3(kTcThreads), (size_t)tc_smem(BN), s, mw, mx, partial, rows, n, kbt, kbs, d_status, w_static);
     return CASS_OK;
 }
 
 int launch_verify_gemm(const uint16_t* W, const uint16_t* X, int rows, int bn, int n, int k, float* partial, uint16_t* y_bf16,
-                       float* y_f32, int32_t* d_status, cudaStream_t s) {
+                       float* y_f32, int32_t* d_status, cudaStream_t s, int w_static) {
     if (rows < 1 || rows > bn || (bn != 16 && bn != 32 && bn != 64) || (k % 8) || n < 1 || !partial || !d_status)
         return CASS_ERR_INVALID_ARG;
     if (((uintptr_t)W & 15) || ((uintptr_t)X & 15)) return CASS_ERR_INVALID_ARG;
@@ -198,9 +215,9 @@ int launch_verify_gemm(const uint16_t* W, const uint16_t* X, int rows, int bn, i
     if (rc) return rc;
     int kbt, kbs, ns;
     split_plan(n, k, &kbt, &kbs, &ns);
-    if (bn == 16) rc = launch_tc<16>(mw, mx, partial, rows, n, kbt, kbs, ns, d_status, s);
-    else if (bn == 32) rc = launch_tc<32>(mw, mx, partial, rows, n, kbt, kbs, ns, d_status, s);
-    else rc = launch_tc<64>(mw, mx, partial, rows, n, kbt, kbs, ns, d_status, s);
+    if (bn == 16) rc = launch_tc<16>(mw, mx, partial, rows, n, kbt, kbs, ns, d_status, w_static, s);
+    else if (bn == 32) rc = launch_tc<32>(mw, mx, partial, rows, n, kbt, kbs, ns, d_status, w_static, s);
+    else rc = launch_tc<64>(mw, mx, partial, rows, n, kbt, kbs, ns, d_status, w_static, s);
     if (rc) return rc;
     if (!y_bf16 && !y_f32) return CASS_OK;          // the caller's next kernel adds the parts itself
     dim3 g2(ceil_div(n, 256), rows);
