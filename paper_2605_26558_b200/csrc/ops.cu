@@ -45,6 +45,13 @@ __global__ void __launch_bounds__(1024) k_residual_rmsnorm(uint16_t* __restrict_
                                                            const uint16_t* __restrict__ gain, uint16_t* __restrict__ out,
                                                            int hidden, float eps) {
     __shared__ float s_red[32];
+    // the gains are weights: they are requested ahead of the wait for the predecessor
+    uint2 gvs[ITERS];
+#pragma unroll
+    for (int it = 0; it < ITERS; ++it) {
+        const int i = threadIdx.x * 4 + it * (int)blockDim.x * 4;
+        gvs[it] = (out && i < hidden) ? __ldg(reinterpret_cast<const uint2*>(gain + i)) : make_uint2(0u, 0u);
+    }
     pdl_early<0>();
     pdl_wait();
     const int r = blockIdx.x;
@@ -88,7 +95,7 @@ __global__ void __launch_bounds__(1024) k_residual_rmsnorm(uint16_t* __restrict_
         for (int it = 0; it < ITERS; ++it) {
             const int i = threadIdx.x * 4 + it * step;
             if (i < hidden) {
-                const uint2 gv = *reinterpret_cast<const uint2*>(gain + i);
+                const uint2 gv = gvs[it];
                 const float gq[4] = {__uint_as_float(gv.x << 16), __uint_as_float(gv.x & 0xFFFF0000u), __uint_as_float(gv.y << 16),
                                      __uint_as_float(gv.y & 0xFFFF0000u)};
                 uint32_t ob[4];
