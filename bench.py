@@ -32,9 +32,9 @@ METRIC = "batch-1 decode tokens/s (8B-shape) + accepted len; draft-kernel HBM GB
 UNIT = "tokens/s"
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one k_draft_gemv launch divided by the blob's bytes, from the ncu
-# capture of the 28672 x 4096 matrix (profiles/draft_gemv_wgu_28672x4096.txt: 71.54 MB for a 70.6 MB blob); a launch
+# capture of the 28672 x 4096 matrix (profiles/draft_gemv_wgu_28672x4096.txt: 71.32 MB for a 70.6 MB blob); a launch
 # reads its blob once plus x and writes the partial sums, so traffic scales with the blob bytes.
-DRAM_BYTES_PER_BLOB_BYTE = 1.013
+DRAM_BYTES_PER_BLOB_BYTE = 1.010
 
 
 def _peaks():
