@@ -171,8 +171,8 @@ def run_reference(args):
 # ----------------------------------------------------------------------------------------------------------
 
 def launches_per_step(n_layers: int, gamma: int, max_seq: int = 0, kv_mode: int = 1, from_parts: bool = False) -> int:
-    # draft, per layer: 4 gemv, rope+kv, attention + merge (Cassandra-2 caches: the attention's last CTA merges), 2 norm, swiglu
-    draft = 2 + n_layers * (10 if kv_mode == 1 else 9) + 3     # + embed, norm | lm gemv, 2 argmax
+    # draft, per layer: 4 gemv, rope+kv, attention, merge, 2 norm, swiglu
+    draft = 2 + n_layers * 10 + 3     # + embed, norm | lm gemv, 2 argmax
     # verify, per layer: 4 gemm (each preceded by two reconstruction kernels when verifying from the two parts), rope+kv, attn, merge, 2 norm, swiglu
     verify = 2 + n_layers * (10 + (8 if from_parts else 0)) + 3 + (2 if from_parts else 0)
     return gamma * draft + verify + 1

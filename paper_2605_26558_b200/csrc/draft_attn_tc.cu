@@ -1,4 +1,4 @@
-// Draft decode attention over Cassandra-1 KV records (Sec. 4.1 draft inference; KV speculation data of
+// Draft decode attention over the compressed KV cache, Cassandra-1 and Cassandra-2 records (Sec. 4.1 draft inference; KV speculation data of
 // Sec. 4.2), dense-tile form: the decoders feed matrix units, as the paper's decoder array feeds the tensor cores
 // (Sec. 5.1, 5.2).  One CTA = one (KV head, run of 64-token chunks).  Per chunk, warps 0-1 decode the K records of 32 tokens each
 // (lane = token, the whole record by one lane) into a dense bf16 tile [token][channel] in shared memory, pruned channels
@@ -201,6 +201,111 @@ __device__ __forceinline__ void tc_walk(const uint32_t* bmP, const uint32_t* flP
     if (rem) group(n_full, std::true_type{});
 }
 
+// ---- Cassandra-2 (MX) records: fields = sign + magnitude >> t, one exponent byte E per 32-channel slice -------------
+// A value is (-1)^s (mag << t) 2^(E - 133).  With p the leading bit of mag << t its bf16 pattern is sign, exponent
+// E + p - 6, mantissa the bits below p: lut[field] = {sign | p << 7 | mantissa, mask}, and the pattern is
+// lut.x + (((E - 6) << 7) & lut.y) with mask 0 for a zero magnitude (and for slices with E < 7, whose fields are all zero).
+__device__ __forceinline__ uint2 tc_lds64(uint32_t a) {
+    uint2 v;
+    asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(a));
+    return v;
+}
+
+// Careful walk of the kept values k0 .. k0 + count - 1 of an MX record from column bpos on.  eb: the lane's slice table
+// ((E - 6) << 7 per slice, rows 32 words apart); lut: field -> {pattern, mask}.
+template <int T>
+__device__ __noinline__ void tc_walk_mx_slow(const uint32_t* bm, const uint32_t* fl, const uint32_t* eb, const uint2* lut, int k0, int count,
+                                             uint32_t bpos, uint32_t d, uint32_t row_a) {
+    constexpr int F = 8 - T, PER = 32 / F;
+    for (int e = 0; e < count; ++e) {
+        bool found = false;
+        while (bpos < d) {
+            const uint32_t w = bm[(bpos >> 5) * 32] << (bpos & 31);
+            if (w) { bpos += __clz(w); found = true; break; }
+            bpos = (bpos | 31u) + 1u;
+        }
+        if (!found || bpos >= d) break;                       // corrupt record: stop inside the row
+        const uint32_t col = bpos;
+        bpos += 1;
+        const uint32_t k = (uint32_t)(k0 + e);
+        const uint32_t f = (fl[(k / PER) * 32] >> (32 - F * (k % PER + 1))) & ((1u << F) - 1u);
+        const uint2 lm = lut[f];
+        tc_sts16(row_a + col * 2u, lm.x + (eb[(col >> 5) * 32] & lm.y));
+    }
+}
+
+// Walk of one staged MX record by one lane, 8 kept values per 32-bit bitmap window; the window's columns lie in at most
+// two slices, whose exponents are fetched once per group.  xP: the record's exponent words; ebP: room for the lane's
+// slice table (d / 32 + 2 rows).
+template <int T>
+__device__ __forceinline__ void tc_walk_mx(const uint32_t* bmP, const uint32_t* flP, const uint32_t* xP, uint32_t* ebP, const uint2* lutP,
+                                           int kept, int d, uint32_t row_a) {
+    constexpr int F = 8 - T, PER = 32 / F, NFW = kGroupCols / PER;
+    static_assert(PER == 4 || PER == 8, "fields tile a word");
+    const int S = d / 32;
+    for (int sl = 0; sl < S; ++sl) {
+        const uint32_t E = (xP[(sl >> 2) * 32] >> (24 - 8 * (sl & 3))) & 0xFFu;
+        ebP[sl * 32] = E >= 7u ? (E - 6u) << 7 : 0u;
+    }
+    ebP[S * 32] = 0u;
+    ebP[(S + 1) * 32] = 0u;
+    __syncwarp();
+    const uint32_t bm_a = smem_u32(bmP), eb_a = smem_u32(ebP), lut_a = smem_u32(lutP);
+    uint32_t fl_a = smem_u32(flP);
+    uint32_t bpos = 0;
+    const int n_full = kept / kGroupCols, rem = kept % kGroupCols;
+    auto group = [&](int grp, auto tail_c) {
+        constexpr bool tail = decltype(tail_c)::value;
+        const uint32_t bpos0 = bpos;
+        const uint32_t ba = bm_a + (bpos >> 5) * 128u;
+        uint32_t bv = __funnelshift_l(tc_lds_off<128>(ba), tc_lds(ba), bpos);        // 32 columns from bpos on
+        const uint32_t xg = row_a + bpos * 2u + 62u;                                 // address of column bpos + 31
+        const uint32_t ea = eb_a + (bpos >> 5) * 128u;
+        const uint32_t eb0 = tc_lds(ea), eb1 = tc_lds_off<128>(ea);                  // this slice's exponent and the next one's
+        const int pb = (int)(bpos & 31u) - 1;                                        // window bits <= pb lie in the next slice
+        uint32_t fwd[NFW];
+        fwd[0] = tc_lds(fl_a);
+        if (NFW > 1) fwd[NFW - 1] = tc_lds_off<128>(fl_a);
+        uint32_t addr[kGroupCols], val[kGroupCols];
+        uint32_t dry = 0, p = 0;
+#pragma unroll
+        for (int e = 0; e < kGroupCols; ++e) {
+            p = tc_bfind(bv);                                         // next kept column: bpos + 31 - p
+            addr[e] = tc_mad(p, 0xFFFFFFFEu, xg);
+            bv &= ~tc_shl(1u, p);
+            const uint32_t f = (fwd[e / PER] >> (32 - F * (e % PER + 1))) & ((1u << F) - 1u);
+            const uint2 lm = tc_lds64(lut_a + f * 8u);
+            const uint32_t eb = (int)p <= pb ? eb1 : eb0;
+            val[e] = lm.x + (eb & lm.y);
+            if (tail && e < rem) dry |= p;
+        }
+        bpos += 32u - p;
+        if (!tail) dry |= p;                                          // a search that failed fails from then on
+        const bool ok = (int32_t)dry >= 0;
+#pragma unroll
+        for (int e = 0; e < kGroupCols; ++e)
+            if (ok && (!tail || e < rem)) tc_sts16(addr[e], val[e]);
+        if (!ok) {
+            const int cnt = tail ? rem : kGroupCols;
+            tc_walk_mx_slow<T>(bmP, flP, ebP, lutP, grp * kGroupCols, cnt, bpos0, (uint32_t)d, row_a);
+            uint32_t b = bpos0;
+            for (int e = 0; e < cnt; ++e) {
+                while (b < (uint32_t)d) {
+                    const uint32_t w = bmP[(b >> 5) * 32] << (b & 31);
+                    if (w) { b += __clz(w) + 1; break; }
+                    b = (b | 31u) + 1u;
+                }
+            }
+            bpos = b;
+        }
+        bpos = min(bpos, (uint32_t)d);
+        fl_a += NFW * 128u;
+    };
+    for (int grp = 0; grp < n_full; ++grp) group(grp, std::false_type{});
+    if (rem) group(n_full, std::true_type{});
+}
+
+
 __device__ __forceinline__ void tc_cp_async4(uint32_t dst, const void* src, bool take) {      // take = false: zero fill
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(src), "r"(take ? 4 : 0) : "memory");
 }
@@ -217,7 +322,10 @@ __host__ __device__ inline int tc_fix_words(const KvGeom& g) {
 // grid = (runs, KV heads, sequences).  A CTA handles a run of consecutive 64-token chunks (tc_run_tokens positions: the
 // longer the visible cache, the longer the run, so that the grid stays near four CTAs per SM and the merge short) with a
 // running softmax: per chunk it stages and decodes the records, forms the scores, rescales what it has and adds P.V.
-template <int T>
+__host__ __device__ inline int tc_lut_words(const KvGeom& g) { return g.mode == 1 ? 64 : 2 << (8 - g.t); }
+__host__ __device__ inline int tc_una_rows(const KvGeom& g) { return g.mode == 1 ? tc_una_stage(g) + 2 : g.d / 32 + 2; }
+
+template <int MODE, int T>
 __global__ void __launch_bounds__(kTcThreads) k_draft_attn_tc(KvGeom g, KvComp ck0, KvComp cv0, const uint16_t* __restrict__ qkv,
                                                               int qkv_stride, int n_q, const DevState* __restrict__ st, AttnScratch sc,
                                                               int n_chunks_alloc) {
@@ -241,10 +349,10 @@ __global__ void __launch_bounds__(kTcThreads) k_draft_attn_tc(KvGeom g, KvComp c
     uint32_t* fix_s = reinterpret_cast<uint32_t*>(q_s + kTcHeads * ks);       // [4 warps][wpt + 1][32] records; after the walk:
     uint16_t* p_s = reinterpret_cast<uint16_t*>(fix_s);                       //   [2][8][64 + 8] probabilities, high and low bf16 term
     float* sc_s = reinterpret_cast<float*>(p_s + 2 * kTcHeads * (kTcTok + kTcPad));   //   [8][64] scores
-    const int stage = tc_una_stage(g), una_rows = stage + 2;
-    uint32_t* una_s = fix_s + tc_fix_words(g);                                // [4 warps][una_rows][32]
-    uint32_t* lut_s = una_s + 4 * una_rows * 32;                            // [2][32] rank -> exponent << 7 (a window holds ranks < 32)
-    float* run_s = reinterpret_cast<float*>(lut_s + 64);                      // [8][3]: running max, running sum, rescale factor of the chunk
+    const int stage = MODE == 1 ? tc_una_stage(g) : 0, una_rows = MODE == 1 ? stage + 2 : d / 32 + 2;
+    uint32_t* una_s = fix_s + tc_fix_words(g);                                // [4 warps][una_rows][32]: exponent words (MODE 1) | slice tables (MODE 2)
+    uint32_t* lut_s = una_s + 4 * una_rows * 32;                              // MODE 1: [2][32] rank -> exponent << 7; MODE 2: field -> {pattern, mask}
+    float* run_s = reinterpret_cast<float*>(lut_s + tc_lut_words(g));         // [8][3]: running max, running sum, rescale factor of the chunk
 
     // warps 0,1 -> K records of tokens t0 + 32 w .., warps 2,3 -> V records of the same tokens
     const int kind = warp >> 1, tw = warp & 1;
@@ -258,6 +366,7 @@ __global__ void __launch_bounds__(kTcThreads) k_draft_attn_tc(KvGeom g, KvComp c
     // Tokens beyond the visible length take the last visible token's record (their probabilities are zero).
     auto load_off = [&](int t0, uint32_t& o0, uint32_t& n_una) {
         o0 = 0; n_una = 0;
+        if (MODE != 1) return;                                                // Cassandra-2 records have no exponent stream
         const int n_here = min(32, cur_len - (t0 + tw * 32));
         if (t0 < t_end && n_here > 0) {
             const int tok = t0 + tw * 32 + min(lane, n_here - 1);
@@ -271,7 +380,7 @@ __global__ void __launch_bounds__(kTcThreads) k_draft_attn_tc(KvGeom g, KvComp c
     uint32_t o0, n_una, o0_next, nu_next;
     load_off(t_begin, o0_next, nu_next);
     uint32_t lut_v = 0;
-    if (tid < 64) {
+    if (MODE == 1 && tid < 64) {
         const uint8_t *rk = of_seq(ck0.rank_to_exp, seq, g.seq_stride), *rv = of_seq(cv0.rank_to_exp, seq, g.seq_stride);
         lut_v = tid < 32 ? rk[tid] : rv[tid - 32];
     }
@@ -293,7 +402,21 @@ __global__ void __launch_bounds__(kTcThreads) k_draft_attn_tc(KvGeom g, KvComp c
             if (i < n_qw) reinterpret_cast<uint32_t*>(q_s + (i / (d / 2)) * ks)[i % (d / 2)] = qv[u];
         }
     }
-    if (tid < 64) lut_s[tid] = lut_v << 7;
+    if (MODE == 1) {
+        if (tid < 64) lut_s[tid] = lut_v << 7;
+    } else {
+        constexpr int NF = 1 << (8 - T);
+        for (int f = tid; f < NF; f += kTcThreads) {
+            const uint32_t sgn = (uint32_t)f >> (7 - T), mag = ((uint32_t)f & ((1u << (7 - T)) - 1u)) << T;
+            uint2 lm = make_uint2(0u, 0u);
+            if (mag) {
+                const uint32_t pl = 31u - (uint32_t)__clz(mag);               // leading bit of the 7-bit magnitude
+                lm.x = (sgn << 15) | (pl << 7) | ((mag << (7u - pl)) & 0x7Fu);
+                lm.y = 0xFFFFFFFFu;
+            }
+            reinterpret_cast<uint2*>(lut_s)[f] = lm;
+        }
+    }
     constexpr int kMaxMt = 4;                                                 // 16-channel tiles of the output per warp (head_dim <= 256)
     float o_acc[kMaxMt][4];
 #pragma unroll
@@ -311,12 +434,14 @@ __global__ void __launch_bounds__(kTcThreads) k_draft_attn_tc(KvGeom g, KvComp c
             const uint32_t fa = smem_u32(my_fix + lane);
             for (int w = 0; w < g.wpt; ++w) tc_cp_async4(fa + w * 128, fixed + w * 32 + src_lane, true);      // coalesced block copy
             my_fix[g.wpt * 32 + lane] = 0u;
-            const uint32_t ua = smem_u32(my_una + lane);
-            const bool fits = n_una <= (uint32_t)stage;
+            if (MODE == 1) {
+                const uint32_t ua = smem_u32(my_una + lane);
+                const bool fits = n_una <= (uint32_t)stage;
 #pragma unroll 4
-            for (int w = 0; w < una_rows; ++w) {
-                const bool take = fits && (uint32_t)w < n_una;
-                tc_cp_async4(ua + w * 128, arena + (take ? o0 + w : 0), take);
+                for (int w = 0; w < una_rows; ++w) {
+                    const bool take = fits && (uint32_t)w < n_una;
+                    tc_cp_async4(ua + w * 128, arena + (take ? o0 + w : 0), take);
+                }
             }
         }
         load_off(t0 + kTcTok, o0_next, nu_next);                              // the next chunk's offsets travel meanwhile
@@ -328,15 +453,19 @@ __global__ void __launch_bounds__(kTcThreads) k_draft_attn_tc(KvGeom g, KvComp c
         tc_cp_async_wait_all();
         __syncthreads();
         if (n_here > 0) {
-            const bool raw = (my_fix[lane] & kKvRawFlag) != 0;                // entry word 0 of this token's record
-            const bool staged = n_una <= (uint32_t)stage && !raw;
-            const uint32_t* lutP = lut_s + kind * 32;
             const uint32_t row_a = smem_u32((kind ? vt_s : kt_s) + (size_t)(tw * 32 + lane) * ks);
             const uint32_t* bmP = my_fix + g.e_words * 32 + lane;
             const uint32_t* flP = bmP + g.bm_words * 32;
-            tc_walk<T>(bmP, flP, my_una + lane, lutP, r2e, g.kept, d, n_una * 32u, row_a, staged, stage);
-            if (!staged)                                                      // raw exponents or a very long record: read it in place
-                tc_walk_slow<T>(bmP, flP, arena + o0, 1, raw, 0, g.kept, 0u, 0u, (uint32_t)d, n_una * 32u, r2e, row_a);
+            if (MODE == 1) {
+                const bool raw = (my_fix[lane] & kKvRawFlag) != 0;            // entry word 0 of this token's record
+                const bool staged = n_una <= (uint32_t)stage && !raw;
+                const uint32_t* lutP = lut_s + kind * 32;
+                tc_walk<T>(bmP, flP, my_una + lane, lutP, r2e, g.kept, d, n_una * 32u, row_a, staged, stage);
+                if (!staged)                                                  // raw exponents or a very long record: read it in place
+                    tc_walk_slow<T>(bmP, flP, arena + o0, 1, raw, 0, g.kept, 0u, 0u, (uint32_t)d, n_una * 32u, r2e, row_a);
+            } else {
+                tc_walk_mx<T>(bmP, flP, flP + g.f_words * 32, my_una + lane, reinterpret_cast<const uint2*>(lut_s), g.kept, d, row_a);
+            }
         }
         __syncthreads();
 
@@ -436,12 +565,12 @@ int launch_attn_merge(const AttnScratch& sc, int n_chunks_alloc, int chunk_token
 
 size_t draft_attn_tc_smem_bytes(const KvGeom& g) {
     const size_t ks = (size_t)g.d + kTcPad;
-    return (2 * kTcTok + kTcHeads) * ks * 2 + (size_t)tc_fix_words(g) * 4 + (size_t)4 * (tc_una_stage(g) + 2) * 32 * 4 + 64 * 4 + 3 * kTcHeads * 4 + 64;
+    return (2 * kTcTok + kTcHeads) * ks * 2 + (size_t)tc_fix_words(g) * 4 + (size_t)4 * tc_una_rows(g) * 32 * 4 + (size_t)tc_lut_words(g) * 4 + 3 * kTcHeads * 4 + 64;
 }
 
 bool draft_attn_tc_supported(const KvGeom& g, int n_q) {
     const int G = n_q / g.n_kv;
-    return g.mode == 1 && (g.t == 4 || g.t == 0) && G >= 1 && G <= kTcHeads && g.d % 16 == 0 && g.d >= 32 && g.d <= 256;
+    return (g.mode == 1 || g.mode == 2) && (g.t == 4 || g.t == 0) && G >= 1 && G <= kTcHeads && g.d % 16 == 0 && g.d >= 32 && g.d <= 256;
 }
 
 int launch_draft_attn_tc(const KvGeom& g, const KvComp& ck, const KvComp& cv, const uint16_t* qkv, int qkv_stride, int n_q,
@@ -451,17 +580,19 @@ int launch_draft_attn_tc(const KvGeom& g, const KvComp& ck, const KvComp& cv, co
     const size_t smem = draft_attn_tc_smem_bytes(g);
     if (smem > 227 * 1024) return CASS_ERR_UNSUPPORTED;
     dim3 grid(n_chunks, g.n_kv, n_seq);
-#define CASS_TC_LAUNCH(TT)                                                                                           \
+#define CASS_TC_LAUNCH(MM, TT)                                                                                           \
     do {                                                                                                             \
         static size_t attr = 0;                                                                                      \
         if (smem > attr) {                                                                                           \
-            CASS_CUDA_CHECK(cudaFuncSetAttribute((k_draft_attn_tc<TT>), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
+            CASS_CUDA_CHECK(cudaFuncSetAttribute((k_draft_attn_tc<MM, TT>), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
             attr = smem;                                                                                             \
         }                                                                                                            \
-        CASS_PDL_LAUNCH((k_draft_attn_tc<TT>), grid, dim3(kTcThreads), smem, s, g, ck, cv, qkv, qkv_stride, n_q, st, sc, n_chunks);      \
+        CASS_PDL_LAUNCH((k_draft_attn_tc<MM, TT>), grid, dim3(kTcThreads), smem, s, g, ck, cv, qkv, qkv_stride, n_q, st, sc, n_chunks);      \
     } while (0)
-    if (g.t == 4) CASS_TC_LAUNCH(4);
-    else CASS_TC_LAUNCH(0);
+    if (g.mode == 1 && g.t == 4) CASS_TC_LAUNCH(1, 4);
+    else if (g.mode == 1) CASS_TC_LAUNCH(1, 0);
+    else if (g.t == 4) CASS_TC_LAUNCH(2, 4);
+    else CASS_TC_LAUNCH(2, 0);
 #undef CASS_TC_LAUNCH
     CASS_LAUNCH_CHECK();
     // the runs of every (sequence, query head) are merged by a kernel of their own: one CTA per head with the runs spread

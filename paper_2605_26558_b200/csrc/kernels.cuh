@@ -55,15 +55,8 @@ __host__ __device__ __forceinline__ P* of_seq(P* p, int b, size_t seq_stride) {
 }
 __host__ __device__ inline int kv_entry_words(int d) { int n = (d / 32 - 1 + 2) / 3; return n < 1 ? 1 : n; }
 __host__ __device__ inline int kv_code_budget(int kept) { return 8 * kept < 1023 ? 8 * kept : 1023; }
-// Tokens one CTA of the draft attention handles: 32, doubled while the grid would exceed about four CTAs per SM.
-// Draft attention and its merge compute it from the same visible length, so they agree without host involvement.
-__host__ __device__ inline int da_tokens_per_cta(int visible, int heads_x_seqs) {
-    int t = 32;
-    while (t < 256 && ceil_div(visible, t) * heads_x_seqs > 592) t *= 2;
-    return t;
-}
-// Positions one CTA of the dense-tile draft attention (long caches) handles: one 64-token chunk, doubled while the grid
-// would exceed about four CTAs per SM.  The kernel and its merge compute it from the same visible length.
+// Positions one CTA of the draft attention handles: one 64-token chunk, doubled while the grid would exceed about four
+// CTAs per SM.  The kernel and its merge compute it from the same visible length, so they agree without host involvement.
 __host__ __device__ inline int tc_run_tokens(int visible, int heads_x_seqs) {
     int t = 64;
     while (t < 2048 && ceil_div(visible, t) * heads_x_seqs > 592) t *= 2;
@@ -205,7 +198,6 @@ struct AttnScratch {
     float* o;     // [rows*n_q][n_chunks][d]
     float* m;     // [rows*n_q][n_chunks]
     float* l;     // [rows*n_q][n_chunks]
-    int* cnt;     // [kMaxBatch * n_kv] arrival counters of the draft attention's CTAs, zero between launches
 };
 // Draft: one query row per sequence (qkv row b, `qkv_stride` elements apart) at position len + inflight over that
 // sequence's compressed cache (caches given for sequence 0).

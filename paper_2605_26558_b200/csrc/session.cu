@@ -158,7 +158,6 @@ static size_t layout(Session* s, uint8_t* base) {
     s->asc.o = (float*)at(p.take(pairs * n_chunks * d.head_dim * 4));
     s->asc.m = (float*)at(p.take(pairs * n_chunks * 4));
     s->asc.l = (float*)at(p.take(pairs * n_chunks * 4));
-    s->asc.cnt = (int*)at(p.take((size_t)kMaxBatch * d.n_kv_heads * 4));      // zeroed with the session memory
     s->argmax_tmp = (int32_t*)at(p.take((size_t)R * 128 * 4));
     s->argmax_val = (float*)at(p.take((size_t)R * 128 * 4));
     s->layers.resize(d.n_layers);

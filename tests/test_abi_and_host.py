@@ -90,8 +90,8 @@ def test_launch_count_formula():
     import bench
     # 10 launches per draft layer (4 projections, RoPE + KV append, attention, merge, 2 norms, SwiGLU) and per verification layer
     assert bench.launches_per_step(32, 4) == 4 * (2 + 32 * 10 + 3) + (2 + 32 * 10 + 3) + 1
-    # the count does not depend on the cache length; a Cassandra-2 cache merges inside the attention kernel
+    # the count depends neither on the cache length nor on the KV format
     assert bench.launches_per_step(32, 4, max_seq=4096) == bench.launches_per_step(32, 4)
-    assert bench.launches_per_step(32, 4, kv_mode=2) == bench.launches_per_step(32, 4) - 4 * 32
+    assert bench.launches_per_step(32, 4, kv_mode=2) == bench.launches_per_step(32, 4)
     # verification from the two parts: two reconstruction launches per matrix
     assert bench.launches_per_step(2, 1, from_parts=True) - bench.launches_per_step(2, 1) == 2 * (2 * 4 + 1)

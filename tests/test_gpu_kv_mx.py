@@ -34,7 +34,8 @@ def _engine(cass, n_q, n_kv, d, max_seq=640, kv_p=400, kv_t=4, batch=1):
 
 
 @pytest.mark.parametrize("n_q,n_kv,d,n_pos,kv_p,kv_t", [(32, 8, 128, 70, 400, 4), (4, 2, 64, 45, 400, 4), (10, 2, 32, 33, 400, 4),
-                                                         (8, 2, 256, 40, 300, 4), (8, 2, 128, 37, 0, 0), (32, 8, 128, 600, 400, 4)])
+                                                         (8, 2, 256, 40, 300, 4), (8, 2, 128, 37, 0, 0), (32, 8, 128, 600, 400, 4),
+                                                         (4, 2, 64, 68, 400, 4), (4, 2, 64, 131, 400, 4), (16, 2, 256, 200, 0, 4)])
 def test_mx_kv_records_and_draft_attention(cass, n_q, n_kv, d, n_pos, kv_p, kv_t):
     """cass_kv_append with kv_mode 2: every record equals the oracle's words (bitmap, fields, slice exponents); the
     draft attention over them equals softmax(q K^T / sqrt(d)) V on the oracle's zero-padded reconstruction.  Tokens
@@ -122,8 +123,12 @@ def test_model_with_a_cassandra_2_cache(cass):
         cass.cass_draft_step(eng.session, eng.toks[i: i + 1], tok, logits)
         want = model.forward_token(Wd, kv2, forced[i], 64 + i, True, 400, 4, kv_mode=2)
         rms = float(np.sqrt(np.mean(want ** 2)))
-        errs.append(float(np.abs(logits.cpu().numpy() - want).max()) / rms)
-    assert min(errs) <= TOL and max(errs) <= 0.1, errs       # whole-model logits: rounding flips, see test_gpu_layer_parity
+        e = np.abs(logits.cpu().numpy() - want) / rms
+        errs.append((float(e.max()), float(np.median(e)), float((e <= TOL).mean())))
+    # Whole-model logits: a single bf16 rounding flip of an activation is amplified by the outlier columns of the weights
+    # (see test_gpu_layer_parity for the per-layer analysis), so the bar is held by the bulk of the logits and the few
+    # elements a flip reaches stay within five times the bar.
+    assert all(mx_ <= 0.1 and med <= 0.5 * TOL and frac >= 0.95 for mx_, med, frac in errs), errs
     assert eng.status()[0] == 0
     eng.close()
     e0, f0 = make()
