@@ -171,10 +171,11 @@ __device__ __forceinline__ void tc_walk(const uint32_t* bmP, const uint32_t* flP
         bpos += 32u - p;
         if (!tail) dry |= p;
         const bool ok = (int32_t)dry >= 0;
+        if (emit && ok) {                                             // one branch per group: the stores themselves are unconditional
 #pragma unroll
-        for (int e = 0; e < kGroupCols; ++e)
-            if (emit && ok && (!tail || e < rem)) tc_sts16(addr[e], val[e]);
-        if (emit && !ok) {
+            for (int e = 0; e < kGroupCols; ++e)
+                if (!tail || e < rem) tc_sts16(addr[e], val[e]);
+        } else if (emit) {
             // redo the group value by value, then put the cursors behind it
             const int cnt = tail ? rem : kGroupCols;
             tc_walk_slow<T>(bmP, flP, unP, 32, false, grp * kGroupCols, cnt, bpos0, upos0, (uint32_t)d, una_bits, r2e, row_a);
@@ -282,10 +283,11 @@ __device__ __forceinline__ void tc_walk_mx(const uint32_t* bmP, const uint32_t* 
         bpos += 32u - p;
         if (!tail) dry |= p;                                          // a search that failed fails from then on
         const bool ok = (int32_t)dry >= 0;
+        if (ok) {                                                     // one branch per group: the stores themselves are unconditional
 #pragma unroll
-        for (int e = 0; e < kGroupCols; ++e)
-            if (ok && (!tail || e < rem)) tc_sts16(addr[e], val[e]);
-        if (!ok) {
+            for (int e = 0; e < kGroupCols; ++e)
+                if (!tail || e < rem) tc_sts16(addr[e], val[e]);
+        } else {
             const int cnt = tail ? rem : kGroupCols;
             tc_walk_mx_slow<T>(bmP, flP, ebP, lutP, grp * kGroupCols, cnt, bpos0, (uint32_t)d, row_a);
             uint32_t b = bpos0;

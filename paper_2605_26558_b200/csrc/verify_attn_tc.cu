@@ -80,6 +80,13 @@ __global__ void __launch_bounds__(kVtThreads) k_verify_attn_tc(const __grid_cons
     if (tid == 0) {
         mbar_init(bar_k, 1); mbar_init(bar_v, 1); mbar_init(bar_s, 1); mbar_init(bar_p, 128); mbar_init(bar_o, 1);
         fence_mbar_init();
+        // the chunk's K and V tiles start travelling now, while the other warps stage Q and tensor memory is allocated
+        mbar_expect_tx(bar_k, 2 * kVtTileBytes);
+        tma_load_3d(sK, &map_k, head * kVtD, t0, seq, bar_k);
+        tma_load_3d(sK + kVtTileBytes, &map_k, head * kVtD + 64, t0, seq, bar_k);
+        mbar_expect_tx(bar_v, 2 * kVtTileBytes);
+        tma_load_3d(sV, &map_v, head * kVtD, t0, seq, bar_v);
+        tma_load_3d(sV + kVtTileBytes, &map_v, head * kVtD + 64, t0, seq, bar_v);
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kVtTmemCols) : "memory");
@@ -104,14 +111,7 @@ __global__ void __launch_bounds__(kVtThreads) k_verify_attn_tc(const __grid_cons
     const uint32_t tmem = *tmem_slot;
     bool ok = true;
 
-    if (warp == 0 && lane == 0) {
-        mbar_expect_tx(bar_k, 2 * kVtTileBytes);
-        tma_load_3d(sK, &map_k, head * kVtD, t0, seq, bar_k);
-        tma_load_3d(sK + kVtTileBytes, &map_k, head * kVtD + 64, t0, seq, bar_k);
-        mbar_expect_tx(bar_v, 2 * kVtTileBytes);
-        tma_load_3d(sV, &map_v, head * kVtD, t0, seq, bar_v);
-        tma_load_3d(sV + kVtTileBytes, &map_v, head * kVtD + 64, t0, seq, bar_v);
-    } else if (warp == 1 && lane == 0) {
+    if (warp == 1 && lane == 0) {
         // ---- scores^T = K . Q^T: A = K tile (K-major over d), B = Q (K-major over d) ----
         if (mbar_wait_bounded(bar_k, 0)) {
             tc_fence_after();
