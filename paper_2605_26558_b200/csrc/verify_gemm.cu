@@ -166,16 +166,26 @@ __global__ void k_verify_gemm_finish(const float* __restrict__ partial, int rows
     if (y_bf16) y_bf16[(size_t)r * n + j] = float_to_bf16_bits(acc);
 }
 
-// K ranges: a function of (n, k) only.  Enough CTAs for about two per SM, at least 4 k-blocks per range.
+// K ranges: a function of (n, k) only.  Enough CTAs for about two per SM, at least 4 k-blocks per range.  A plan that
+// needs a few CTAs more than the 296 that run at once pays a second, nearly empty wave for them (320 CTAs for the
+// 4096 x 4096 matrix: 12.5 us; 256: see the microbenchmark summary), so such a plan gives up ranges until it fits.
 static void split_plan(int n, int k, int* kb_total, int* kb_per_split, int* n_split) {
+    constexpr int kSlots = 296;
     const int tiles = ceil_div(n, kTcBM);
     *kb_total = ceil_div(k, kTcBK);
-    int want = ceil_div(296, tiles);
+    int want = ceil_div(kSlots, tiles);
     int max_split = *kb_total / 4 > 0 ? *kb_total / 4 : 1;
     if (want > max_split) want = max_split;
     if (want < 1) want = 1;
-    *kb_per_split = ceil_div(*kb_total, want);
-    *n_split = ceil_div(*kb_total, *kb_per_split);
+    auto plan = [&](int w, int* per, int* ns) { *per = ceil_div(*kb_total, w); *ns = ceil_div(*kb_total, *per); return tiles * *ns; };
+    int ctas = plan(want, kb_per_split, n_split);
+    while (ctas > kSlots && 2 * ctas <= 3 * kSlots && want > 1) {             // a little over one wave
+        int per, ns;
+        const int fewer = plan(want - 1, &per, &ns);
+        if (fewer <= kSlots && 5 * fewer < 4 * kSlots) break;                 // would leave the single wave too empty: keep the plan
+        --want;
+        *kb_per_split = per; *n_split = ns; ctas = fewer;
+    }
 }
 
 Partials verify_gemm_partials(const float* partial, int n, int k, int bn) {

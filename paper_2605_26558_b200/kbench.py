@@ -201,6 +201,7 @@ def step_breakdown(gamma=4, n_prompt=512, steps=3, batch=1):
     evs.sort(key=lambda ev: ev.time_range.start)
     per_pass = 4 * shape.n_layers + 1              # draft projections of one pass, in launch order: (wqkv, wo, wgu, wd) per layer, lm_head
     n_gemv = 0
+    n_vgemm = 0
     for ev in evs:
         if True:
             name = re.sub(r"<.*|\(.*", "", ev.name).replace("void ", "").replace("cass::", "")
@@ -208,6 +209,10 @@ def step_breakdown(gamma=4, n_prompt=512, steps=3, batch=1):
                 c = n_gemv % per_pass
                 name += "[" + ("lm_head" if c == per_pass - 1 else ("wqkv", "wo", "wgu", "wd")[c % 4]) + "]"
                 n_gemv += 1
+            if name == "k_verify_gemm_tc":                   # the verification pass launches its projections in the same order
+                c = n_vgemm % per_pass
+                name += "[" + ("lm_head" if c == per_pass - 1 else ("wqkv", "wo", "wgu", "wd")[c % 4]) + "]"
+                n_vgemm += 1
             agg[name][0] += 1
             agg[name][1] += ev.device_time_total if hasattr(ev, "device_time_total") else ev.cuda_time_total
     tot = sum(v[1] for v in agg.values())
