@@ -571,6 +571,9 @@ int launch_draft_gemv(const void* blob, const cass_blob_info& bi, const void* x_
     int g = ceil_div(sm_count() * per_sm, bi.n_seg);
     if (g > bi.n_rowblocks) g = bi.n_rowblocks;
     if (g < 1) g = 1;
+    { static const int one = [] { const char* e = std::getenv("CASS_GEMV_ONE_TILE"); return e ? atoi(e) : 0; }();
+      if (one == 1) g = bi.n_rowblocks;
+      if (one > 1) { int tpc = ceil_div(bi.n_rowblocks, g); tpc = ceil_div(tpc, one); g = ceil_div(bi.n_rowblocks, tpc); } }
     dim3 grid(bi.n_seg, g), block(threads);
     const uint32_t* b = (const uint32_t*)blob;
     const uint16_t* x = (const uint16_t*)x_bf16;
