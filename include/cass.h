@@ -246,7 +246,7 @@ size_t cass_calib_norms_count(const cass_model_desc* desc);
  * order: start_pos may not exceed the number of positions already in the compressed cache of that layer.
  * The compressed cache uses the layer's frozen codebooks (cass_kv_build_codebook).
  * Record of one (token, head, K|V) in the compressed cache, kv_mode 1: entry words (a 10-bit code-bit offset for every
- * 32-channel slice after the first, three per word from bit 29 down: the d/32 slices of a record decode side by side;
+ * 32-channel slice after the first, three per word from bit 29 down: a decoder can enter a record at any slice;
  * bit 31 of the first word = raw flag), bitmap, sign+mantissa fields, and in the arena the unary exponent stream -- or,
  * when that stream would take more than min(8 * kept, 1023) bits, the kept exponents as raw bytes, so that a record
  * never takes more than ceil(8 * kept / 32) arena words and the arena is sized for that: a codebook that fits the later
@@ -287,7 +287,8 @@ int cass_verify(void* session, const int32_t* toks, int g, int32_t* target_argma
 /* Stand-alone draft attention of one layer (Sec. 4.1 draft inference over the KV speculation data of Sec. 4.2):
  * q: bf16 [max_batch][n_q_heads][head_dim] (post-RoPE); sequence b's query sees the first len_b + 1 positions of its
  * compressed cache of that layer (len = committed length, see cass_set_len; no draft in flight);
- * out: bf16 [max_batch][n_q_heads][head_dim]. */
+ * out: bf16 [max_batch][n_q_heads][head_dim].  Returns CASS_ERR_UNSUPPORTED for KV truncations other than 0 and 4,
+ * more than 8 query heads per KV head, or a head size that is not a multiple of 32 (cass_draft_step likewise). */
 int cass_draft_attention(void* session, int layer, const void* q_bf16, void* out_bf16, void* stream);
 
 /* Stand-alone verification projection (Sec. 2.2: the gamma+1 rows are processed as one small batch, bound by
