@@ -21,7 +21,23 @@ __global__ void k_embed(const int32_t* __restrict__ toks, int tok_stride, const 
     pdl_wait();
     int r = blockIdx.x;
     const uint16_t* src = embed + (size_t)toks[(size_t)r * tok_stride] * hidden;
-    for (int i = threadIdx.x; i < hidden; i += blockDim.x) h[(size_t)r * hidden + i] = src[i];
+    uint16_t* dst = h + (size_t)r * hidden;
+    if ((hidden & 7) == 0 && (((uintptr_t)src | (uintptr_t)dst) & 15) == 0) {
+        // 16 bytes per load, two loads in flight per thread: the row costs one or two round trips
+        const uint4* s4 = reinterpret_cast<const uint4*>(src);
+        uint4* d4 = reinterpret_cast<uint4*>(dst);
+        const int n16 = hidden / 8;
+        for (int i = threadIdx.x; i < n16; i += 2 * blockDim.x) {
+            const int j = i + blockDim.x;
+            const uint4 a = s4[i];
+            uint4 b = make_uint4(0u, 0u, 0u, 0u);
+            if (j < n16) b = s4[j];
+            d4[i] = a;
+            if (j < n16) d4[j] = b;
+        }
+        return;
+    }
+    for (int i = threadIdx.x; i < hidden; i += blockDim.x) dst[i] = src[i];
 }
 
 __device__ __forceinline__ float block_sum(float v, float* s_red) {
