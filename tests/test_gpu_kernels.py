@@ -61,7 +61,8 @@ def test_verify_gemm_rows_do_not_depend_on_the_batch(cass):
     assert torch.equal(alone[0], full[0])
 
 
-@pytest.mark.parametrize("n_pos,n_q", [(1, 32), (63, 32), (64, 32), (65, 32), (700, 32), (4096, 32), (300, 40), (130, 64)])
+@pytest.mark.parametrize("n_pos,n_q", [(1, 32), (63, 32), (64, 32), (65, 32), (700, 32), (4096, 32), (300, 40), (130, 64),
+                                         (6000, 32)])      # 6000 positions: runs of two chunks per CTA (running softmax)
 def test_draft_attention_llama_layer_shape(cass, n_pos, n_q):
     """Draft attention of one Llama-3-8B-shaped layer (32 q / 8 kv heads of 128; also 5 and 8 query heads per KV head,
     the Qwen-style grouping) over synthetic KV (N(0,1), outlier channels in K) against the oracle:
@@ -72,7 +73,7 @@ def test_draft_attention_llama_layer_shape(cass, n_pos, n_q):
     wt = synth.model_weights(shape, 0, device="cuda")
     gw = {"layers": [engine.fuse_layer_weights(lw) for lw in wt["layers"]], "embed": wt["embed"], "lm_head": wt["lm_head"],
           "norm_final": wt["norm_final"]}
-    eng = engine.Engine(shape, gw, max_seq=4096 + 64, gamma_max=4)
+    eng = engine.Engine(shape, gw, max_seq=max(4096, n_pos) + 64, gamma_max=4)
     k, v = synth.kv_fill(n_pos, 8, 128, 1, "ka/kv")
     n0 = max(1, min(n_pos, 512))                     # codebooks come from the first positions, the rest is appended
     cass.cass_kv_append(eng.session, 0, k[:n0].cuda().contiguous(), v[:n0].cuda().contiguous(), 0, n0, cass.KV_BF16)

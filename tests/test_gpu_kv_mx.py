@@ -35,12 +35,13 @@ def _engine(cass, n_q, n_kv, d, max_seq=640, kv_p=400, kv_t=4, batch=1):
 
 @pytest.mark.parametrize("n_q,n_kv,d,n_pos,kv_p,kv_t", [(32, 8, 128, 70, 400, 4), (4, 2, 64, 45, 400, 4), (10, 2, 32, 33, 400, 4),
                                                          (8, 2, 256, 40, 300, 4), (8, 2, 128, 37, 0, 0), (32, 8, 128, 600, 400, 4),
-                                                         (4, 2, 64, 68, 400, 4), (4, 2, 64, 131, 400, 4), (16, 2, 256, 200, 0, 4)])
+                                                         (4, 2, 64, 68, 400, 4), (4, 2, 64, 131, 400, 4), (16, 2, 256, 200, 0, 4),
+                                                         (32, 8, 128, 5000, 400, 4), (32, 16, 128, 5000, 400, 4)])     # runs of two and of four chunks per CTA
 def test_mx_kv_records_and_draft_attention(cass, n_q, n_kv, d, n_pos, kv_p, kv_t):
     """cass_kv_append with kv_mode 2: every record equals the oracle's words (bitmap, fields, slice exponents); the
     draft attention over them equals softmax(q K^T / sqrt(d)) V on the oracle's zero-padded reconstruction.  Tokens
     with a wide exponent spread (values below their slice's quantum), equal magnitudes (tie rule) and zeros included."""
-    eng = _engine(cass, n_q, n_kv, d, kv_p=kv_p, kv_t=kv_t)
+    eng = _engine(cass, n_q, n_kv, d, max_seq=max(640, (n_pos + 64 + 31) // 32 * 32), kv_p=kv_p, kv_t=kv_t)
     k, v = synth.kv_fill(n_pos, n_kv, d, 7, "kvmx/kv")
     g = torch.Generator().manual_seed(d + n_pos)
     sign = torch.where(torch.rand(n_kv, d, generator=g) < 0.5, -1.0, 1.0)
